@@ -1,0 +1,175 @@
+/*
+ * loopspec.h -- C ABI of the LoopSpec pipelined decode path for looped transformers on B200 (sm_100a).
+ *
+ * The library runs the decode loop of Algorithm 1 (App. G) of "LoopSpec: Pipelined Self-Speculative
+ * Decoding for Looped Transformers": in every step all active branches -- the token being verified at
+ * recurrent depth R, first-proposal drafts spawned at depth d1 and, when the gate of Eq. 6 opens,
+ * residual second proposals spawned at depth d2 (Eq. 5) -- go through the shared block stack in ONE
+ * batched pass (Sec. 4.2 step 1), so the shared weights are read from HBM once per step.
+ *
+ * Conventions (all entry points):
+ *   - Every call returns a loopspec_status; nothing throws or aborts across this boundary.
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers are ordinary host memory.
+ *   - Weights and the workspace are allocated by the caller, borrowed for the life of the context and never
+ *     freed by the library; weights are never written.  The library itself allocates only host memory, CUDA
+ *     graphs/events and two small pinned host buffers; it never allocates device memory.
+ *   - Linear weights are row-major [out_features][in_features]; bf16 weights are raw 16-bit bfloat16,
+ *     fp32 weights IEEE binary32.  Norm gains are always fp32.
+ *   - Argument errors are detected on the host before any launch and leave the context usable.
+ *     LOOPSPEC_ECUDA is sticky (the context must be destroyed).
+ *   - A context is not thread safe; all work is issued on the stream given at init.
+ */
+#ifndef LOOPSPEC_H
+#define LOOPSPEC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct loopspec_ctx loopspec_ctx; /* opaque, owned by the library */
+
+typedef enum {
+  LOOPSPEC_OK = 0,
+  LOOPSPEC_EINVAL = -1,       /* bad argument */
+  LOOPSPEC_ESTATE = -2,       /* call out of order (step before prefill, verify with nothing at depth R, ...) */
+  LOOPSPEC_ECAPACITY = -3,    /* max_ctx, max_seqs, node table or workspace too small */
+  LOOPSPEC_ECUDA = -4,        /* a CUDA call failed; see loopspec_last_error */
+  LOOPSPEC_ETIMEOUT = -5,     /* reserved: a bounded device-side wait ran out */
+  LOOPSPEC_EUNSUPPORTED = -6  /* shape outside what the kernels support */
+} loopspec_status;
+
+/* Looped transformer of Sec. 3.1 (Eq. 1).  Ouro layout: n_prelude = n_coda = 0, P = embedding, C = final
+ * RMSNorm + lm_head.  Blocks are pre-RMSNorm, rotary attention (rotate-half pairing), SwiGLU, no biases. */
+typedef struct {
+  int32_t vocab, hidden, n_q_heads, n_kv_heads, head_dim, ffn;
+  int32_t n_prelude, n_recurrent, n_coda; /* layers in P, B, C; only n_prelude = n_coda = 0 is supported */
+  int32_t R;                              /* recurrences of B */
+  int32_t weight_dtype;                   /* 0 = fp32, 1 = bf16 (all matrices incl. embedding) */
+  int32_t tied_lm_head;                   /* 1: lm_head pointer ignored, the embedding is used */
+  float rms_eps, rope_theta;
+} loopspec_model;
+
+/* Scheduler settings (Sec. 4.2-4.3, App. B "Depth Configuration").
+ * d1 < d2 < R with d1 | d2 and d1 | R; d2 == 0 selects the single-proposal pipeline of Sec. 4.2;
+ * d1 == d2 == 0 picks the pair from the closed form of Theorem 2 using (alpha, beta).
+ * gate = 1 applies Eq. 6, gate = 0 always creates the second proposal; residual_q2 = 1 drafts it from
+ * p_{d2} (-) p_{d1} (Eq. 5), 0 from p_{d2} itself.  temperature 0 = greedy.  max_prefill_rows (0 = default)
+ * bounds how many prompt positions one prefill pass carries. */
+typedef struct {
+  int32_t d1, d2;
+  float alpha, beta;
+  int32_t gate, residual_q2;
+  float temperature;
+  uint64_t seed;
+  int32_t max_seqs, max_ctx;
+  int32_t max_prefill_rows;
+} loopspec_sched;
+
+/* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:
+ * norm1 [H], wqkv [(nq + 2 nkv) * d][H] (q rows, then k rows, then v rows), wo [H][nq * d], norm2 [H],
+ * wgateup [2F][H] (gate rows, then up rows), wdown [H][F].  adapter must be NULL. */
+typedef struct {
+  const void* embed;      /* [V][H] */
+  const void* lm_head;    /* [V][H], ignored when tied */
+  const void* final_norm; /* fp32 [H] */
+  const void* adapter;
+  const void* const* layer_ptrs;
+} loopspec_weights;
+
+/* One committed token (Algorithm 1, main loop: "commit a new decoded token"). source: 1 = accepted first
+ * proposal, 2 = accepted second proposal, 3 = resampled at depth R (restart). step = index (from 1) of the
+ * batched pass after which it was committed. */
+typedef struct {
+  int32_t seq, n_committed, token, source, accepted1, accepted2, gate_open, step;
+} loopspec_commit;
+
+/* Counters of Sec. 5 (gamma), App. C (gate openings, effective batch size) and App. D (commit sources). */
+typedef struct {
+  int64_t steps, n_decode, n_accept1, n_accept2, n_restart, gate_evals, gate_opens, rows_total, rows_max,
+      readout_rows_total;
+  double gamma;
+} loopspec_stats;
+
+/* Bytes of device workspace loopspec_init needs for this model and scheduler (0 on invalid input). */
+size_t loopspec_workspace_bytes(const loopspec_model*, const loopspec_sched*);
+
+/* Create a context.  workspace: device memory, 256-byte aligned, at least loopspec_workspace_bytes large.
+ * cuda_stream: a cudaStream_t (may be NULL for the legacy stream is NOT allowed: pass a real stream).
+ * Host structs are copied.  Synchronous; uploads the rotary table and clears the workspace tables. */
+int loopspec_init(const loopspec_model*, const loopspec_sched*, const loopspec_weights*, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream, loopspec_ctx** out);
+
+/* Algorithm 1, lines before the main loop: run all R recurrences over the prompt of sequence `seq`
+ * (host array of n ids), fill every (layer, recurrence) KV plane, commit the first token drawn from C(H^R)
+ * and spawn the initial branch on prompt||token.  first_token (host, may be NULL) receives that token.
+ * Synchronous.  Calling it again for the same seq restarts that sequence. */
+int loopspec_prefill(loopspec_ctx*, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* first_token);
+
+/* One iteration of the body of Algorithm 1's main loop up to, not including, verification: advance every
+ * active branch by one recurrent depth in one batched pass, read out branches reaching d1 / d2 / R, draw
+ * first proposals, evaluate the gate, draw second proposals, spawn their children.  n_rows_out: branches
+ * advanced; n_need_verify_out: sequences whose deepest branch reached R (call loopspec_verify before the
+ * next step if > 0).  Synchronous. */
+int loopspec_step(loopspec_ctx*, int32_t* n_rows_out, int32_t* n_need_verify_out);
+
+/* Cascade verification (Sec. 4.3; Algorithm 1 Verify + Reroot) for every sequence whose deepest branch is
+ * at depth R: accept the first candidate w.p. min{1, p/q1}, else the second against p (-) q1, else
+ * resample; commit, keep the chosen child's subtree, release the rest, make the kept branch's KV part of
+ * the committed prefix.  out: host array of max_out entries.  ESTATE if nothing is at depth R. */
+int loopspec_verify(loopspec_ctx*, loopspec_commit* out, int32_t max_out, int32_t* n_out);
+
+/* Run step+verify until every prefilled sequence has committed n_tokens more tokens, as CUDA-graph
+ * replays with the branch table on the device.  ids_out: host [max_seqs][n_tokens] (rows of sequences
+ * that were not prefilled are left untouched).  Produces exactly the tokens of alternating step/verify. */
+int loopspec_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
+
+/* Baseline of Fig. 1(a): all R recurrences of a token before the next, from the same kernels. */
+int loopspec_vanilla_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
+
+/* Theorem 2 / Eq. 8: real-valued optimum and the admissible integer pair (d1 | d2, d1 | R, d1 < d2 < R)
+ * minimising the bound d1 + beta d1^-alpha d2 + 2 beta d2^-alpha R.  Host only; any output may be NULL. */
+int loopspec_pick_depths(float alpha, float beta, int32_t R, double* d1_star, double* d2_star, int32_t* d1,
+                         int32_t* d2);
+
+/* Maximum number of simultaneously active branches (Sec. 4.3 recurrence); d2 = 0: single proposal. */
+int32_t loopspec_max_branches(int32_t R, int32_t d1, int32_t d2);
+
+int loopspec_get_stats(loopspec_ctx*, loopspec_stats*);
+/* Commit records of the last decode/verify calls of sequence seq since its prefill (host array). */
+int loopspec_get_commits(loopspec_ctx*, int32_t seq, loopspec_commit* out, int32_t max_out, int32_t* n_out);
+/* Rows advanced by each step since the last prefill of any sequence (host array of int32). */
+int loopspec_get_row_trace(loopspec_ctx*, int32_t* out, int32_t max_out, int32_t* n_out);
+
+/* Copy fp32 logits (before temperature) to host out_V[vocab]: which = 0 the last verified target p_R
+ * (or the prefill / vanilla readout), 1 / 2 the root branch's stored first / second proposal readout. */
+int loopspec_debug_logits(loopspec_ctx*, int32_t seq, int32_t which, float* out_V);
+
+/* Algorithmic HBM bytes of one batched pass with the current rows (weights + KV read + lm_head if any
+ * branch reads out), and of one vanilla token at the current context.  Host arithmetic only. */
+int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);
+
+/* Time `iters` back-to-back launches of one kernel of the pass in the decode launch configuration, cycling
+ * over the layers' weights (so successive launches read different memory): which = 0 qkv, 1 o-proj,
+ * 2 gate/up, 3 down, 4 lm_head.  rows = token rows carried.  ms_out: mean milliseconds per launch measured
+ * with CUDA events on the context's stream; bytes_out: weight bytes one launch streams. */
+int loopspec_time_kernel(loopspec_ctx*, int32_t which, int32_t rows, int32_t iters, float* ms_out,
+                         double* bytes_out);
+
+/* Stand-alone linear map y[M][N] = x[M][K] * W[N][K]^T through the same weight-streaming kernel (token
+ * activations split into three bf16 terms, fp32 accumulation; fp32 weights use the CUDA-core path).
+ * All pointers device; x, y fp32; scratch: device, loopspec_linear_scratch_bytes(M, N, K) bytes, zeroed
+ * once by the caller before first use (the kernel leaves it zeroed where it must be).  M <= 64. */
+size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K);
+int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N,
+                       int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream);
+
+const char* loopspec_last_error(loopspec_ctx*);
+int loopspec_destroy(loopspec_ctx*);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOOPSPEC_H */

@@ -1,0 +1,8 @@
+"""B200-native LoopSpec decode path: a thin ctypes binding over the C-ABI library `libloopspec.so`.
+
+Every step of the path (batched recurrence, readouts, drafting, gate, cascade verification, KV rollback,
+scheduling) runs in the library's CUDA kernels; this package only marshals arguments.  PyTorch is used for
+device memory and streams.  There is no CPU fallback: importing fails if the library cannot be loaded.
+"""
+from .binding import (LoopSpec, LoopSpecError, lib, linear, linear_scratch_bytes, max_branches, pick_depths,  # noqa: F401
+                      upload_weights, EXPORTS)

@@ -1,0 +1,89 @@
+// Shared device-side declarations of the LoopSpec decode path: the row table every kernel of a batched
+// pass reads, the branch (node) table of Algorithm 1, and small numeric helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ls {
+
+constexpr int MAX_ROWS = 64;  // rows (branches) one batched pass can carry: 8 token columns x up to 8 groups
+constexpr int MAX_SPEC = 8;   // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
+constexpr int ATT_CHUNK = 64; // key positions per attention work item (fixed by absolute position)
+
+// readout kinds of a row after its advance (Algorithm 1: r_b = d1, r_b = d2, r_b = R)
+enum { RO_NONE = 0, RO_D1 = 1, RO_D2 = 2, RO_VERIFY = 3, RO_TARGET = 4 /* x ~ C(H): prefill, vanilla */ };
+
+// One batched pass = the rows below.  A row is one branch: one token position at one recurrent depth.
+struct RowTable {
+  int n_rows;
+  int n_readout;             // rows whose new depth is d1, d2 or R
+  int attn_items;            // sum over rows of attention chunks
+  int n_layers_done;         // unused, keeps the header 16 bytes
+  int seq[MAX_ROWS];         // sequence of the row
+  int r[MAX_ROWS];           // recurrence the row is advanced TO (1..R): KV plane it writes and reads
+  int pos[MAX_ROWS];         // position of the row's token (rotary index)
+  int kv_slot[MAX_ROWS];     // slot its K,V are written to
+  int n_canon[MAX_ROWS];     // committed slots [0, n_canon) it attends to
+  int n_spec[MAX_ROWS];      // speculative slots it attends to (its uncommitted ancestors and itself)
+  int spec_slot[MAX_ROWS][MAX_SPEC];
+  int hid_idx[MAX_ROWS];     // where its hidden state lives (updated in place)
+  int readout[MAX_ROWS];     // RO_*
+  int logit_idx[MAX_ROWS];   // which logits vector its readout fills
+  int node[MAX_ROWS];        // global node index (seq * NB + node), -1 for prefill rows
+  int ro_rows[MAX_ROWS];     // compact list of rows with readout != 0
+  int chunk_start[MAX_ROWS + 1];  // exclusive prefix sum of attention chunks per row
+};
+
+// Branch table of Algorithm 1 (a branch: prefix, hidden state, depth, proposal records), per sequence NB nodes.
+struct NodeTable {
+  int* state;    // 0 free, 1 active
+  int* depth;    // r_b
+  int* pos;      // position of the last token of the prefix
+  int* token;    // that token
+  int* parent;   // node index within the sequence, -1 for the root (whole prefix committed)
+  int* child1;   // record 1: child spawned for the first proposal
+  int* child2;   // record 2
+  int* tok1;
+  int* tok2;
+  int* has2;     // the gate opened and record 2 exists
+  float* lse1;   // log-sum-exp of z/T of the first readout
+  float* lse2;
+  float* z2;     // sum of [q2~ - q1]_+ (normaliser of the residual proposal), 0 if it had no mass
+};
+
+struct SeqState {
+  int* root;         // node index of the root branch, -1 if the sequence is idle
+  int* n_ids;        // committed tokens (prompt + decoded)
+  int* n_dec;        // decoded tokens since prefill (excluding the prefill token)
+  int* n_target;     // decode stops committing for the sequence at this many
+  int* need_verify;  // set by the step phase when the root reached R
+};
+
+struct Counters {  // App. C / App. D statistics
+  unsigned long long steps, n_decode, n_accept1, n_accept2, n_restart, gate_evals, gate_opens, rows_total, rows_max,
+      readout_rows_total;
+};
+
+struct KvCopyCmd {
+  int src_slot, dst_slot, n_planes, pad;
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(unsigned short b) { return __uint_as_float(((unsigned)b) << 16); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// programmatic dependent launch: wait for the kernels this launch depends on / let dependents start launching
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+}  // namespace ls

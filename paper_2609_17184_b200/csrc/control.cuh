@@ -1,0 +1,408 @@
+// Device-resident scheduler: the branch bookkeeping of Algorithm 1 (Spawn, the readout branches at d1/d2,
+// Verify's outcome, Reroot) and the construction of the next pass's row table, so that a decode step is a
+// CUDA-graph replay with no host round trip.  All kernels here run as ONE CTA: the tables are a few KB,
+// are pulled into shared memory, updated there (one thread per sequence) and written back.
+#pragma once
+#include "common.cuh"
+
+namespace ls {
+
+constexpr int CTRL_THREADS = 256;
+constexpr int MAX_NODES = 512;   // max_seqs * nodes-per-sequence
+enum { PH_ADVANCE = 1, PH_VERIFY = 2, PH_BUILD = 4 };
+enum { HF_ERROR = 0, HF_MIN_DEC = 1, HF_N_ROWS = 2, HF_NEED_VERIFY = 3, HF_FIRST_TOKEN = 4, HF_COUNT = 8 };
+enum { ERR_NODES = 1, ERR_CTX = 2, ERR_SPEC = 3 };
+
+struct ControlParams {
+  RowTable* tab;
+  NodeTable nodes;
+  SeqState seqs;
+  Counters* ctr;
+  int S, NB, R, d1, d2, ctx_cap;
+  const int* sel_tok;
+  const int* sel_aux;
+  const float* sel_lse;
+  const float* sel_z2;
+  int phases;
+  int* out_ids;      // [S][ids_cap] decoded tokens since prefill
+  int ids_cap;
+  int* commits;      // [S][ids_cap][8]
+  int* row_trace;    // [trace_cap], trace_n[0] entries used
+  int* trace_n;
+  int trace_cap;
+  KvCopyCmd* kvcopy; // [S]
+  float* hid;        // [hid_idx][H]
+  int H;
+  const void* embed; // [V][H]
+  int weight_dtype;
+  int p_logit_base;  // logits index of sequence 0's target readout
+  volatile int* host_flags;  // pinned, host-mapped
+};
+
+struct NodeSmem {
+  int state[MAX_NODES], depth[MAX_NODES], pos[MAX_NODES], token[MAX_NODES], parent[MAX_NODES], child1[MAX_NODES],
+      child2[MAX_NODES], tok1[MAX_NODES], tok2[MAX_NODES], has2[MAX_NODES];
+  float lse1[MAX_NODES], lse2[MAX_NODES], z2[MAX_NODES];
+};
+
+__device__ __forceinline__ void nodes_load(NodeSmem& s, const NodeTable& g, int n) {
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    s.state[i] = g.state[i], s.depth[i] = g.depth[i], s.pos[i] = g.pos[i], s.token[i] = g.token[i];
+    s.parent[i] = g.parent[i], s.child1[i] = g.child1[i], s.child2[i] = g.child2[i], s.tok1[i] = g.tok1[i];
+    s.tok2[i] = g.tok2[i], s.has2[i] = g.has2[i], s.lse1[i] = g.lse1[i], s.lse2[i] = g.lse2[i], s.z2[i] = g.z2[i];
+  }
+}
+__device__ __forceinline__ void nodes_store(const NodeSmem& s, const NodeTable& g, int n) {
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    g.state[i] = s.state[i], g.depth[i] = s.depth[i], g.pos[i] = s.pos[i], g.token[i] = s.token[i];
+    g.parent[i] = s.parent[i], g.child1[i] = s.child1[i], g.child2[i] = s.child2[i], g.tok1[i] = s.tok1[i];
+    g.tok2[i] = s.tok2[i], g.has2[i] = s.has2[i], g.lse1[i] = s.lse1[i], g.lse2[i] = s.lse2[i], g.z2[i] = s.z2[i];
+  }
+}
+
+// P of Eq. 1 for the Ouro layout: hidden state at depth 0 = embedding row of the prefix's last token
+__device__ __forceinline__ void embed_rows(const int (*list)[2], int n, float* hid, int H, const void* embed, int wdt) {
+  for (int e = 0; e < n; ++e) {
+    float* dst = hid + (size_t)list[e][0] * H;
+    if (wdt == 1) {
+      const unsigned short* src = static_cast<const unsigned short*>(embed) + (size_t)list[e][1] * H;
+      for (int i = threadIdx.x; i < H; i += blockDim.x) dst[i] = bf16_bits_to_float(src[i]);
+    } else {
+      const float* src = static_cast<const float*>(embed) + (size_t)list[e][1] * H;
+      for (int i = threadIdx.x; i < H; i += blockDim.x) dst[i] = src[i];
+    }
+  }
+}
+
+__device__ __forceinline__ int alloc_node(int* state, int NB) {
+  for (int i = 0; i < NB; ++i)
+    if (!state[i]) return i;
+  return -1;
+}
+
+// Fill the row table from the active branches (thread 0; tables live in shared memory).
+__device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, const int* n_dec, const int* n_target,
+                           const ControlParams& p, int* err) {
+  int n_rows = 0, n_ro = 0, items = 0;
+  for (int s = 0; s < p.S; ++s) {
+    if (root[s] < 0 || n_dec[s] >= n_target[s]) continue;
+    const int o = s * p.NB;
+    const int rt = root[s];
+    for (int n = 0; n < p.NB; ++n) {
+      if (!nd.state[o + n]) continue;
+      if (n_rows >= MAX_ROWS) { *err = ERR_NODES; break; }
+      const int i = n_rows++;
+      const int r = nd.depth[o + n] + 1;
+      const bool is_root = nd.parent[o + n] < 0;
+      t.seq[i] = s, t.r[i] = r, t.pos[i] = nd.pos[o + n], t.node[i] = o + n, t.hid_idx[i] = o + n;
+      t.kv_slot[i] = is_root ? nd.pos[o + n] : p.ctx_cap + n;
+      t.n_canon[i] = nd.pos[o + rt] + 1;
+      if (nd.pos[o + n] + 2 >= p.ctx_cap) *err = ERR_CTX;
+      int chain[MAX_SPEC], len = 0;
+      for (int a = n; a >= 0 && nd.parent[o + a] >= 0; a = nd.parent[o + a]) {
+        if (len >= MAX_SPEC) { *err = ERR_SPEC; break; }
+        chain[len++] = a;
+      }
+      t.n_spec[i] = len;
+      for (int j = 0; j < len; ++j) t.spec_slot[i][j] = p.ctx_cap + chain[len - 1 - j];
+      int ro = RO_NONE, li = 0;
+      if (r == p.d1) ro = RO_D1, li = (o + n) * 2;
+      else if (p.d2 > 0 && r == p.d2) ro = RO_D2, li = (o + n) * 2 + 1;
+      else if (r == p.R) ro = RO_VERIFY, li = p.p_logit_base + s;
+      t.readout[i] = ro, t.logit_idx[i] = li;
+      if (ro) t.ro_rows[n_ro++] = i;
+      t.chunk_start[i] = items;
+      items += (t.n_canon[i] + ATT_CHUNK - 1) / ATT_CHUNK + (len > 0 ? 1 : 0);
+    }
+  }
+  t.chunk_start[n_rows] = items;
+  t.n_rows = n_rows, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
+}
+
+__global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const ControlParams p) {
+  __shared__ NodeSmem nd;
+  __shared__ RowTable t;
+  __shared__ int s_root[MAX_ROWS], s_nids[MAX_ROWS], s_ndec[MAX_ROWS], s_ntarget[MAX_ROWS], s_needv[MAX_ROWS];
+  __shared__ int s_emb[2 * MAX_ROWS][2];
+  __shared__ int s_nemb, s_err;
+  const int tid = threadIdx.x;
+  const int n_nodes = p.S * p.NB;
+  nodes_load(nd, p.nodes, n_nodes);
+  {
+    const int* src = reinterpret_cast<const int*>(p.tab);
+    int* dst = reinterpret_cast<int*>(&t);
+    for (int i = tid; i < (int)(sizeof(RowTable) / 4); i += CTRL_THREADS) dst[i] = src[i];
+  }
+  if (tid < p.S) {
+    s_root[tid] = p.seqs.root[tid], s_nids[tid] = p.seqs.n_ids[tid], s_ndec[tid] = p.seqs.n_dec[tid];
+    s_ntarget[tid] = p.seqs.n_target[tid], s_needv[tid] = p.seqs.need_verify[tid];
+  }
+  if (tid == 0) s_nemb = 0, s_err = 0;
+  __syncthreads();
+
+  if (tid < p.S) {
+    const int s = tid, o = s * p.NB;
+    int* st = nd.state + o;
+    // ---- advance, first proposal at d1, gated second proposal at d2 (Algorithm 1 main loop body) ----
+    if (p.phases & PH_ADVANCE) {
+      for (int i = 0; i < t.n_rows; ++i)
+        if (t.seq[i] == s) nd.depth[t.node[i]] = t.r[i];
+      for (int i = 0; i < t.n_rows; ++i) {
+        if (t.seq[i] != s) continue;
+        const int gn = t.node[i], ro = t.readout[i];
+        if (ro == RO_D1 || (ro == RO_D2 && p.sel_aux[i])) {
+          int c = alloc_node(st, p.NB);
+          if (c < 0) { s_err = ERR_NODES; continue; }
+          st[c] = 1, nd.depth[o + c] = 0, nd.pos[o + c] = nd.pos[gn] + 1, nd.token[o + c] = p.sel_tok[i];
+          nd.parent[o + c] = gn - o, nd.child1[o + c] = nd.child2[o + c] = -1, nd.has2[o + c] = 0;
+          if (ro == RO_D1) {
+            nd.tok1[gn] = p.sel_tok[i], nd.child1[gn] = c, nd.lse1[gn] = p.sel_lse[i], nd.has2[gn] = 0, nd.child2[gn] = -1;
+          } else {
+            nd.tok2[gn] = p.sel_tok[i], nd.child2[gn] = c, nd.lse2[gn] = p.sel_lse[i], nd.z2[gn] = p.sel_z2[i], nd.has2[gn] = 1;
+            atomicAdd(&p.ctr->gate_opens, 1ull);
+          }
+          int e = atomicAdd(&s_nemb, 1);
+          s_emb[e][0] = o + c, s_emb[e][1] = p.sel_tok[i];
+        }
+        if (ro == RO_D2) atomicAdd(&p.ctr->gate_evals, 1ull);
+        if (ro == RO_VERIFY) s_needv[s] = 1;
+      }
+    }
+    // ---- the deepest branch reached R: commit and Reroot ---------------------------------------------
+    p.kvcopy[s].n_planes = 0;
+    if ((p.phases & PH_VERIFY) && s_needv[s]) {
+      int vrow = -1;
+      for (int i = 0; i < t.n_rows; ++i)
+        if (t.seq[i] == s && t.readout[i] == RO_VERIFY) vrow = i;
+      const int rt = s_root[s];
+      const int tok = p.sel_tok[vrow], src = p.sel_aux[vrow];
+      const int k = s_ndec[s];
+      if (k < p.ids_cap) {
+        p.out_ids[(size_t)s * p.ids_cap + k] = tok;
+        int* cm = p.commits + ((size_t)s * p.ids_cap + k) * 8;
+        cm[0] = s, cm[1] = 1, cm[2] = tok, cm[3] = src, cm[4] = (src == 1), cm[5] = (src == 2), cm[6] = nd.has2[o + rt];
+        cm[7] = (int)p.ctr->steps + ((p.phases & PH_ADVANCE) ? 1 : 0);
+      }
+      s_ndec[s] = k + 1, s_nids[s] += 1;
+      atomicAdd(&p.ctr->n_decode, 1ull);
+      atomicAdd(src == 1 ? &p.ctr->n_accept1 : (src == 2 ? &p.ctr->n_accept2 : &p.ctr->n_restart), 1ull);
+      const int keep = src == 1 ? nd.child1[o + rt] : (src == 2 ? nd.child2[o + rt] : -1);
+      const int new_pos = nd.pos[o + rt] + 1;
+      for (int n = 0; n < p.NB; ++n) {
+        if (!st[n]) continue;
+        bool in = false;
+        for (int a = n; a >= 0; a = nd.parent[o + a])
+          if (a == keep) { in = true; break; }
+        if (!in) st[n] = 0;
+      }
+      if (keep < 0) {  // restart: fresh branch on the verified prefix
+        const int c = alloc_node(st, p.NB);
+        st[c] = 1, nd.depth[o + c] = 0, nd.pos[o + c] = new_pos, nd.token[o + c] = tok, nd.parent[o + c] = -1;
+        nd.child1[o + c] = nd.child2[o + c] = -1, nd.has2[o + c] = 0;
+        s_root[s] = c;
+        int e = atomicAdd(&s_nemb, 1);
+        s_emb[e][0] = o + c, s_emb[e][1] = tok;
+      } else {         // keep the chosen child and its descendants; its KV joins the committed prefix
+        nd.parent[o + keep] = -1;
+        s_root[s] = keep;
+        p.kvcopy[s].src_slot = p.ctx_cap + keep, p.kvcopy[s].dst_slot = nd.pos[o + keep];
+        p.kvcopy[s].n_planes = nd.depth[o + keep];
+      }
+      s_needv[s] = 0;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    if (p.phases & PH_ADVANCE) {
+      p.ctr->steps += 1, p.ctr->rows_total += t.n_rows, p.ctr->readout_rows_total += t.n_readout;
+      if ((unsigned long long)t.n_rows > p.ctr->rows_max) p.ctr->rows_max = t.n_rows;
+      int k = *p.trace_n;
+      if (k < p.trace_cap) p.row_trace[k] = t.n_rows;
+      *p.trace_n = k + 1;
+    }
+    int need = 0, min_dec = 0x7fffffff;
+    for (int s = 0; s < p.S; ++s) {
+      need += s_needv[s];
+      if (s_root[s] >= 0) min_dec = min(min_dec, s_ndec[s]);
+    }
+    int err = s_err;
+    // rows are rebuilt only when no verification is pending (the verify phase needs the current rows)
+    if ((p.phases & PH_BUILD) && need == 0) build_rows(t, nd, s_root, s_ndec, s_ntarget, p, &err);
+    p.host_flags[HF_MIN_DEC] = min_dec, p.host_flags[HF_N_ROWS] = t.n_rows, p.host_flags[HF_NEED_VERIFY] = need;
+    if (err) p.host_flags[HF_ERROR] = err;
+  }
+  __syncthreads();
+  nodes_store(nd, p.nodes, n_nodes);
+  {
+    int* dst = reinterpret_cast<int*>(p.tab);
+    const int* src = reinterpret_cast<const int*>(&t);
+    for (int i = tid; i < (int)(sizeof(RowTable) / 4); i += CTRL_THREADS) dst[i] = src[i];
+  }
+  if (tid < p.S) {
+    p.seqs.root[tid] = s_root[tid], p.seqs.n_ids[tid] = s_nids[tid], p.seqs.n_dec[tid] = s_ndec[tid];
+    p.seqs.need_verify[tid] = s_needv[tid];
+  }
+  embed_rows(s_emb, s_nemb, p.hid, p.H, p.embed, p.weight_dtype);
+}
+
+// ---- vanilla decoding (Fig. 1a): one row per sequence, R passes per token ---------------------------
+struct VanillaParams {
+  RowTable* tabs;   // [R] one table per recurrence
+  NodeTable nodes;
+  SeqState seqs;
+  int S, NB, R;
+  const int* sel_tok;
+  int commit;       // 0: set up from the current committed prefix; 1: commit sel_tok of each sequence first
+  int* out_ids;
+  int ids_cap;
+  float* hid;
+  int H;
+  const void* embed;
+  int weight_dtype, p_logit_base, ctx_cap;
+  volatile int* host_flags;
+};
+
+__global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const VanillaParams p) {
+  __shared__ int s_emb[MAX_ROWS][2];
+  __shared__ int s_rowof[MAX_ROWS];
+  __shared__ int s_n;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    int n = 0;
+    const RowTable& cur = p.tabs[p.R - 1];
+    for (int s = 0; s < p.S; ++s) {
+      int rt = p.seqs.root[s];
+      if (rt < 0) continue;
+      const int o = s * p.NB;
+      if (p.commit) {
+        int row = -1;
+        for (int i = 0; i < cur.n_rows; ++i)
+          if (cur.seq[i] == s) row = i;
+        int tok = p.sel_tok[row];
+        int k = p.seqs.n_dec[s];
+        if (k < p.ids_cap) p.out_ids[(size_t)s * p.ids_cap + k] = tok;
+        p.seqs.n_dec[s] = k + 1, p.seqs.n_ids[s] += 1;
+        p.nodes.token[o + rt] = tok, p.nodes.pos[o + rt] += 1;
+      } else {
+        for (int i = 0; i < p.NB; ++i)
+          if (i != rt) p.nodes.state[o + i] = 0;
+      }
+      p.nodes.depth[o + rt] = 0, p.nodes.child1[o + rt] = p.nodes.child2[o + rt] = -1, p.nodes.has2[o + rt] = 0;
+      p.seqs.need_verify[s] = 0;
+      if (p.nodes.pos[o + rt] + 2 >= p.ctx_cap) p.host_flags[HF_ERROR] = ERR_CTX;
+      s_emb[n][0] = o + rt, s_emb[n][1] = p.nodes.token[o + rt];
+      s_rowof[n] = s;
+      ++n;
+    }
+    s_n = n;
+    for (int r = 1; r <= p.R; ++r) {
+      RowTable& t = p.tabs[r - 1];
+      int items = 0;
+      for (int i = 0; i < n; ++i) {
+        int s = s_rowof[i], gn = s_emb[i][0], pos = p.nodes.pos[gn];
+        t.seq[i] = s, t.r[i] = r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
+        t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE;
+        t.logit_idx[i] = p.p_logit_base + s, t.ro_rows[i] = i, t.chunk_start[i] = items;
+        items += (pos + 1 + ATT_CHUNK - 1) / ATT_CHUNK;
+      }
+      t.chunk_start[n] = items;
+      t.n_rows = n, t.n_readout = (r == p.R) ? n : 0, t.attn_items = items, t.n_layers_done = 0;
+    }
+  }
+  __syncthreads();
+  embed_rows(s_emb, s_n, p.hid, p.H, p.embed, p.weight_dtype);
+}
+
+// ---- prefill (Algorithm 1, lines before the main loop): rows = consecutive prompt positions ---------
+struct PrefillParams {
+  RowTable* tab;
+  const int* prompt;  // device ids of the sequence
+  int seq, p0, count, r, R, n_prompt;
+  int hid_base;       // first hidden-state index of the prefill rows
+  int p_logit_base;
+  float* hid;
+  int H;
+  const void* embed;
+  int weight_dtype;
+};
+
+__global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const PrefillParams p) {
+  __shared__ int s_emb[MAX_ROWS][2];
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    RowTable& t = *p.tab;
+    int items = 0, n_ro = 0;
+    for (int i = 0; i < p.count; ++i) {
+      int pos = p.p0 + i;
+      t.seq[i] = p.seq, t.r[i] = p.r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
+      t.hid_idx[i] = p.hid_base + i, t.node[i] = -1;
+      bool last = (p.r == p.R) && (pos == p.n_prompt - 1);
+      t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;
+      if (last) t.ro_rows[n_ro++] = i;
+      t.chunk_start[i] = items;
+      items += (pos + 1 + ATT_CHUNK - 1) / ATT_CHUNK;
+      s_emb[i][0] = p.hid_base + i, s_emb[i][1] = p.prompt[pos];
+    }
+    t.chunk_start[p.count] = items;
+    t.n_rows = p.count, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
+  }
+  __syncthreads();
+  if (p.r == 1) embed_rows(s_emb, p.count, p.hid, p.H, p.embed, p.weight_dtype);
+}
+
+struct PrefillFinishParams {
+  const RowTable* tab;
+  NodeTable nodes;
+  SeqState seqs;
+  int seq, NB, n_prompt, n_target;
+  const int* sel_tok;
+  float* hid;
+  int H;
+  const void* embed;
+  int weight_dtype;
+  volatile int* host_flags;
+};
+
+// commit the first token and Spawn(prompt || token) as the root branch at depth 0
+__global__ void __launch_bounds__(CTRL_THREADS) prefill_finish_kernel(const PrefillFinishParams p) {
+  __shared__ int s_emb[1][2];
+  if (threadIdx.x == 0) {
+    const int o = p.seq * p.NB;
+    const int tok = p.sel_tok[p.tab->ro_rows[0]];
+    for (int i = 0; i < p.NB; ++i) p.nodes.state[o + i] = 0;
+    p.nodes.state[o] = 1, p.nodes.depth[o] = 0, p.nodes.pos[o] = p.n_prompt, p.nodes.token[o] = tok, p.nodes.parent[o] = -1;
+    p.nodes.child1[o] = p.nodes.child2[o] = -1, p.nodes.has2[o] = 0;
+    p.seqs.root[p.seq] = 0, p.seqs.n_ids[p.seq] = p.n_prompt + 1, p.seqs.n_dec[p.seq] = 0;
+    p.seqs.n_target[p.seq] = p.n_target, p.seqs.need_verify[p.seq] = 0;
+    p.host_flags[HF_FIRST_TOKEN] = tok;
+    s_emb[0][0] = o, s_emb[0][1] = tok;
+  }
+  __syncthreads();
+  embed_rows(s_emb, 1, p.hid, p.H, p.embed, p.weight_dtype);
+}
+
+// ---- KV rollback / commit: the kept branch's keys and values become the committed ones of its position ---
+struct KvCommitParams {
+  const KvCopyCmd* cmds;  // [S]
+  __nv_bfloat16* kv;      // whole pool [L][R][2][S][n_kv][slots][d]
+  long long layer_stride, plane_stride, sel_stride;
+  int S, L, n_kv_heads, slots, d;
+};
+
+__global__ void kv_commit_kernel(const KvCommitParams p) {
+  // grid: (L, R, 2 * S); one CTA copies n_kv_heads rows of d bf16
+  const int l = blockIdx.x, plane = blockIdx.y, sel = blockIdx.z & 1, s = blockIdx.z >> 1;
+  const KvCopyCmd c = p.cmds[s];
+  if (plane >= c.n_planes) return;
+  __nv_bfloat16* base = p.kv + (size_t)l * p.layer_stride + (size_t)plane * p.plane_stride + (size_t)sel * p.sel_stride;
+  const int per_head = p.d / 8;  // uint4 per head row
+  for (int i = threadIdx.x; i < p.n_kv_heads * per_head; i += blockDim.x) {
+    int h = i / per_head, j = i % per_head;
+    size_t hb = (size_t)(s * p.n_kv_heads + h) * p.slots;
+    const uint4* src = reinterpret_cast<const uint4*>(base + (hb + c.src_slot) * p.d) + j;
+    uint4* dst = reinterpret_cast<uint4*>(base + (hb + c.dst_slot) * p.d) + j;
+    *dst = *src;
+  }
+}
+
+}  // namespace ls

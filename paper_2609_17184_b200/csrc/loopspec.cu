@@ -1,0 +1,942 @@
+// C ABI of the LoopSpec decode path (see include/loopspec.h): context, workspace layout, the launch
+// sequence of one batched pass, CUDA-graph capture of the decode step and the host side of the scheduler.
+#include "../../include/loopspec.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "control.cuh"
+#include "gemm.cuh"
+#include "select.cuh"
+
+using namespace ls;
+
+namespace {
+
+constexpr int kCtasPerSm = 2;
+
+struct GemmPlan {
+  int n_rb, kpr, upc, total, grid, max_contrib;
+};
+
+GemmPlan plan_gemm(int n_rb, int K, int target_ctas) {
+  GemmPlan g;
+  g.n_rb = n_rb;
+  g.kpr = (K + 31) / 32;
+  g.total = g.n_rb * g.kpr;
+  int grid = std::min(target_ctas, g.total);
+  g.upc = (g.total + grid - 1) / grid;
+  g.grid = (g.total + g.upc - 1) / g.upc;
+  g.max_contrib = 1;
+  for (int rb = 0; rb < n_rb; ++rb) {
+    int cf = (rb * g.kpr) / g.upc, cl = ((rb + 1) * g.kpr - 1) / g.upc;
+    g.max_contrib = std::max(g.max_contrib, cl - cf + 1);
+  }
+  return g;
+}
+
+size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
+
+struct Layout {  // byte offsets into the workspace
+  size_t rope, kv, hid, qbuf, abuf, sbuf, sumsq, logits, gpart, gcnt, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
+      tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
+};
+
+struct Derived {
+  int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, max_chunks,
+      trace_cap, Hq, Hkv, d1, d2;
+  size_t gpart_floats, gcnt_ints;
+};
+
+int max_branches(int R, int d1, int d2) {
+  int n = R / d1;
+  if (d2 == 0) return n;
+  int lag = d2 / d1;
+  std::vector<long long> s(n);
+  long long tot = 0;
+  for (int k = 0; k < n; ++k) {
+    s[k] = k < lag ? 1 : s[k - 1] + s[k - lag];
+    tot += s[k];
+  }
+  return (int)std::min<long long>(tot, 1 << 20);
+}
+
+// Theorem 2 / Eq. 8
+void closed_form(double a, double b, double R, double* d1, double* d2) {
+  double D = a * a + a + 1.0, ab = a * b, tar = 2.0 * a * R;
+  *d1 = std::pow(ab, (a + 1.0) / D) * std::pow(tar, 1.0 / D);
+  *d2 = std::pow(ab, a / D) * std::pow(tar, (a + 1.0) / D);
+}
+double steps_bound(double d1, double d2, double a, double b, double R) {
+  return d1 + b * std::pow(d1, -a) * d2 + 2.0 * b * std::pow(d2, -a) * R;
+}
+bool snap_depths(double a, double b, int R, int* o1, int* o2) {
+  double best = 0;
+  bool found = false;
+  for (int x = 1; x < R; ++x)
+    for (int y = x + 1; y < R; ++y) {
+      if (y % x || R % x) continue;
+      double f = steps_bound(x, y, a, b, R);
+      if (!found || f < best) best = f, *o1 = x, *o2 = y, found = true;
+    }
+  return found;
+}
+
+bool validate_model(const loopspec_model* m, int* why) {
+  *why = LOOPSPEC_EINVAL;
+  if (!m) return false;
+  if (m->vocab <= 0 || m->hidden <= 0 || m->n_q_heads <= 0 || m->n_kv_heads <= 0 || m->ffn <= 0 || m->R < 2 ||
+      m->n_recurrent <= 0 || (m->weight_dtype != 0 && m->weight_dtype != 1) || !(m->rms_eps > 0) || !(m->rope_theta > 0))
+    return false;
+  if (m->n_q_heads % m->n_kv_heads) return false;
+  *why = LOOPSPEC_EUNSUPPORTED;
+  if (m->n_prelude || m->n_coda) return false;
+  if (m->head_dim != 64 && m->head_dim != 128) return false;
+  int g = m->n_q_heads / m->n_kv_heads;
+  if (g != 1 && g != 4) return false;
+  if (m->hidden % 128 || (m->n_q_heads * m->head_dim) % 128 || (m->n_kv_heads * m->head_dim) % 128) return false;
+  if (m->ffn % 16 || m->vocab % 16) return false;
+  return true;
+}
+
+bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d, int* why) {
+  *why = LOOPSPEC_EINVAL;
+  if (!s || s->max_seqs <= 0 || s->max_ctx < 4 || s->temperature < 0 || s->max_prefill_rows < 0) return false;
+  int d1 = s->d1, d2 = s->d2;
+  if (d1 == 0 && d2 == 0) {
+    if (!(s->alpha > 0) || !(s->beta > 0)) return false;
+    if (!snap_depths(s->alpha, s->beta, m->R, &d1, &d2)) {  // R too small for two proposals
+      d1 = 1, d2 = 0;
+    }
+  }
+  if (d1 < 1 || d1 >= m->R || m->R % d1) return false;
+  if (d2 != 0 && (d2 <= d1 || d2 >= m->R || d2 % d1)) return false;
+  d->d1 = d1, d->d2 = d2;
+  *why = LOOPSPEC_ECAPACITY;
+  d->S = s->max_seqs;
+  d->B = max_branches(m->R, d1, d2);
+  d->NB = 2 * d->B + 1;
+  if (m->R / d1 > MAX_SPEC) return false;
+  if (d->S > MAX_ROWS || d->S * d->NB > MAX_NODES || d->S * d->B > MAX_ROWS) return false;
+  d->max_rows_dec = d->S * d->B;
+  d->max_rows_pf = s->max_prefill_rows ? s->max_prefill_rows : 32;
+  if (d->max_rows_pf > MAX_ROWS) return false;
+  d->max_rows = 8 * ng_for_rows(std::max(d->max_rows_dec, d->max_rows_pf));
+  d->slots = s->max_ctx + d->NB;
+  d->ids_cap = s->max_ctx;
+  d->n_hid = d->S * d->NB + MAX_ROWS;
+  d->p_logit_base = d->S * d->NB * 2;
+  d->n_logit_vecs = d->p_logit_base + d->S;
+  d->n_sq = m->hidden / 128;
+  d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK + 1;
+  d->trace_cap = 4 * s->max_ctx + 64;
+  d->Hq = m->n_q_heads * m->head_dim;
+  d->Hkv = m->n_kv_heads * m->head_dim;
+  return true;
+}
+
+Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Derived& d, int n_sm) {
+  Layout L;
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o = align_up(o + bytes);
+    return at;
+  };
+  const size_t MR = d.max_rows;
+  L.rope = take((size_t)s->max_ctx * (m->head_dim / 2) * sizeof(float2));
+  L.kv = take((size_t)m->n_recurrent * m->R * 2 * d.S * m->n_kv_heads * d.slots * m->head_dim * 2);
+  L.hid = take((size_t)d.n_hid * m->hidden * 4);
+  L.qbuf = take(MR * d.Hq * 4);
+  L.abuf = take(MR * d.Hq * 4);
+  L.sbuf = take(MR * m->ffn * 4);
+  L.sumsq = take(MR * d.n_sq * 4);
+  L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
+  // split-k scratch: the largest of the five GEMMs at the widest token-group count in use
+  int target = n_sm * kCtasPerSm;
+  GemmPlan plans[5] = {plan_gemm((d.Hq + 2 * d.Hkv) / 128, m->hidden, target), plan_gemm(m->hidden / 128, d.Hq, target),
+                       plan_gemm((m->ffn + 63) / 64, m->hidden, target), plan_gemm(m->hidden / 128, m->ffn, target),
+                       plan_gemm((m->vocab + 127) / 128, m->hidden, target)};
+  size_t pf = 0, cnt = 0;
+  for (auto& g : plans) pf = std::max(pf, (size_t)g.n_rb * g.max_contrib), cnt = std::max(cnt, (size_t)g.n_rb);
+  L.gpart = take(pf * MR * 128 * 4);
+  L.gcnt = take(cnt * 4);
+  int G = m->n_q_heads / m->n_kv_heads;
+  L.apart = take(MR * m->n_kv_heads * d.max_chunks * G * (m->head_dim + 2) * 4);
+  L.acnt = take(MR * m->n_kv_heads * 4);
+  L.nodes = take((size_t)13 * MAX_NODES * 4);
+  L.seqs = take((size_t)5 * MAX_ROWS * 4);
+  L.ctr = take(sizeof(Counters));
+  L.tab_dec = take(sizeof(RowTable));
+  L.tab_pf = take(sizeof(RowTable));
+  L.tab_van = take(sizeof(RowTable) * m->R);
+  L.sel_tok = take(MAX_ROWS * 4);
+  L.sel_aux = take(MAX_ROWS * 4);
+  L.sel_lse = take(MAX_ROWS * 4);
+  L.sel_z2 = take(MAX_ROWS * 4);
+  L.kvcopy = take(MAX_ROWS * sizeof(KvCopyCmd));
+  L.out_ids = take((size_t)d.S * d.ids_cap * 4);
+  L.commits = take((size_t)d.S * d.ids_cap * 8 * 4);
+  L.trace = take((size_t)d.trace_cap * 4);
+  L.trace_n = take(4);
+  L.prompt = take((size_t)s->max_ctx * 4);
+  L.total = o;
+  return L;
+}
+
+}  // namespace
+
+struct loopspec_ctx {
+  loopspec_model m;
+  loopspec_sched s;
+  Derived d;
+  Layout L;
+  cudaStream_t stream = nullptr;
+  unsigned char* ws = nullptr;
+  const void* embed = nullptr;
+  const void* lm_head = nullptr;
+  const float* final_norm = nullptr;
+  std::vector<const void*> layers;  // 6 per layer
+  int n_sm = 148;
+  int ng_dec = 1, ng_pf = 1;
+  GemmPlan plan[5];
+  volatile int* host_flags = nullptr;  // pinned + mapped
+  int* host_flags_dev = nullptr;
+  int* pin_ids = nullptr;              // pinned staging for prompt / ids
+  size_t pin_ids_cap = 0;
+  cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  std::vector<char> prefilled;
+  bool pending_verify = false, sticky = false, vanilla_mode = false;
+  int launches_per_step = 0;
+  std::string err;
+
+  template <typename T>
+  T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  NodeTable nodes() const {
+    int* b = at<int>(L.nodes);
+    NodeTable n;
+    n.state = b, n.depth = b + MAX_NODES, n.pos = b + 2 * MAX_NODES, n.token = b + 3 * MAX_NODES;
+    n.parent = b + 4 * MAX_NODES, n.child1 = b + 5 * MAX_NODES, n.child2 = b + 6 * MAX_NODES, n.tok1 = b + 7 * MAX_NODES;
+    n.tok2 = b + 8 * MAX_NODES, n.has2 = b + 9 * MAX_NODES;
+    n.lse1 = reinterpret_cast<float*>(b + 10 * MAX_NODES), n.lse2 = reinterpret_cast<float*>(b + 11 * MAX_NODES);
+    n.z2 = reinterpret_cast<float*>(b + 12 * MAX_NODES);
+    return n;
+  }
+  SeqState seqs() const {
+    int* b = at<int>(L.seqs);
+    SeqState q;
+    q.root = b, q.n_ids = b + MAX_ROWS, q.n_dec = b + 2 * MAX_ROWS, q.n_target = b + 3 * MAX_ROWS, q.need_verify = b + 4 * MAX_ROWS;
+    return q;
+  }
+  long long kv_sel_stride() const { return (long long)d.S * m.n_kv_heads * d.slots * m.head_dim; }
+  long long kv_plane_stride() const { return 2 * kv_sel_stride(); }
+  long long kv_layer_stride() const { return (long long)m.R * kv_plane_stride(); }
+};
+
+namespace {
+
+int fail(loopspec_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    c->err = buf;
+    if (code == LOOPSPEC_ECUDA) c->sticky = true;
+  }
+  return code;
+}
+
+#define CU(c, call)                                                                                       \
+  do {                                                                                                    \
+    cudaError_t e_ = (call);                                                                              \
+    if (e_ != cudaSuccess) return fail(c, LOOPSPEC_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+// ---- kernel dispatch ---------------------------------------------------------------------------------
+using GemmFn = void (*)(const GemmParams);
+
+template <typename WT, int NG>
+GemmFn gemm_fn_epi(int epi) {
+  switch (epi) {
+    case EPI_PLAIN: return gemm_kernel<WT, NG, EPI_PLAIN>;
+    case EPI_QKV: return gemm_kernel<WT, NG, EPI_QKV>;
+    case EPI_RESID: return gemm_kernel<WT, NG, EPI_RESID>;
+    case EPI_SWIGLU: return gemm_kernel<WT, NG, EPI_SWIGLU>;
+    default: return gemm_kernel<WT, NG, EPI_LOGITS>;
+  }
+}
+template <typename WT>
+GemmFn gemm_fn_ng(int ng, int epi) {
+  switch (ng) {
+    case 1: return gemm_fn_epi<WT, 1>(epi);
+    case 2: return gemm_fn_epi<WT, 2>(epi);
+    case 4: return gemm_fn_epi<WT, 4>(epi);
+    default: return gemm_fn_epi<WT, 8>(epi);
+  }
+}
+GemmFn gemm_fn(int wdt, int ng, int epi) {
+  return wdt == 1 ? gemm_fn_ng<__nv_bfloat16>(ng, epi) : gemm_fn_ng<float>(ng, epi);
+}
+
+cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, int grid, cudaStream_t st) {
+  GemmFn fn = gemm_fn(wdt, ng, epi);
+  int smem = gemm_smem_bytes(ng);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+  }
+  fn<<<grid, GEMM_THREADS, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+using AttnFn = void (*)(const AttnParams);
+AttnFn attn_fn(int d, int G) {
+  if (d == 128) return G == 1 ? attn_kernel<128, 1> : attn_kernel<128, 4>;
+  return G == 1 ? attn_kernel<64, 1> : attn_kernel<64, 4>;
+}
+
+// ---- one batched pass through the shared block stack (all layers) on the rows of `tab` ------------------
+enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_LM = 4 };
+
+GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
+  const loopspec_model& m = c->m;
+  const Derived& d = c->d;
+  GemmParams p;
+  memset(&p, 0, sizeof p);
+  const GemmPlan& g = c->plan[which];
+  p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.units_per_cta = g.upc, p.total_units = g.total, p.max_contrib = g.max_contrib;
+  p.partials = c->at<float>(c->L.gpart), p.counters = c->at<int>(c->L.gcnt);
+  p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
+  const void* const* lp = which == G_LM ? nullptr : &c->layers[6 * layer];
+  switch (which) {
+    case G_QKV:
+      p.W = lp[1], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
+      p.xs_kind = XS_HID_NORM, p.gain = static_cast<const float*>(lp[0]);
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 0 : d.n_sq;
+      p.qbuf = c->at<float>(c->L.qbuf);
+      p.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)layer * c->kv_layer_stride();
+      p.kv_plane_stride = c->kv_plane_stride(), p.kv_sel_stride = c->kv_sel_stride();
+      p.slots = d.slots, p.n_kv_heads = m.n_kv_heads, p.n_q_heads = m.n_q_heads, p.head_dim = m.head_dim;
+      p.rope = c->at<float2>(c->L.rope);
+      break;
+    case G_O:
+      p.W = lp[2], p.N = m.hidden, p.K = d.Hq;
+      p.xs_kind = XS_BUF, p.xbuf = c->at<float>(c->L.abuf), p.x_ld = d.Hq;
+      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      break;
+    case G_GU:
+      p.W = lp[4], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
+      p.xs_kind = XS_HID_NORM, p.gain = static_cast<const float*>(lp[3]);
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq;
+      p.out = c->at<float>(c->L.sbuf), p.out_ld = m.ffn;
+      break;
+    case G_DOWN:
+      p.W = lp[5], p.N = m.hidden, p.K = m.ffn;
+      p.xs_kind = XS_BUF, p.xbuf = c->at<float>(c->L.sbuf), p.x_ld = m.ffn;
+      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      break;
+    default:
+      p.W = c->lm_head, p.N = m.vocab, p.K = m.hidden;
+      p.xs_kind = XS_HID_NORM_RO, p.gain = c->final_norm;
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq;
+      p.logits = c->at<float>(c->L.logits);
+      break;
+  }
+  return p;
+}
+
+const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
+
+cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch) {
+  const loopspec_model& m = c->m;
+  const Derived& d = c->d;
+  const int G = m.n_q_heads / m.n_kv_heads;
+  cudaError_t e;
+  for (int l = 0; l < m.n_recurrent; ++l) {
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->plan[G_QKV].grid, c->stream))) return e;
+    AttnParams a;
+    a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.abuf = c->at<float>(c->L.abuf);
+    a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
+    a.kv_plane_stride = c->kv_plane_stride(), a.kv_sel_stride = c->kv_sel_stride();
+    a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
+    a.scale = 1.0f / sqrtf((float)m.head_dim);
+    a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
+    attn_fn(m.head_dim, G)<<<c->n_sm * 4, ATT_THREADS, 0, c->stream>>>(a);
+    if ((e = cudaGetLastError())) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->plan[G_O].grid, c->stream))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->plan[G_GU].grid, c->stream))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->plan[G_DOWN].grid, c->stream))) return e;
+    if (n_launch) *n_launch += 5;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
+  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->plan[G_LM].grid, c->stream);
+}
+
+cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) {
+  SelectParams sp;
+  sp.tab = tab, sp.logits = c->at<float>(c->L.logits), sp.V = c->m.vocab, sp.NB = c->d.NB, sp.nodes = c->nodes();
+  sp.temperature = c->s.temperature, sp.gate = c->s.gate, sp.residual_q2 = c->s.residual_q2, sp.seed = c->s.seed;
+  sp.kinds_mask = kinds_mask;
+  sp.sel_tok = c->at<int>(c->L.sel_tok), sp.sel_aux = c->at<int>(c->L.sel_aux);
+  sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);
+  select_kernel<<<c->d.max_rows, SEL_THREADS, 0, c->stream>>>(sp);
+  return cudaGetLastError();
+}
+
+ControlParams control_params(loopspec_ctx* c, int phases) {
+  ControlParams p;
+  memset(&p, 0, sizeof p);
+  p.tab = c->at<RowTable>(c->L.tab_dec), p.nodes = c->nodes(), p.seqs = c->seqs(), p.ctr = c->at<Counters>(c->L.ctr);
+  p.S = c->d.S, p.NB = c->d.NB, p.R = c->m.R, p.d1 = c->d.d1, p.d2 = c->d.d2, p.ctx_cap = c->s.max_ctx;
+  p.sel_tok = c->at<int>(c->L.sel_tok), p.sel_aux = c->at<int>(c->L.sel_aux);
+  p.sel_lse = c->at<float>(c->L.sel_lse), p.sel_z2 = c->at<float>(c->L.sel_z2);
+  p.phases = phases;
+  p.out_ids = c->at<int>(c->L.out_ids), p.ids_cap = c->d.ids_cap, p.commits = c->at<int>(c->L.commits);
+  p.row_trace = c->at<int>(c->L.trace), p.trace_n = c->at<int>(c->L.trace_n), p.trace_cap = c->d.trace_cap;
+  p.kvcopy = c->at<KvCopyCmd>(c->L.kvcopy);
+  p.hid = c->at<float>(c->L.hid), p.H = c->m.hidden, p.embed = c->embed, p.weight_dtype = c->m.weight_dtype;
+  p.p_logit_base = c->d.p_logit_base, p.host_flags = c->host_flags_dev;
+  return p;
+}
+
+cudaError_t launch_control(loopspec_ctx* c, int phases) {
+  control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(control_params(c, phases));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_kv_commit(loopspec_ctx* c) {
+  KvCommitParams k;
+  k.cmds = c->at<KvCopyCmd>(c->L.kvcopy), k.kv = c->at<__nv_bfloat16>(c->L.kv);
+  k.layer_stride = c->kv_layer_stride(), k.plane_stride = c->kv_plane_stride(), k.sel_stride = c->kv_sel_stride();
+  k.S = c->d.S, k.L = c->m.n_recurrent, k.n_kv_heads = c->m.n_kv_heads, k.slots = c->d.slots, k.d = c->m.head_dim;
+  dim3 grid(c->m.n_recurrent, c->m.R, 2 * c->d.S);
+  kv_commit_kernel<<<grid, 128, 0, c->stream>>>(k);
+  return cudaGetLastError();
+}
+
+// the whole decode step: pass, readouts, decisions, bookkeeping, KV commit
+cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_commit, int* n_launch) {
+  const RowTable* tab = c->at<RowTable>(c->L.tab_dec);
+  cudaError_t e;
+  if ((e = launch_layers(c, tab, c->ng_dec, n_launch))) return e;
+  if ((e = launch_lm_head(c, tab, c->ng_dec))) return e;
+  if ((e = launch_select(c, tab, kinds_mask))) return e;
+  if ((e = launch_control(c, phases))) return e;
+  if (n_launch) *n_launch += 3;
+  if (kv_commit) {
+    if ((e = launch_kv_commit(c))) return e;
+    if (n_launch) *n_launch += 1;
+  }
+  return cudaSuccess;
+}
+
+VanillaParams vanilla_params(loopspec_ctx* c, int commit) {
+  VanillaParams v;
+  memset(&v, 0, sizeof v);
+  v.tabs = c->at<RowTable>(c->L.tab_van), v.nodes = c->nodes(), v.seqs = c->seqs();
+  v.S = c->d.S, v.NB = c->d.NB, v.R = c->m.R, v.sel_tok = c->at<int>(c->L.sel_tok), v.commit = commit;
+  v.out_ids = c->at<int>(c->L.out_ids), v.ids_cap = c->d.ids_cap;
+  v.hid = c->at<float>(c->L.hid), v.H = c->m.hidden, v.embed = c->embed, v.weight_dtype = c->m.weight_dtype;
+  v.p_logit_base = c->d.p_logit_base, v.ctx_cap = c->s.max_ctx, v.host_flags = c->host_flags_dev;
+  return v;
+}
+
+cudaError_t launch_vanilla_token(loopspec_ctx* c) {
+  cudaError_t e;
+  RowTable* tabs = c->at<RowTable>(c->L.tab_van);
+  for (int r = 0; r < c->m.R; ++r)
+    if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr))) return e;
+  if ((e = launch_lm_head(c, tabs + c->m.R - 1, c->ng_dec))) return e;
+  if ((e = launch_select(c, tabs + c->m.R - 1, 1 << RO_TARGET))) return e;
+  vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 1));
+  return cudaGetLastError();
+}
+
+int check_device_error(loopspec_ctx* c) {
+  int e = c->host_flags[HF_ERROR];
+  if (!e) return LOOPSPEC_OK;
+  c->host_flags[HF_ERROR] = 0;
+  return fail(c, LOOPSPEC_ECAPACITY, "device scheduler reported %s",
+              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : "speculative chain too deep");
+}
+
+int capture(loopspec_ctx* c, cudaGraphExec_t* out, bool vanilla) {
+  cudaGraph_t g = nullptr;
+  CU(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+  cudaError_t e;
+  if (vanilla) e = launch_vanilla_token(c);
+  else {
+    int n = 0;
+    e = launch_step(c, 0x1e, PH_ADVANCE | PH_VERIFY | PH_BUILD, true, &n);
+    c->launches_per_step = n;
+  }
+  cudaError_t e2 = cudaStreamEndCapture(c->stream, &g);
+  if (e != cudaSuccess || e2 != cudaSuccess) {
+    if (g) cudaGraphDestroy(g);
+    return fail(c, LOOPSPEC_ECUDA, "graph capture failed: %s", cudaGetErrorString(e != cudaSuccess ? e : e2));
+  }
+  e = cudaGraphInstantiate(out, g, 0);
+  cudaGraphDestroy(g);
+  if (e != cudaSuccess) return fail(c, LOOPSPEC_ECUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e));
+  return LOOPSPEC_OK;
+}
+
+bool any_prefilled(loopspec_ctx* c) {
+  for (char p : c->prefilled)
+    if (p) return true;
+  return false;
+}
+
+}  // namespace
+
+// =============================================== C ABI =================================================
+extern "C" {
+
+size_t loopspec_workspace_bytes(const loopspec_model* m, const loopspec_sched* s) {
+  int why;
+  Derived d;
+  if (!validate_model(m, &why) || !resolve_sched(m, s, &d, &why)) return 0;
+  int n_sm = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n_sm = v;
+  }
+  (void)cudaGetLastError();
+  return make_layout(m, s, d, n_sm).total;
+}
+
+int loopspec_pick_depths(float alpha, float beta, int32_t R, double* d1_star, double* d2_star, int32_t* d1, int32_t* d2) {
+  if (!(alpha > 0) || !(beta > 0) || R < 2) return LOOPSPEC_EINVAL;
+  double a, b;
+  closed_form(alpha, beta, R, &a, &b);
+  if (d1_star) *d1_star = a;
+  if (d2_star) *d2_star = b;
+  int x = 1, y = 0;
+  if (!snap_depths(alpha, beta, R, &x, &y)) x = 1, y = 0;
+  if (d1) *d1 = x;
+  if (d2) *d2 = y;
+  return LOOPSPEC_OK;
+}
+
+int32_t loopspec_max_branches(int32_t R, int32_t d1, int32_t d2) {
+  if (d1 < 1 || R < 2 || d1 >= R || R % d1 || (d2 && (d2 <= d1 || d2 >= R || d2 % d1))) return 0;
+  return max_branches(R, d1, d2);
+}
+
+int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopspec_weights* w, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream, loopspec_ctx** out) {
+  if (!out) return LOOPSPEC_EINVAL;
+  *out = nullptr;
+  int why;
+  Derived d;
+  if (!validate_model(m, &why)) return why;
+  if (!resolve_sched(m, s, &d, &why)) return why;
+  if (!w || !w->embed || !w->final_norm || !w->layer_ptrs || (!m->tied_lm_head && !w->lm_head) || w->adapter) return LOOPSPEC_EINVAL;
+  for (int i = 0; i < 6 * m->n_recurrent; ++i)
+    if (!w->layer_ptrs[i]) return LOOPSPEC_EINVAL;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LOOPSPEC_EINVAL;
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return LOOPSPEC_ECUDA;
+  Layout L = make_layout(m, s, d, n_sm);
+  if (workspace_bytes < L.total) return LOOPSPEC_ECAPACITY;
+
+  loopspec_ctx* c = new loopspec_ctx();
+  c->m = *m, c->s = *s, c->d = d, c->L = L, c->n_sm = n_sm;
+  c->s.d1 = d.d1, c->s.d2 = d.d2;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->ws = static_cast<unsigned char*>(workspace);
+  c->embed = w->embed, c->lm_head = m->tied_lm_head ? w->embed : w->lm_head;
+  c->final_norm = static_cast<const float*>(w->final_norm);
+  c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * m->n_recurrent);
+  c->ng_dec = ng_for_rows(d.max_rows_dec), c->ng_pf = ng_for_rows(d.max_rows_pf);
+  c->prefilled.assign(d.S, 0);
+  int target = n_sm * kCtasPerSm;
+  c->plan[G_QKV] = plan_gemm((d.Hq + 2 * d.Hkv) / 128, m->hidden, target);
+  c->plan[G_O] = plan_gemm(m->hidden / 128, d.Hq, target);
+  c->plan[G_GU] = plan_gemm((m->ffn + 63) / 64, m->hidden, target);
+  c->plan[G_DOWN] = plan_gemm(m->hidden / 128, m->ffn, target);
+  c->plan[G_LM] = plan_gemm((m->vocab + 127) / 128, m->hidden, target);
+
+  for (int ng : {c->ng_dec, c->ng_pf})
+    if (gemm_smem_bytes(ng) > 48 * 1024)
+      for (int epi = 0; epi < 5; ++epi)
+        cudaFuncSetAttribute(gemm_fn(m->weight_dtype, ng, epi), cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(ng));
+  auto bail = [&](int code, const char* what) {
+    loopspec_destroy(c);
+    (void)what;
+    return code;
+  };
+  int* hf = nullptr;
+  if (cudaHostAlloc(reinterpret_cast<void**>(&hf), HF_COUNT * sizeof(int), cudaHostAllocMapped) != cudaSuccess)
+    return bail(LOOPSPEC_ECUDA, "cudaHostAlloc");
+  memset(hf, 0, HF_COUNT * sizeof(int));
+  c->host_flags = hf;
+  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_flags_dev), hf, 0) != cudaSuccess)
+    return bail(LOOPSPEC_ECUDA, "cudaHostGetDevicePointer");
+  c->pin_ids_cap = (size_t)std::max(s->max_ctx, d.S * d.ids_cap) * 8 + 64;
+  if (cudaHostAlloc(reinterpret_cast<void**>(&c->pin_ids), c->pin_ids_cap * sizeof(int), cudaHostAllocDefault) != cudaSuccess)
+    return bail(LOOPSPEC_ECUDA, "cudaHostAlloc");
+  if (cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "event");
+
+  // rotary table in double precision on the host: cos/sin(pos * theta^(-2i/d))
+  {
+    const int hd2 = m->head_dim / 2;
+    std::vector<float2> tab((size_t)s->max_ctx * hd2);
+    for (int i = 0; i < hd2; ++i) {
+      double inv = std::pow((double)m->rope_theta, -2.0 * i / m->head_dim);
+      for (int p = 0; p < s->max_ctx; ++p) {
+        double a = p * inv;
+        tab[(size_t)p * hd2 + i] = make_float2((float)std::cos(a), (float)std::sin(a));
+      }
+    }
+    if (cudaMemcpyAsync(c->ws + L.rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+      return bail(LOOPSPEC_ECUDA, "rope upload");
+  }
+  // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
+  if (cudaMemsetAsync(c->ws + L.gcnt, 0, L.apart - L.gcnt, c->stream) != cudaSuccess ||
+      cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
+      cudaMemsetAsync(c->ws + L.seqs, 0xff, (size_t)MAX_ROWS * 4, c->stream) != cudaSuccess ||  // root = -1
+      cudaStreamSynchronize(c->stream) != cudaSuccess)
+    return bail(LOOPSPEC_ECUDA, "workspace clear");
+  *out = c;
+  return LOOPSPEC_OK;
+}
+
+int loopspec_destroy(loopspec_ctx* c) {
+  if (!c) return LOOPSPEC_OK;
+  if (c->g_step) cudaGraphExecDestroy(c->g_step);
+  if (c->g_vanilla) cudaGraphExecDestroy(c->g_vanilla);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+  if (c->host_flags) cudaFreeHost(const_cast<int*>(c->host_flags));
+  if (c->pin_ids) cudaFreeHost(c->pin_ids);
+  delete c;
+  return LOOPSPEC_OK;
+}
+
+const char* loopspec_last_error(loopspec_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* first_token) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (seq < 0 || seq >= c->d.S || !prompt_ids || n < 1) return fail(c, LOOPSPEC_EINVAL, "bad prefill arguments");
+  if (n + 3 >= c->s.max_ctx) return fail(c, LOOPSPEC_ECAPACITY, "prompt of %d tokens does not fit max_ctx %d", n, c->s.max_ctx);
+  for (int i = 0; i < n; ++i)
+    if (prompt_ids[i] < 0 || prompt_ids[i] >= c->m.vocab) return fail(c, LOOPSPEC_EINVAL, "prompt id out of range");
+  if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
+  memcpy(c->pin_ids, prompt_ids, (size_t)n * 4);
+  CU(c, cudaMemcpyAsync(c->ws + c->L.prompt, c->pin_ids, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
+  RowTable* tab = c->at<RowTable>(c->L.tab_pf);
+  const int chunk = c->d.max_rows_pf;
+  for (int p0 = 0; p0 < n; p0 += chunk) {
+    int cnt = std::min(chunk, n - p0);
+    for (int r = 1; r <= c->m.R; ++r) {
+      PrefillParams pp;
+      pp.tab = tab, pp.prompt = c->at<int>(c->L.prompt), pp.seq = seq, pp.p0 = p0, pp.count = cnt, pp.r = r, pp.R = c->m.R;
+      pp.n_prompt = n, pp.hid_base = c->d.S * c->d.NB, pp.p_logit_base = c->d.p_logit_base;
+      pp.hid = c->at<float>(c->L.hid), pp.H = c->m.hidden, pp.embed = c->embed, pp.weight_dtype = c->m.weight_dtype;
+      prefill_setup_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(pp);
+      CU(c, cudaGetLastError());
+      CU(c, launch_layers(c, tab, c->ng_pf, nullptr));
+    }
+  }
+  CU(c, launch_lm_head(c, tab, c->ng_pf));
+  CU(c, launch_select(c, tab, 1 << RO_TARGET));
+  PrefillFinishParams fp;
+  fp.tab = tab, fp.nodes = c->nodes(), fp.seqs = c->seqs(), fp.seq = seq, fp.NB = c->d.NB, fp.n_prompt = n, fp.n_target = 0;
+  fp.sel_tok = c->at<int>(c->L.sel_tok), fp.hid = c->at<float>(c->L.hid), fp.H = c->m.hidden, fp.embed = c->embed;
+  fp.weight_dtype = c->m.weight_dtype, fp.host_flags = c->host_flags_dev;
+  prefill_finish_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(fp);
+  CU(c, cudaGetLastError());
+  // statistics and traces restart with the sequence set
+  CU(c, cudaMemsetAsync(c->ws + c->L.ctr, 0, sizeof(Counters), c->stream));
+  CU(c, cudaMemsetAsync(c->ws + c->L.trace_n, 0, 4, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  c->prefilled[seq] = 1;
+  c->vanilla_mode = false;
+  if (first_token) *first_token = c->host_flags[HF_FIRST_TOKEN];
+  return check_device_error(c);
+}
+
+// set every prefilled sequence's target to n more tokens and (re)build the decode rows
+static int arm_decode(loopspec_ctx* c, int n_tokens, bool unlimited = false) {
+  std::vector<int> ndec(MAX_ROWS), tgt(MAX_ROWS, 0);
+  CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (int s = 0; s < c->d.S; ++s) {
+    if (!c->prefilled[s]) continue;
+    if (unlimited) {
+      tgt[s] = c->d.ids_cap;
+      continue;
+    }
+    if ((long long)ndec[s] + n_tokens > c->d.ids_cap) return fail(c, LOOPSPEC_ECAPACITY, "decode would exceed max_ctx");
+    tgt[s] = ndec[s] + n_tokens;
+  }
+  memcpy(c->pin_ids, tgt.data(), MAX_ROWS * 4);
+  CU(c, cudaMemcpyAsync(c->seqs().n_target, c->pin_ids, MAX_ROWS * 4, cudaMemcpyHostToDevice, c->stream));
+  if (c->vanilla_mode) {  // drop back from vanilla decoding: the root restarts at depth 0
+    vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 0));
+    CU(c, cudaGetLastError());
+    c->vanilla_mode = false;
+  }
+  CU(c, launch_control(c, PH_BUILD));
+  CU(c, cudaStreamSynchronize(c->stream));
+  return check_device_error(c);
+}
+
+int loopspec_step(loopspec_ctx* c, int32_t* n_rows_out, int32_t* n_need_verify_out) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "step before prefill");
+  if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending: call loopspec_verify first");
+  // a manual step never stops on a token target; (re)building the rows is idempotent
+  int rc = arm_decode(c, 0, true);
+  if (rc) return rc;
+  int rows = c->host_flags[HF_N_ROWS];
+  CU(c, launch_step(c, (1 << RO_D1) | (1 << RO_D2), PH_ADVANCE | PH_BUILD, false, nullptr));
+  CU(c, cudaStreamSynchronize(c->stream));
+  int need = c->host_flags[HF_NEED_VERIFY];
+  c->pending_verify = need > 0;
+  if (n_rows_out) *n_rows_out = rows;
+  if (n_need_verify_out) *n_need_verify_out = need;
+  return check_device_error(c);
+}
+
+int loopspec_verify(loopspec_ctx* c, loopspec_commit* out, int32_t max_out, int32_t* n_out) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (!c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "no branch is at depth R");
+  if (max_out < 0 || (max_out > 0 && !out)) return fail(c, LOOPSPEC_EINVAL, "bad output array");
+  std::vector<int> before(MAX_ROWS), after(MAX_ROWS);
+  CU(c, cudaMemcpyAsync(before.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, launch_select(c, c->at<RowTable>(c->L.tab_dec), 1 << RO_VERIFY));
+  CU(c, launch_control(c, PH_VERIFY | PH_BUILD));
+  CU(c, launch_kv_commit(c));
+  CU(c, cudaMemcpyAsync(after.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  c->pending_verify = false;
+  int n = 0;
+  for (int s = 0; s < c->d.S; ++s) {
+    if (after[s] == before[s]) continue;
+    if (n < max_out) {
+      int rec[8];
+      CU(c, cudaMemcpy(rec, c->at<int>(c->L.commits) + ((size_t)s * c->d.ids_cap + before[s]) * 8, sizeof rec, cudaMemcpyDeviceToHost));
+      out[n] = loopspec_commit{rec[0], rec[1], rec[2], rec[3], rec[4], rec[5], rec[6], rec[7]};
+    }
+    ++n;
+  }
+  if (n_out) *n_out = n;
+  return check_device_error(c);
+}
+
+static int copy_ids_out(loopspec_ctx* c, const std::vector<int>& start, int n_tokens, int32_t* ids_out) {
+  if (!ids_out) return LOOPSPEC_OK;
+  for (int s = 0; s < c->d.S; ++s) {
+    if (!c->prefilled[s]) continue;
+    CU(c, cudaMemcpyAsync(c->pin_ids + (size_t)s * n_tokens, c->at<int>(c->L.out_ids) + (size_t)s * c->d.ids_cap + start[s],
+                          (size_t)n_tokens * 4, cudaMemcpyDeviceToHost, c->stream));
+  }
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (int s = 0; s < c->d.S; ++s)
+    if (c->prefilled[s]) memcpy(ids_out + (size_t)s * n_tokens, c->pin_ids + (size_t)s * n_tokens, (size_t)n_tokens * 4);
+  return LOOPSPEC_OK;
+}
+
+int loopspec_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
+  if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "decode before prefill");
+  if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
+  std::vector<int> start(MAX_ROWS);
+  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  int rc = arm_decode(c, n_tokens);
+  if (rc) return rc;
+  if (!c->g_step && (rc = capture(c, &c->g_step, false))) return rc;
+  // every commit needs at least d1 more passes, so `remaining * d1` replays can never overshoot
+  std::vector<int> ndec(MAX_ROWS);
+  for (;;) {
+    CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaStreamSynchronize(c->stream));
+    if ((rc = check_device_error(c))) return rc;
+    int remaining = 0;
+    for (int s = 0; s < c->d.S; ++s)
+      if (c->prefilled[s]) remaining = std::max(remaining, start[s] + n_tokens - ndec[s]);
+    if (remaining <= 0) break;
+    for (int i = 0; i < remaining * c->d.d1; ++i) CU(c, cudaGraphLaunch(c->g_step, c->stream));
+  }
+  return copy_ids_out(c, start, n_tokens, ids_out);
+}
+
+int loopspec_vanilla_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
+  if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "decode before prefill");
+  if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
+  std::vector<int> start(MAX_ROWS);
+  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (int s = 0; s < c->d.S; ++s)
+    if (c->prefilled[s] && (long long)start[s] + n_tokens > c->d.ids_cap) return fail(c, LOOPSPEC_ECAPACITY, "decode would exceed max_ctx");
+  vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 0));
+  CU(c, cudaGetLastError());
+  c->vanilla_mode = true;
+  int rc;
+  if (!c->g_vanilla && (rc = capture(c, &c->g_vanilla, true))) return rc;
+  for (int i = 0; i < n_tokens; ++i) CU(c, cudaGraphLaunch(c->g_vanilla, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  if ((rc = check_device_error(c))) return rc;
+  return copy_ids_out(c, start, n_tokens, ids_out);
+}
+
+int loopspec_get_stats(loopspec_ctx* c, loopspec_stats* out) {
+  if (!c || !out) return LOOPSPEC_EINVAL;
+  Counters k;
+  CU(c, cudaMemcpyAsync(&k, c->ws + c->L.ctr, sizeof k, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  out->steps = k.steps, out->n_decode = k.n_decode, out->n_accept1 = k.n_accept1, out->n_accept2 = k.n_accept2;
+  out->n_restart = k.n_restart, out->gate_evals = k.gate_evals, out->gate_opens = k.gate_opens;
+  out->rows_total = k.rows_total, out->rows_max = k.rows_max, out->readout_rows_total = k.readout_rows_total;
+  double den = (double)k.n_accept1 * c->d.d1 + (double)k.n_accept2 * c->d.d2 + (double)k.n_restart * c->m.R;
+  out->gamma = den > 0 ? (double)k.n_decode * c->m.R / den : 0.0;  // Sec. 5, definition of gamma
+  return LOOPSPEC_OK;
+}
+
+int loopspec_get_commits(loopspec_ctx* c, int32_t seq, loopspec_commit* out, int32_t max_out, int32_t* n_out) {
+  if (!c || seq < 0 || seq >= c->d.S || max_out < 0 || (max_out && !out)) return LOOPSPEC_EINVAL;
+  int n = 0;
+  CU(c, cudaMemcpyAsync(&n, c->seqs().n_dec + seq, 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  int k = std::min(n, (int)max_out);
+  if (k > 0) {
+    std::vector<int> rec((size_t)k * 8);
+    CU(c, cudaMemcpy(rec.data(), c->at<int>(c->L.commits) + (size_t)seq * c->d.ids_cap * 8, rec.size() * 4, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < k; ++i) {
+      const int* r = &rec[(size_t)i * 8];
+      out[i] = loopspec_commit{r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7]};
+    }
+  }
+  if (n_out) *n_out = n;
+  return LOOPSPEC_OK;
+}
+
+int loopspec_get_row_trace(loopspec_ctx* c, int32_t* out, int32_t max_out, int32_t* n_out) {
+  if (!c || max_out < 0 || (max_out && !out)) return LOOPSPEC_EINVAL;
+  int n = 0;
+  CU(c, cudaMemcpyAsync(&n, c->ws + c->L.trace_n, 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  int k = std::min(std::min(n, c->d.trace_cap), (int)max_out);
+  if (k > 0) CU(c, cudaMemcpy(out, c->ws + c->L.trace, (size_t)k * 4, cudaMemcpyDeviceToHost));
+  if (n_out) *n_out = n;
+  return LOOPSPEC_OK;
+}
+
+int loopspec_debug_logits(loopspec_ctx* c, int32_t seq, int32_t which, float* out_V) {
+  if (!c || !out_V || seq < 0 || seq >= c->d.S || which < 0 || which > 2) return LOOPSPEC_EINVAL;
+  size_t idx;
+  if (which == 0) idx = c->d.p_logit_base + seq;
+  else {
+    int root = -1;
+    CU(c, cudaMemcpy(&root, c->seqs().root + seq, 4, cudaMemcpyDeviceToHost));
+    if (root < 0) return fail(c, LOOPSPEC_ESTATE, "sequence has no root branch");
+    idx = (size_t)(seq * c->d.NB + root) * 2 + (which - 1);
+  }
+  CU(c, cudaStreamSynchronize(c->stream));
+  CU(c, cudaMemcpy(out_V, c->at<float>(c->L.logits) + idx * c->m.vocab, (size_t)c->m.vocab * 4, cudaMemcpyDeviceToHost));
+  return LOOPSPEC_OK;
+}
+
+int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
+  if (!c || !out) return LOOPSPEC_EINVAL;
+  *out = c->m.n_recurrent * 5 + 4;
+  return LOOPSPEC_OK;
+}
+
+int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_out, double* bytes_out) {
+  if (!c || which < 0 || which > 4 || rows < 1 || rows > 8 * c->ng_dec || iters < 1 || !ms_out) return LOOPSPEC_EINVAL;
+  if (c->sticky) return LOOPSPEC_ECUDA;
+  if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
+  // a scratch row table with `rows` plain rows on sequence 0 (hidden states of the prefill area; outputs go to
+  // the pass buffers and to KV slot 0 of plane 1, which the next prefill overwrites)
+  RowTable t;
+  memset(&t, 0, sizeof t);
+  t.n_rows = rows, t.n_readout = rows;
+  for (int i = 0; i < rows; ++i) {
+    t.r[i] = 1, t.hid_idx[i] = c->d.S * c->d.NB + i, t.ro_rows[i] = i, t.readout[i] = RO_TARGET, t.n_canon[i] = 1;
+    t.logit_idx[i] = c->d.p_logit_base, t.node[i] = -1, t.chunk_start[i] = i;
+  }
+  t.chunk_start[rows] = rows, t.attn_items = rows;
+  CU(c, cudaMemcpyAsync(c->ws + c->L.tab_pf, &t, sizeof t, cudaMemcpyHostToDevice, c->stream));
+  CU(c, cudaMemsetAsync(c->ws + c->L.hid + (size_t)c->d.S * c->d.NB * c->m.hidden * 4, 0, (size_t)rows * c->m.hidden * 4, c->stream));
+  const RowTable* tab = c->at<RowTable>(c->L.tab_pf);
+  const int L = c->m.n_recurrent;
+  auto run = [&](int n) -> cudaError_t {
+    for (int i = 0; i < n; ++i) {
+      GemmParams p = gemm_params(c, which, i % L, tab);
+      if (which == G_QKV) p.n_sq = 0;
+      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->plan[which].grid, c->stream);
+      if (e) return e;
+    }
+    return cudaSuccess;
+  };
+  CU(c, run(std::min(iters, 8)));
+  CU(c, cudaEventRecord(c->ev0, c->stream));
+  CU(c, run(iters));
+  CU(c, cudaEventRecord(c->ev1, c->stream));
+  CU(c, cudaEventSynchronize(c->ev1));
+  float ms = 0;
+  CU(c, cudaEventElapsedTime(&ms, c->ev0, c->ev1));
+  *ms_out = ms / iters;
+  const size_t wb = c->m.weight_dtype ? 2 : 4;
+  const Derived& d = c->d;
+  double nk[5] = {(double)(d.Hq + 2 * d.Hkv) * c->m.hidden, (double)c->m.hidden * d.Hq, 2.0 * c->m.ffn * c->m.hidden,
+                  (double)c->m.hidden * c->m.ffn, (double)c->m.vocab * c->m.hidden};
+  if (bytes_out) *bytes_out = nk[which] * wb;
+  // the timed launches touched sequence state only through scratch; mark sequences as needing a new prefill
+  std::fill(c->prefilled.begin(), c->prefilled.end(), 0);
+  return LOOPSPEC_OK;
+}
+
+size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K) {
+  if (M < 1 || M > 64 || N < 16 || K < 8 || N % 16 || K % 8) return 0;
+  int n_rb = (N + 127) / 128;
+  GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
+  return align_up((size_t)n_rb * 4) + (size_t)n_rb * g.max_contrib * 8 * ng_for_rows(M) * 128 * 4;
+}
+
+int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N, int32_t K,
+                       void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!W || !x || !y || (weight_dtype != 0 && weight_dtype != 1)) return LOOPSPEC_EINVAL;
+  size_t need = loopspec_linear_scratch_bytes(M, N, K);
+  if (!need) return LOOPSPEC_EINVAL;
+  if (!scratch || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) & 15)) return LOOPSPEC_ECAPACITY;
+  int n_rb = (N + 127) / 128;
+  GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
+  GemmParams p;
+  memset(&p, 0, sizeof p);
+  p.W = W, p.N = N, p.K = K, p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.units_per_cta = g.upc, p.total_units = g.total;
+  p.xs_kind = XS_BUF, p.xbuf = x, p.x_ld = K, p.m_fixed = M, p.max_contrib = g.max_contrib;
+  p.counters = static_cast<int*>(scratch);
+  p.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + align_up((size_t)n_rb * 4));
+  p.out = y, p.out_ld = N;
+  cudaError_t e = launch_gemm(weight_dtype, ng_for_rows(M), EPI_PLAIN, p, g.grid, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,217 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same seeded inputs.
+
+Bar: token ids, accept/reject decisions, commit sources, gate bits, commit steps, per-step row counts and the
+App. C/D counters bit-exact; logits within max-abs 3e-2 + 2e-2 relative (the stated bf16 bound) -- and, because
+the kernels keep activations fp32-faithful, within 2e-3 absolute in practice, which is also asserted.
+"""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+# ---- the weight-streaming GEMM against its definition -----------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("M,N,K", [(1, 128, 256), (4, 768, 256), (7, 1408, 256), (8, 256, 704), (5, 2000, 768),
+                                   (3, 2048, 2048), (8, 4000, 768), (16, 768, 768), (29, 512, 2000), (64, 256, 256),
+                                   (2, 11264, 2048), (6, 2048, 5632), (4, 256, 688)])
+def test_linear_matches_definition(dtype, M, N, K):
+    import paper_2609_17184_b200 as ls
+    rng = np.random.default_rng(N * 7 + K + M)
+    Wn = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    if dtype == "bf16":
+        Wn = W.bf16_round(Wn)
+    x = rng.standard_normal((M, K)).astype(np.float32) * rng.uniform(0.1, 3.0, (M, 1)).astype(np.float32)
+    Wt = torch.from_numpy(Wn).cuda().to(torch.bfloat16 if dtype == "bf16" else torch.float32)
+    xt = torch.from_numpy(x).cuda()
+    y = ls.linear(Wt, xt).cpu().numpy()
+    ref = x.astype(np.float64) @ Wn.astype(np.float64).T
+    scale = np.abs(x).astype(np.float64) @ np.abs(Wn).astype(np.float64).T
+    assert (np.abs(y - ref) <= 2e-6 * scale + 1e-30).all(), np.abs(y - ref).max()
+    # batch invariance: a row's bits do not depend on which other rows share the call
+    y1 = ls.linear(Wt, xt[:1].contiguous()).cpu().numpy()
+    assert np.array_equal(y1[0].view(np.uint32), y[0].view(np.uint32))
+    # reproducible bit for bit
+    assert np.array_equal(ls.linear(Wt, xt).cpu().numpy().view(np.uint32), y.view(np.uint32))
+
+
+# ---- end-to-end parity -------------------------------------------------------------------------------
+GREEDY_CASES = [
+    ("tiny", 16, 64, 1, 0, True),            # BASELINE config 0 as given
+    ("tiny", 16, 40, 1, 2, True),
+    ("tiny", 9, 30, 2, 0, True),
+    ("tiny_bf16", 16, 64, 1, 2, True),
+    ("tiny_bf16", 16, 48, 1, 3, True),
+    ("tiny_bf16", 16, 48, 1, 2, False),      # gate forced open: 7 rows
+    ("tiny_bf16", 5, 40, 2, 0, True),
+    ("small_bf16", 70, 48, 1, 2, True),      # context spans two attention chunks, ragged GEMM tails
+    ("small_bf16", 130, 24, 1, 0, True),
+]
+
+
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,gate", GREEDY_CASES)
+def test_greedy_decode_matches_oracle(name, n_prompt, n_decode, d1, d2, gate):
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, gate=gate)
+    ctx = U.make_ctx(name, d1, d2, gate=gate, max_ctx=n_prompt + n_decode + 8)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    np.testing.assert_allclose(ctx.debug_logits(0, 0), ref["dec"].first_logits, atol=2e-3, rtol=0)
+    out = ctx.decode(n_decode)
+    assert out[0].tolist() == ref["tokens"], (U.first_diff(out[0].tolist(), ref["tokens"]), U.min_margin(ref["dec"]))
+    err = U.assert_same_run(ctx, ref, n_decode)
+    assert err < 2e-3
+    st, so = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_decode", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total",
+              "rows_max", "readout_rows_total"):
+        assert st[k] == so[k], (k, st[k], so[k])
+    assert abs(st["gamma"] - so["gamma"]) < 1e-12
+    assert ctx.row_trace().tolist() == ref["dec"].rows_per_step
+    ctx.close()
+
+
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2", [("tiny", 16, 64, 1, 0), ("tiny_bf16", 16, 64, 1, 2),
+                                                           ("small_bf16", 70, 40, 1, 2)])
+def test_greedy_loopspec_equals_vanilla_on_gpu(name, n_prompt, n_decode, d1, d2):
+    """Losslessness on the device: same tokens from the pipelined path and from all-R decoding (same kernels)."""
+    prompt = W.make_prompt(W.CONFIGS[name].vocab, n_prompt)
+    a = U.make_ctx(name, d1, d2, max_ctx=n_prompt + 2 * n_decode + 8)
+    fa = a.prefill(prompt)
+    van = a.vanilla_decode(n_decode)[0].tolist()
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, vanilla=True)
+    assert fa == ref["first"] and van == ref["tokens"]
+    np.testing.assert_allclose(a.debug_logits(0, 0), ref["dec"].verify_logits[-1], atol=2e-3, rtol=0)
+    # continue with the pipelined path from the vanilla state, and compare with a fresh pipelined run
+    cont = a.decode(n_decode)[0].tolist()
+    b = U.make_ctx(name, d1, d2, max_ctx=n_prompt + 2 * n_decode + 8)
+    b.prefill(prompt)
+    both = b.decode(2 * n_decode)[0].tolist()
+    assert both[:n_decode] == van and both[n_decode:] == cont
+    a.close(), b.close()
+
+
+SAMPLED_CASES = [
+    ("tiny_bf16", 16, 64, 1, 2, 1.0, True, True),
+    ("tiny_bf16", 16, 64, 1, 2, 0.7, True, True),
+    ("tiny_bf16", 16, 48, 1, 3, 1.0, True, True),
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, False, True),     # ungated
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, True, False),     # non-residual second proposal
+    ("tiny", 16, 48, 1, 2, 1.0, True, True),
+    ("tiny", 16, 48, 2, 0, 1.3, True, True),
+    ("small_bf16", 70, 40, 1, 2, 1.0, True, True),
+]
+
+
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,gate,residual", SAMPLED_CASES)
+def test_sampled_decode_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate, residual):
+    """Rejection-sampling verification: same draws, same accept/reject decisions, same resampled tokens."""
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=2, gate=gate, residual_q2=residual)
+    ctx = U.make_ctx(name, d1, d2, T=T, seed=2, gate=gate, residual_q2=residual, max_ctx=n_prompt + n_decode + 8)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(n_decode)
+    U.assert_same_run(ctx, ref, n_decode)
+    st, so = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
+        assert st[k] == so[k], (k, st[k], so[k])
+    srcs = {c["source"] for c in ref["dec"].commits}
+    assert len(srcs) >= 2          # the case exercises acceptance and rejection
+    ctx.close()
+
+
+def test_sampled_vanilla_matches_oracle():
+    ref = U.oracle_run("tiny_bf16", 16, 40, 1, 0, T=1.0, seed=5, vanilla=True)
+    ctx = U.make_ctx("tiny_bf16", 1, 0, T=1.0, seed=5, max_ctx=80)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    assert ctx.vanilla_decode(40)[0].tolist() == ref["tokens"]
+    ctx.close()
+
+
+def test_step_verify_calls_equal_decode():
+    """loopspec_decode produces exactly the tokens of alternating loopspec_step / loopspec_verify."""
+    name, n_prompt, n = "tiny_bf16", 16, 32
+    ref = U.oracle_run(name, n_prompt, n, 1, 2, T=1.0, seed=2)
+    ctx = U.make_ctx(name, 1, 2, T=1.0, seed=2, max_ctx=80)
+    ctx.prefill(ref["prompt"])
+    toks, rows, commits = [], [], []
+    while len(toks) < n:
+        n_rows, need = ctx.step()
+        rows.append(n_rows)
+        if need:
+            for c in ctx.verify():
+                toks.append(c["token"])
+                commits.append(c)
+    assert toks == ref["tokens"]
+    assert rows == ref["dec"].rows_per_step[: len(rows)]
+    for g, o in zip(commits, ref["dec"].commits):
+        assert tuple(g[k] for k in U.COMMIT_KEYS) == tuple(o[k] for k in U.COMMIT_KEYS)
+    with pytest.raises(Exception) as e:
+        ctx.verify()
+    assert "ESTATE" in str(e.value)
+    ctx.close()
+
+
+def test_batch_of_sequences_equals_each_alone():
+    """Independent sequences share the passes; each must decode exactly as it does alone (and as the oracle)."""
+    name, n_prompt, n = "tiny_bf16", 12, 32
+    S = 3
+    refs = [U.oracle_run(name, n_prompt + 3 * s, n, 1, 2, T=0.9, seed=7, seq=s) for s in range(S)]
+    ctx = U.make_ctx(name, 1, 2, T=0.9, seed=7, max_seqs=S, max_ctx=96)
+    for s in range(S):
+        assert ctx.prefill(refs[s]["prompt"], seq=s) == refs[s]["first"]
+    out = ctx.decode(n)
+    for s in range(S):
+        assert out[s].tolist() == refs[s]["tokens"], s
+        got = ctx.commits(s)
+        assert [c["source"] for c in got] == [c["source"] for c in refs[s]["dec"].commits]
+    ctx.close()
+
+
+def test_prefill_chunking_does_not_change_results():
+    name = "tiny_bf16"
+    ref = U.oracle_run(name, 37, 16, 1, 2)
+    outs = []
+    for rows in (5, 8, 32, 64):
+        ctx = U.make_ctx(name, 1, 2, max_ctx=80, max_prefill_rows=rows)
+        assert ctx.prefill(ref["prompt"]) == ref["first"]
+        outs.append(ctx.debug_logits(0, 0).copy())
+        assert ctx.decode(16)[0].tolist() == ref["tokens"]
+        ctx.close()
+    for o in outs[1:]:
+        assert np.array_equal(o.view(np.uint32), outs[0].view(np.uint32))   # bit-identical across chunkings
+
+
+def test_norm_gains_are_applied():
+    ref = U.oracle_run("tiny_bf16", 16, 24, 1, 2, wseed=3, gain_jitter=0.2)
+    ctx = U.make_ctx("tiny_bf16", 1, 2, max_ctx=64, wseed=3, gain_jitter=0.2)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    assert ctx.decode(24)[0].tolist() == ref["tokens"]
+    U.assert_same_run(ctx, ref, 24)
+    ctx.close()
+
+
+def test_error_paths_leave_the_context_usable():
+    import paper_2609_17184_b200 as ls
+    ctx = U.make_ctx("tiny_bf16", 1, 2, max_ctx=64)
+    for call in (ctx.step, lambda: ctx.decode(4), lambda: ctx.vanilla_decode(4)):
+        with pytest.raises(ls.LoopSpecError) as e:
+            call()
+        assert e.value.status == "ESTATE"
+    with pytest.raises(ls.LoopSpecError) as e:
+        ctx.prefill(np.arange(100) % 512)
+    assert e.value.status == "ECAPACITY"
+    with pytest.raises(ls.LoopSpecError) as e:
+        ctx.prefill([1, 2, 9999])
+    assert e.value.status == "EINVAL"
+    prompt = W.make_prompt(512, 16)
+    ctx.prefill(prompt)
+    with pytest.raises(ls.LoopSpecError) as e:
+        ctx.decode(1000)
+    assert e.value.status == "ECAPACITY"
+    ref = U.oracle_run("tiny_bf16", 16, 8, 1, 2)
+    assert ctx.decode(8)[0].tolist() == ref["tokens"]
+    with pytest.raises(ls.LoopSpecError) as e:
+        U.make_ctx("tiny_bf16", 3, 0)
+    assert e.value.status == "EINVAL"
+    ctx.close()
