@@ -97,7 +97,8 @@ typedef struct {
 size_t loopspec_workspace_bytes(const loopspec_model*, const loopspec_sched*);
 
 /* Create a context.  workspace: device memory, 256-byte aligned, at least loopspec_workspace_bytes large.
- * cuda_stream: a cudaStream_t (may be NULL for the legacy stream is NOT allowed: pass a real stream).
+ * cuda_stream: a cudaStream_t created by the caller; NULL (the legacy default stream) is rejected with EINVAL
+ * because the decode step is captured into a CUDA graph on it.
  * Host structs are copied.  Synchronous; uploads the rotary table and clears the workspace tables. */
 int loopspec_init(const loopspec_model*, const loopspec_sched*, const loopspec_weights*, void* workspace,
                   size_t workspace_bytes, void* cuda_stream, loopspec_ctx** out);
@@ -147,8 +148,7 @@ int loopspec_get_row_trace(loopspec_ctx*, int32_t* out, int32_t max_out, int32_t
  * (or the prefill / vanilla readout), 1 / 2 the root branch's stored first / second proposal readout. */
 int loopspec_debug_logits(loopspec_ctx*, int32_t seq, int32_t which, float* out_V);
 
-/* Algorithmic HBM bytes of one batched pass with the current rows (weights + KV read + lm_head if any
- * branch reads out), and of one vanilla token at the current context.  Host arithmetic only. */
+/* Number of kernels one decode step (one graph replay of loopspec_decode) launches. */
 int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);
 
 /* Time `iters` back-to-back launches of one kernel of the pass in the decode launch configuration, cycling

@@ -150,7 +150,9 @@ class LoopSpec:
         self.shape = shape
         self.h = None
         self.weights = weights  # keep the tensors alive: the library borrows them
-        self.stream = stream or torch.cuda.current_stream()
+        # CUDA graphs cannot be captured on the legacy default stream: the context gets a stream of its own
+        self.stream = stream or torch.cuda.Stream()
+        torch.cuda.synchronize()  # weights were uploaded on other streams
         self.model = Model(shape.vocab, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                            shape.n_prelude, shape.n_recurrent, shape.n_coda, shape.R,
                            1 if shape.weight_dtype == "bf16" else 0, 1 if shape.tied else 0, shape.rms_eps, shape.rope_theta)

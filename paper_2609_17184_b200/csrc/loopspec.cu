@@ -548,6 +548,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   for (int i = 0; i < 6 * m->n_recurrent; ++i)
     if (!w->layer_ptrs[i]) return LOOPSPEC_EINVAL;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LOOPSPEC_EINVAL;
+  if (!cuda_stream) return LOOPSPEC_EINVAL;  // the legacy default stream cannot be captured into a graph
   int dev = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return LOOPSPEC_ECUDA;
