@@ -102,6 +102,23 @@ def vanilla_bytes(shape, n_prompt, n_decode):
     return n_decode * (shape.R * (w_b + kv_row) + w_c)
 
 
+KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
+
+
+def run_kernel_only(args):
+    """Time one kernel of the pass alone (used for profiling captures): prints its own JSON line."""
+    import torch
+    import paper_2609_17184_b200 as ls
+    wl = W.WORKLOADS[args.workload]
+    shape = W.CONFIGS[wl.model]
+    weights = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed))
+    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, max_seqs=1, max_ctx=wl.prompt_len + wl.decode_len + 16)
+    ms, nbytes = ctx.time_kernel(KERNELS.index(args.kernel_only), args.rows, args.iters)
+    print(json.dumps({"kernel": args.kernel_only, "rows": args.rows, "iters": args.iters, "us_per_launch": ms * 1e3,
+                      "GBps": nbytes / (ms / 1e3) / 1e9}))
+    ctx.close()
+
+
 def run_ours(args):
     import torch
     import paper_2609_17184_b200 as ls
@@ -346,7 +363,12 @@ def main():
     ap.add_argument("--decode-len", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--calibrated", action="store_true", help="also run the acceptance-calibrated variant")
+    ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")
+    ap.add_argument("--rows", type=int, default=4)
+    ap.add_argument("--iters", type=int, default=10)
     args = ap.parse_args()
+    if args.kernel_only:
+        return run_kernel_only(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
