@@ -15,7 +15,7 @@ constexpr int ATT_THREADS = 128;
 struct AttnParams {
   const RowTable* tab;
   const float* qbuf;          // [row][n_q_heads * d], rotary applied, unscaled
-  float* abuf;                // [row][n_q_heads * d]
+  __nv_bfloat16* aplanes;     // out: three bf16 planes per row [row][3][n_q_heads * d]
   const __nv_bfloat16* kv;    // this layer's pool [R][2][S][n_kv][slots][d]
   long long kv_plane_stride, kv_sel_stride;
   int slots, n_kv_heads, n_q_heads;
@@ -26,7 +26,7 @@ struct AttnParams {
 };
 
 template <int D, int G>
-__global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant__ AttnParams p) {
   constexpr int LPP = D / 8;            // lanes per key position (8 bf16 = 16 bytes per lane)
   constexpr int PPW = 32 / LPP;         // positions per warp per load
   constexpr int PPR = PPW * (ATT_THREADS / 32);  // positions per round of the whole CTA
@@ -39,9 +39,12 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const AttnParams p) {
   __shared__ int s_slot[ATT_CHUNK];
   __shared__ int s_last;
 
+  pdl_launch_dependents();
+  pdl_wait();
   const RowTable* tab = p.tab;
   const int n_rows = tab->n_rows;
   if (n_rows <= 0) return;
+  const int HQ = p.n_q_heads * D;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int sub = lane / LPP, dl = lane % LPP;  // which position of the warp's group, which 8-dim slice
   const int total = tab->attn_items * p.n_kv_heads;
@@ -173,7 +176,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const AttnParams p) {
         float v = 0.f;
 #pragma unroll
         for (int w2 = 0; w2 < ATT_THREADS / 32; ++w2) v += s_red[w2][gq][dd];
-        p.abuf[(size_t)row * p.n_q_heads * D + (size_t)(kvh * G + gq) * D + dd] = v / s_stat[gq][1];
+        store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, (kvh * G + gq) * D + dd, v / s_stat[gq][1]);
       }
       continue;
     }
@@ -206,7 +209,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const AttnParams p) {
           l = fmaf(__ldcg(pc + D + 1), wgt, l);
           acc = fmaf(__ldcg(pc + dd), wgt, acc);
         }
-        p.abuf[(size_t)row * p.n_q_heads * D + (size_t)(kvh * G + gq) * D + dd] = acc / l;
+        store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, (kvh * G + gq) * D + dd, acc / l);
       }
       if (tid == 0) p.counters[pair] = 0;
     }

@@ -82,6 +82,26 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
+// x = hi + mid + lo with hi, mid, lo bf16 (round-to-nearest at each stage; the remainders are exact in fp32)
+__device__ __forceinline__ void split3(float x, unsigned short& hi, unsigned short& mid, unsigned short& lo) {
+  __nv_bfloat16 h = __float2bfloat16_rn(x);
+  float r1 = x - __bfloat162float(h);
+  __nv_bfloat16 m = __float2bfloat16_rn(r1);
+  float r2 = r1 - __bfloat162float(m);
+  __nv_bfloat16 l = __float2bfloat16_rn(r2);
+  hi = __bfloat16_as_ushort(h);
+  mid = __bfloat16_as_ushort(m);
+  lo = __bfloat16_as_ushort(l);
+}
+// write one value into the three planes of a row: planes + plane * ld
+__device__ __forceinline__ void store_split(__nv_bfloat16* row_planes, int ld, int k, float v) {
+  unsigned short h, m, l;
+  split3(v, h, m, l);
+  row_planes[k] = __ushort_as_bfloat16(h);
+  row_planes[ld + k] = __ushort_as_bfloat16(m);
+  row_planes[2 * ld + k] = __ushort_as_bfloat16(l);
+}
+
 // programmatic dependent launch: wait for the kernels this launch depends on / let dependents start launching
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

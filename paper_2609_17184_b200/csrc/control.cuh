@@ -119,7 +119,7 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
   t.n_rows = n_rows, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
 }
 
-__global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const ControlParams p) {
+__global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_constant__ ControlParams p) {
   __shared__ NodeSmem nd;
   __shared__ RowTable t;
   __shared__ int s_root[MAX_ROWS], s_nids[MAX_ROWS], s_ndec[MAX_ROWS], s_ntarget[MAX_ROWS], s_needv[MAX_ROWS];
@@ -127,6 +127,8 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const ControlPara
   __shared__ int s_nemb, s_err;
   const int tid = threadIdx.x;
   const int n_nodes = p.S * p.NB;
+  pdl_launch_dependents();
+  pdl_wait();
   nodes_load(nd, p.nodes, n_nodes);
   {
     const int* src = reinterpret_cast<const int*>(p.tab);
@@ -262,11 +264,13 @@ struct VanillaParams {
   volatile int* host_flags;
 };
 
-__global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const VanillaParams p) {
+__global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __grid_constant__ VanillaParams p) {
   __shared__ int s_emb[MAX_ROWS][2];
   __shared__ int s_rowof[MAX_ROWS];
   __shared__ int s_n;
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   if (tid == 0) {
     int n = 0;
     const RowTable& cur = p.tabs[p.R - 1];
@@ -389,8 +393,10 @@ struct KvCommitParams {
   int S, L, n_kv_heads, slots, d;
 };
 
-__global__ void kv_commit_kernel(const KvCommitParams p) {
+__global__ void kv_commit_kernel(const __grid_constant__ KvCommitParams p) {
   // grid: (L, R, 2 * S); one CTA copies n_kv_heads rows of d bf16
+  pdl_launch_dependents();
+  pdl_wait();
   const int l = blockIdx.x, plane = blockIdx.y, sel = blockIdx.z & 1, s = blockIdx.z >> 1;
   const KvCopyCmd c = p.cmds[s];
   if (plane >= c.n_planes) return;

@@ -19,7 +19,7 @@ using namespace ls;
 
 namespace {
 
-constexpr int kCtasPerSm = 2;
+constexpr int kCtasPerSm = 1;
 
 struct GemmPlan {
   int n_rb, kpr, upc, total, grid, max_contrib;
@@ -45,7 +45,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t rope, kv, hid, qbuf, abuf, sbuf, sumsq, logits, gpart, gcnt, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, gpart, gcnt, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -155,9 +155,11 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.kv = take((size_t)m->n_recurrent * m->R * 2 * d.S * m->n_kv_heads * d.slots * m->head_dim * 2);
   L.hid = take((size_t)d.n_hid * m->hidden * 4);
   L.qbuf = take(MR * d.Hq * 4);
-  L.abuf = take(MR * d.Hq * 4);
-  L.sbuf = take(MR * m->ffn * 4);
+  L.xplanes = take(MR * 3 * m->hidden * 2);
+  L.aplanes = take(MR * 3 * d.Hq * 2);
+  L.splanes = take(MR * 3 * m->ffn * 2);
   L.sumsq = take(MR * d.n_sq * 4);
+  L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
   // split-k scratch: the largest of the five GEMMs at the widest token-group count in use
   int target = n_sm * kCtasPerSm;
@@ -214,7 +216,7 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true;
   int launches_per_step = 0;
   std::string err;
 
@@ -265,38 +267,51 @@ int fail(loopspec_ctx* c, int code, const char* fmt, ...) {
 // ---- kernel dispatch ---------------------------------------------------------------------------------
 using GemmFn = void (*)(const GemmParams);
 
-template <typename WT, int NG>
-GemmFn gemm_fn_epi(int epi) {
-  switch (epi) {
-    case EPI_PLAIN: return gemm_kernel<WT, NG, EPI_PLAIN>;
-    case EPI_QKV: return gemm_kernel<WT, NG, EPI_QKV>;
-    case EPI_RESID: return gemm_kernel<WT, NG, EPI_RESID>;
-    case EPI_SWIGLU: return gemm_kernel<WT, NG, EPI_SWIGLU>;
-    default: return gemm_kernel<WT, NG, EPI_LOGITS>;
+template <int NG>
+GemmFn gemm_fn_epi(int wdt, int epi) {
+  if (wdt == 1) {
+    switch (epi) {
+      case EPI_PLAIN: return gemm_bf16_kernel<NG, EPI_PLAIN>;
+      case EPI_QKV: return gemm_bf16_kernel<NG, EPI_QKV>;
+      case EPI_RESID: return gemm_bf16_kernel<NG, EPI_RESID>;
+      case EPI_SWIGLU: return gemm_bf16_kernel<NG, EPI_SWIGLU>;
+      default: return gemm_bf16_kernel<NG, EPI_LOGITS>;
+    }
   }
-}
-template <typename WT>
-GemmFn gemm_fn_ng(int ng, int epi) {
-  switch (ng) {
-    case 1: return gemm_fn_epi<WT, 1>(epi);
-    case 2: return gemm_fn_epi<WT, 2>(epi);
-    case 4: return gemm_fn_epi<WT, 4>(epi);
-    default: return gemm_fn_epi<WT, 8>(epi);
+  switch (epi) {
+    case EPI_PLAIN: return gemm_f32_kernel<NG, EPI_PLAIN>;
+    case EPI_QKV: return gemm_f32_kernel<NG, EPI_QKV>;
+    case EPI_RESID: return gemm_f32_kernel<NG, EPI_RESID>;
+    case EPI_SWIGLU: return gemm_f32_kernel<NG, EPI_SWIGLU>;
+    default: return gemm_f32_kernel<NG, EPI_LOGITS>;
   }
 }
 GemmFn gemm_fn(int wdt, int ng, int epi) {
-  return wdt == 1 ? gemm_fn_ng<__nv_bfloat16>(ng, epi) : gemm_fn_ng<float>(ng, epi);
+  switch (ng) {
+    case 1: return gemm_fn_epi<1>(wdt, epi);
+    case 2: return gemm_fn_epi<2>(wdt, epi);
+    case 4: return gemm_fn_epi<4>(wdt, epi);
+    default: return gemm_fn_epi<8>(wdt, epi);
+  }
+}
+int gemm_smem(int wdt, int ng) { return wdt == 1 ? gemm_smem_bytes(ng) : gemm_f32_smem_bytes(ng); }
+
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream is
+// still running; it orders itself with griddepcontrol.wait before touching anything the predecessor writes.
+template <typename P>
+cudaError_t launch_k(void (*fn)(const P), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const P& params, bool pdl) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, fn, params);
 }
 
-cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, int grid, cudaStream_t st) {
-  GemmFn fn = gemm_fn(wdt, ng, epi);
-  int smem = gemm_smem_bytes(ng);
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-  }
-  fn<<<grid, GEMM_THREADS, smem, st>>>(p);
-  return cudaGetLastError();
+cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, int grid, cudaStream_t st, bool pdl = true) {
+  return launch_k(gemm_fn(wdt, ng, epi), dim3(grid), dim3(GEMM_THREADS), (size_t)gemm_smem(wdt, ng), st, p, pdl);
 }
 
 using AttnFn = void (*)(const AttnParams);
@@ -318,11 +333,13 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   p.partials = c->at<float>(c->L.gpart), p.counters = c->at<int>(c->L.gcnt);
   p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
   const void* const* lp = which == G_LM ? nullptr : &c->layers[6 * layer];
+  __nv_bfloat16* xpl = c->at<__nv_bfloat16>(c->L.xplanes);
   switch (which) {
     case G_QKV:
       p.W = lp[1], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
-      p.xs_kind = XS_HID_NORM, p.gain = static_cast<const float*>(lp[0]);
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 0 : d.n_sq;
+      p.xplanes = xpl, p.x_ld = m.hidden;
+      // layer 0 reads the full sums the preparation kernel wrote; later layers the down-projection's partials
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.n_sq;
       p.qbuf = c->at<float>(c->L.qbuf);
       p.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)layer * c->kv_layer_stride();
       p.kv_plane_stride = c->kv_plane_stride(), p.kv_sel_stride = c->kv_sel_stride();
@@ -331,28 +348,41 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       break;
     case G_O:
       p.W = lp[2], p.N = m.hidden, p.K = d.Hq;
-      p.xs_kind = XS_BUF, p.xbuf = c->at<float>(c->L.abuf), p.x_ld = d.Hq;
+      p.xplanes = c->at<__nv_bfloat16>(c->L.aplanes), p.x_ld = d.Hq;
       p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(lp[3]);
       break;
     case G_GU:
       p.W = lp[4], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
-      p.xs_kind = XS_HID_NORM, p.gain = static_cast<const float*>(lp[3]);
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq;
-      p.out = c->at<float>(c->L.sbuf), p.out_ld = m.ffn;
+      p.xplanes = xpl, p.x_ld = m.hidden;
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.n_sq;
+      p.out_planes = c->at<__nv_bfloat16>(c->L.splanes), p.planes_ld = m.ffn;
       break;
     case G_DOWN:
       p.W = lp[5], p.N = m.hidden, p.K = m.ffn;
-      p.xs_kind = XS_BUF, p.xbuf = c->at<float>(c->L.sbuf), p.x_ld = m.ffn;
+      p.xplanes = c->at<__nv_bfloat16>(c->L.splanes), p.x_ld = m.ffn;
       p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      if (layer + 1 < m.n_recurrent) {
+        p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(c->layers[6 * (layer + 1)]);
+      }
       break;
     default:
       p.W = c->lm_head, p.N = m.vocab, p.K = m.hidden;
-      p.xs_kind = XS_HID_NORM_RO, p.gain = c->final_norm;
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq;
+      p.xplanes = xpl, p.x_ld = m.hidden, p.cols_from_readout = 1;
+      p.sumsq = c->at<float>(c->L.sumsq_ro), p.n_sq = 1, p.sq_stride = 1;
       p.logits = c->at<float>(c->L.logits);
       break;
   }
   return p;
+}
+
+cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
+  PrepParams q;
+  memset(&q, 0, sizeof q);
+  q.tab = tab, q.hid = c->at<float>(c->L.hid), q.K = c->m.hidden, q.planes = c->at<__nv_bfloat16>(c->L.xplanes);
+  if (readout) q.gain = c->final_norm, q.sumsq = c->at<float>(c->L.sumsq_ro), q.sq_stride = 1, q.readout_only = 1;
+  else q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.n_sq;
+  return launch_k(prep_planes_kernel, dim3(c->d.max_rows), dim3(256), 0, c->stream, q, c->use_pdl);
 }
 
 const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
@@ -361,28 +391,32 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
+  const bool pdl = c->use_pdl;
   cudaError_t e;
+  if ((e = launch_prep(c, tab, false))) return e;
+  if (n_launch) *n_launch += 1;
   for (int l = 0; l < m.n_recurrent; ++l) {
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->plan[G_QKV].grid, c->stream))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->plan[G_QKV].grid, c->stream, pdl))) return e;
     AttnParams a;
-    a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.abuf = c->at<float>(c->L.abuf);
+    a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
     a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
     a.kv_plane_stride = c->kv_plane_stride(), a.kv_sel_stride = c->kv_sel_stride();
     a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
-    attn_fn(m.head_dim, G)<<<c->n_sm * 4, ATT_THREADS, 0, c->stream>>>(a);
-    if ((e = cudaGetLastError())) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->plan[G_O].grid, c->stream))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->plan[G_GU].grid, c->stream))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->plan[G_DOWN].grid, c->stream))) return e;
+    if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 4), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->plan[G_O].grid, c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->plan[G_GU].grid, c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->plan[G_DOWN].grid, c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
   }
   return cudaSuccess;
 }
 
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
-  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->plan[G_LM].grid, c->stream);
+  cudaError_t e;
+  if ((e = launch_prep(c, tab, true))) return e;
+  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->plan[G_LM].grid, c->stream, c->use_pdl);
 }
 
 cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) {
@@ -392,8 +426,7 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   sp.kinds_mask = kinds_mask;
   sp.sel_tok = c->at<int>(c->L.sel_tok), sp.sel_aux = c->at<int>(c->L.sel_aux);
   sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);
-  select_kernel<<<c->d.max_rows, SEL_THREADS, 0, c->stream>>>(sp);
-  return cudaGetLastError();
+  return launch_k(select_kernel, dim3(c->d.max_rows), dim3(SEL_THREADS), 0, c->stream, sp, c->use_pdl);
 }
 
 ControlParams control_params(loopspec_ctx* c, int phases) {
@@ -413,8 +446,7 @@ ControlParams control_params(loopspec_ctx* c, int phases) {
 }
 
 cudaError_t launch_control(loopspec_ctx* c, int phases) {
-  control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(control_params(c, phases));
-  return cudaGetLastError();
+  return launch_k(control_kernel, dim3(1), dim3(CTRL_THREADS), 0, c->stream, control_params(c, phases), c->use_pdl);
 }
 
 cudaError_t launch_kv_commit(loopspec_ctx* c) {
@@ -423,8 +455,7 @@ cudaError_t launch_kv_commit(loopspec_ctx* c) {
   k.layer_stride = c->kv_layer_stride(), k.plane_stride = c->kv_plane_stride(), k.sel_stride = c->kv_sel_stride();
   k.S = c->d.S, k.L = c->m.n_recurrent, k.n_kv_heads = c->m.n_kv_heads, k.slots = c->d.slots, k.d = c->m.head_dim;
   dim3 grid(c->m.n_recurrent, c->m.R, 2 * c->d.S);
-  kv_commit_kernel<<<grid, 128, 0, c->stream>>>(k);
-  return cudaGetLastError();
+  return launch_k(kv_commit_kernel, grid, dim3(128), 0, c->stream, k, c->use_pdl);
 }
 
 // the whole decode step: pass, readouts, decisions, bookkeeping, KV commit
@@ -435,7 +466,7 @@ cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_com
   if ((e = launch_lm_head(c, tab, c->ng_dec))) return e;
   if ((e = launch_select(c, tab, kinds_mask))) return e;
   if ((e = launch_control(c, phases))) return e;
-  if (n_launch) *n_launch += 3;
+  if (n_launch) *n_launch += 4;
   if (kv_commit) {
     if ((e = launch_kv_commit(c))) return e;
     if (n_launch) *n_launch += 1;
@@ -461,8 +492,7 @@ cudaError_t launch_vanilla_token(loopspec_ctx* c) {
     if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr))) return e;
   if ((e = launch_lm_head(c, tabs + c->m.R - 1, c->ng_dec))) return e;
   if ((e = launch_select(c, tabs + c->m.R - 1, 1 << RO_TARGET))) return e;
-  vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 1));
-  return cudaGetLastError();
+  return launch_k(vanilla_control_kernel, dim3(1), dim3(CTRL_THREADS), 0, c->stream, vanilla_params(c, 1), c->use_pdl);
 }
 
 int check_device_error(loopspec_ctx* c) {
@@ -573,9 +603,14 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->plan[G_LM] = plan_gemm((m->vocab + 127) / 128, m->hidden, target);
 
   for (int ng : {c->ng_dec, c->ng_pf})
-    if (gemm_smem_bytes(ng) > 48 * 1024)
+    if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
-        cudaFuncSetAttribute(gemm_fn(m->weight_dtype, ng, epi), cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(ng));
+        if (cudaFuncSetAttribute(gemm_fn(m->weight_dtype, ng, epi), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 gemm_smem(m->weight_dtype, ng)) != cudaSuccess) {
+          delete c;
+          return LOOPSPEC_ECUDA;
+        }
+  if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
     (void)what;
@@ -865,7 +900,7 @@ int loopspec_debug_logits(loopspec_ctx* c, int32_t seq, int32_t which, float* ou
 
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
-  *out = c->m.n_recurrent * 5 + 4;
+  *out = c->m.n_recurrent * 5 + 6;
   return LOOPSPEC_OK;
 }
 
@@ -890,8 +925,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
-      if (which == G_QKV) p.n_sq = 0;
-      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->plan[which].grid, c->stream);
+      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->plan[which].grid, c->stream, c->use_pdl);
       if (e) return e;
     }
     return cudaSuccess;
@@ -918,7 +952,7 @@ size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K) {
   if (M < 1 || M > 64 || N < 16 || K < 8 || N % 16 || K % 8) return 0;
   int n_rb = (N + 127) / 128;
   GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
-  return align_up((size_t)n_rb * 4) + (size_t)n_rb * g.max_contrib * 8 * ng_for_rows(M) * 128 * 4;
+  return align_up((size_t)n_rb * 4) + align_up((size_t)n_rb * g.max_contrib * 8 * ng_for_rows(M) * 128 * 4) + (size_t)M * 3 * K * 2;
 }
 
 int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N, int32_t K,
@@ -927,16 +961,29 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
   size_t need = loopspec_linear_scratch_bytes(M, N, K);
   if (!need) return LOOPSPEC_EINVAL;
   if (!scratch || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) & 15)) return LOOPSPEC_ECAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int ng = ng_for_rows(M);
   int n_rb = (N + 127) / 128;
   GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
+  unsigned char* sc = static_cast<unsigned char*>(scratch);
+  size_t off_part = align_up((size_t)n_rb * 4);
+  size_t off_planes = off_part + align_up((size_t)n_rb * g.max_contrib * 8 * ng * 128 * 4);
+  PrepParams q;
+  memset(&q, 0, sizeof q);
+  q.m_fixed = M, q.x = x, q.K = K, q.planes = reinterpret_cast<__nv_bfloat16*>(sc + off_planes);
+  if (launch_k(prep_planes_kernel, dim3(M), dim3(256), 0, st, q, false) != cudaSuccess) return LOOPSPEC_ECUDA;
   GemmParams p;
   memset(&p, 0, sizeof p);
   p.W = W, p.N = N, p.K = K, p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.units_per_cta = g.upc, p.total_units = g.total;
-  p.xs_kind = XS_BUF, p.xbuf = x, p.x_ld = K, p.m_fixed = M, p.max_contrib = g.max_contrib;
-  p.counters = static_cast<int*>(scratch);
-  p.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(scratch) + align_up((size_t)n_rb * 4));
+  p.xplanes = q.planes, p.x_ld = K, p.m_fixed = M, p.max_contrib = g.max_contrib;
+  p.counters = reinterpret_cast<int*>(sc);
+  p.partials = reinterpret_cast<float*>(sc + off_part);
   p.out = y, p.out_ld = N;
-  cudaError_t e = launch_gemm(weight_dtype, ng_for_rows(M), EPI_PLAIN, p, g.grid, static_cast<cudaStream_t>(cuda_stream));
+  GemmFn fn = gemm_fn(weight_dtype, ng, EPI_PLAIN);
+  if (gemm_smem(weight_dtype, ng) > 48 * 1024 &&
+      cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem(weight_dtype, ng)) != cudaSuccess)
+    return LOOPSPEC_ECUDA;
+  cudaError_t e = launch_gemm(weight_dtype, ng, EPI_PLAIN, p, g.grid, st, false);
   return e == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
 }
 

@@ -83,9 +83,11 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
   return r;
 }
 
-__global__ void __launch_bounds__(SEL_THREADS) select_kernel(const SelectParams p) {
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_constant__ SelectParams p) {
   __shared__ ArgMax sh_am[SEL_THREADS / 32];
   __shared__ float sh_f[SEL_THREADS / 32];
+  pdl_launch_dependents();
+  pdl_wait();
   const RowTable* tab = p.tab;
   if ((int)blockIdx.x >= tab->n_readout) return;
   const int row = tab->ro_rows[blockIdx.x];
