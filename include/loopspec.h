@@ -93,7 +93,8 @@ typedef struct {
   double gamma;
 } loopspec_stats;
 
-/* Bytes of device workspace loopspec_init needs for this model and scheduler (0 on invalid input). */
+/* Bytes of device workspace loopspec_init needs for this model and scheduler (0 on invalid input).  For bf16
+ * weights this includes a second, tile-major copy of every matrix that the kernels stream from. */
 size_t loopspec_workspace_bytes(const loopspec_model*, const loopspec_sched*);
 
 /* Create a context.  workspace: device memory, 256-byte aligned, at least loopspec_workspace_bytes large.
@@ -160,8 +161,9 @@ int loopspec_time_kernel(loopspec_ctx*, int32_t which, int32_t rows, int32_t ite
 
 /* Stand-alone linear map y[M][N] = x[M][K] * W[N][K]^T through the same weight-streaming kernel (token
  * activations split into three bf16 terms, fp32 accumulation; fp32 weights use the CUDA-core path).
- * All pointers device; x, y fp32; scratch: device, loopspec_linear_scratch_bytes(M, N, K) bytes, zeroed
- * once by the caller before first use (the kernel leaves it zeroed where it must be).  M <= 64. */
+ * All pointers device; x, y fp32; scratch: device, 16-byte aligned, loopspec_linear_scratch_bytes(M, N, K)
+ * bytes (it receives the bf16 planes of x and, for bf16 weights, a tile-major copy of W; contents on entry are
+ * irrelevant).  M <= 64, N % 16 == 0, K % 8 == 0. */
 size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N,
                        int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream);

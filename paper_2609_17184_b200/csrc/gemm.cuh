@@ -8,48 +8,49 @@
 // the split) and 1/rms (by the consumer's epilogue, from the per-row sums of squares) -- both linear.
 //
 // Mapping.  The weights are the 16-row A operand of mma.sync.m16n8k16 (bf16, fp32 accumulate); the token rows
-// are the 8 B columns.  A CTA of 8 warps owns blocks of 128 output rows (one 16-row tile per warp) over a
-// contiguous range of 32-wide k-blocks.  The work (row block x k-block) is linearised and cut into equal
-// shares, one per CTA (stream-K); a row block shared by several CTAs is reduced in fixed order by whichever
-// CTA arrives last, which then runs the epilogue.  No atomics touch data, so results are bit-reproducible.
-// Weight tiles stream through a deep thread-private cp.async ring in shared memory; the first stages are
-// issued before the kernel waits for its predecessor (programmatic dependent launch).
+// are the 8 B columns.  A thread-block cluster owns a block of 128 output rows; its CTAs split K into
+// contiguous ranges (one 16-row tile per warp, 32-wide k-blocks).  Each CTA leaves its partial tile in its
+// own shared memory; after a cluster barrier the CTAs sum the partials over distributed shared memory in rank
+// order -- each CTA finishing a subset of the token columns -- and run the epilogue.  No global scratch, no
+// atomics: results are bit-reproducible.  Weight tiles stream through a deep thread-private cp.async ring
+// whose first stages are issued before the kernel waits for its predecessor (programmatic dependent launch).
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace ls {
+namespace cg = cooperative_groups;
 
 enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4 };
 
 constexpr int GEMM_THREADS = 256;
 constexpr int RB_ROWS = 128;   // output rows per row block
-constexpr int TILE_LD = 132;   // padded leading dimension of the epilogue tile
+constexpr int TILE_LD = 132;   // padded leading dimension of the partial tile
 constexpr int RING = 8;        // weight stages in flight per thread (8 KB per stage per CTA)
+constexpr int MAX_XCH_BLOCKS = 24;  // k-blocks of activations one CTA keeps staged when NG = 1
 
-__host__ __device__ constexpr int xchunk_kblocks(int NG) { return NG >= 4 ? 2 : 8 / NG; }
+__host__ __device__ constexpr int xchunk_kblocks(int NG) { return MAX_XCH_BLOCKS / NG; }
 __host__ __device__ constexpr int xbuf_uint4(int NG) { return 3 * xchunk_kblocks(NG) * 8 * NG * 4; }
 __host__ __device__ constexpr int gemm_smem_bytes(int NG) {
-  return RING * 2 * GEMM_THREADS * 16 + 2 * xbuf_uint4(NG) * 16 + 8 * NG * TILE_LD * 4 + 8 * NG * 4 + 16;
+  return RING * 2 * GEMM_THREADS * 16 + xbuf_uint4(NG) * 16 + 8 * NG * TILE_LD * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
 }
 
 struct GemmParams {
   const void* W;
   int N, K;
-  int n_rb, kb_per_rb, units_per_cta, total_units;
+  int n_rb, kb_per_rb;    // row blocks; 32-wide k-blocks per row
+  int cluster_size, n_clusters;
   // activations: bf16 planes [col][3][x_ld]
   const __nv_bfloat16* xplanes;
   int x_ld;
   const RowTable* tab;
   int m_fixed;            // tab == nullptr: number of rows of a stand-alone call
   int cols_from_readout;  // columns are the reading-out rows (lm_head)
-  // fused RMSNorm: scale row c by 1/sqrt(sum_j sumsq[c*sq_stride + j] / H + eps); sumsq == nullptr: none
+  // fused RMSNorm: scale column c by 1/sqrt(sum_j sumsq[c*sq_stride + j] / H + eps); sumsq == nullptr: none
   const float* sumsq;
   int n_sq, sq_stride, H;
   float eps;
-  // split-k scratch
-  float* partials;        // [n_rb][max_contrib][8*NG][128]
-  int max_contrib;
-  int* counters;          // [n_rb], zero between launches
   // epilogue outputs
   float* out;             // PLAIN y [m][out_ld]
   int out_ld;
@@ -85,149 +86,6 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// ---- epilogue over the finished tile [col][TILE_LD] of row block rb ------------------------------------
-template <int EPI>
-__device__ __forceinline__ void gemm_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, const float* tile,
-                                              const float* s_rstd) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (EPI == EPI_PLAIN || EPI == EPI_LOGITS) {
-    int n0 = rb * RB_ROWS;
-    for (int idx = tid; idx < n_cols * RB_ROWS; idx += GEMM_THREADS) {
-      int c = idx / RB_ROWS, j = idx % RB_ROWS;
-      if (n0 + j < p.N) {
-        float v = tile[c * TILE_LD + j] * s_rstd[c];
-        if (EPI == EPI_PLAIN) p.out[(size_t)c * p.out_ld + n0 + j] = v;
-        else p.logits[(size_t)tab->logit_idx[tab->ro_rows[c]] * p.N + n0 + j] = v;
-      }
-    }
-  } else if (EPI == EPI_RESID) {
-    int n0 = rb * RB_ROWS;
-    for (int c = warp; c < n_cols; c += GEMM_THREADS / 32) {
-      float4* h = reinterpret_cast<float4*>(p.hid + (size_t)tab->hid_idx[c] * p.H + n0) + lane;
-      float4 v = *h;
-      const float* tr = tile + c * TILE_LD + lane * 4;
-      v.x += tr[0], v.y += tr[1], v.z += tr[2], v.w += tr[3];
-      *h = v;
-      float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
-      if (lane == 0) p.sumsq_out[c * p.n_sq_out + rb] = ss;
-      if (p.out_planes) {  // the next norm's gain, then the three-way split, once for every consumer
-        float4 gn = *reinterpret_cast<const float4*>(p.gain_next + n0 + lane * 4);
-        float xv[4] = {v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w};
-        unsigned short hh[4], mm[4], ll[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) split3(xv[i], hh[i], mm[i], ll[i]);
-        __nv_bfloat16* dst = p.out_planes + (size_t)c * 3 * p.planes_ld + n0 + lane * 4;
-        *reinterpret_cast<uint2*>(dst) = make_uint2(hh[0] | ((unsigned)hh[1] << 16), hh[2] | ((unsigned)hh[3] << 16));
-        *reinterpret_cast<uint2*>(dst + p.planes_ld) = make_uint2(mm[0] | ((unsigned)mm[1] << 16), mm[2] | ((unsigned)mm[3] << 16));
-        *reinterpret_cast<uint2*>(dst + 2 * p.planes_ld) = make_uint2(ll[0] | ((unsigned)ll[1] << 16), ll[2] | ((unsigned)ll[3] << 16));
-      }
-    }
-  } else if (EPI == EPI_SWIGLU) {
-    int j0 = rb * 64;
-    for (int idx = tid; idx < n_cols * 64; idx += GEMM_THREADS) {
-      int c = idx >> 6, jj = idx & 63;
-      if (j0 + jj < p.F) {
-        float gt = tile[c * TILE_LD + jj] * s_rstd[c], up = tile[c * TILE_LD + 64 + jj] * s_rstd[c];
-        store_split(p.out_planes + (size_t)c * 3 * p.planes_ld, p.planes_ld, j0 + jj, gt / (1.0f + expf(-gt)) * up);
-      }
-    }
-  } else if (EPI == EPI_QKV) {
-    const int d = p.head_dim, hd2 = d >> 1;
-    const int Hq = p.n_q_heads * d, Hk = p.n_kv_heads * d;
-    int n0 = rb * RB_ROWS;
-    int region = n0 < Hq ? 0 : (n0 < Hq + Hk ? 1 : 2);
-    int base = region == 0 ? 0 : (region == 1 ? Hq : Hq + Hk);
-    for (int idx = tid; idx < n_cols * 64; idx += GEMM_THREADS) {
-      int c = idx >> 6, pr = idx & 63;        // pair index inside the 128-row block
-      int hh = pr / hd2, i = pr - hh * hd2;   // head inside the block, rotary pair
-      float x1 = tile[c * TILE_LD + hh * d + i] * s_rstd[c], x2 = tile[c * TILE_LD + hh * d + i + hd2] * s_rstd[c];
-      float y1 = x1, y2 = x2;
-      if (region < 2) {
-        float2 cs = p.rope[(size_t)tab->pos[c] * hd2 + i];
-        y1 = x1 * cs.x - x2 * cs.y;
-        y2 = x2 * cs.x + x1 * cs.y;
-      }
-      int head = (n0 - base) / d + hh;
-      if (region == 0) {
-        float* q = p.qbuf + (size_t)c * Hq + head * d + i;
-        q[0] = y1;
-        q[hd2] = y2;
-      } else {
-        __nv_bfloat16* dst = p.kv + (size_t)(tab->r[c] - 1) * p.kv_plane_stride + (size_t)(region - 1) * p.kv_sel_stride +
-                             ((size_t)(tab->seq[c] * p.n_kv_heads + head) * p.slots + tab->kv_slot[c]) * d + i;
-        dst[0] = __float2bfloat16_rn(y1);
-        dst[hd2] = __float2bfloat16_rn(y2);
-      }
-    }
-  }
-}
-
-// ---- a row block's share is complete: publish it, and reduce + finish if this CTA is the last one -------
-// acc: this thread's MMA accumulator fragments (rows warp*16+g / +8, columns n*8+2t / +1)
-template <int NG, int EPI>
-__device__ __forceinline__ void gemm_finish_segment(const GemmParams& p, const RowTable* tab, int rb, int n_cols,
-                                                    const float (&acc)[NG][4], float* tile, const float* s_rstd, int* s_flag) {
-  constexpr int NTOK = 8 * NG;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int kpr = p.kb_per_rb;
-  int c_first = (rb * kpr) / p.units_per_cta;
-  int c_last = ((rb + 1) * kpr - 1) / p.units_per_cta;
-  int n_contrib = c_last - c_first + 1;
-  int rl = warp * 16 + g;
-  if (n_contrib == 1) {
-#pragma unroll
-    for (int n = 0; n < NG; ++n) {
-      int c0 = n * 8 + 2 * t;
-      tile[c0 * TILE_LD + rl] = acc[n][0];
-      tile[(c0 + 1) * TILE_LD + rl] = acc[n][1];
-      tile[c0 * TILE_LD + rl + 8] = acc[n][2];
-      tile[(c0 + 1) * TILE_LD + rl + 8] = acc[n][3];
-    }
-    __syncthreads();
-    gemm_epilogue<EPI>(p, tab, rb, n_cols, tile, s_rstd);
-  } else {
-    int ord = blockIdx.x - c_first;
-    float* dst = p.partials + ((size_t)rb * p.max_contrib + ord) * (NTOK * RB_ROWS);
-#pragma unroll
-    for (int n = 0; n < NG; ++n) {
-      int c0 = n * 8 + 2 * t;
-      if (c0 < n_cols) {  // columns beyond the live rows are never read back
-        __stcg(dst + c0 * RB_ROWS + rl, acc[n][0]);
-        __stcg(dst + c0 * RB_ROWS + rl + 8, acc[n][2]);
-        if (c0 + 1 < n_cols) {
-          __stcg(dst + (c0 + 1) * RB_ROWS + rl, acc[n][1]);
-          __stcg(dst + (c0 + 1) * RB_ROWS + rl + 8, acc[n][3]);
-        }
-      }
-    }
-    __syncthreads();
-    if (tid == 0) {
-      __threadfence();  // the CTA's partials (ordered before this by the barrier) are visible device-wide
-      int old = atomicAdd(p.counters + rb, 1);
-      *s_flag = (old == n_contrib - 1);
-      __threadfence();
-    }
-    __syncthreads();
-    if (*s_flag) {
-      const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)rb * p.max_contrib * (NTOK * RB_ROWS));
-      for (int idx = tid; idx < n_cols * (RB_ROWS / 4); idx += GEMM_THREADS) {
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int o = 0; o < n_contrib; ++o) {
-          float4 v = __ldcg(src + (size_t)o * (NTOK * RB_ROWS / 4) + idx);
-          s.x += v.x, s.y += v.y, s.z += v.z, s.w += v.w;
-        }
-        int c = idx / (RB_ROWS / 4), j = (idx % (RB_ROWS / 4)) * 4;
-        float* tr = tile + c * TILE_LD + j;
-        tr[0] = s.x, tr[1] = s.y, tr[2] = s.z, tr[3] = s.w;
-      }
-      if (tid == 0) p.counters[rb] = 0;
-      __syncthreads();
-      gemm_epilogue<EPI>(p, tab, rb, n_cols, tile, s_rstd);
-    }
-  }
-  __syncthreads();  // tile and s_flag are reused by the next segment
-}
-
 // first weight row this warp streams for row block rb (-1: outside the matrix)
 template <int EPI>
 __device__ __forceinline__ int gemm_row0(const GemmParams& p, int rb, int warp) {
@@ -238,6 +96,96 @@ __device__ __forceinline__ int gemm_row0(const GemmParams& p, int rb, int warp) 
   }
   int r = rb * RB_ROWS + warp * 16;
   return r < p.N ? r : -1;
+}
+
+// k-blocks [lo, hi) of cluster rank `rank`
+__device__ __forceinline__ void gemm_krange(int kpr, int cs, int rank, int& lo, int& hi) {
+  int q = kpr / cs, r = kpr % cs;
+  lo = rank * q + min(rank, r);
+  hi = lo + q + (rank < r ? 1 : 0);
+}
+
+// ---- the cluster's partial tiles are complete: sum them in rank order and finish this CTA's columns ------
+// Column c of row block rb is finished by rank (c mod cluster size); threads 0..127 take one column, threads
+// 128..255 the next one of this rank, one output row each.
+template <int EPI>
+__device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, float* tile,
+                                                     float* colbuf, const float* s_rstd, cg::cluster_group& cluster) {
+  const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
+  const int cs = p.cluster_size, rank = (int)cluster.block_rank();
+  __shared__ float s_ss[2][4];
+  for (int base = rank; base < n_cols; base += 2 * cs) {
+    const int c = base + cs * half;
+    const bool live = c < n_cols;
+    float v = 0.f;
+    if (live) {
+      for (int rk = 0; rk < cs; ++rk) {
+        const float* remote = cs > 1 ? cluster.map_shared_rank(tile, rk) : tile;
+        v += remote[c * TILE_LD + j];
+      }
+      v *= s_rstd[c];
+    }
+    if (EPI == EPI_PLAIN || EPI == EPI_LOGITS) {
+      const int n = rb * RB_ROWS + j;
+      if (live && n < p.N) {
+        if (EPI == EPI_PLAIN) p.out[(size_t)c * p.out_ld + n] = v;
+        else p.logits[(size_t)tab->logit_idx[tab->ro_rows[c]] * p.N + n] = v;
+      }
+    } else if (EPI == EPI_RESID) {
+      const int n = rb * RB_ROWS + j;
+      float xn = 0.f;
+      if (live) {
+        float* h = p.hid + (size_t)tab->hid_idx[c] * p.H + n;
+        xn = *h + v;
+        *h = xn;
+        if (p.out_planes) store_split(p.out_planes + (size_t)c * 3 * p.planes_ld, p.planes_ld, n, xn * p.gain_next[n]);
+      }
+      float ss = warp_sum(xn * xn);
+      if (lane == 0) s_ss[half][hw] = ss;
+      __syncthreads();
+      if (live && j == 0) p.sumsq_out[c * p.n_sq_out + rb] = (s_ss[half][0] + s_ss[half][1]) + (s_ss[half][2] + s_ss[half][3]);
+      __syncthreads();
+    } else {
+      colbuf[half * RB_ROWS + j] = v;
+      __syncthreads();
+      if (live && j < 64) {
+        const float* col = colbuf + half * RB_ROWS;
+        if (EPI == EPI_SWIGLU) {
+          const int f = rb * 64 + j;
+          if (f < p.F) {
+            float gt = col[j], up = col[64 + j];
+            store_split(p.out_planes + (size_t)c * 3 * p.planes_ld, p.planes_ld, f, gt / (1.0f + expf(-gt)) * up);
+          }
+        } else {  // EPI_QKV: rotary pair j of the 128-row block, then q to the query buffer, k/v to the cache
+          const int d = p.head_dim, hd2 = d >> 1;
+          const int Hq = p.n_q_heads * d, Hk = p.n_kv_heads * d;
+          const int n0 = rb * RB_ROWS;
+          const int region = n0 < Hq ? 0 : (n0 < Hq + Hk ? 1 : 2);
+          const int rbase = region == 0 ? 0 : (region == 1 ? Hq : Hq + Hk);
+          const int hh = j / hd2, i = j - hh * hd2;
+          const float x1 = col[hh * d + i], x2 = col[hh * d + i + hd2];
+          float y1 = x1, y2 = x2;
+          if (region < 2) {
+            float2 csn = p.rope[(size_t)tab->pos[c] * hd2 + i];
+            y1 = x1 * csn.x - x2 * csn.y;
+            y2 = x2 * csn.x + x1 * csn.y;
+          }
+          const int head = (n0 - rbase) / d + hh;
+          if (region == 0) {
+            float* q = p.qbuf + (size_t)c * Hq + head * d + i;
+            q[0] = y1;
+            q[hd2] = y2;
+          } else {
+            __nv_bfloat16* dst = p.kv + (size_t)(tab->r[c] - 1) * p.kv_plane_stride + (size_t)(region - 1) * p.kv_sel_stride +
+                                 ((size_t)(tab->seq[c] * p.n_kv_heads + head) * p.slots + tab->kv_slot[c]) * d + i;
+            dst[0] = __float2bfloat16_rn(y1);
+            dst[hd2] = __float2bfloat16_rn(y2);
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
 }
 
 __device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float* s_rstd) {
@@ -253,43 +201,66 @@ __device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float
   }
 }
 
+// write this thread's accumulator fragments (rows warp*16+g / +8, columns n*8+2t / +1) into the partial tile
+template <int NG>
+__device__ __forceinline__ void gemm_store_tile(const float (&acc)[NG][4], float* tile) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int rl = warp * 16 + g;
+#pragma unroll
+  for (int n = 0; n < NG; ++n) {
+    const int c0 = n * 8 + 2 * t;
+    tile[c0 * TILE_LD + rl] = acc[n][0];
+    tile[(c0 + 1) * TILE_LD + rl] = acc[n][1];
+    tile[c0 * TILE_LD + rl + 8] = acc[n][2];
+    tile[(c0 + 1) * TILE_LD + rl + 8] = acc[n][3];
+  }
+}
+
 // ======================================= bf16 weights: tensor cores ========================================
 template <int NG, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
   constexpr int NTOK = 8 * NG;
   constexpr int XCH = xchunk_kblocks(NG);
-  constexpr int XBUF = xbuf_uint4(NG);
   constexpr int PIECES = 3 * XCH * NTOK * 4;
   constexpr int PPT = (PIECES + GEMM_THREADS - 1) / GEMM_THREADS;
-  constexpr int NCH = 3;  // independent accumulator chains, one per split term (the same for every NG:
-                          // a row's bits must not depend on how many rows share the pass)
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);            // [RING][2][256], slot of thread tid only
-  uint4* xbuf = ring + RING * 2 * GEMM_THREADS;                // [2][3][XCH][NTOK][4]
-  float* tile = reinterpret_cast<float*>(xbuf + 2 * XBUF);     // [NTOK][TILE_LD]
-  float* s_rstd = tile + NTOK * TILE_LD;
-  int* s_flag = reinterpret_cast<int*>(s_rstd + NTOK);
+  uint4* xbuf = ring + RING * 2 * GEMM_THREADS;                // [3][XCH][NTOK][4]
+  float* tile = reinterpret_cast<float*>(xbuf + xbuf_uint4(NG));  // [NTOK][TILE_LD]
+  float* colbuf = tile + NTOK * TILE_LD;                       // [2][128]
+  float* s_rstd = colbuf + 2 * RB_ROWS;
 
+  cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int cs = p.cluster_size, rank = (int)cluster.block_rank(), cid = blockIdx.x / cs;
   const int kpr = p.kb_per_rb;
-  const int u_begin = blockIdx.x * p.units_per_cta;
-  const int u_end = min(u_begin + p.units_per_cta, p.total_units);
-  const int n_units = u_end - u_begin;  // >= 1 by construction of the grid
+  int kb_lo, kb_hi;
+  gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
+  const int upt = kb_hi - kb_lo;                                 // units per task
+  const int n_tasks = (p.n_rb - cid + p.n_clusters - 1) / p.n_clusters;  // row blocks cid, cid + n_clusters, ...
+  const int n_units = n_tasks * upt;
 
-  // ---- weight ring: issue side ---------------------------------------------------------------------------
-  int i_rb = u_begin / kpr, i_kb = u_begin - i_rb * kpr, i_row0 = gemm_row0<EPI>(p, i_rb, warp), i_cnt = 0;
+  // ---- weight ring: issue side.  The weights are stored tile-major (see pack_weights_kernel): the 1 KB a warp
+  // consumes per unit is contiguous and consecutive k-blocks of a 16-row tile follow each other, so every warp
+  // streams one contiguous region and every request covers whole 128-byte lines.
+  int i_rb = cid, i_kb = kb_lo, i_cnt = 0;
+  const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
+  const __nv_bfloat16* i_ptr = Wb;
+  bool i_ok = false;
+  auto i_setup = [&]() {
+    int r0 = gemm_row0<EPI>(p, i_rb, warp);
+    i_ok = r0 >= 0;
+    i_ptr = Wb + (i_ok ? ((size_t)(r0 >> 4) * kpr + i_kb) * 512 : 0) + lane * 8;
+  };
+  i_setup();
   auto issue_unit = [&]() {
     if (i_cnt < n_units) {
-      const int k = i_kb * 32 + t * 8;
-      const bool valid = i_row0 >= 0 && k < p.K;
-      const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(p.W);
-      if (valid) src += (size_t)(i_row0 + g) * p.K + k;
-      uint4* slot = ring + (size_t)(i_cnt % RING) * 2 * GEMM_THREADS + tid;
-      cp_async16(slot, src, valid);
-      cp_async16(slot + GEMM_THREADS, valid ? src + (size_t)8 * p.K : src, valid);
-      ++i_cnt;
-      if (++i_kb == kpr) i_kb = 0, ++i_rb, i_row0 = gemm_row0<EPI>(p, i_rb, warp);
+      uint4* slot = ring + (i_cnt & (RING - 1)) * 2 * GEMM_THREADS + tid;
+      cp_async16(slot, i_ok ? i_ptr : Wb, i_ok);
+      cp_async16(slot + GEMM_THREADS, i_ok ? i_ptr + 256 : Wb, i_ok);
+      ++i_cnt, i_ptr += 512;
+      if (++i_kb == kb_hi) i_kb = kb_lo, i_rb += p.n_clusters, i_setup();
     }
     cp_async_commit();
   };
@@ -300,105 +271,91 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   pdl_launch_dependents();
   pdl_wait();
 
-  const RowTable* tab = p.tab;
-  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
-  if (n_cols > NTOK) n_cols = NTOK;
-  if (n_cols <= 0) {
-    cp_async_wait<0>();
-    return;
-  }
-  gemm_rstd(p, n_cols, s_rstd);
-
-  // ---- activation chunks: gathered into registers one chunk ahead, then stored in MMA-fragment order -----
+  // ---- activations of this CTA's k-range: piece idx -> (plane s, k-block kbl, column c, quarter tt) ---------
+  // Columns beyond the live rows may hold stale values: every column is an independent dot product and the
+  // epilogue never reads them.
   uint4 xr[PPT];
   auto x_fetch = [&](int kb0, int nkb) {
 #pragma unroll
     for (int i = 0; i < PPT; ++i) {
-      int idx = tid + i * GEMM_THREADS;
+      const int idx = tid + i * GEMM_THREADS;
+      const int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % XCH, s = r / XCH;
+      const int k = (kb0 + kbl) * 32 + tt * 8;
       xr[i] = make_uint4(0, 0, 0, 0);
-      if (idx < 3 * nkb * NTOK * 4) {
-        int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % nkb, s = r / nkb;
-        int k = (kb0 + kbl) * 32 + tt * 8;
-        if (c < n_cols && k < p.K)
-          xr[i] = *reinterpret_cast<const uint4*>(p.xplanes + ((size_t)c * 3 + s) * p.x_ld + k);
-      }
+      if (idx < PIECES && kbl < nkb && k < p.K)
+        xr[i] = *reinterpret_cast<const uint4*>(p.xplanes + ((size_t)c * 3 + s) * p.x_ld + k);
     }
   };
-  auto x_store = [&](int nkb, int buf) {
+  auto x_store = [&]() {
 #pragma unroll
     for (int i = 0; i < PPT; ++i) {
-      int idx = tid + i * GEMM_THREADS;
-      if (idx < 3 * nkb * NTOK * 4) {
-        int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % nkb, s = r / nkb;
-        xbuf[buf * XBUF + ((s * XCH + kbl) * NTOK + c) * 4 + tt] = xr[i];
-      }
+      const int idx = tid + i * GEMM_THREADS;
+      if (idx < PIECES) xbuf[idx] = xr[i];   // [s][kbl][c][tt] is exactly the piece order
     }
   };
+  const bool one_chunk = upt <= XCH;  // the whole k-range stays staged for every row block of this CTA
+  x_fetch(kb_lo, min(XCH, upt));
 
-  float acc[NCH][NG][4];
-  auto zero_acc = [&]() {
+  const RowTable* tab = p.tab;
+  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
+  if (n_cols > NTOK) n_cols = NTOK;
+  if (n_cols <= 0) {  // uniform over the cluster: nobody reaches a cluster barrier
+    cp_async_wait<0>();
+    return;
+  }
+  gemm_rstd(p, n_cols, s_rstd);
+  x_store();
+  __syncthreads();
+
+  float acc[3][NG][4];  // one chain per split term, the same for every NG: a row's bits must not depend on
+                        // how many rows share the pass
+  const uint4* xs = xbuf + g * 4 + t;
+  int j = 0;
+  for (int task = 0; task < n_tasks; ++task) {
+    const int rb = cid + task * p.n_clusters;
+    const bool warp_valid = gemm_row0<EPI>(p, rb, warp) >= 0;
 #pragma unroll
-    for (int h = 0; h < NCH; ++h)
+    for (int h = 0; h < 3; ++h)
 #pragma unroll
       for (int n = 0; n < NG; ++n)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[h][n][i] = 0.f;
-  };
-  zero_acc();
-
-  // ---- consume side: segments (one row block each) of chunks of units ------------------------------------
-  int c_rb = u_begin / kpr, c_kb = u_begin - c_rb * kpr;
-  int j = 0, xb = 0;
-  {
-    int seg_len = min(kpr - c_kb, n_units);
-    x_fetch(c_kb, min(XCH, seg_len));
-  }
-  while (j < n_units) {
-    const int seg_len = min(kpr - c_kb, n_units - j);
-    const bool warp_valid = gemm_row0<EPI>(p, c_rb, warp) >= 0;
-    for (int ck = 0; ck < seg_len; ck += XCH) {
-      const int nkb = min(XCH, seg_len - ck);
-      x_store(nkb, xb);
-      __syncthreads();
-      {  // fetch the next chunk (of this segment, or the first of the next) while this one is consumed
-        int nk0 = ck + XCH;
-        if (nk0 < seg_len) x_fetch(c_kb + nk0, min(XCH, seg_len - nk0));
-        else if (j + (seg_len - ck) < n_units) x_fetch(0, min(XCH, min(kpr, n_units - j - (seg_len - ck))));
+    for (int ck = 0; ck < upt; ck += XCH) {
+      const int nkb = min(XCH, upt - ck);
+      if (!one_chunk) {  // wide passes (prefill): restage the activations chunk by chunk
+        __syncthreads();
+        x_fetch(kb_lo + ck, nkb);
+        x_store();
+        __syncthreads();
       }
-      const uint4* xs = xbuf + xb * XBUF;
       for (int kbl = 0; kbl < nkb; ++kbl, ++j) {
         issue_unit();
         cp_async_wait<RING - 1>();
         if (warp_valid) {
-          const uint4* slot = ring + (size_t)(j % RING) * 2 * GEMM_THREADS + tid;
+          const uint4* slot = ring + (j & (RING - 1)) * 2 * GEMM_THREADS + tid;
           const uint4 a_lo = slot[0], a_hi = slot[GEMM_THREADS];
 #pragma unroll
           for (int s = 0; s < 3; ++s) {
 #pragma unroll
             for (int n = 0; n < NG; ++n) {
-              const uint4 b = xs[((s * XCH + kbl) * NTOK + n * 8 + g) * 4 + t];
-              float(&c)[4] = acc[NCH == 3 ? s : 0][n];
-              mma_bf16(c, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
-              mma_bf16(c, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
+              const uint4 b = xs[((s * XCH + kbl) * NTOK + n * 8) * 4];
+              mma_bf16(acc[s][n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
+              mma_bf16(acc[s][n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
             }
           }
         }
       }
-      xb ^= 1;
     }
-    // fold the chains in fixed order: hi + (mid + lo)
+    // fold the chains in fixed order, hi + (mid + lo), and publish this CTA's partial tile
     float tot[NG][4];
 #pragma unroll
     for (int n = 0; n < NG; ++n)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if constexpr (NCH == 3) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
-        else tot[n][i] = acc[0][n][i];
-      }
-    gemm_finish_segment<NG, EPI>(p, tab, c_rb, n_cols, tot, tile, s_rstd, s_flag);
-    zero_acc();
-    c_kb += seg_len;
-    if (c_kb == kpr) c_kb = 0, ++c_rb;
+      for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
+    gemm_store_tile<NG>(tot, tile);
+    cluster.sync();
+    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, tile, colbuf, s_rstd, cluster);
+    cluster.sync();  // nobody overwrites (or leaves with) a tile another rank is still reading
   }
   cp_async_wait<0>();
 }
@@ -413,14 +370,17 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* xf = reinterpret_cast<float*>(smem_raw);              // [XCH][NTOK][32]
   float* tile = xf + XCH * NTOK * 32;                          // [NTOK][TILE_LD]
-  float* s_rstd = tile + NTOK * TILE_LD;
-  int* s_flag = reinterpret_cast<int*>(s_rstd + NTOK);
+  float* colbuf = tile + NTOK * TILE_LD;
+  float* s_rstd = colbuf + 2 * RB_ROWS;
 
+  cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int cs = p.cluster_size, rank = (int)cluster.block_rank(), cid = blockIdx.x / cs;
   const int kpr = p.kb_per_rb;
-  const int u_begin = blockIdx.x * p.units_per_cta;
-  const int u_end = min(u_begin + p.units_per_cta, p.total_units);
-  const int n_units = u_end - u_begin;
+  int kb_lo, kb_hi;
+  gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
+  const int upt = kb_hi - kb_lo;
+  const int n_tasks = (p.n_rb - cid + p.n_clusters - 1) / p.n_clusters;
   pdl_launch_dependents();
   pdl_wait();
   const RowTable* tab = p.tab;
@@ -429,21 +389,20 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   if (n_cols <= 0) return;
   gemm_rstd(p, n_cols, s_rstd);
 
-  int c_rb = u_begin / kpr, c_kb = u_begin - c_rb * kpr, j = 0;
-  while (j < n_units) {
-    const int seg_len = min(kpr - c_kb, n_units - j);
-    const int row0 = gemm_row0<EPI>(p, c_rb, warp);
+  for (int task = 0; task < n_tasks; ++task) {
+    const int rb = cid + task * p.n_clusters;
+    const int row0 = gemm_row0<EPI>(p, rb, warp);
     float accf[NG][8][2];
 #pragma unroll
     for (int n = 0; n < NG; ++n)
 #pragma unroll
       for (int c = 0; c < 8; ++c) accf[n][c][0] = accf[n][c][1] = 0.f;
-    for (int ck = 0; ck < seg_len; ck += XCH) {
-      const int nkb = min(XCH, seg_len - ck);
+    for (int ck = 0; ck < upt; ck += XCH) {
+      const int nkb = min(XCH, upt - ck);
       __syncthreads();
       for (int idx = tid; idx < nkb * NTOK * 32; idx += GEMM_THREADS) {
         int e = idx & 31, c = (idx >> 5) % NTOK, kbl = idx / (32 * NTOK);
-        int k = (c_kb + ck + kbl) * 32 + e;
+        int k = (kb_lo + ck + kbl) * 32 + e;
         float v = 0.f;
         if (c < n_cols && k < p.K) {
           const __nv_bfloat16* pl = p.xplanes + (size_t)c * 3 * p.x_ld + k;
@@ -454,7 +413,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
       __syncthreads();
       if (row0 >= 0) {
         for (int kbl = 0; kbl < nkb; ++kbl) {
-          const int k = (c_kb + ck + kbl) * 32 + t * 8;
+          const int k = (kb_lo + ck + kbl) * 32 + t * 8;
           if (k < p.K) {
             const float* wl = static_cast<const float*>(p.W) + (size_t)(row0 + g) * p.K + k;
             const float* wh = wl + (size_t)8 * p.K;
@@ -477,7 +436,6 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
         }
       }
     }
-    j += seg_len;
     // fold the four k-lanes, then take the MMA accumulator layout the shared epilogue expects
     float tot[NG][4];
 #pragma unroll
@@ -492,12 +450,40 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
           if (c == 2 * t) tot[n][2 * h] = v;
           if (c == 2 * t + 1) tot[n][2 * h + 1] = v;
         }
-    gemm_finish_segment<NG, EPI>(p, tab, c_rb, n_cols, tot, tile, s_rstd, s_flag);
-    c_kb += seg_len;
-    if (c_kb == kpr) c_kb = 0, ++c_rb;
+    gemm_store_tile<NG>(tot, tile);
+    cluster.sync();
+    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, tile, colbuf, s_rstd, cluster);
+    cluster.sync();
   }
 }
-__host__ __device__ constexpr int gemm_f32_smem_bytes(int NG) { return 4 * 8 * NG * 32 * 4 + 8 * NG * TILE_LD * 4 + 8 * NG * 4 + 16; }
+__host__ __device__ constexpr int gemm_f32_smem_bytes(int NG) {
+  return 4 * 8 * NG * 32 * 4 + 8 * NG * TILE_LD * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
+}
+
+// ---- one-time repacking of a bf16 weight matrix [N][K] into the tile-major streaming layout ----------------
+// unit (rt, kb) = rows rt*16 .. +15, k = kb*32 .. +31, 1 KB: first the 512 bytes of the "low" pieces (lane g*4+t
+// holds row rt*16+g, k = kb*32 + t*8 .. +7), then the 512 bytes of the "high" pieces (row rt*16+g+8); k beyond
+// K is zero.  Units of one row tile are consecutive in kb.
+struct PackParams {
+  const __nv_bfloat16* src;  // [N][K]
+  __nv_bfloat16* dst;        // [N/16][kpr][2][32][8]
+  int N, K, kpr;
+};
+__global__ void pack_weights_kernel(const __grid_constant__ PackParams p) {
+  const size_t n_pieces = (size_t)(p.N / 16) * p.kpr * 64;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_pieces; i += (size_t)gridDim.x * blockDim.x) {
+    const int lane = (int)(i & 31), hi = (int)((i >> 5) & 1);
+    const size_t unit = i >> 6;
+    const int kb = (int)(unit % p.kpr);
+    const size_t rt = unit / p.kpr;
+    const int g = lane >> 2, t = lane & 3;
+    const size_t row = rt * 16 + g + 8 * hi;
+    const int k = kb * 32 + t * 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (k < p.K) v = *reinterpret_cast<const uint4*>(p.src + row * p.K + k);
+    reinterpret_cast<uint4*>(p.dst)[i] = v;
+  }
+}
 
 // ---- fp32 rows -> three bf16 planes, optionally through RMSNorm's gain, with the row's sum of squares -----
 struct PrepParams {

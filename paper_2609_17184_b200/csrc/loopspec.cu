@@ -19,25 +19,34 @@ using namespace ls;
 
 namespace {
 
-constexpr int kCtasPerSm = 1;
+constexpr int kCtasPerSm = 2;
 
 struct GemmPlan {
-  int n_rb, kpr, upc, total, grid, max_contrib;
+  int n_rb, kpr, cs, n_clusters, grid;
 };
 
-GemmPlan plan_gemm(int n_rb, int K, int target_ctas) {
+// Cluster size = how many CTAs split K for one block of 128 output rows.  Enough CTAs to fill the resident
+// slots (two per SM), a k-range short enough that a decode pass keeps its activations staged once, and whole
+// rounds of row blocks per cluster so that every CTA streams the same number of bytes.
+GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only) {
   GemmPlan g;
   g.n_rb = n_rb;
   g.kpr = (K + 31) / 32;
-  g.total = g.n_rb * g.kpr;
-  int grid = std::min(target_ctas, g.total);
-  g.upc = (g.total + grid - 1) / grid;
-  g.grid = (g.total + g.upc - 1) / g.upc;
-  g.max_contrib = 1;
-  for (int rb = 0; rb < n_rb; ++rb) {
-    int cf = (rb * g.kpr) / g.upc, cl = ((rb + 1) * g.kpr - 1) / g.upc;
-    g.max_contrib = std::max(g.max_contrib, cl - cf + 1);
+  int cs_min = (g.kpr + MAX_XCH_BLOCKS - 1) / MAX_XCH_BLOCKS;
+  int cs = std::max(1, slots / std::max(n_rb, 1));
+  cs = std::max(cs, cs_min);
+  cs = std::min(std::min(cs, 8), g.kpr);
+  if (pow2_only) {
+    int q = 1;
+    while (q < cs) q <<= 1;
+    cs = std::min(std::min(q, 8), g.kpr);
+    while (cs & (cs - 1)) --cs;
   }
+  g.cs = cs;
+  int max_clusters = std::max(1, slots / cs);
+  int rounds = (n_rb + max_clusters - 1) / max_clusters;
+  g.n_clusters = (n_rb + rounds - 1) / rounds;
+  g.grid = g.n_clusters * cs;
   return g;
 }
 
@@ -45,7 +54,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, gpart, gcnt, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -142,7 +151,16 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   return true;
 }
 
-Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Derived& d, int n_sm) {
+// bytes of one matrix in the tile-major streaming layout (bf16 weights only; fp32 weights are used in place)
+size_t packed_bytes(int N, int K) { return align_up((size_t)(N / 16) * ((K + 31) / 32) * 1024); }
+size_t packed_total_bytes(const loopspec_model* m, const Derived& d) {
+  if (m->weight_dtype != 1) return 0;
+  size_t per_layer = packed_bytes(d.Hq + 2 * d.Hkv, m->hidden) + packed_bytes(m->hidden, d.Hq) +
+                     packed_bytes(2 * m->ffn, m->hidden) + packed_bytes(m->hidden, m->ffn);
+  return per_layer * m->n_recurrent + packed_bytes(m->vocab, m->hidden);
+}
+
+Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Derived& d) {
   Layout L;
   size_t o = 0;
   auto take = [&](size_t bytes) {
@@ -151,6 +169,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
     return at;
   };
   const size_t MR = d.max_rows;
+  L.wpack = take(packed_total_bytes(m, d));
   L.rope = take((size_t)s->max_ctx * (m->head_dim / 2) * sizeof(float2));
   L.kv = take((size_t)m->n_recurrent * m->R * 2 * d.S * m->n_kv_heads * d.slots * m->head_dim * 2);
   L.hid = take((size_t)d.n_hid * m->hidden * 4);
@@ -161,15 +180,6 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sumsq = take(MR * d.n_sq * 4);
   L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
-  // split-k scratch: the largest of the five GEMMs at the widest token-group count in use
-  int target = n_sm * kCtasPerSm;
-  GemmPlan plans[5] = {plan_gemm((d.Hq + 2 * d.Hkv) / 128, m->hidden, target), plan_gemm(m->hidden / 128, d.Hq, target),
-                       plan_gemm((m->ffn + 63) / 64, m->hidden, target), plan_gemm(m->hidden / 128, m->ffn, target),
-                       plan_gemm((m->vocab + 127) / 128, m->hidden, target)};
-  size_t pf = 0, cnt = 0;
-  for (auto& g : plans) pf = std::max(pf, (size_t)g.n_rb * g.max_contrib), cnt = std::max(cnt, (size_t)g.n_rb);
-  L.gpart = take(pf * MR * 128 * 4);
-  L.gcnt = take(cnt * 4);
   int G = m->n_q_heads / m->n_kv_heads;
   L.apart = take(MR * m->n_kv_heads * d.max_chunks * G * (m->head_dim + 2) * 4);
   L.acnt = take(MR * m->n_kv_heads * 4);
@@ -206,6 +216,7 @@ struct loopspec_ctx {
   const void* lm_head = nullptr;
   const float* final_norm = nullptr;
   std::vector<const void*> layers;  // 6 per layer
+  std::vector<const void*> packed;  // 4 per layer (qkv, o, gate/up, down) + lm_head; empty for fp32 weights
   int n_sm = 148;
   int ng_dec = 1, ng_pf = 1;
   GemmPlan plan[5];
@@ -299,19 +310,30 @@ int gemm_smem(int wdt, int ng) { return wdt == 1 ? gemm_smem_bytes(ng) : gemm_f3
 // Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream is
 // still running; it orders itself with griddepcontrol.wait before touching anything the predecessor writes.
 template <typename P>
-cudaError_t launch_k(void (*fn)(const P), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const P& params, bool pdl) {
+cudaError_t launch_k(void (*fn)(const P), dim3 grid, dim3 block, size_t smem, cudaStream_t st, const P& params, bool pdl,
+                     int cluster = 1) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at, cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchAttribute at[2];
+  int n = 0;
+  if (pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = cluster, at[n].val.clusterDim.y = 1, at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = at, cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, fn, params);
 }
 
-cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, int grid, cudaStream_t st, bool pdl = true) {
-  return launch_k(gemm_fn(wdt, ng, epi), dim3(grid), dim3(GEMM_THREADS), (size_t)gemm_smem(wdt, ng), st, p, pdl);
+cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, cudaStream_t st, bool pdl = true) {
+  return launch_k(gemm_fn(wdt, ng, epi), dim3(p.n_clusters * p.cluster_size), dim3(GEMM_THREADS), (size_t)gemm_smem(wdt, ng), st, p,
+                  pdl, p.cluster_size);
 }
 
 using AttnFn = void (*)(const AttnParams);
@@ -322,6 +344,7 @@ AttnFn attn_fn(int d, int G) {
 
 // ---- one batched pass through the shared block stack (all layers) on the rows of `tab` ------------------
 enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_LM = 4 };
+const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
 
 GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
   const loopspec_model& m = c->m;
@@ -329,14 +352,13 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   GemmParams p;
   memset(&p, 0, sizeof p);
   const GemmPlan& g = c->plan[which];
-  p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.units_per_cta = g.upc, p.total_units = g.total, p.max_contrib = g.max_contrib;
-  p.partials = c->at<float>(c->L.gpart), p.counters = c->at<int>(c->L.gcnt);
+  p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.cluster_size = g.cs, p.n_clusters = g.n_clusters;
   p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
   const void* const* lp = which == G_LM ? nullptr : &c->layers[6 * layer];
   __nv_bfloat16* xpl = c->at<__nv_bfloat16>(c->L.xplanes);
   switch (which) {
     case G_QKV:
-      p.W = lp[1], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
+      p.W = c->packed.empty() ? lp[1] : c->packed[4 * layer + 0], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden;
       // layer 0 reads the full sums the preparation kernel wrote; later layers the down-projection's partials
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.n_sq;
@@ -347,19 +369,19 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.rope = c->at<float2>(c->L.rope);
       break;
     case G_O:
-      p.W = lp[2], p.N = m.hidden, p.K = d.Hq;
+      p.W = c->packed.empty() ? lp[2] : c->packed[4 * layer + 1], p.N = m.hidden, p.K = d.Hq;
       p.xplanes = c->at<__nv_bfloat16>(c->L.aplanes), p.x_ld = d.Hq;
       p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
       p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(lp[3]);
       break;
     case G_GU:
-      p.W = lp[4], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
+      p.W = c->packed.empty() ? lp[4] : c->packed[4 * layer + 2], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
       p.xplanes = xpl, p.x_ld = m.hidden;
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.n_sq;
       p.out_planes = c->at<__nv_bfloat16>(c->L.splanes), p.planes_ld = m.ffn;
       break;
     case G_DOWN:
-      p.W = lp[5], p.N = m.hidden, p.K = m.ffn;
+      p.W = c->packed.empty() ? lp[5] : c->packed[4 * layer + 3], p.N = m.hidden, p.K = m.ffn;
       p.xplanes = c->at<__nv_bfloat16>(c->L.splanes), p.x_ld = m.ffn;
       p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
       if (layer + 1 < m.n_recurrent) {
@@ -367,7 +389,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       }
       break;
     default:
-      p.W = c->lm_head, p.N = m.vocab, p.K = m.hidden;
+      p.W = c->packed.empty() ? c->lm_head : c->packed[4 * m.n_recurrent], p.N = m.vocab, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden, p.cols_from_readout = 1;
       p.sumsq = c->at<float>(c->L.sumsq_ro), p.n_sq = 1, p.sq_stride = 1;
       p.logits = c->at<float>(c->L.logits);
@@ -385,7 +407,6 @@ cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
   return launch_k(prep_planes_kernel, dim3(c->d.max_rows), dim3(256), 0, c->stream, q, c->use_pdl);
 }
 
-const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
 
 cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch) {
   const loopspec_model& m = c->m;
@@ -396,7 +417,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   if ((e = launch_prep(c, tab, false))) return e;
   if (n_launch) *n_launch += 1;
   for (int l = 0; l < m.n_recurrent; ++l) {
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->plan[G_QKV].grid, c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->stream, pdl))) return e;
     AttnParams a;
     a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
     a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
@@ -405,9 +426,9 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
     if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 4), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->plan[G_O].grid, c->stream, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->plan[G_GU].grid, c->stream, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->plan[G_DOWN].grid, c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->stream, pdl))) return e;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
   }
   return cudaSuccess;
@@ -416,7 +437,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
   cudaError_t e;
   if ((e = launch_prep(c, tab, true))) return e;
-  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->plan[G_LM].grid, c->stream, c->use_pdl);
+  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->stream, c->use_pdl);
 }
 
 cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) {
@@ -539,13 +560,7 @@ size_t loopspec_workspace_bytes(const loopspec_model* m, const loopspec_sched* s
   int why;
   Derived d;
   if (!validate_model(m, &why) || !resolve_sched(m, s, &d, &why)) return 0;
-  int n_sm = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) {
-    int v = 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n_sm = v;
-  }
-  (void)cudaGetLastError();
-  return make_layout(m, s, d, n_sm).total;
+  return make_layout(m, s, d).total;
 }
 
 int loopspec_pick_depths(float alpha, float beta, int32_t R, double* d1_star, double* d2_star, int32_t* d1, int32_t* d2) {
@@ -582,7 +597,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   int dev = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return LOOPSPEC_ECUDA;
-  Layout L = make_layout(m, s, d, n_sm);
+  Layout L = make_layout(m, s, d);
   if (workspace_bytes < L.total) return LOOPSPEC_ECAPACITY;
 
   loopspec_ctx* c = new loopspec_ctx();
@@ -595,13 +610,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * m->n_recurrent);
   c->ng_dec = ng_for_rows(d.max_rows_dec), c->ng_pf = ng_for_rows(d.max_rows_pf);
   c->prefilled.assign(d.S, 0);
-  int target = n_sm * kCtasPerSm;
-  c->plan[G_QKV] = plan_gemm((d.Hq + 2 * d.Hkv) / 128, m->hidden, target);
-  c->plan[G_O] = plan_gemm(m->hidden / 128, d.Hq, target);
-  c->plan[G_GU] = plan_gemm((m->ffn + 63) / 64, m->hidden, target);
-  c->plan[G_DOWN] = plan_gemm(m->hidden / 128, m->ffn, target);
-  c->plan[G_LM] = plan_gemm((m->vocab + 127) / 128, m->hidden, target);
-
+  const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / 128, (m->ffn + 63) / 64, m->hidden / 128, (m->vocab + 127) / 128};
+  const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
+  for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], n_sm * kCtasPerSm, false);
   for (int ng : {c->ng_dec, c->ng_pf})
     if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
@@ -611,6 +622,36 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           return LOOPSPEC_ECUDA;
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
+  if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
+    int v[5];
+    if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
+      for (int i = 0; i < 5; ++i) {
+        GemmPlan& g = c->plan[i];
+        if (v[i] < 1 || v[i] > 8) continue;
+        g.cs = std::min(v[i], g.kpr);
+        int max_clusters = std::max(1, n_sm * kCtasPerSm / g.cs);
+        int rounds = (g.n_rb + max_clusters - 1) / max_clusters;
+        g.n_clusters = (g.n_rb + rounds - 1) / rounds, g.grid = g.n_clusters * g.cs;
+      }
+  }
+  // cluster sizes that are not powers of two are used only if the device can co-schedule them
+  for (int i = 0; i < 5; ++i) {
+    GemmPlan& g = c->plan[i];
+    if ((g.cs & (g.cs - 1)) == 0) continue;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(g.grid), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = gemm_smem(m->weight_dtype, c->ng_dec);
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = g.cs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+    cfg.attrs = at, cfg.numAttrs = 1;
+    int n_active = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
+    if (e != cudaSuccess || n_active < 1) {
+      (void)cudaGetLastError();
+      g = plan_gemm(n_rbs[i], Ks[i], n_sm * kCtasPerSm, true);
+    }
+  }
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
     (void)what;
@@ -643,9 +684,29 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         cudaStreamSynchronize(c->stream) != cudaSuccess)
       return bail(LOOPSPEC_ECUDA, "rope upload");
   }
+  // bf16 weights: repack every matrix once into the tile-major streaming layout held in the workspace
+  if (m->weight_dtype == 1) {
+    unsigned char* dst = c->ws + L.wpack;
+    auto pack = [&](const void* src, int N, int K) -> bool {
+      PackParams pp;
+      pp.src = static_cast<const __nv_bfloat16*>(src), pp.dst = reinterpret_cast<__nv_bfloat16*>(dst), pp.N = N, pp.K = K;
+      pp.kpr = (K + 31) / 32;
+      pack_weights_kernel<<<n_sm * 8, 256, 0, c->stream>>>(pp);
+      c->packed.push_back(dst);
+      dst += packed_bytes(N, K);
+      return cudaGetLastError() == cudaSuccess;
+    };
+    bool ok = true;
+    for (int l = 0; l < m->n_recurrent && ok; ++l) {
+      const void* const* lp = &c->layers[6 * l];
+      ok = pack(lp[1], d.Hq + 2 * d.Hkv, m->hidden) && pack(lp[2], m->hidden, d.Hq) && pack(lp[4], 2 * m->ffn, m->hidden) &&
+           pack(lp[5], m->hidden, m->ffn);
+    }
+    ok = ok && pack(c->lm_head, m->vocab, m->hidden);
+    if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
+  }
   // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
-  if (cudaMemsetAsync(c->ws + L.gcnt, 0, L.apart - L.gcnt, c->stream) != cudaSuccess ||
-      cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
+  if (cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
       cudaMemsetAsync(c->ws + L.seqs, 0xff, (size_t)MAX_ROWS * 4, c->stream) != cudaSuccess ||  // root = -1
       cudaStreamSynchronize(c->stream) != cudaSuccess)
     return bail(LOOPSPEC_ECUDA, "workspace clear");
@@ -925,7 +986,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
-      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->plan[which].grid, c->stream, c->use_pdl);
+      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }
     return cudaSuccess;
@@ -950,9 +1011,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
 
 size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K) {
   if (M < 1 || M > 64 || N < 16 || K < 8 || N % 16 || K % 8) return 0;
-  int n_rb = (N + 127) / 128;
-  GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
-  return align_up((size_t)n_rb * 4) + align_up((size_t)n_rb * g.max_contrib * 8 * ng_for_rows(M) * 128 * 4) + (size_t)M * 3 * K * 2;
+  return align_up((size_t)M * 3 * K * 2) + packed_bytes(N, K);
 }
 
 int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N, int32_t K,
@@ -963,27 +1022,29 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
   if (!scratch || scratch_bytes < need || (reinterpret_cast<uintptr_t>(scratch) & 15)) return LOOPSPEC_ECAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int ng = ng_for_rows(M);
-  int n_rb = (N + 127) / 128;
-  GemmPlan g = plan_gemm(n_rb, K, 148 * kCtasPerSm);
-  unsigned char* sc = static_cast<unsigned char*>(scratch);
-  size_t off_part = align_up((size_t)n_rb * 4);
-  size_t off_planes = off_part + align_up((size_t)n_rb * g.max_contrib * 8 * ng * 128 * 4);
+  GemmPlan g = plan_gemm((N + 127) / 128, K, 148 * kCtasPerSm, true);
   PrepParams q;
   memset(&q, 0, sizeof q);
-  q.m_fixed = M, q.x = x, q.K = K, q.planes = reinterpret_cast<__nv_bfloat16*>(sc + off_planes);
+  q.m_fixed = M, q.x = x, q.K = K, q.planes = static_cast<__nv_bfloat16*>(scratch);
   if (launch_k(prep_planes_kernel, dim3(M), dim3(256), 0, st, q, false) != cudaSuccess) return LOOPSPEC_ECUDA;
+  if (weight_dtype == 1) {  // stream from a tile-major copy, as the decode path does
+    PackParams pp;
+    pp.src = static_cast<const __nv_bfloat16*>(W), pp.N = N, pp.K = K, pp.kpr = (K + 31) / 32;
+    pp.dst = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(scratch) + align_up((size_t)M * 3 * K * 2));
+    pack_weights_kernel<<<296, 256, 0, st>>>(pp);
+    if (cudaGetLastError() != cudaSuccess) return LOOPSPEC_ECUDA;
+    W = pp.dst;
+  }
   GemmParams p;
   memset(&p, 0, sizeof p);
-  p.W = W, p.N = N, p.K = K, p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.units_per_cta = g.upc, p.total_units = g.total;
-  p.xplanes = q.planes, p.x_ld = K, p.m_fixed = M, p.max_contrib = g.max_contrib;
-  p.counters = reinterpret_cast<int*>(sc);
-  p.partials = reinterpret_cast<float*>(sc + off_part);
+  p.W = W, p.N = N, p.K = K, p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.cluster_size = g.cs, p.n_clusters = g.n_clusters;
+  p.xplanes = q.planes, p.x_ld = K, p.m_fixed = M;
   p.out = y, p.out_ld = N;
   GemmFn fn = gemm_fn(weight_dtype, ng, EPI_PLAIN);
   if (gemm_smem(weight_dtype, ng) > 48 * 1024 &&
       cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem(weight_dtype, ng)) != cudaSuccess)
     return LOOPSPEC_ECUDA;
-  cudaError_t e = launch_gemm(weight_dtype, ng, EPI_PLAIN, p, g.grid, st, false);
+  cudaError_t e = launch_gemm(weight_dtype, ng, EPI_PLAIN, p, st, false);
   return e == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
 }
 
