@@ -119,6 +119,22 @@ def run_kernel_only(args):
     ctx.close()
 
 
+def run_profile_pass(args):
+    """Prefill, then decode a few tokens and exit: the command profilers capture a steady-state pass from."""
+    import paper_2609_17184_b200 as ls
+    wl = W.WORKLOADS[args.workload]
+    shape = W.CONFIGS[wl.model]
+    weights = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed))
+    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
+                      max_seqs=1, max_ctx=wl.prompt_len + wl.decode_len + 16, max_prefill_rows=64)
+    ctx.prefill(W.make_prompt(shape.vocab, wl.prompt_len, seed=wl.prompt_seed))
+    ctx.decode(args.profile_pass)
+    st = ctx.stats()
+    print(json.dumps({"profile_pass": args.profile_pass, "passes": st["steps"], "rows_total": st["rows_total"],
+                      "launches_per_pass": ctx.launches_per_step()}))
+    ctx.close()
+
+
 def run_ours(args):
     import torch
     import paper_2609_17184_b200 as ls
@@ -364,11 +380,14 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--calibrated", action="store_true", help="also run the acceptance-calibrated variant")
     ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")
+    ap.add_argument("--profile-pass", type=int, default=0, help="prefill, decode this many tokens, exit (for profilers)")
     ap.add_argument("--rows", type=int, default=4)
     ap.add_argument("--iters", type=int, default=10)
     args = ap.parse_args()
     if args.kernel_only:
         return run_kernel_only(args)
+    if args.profile_pass:
+        return run_profile_pass(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -30,24 +30,22 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
   constexpr int LPP = D / 8;            // lanes per key position (8 bf16 = 16 bytes per lane)
   constexpr int PPW = 32 / LPP;         // positions per warp per load
   constexpr int PPR = PPW * (ATT_THREADS / 32);  // positions per round of the whole CTA
-  constexpr int ROUNDS = ATT_CHUNK / PPR;
+  constexpr int NPOS = ATT_CHUNK + MAX_SPEC;     // the last chunk of a row also carries its speculative slots
+  constexpr int ROUNDS = (NPOS + PPR - 1) / PPR;
   constexpr int PSTRIDE = D + 2;
 
-  __shared__ float s_score[G][ATT_CHUNK];
+  __shared__ float s_score[G][ROUNDS * PPR];
   __shared__ float s_red[ATT_THREADS / 32][G][D];
   __shared__ float s_stat[G][2];
-  __shared__ int s_slot[ATT_CHUNK];
   __shared__ int s_last;
 
-  pdl_launch_dependents();
-  pdl_wait();
-  const RowTable* tab = p.tab;
+  const RowTable* tab = p.tab;   // written before this pass started: safe to read ahead of the predecessor
   const int n_rows = tab->n_rows;
-  if (n_rows <= 0) return;
   const int HQ = p.n_q_heads * D;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int sub = lane / LPP, dl = lane % LPP;  // which position of the warp's group, which 8-dim slice
   const int total = tab->attn_items * p.n_kv_heads;
+  bool waited = false;
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     const int kvh = item % p.n_kv_heads;
@@ -56,19 +54,42 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
     while (row + 1 < n_rows && tab->chunk_start[row + 1] <= rc) ++row;
     const int chunk = rc - tab->chunk_start[row];
     const int n_chunks = tab->chunk_start[row + 1] - tab->chunk_start[row];
-    const int n_canon = tab->n_canon[row], n_spec = tab->n_spec[row];
-    const int n_canon_chunks = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK;
-    const bool spec_chunk = chunk >= n_canon_chunks;
+    const int n_canon = tab->n_canon[row];
     const int p0 = chunk * ATT_CHUNK;
-    const int n_here = spec_chunk ? n_spec : min(ATT_CHUNK, n_canon - p0);
-
-    __syncthreads();  // shared buffers of the previous item are free
-    if (tid < ATT_CHUNK) s_slot[tid] = tid < n_here ? (spec_chunk ? tab->spec_slot[row][tid] : p0 + tid) : 0;
+    const int n_can_here = min(ATT_CHUNK, n_canon - p0);
+    const int n_spec = (chunk == n_chunks - 1) ? tab->n_spec[row] : 0;
+    const int n_here = n_can_here + n_spec;
+    // positions below n_safe were cached by earlier passes; the others are written by this pass's QKV kernel
+    const int n_safe_can = min(n_can_here, max(0, tab->n_safe[row] - p0));
+    const int n_safe = (n_spec > 0) ? n_can_here + n_spec - 1 : n_safe_can;
 
     const size_t plane = (size_t)(tab->r[row] - 1) * p.kv_plane_stride;
     const size_t headbase = (size_t)(tab->seq[row] * p.n_kv_heads + kvh) * p.slots * D;
     const __nv_bfloat16* Kb = p.kv + plane + headbase;
     const __nv_bfloat16* Vb = p.kv + plane + p.kv_sel_stride + headbase;
+
+    auto slot_of = [&](int jpos) -> int { return jpos < n_can_here ? p0 + jpos : tab->spec_slot[row][jpos - n_can_here]; };
+    uint4 kreg[ROUNDS], vreg[ROUNDS];
+    auto load_kv = [&](int lo, int hi) {
+#pragma unroll
+      for (int rd = 0; rd < ROUNDS; ++rd) {
+        const int jpos = rd * PPR + warp * PPW + sub;
+        if (jpos >= lo && jpos < hi) {
+          const size_t off = (size_t)slot_of(jpos) * D + dl * 8;
+          kreg[rd] = *reinterpret_cast<const uint4*>(Kb + off);
+          vreg[rd] = *reinterpret_cast<const uint4*>(Vb + off);
+        }
+      }
+    };
+#pragma unroll
+    for (int rd = 0; rd < ROUNDS; ++rd) kreg[rd] = vreg[rd] = make_uint4(0, 0, 0, 0);
+    load_kv(0, n_safe);
+    if (!waited) {
+      pdl_launch_dependents();
+      pdl_wait();
+      waited = true;
+    }
+    load_kv(n_safe, n_here);
 
     float q[G][8];
 #pragma unroll
@@ -79,19 +100,12 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       q[gq][0] = a.x, q[gq][1] = a.y, q[gq][2] = a.z, q[gq][3] = a.w;
       q[gq][4] = b.x, q[gq][5] = b.y, q[gq][6] = b.z, q[gq][7] = b.w;
     }
-    __syncthreads();
+    __syncthreads();  // shared buffers of the previous item are free
 
     // ---- scores ------------------------------------------------------------------------------------
-    uint4 kreg[ROUNDS];
 #pragma unroll
     for (int rd = 0; rd < ROUNDS; ++rd) {
-      int j = rd * PPR + warp * PPW + sub;
-      kreg[rd] = make_uint4(0, 0, 0, 0);
-      if (j < n_here) kreg[rd] = *reinterpret_cast<const uint4*>(Kb + (size_t)s_slot[j] * D + dl * 8);
-    }
-#pragma unroll
-    for (int rd = 0; rd < ROUNDS; ++rd) {
-      int j = rd * PPR + warp * PPW + sub;
+      const int jpos = rd * PPR + warp * PPW + sub;
       const unsigned w[4] = {kreg[rd].x, kreg[rd].y, kreg[rd].z, kreg[rd].w};
       float kf[8];
 #pragma unroll
@@ -106,7 +120,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
         for (int i = 0; i < 8; ++i) s = fmaf(q[gq][i], kf[i], s);
 #pragma unroll
         for (int o = LPP / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (dl == 0) s_score[gq][j] = (j < n_here) ? s * p.scale : -INFINITY;
+        if (dl == 0) s_score[gq][jpos] = (jpos < n_here) ? s * p.scale : -INFINITY;
       }
     }
     __syncthreads();
@@ -114,12 +128,12 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
     // ---- chunk softmax statistics (one warp per query head, round robin) ----------------------------
     for (int gq = warp; gq < G; gq += ATT_THREADS / 32) {
       float m = -INFINITY;
-      for (int j = lane; j < ATT_CHUNK; j += 32) m = fmaxf(m, s_score[gq][j]);
+      for (int jj = lane; jj < ROUNDS * PPR; jj += 32) m = fmaxf(m, s_score[gq][jj]);
       m = warp_max(m);
       float l = 0.f;
-      for (int j = lane; j < ATT_CHUNK; j += 32) {
-        float e = (j < n_here) ? expf(s_score[gq][j] - m) : 0.f;
-        s_score[gq][j] = e;
+      for (int jj = lane; jj < ROUNDS * PPR; jj += 32) {
+        float e = (jj < n_here) ? expf(s_score[gq][jj] - m) : 0.f;
+        s_score[gq][jj] = e;
         l += e;
       }
       l = warp_sum(l);
@@ -135,14 +149,8 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       for (int i = 0; i < 8; ++i) o[gq][i] = 0.f;
 #pragma unroll
     for (int rd = 0; rd < ROUNDS; ++rd) {
-      int j = rd * PPR + warp * PPW + sub;
-      kreg[rd] = make_uint4(0, 0, 0, 0);
-      if (j < n_here) kreg[rd] = *reinterpret_cast<const uint4*>(Vb + (size_t)s_slot[j] * D + dl * 8);
-    }
-#pragma unroll
-    for (int rd = 0; rd < ROUNDS; ++rd) {
-      int j = rd * PPR + warp * PPW + sub;
-      const unsigned w[4] = {kreg[rd].x, kreg[rd].y, kreg[rd].z, kreg[rd].w};
+      const int jpos = rd * PPR + warp * PPW + sub;
+      const unsigned w[4] = {vreg[rd].x, vreg[rd].y, vreg[rd].z, vreg[rd].w};
       float vf[8];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -151,7 +159,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       }
 #pragma unroll
       for (int gq = 0; gq < G; ++gq) {
-        float pw = s_score[gq][j];
+        float pw = s_score[gq][jpos];
 #pragma unroll
         for (int i = 0; i < 8; ++i) o[gq][i] = fmaf(pw, vf[i], o[gq][i]);
       }
@@ -185,34 +193,55 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       float v = 0.f;
 #pragma unroll
       for (int w2 = 0; w2 < ATT_THREADS / 32; ++w2) v += s_red[w2][gq][dd];
-      mypart[gq * PSTRIDE + dd] = v;
+      __stcg(mypart + gq * PSTRIDE + dd, v);
     }
-    if (tid < G) mypart[tid * PSTRIDE + D] = s_stat[tid][0], mypart[tid * PSTRIDE + D + 1] = s_stat[tid][1];
-    __threadfence();
+    if (tid < G) __stcg(mypart + tid * PSTRIDE + D, s_stat[tid][0]), __stcg(mypart + tid * PSTRIDE + D + 1, s_stat[tid][1]);
     __syncthreads();
     if (tid == 0) {
+      __threadfence();
       int old = atomicAdd(p.counters + pair, 1);
       s_last = (old == n_chunks - 1);
+      __threadfence();
     }
     __syncthreads();
-    if (s_last) {
-      __threadfence();
+    if (s_last) {  // combine the chunks in ascending order
       const float* base = p.part + (size_t)pair * p.max_chunks * G * PSTRIDE;
       for (int idx = tid; idx < G * D; idx += ATT_THREADS) {
         int gq = idx / D, dd = idx % D;
         float m = -INFINITY;
-        for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, __ldcg(base + ((size_t)c * G + gq) * PSTRIDE + D));
+        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+          float mm[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) mm[u] = (c0 + u < n_chunks) ? __ldcg(base + ((size_t)(c0 + u) * G + gq) * PSTRIDE + D) : -INFINITY;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) m = fmaxf(m, mm[u]);
+        }
         float l = 0.f, acc = 0.f;
-        for (int c = 0; c < n_chunks; ++c) {
-          const float* pc = base + ((size_t)c * G + gq) * PSTRIDE;
-          float wgt = expf(__ldcg(pc + D) - m);
-          l = fmaf(__ldcg(pc + D + 1), wgt, l);
-          acc = fmaf(__ldcg(pc + dd), wgt, acc);
+        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+          float mc[8], lc[8], oc[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const bool ok = c0 + u < n_chunks;
+            const float* pc = base + ((size_t)(ok ? c0 + u : 0) * G + gq) * PSTRIDE;
+            mc[u] = ok ? __ldcg(pc + D) : -INFINITY;
+            lc[u] = ok ? __ldcg(pc + D + 1) : 0.f;
+            oc[u] = ok ? __ldcg(pc + dd) : 0.f;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            float wgt = expf(mc[u] - m);
+            l = fmaf(lc[u], wgt, l);
+            acc = fmaf(oc[u], wgt, acc);
+          }
         }
         store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, (kvh * G + gq) * D + dd, acc / l);
       }
       if (tid == 0) p.counters[pair] = 0;
     }
+  }
+  if (!waited) {
+    pdl_launch_dependents();
+    pdl_wait();
   }
 }
 

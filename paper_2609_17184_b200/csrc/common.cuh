@@ -26,6 +26,7 @@ struct RowTable {
   int kv_slot[MAX_ROWS];     // slot its K,V are written to
   int n_canon[MAX_ROWS];     // committed slots [0, n_canon) it attends to
   int n_spec[MAX_ROWS];      // speculative slots it attends to (its uncommitted ancestors and itself)
+  int n_safe[MAX_ROWS];      // committed slots [0, n_safe) were cached by earlier passes (not written in this one)
   int spec_slot[MAX_ROWS][MAX_SPEC];
   int hid_idx[MAX_ROWS];     // where its hidden state lives (updated in place)
   int readout[MAX_ROWS];     // RO_*

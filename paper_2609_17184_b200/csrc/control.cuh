@@ -97,6 +97,7 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       t.seq[i] = s, t.r[i] = r, t.pos[i] = nd.pos[o + n], t.node[i] = o + n, t.hid_idx[i] = o + n;
       t.kv_slot[i] = is_root ? nd.pos[o + n] : p.ctx_cap + n;
       t.n_canon[i] = nd.pos[o + rt] + 1;
+      t.n_safe[i] = is_root ? nd.pos[o + n] : t.n_canon[i];
       if (nd.pos[o + n] + 2 >= p.ctx_cap) *err = ERR_CTX;
       int chain[MAX_SPEC], len = 0;
       for (int a = n; a >= 0 && nd.parent[o + a] >= 0; a = nd.parent[o + a]) {
@@ -112,7 +113,7 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       t.readout[i] = ro, t.logit_idx[i] = li;
       if (ro) t.ro_rows[n_ro++] = i;
       t.chunk_start[i] = items;
-      items += (t.n_canon[i] + ATT_CHUNK - 1) / ATT_CHUNK + (len > 0 ? 1 : 0);
+      items += (t.n_canon[i] + ATT_CHUNK - 1) / ATT_CHUNK;
     }
   }
   t.chunk_start[n_rows] = items;
@@ -305,6 +306,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
       for (int i = 0; i < n; ++i) {
         int s = s_rowof[i], gn = s_emb[i][0], pos = p.nodes.pos[gn];
         t.seq[i] = s, t.r[i] = r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
+        t.n_safe[i] = pos;
         t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE;
         t.logit_idx[i] = p.p_logit_base + s, t.ro_rows[i] = i, t.chunk_start[i] = items;
         items += (pos + 1 + ATT_CHUNK - 1) / ATT_CHUNK;
@@ -339,6 +341,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
     for (int i = 0; i < p.count; ++i) {
       int pos = p.p0 + i;
       t.seq[i] = p.seq, t.r[i] = p.r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
+      t.n_safe[i] = p.p0;
       t.hid_idx[i] = p.hid_base + i, t.node[i] = -1;
       bool last = (p.r == p.R) && (pos == p.n_prompt - 1);
       t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;

@@ -117,14 +117,28 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
   for (int base = rank; base < n_cols; base += 2 * cs) {
     const int c = base + cs * half;
     const bool live = c < n_cols;
-    float v = 0.f;
-    if (live) {
-      for (int rk = 0; rk < cs; ++rk) {
-        const float* remote = cs > 1 ? cluster.map_shared_rank(tile, rk) : tile;
-        v += remote[c * TILE_LD + j];
-      }
-      v *= s_rstd[c];
+    // global operands of the epilogue are requested first so that their latency overlaps the remote reads
+    float h_old = 0.f, g_next = 1.f;
+    float* h_ptr = nullptr;
+    if (EPI == EPI_RESID && live) {
+      h_ptr = p.hid + (size_t)tab->hid_idx[c] * p.H + rb * RB_ROWS + j;
+      h_old = *h_ptr;
+      if (p.out_planes) g_next = p.gain_next[rb * RB_ROWS + j];
     }
+    float part[8];
+#pragma unroll
+    for (int rk = 0; rk < 8; ++rk) {
+      part[rk] = 0.f;
+      if (live && rk < cs) {
+        const float* remote = cs > 1 ? cluster.map_shared_rank(tile, rk) : tile;
+        part[rk] = remote[c * TILE_LD + j];
+      }
+    }
+    float v = part[0];
+#pragma unroll
+    for (int rk = 1; rk < 8; ++rk)
+      if (rk < cs) v += part[rk];  // rank order, the same for every launch
+    v *= live ? s_rstd[c] : 0.f;
     if (EPI == EPI_PLAIN || EPI == EPI_LOGITS) {
       const int n = rb * RB_ROWS + j;
       if (live && n < p.N) {
@@ -135,10 +149,9 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
       const int n = rb * RB_ROWS + j;
       float xn = 0.f;
       if (live) {
-        float* h = p.hid + (size_t)tab->hid_idx[c] * p.H + n;
-        xn = *h + v;
-        *h = xn;
-        if (p.out_planes) store_split(p.out_planes + (size_t)c * 3 * p.planes_ld, p.planes_ld, n, xn * p.gain_next[n]);
+        xn = h_old + v;
+        *h_ptr = xn;
+        if (p.out_planes) store_split(p.out_planes + (size_t)c * 3 * p.planes_ld, p.planes_ld, n, xn * g_next);
       }
       float ss = warp_sum(xn * xn);
       if (lane == 0) s_ss[half][hw] = ss;

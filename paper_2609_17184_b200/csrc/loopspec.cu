@@ -36,11 +36,22 @@ GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only) {
   int cs = std::max(1, slots / std::max(n_rb, 1));
   cs = std::max(cs, cs_min);
   cs = std::min(std::min(cs, 8), g.kpr);
-  if (pow2_only) {
+  auto pow2_at_least = [&](int v) {
     int q = 1;
-    while (q < cs) q <<= 1;
-    cs = std::min(std::min(q, 8), g.kpr);
-    while (cs & (cs - 1)) --cs;
+    while (q < v) q <<= 1;
+    q = std::min(std::min(q, 8), g.kpr);
+    while (q & (q - 1)) --q;
+    return q;
+  };
+  if (pow2_only || n_rb * cs_min > slots) {
+    cs = pow2_at_least(cs);  // several rounds of row blocks per cluster: measured best with power-of-two clusters
+  } else {
+    // equal k-ranges stream best: the largest cluster size up to `cs` that divides the k-blocks, if long enough
+    for (int v = cs; v >= std::max(cs_min, 1); --v)
+      if (g.kpr % v == 0) {
+        cs = v;
+        break;
+      }
   }
   g.cs = cs;
   int max_clusters = std::max(1, slots / cs);
@@ -144,7 +155,7 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
   d->n_sq = m->hidden / 128;
-  d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK + 1;
+  d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
   d->trace_cap = 4 * s->max_ctx + 64;
   d->Hq = m->n_q_heads * m->head_dim;
   d->Hkv = m->n_kv_heads * m->head_dim;
@@ -425,7 +436,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
-    if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 4), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
+    if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->stream, pdl))) return e;
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->stream, pdl))) return e;
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->stream, pdl))) return e;
@@ -612,7 +623,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->prefilled.assign(d.S, 0);
   const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / 128, (m->ffn + 63) / 64, m->hidden / 128, (m->vocab + 127) / 128};
   const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
-  for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], n_sm * kCtasPerSm, false);
+  int slots = n_sm * kCtasPerSm;
+  if (const char* env = getenv("LOOPSPEC_SLOTS")) slots = std::max(1, atoi(env));  // tuning aid
+  for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
   for (int ng : {c->ng_dec, c->ng_pf})
     if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
@@ -629,7 +642,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         GemmPlan& g = c->plan[i];
         if (v[i] < 1 || v[i] > 8) continue;
         g.cs = std::min(v[i], g.kpr);
-        int max_clusters = std::max(1, n_sm * kCtasPerSm / g.cs);
+        int max_clusters = std::max(1, slots / g.cs);
         int rounds = (g.n_rb + max_clusters - 1) / max_clusters;
         g.n_clusters = (g.n_rb + rounds - 1) / rounds, g.grid = g.n_clusters * g.cs;
       }
@@ -649,7 +662,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
     if (e != cudaSuccess || n_active < 1) {
       (void)cudaGetLastError();
-      g = plan_gemm(n_rbs[i], Ks[i], n_sm * kCtasPerSm, true);
+      g = plan_gemm(n_rbs[i], Ks[i], slots, true);
     }
   }
   auto bail = [&](int code, const char* what) {
@@ -975,7 +988,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   memset(&t, 0, sizeof t);
   t.n_rows = rows, t.n_readout = rows;
   for (int i = 0; i < rows; ++i) {
-    t.r[i] = 1, t.hid_idx[i] = c->d.S * c->d.NB + i, t.ro_rows[i] = i, t.readout[i] = RO_TARGET, t.n_canon[i] = 1;
+    t.r[i] = 1, t.hid_idx[i] = c->d.S * c->d.NB + i, t.ro_rows[i] = i, t.readout[i] = RO_TARGET, t.n_canon[i] = 1, t.n_safe[i] = 0;
     t.logit_idx[i] = c->d.p_logit_base, t.node[i] = -1, t.chunk_start[i] = i;
   }
   t.chunk_start[rows] = rows, t.attn_items = rows;
