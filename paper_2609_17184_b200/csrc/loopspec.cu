@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "control.cuh"
 #include "gemm.cuh"
+#include "pass.cuh"
 #include "select.cuh"
 
 using namespace ls;
@@ -65,7 +66,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -191,9 +192,14 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sumsq = take(MR * d.n_sq * 4);
   L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
+  // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
+  L.gpart = take((size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4 * MR * 128 * 4);
+  L.ptrs = take((size_t)m->n_recurrent * 10 * sizeof(void*));
   int G = m->n_q_heads / m->n_kv_heads;
   L.apart = take(MR * m->n_kv_heads * d.max_chunks * G * (m->head_dim + 2) * 4);
   L.acnt = take(MR * m->n_kv_heads * 4);
+  L.gcnt = take((size_t)((m->ffn + 63) / 64 + (d.Hq + 2 * d.Hkv) / 128 + 16) * 4);
+  L.bar = take(256);
   L.nodes = take((size_t)13 * MAX_NODES * 4);
   L.seqs = take((size_t)5 * MAX_ROWS * 4);
   L.ctr = take(sizeof(Counters));
@@ -238,7 +244,9 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false;
+  PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
+  int pass_grid = 0;
   int launches_per_step = 0;
   std::string err;
 
@@ -419,6 +427,23 @@ cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
 }
 
 
+using PassFn = void (*)(const PassParams);
+PassFn pass_fn(int d, int G) {
+  if (d == 128) return G == 1 ? pass_kernel<1, 128, 1> : pass_kernel<1, 128, 4>;
+  return G == 1 ? pass_kernel<1, 64, 1> : pass_kernel<1, 64, 4>;
+}
+
+cudaError_t launch_pass(loopspec_ctx* c, const PassParams& pp) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(c->pass_grid), cfg.blockDim = dim3(PASS_THREADS), cfg.dynamicSmemBytes = pass_smem_bytes(1), cfg.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they meet at grid barriers
+  at[0].val.cooperative = 1;
+  cfg.attrs = at, cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, pass_fn(c->m.head_dim, c->m.n_q_heads / c->m.n_kv_heads), pp);
+}
+
 cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
@@ -427,6 +452,14 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   cudaError_t e;
   if ((e = launch_prep(c, tab, false))) return e;
   if (n_launch) *n_launch += 1;
+  if (c->use_mega && ng == 1) {
+    if ((e = cudaMemsetAsync(c->ws + c->L.bar, 0, 4, c->stream))) return e;
+    PassParams pp = c->pass;
+    pp.tab = tab;
+    if ((e = launch_pass(c, pp))) return e;
+    if (n_launch) *n_launch += 1;
+    return cudaSuccess;
+  }
   for (int l = 0; l < m.n_recurrent; ++l) {
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->stream, pdl))) return e;
     AttnParams a;
@@ -532,7 +565,7 @@ int check_device_error(loopspec_ctx* c) {
   if (!e) return LOOPSPEC_OK;
   c->host_flags[HF_ERROR] = 0;
   return fail(c, LOOPSPEC_ECAPACITY, "device scheduler reported %s",
-              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : "speculative chain too deep");
+              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : e == 4 ? "a grid barrier timed out" : "speculative chain too deep");
 }
 
 int capture(loopspec_ctx* c, cudaGraphExec_t* out, bool vanilla) {
@@ -717,6 +750,55 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     }
     ok = ok && pack(c->lm_head, m->vocab, m->hidden);
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
+  }
+  // persistent pass kernel: available for bf16 weights when a decode pass carries at most 8 rows
+  if (m->weight_dtype == 1 && c->ng_dec == 1) {
+    PassFn fn = pass_fn(m->head_dim, m->n_q_heads / m->n_kv_heads);
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pass_smem_bytes(1)) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, PASS_THREADS, pass_smem_bytes(1)) == cudaSuccess && per_sm >= 1) {
+      c->pass_grid = n_sm * std::min(per_sm, 2);
+      std::vector<const void*> tabs((size_t)m->n_recurrent * 10);
+      for (int l = 0; l < m->n_recurrent; ++l) {
+        for (int i = 0; i < 4; ++i) tabs[(size_t)l * 4 + i] = c->packed[(size_t)l * 4 + i];
+        for (int i = 0; i < 6; ++i) tabs[(size_t)m->n_recurrent * 4 + (size_t)l * 6 + i] = c->layers[(size_t)l * 6 + i];
+      }
+      if (cudaMemcpyAsync(c->ws + L.ptrs, tabs.data(), tabs.size() * sizeof(void*), cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+          cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return bail(LOOPSPEC_ECUDA, "pointer table upload");
+      PassParams& q = c->pass;
+      memset(&q, 0, sizeof q);
+      q.L = m->n_recurrent;
+      q.wpacked = c->at<const void*>(L.ptrs), q.layer_w = c->at<const void*>(L.ptrs) + (size_t)m->n_recurrent * 4;
+      q.H = m->hidden, q.Hq = d.Hq, q.Hkv = d.Hkv, q.F = m->ffn, q.n_q_heads = m->n_q_heads, q.n_kv_heads = m->n_kv_heads;
+      q.head_dim = m->head_dim, q.slots = d.slots, q.eps = m->rms_eps, q.scale = 1.0f / sqrtf((float)m->head_dim);
+      q.hid = c->at<float>(L.hid), q.xplanes = c->at<__nv_bfloat16>(L.xplanes), q.aplanes = c->at<__nv_bfloat16>(L.aplanes);
+      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq), q.n_sq = d.n_sq;
+      q.kv = c->at<__nv_bfloat16>(L.kv), q.kv_layer_stride = c->kv_layer_stride(), q.kv_plane_stride = c->kv_plane_stride();
+      q.kv_sel_stride = c->kv_sel_stride(), q.rope = c->at<float2>(L.rope);
+      q.gpart = c->at<float>(L.gpart), q.gcnt = c->at<int>(L.gcnt), q.apart = c->at<float>(L.apart), q.acnt = c->at<int>(L.acnt);
+      q.max_chunks = d.max_chunks, q.bar = c->at<unsigned>(L.bar), q.err = c->host_flags_dev + HF_ERROR;
+      const int Ns[4] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden};
+      bool fits = true;
+      for (int i = 0; i < 4; ++i) {
+        q.n_rb[i] = n_rbs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.N[i] = Ns[i], q.K[i] = Ks[i];
+        int total = q.n_rb[i] * q.kpr[i];
+        q.upc[i] = (total + c->pass_grid - 1) / c->pass_grid;
+        int mc = 1;
+        for (int rb = 0; rb < q.n_rb[i]; ++rb)
+          mc = std::max(mc, ((rb + 1) * q.kpr[i] - 1) / q.upc[i] - (rb * q.kpr[i]) / q.upc[i] + 1);
+        q.max_contrib[i] = mc;
+        if ((size_t)q.n_rb[i] * mc > (size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4) fits = false;
+      }
+      // measured slower than the chain of cluster kernels (its stage hand-over through global partials and a
+      // grid barrier costs more than a kernel boundary), so it is opt-in: LOOPSPEC_MEGA=1
+      c->use_mega = false;
+      if (const char* env = getenv("LOOPSPEC_MEGA")) c->use_mega = fits && env[0] == '1';
+      if (getenv("LOOPSPEC_DBG")) {  // tuning aid: timestamps land in the unused tail of the partial buffer
+        q.dbg = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + (1 << 20);
+        fprintf(stderr, "LOOPSPEC_DBG offset %zu\n", L.gpart + ((size_t)8 << 20));
+      }
+    }
   }
   // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
   if (cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
@@ -974,7 +1056,7 @@ int loopspec_debug_logits(loopspec_ctx* c, int32_t seq, int32_t which, float* ou
 
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
-  *out = c->m.n_recurrent * 5 + 6;
+  *out = c->use_mega ? 8 : c->m.n_recurrent * 5 + 6;
   return LOOPSPEC_OK;
 }
 

@@ -1,0 +1,92 @@
+"""Full-size parity on the Ouro-1.4B-shaped model (BASELINE config 1), in the launch configuration bench.py times.
+
+The oracle cannot decode 512 tokens of a 1.4B model in test time, so:
+  * the first tokens of the run (greedy and temperature 1) are compared with values the oracle computed once
+    (tests/golden/ouro_1p4b_oracle.json, written by tests/golden/make_ouro_golden.py, which calls only oracle/);
+  * the whole 512-token run is checked through properties that hold at any size: greedy LoopSpec == greedy
+    vanilla decoding on the device, the commit-gap schedule, and the counters' identities.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import workloads as W
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "ouro_1p4b_oracle.json")
+
+
+@pytest.fixture(scope="module")
+def setup():
+    import paper_2609_17184_b200 as ls
+    wl = W.WORKLOADS["ouro_1p4b"]
+    shape = W.CONFIGS[wl.model]
+    weights = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed))
+    prompt = W.make_prompt(shape.vocab, wl.prompt_len, seed=wl.prompt_seed)
+    return ls, wl, shape, weights, prompt, json.load(open(GOLD))
+
+
+def make(setup, T):
+    ls, wl, shape, weights, prompt, gold = setup
+    return ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=T, seed=wl.sample_seed, gate=wl.gate, max_seqs=1,
+                       max_ctx=wl.prompt_len + wl.decode_len + 16, max_prefill_rows=64)
+
+
+@pytest.mark.parametrize("run", ["greedy", "sampled_T1"])
+def test_first_tokens_match_the_oracle(setup, run):
+    ls, wl, shape, weights, prompt, gold = setup
+    g = gold["runs"][run]
+    n = gold["n_tokens"]
+    ctx = make(setup, g["temperature"])
+    assert ctx.prefill(prompt) == g["first_token"]
+    z = ctx.debug_logits(0, 0)
+    assert int(np.argmax(z)) == g["first_logits_argmax"]
+    for i, v in g["first_logits_probe"].items():
+        assert abs(z[int(i)] - v) <= 3e-2 + 2e-2 * abs(v)
+        assert abs(z[int(i)] - v) < 5e-3
+    out = ctx.decode(n)[0].tolist()
+    assert out == g["tokens"], ("oracle min margin", g["min_margin"])
+    commits = ctx.commits(0)
+    assert [[c["source"], c["gate_open"], c["step"]] for c in commits] == g["commits"]
+    assert ctx.row_trace().tolist() == g["rows_per_step"]
+    st = ctx.stats()
+    for k, v in g["stats"].items():
+        if k != "gamma":
+            assert st[k] == v, k
+    z = ctx.debug_logits(0, 0)
+    for i, v in g["last_verify_logits_probe"].items():
+        assert abs(z[int(i)] - v) < 5e-3
+    if run == "greedy":
+        ctx.prefill(prompt)
+        assert ctx.vanilla_decode(n)[0].tolist() == gold["vanilla_greedy_tokens"] == g["tokens"]
+    ctx.close()
+
+
+def test_full_run_properties(setup):
+    ls, wl, shape, weights, prompt, gold = setup
+    n, R = wl.decode_len, shape.R
+    ctx = make(setup, 0.0)
+    ctx.prefill(prompt)
+    out = ctx.decode(n)[0].tolist()
+    commits, st, trace = ctx.commits(0), ctx.stats(), ctx.row_trace()
+    assert out[: gold["n_tokens"]] == gold["runs"]["greedy"]["tokens"]
+    # schedule: first commit after R passes, then d1 / d2 / R passes after a first / second / resampled commit
+    cost = {1: wl.d1, 2: wl.d2, 3: R}
+    steps = [c["step"] for c in commits]
+    assert steps[0] == R and list(np.diff(steps)) == [cost[c["source"]] for c in commits[:-1]]
+    assert st["n_decode"] == n == st["n_accept1"] + st["n_accept2"] + st["n_restart"]
+    assert st["steps"] == steps[-1] == len(trace) and st["rows_total"] == int(trace.sum()) and st["rows_max"] == int(trace.max())
+    assert st["rows_max"] <= ls.max_branches(R, wl.d1, wl.d2)
+    den = st["n_accept1"] * wl.d1 + st["n_accept2"] * wl.d2 + st["n_restart"] * R
+    assert abs(st["gamma"] - n * R / den) < 1e-12
+    # losslessness at full size: the pipelined greedy stream is the vanilla all-R stream
+    ctx.prefill(prompt)
+    assert ctx.vanilla_decode(n)[0].tolist() == out
+    # and the run is reproducible bit for bit (logits of the last verification)
+    z1 = ctx.debug_logits(0, 0).copy()
+    ctx.prefill(prompt)
+    ctx.vanilla_decode(n)
+    assert np.array_equal(z1.view(np.uint32), ctx.debug_logits(0, 0).view(np.uint32))
+    ctx.close()
