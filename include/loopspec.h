@@ -168,6 +168,24 @@ size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N,
                        int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* The same linear map for callers that cannot allocate device memory at all.  (The paper has no counterpart;
+ * this is a packaging convenience.)  Two kinds of caller are meant: a serving process whose allocator has reserved
+ * the whole device up front, so that a later cudaMalloc -- theirs or ours -- fails or fragments the pool; and a
+ * latency-critical thread for which cudaMalloc/cudaFree are off limits because they synchronise the device and stall
+ * every other stream.  Such callers pass only inputs and the output; the scratch that loopspec_op_linear wants lives
+ * in a fixed 16 MiB array inside the library's device image (every GPU that loads the library carries it until the
+ * process exits).  The call allocates nothing and frees nothing.
+ *   - Sizes: loopspec_linear_scratch_bytes(M, N, K) must not exceed 16 MiB (roughly N*K <= 8M bf16 weights);
+ *     larger requests return LOOPSPEC_ECAPACITY and do nothing.  Bad shapes return LOOPSPEC_EINVAL.
+ *   - The first call on each device looks up the array's device address (with that device current); make that
+ *     first call outside any stream capture.  Later calls only launch kernels on cuda_stream.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left there.  Nothing in
+ *     it has to start at zero: every call overwrites the part it reads.  Two calls that overlap on the GPU (different
+ *     streams, or threads racing on one stream's ordering) overwrite each other's scratch and give wrong results:
+ *     serialise them. */
+int loopspec_op_linear_static(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N,
+                              int32_t K, void* cuda_stream);
+
 const char* loopspec_last_error(loopspec_ctx*);
 int loopspec_destroy(loopspec_ctx*);
 

@@ -13,6 +13,7 @@ EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loo
            "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
            "loopspec_launches_per_step", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
+           "loopspec_op_linear_static",
            "loopspec_last_error", "loopspec_destroy"]
 
 STATUS = {0: "OK", -1: "EINVAL", -2: "ESTATE", -3: "ECAPACITY", -4: "ECUDA", -5: "ETIMEOUT", -6: "EUNSUPPORTED"}
@@ -82,6 +83,7 @@ def _load():
     lib.loopspec_linear_scratch_bytes.restype = C.c_size_t
     lib.loopspec_linear_scratch_bytes.argtypes = [I, I, I]
     lib.loopspec_op_linear.argtypes = [V, I, V, V, I, I, I, V, C.c_size_t, V]
+    lib.loopspec_op_linear_static.argtypes = [V, I, V, V, I, I, I, V]
     lib.loopspec_last_error.restype = C.c_char_p
     lib.loopspec_last_error.argtypes = [V]
     lib.loopspec_destroy.argtypes = [V]
@@ -137,6 +139,20 @@ def linear(W, x, scratch=None):
                                 scratch.data_ptr(), scratch.numel(), torch.cuda.current_stream().cuda_stream)
     if rc:
         raise LoopSpecError(rc)
+    return y
+
+
+def linear_static(W, x):
+    """y = x @ W.T like `linear`, but through the entry point that needs no scratch buffer from the caller: for
+    processes that may not allocate device memory while serving.  Only the output tensor is created here."""
+    import torch
+    M, K = x.shape
+    N = W.shape[0]
+    y = torch.empty(M, N, dtype=torch.float32, device=x.device)
+    rc = lib.loopspec_op_linear_static(W.data_ptr(), 1 if W.dtype == torch.bfloat16 else 0, x.data_ptr(), y.data_ptr(), M, N, K,
+                                       torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise LoopSpecError(rc, "op_linear_static")
     return y
 
 

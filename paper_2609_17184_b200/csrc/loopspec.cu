@@ -1143,4 +1143,29 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
   return e == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
 }
 
+// ---- linear map without any caller- or library-side allocation ---------------------------------------------
+// Scratch for loopspec_op_linear_static: one fixed array in the library's device image.  Host code may only use
+// the symbol through cudaGetSymbolAddress; the address is looked up once per device and cached.
+#define LOOPSPEC_STATIC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[LOOPSPEC_STATIC_SCRATCH_BYTES];
+
+int loopspec_op_linear_static(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N, int32_t K,
+                              void* cuda_stream) {
+  static void* scratch_of_device[64] = {nullptr};
+  size_t need = loopspec_linear_scratch_bytes(M, N, K);
+  if (!need) return LOOPSPEC_EINVAL;
+  if (need > LOOPSPEC_STATIC_SCRATCH_BYTES) return LOOPSPEC_ECAPACITY;  // beyond the built-in scratch: use loopspec_op_linear
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOOPSPEC_ECUDA;
+  void* ptr = scratch_of_device[dev];
+  if (!ptr) {  // first call on this device (it is the current one): resolve the array's device address
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+      (void)cudaGetLastError();
+      return LOOPSPEC_ECUDA;
+    }
+    scratch_of_device[dev] = ptr;
+  }
+  return loopspec_op_linear(W, weight_dtype, x, y, M, N, K, ptr, LOOPSPEC_STATIC_SCRATCH_BYTES, cuda_stream);
+}
+
 }  // extern "C"
