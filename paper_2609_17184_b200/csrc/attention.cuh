@@ -23,6 +23,8 @@ struct AttnParams {
   float* part;                // [row][n_kv][max_chunks][G][D + 2]
   int max_chunks;
   int* counters;              // [row][n_kv]
+  const void* pf_ptr;         // region to prefetch into L2 for a later kernel of the chain (may be null)
+  long long pf_bytes;
 };
 
 template <int D, int G>
@@ -39,6 +41,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
   __shared__ float s_stat[G][2];
   __shared__ int s_last;
 
+  if (threadIdx.x == 0) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
   const RowTable* tab = p.tab;   // written before this pass started: safe to read ahead of the predecessor
   const int n_rows = tab->n_rows;
   const int HQ = p.n_q_heads * D;

@@ -32,8 +32,10 @@ constexpr int MAX_XCH_BLOCKS = 24;  // k-blocks of activations one CTA keeps sta
 
 __host__ __device__ constexpr int xchunk_kblocks(int NG) { return MAX_XCH_BLOCKS / NG; }
 __host__ __device__ constexpr int xbuf_uint4(int NG) { return 3 * xchunk_kblocks(NG) * 8 * NG * 4; }
+// partial columns received from the cluster's ranks: [rank][owned column][128 rows]
+__host__ __device__ constexpr int recv_floats(int NG) { return (8 * NG + 7) * RB_ROWS; }
 __host__ __device__ constexpr int gemm_smem_bytes(int NG) {
-  return RING * 2 * GEMM_THREADS * 16 + xbuf_uint4(NG) * 16 + 8 * NG * TILE_LD * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
+  return RING * 2 * GEMM_THREADS * 16 + xbuf_uint4(NG) * 16 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
 }
 
 struct GemmParams {
@@ -67,6 +69,9 @@ struct GemmParams {
   const float2* rope;     // [pos][d/2] (cos, sin)
   float* logits;          // LOGITS: [logit_idx][V]
   int F;                  // SWIGLU: ffn width
+  const void* pf_ptr;     // region to prefetch into L2 for a later kernel of the chain (may be null)
+  long long pf_bytes;
+  long long* dbg;         // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
 };
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
@@ -105,19 +110,19 @@ __device__ __forceinline__ void gemm_krange(int kpr, int cs, int rank, int& lo, 
   hi = lo + q + (rank < r ? 1 : 0);
 }
 
-// ---- the cluster's partial tiles are complete: sum them in rank order and finish this CTA's columns ------
-// Column c of row block rb is finished by rank (c mod cluster size); threads 0..127 take one column, threads
-// 128..255 the next one of this rank, one output row each.
+// ---- every rank has pushed its partial columns into the owners' receive buffers: sum them in rank order and
+// finish this CTA's columns.  Column c of row block rb is finished by rank (c mod cluster size); threads 0..127
+// take one column, threads 128..255 the next one of this rank, one output row each.
 template <int EPI>
-__device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, float* tile,
-                                                     float* colbuf, const float* s_rstd, cg::cluster_group& cluster) {
+__device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, const float* recv,
+                                                     int own_max, float* colbuf, const float* s_rstd, int rank) {
   const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
-  const int cs = p.cluster_size, rank = (int)cluster.block_rank();
+  const int cs = p.cluster_size;
   __shared__ float s_ss[2][4];
   for (int base = rank; base < n_cols; base += 2 * cs) {
     const int c = base + cs * half;
     const bool live = c < n_cols;
-    // global operands of the epilogue are requested first so that their latency overlaps the remote reads
+    // global operands of the epilogue are requested first so that their latency overlaps the summation
     float h_old = 0.f, g_next = 1.f;
     float* h_ptr = nullptr;
     if (EPI == EPI_RESID && live) {
@@ -125,20 +130,13 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
       h_old = *h_ptr;
       if (p.out_planes) g_next = p.gain_next[rb * RB_ROWS + j];
     }
-    float part[8];
-#pragma unroll
-    for (int rk = 0; rk < 8; ++rk) {
-      part[rk] = 0.f;
-      if (live && rk < cs) {
-        const float* remote = cs > 1 ? cluster.map_shared_rank(tile, rk) : tile;
-        part[rk] = remote[c * TILE_LD + j];
-      }
+    float v = 0.f;
+    if (live) {
+      const float* src = recv + (size_t)(c / cs) * RB_ROWS + j;
+      v = src[0];
+      for (int rk = 1; rk < cs; ++rk) v += src[(size_t)rk * own_max * RB_ROWS];  // rank order, the same for every launch
+      v *= s_rstd[c];
     }
-    float v = part[0];
-#pragma unroll
-    for (int rk = 1; rk < 8; ++rk)
-      if (rk < cs) v += part[rk];  // rank order, the same for every launch
-    v *= live ? s_rstd[c] : 0.f;
     if (EPI == EPI_PLAIN || EPI == EPI_LOGITS) {
       const int n = rb * RB_ROWS + j;
       if (live && n < p.N) {
@@ -214,19 +212,25 @@ __device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float
   }
 }
 
-// write this thread's accumulator fragments (rows warp*16+g / +8, columns n*8+2t / +1) into the partial tile
+// push this thread's accumulator fragments (rows warp*16+g / +8, columns n*8+2t / +1) into the receive buffers of
+// the ranks that own the columns (distributed shared memory stores; made visible by the cluster barrier)
 template <int NG>
-__device__ __forceinline__ void gemm_store_tile(const float (&acc)[NG][4], float* tile) {
+__device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float* recv, int own_max, int n_cols, int cs, int rank,
+                                               cg::cluster_group& cluster) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int rl = warp * 16 + g;
 #pragma unroll
-  for (int n = 0; n < NG; ++n) {
-    const int c0 = n * 8 + 2 * t;
-    tile[c0 * TILE_LD + rl] = acc[n][0];
-    tile[(c0 + 1) * TILE_LD + rl] = acc[n][1];
-    tile[c0 * TILE_LD + rl + 8] = acc[n][2];
-    tile[(c0 + 1) * TILE_LD + rl + 8] = acc[n][3];
-  }
+  for (int n = 0; n < NG; ++n)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int c = n * 8 + 2 * t + e;
+      if (c < n_cols) {
+        const int owner = c % cs, slot = c / cs;
+        float* dst = (cs > 1 ? cluster.map_shared_rank(recv, owner) : recv) + ((size_t)rank * own_max + slot) * RB_ROWS + rl;
+        dst[0] = acc[n][e];
+        dst[8] = acc[n][2 + e];
+      }
+    }
 }
 
 // ======================================= bf16 weights: tensor cores ========================================
@@ -240,13 +244,19 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);            // [RING][2][256], slot of thread tid only
   uint4* xbuf = ring + RING * 2 * GEMM_THREADS;                // [3][XCH][NTOK][4]
-  float* tile = reinterpret_cast<float*>(xbuf + xbuf_uint4(NG));  // [NTOK][TILE_LD]
-  float* colbuf = tile + NTOK * TILE_LD;                       // [2][128]
+  float* recv = reinterpret_cast<float*>(xbuf + xbuf_uint4(NG));  // [cs][own_max][128]
+  float* colbuf = recv + recv_floats(NG);                      // [2][128]
   float* s_rstd = colbuf + 2 * RB_ROWS;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int cs = p.cluster_size, rank = (int)cluster.block_rank(), cid = blockIdx.x / cs;
+  const int own_max = (NTOK + cs - 1) / cs;
+  int dbg_n = 0;
+  auto stamp = [&]() {
+    if (p.dbg && blockIdx.x == 0 && tid == 0) p.dbg[dbg_n++] = clock64();
+  };
+  stamp();
   const int kpr = p.kb_per_rb;
   int kb_lo, kb_hi;
   gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
@@ -256,74 +266,85 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
 
   // ---- weight ring: issue side.  The weights are stored tile-major (see pack_weights_kernel): the 1 KB a warp
   // consumes per unit is contiguous and consecutive k-blocks of a 16-row tile follow each other, so every warp
-  // streams one contiguous region and every request covers whole 128-byte lines.
-  int i_rb = cid, i_kb = kb_lo, i_cnt = 0;
+  // streams one contiguous region and every request covers whole 128-byte lines.  The loop is kept to a few
+  // instructions per unit: shared-memory addresses are 32-bit registers advanced by constants.
+  constexpr unsigned SLOT_BYTES = 2 * GEMM_THREADS * 16, RING_MASK = RING * SLOT_BYTES - 1, HI_OFF = GEMM_THREADS * 16;
+  static_assert((RING & (RING - 1)) == 0, "ring depth must be a power of two");
+  const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring) + tid * 16;
   const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
-  const __nv_bfloat16* i_ptr = Wb;
-  bool i_ok = false;
+  const char* i_ptr = reinterpret_cast<const char*>(Wb);
+  unsigned i_slot = 0;
+  int i_rb = cid, i_left = upt, i_tasks = n_tasks, i_size = 0;
   auto i_setup = [&]() {
     int r0 = gemm_row0<EPI>(p, i_rb, warp);
-    i_ok = r0 >= 0;
-    i_ptr = Wb + (i_ok ? ((size_t)(r0 >> 4) * kpr + i_kb) * 512 : 0) + lane * 8;
+    i_size = r0 >= 0 ? 16 : 0;  // rows beyond the matrix: zero-fill, nothing is read
+    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)(r0 >= 0 ? (r0 >> 4) : 0) * kpr + kb_lo) * 512 + lane * 8);
   };
   i_setup();
   auto issue_unit = [&]() {
-    if (i_cnt < n_units) {
-      uint4* slot = ring + (i_cnt & (RING - 1)) * 2 * GEMM_THREADS + tid;
-      cp_async16(slot, i_ok ? i_ptr : Wb, i_ok);
-      cp_async16(slot + GEMM_THREADS, i_ok ? i_ptr + 256 : Wb, i_ok);
-      ++i_cnt, i_ptr += 512;
-      if (++i_kb == kb_hi) i_kb = kb_lo, i_rb += p.n_clusters, i_setup();
+    if (i_tasks > 0) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(ring_s + i_slot), "l"(i_ptr), "r"(i_size) : "memory");
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(ring_s + i_slot + HI_OFF), "l"(i_ptr + 512), "r"(i_size)
+                   : "memory");
+      i_ptr += 1024;
+      i_slot = (i_slot + SLOT_BYTES) & RING_MASK;
+      if (--i_left == 0) {
+        i_left = upt, i_rb += p.n_clusters;
+        if (--i_tasks > 0) i_setup();
+      }
     }
     cp_async_commit();
   };
 #pragma unroll
   for (int s = 0; s < RING - 1; ++s) issue_unit();
 
-  // the weights above are constants; everything below reads what earlier kernels of the pass produced
-  pdl_launch_dependents();
-  pdl_wait();
-
-  // ---- activations of this CTA's k-range: piece idx -> (plane s, k-block kbl, column c, quarter tt) ---------
-  // Columns beyond the live rows may hold stale values: every column is an independent dot product and the
-  // epilogue never reads them.
-  uint4 xr[PPT];
-  auto x_fetch = [&](int kb0, int nkb) {
-#pragma unroll
-    for (int i = 0; i < PPT; ++i) {
-      const int idx = tid + i * GEMM_THREADS;
-      const int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % XCH, s = r / XCH;
-      const int k = (kb0 + kbl) * 32 + tt * 8;
-      xr[i] = make_uint4(0, 0, 0, 0);
-      if (idx < PIECES && kbl < nkb && k < p.K)
-        xr[i] = *reinterpret_cast<const uint4*>(p.xplanes + ((size_t)c * 3 + s) * p.x_ld + k);
-    }
-  };
-  auto x_store = [&]() {
-#pragma unroll
-    for (int i = 0; i < PPT; ++i) {
-      const int idx = tid + i * GEMM_THREADS;
-      if (idx < PIECES) xbuf[idx] = xr[i];   // [s][kbl][c][tt] is exactly the piece order
-    }
-  };
-  const bool one_chunk = upt <= XCH;  // the whole k-range stays staged for every row block of this CTA
-  x_fetch(kb_lo, min(XCH, upt));
-
+  // the row table was written before this pass started, so the live row count can be read ahead of the predecessor
   const RowTable* tab = p.tab;
   int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
   if (n_cols > NTOK) n_cols = NTOK;
+  // the weights above are constants; everything below reads what earlier kernels of the pass produced
+  stamp();
+  if (tid == GEMM_THREADS - 1) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
+  pdl_launch_dependents();
+  pdl_wait();
+  stamp();
   if (n_cols <= 0) {  // uniform over the cluster: nobody reaches a cluster barrier
     cp_async_wait<0>();
     return;
   }
+
+  // ---- activations of this CTA's k-range, copied asynchronously into MMA-fragment order: piece idx -> (plane s,
+  // k-block kbl, column c, quarter tt).  Columns beyond the live rows are zero-filled without being read.
+  auto x_stage = [&](int kb0, int nkb) {
+#pragma unroll
+    for (int i = 0; i < PPT; ++i) {
+      const int idx = tid + i * GEMM_THREADS;
+      if (idx < PIECES) {
+        const int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % XCH, s = r / XCH;
+        const int k = (kb0 + kbl) * 32 + tt * 8;
+        const bool ok = kbl < nkb && k < p.K && c < n_cols;
+        cp_async16(xbuf + idx, ok ? p.xplanes + ((size_t)c * 3 + s) * p.x_ld + k : p.xplanes, ok);
+      }
+    }
+    cp_async_commit();
+  };
+  const bool one_chunk = upt <= XCH;  // the whole k-range stays staged for every row block of this CTA
+  x_stage(kb_lo, min(XCH, upt));
   gemm_rstd(p, n_cols, s_rstd);
-  x_store();
+  cp_async_wait<0>();
   __syncthreads();
+  stamp();
 
   float acc[3][NG][4];  // one chain per split term, the same for every NG: a row's bits must not depend on
                         // how many rows share the pass
-  const uint4* xs = xbuf + g * 4 + t;
-  int j = 0;
+  const unsigned xs_s = (unsigned)__cvta_generic_to_shared(xbuf) + (g * 4 + t) * 16;
+  constexpr unsigned X_KB = NTOK * 64, X_PLANE = XCH * NTOK * 64;  // bytes per k-block / per plane in xbuf
+  unsigned c_slot = 0;
+  auto lds128 = [](unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+  };
   for (int task = 0; task < n_tasks; ++task) {
     const int rb = cid + task * p.n_clusters;
     const bool warp_valid = gemm_row0<EPI>(p, rb, warp) >= 0;
@@ -337,26 +358,28 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
       const int nkb = min(XCH, upt - ck);
       if (!one_chunk) {  // wide passes (prefill): restage the activations chunk by chunk
         __syncthreads();
-        x_fetch(kb_lo + ck, nkb);
-        x_store();
+        x_stage(kb_lo + ck, nkb);
+        cp_async_wait<0>();
         __syncthreads();
       }
-      for (int kbl = 0; kbl < nkb; ++kbl, ++j) {
+      unsigned xk = xs_s;
+      for (int kbl = 0; kbl < nkb; ++kbl) {
         issue_unit();
         cp_async_wait<RING - 1>();
         if (warp_valid) {
-          const uint4* slot = ring + (j & (RING - 1)) * 2 * GEMM_THREADS + tid;
-          const uint4 a_lo = slot[0], a_hi = slot[GEMM_THREADS];
+          const uint4 a_lo = lds128(ring_s + c_slot), a_hi = lds128(ring_s + c_slot + HI_OFF);
 #pragma unroll
           for (int s = 0; s < 3; ++s) {
 #pragma unroll
             for (int n = 0; n < NG; ++n) {
-              const uint4 b = xs[((s * XCH + kbl) * NTOK + n * 8) * 4];
+              const uint4 b = lds128(xk + s * X_PLANE + n * 512);
               mma_bf16(acc[s][n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
               mma_bf16(acc[s][n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
             }
           }
         }
+        c_slot = (c_slot + SLOT_BYTES) & RING_MASK;
+        xk += X_KB;
       }
     }
     // fold the chains in fixed order, hi + (mid + lo), and publish this CTA's partial tile
@@ -365,10 +388,13 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
     for (int n = 0; n < NG; ++n)
 #pragma unroll
       for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
-    gemm_store_tile<NG>(tot, tile);
+    stamp();
+    gemm_push_tile<NG>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
-    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, tile, colbuf, s_rstd, cluster);
-    cluster.sync();  // nobody overwrites (or leaves with) a tile another rank is still reading
+    stamp();
+    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+    stamp();
+    if (task + 1 < n_tasks) cluster.sync();  // the owners are done with the receive buffer before it is refilled
   }
   cp_async_wait<0>();
 }
@@ -382,8 +408,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   constexpr int XCH = 4;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* xf = reinterpret_cast<float*>(smem_raw);              // [XCH][NTOK][32]
-  float* tile = xf + XCH * NTOK * 32;                          // [NTOK][TILE_LD]
-  float* colbuf = tile + NTOK * TILE_LD;
+  float* recv = xf + XCH * NTOK * 32;                          // [cs][own_max][128]
+  float* colbuf = recv + recv_floats(NG);
   float* s_rstd = colbuf + 2 * RB_ROWS;
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -394,6 +420,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
   const int upt = kb_hi - kb_lo;
   const int n_tasks = (p.n_rb - cid + p.n_clusters - 1) / p.n_clusters;
+  const int own_max = (NTOK + cs - 1) / cs;
   pdl_launch_dependents();
   pdl_wait();
   const RowTable* tab = p.tab;
@@ -463,14 +490,14 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
           if (c == 2 * t) tot[n][2 * h] = v;
           if (c == 2 * t + 1) tot[n][2 * h + 1] = v;
         }
-    gemm_store_tile<NG>(tot, tile);
+    gemm_push_tile<NG>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
-    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, tile, colbuf, s_rstd, cluster);
-    cluster.sync();
+    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+    if (task + 1 < n_tasks) cluster.sync();
   }
 }
 __host__ __device__ constexpr int gemm_f32_smem_bytes(int NG) {
-  return 4 * 8 * NG * 32 * 4 + 8 * NG * TILE_LD * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
+  return 4 * 8 * NG * 32 * 4 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
 }
 
 // ---- one-time repacking of a bf16 weight matrix [N][K] into the tile-major streaming layout ----------------

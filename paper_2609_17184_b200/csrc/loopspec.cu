@@ -244,7 +244,7 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = true;
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
   int launches_per_step = 0;
@@ -417,6 +417,17 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   return p;
 }
 
+// the region a kernel of the chain asks L2 to fetch for a later one: the packed weights of GEMM `which`, layer l
+void prefetch_target(loopspec_ctx* c, int which, int l, const void** ptr, long long* bytes) {
+  *ptr = nullptr, *bytes = 0;
+  if (c->packed.empty() || !c->use_l2pf || l >= c->m.n_recurrent) return;
+  const Derived& d = c->d;
+  const int Ns[4] = {d.Hq + 2 * d.Hkv, c->m.hidden, 2 * c->m.ffn, c->m.hidden};
+  const int Ks[4] = {c->m.hidden, d.Hq, c->m.hidden, c->m.ffn};
+  *ptr = c->packed[4 * l + which];
+  *bytes = (long long)packed_bytes(Ns[which], Ks[which]);
+}
+
 cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
   PrepParams q;
   memset(&q, 0, sizeof q);
@@ -461,18 +472,26 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     return cudaSuccess;
   }
   for (int l = 0; l < m.n_recurrent; ++l) {
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gemm_params(c, G_QKV, l, tab), c->stream, pdl))) return e;
+    GemmParams gq = gemm_params(c, G_QKV, l, tab);
+    prefetch_target(c, G_O, l, &gq.pf_ptr, &gq.pf_bytes);          // QKV runs: fetch W_o
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
     AttnParams a;
+    memset(&a, 0, sizeof a);
     a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
     a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
     a.kv_plane_stride = c->kv_plane_stride(), a.kv_sel_stride = c->kv_sel_stride();
     a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
+    prefetch_target(c, G_GU, l, &a.pf_ptr, &a.pf_bytes);           // attention runs: fetch W_gate/up
     if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->stream, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gemm_params(c, G_GU, l, tab), c->stream, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_DOWN, l, tab), c->stream, pdl))) return e;
+    GemmParams gg = gemm_params(c, G_GU, l, tab);
+    prefetch_target(c, G_DOWN, l, &gg.pf_ptr, &gg.pf_bytes);       // gate/up runs: fetch W_down
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
+    GemmParams gd = gemm_params(c, G_DOWN, l, tab);
+    prefetch_target(c, G_QKV, l + 1, &gd.pf_ptr, &gd.pf_bytes);    // down runs: fetch the next layer's W_qkv
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
   }
   return cudaSuccess;
@@ -668,6 +687,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           return LOOPSPEC_ECUDA;
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
+  if (const char* env = getenv("LOOPSPEC_NO_L2PF")) c->use_l2pf = !(env[0] == '1');
+  if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
   if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
     int v[5];
     if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
@@ -1081,6 +1102,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
+      if (getenv("LOOPSPEC_DBG")) p.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart);  // tuning aid
       cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }
