@@ -25,6 +25,9 @@ struct AttnParams {
   int* counters;              // [row][n_kv]
   const void* pf_ptr;         // region to prefetch into L2 for a later kernel of the chain (may be null)
   long long pf_bytes;
+  long long* dbg;             // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
+  unsigned long long* tl;     // tuning aid: kernel timeline (null in production)
+  int tl_id;
 };
 
 template <int D, int G>
@@ -41,6 +44,12 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
   __shared__ float s_stat[G][2];
   __shared__ int s_last;
 
+  int dbg_n = 0;
+  auto stamp = [&]() {
+    if (p.dbg && blockIdx.x == 0 && threadIdx.x == 0) p.dbg[dbg_n++] = clock64();
+  };
+  stamp();
+  timeline_mark(p.tl, p.tl_id, false);
   if (threadIdx.x == 0) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
   const RowTable* tab = p.tab;   // written before this pass started: safe to read ahead of the predecessor
   const int n_rows = tab->n_rows;
@@ -86,12 +95,16 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
     };
 #pragma unroll
     for (int rd = 0; rd < ROUNDS; ++rd) kreg[rd] = vreg[rd] = make_uint4(0, 0, 0, 0);
+    stamp();
     load_kv(0, n_safe);
+    stamp();
     if (!waited) {
       pdl_launch_dependents();
       pdl_wait();
       waited = true;
+      timeline_mark(p.tl, p.tl_id + 256, false);
     }
+    stamp();
     load_kv(n_safe, n_here);
 
     float q[G][8];
@@ -104,6 +117,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       q[gq][4] = b.x, q[gq][5] = b.y, q[gq][6] = b.z, q[gq][7] = b.w;
     }
     __syncthreads();  // shared buffers of the previous item are free
+    stamp();
 
     // ---- scores ------------------------------------------------------------------------------------
 #pragma unroll
@@ -127,6 +141,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       }
     }
     __syncthreads();
+    stamp();
 
     // ---- chunk softmax statistics (one warp per query head, round robin) ----------------------------
     for (int gq = warp; gq < G; gq += ATT_THREADS / 32) {
@@ -143,6 +158,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       if (lane == 0) s_stat[gq][0] = m, s_stat[gq][1] = l;
     }
     __syncthreads();
+    stamp();
 
     // ---- weighted values ----------------------------------------------------------------------------
     float o[G][8];
@@ -178,6 +194,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
         if (sub == 0) s_red[warp][gq][dl * 8 + i] = v;
       }
     __syncthreads();
+    stamp();
 
     const int pair = row * p.n_kv_heads + kvh;
     float* mypart = p.part + ((size_t)pair * p.max_chunks + chunk) * G * PSTRIDE;
@@ -207,6 +224,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       __threadfence();
     }
     __syncthreads();
+    stamp();
     if (s_last) {  // combine the chunks in ascending order
       const float* base = p.part + (size_t)pair * p.max_chunks * G * PSTRIDE;
       for (int idx = tid; idx < G * D; idx += ATT_THREADS) {
@@ -241,11 +259,13 @@ __global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant
       }
       if (tid == 0) p.counters[pair] = 0;
     }
+    stamp();
   }
   if (!waited) {
     pdl_launch_dependents();
     pdl_wait();
   }
+  timeline_mark(p.tl, p.tl_id, true);
 }
 
 }  // namespace ls

@@ -121,6 +121,18 @@ __device__ __forceinline__ void l2_prefetch_slice(const void* ptr, long long byt
   }
 }
 
+// tuning aid: earliest CTA start / latest CTA end of kernel `id` on the global nanosecond timer
+__device__ __forceinline__ void timeline_mark(unsigned long long* tl, int id, bool end) {
+  if (tl == nullptr || threadIdx.x != 0) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  if (end) atomicMax(tl + 2 * id + 1, t);
+  else {
+    atomicMin(tl + 2 * id, t);
+    if (id < 256) atomicMax(tl + 2 * (id + 512) + 1, t);  // the latest CTA start
+  }
+}
+
 // programmatic dependent launch: wait for the kernels this launch depends on / let dependents start launching
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -72,6 +72,8 @@ struct GemmParams {
   const void* pf_ptr;     // region to prefetch into L2 for a later kernel of the chain (may be null)
   long long pf_bytes;
   long long* dbg;         // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
+  unsigned long long* tl; // tuning aid: kernel timeline (null in production)
+  int tl_id;
 };
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
@@ -92,14 +94,15 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // first weight row this warp streams for row block rb (-1: outside the matrix)
-template <int EPI>
+template <int EPI, int KH = 1>
 __device__ __forceinline__ int gemm_row0(const GemmParams& p, int rb, int warp) {
   if (EPI == EPI_SWIGLU) {  // 64 gate rows and the 64 matching up rows
     int j = rb * 64 + (warp & 3) * 16;
     if (j >= p.F) return -1;
     return (warp < 4) ? j : p.F + j;
   }
-  int r = rb * RB_ROWS + warp * 16;
+  // KH = 2: blocks of 64 rows; warps 0-3 and 4-7 take the same four row tiles and alternate k-blocks
+  int r = rb * (RB_ROWS / KH) + (warp % (8 / KH)) * 16;
   return r < p.N ? r : -1;
 }
 
@@ -113,28 +116,29 @@ __device__ __forceinline__ void gemm_krange(int kpr, int cs, int rank, int& lo, 
 // ---- every rank has pushed its partial columns into the owners' receive buffers: sum them in rank order and
 // finish this CTA's columns.  Column c of row block rb is finished by rank (c mod cluster size); threads 0..127
 // take one column, threads 128..255 the next one of this rank, one output row each.
-template <int EPI>
+template <int EPI, int KH = 1>
 __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, const float* recv,
                                                      int own_max, float* colbuf, const float* s_rstd, int rank) {
+  constexpr int RBW = RB_ROWS / KH;  // rows of this row block
   const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
-  const int cs = p.cluster_size;
+  const int cs = p.cluster_size, vcs = cs * KH;
   __shared__ float s_ss[2][4];
   for (int base = rank; base < n_cols; base += 2 * cs) {
     const int c = base + cs * half;
-    const bool live = c < n_cols;
+    const bool live = c < n_cols && j < RBW;
     // global operands of the epilogue are requested first so that their latency overlaps the summation
     float h_old = 0.f, g_next = 1.f;
     float* h_ptr = nullptr;
     if (EPI == EPI_RESID && live) {
-      h_ptr = p.hid + (size_t)tab->hid_idx[c] * p.H + rb * RB_ROWS + j;
+      h_ptr = p.hid + (size_t)tab->hid_idx[c] * p.H + rb * RBW + j;
       h_old = *h_ptr;
-      if (p.out_planes) g_next = p.gain_next[rb * RB_ROWS + j];
+      if (p.out_planes) g_next = p.gain_next[rb * RBW + j];
     }
     float v = 0.f;
     if (live) {
-      const float* src = recv + (size_t)(c / cs) * RB_ROWS + j;
+      const float* src = recv + (size_t)(c / cs) * RBW + j;
       v = src[0];
-      for (int rk = 1; rk < cs; ++rk) v += src[(size_t)rk * own_max * RB_ROWS];  // rank order, the same for every launch
+      for (int rk = 1; rk < vcs; ++rk) v += src[(size_t)rk * own_max * RBW];  // rank order, the same for every launch
       v *= s_rstd[c];
     }
     if (EPI == EPI_PLAIN || EPI == EPI_LOGITS) {
@@ -144,7 +148,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
         else p.logits[(size_t)tab->logit_idx[tab->ro_rows[c]] * p.N + n] = v;
       }
     } else if (EPI == EPI_RESID) {
-      const int n = rb * RB_ROWS + j;
+      const int n = rb * RBW + j;
       float xn = 0.f;
       if (live) {
         xn = h_old + v;
@@ -154,7 +158,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
       float ss = warp_sum(xn * xn);
       if (lane == 0) s_ss[half][hw] = ss;
       __syncthreads();
-      if (live && j == 0) p.sumsq_out[c * p.n_sq_out + rb] = (s_ss[half][0] + s_ss[half][1]) + (s_ss[half][2] + s_ss[half][3]);
+      if (c < n_cols && j == 0) p.sumsq_out[c * p.n_sq_out + rb] = (s_ss[half][0] + s_ss[half][1]) + (s_ss[half][2] + s_ss[half][3]);
       __syncthreads();
     } else {
       colbuf[half * RB_ROWS + j] = v;
@@ -214,11 +218,13 @@ __device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float
 
 // push this thread's accumulator fragments (rows warp*16+g / +8, columns n*8+2t / +1) into the receive buffers of
 // the ranks that own the columns (distributed shared memory stores; made visible by the cluster barrier)
-template <int NG>
+template <int NG, int KH = 1>
 __device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float* recv, int own_max, int n_cols, int cs, int rank,
                                                cg::cluster_group& cluster) {
+  constexpr int RBW = RB_ROWS / KH;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int rl = warp * 16 + g;
+  const int rl = (warp % (8 / KH)) * 16 + g;
+  rank = rank * KH + warp / (8 / KH);  // the two k-halves of a CTA count as separate contributors
 #pragma unroll
   for (int n = 0; n < NG; ++n)
 #pragma unroll
@@ -226,7 +232,7 @@ __device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float*
       const int c = n * 8 + 2 * t + e;
       if (c < n_cols) {
         const int owner = c % cs, slot = c / cs;
-        float* dst = (cs > 1 ? cluster.map_shared_rank(recv, owner) : recv) + ((size_t)rank * own_max + slot) * RB_ROWS + rl;
+        float* dst = (cs > 1 ? cluster.map_shared_rank(recv, owner) : recv) + ((size_t)rank * own_max + slot) * RBW + rl;
         dst[0] = acc[n][e];
         dst[8] = acc[n][2 + e];
       }
@@ -236,6 +242,8 @@ __device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float*
 // ======================================= bf16 weights: tensor cores ========================================
 template <int NG, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
+  // the residual GEMMs have few output rows: 64-row blocks with two k-halves per CTA double the CTAs that stream
+  constexpr int KH = (EPI == EPI_RESID) ? 2 : 1;
   constexpr int NTOK = 8 * NG;
   constexpr int XCH = xchunk_kblocks(NG);
   constexpr int PIECES = 3 * XCH * NTOK * 4;
@@ -257,12 +265,14 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
     if (p.dbg && blockIdx.x == 0 && tid == 0) p.dbg[dbg_n++] = clock64();
   };
   stamp();
+  timeline_mark(p.tl, p.tl_id, false);
   const int kpr = p.kb_per_rb;
   int kb_lo, kb_hi;
   gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
-  const int upt = kb_hi - kb_lo;                                 // units per task
+  const int upt = kb_hi - kb_lo;                                 // k-blocks per task (whole CTA)
+  const int khalf = warp / (8 / KH);                             // which k-blocks of the range this warp takes
+  const int my_upt = (upt - khalf + KH - 1) / KH;                // units per task of this warp
   const int n_tasks = (p.n_rb - cid + p.n_clusters - 1) / p.n_clusters;  // row blocks cid, cid + n_clusters, ...
-  const int n_units = n_tasks * upt;
 
   // ---- weight ring: issue side.  The weights are stored tile-major (see pack_weights_kernel): the 1 KB a warp
   // consumes per unit is contiguous and consecutive k-blocks of a 16-row tile follow each other, so every warp
@@ -274,11 +284,11 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
   const char* i_ptr = reinterpret_cast<const char*>(Wb);
   unsigned i_slot = 0;
-  int i_rb = cid, i_left = upt, i_tasks = n_tasks, i_size = 0;
+  int i_rb = cid, i_left = my_upt, i_tasks = my_upt > 0 ? n_tasks : 0, i_size = 0;
   auto i_setup = [&]() {
-    int r0 = gemm_row0<EPI>(p, i_rb, warp);
+    int r0 = gemm_row0<EPI, KH>(p, i_rb, warp);
     i_size = r0 >= 0 ? 16 : 0;  // rows beyond the matrix: zero-fill, nothing is read
-    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)(r0 >= 0 ? (r0 >> 4) : 0) * kpr + kb_lo) * 512 + lane * 8);
+    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)(r0 >= 0 ? (r0 >> 4) : 0) * kpr + kb_lo + khalf) * 512 + lane * 8);
   };
   i_setup();
   auto issue_unit = [&]() {
@@ -286,10 +296,10 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(ring_s + i_slot), "l"(i_ptr), "r"(i_size) : "memory");
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(ring_s + i_slot + HI_OFF), "l"(i_ptr + 512), "r"(i_size)
                    : "memory");
-      i_ptr += 1024;
+      i_ptr += 1024 * KH;
       i_slot = (i_slot + SLOT_BYTES) & RING_MASK;
       if (--i_left == 0) {
-        i_left = upt, i_rb += p.n_clusters;
+        i_left = my_upt, i_rb += p.n_clusters;
         if (--i_tasks > 0) i_setup();
       }
     }
@@ -308,6 +318,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   pdl_launch_dependents();
   pdl_wait();
   stamp();
+  timeline_mark(p.tl, p.tl_id + 256, false);
   if (n_cols <= 0) {  // uniform over the cluster: nobody reaches a cluster barrier
     cp_async_wait<0>();
     return;
@@ -347,7 +358,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   };
   for (int task = 0; task < n_tasks; ++task) {
     const int rb = cid + task * p.n_clusters;
-    const bool warp_valid = gemm_row0<EPI>(p, rb, warp) >= 0;
+    const bool warp_valid = gemm_row0<EPI, KH>(p, rb, warp) >= 0;
 #pragma unroll
     for (int h = 0; h < 3; ++h)
 #pragma unroll
@@ -362,8 +373,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
         cp_async_wait<0>();
         __syncthreads();
       }
-      unsigned xk = xs_s;
-      for (int kbl = 0; kbl < nkb; ++kbl) {
+      const int kbl0 = (khalf + KH - (ck % KH)) % KH;  // this warp's first k-block of the chunk
+      unsigned xk = xs_s + kbl0 * X_KB;
+      for (int kbl = kbl0; kbl < nkb; kbl += KH) {
         issue_unit();
         cp_async_wait<RING - 1>();
         if (warp_valid) {
@@ -379,7 +391,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
           }
         }
         c_slot = (c_slot + SLOT_BYTES) & RING_MASK;
-        xk += X_KB;
+        xk += X_KB * KH;
       }
     }
     // fold the chains in fixed order, hi + (mid + lo), and publish this CTA's partial tile
@@ -389,14 +401,15 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
 #pragma unroll
       for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
     stamp();
-    gemm_push_tile<NG>(tot, recv, own_max, n_cols, cs, rank, cluster);
+    gemm_push_tile<NG, KH>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
     stamp();
-    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+    gemm_reduce_epilogue<EPI, KH>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
     stamp();
     if (task + 1 < n_tasks) cluster.sync();  // the owners are done with the receive buffer before it is refilled
   }
   cp_async_wait<0>();
+  timeline_mark(p.tl, p.tl_id, true);
 }
 
 // ======================================= fp32 weights: CUDA cores ==========================================

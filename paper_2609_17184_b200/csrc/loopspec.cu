@@ -155,7 +155,7 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->n_hid = d->S * d->NB + MAX_ROWS;
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
-  d->n_sq = m->hidden / 128;
+  d->n_sq = m->hidden / (m->weight_dtype == 1 ? 64 : 128);  // residual row blocks: 64 rows (bf16 kernels), 128 (fp32)
   d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
   d->trace_cap = 4 * s->max_ctx + 64;
   d->Hq = m->n_q_heads * m->head_dim;
@@ -244,7 +244,7 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = true;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = false;
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
   int launches_per_step = 0;
@@ -472,7 +472,9 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     return cudaSuccess;
   }
   for (int l = 0; l < m.n_recurrent; ++l) {
+    unsigned long long* tl = getenv("LOOPSPEC_DBG") ? reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024 : nullptr;  // tuning aid
     GemmParams gq = gemm_params(c, G_QKV, l, tab);
+    gq.tl = tl, gq.tl_id = l * 5 + 0;
     prefetch_target(c, G_O, l, &gq.pf_ptr, &gq.pf_bytes);          // QKV runs: fetch W_o
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
     AttnParams a;
@@ -484,12 +486,18 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
     prefetch_target(c, G_GU, l, &a.pf_ptr, &a.pf_bytes);           // attention runs: fetch W_gate/up
+    if (l == 3 && getenv("LOOPSPEC_DBG")) a.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart) + 64;  // tuning aid
+    a.tl = tl, a.tl_id = l * 5 + 1;
     if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_O, l, tab), c->stream, pdl))) return e;
+    GemmParams go = gemm_params(c, G_O, l, tab);
+    go.tl = tl, go.tl_id = l * 5 + 2;
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
     GemmParams gg = gemm_params(c, G_GU, l, tab);
+    gg.tl = tl, gg.tl_id = l * 5 + 3;
     prefetch_target(c, G_DOWN, l, &gg.pf_ptr, &gg.pf_bytes);       // gate/up runs: fetch W_down
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
     GemmParams gd = gemm_params(c, G_DOWN, l, tab);
+    gd.tl = tl, gd.tl_id = l * 5 + 4;
     prefetch_target(c, G_QKV, l + 1, &gd.pf_ptr, &gd.pf_bytes);    // down runs: fetch the next layer's W_qkv
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
@@ -673,7 +681,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * m->n_recurrent);
   c->ng_dec = ng_for_rows(d.max_rows_dec), c->ng_pf = ng_for_rows(d.max_rows_pf);
   c->prefilled.assign(d.S, 0);
-  const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / 128, (m->ffn + 63) / 64, m->hidden / 128, (m->vocab + 127) / 128};
+  const int resid_rows = m->weight_dtype == 1 ? 64 : 128;
+  const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / resid_rows, (m->ffn + 63) / 64, m->hidden / resid_rows, (m->vocab + 127) / 128};
   const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
   int slots = n_sm * kCtasPerSm;
   if (const char* env = getenv("LOOPSPEC_SLOTS")) slots = std::max(1, atoi(env));  // tuning aid
@@ -687,7 +696,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           return LOOPSPEC_ECUDA;
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
-  if (const char* env = getenv("LOOPSPEC_NO_L2PF")) c->use_l2pf = !(env[0] == '1');
+  if (const char* env = getenv("LOOPSPEC_L2PF")) c->use_l2pf = env[0] == '1';  // measured no gain: off by default
   if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
   if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
     int v[5];
@@ -794,7 +803,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       q.H = m->hidden, q.Hq = d.Hq, q.Hkv = d.Hkv, q.F = m->ffn, q.n_q_heads = m->n_q_heads, q.n_kv_heads = m->n_kv_heads;
       q.head_dim = m->head_dim, q.slots = d.slots, q.eps = m->rms_eps, q.scale = 1.0f / sqrtf((float)m->head_dim);
       q.hid = c->at<float>(L.hid), q.xplanes = c->at<__nv_bfloat16>(L.xplanes), q.aplanes = c->at<__nv_bfloat16>(L.aplanes);
-      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq), q.n_sq = d.n_sq;
+      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq), q.n_sq = m->hidden / 128;
+      q.sq_stride = d.n_sq;
       q.kv = c->at<__nv_bfloat16>(L.kv), q.kv_layer_stride = c->kv_layer_stride(), q.kv_plane_stride = c->kv_plane_stride();
       q.kv_sel_stride = c->kv_sel_stride(), q.rope = c->at<float2>(L.rope);
       q.gpart = c->at<float>(L.gpart), q.gcnt = c->at<int>(L.gcnt), q.apart = c->at<float>(L.apart), q.acnt = c->at<int>(L.acnt);
@@ -802,7 +812,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       const int Ns[4] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden};
       bool fits = true;
       for (int i = 0; i < 4; ++i) {
-        q.n_rb[i] = n_rbs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.N[i] = Ns[i], q.K[i] = Ks[i];
+        q.n_rb[i] = (i == 1 || i == 3) ? m->hidden / 128 : n_rbs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.N[i] = Ns[i], q.K[i] = Ks[i];
         int total = q.n_rb[i] * q.kpr[i];
         q.upc[i] = (total + c->pass_grid - 1) / c->pass_grid;
         int mc = 1;
@@ -1103,6 +1113,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
       if (getenv("LOOPSPEC_DBG")) p.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart);  // tuning aid
+      if (getenv("LOOPSPEC_PFSELF") && which < 4) prefetch_target(c, which, (i + 1) % L, &p.pf_ptr, &p.pf_bytes);  // tuning aid
       cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }

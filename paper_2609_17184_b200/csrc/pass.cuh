@@ -33,7 +33,7 @@ struct PassParams {
   __nv_bfloat16 *xplanes, *aplanes, *splanes;
   float* qbuf;
   float* sumsq;                 // [row][n_sq]
-  int n_sq;
+  int n_sq, sq_stride;
   __nv_bfloat16* kv;            // whole pool
   long long kv_layer_stride, kv_plane_stride, kv_sel_stride;
   const float2* rope;
@@ -133,7 +133,7 @@ __device__ __forceinline__ void pass_epilogue(const PassParams& p, const RowTabl
       v.x += tr[0], v.y += tr[1], v.z += tr[2], v.w += tr[3];
       *h = v;
       float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
-      if (lane == 0) p.sumsq[c * p.n_sq + rb] = ss;
+      if (lane == 0) p.sumsq[c * p.sq_stride + rb] = ss;
       if (gain_next) {
         float4 gn = *reinterpret_cast<const float4*>(gain_next + n0 + lane * 4);
         float xv[4] = {v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w};
@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
           if (normed) {
             const int n_sq = (st == ST_QKV && l == 0) ? 1 : p.n_sq;
             float ss = 0.f;
-            for (int q = 0; q < n_sq; ++q) ss += __ldcg(p.sumsq + tid * p.n_sq + q);
+            for (int q = 0; q < n_sq; ++q) ss += __ldcg(p.sumsq + tid * p.sq_stride + q);
             r = 1.0f / sqrtf(ss / (float)p.H + p.eps);
           }
           s_rstd[tid] = r;
