@@ -277,7 +277,7 @@ def run_calibrated(ls, shape, wl, prompt, n_prompt, n_decode, args):
     draft like trained checkpoints do (first-proposal share in the band the paper reports for Ouro-1.4B)."""
     import torch
     res = None
-    for scale in (0.01, 0.003, 0.03, 0.001):
+    for scale in (0.0003, 0.0001, 0.001, 0.00003):
         w = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed, out_scale=scale))
         ctx = ls.LoopSpec(shape, w, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
                           max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64)

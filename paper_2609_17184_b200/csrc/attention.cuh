@@ -10,7 +10,8 @@
 
 namespace ls {
 
-constexpr int ATT_THREADS = 128;
+constexpr int ATT_THREADS = 256;  // 8 warps per work item; at most 64 registers per thread so that the
+                                   // neighbouring GEMM kernels' CTAs can be resident (and prefetching) alongside
 
 struct AttnParams {
   const RowTable* tab;
@@ -31,7 +32,7 @@ struct AttnParams {
 };
 
 template <int D, int G>
-__global__ void __launch_bounds__(ATT_THREADS) attn_kernel(const __grid_constant__ AttnParams p) {
+__global__ void __launch_bounds__(ATT_THREADS, 4) attn_kernel(const __grid_constant__ AttnParams p) {
   constexpr int LPP = D / 8;            // lanes per key position (8 bf16 = 16 bytes per lane)
   constexpr int PPW = 32 / LPP;         // positions per warp per load
   constexpr int PPR = PPW * (ATT_THREADS / 32);  // positions per round of the whole CTA

@@ -126,10 +126,19 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
   __shared__ int s_root[MAX_ROWS], s_nids[MAX_ROWS], s_ndec[MAX_ROWS], s_ntarget[MAX_ROWS], s_needv[MAX_ROWS];
   __shared__ int s_emb[2 * MAX_ROWS][2];
   __shared__ int s_nemb, s_err;
+  __shared__ int s_sel_tok[MAX_ROWS], s_sel_aux[MAX_ROWS];
+  __shared__ float s_sel_lse[MAX_ROWS], s_sel_z2[MAX_ROWS];
+  __shared__ unsigned long long s_steps;
   const int tid = threadIdx.x;
   const int n_nodes = p.S * p.NB;
   pdl_launch_dependents();
   pdl_wait();
+  // everything the serial bookkeeping reads is pulled into shared memory with one round of parallel loads
+  if (tid < MAX_ROWS) {
+    s_sel_tok[tid] = p.sel_tok[tid], s_sel_aux[tid] = p.sel_aux[tid];
+    s_sel_lse[tid] = p.sel_lse[tid], s_sel_z2[tid] = p.sel_z2[tid];
+  }
+  if (tid == MAX_ROWS) s_steps = p.ctr->steps;
   nodes_load(nd, p.nodes, n_nodes);
   {
     const int* src = reinterpret_cast<const int*>(p.tab);
@@ -153,19 +162,19 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
       for (int i = 0; i < t.n_rows; ++i) {
         if (t.seq[i] != s) continue;
         const int gn = t.node[i], ro = t.readout[i];
-        if (ro == RO_D1 || (ro == RO_D2 && p.sel_aux[i])) {
+        if (ro == RO_D1 || (ro == RO_D2 && s_sel_aux[i])) {
           int c = alloc_node(st, p.NB);
           if (c < 0) { s_err = ERR_NODES; continue; }
-          st[c] = 1, nd.depth[o + c] = 0, nd.pos[o + c] = nd.pos[gn] + 1, nd.token[o + c] = p.sel_tok[i];
+          st[c] = 1, nd.depth[o + c] = 0, nd.pos[o + c] = nd.pos[gn] + 1, nd.token[o + c] = s_sel_tok[i];
           nd.parent[o + c] = gn - o, nd.child1[o + c] = nd.child2[o + c] = -1, nd.has2[o + c] = 0;
           if (ro == RO_D1) {
-            nd.tok1[gn] = p.sel_tok[i], nd.child1[gn] = c, nd.lse1[gn] = p.sel_lse[i], nd.has2[gn] = 0, nd.child2[gn] = -1;
+            nd.tok1[gn] = s_sel_tok[i], nd.child1[gn] = c, nd.lse1[gn] = s_sel_lse[i], nd.has2[gn] = 0, nd.child2[gn] = -1;
           } else {
-            nd.tok2[gn] = p.sel_tok[i], nd.child2[gn] = c, nd.lse2[gn] = p.sel_lse[i], nd.z2[gn] = p.sel_z2[i], nd.has2[gn] = 1;
+            nd.tok2[gn] = s_sel_tok[i], nd.child2[gn] = c, nd.lse2[gn] = s_sel_lse[i], nd.z2[gn] = s_sel_z2[i], nd.has2[gn] = 1;
             atomicAdd(&p.ctr->gate_opens, 1ull);
           }
           int e = atomicAdd(&s_nemb, 1);
-          s_emb[e][0] = o + c, s_emb[e][1] = p.sel_tok[i];
+          s_emb[e][0] = o + c, s_emb[e][1] = s_sel_tok[i];
         }
         if (ro == RO_D2) atomicAdd(&p.ctr->gate_evals, 1ull);
         if (ro == RO_VERIFY) s_needv[s] = 1;
@@ -178,13 +187,13 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
       for (int i = 0; i < t.n_rows; ++i)
         if (t.seq[i] == s && t.readout[i] == RO_VERIFY) vrow = i;
       const int rt = s_root[s];
-      const int tok = p.sel_tok[vrow], src = p.sel_aux[vrow];
+      const int tok = s_sel_tok[vrow], src = s_sel_aux[vrow];
       const int k = s_ndec[s];
       if (k < p.ids_cap) {
         p.out_ids[(size_t)s * p.ids_cap + k] = tok;
         int* cm = p.commits + ((size_t)s * p.ids_cap + k) * 8;
         cm[0] = s, cm[1] = 1, cm[2] = tok, cm[3] = src, cm[4] = (src == 1), cm[5] = (src == 2), cm[6] = nd.has2[o + rt];
-        cm[7] = (int)p.ctr->steps + ((p.phases & PH_ADVANCE) ? 1 : 0);
+        cm[7] = (int)s_steps + ((p.phases & PH_ADVANCE) ? 1 : 0);
       }
       s_ndec[s] = k + 1, s_nids[s] += 1;
       atomicAdd(&p.ctr->n_decode, 1ull);
