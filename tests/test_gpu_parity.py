@@ -215,3 +215,28 @@ def test_error_paths_leave_the_context_usable():
         U.make_ctx("tiny_bf16", 3, 0)
     assert e.value.status == "EINVAL"
     ctx.close()
+
+
+def test_depths_from_the_closed_form_are_used_when_none_are_given():
+    """d1 = d2 = 0 at init: the library picks the admissible pair minimising Theorem 2's bound, like the oracle."""
+    from oracle import depths as dp
+    alpha, beta = 1.0, 0.3
+    R = W.CONFIGS["tiny_bf16"].R
+    d1, d2 = dp.snap_depths(float(np.float32(alpha)), float(np.float32(beta)), R)
+    ref = U.oracle_run("tiny_bf16", 16, 40, d1, d2, T=1.0, seed=2)
+    ctx = U.make_ctx("tiny_bf16", 0, 0, T=1.0, seed=2, max_ctx=64, alpha=alpha, beta=beta)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(40)
+    U.assert_same_run(ctx, ref, 40)
+    assert ctx.stats()["steps"] == ref["dec"].stats["steps"]
+    ctx.close()
+
+
+def test_longer_context_spans_many_attention_chunks():
+    """A 300-token prompt: five 64-position attention chunks plus the speculative slots, prefill in 64-row passes."""
+    ref = U.oracle_run("tiny_bf16", 300, 24, 1, 2, T=1.0, seed=4)
+    ctx = U.make_ctx("tiny_bf16", 1, 2, T=1.0, seed=4, max_ctx=340, max_prefill_rows=64)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(24)
+    U.assert_same_run(ctx, ref, 24)
+    ctx.close()
