@@ -105,6 +105,19 @@ def vanilla_bytes(shape, n_prompt, n_decode):
 KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
 
 
+def replica_throughput(tokens_per_rank, device_ms, wall_s, dist=None, device=None):
+    """Whole-job tokens/s of N independent replicas: every rank decodes `tokens_per_rank`; the job takes as long
+    as its slowest rank (MAX over ranks of the device time and of the wall time).  Returns (value, e2e, max_ms)."""
+    world = 1
+    if dist is not None:
+        import torch
+        t = torch.tensor([device_ms, wall_s], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        device_ms, wall_s = t.tolist()
+        world = dist.get_world_size()
+    return world * tokens_per_rank / (device_ms / 1e3), world * tokens_per_rank / wall_s, device_ms
+
+
 def run_kernel_only(args):
     """Time one kernel of the pass alone (used for profiling captures): prints its own JSON line."""
     import torch
@@ -205,15 +218,7 @@ def run_ours(args):
         van_ms.append(ms)
     lossless = bool((vout[0] == out[0]).all()) if wl.temperature == 0 else None
 
-    tot_ms = sum(dec_ms)
-    if dist is not None:
-        t = torch.tensor([tot_ms, sum(wall_s)], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        tot_ms, wall_tot = t.tolist()
-    else:
-        wall_tot = sum(wall_s)
-    value = world * args.steps * n_decode / (tot_ms / 1e3)
-    e2e = world * args.steps * n_decode / wall_tot
+    value, e2e, tot_ms = replica_throughput(args.steps * n_decode, sum(dec_ms), sum(wall_s), dist, "cuda")
     ms_per_step = tot_ms / args.steps
 
     # roofline of the dominant kernel (gate/up GEMM), timed alone over the 24 layers' weights
