@@ -118,7 +118,8 @@ __device__ __forceinline__ void gemm_krange(int kpr, int cs, int rank, int& lo, 
 // take one column, threads 128..255 the next one of this rank, one output row each.
 template <int EPI, int KH = 1>
 __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, const float* recv,
-                                                     int own_max, float* colbuf, const float* s_rstd, int rank) {
+                                                     int own_max, float* colbuf, const float* s_rstd, int rank, float pre_h = 0.f,
+                                                     float pre_g = 1.f, bool pre_valid = false) {
   constexpr int RBW = RB_ROWS / KH;  // rows of this row block
   const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
   const int cs = p.cluster_size, vcs = cs * KH;
@@ -131,8 +132,12 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
     float* h_ptr = nullptr;
     if (EPI == EPI_RESID && live) {
       h_ptr = p.hid + (size_t)tab->hid_idx[c] * p.H + rb * RBW + j;
-      h_old = *h_ptr;
-      if (p.out_planes) g_next = p.gain_next[rb * RBW + j];
+      if (pre_valid && base == rank) {  // requested before the cluster barrier
+        h_old = pre_h, g_next = pre_g;
+      } else {
+        h_old = *h_ptr;
+        if (p.out_planes) g_next = p.gain_next[rb * RBW + j];
+      }
     }
     float v = 0.f;
     if (live) {
@@ -401,10 +406,19 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
 #pragma unroll
       for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
     stamp();
+    // the residual stream and the next gain of this CTA's first output column are requested before the barrier
+    float pre_h = 0.f, pre_g = 1.f;
+    if (EPI == EPI_RESID) {
+      const int c = rank + cs * (tid >> 7), jr = tid & 127;
+      if (c < n_cols && jr < RB_ROWS / KH) {
+        pre_h = p.hid[(size_t)tab->hid_idx[c] * p.H + rb * (RB_ROWS / KH) + jr];
+        if (p.out_planes) pre_g = p.gain_next[rb * (RB_ROWS / KH) + jr];
+      }
+    }
     gemm_push_tile<NG, KH>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
     stamp();
-    gemm_reduce_epilogue<EPI, KH>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+    gemm_reduce_epilogue<EPI, KH>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank, pre_h, pre_g, EPI == EPI_RESID);
     stamp();
     if (task + 1 < n_tasks) cluster.sync();  // the owners are done with the receive buffer before it is refilled
   }

@@ -244,7 +244,7 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = false;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = false, l2pf_only_o = false;
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
   int launches_per_step = 0;
@@ -421,6 +421,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
 void prefetch_target(loopspec_ctx* c, int which, int l, const void** ptr, long long* bytes) {
   *ptr = nullptr, *bytes = 0;
   if (c->packed.empty() || !c->use_l2pf || l >= c->m.n_recurrent) return;
+  if (c->l2pf_only_o && which != G_O) return;
   const Derived& d = c->d;
   const int Ns[4] = {d.Hq + 2 * d.Hkv, c->m.hidden, 2 * c->m.ffn, c->m.hidden};
   const int Ks[4] = {c->m.hidden, d.Hq, c->m.hidden, c->m.ffn};
@@ -696,7 +697,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           return LOOPSPEC_ECUDA;
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
-  if (const char* env = getenv("LOOPSPEC_L2PF")) c->use_l2pf = env[0] == '1';  // measured no gain: off by default
+  if (const char* env = getenv("LOOPSPEC_L2PF")) c->use_l2pf = env[0] != '0', c->l2pf_only_o = env[0] == '2';  // tuning aid
   if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
   if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
     int v[5];
