@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_kernel(const __grid_const
 
   int dbg_n = 0;
   auto stamp = [&]() {
-    if (p.dbg && blockIdx.x == 0 && threadIdx.x == 0) p.dbg[dbg_n++] = clock64();
+    if (kTune && p.dbg && blockIdx.x == 0 && threadIdx.x == 0) p.dbg[dbg_n++] = clock64();
   };
   stamp();
   timeline_mark(p.tl, p.tl_id, false);

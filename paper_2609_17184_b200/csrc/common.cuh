@@ -7,6 +7,14 @@
 
 namespace ls {
 
+// tuning aids (cycle stamps, kernel timeline, L2 prefetch requests) are compiled in only with -DLOOPSPEC_TUNE:
+// the decode kernels run for a few microseconds each and every kilobyte of code they carry costs fetch time
+#ifdef LOOPSPEC_TUNE
+constexpr bool kTune = true;
+#else
+constexpr bool kTune = false;
+#endif
+
 constexpr int MAX_ROWS = 64;  // rows (branches) one batched pass can carry: 8 token columns x up to 8 groups
 constexpr int MAX_SPEC = 8;   // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
 constexpr int ATT_CHUNK = 64; // key positions per attention work item (fixed by absolute position)
@@ -107,7 +115,7 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* row_planes, int ld, i
 // CTA; the region is cut into equal 16-byte-aligned slices).  Used to keep HBM busy with the NEXT kernel's
 // weights while the current kernel is in its latency-bound prologue / epilogue.
 __device__ __forceinline__ void l2_prefetch_slice(const void* ptr, long long bytes, int slice, int n_slices) {
-  if (ptr == nullptr || bytes <= 0) return;
+  if (!kTune || ptr == nullptr || bytes <= 0) return;
   long long per = ((bytes + n_slices - 1) / n_slices + 15) & ~15ll;
   long long off = (long long)slice * per;
   if (off >= bytes) return;
@@ -123,7 +131,7 @@ __device__ __forceinline__ void l2_prefetch_slice(const void* ptr, long long byt
 
 // tuning aid: earliest CTA start / latest CTA end of kernel `id` on the global nanosecond timer
 __device__ __forceinline__ void timeline_mark(unsigned long long* tl, int id, bool end) {
-  if (tl == nullptr || threadIdx.x != 0) return;
+  if (!kTune || tl == nullptr || threadIdx.x != 0) return;
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   if (end) atomicMax(tl + 2 * id + 1, t);

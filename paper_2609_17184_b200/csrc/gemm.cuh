@@ -29,13 +29,15 @@ constexpr int RB_ROWS = 128;   // output rows per row block
 constexpr int TILE_LD = 132;   // padded leading dimension of the partial tile
 constexpr int RING = 8;        // weight stages in flight per thread (8 KB per stage per CTA)
 constexpr int MAX_XCH_BLOCKS = 24;  // k-blocks of activations one CTA keeps staged when NG = 1
+// per-column copies of the row-table fields the epilogues need ([field][column] in shared memory)
+enum { CT_POS = 0, CT_R = 1, CT_SEQ = 2, CT_SLOT = 3, CT_HID = 4, CT_LOGIT = 5, CT_FIELDS = 6 };
 
 __host__ __device__ constexpr int xchunk_kblocks(int NG) { return MAX_XCH_BLOCKS / NG; }
 __host__ __device__ constexpr int xbuf_uint4(int NG) { return 3 * xchunk_kblocks(NG) * 8 * NG * 4; }
 // partial columns received from the cluster's ranks: [rank][owned column][128 rows]
 __host__ __device__ constexpr int recv_floats(int NG) { return (8 * NG + 7) * RB_ROWS; }
 __host__ __device__ constexpr int gemm_smem_bytes(int NG) {
-  return RING * 2 * GEMM_THREADS * 16 + xbuf_uint4(NG) * 16 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
+  return RING * 2 * GEMM_THREADS * 16 + xbuf_uint4(NG) * 16 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 * (1 + CT_FIELDS) + 64;
 }
 
 struct GemmParams {
@@ -69,6 +71,7 @@ struct GemmParams {
   const float2* rope;     // [pos][d/2] (cos, sin)
   float* logits;          // LOGITS: [logit_idx][V]
   int F;                  // SWIGLU: ffn width
+  int perm, perm_a, perm_d;  // order of the row tiles in the packed weights (see packed_tile)
   const void* pf_ptr;     // region to prefetch into L2 for a later kernel of the chain (may be null)
   long long pf_bytes;
   long long* dbg;         // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
@@ -92,6 +95,28 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, boo
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Row tile order of the packed weights.  perm 0: natural.  perm 1 (gate/up, a = ffn width): gate tile u and up
+// tile u are adjacent (2u, 2u + 1).  perm 2 (QKV, a = tiles per rotary half, d = head size): the tile holding
+// rows i of a head and the tile holding their rotary partners i + d/2 are adjacent.
+__host__ __device__ __forceinline__ int packed_tile(int perm, int a, int d, int row0) {
+  const int tt = row0 >> 4;
+  if (perm == 1) return row0 < a ? 2 * tt : 2 * ((row0 - a) >> 4) + 1;
+  if (perm == 2) {  // a is 2 or 4 (head size 64 or 128): shifts, no divisions
+    const int la = a == 4 ? 2 : 1, h = tt >> (la + 1), w = tt & (2 * a - 1);
+    return 2 * (h * a + (w & (a - 1))) + (w >> la);
+  }
+  return tt;
+}
+// first row of packed tile pt in the source matrix (inverse of packed_tile)
+__host__ __device__ __forceinline__ int packed_tile_row0(int perm, int a, int d, int pt) {
+  if (perm == 1) return (pt & 1) * a + (pt >> 1) * 16;
+  if (perm == 2) {
+    const int grp = pt >> 1, h = grp / a, j = grp - h * a;
+    return h * d + (j + (pt & 1) * a) * 16;
+  }
+  return pt * 16;
+}
 
 // first weight row this warp streams for row block rb (-1: outside the matrix)
 template <int EPI, int KH = 1>
@@ -117,9 +142,9 @@ __device__ __forceinline__ void gemm_krange(int kpr, int cs, int rank, int& lo, 
 // finish this CTA's columns.  Column c of row block rb is finished by rank (c mod cluster size); threads 0..127
 // take one column, threads 128..255 the next one of this rank, one output row each.
 template <int EPI, int KH = 1>
-__device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const RowTable* tab, int rb, int n_cols, const float* recv,
+__device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const int* ct, int ntok, int rb, int n_cols, const float* recv,
                                                      int own_max, float* colbuf, const float* s_rstd, int rank, float pre_h = 0.f,
-                                                     float pre_g = 1.f, bool pre_valid = false) {
+                                                     float pre_g = 1.f, float2 pre_rope = make_float2(1.f, 0.f), bool pre_valid = false) {
   constexpr int RBW = RB_ROWS / KH;  // rows of this row block
   const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
   const int cs = p.cluster_size, vcs = cs * KH;
@@ -131,7 +156,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
     float h_old = 0.f, g_next = 1.f;
     float* h_ptr = nullptr;
     if (EPI == EPI_RESID && live) {
-      h_ptr = p.hid + (size_t)tab->hid_idx[c] * p.H + rb * RBW + j;
+      h_ptr = p.hid + (size_t)ct[CT_HID * ntok + c] * p.H + rb * RBW + j;
       if (pre_valid && base == rank) {  // requested before the cluster barrier
         h_old = pre_h, g_next = pre_g;
       } else {
@@ -150,7 +175,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
       const int n = rb * RB_ROWS + j;
       if (live && n < p.N) {
         if (EPI == EPI_PLAIN) p.out[(size_t)c * p.out_ld + n] = v;
-        else p.logits[(size_t)tab->logit_idx[tab->ro_rows[c]] * p.N + n] = v;
+        else p.logits[(size_t)ct[CT_LOGIT * ntok + c] * p.N + n] = v;
       }
     } else if (EPI == EPI_RESID) {
       const int n = rb * RBW + j;
@@ -186,7 +211,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
           const float x1 = col[hh * d + i], x2 = col[hh * d + i + hd2];
           float y1 = x1, y2 = x2;
           if (region < 2) {
-            float2 csn = p.rope[(size_t)tab->pos[c] * hd2 + i];
+            const float2 csn = (pre_valid && base == rank) ? pre_rope : p.rope[(size_t)ct[CT_POS * ntok + c] * hd2 + i];
             y1 = x1 * csn.x - x2 * csn.y;
             y2 = x2 * csn.x + x1 * csn.y;
           }
@@ -196,8 +221,8 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
             q[0] = y1;
             q[hd2] = y2;
           } else {
-            __nv_bfloat16* dst = p.kv + (size_t)(tab->r[c] - 1) * p.kv_plane_stride + (size_t)(region - 1) * p.kv_sel_stride +
-                                 ((size_t)(tab->seq[c] * p.n_kv_heads + head) * p.slots + tab->kv_slot[c]) * d + i;
+            __nv_bfloat16* dst = p.kv + (size_t)(ct[CT_R * ntok + c] - 1) * p.kv_plane_stride + (size_t)(region - 1) * p.kv_sel_stride +
+                                 ((size_t)(ct[CT_SEQ * ntok + c] * p.n_kv_heads + head) * p.slots + ct[CT_SLOT * ntok + c]) * d + i;
             dst[0] = __float2bfloat16_rn(y1);
             dst[hd2] = __float2bfloat16_rn(y2);
           }
@@ -208,16 +233,27 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
   }
 }
 
+// 1/rms of every live column: warp w sums the partial sums of squares of columns w, w + 8, ... (one partial per lane,
+// butterfly sum: the same order in every launch)
 __device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float* s_rstd) {
-  const int tid = threadIdx.x;
-  if (tid < n_cols) {
-    float r = 1.0f;
-    if (p.sumsq) {
-      float ss = 0.f;
-      for (int j = 0; j < p.n_sq; ++j) ss += p.sumsq[tid * p.sq_stride + j];
-      r = 1.0f / sqrtf(ss / (float)p.H + p.eps);
-    }
-    s_rstd[tid] = r;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int c = warp; c < n_cols; c += GEMM_THREADS / 32) {
+    float ss = 0.f;
+    if (p.sumsq)
+      for (int j = lane; j < p.n_sq; j += 32) ss += p.sumsq[c * p.sq_stride + j];
+    ss = warp_sum(ss);
+    if (lane == 0) s_rstd[c] = p.sumsq ? 1.0f / sqrtf(ss / (float)p.H + p.eps) : 1.0f;
+  }
+}
+
+// The row table of a pass is final before the pass starts, so its fields can be copied ahead of the predecessor.
+__device__ __forceinline__ void gemm_load_cols(const GemmParams& p, int n_cols, int ntok, int* ct) {
+  const int c = threadIdx.x;
+  const RowTable* tab = p.tab;
+  if (tab && c < n_cols) {
+    const int row = p.cols_from_readout ? tab->ro_rows[c] : c;
+    ct[CT_POS * ntok + c] = tab->pos[row], ct[CT_R * ntok + c] = tab->r[row], ct[CT_SEQ * ntok + c] = tab->seq[row];
+    ct[CT_SLOT * ntok + c] = tab->kv_slot[row], ct[CT_HID * ntok + c] = tab->hid_idx[row], ct[CT_LOGIT * ntok + c] = tab->logit_idx[row];
   }
 }
 
@@ -251,8 +287,6 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   constexpr int KH = (EPI == EPI_RESID) ? 2 : 1;
   constexpr int NTOK = 8 * NG;
   constexpr int XCH = xchunk_kblocks(NG);
-  constexpr int PIECES = 3 * XCH * NTOK * 4;
-  constexpr int PPT = (PIECES + GEMM_THREADS - 1) / GEMM_THREADS;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);            // [RING][2][256], slot of thread tid only
@@ -260,6 +294,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   float* recv = reinterpret_cast<float*>(xbuf + xbuf_uint4(NG));  // [cs][own_max][128]
   float* colbuf = recv + recv_floats(NG);                      // [2][128]
   float* s_rstd = colbuf + 2 * RB_ROWS;
+  int* s_ct = reinterpret_cast<int*>(s_rstd + NTOK);           // [CT_FIELDS][NTOK]
 
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -267,7 +302,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   const int own_max = (NTOK + cs - 1) / cs;
   int dbg_n = 0;
   auto stamp = [&]() {
-    if (p.dbg && blockIdx.x == 0 && tid == 0) p.dbg[dbg_n++] = clock64();
+    if (kTune && p.dbg && blockIdx.x == 0 && tid == 0) p.dbg[dbg_n++] = clock64();
   };
   stamp();
   timeline_mark(p.tl, p.tl_id, false);
@@ -293,7 +328,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   auto i_setup = [&]() {
     int r0 = gemm_row0<EPI, KH>(p, i_rb, warp);
     i_size = r0 >= 0 ? 16 : 0;  // rows beyond the matrix: zero-fill, nothing is read
-    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)(r0 >= 0 ? (r0 >> 4) : 0) * kpr + kb_lo + khalf) * 512 + lane * 8);
+    const int pt = r0 >= 0 ? packed_tile(p.perm, p.perm_a, p.perm_d, r0) : 0;
+    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)pt * kpr + kb_lo + khalf) * 512 + lane * 8);
   };
   i_setup();
   auto issue_unit = [&]() {
@@ -310,13 +346,14 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
     }
     cp_async_commit();
   };
-#pragma unroll
+#pragma unroll 1
   for (int s = 0; s < RING - 1; ++s) issue_unit();
 
   // the row table was written before this pass started, so the live row count can be read ahead of the predecessor
   const RowTable* tab = p.tab;
   int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
   if (n_cols > NTOK) n_cols = NTOK;
+  gemm_load_cols(p, n_cols, NTOK, s_ct);
   // the weights above are constants; everything below reads what earlier kernels of the pass produced
   stamp();
   if (tid == GEMM_THREADS - 1) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
@@ -331,25 +368,28 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
 
   // ---- activations of this CTA's k-range, copied asynchronously into MMA-fragment order: piece idx -> (plane s,
   // k-block kbl, column c, quarter tt).  Columns beyond the live rows are zero-filled without being read.
+  // Thread tid always copies quarter tt of column c; 256 threads cover 256 / (4 NTOK) k-blocks of one plane per
+  // round.  Dead columns are left as they are: an MMA output column depends on its own B column only, and dead
+  // columns are never read back.
   auto x_stage = [&](int kb0, int nkb) {
+    constexpr int KPR = GEMM_THREADS / (4 * NTOK);  // k-blocks per round
+    const int tt = tid & 3, c = (tid >> 2) % NTOK, kq = tid / (4 * NTOK);
+    if (c < n_cols) {
 #pragma unroll
-    for (int i = 0; i < PPT; ++i) {
-      const int idx = tid + i * GEMM_THREADS;
-      if (idx < PIECES) {
-        const int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % XCH, s = r / XCH;
-        const int k = (kb0 + kbl) * 32 + tt * 8;
-        const bool ok = kbl < nkb && k < p.K && c < n_cols;
-        cp_async16(xbuf + idx, ok ? p.xplanes + ((size_t)c * 3 + s) * p.x_ld + k : p.xplanes, ok);
+      for (int s = 0; s < 3; ++s) {
+        const __nv_bfloat16* src = p.xplanes + ((size_t)c * 3 + s) * p.x_ld + (kb0 + kq) * 32 + tt * 8;
+        uint4* dst = xbuf + ((s * XCH + kq) * NTOK + c) * 4 + tt;
+#pragma unroll
+        for (int j = 0; j < XCH; j += KPR) {
+          const int kbl = kq + j;
+          const bool ok = (kb0 + kbl) * 32 + tt * 8 < p.K;
+          if (kbl < nkb) cp_async16(dst + j * NTOK * 4, ok ? src + j * 32 : p.xplanes, ok);
+        }
       }
     }
     cp_async_commit();
   };
   const bool one_chunk = upt <= XCH;  // the whole k-range stays staged for every row block of this CTA
-  x_stage(kb_lo, min(XCH, upt));
-  gemm_rstd(p, n_cols, s_rstd);
-  cp_async_wait<0>();
-  __syncthreads();
-  stamp();
 
   float acc[3][NG][4];  // one chain per split term, the same for every NG: a row's bits must not depend on
                         // how many rows share the pass
@@ -361,6 +401,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
   };
+  float pre_h = 0.f, pre_g = 1.f;
+  float2 pre_rope = make_float2(1.f, 0.f);
   for (int task = 0; task < n_tasks; ++task) {
     const int rb = cid + task * p.n_clusters;
     const bool warp_valid = gemm_row0<EPI, KH>(p, rb, warp) >= 0;
@@ -372,11 +414,25 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
         for (int i = 0; i < 4; ++i) acc[h][n][i] = 0.f;
     for (int ck = 0; ck < upt; ck += XCH) {
       const int nkb = min(XCH, upt - ck);
-      if (!one_chunk) {  // wide passes (prefill): restage the activations chunk by chunk
-        __syncthreads();
+      const bool first = task == 0 && ck == 0;
+      if (first || !one_chunk) {  // wide passes (prefill) restage the activations chunk by chunk
+        if (!first) __syncthreads();
         x_stage(kb_lo + ck, nkb);
+        if (first) gemm_rstd(p, n_cols, s_rstd);
         cp_async_wait<0>();
         __syncthreads();
+        if (first) stamp();
+      }
+      if (ck == 0) {  // operands of this CTA's first output column, requested ahead of the main loop
+        const int c = rank + cs * (tid >> 7), jr = tid & 127;
+        if (EPI == EPI_RESID && c < n_cols && jr < RB_ROWS / KH) {
+          pre_h = p.hid[(size_t)s_ct[CT_HID * NTOK + c] * p.H + rb * (RB_ROWS / KH) + jr];
+          if (p.out_planes) pre_g = p.gain_next[rb * (RB_ROWS / KH) + jr];
+        }
+        if (EPI == EPI_QKV && c < n_cols && jr < 64) {
+          const int hd2 = p.head_dim >> 1;
+          pre_rope = p.rope[(size_t)s_ct[CT_POS * NTOK + c] * hd2 + jr % hd2];
+        }
       }
       const int kbl0 = (khalf + KH - (ck % KH)) % KH;  // this warp's first k-block of the chunk
       unsigned xk = xs_s + kbl0 * X_KB;
@@ -406,19 +462,11 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
 #pragma unroll
       for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
     stamp();
-    // the residual stream and the next gain of this CTA's first output column are requested before the barrier
-    float pre_h = 0.f, pre_g = 1.f;
-    if (EPI == EPI_RESID) {
-      const int c = rank + cs * (tid >> 7), jr = tid & 127;
-      if (c < n_cols && jr < RB_ROWS / KH) {
-        pre_h = p.hid[(size_t)tab->hid_idx[c] * p.H + rb * (RB_ROWS / KH) + jr];
-        if (p.out_planes) pre_g = p.gain_next[rb * (RB_ROWS / KH) + jr];
-      }
-    }
     gemm_push_tile<NG, KH>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
     stamp();
-    gemm_reduce_epilogue<EPI, KH>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank, pre_h, pre_g, EPI == EPI_RESID);
+    gemm_reduce_epilogue<EPI, KH>(p, s_ct, NTOK, rb, n_cols, recv, own_max, colbuf, s_rstd, rank, pre_h, pre_g, pre_rope,
+                                  EPI == EPI_RESID || EPI == EPI_QKV);
     stamp();
     if (task + 1 < n_tasks) cluster.sync();  // the owners are done with the receive buffer before it is refilled
   }
@@ -438,6 +486,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   float* recv = xf + XCH * NTOK * 32;                          // [cs][own_max][128]
   float* colbuf = recv + recv_floats(NG);
   float* s_rstd = colbuf + 2 * RB_ROWS;
+  int* s_ct = reinterpret_cast<int*>(s_rstd + NTOK);
 
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -454,6 +503,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
   if (n_cols > NTOK) n_cols = NTOK;
   if (n_cols <= 0) return;
+  gemm_load_cols(p, n_cols, NTOK, s_ct);
   gemm_rstd(p, n_cols, s_rstd);
 
   for (int task = 0; task < n_tasks; ++task) {
@@ -519,12 +569,12 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
         }
     gemm_push_tile<NG>(tot, recv, own_max, n_cols, cs, rank, cluster);
     cluster.sync();
-    gemm_reduce_epilogue<EPI>(p, tab, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+    gemm_reduce_epilogue<EPI>(p, s_ct, NTOK, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
     if (task + 1 < n_tasks) cluster.sync();
   }
 }
 __host__ __device__ constexpr int gemm_f32_smem_bytes(int NG) {
-  return 4 * 8 * NG * 32 * 4 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 + 64;
+  return 4 * 8 * NG * 32 * 4 + recv_floats(NG) * 4 + 2 * RB_ROWS * 4 + 8 * NG * 4 * (1 + CT_FIELDS) + 64;
 }
 
 // ---- one-time repacking of a bf16 weight matrix [N][K] into the tile-major streaming layout ----------------
@@ -535,6 +585,7 @@ struct PackParams {
   const __nv_bfloat16* src;  // [N][K]
   __nv_bfloat16* dst;        // [N/16][kpr][2][32][8]
   int N, K, kpr;
+  int perm, perm_a, perm_d;  // row tile order (see packed_tile)
 };
 __global__ void pack_weights_kernel(const __grid_constant__ PackParams p) {
   const size_t n_pieces = (size_t)(p.N / 16) * p.kpr * 64;
@@ -544,7 +595,7 @@ __global__ void pack_weights_kernel(const __grid_constant__ PackParams p) {
     const int kb = (int)(unit % p.kpr);
     const size_t rt = unit / p.kpr;
     const int g = lane >> 2, t = lane & 3;
-    const size_t row = rt * 16 + g + 8 * hi;
+    const size_t row = (size_t)packed_tile_row0(p.perm, p.perm_a, p.perm_d, (int)rt) + g + 8 * hi;
     const int k = kb * 32 + t * 8;
     uint4 v = make_uint4(0, 0, 0, 0);
     if (k < p.K) v = *reinterpret_cast<const uint4*>(p.src + row * p.K + k);

@@ -71,7 +71,7 @@ struct Layout {  // byte offsets into the workspace
 };
 
 struct Derived {
-  int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, max_chunks,
+  int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, sq_stride, max_chunks,
       trace_cap, Hq, Hkv, d1, d2;
   size_t gpart_floats, gcnt_ints;
 };
@@ -156,6 +156,7 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
   d->n_sq = m->hidden / (m->weight_dtype == 1 ? 64 : 128);  // residual row blocks: 64 rows (bf16 kernels), 128 (fp32)
+  d->sq_stride = std::max(d->n_sq, 64);  // room for one partial per cluster of the persistent pass kernel
   d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
   d->trace_cap = 4 * s->max_ctx + 64;
   d->Hq = m->n_q_heads * m->head_dim;
@@ -189,7 +190,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.xplanes = take(MR * 3 * m->hidden * 2);
   L.aplanes = take(MR * 3 * d.Hq * 2);
   L.splanes = take(MR * 3 * m->ffn * 2);
-  L.sumsq = take(MR * d.n_sq * 4);
+  L.sumsq = take(MR * d.sq_stride * 4);
   L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
   // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
@@ -247,6 +248,7 @@ struct loopspec_ctx {
   bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = false, l2pf_only_o = false;
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
+  bool pass_coop = true, use_perm = true;
   int launches_per_step = 0;
   std::string err;
 
@@ -380,7 +382,8 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.W = c->packed.empty() ? lp[1] : c->packed[4 * layer + 0], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden;
       // layer 0 reads the full sums the preparation kernel wrote; later layers the down-projection's partials
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.n_sq;
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.sq_stride;
+      if (!c->packed.empty() && c->use_perm) p.perm = 2, p.perm_a = m.head_dim / 32, p.perm_d = m.head_dim;
       p.qbuf = c->at<float>(c->L.qbuf);
       p.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)layer * c->kv_layer_stride();
       p.kv_plane_stride = c->kv_plane_stride(), p.kv_sel_stride = c->kv_sel_stride();
@@ -390,19 +393,20 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
     case G_O:
       p.W = c->packed.empty() ? lp[2] : c->packed[4 * layer + 1], p.N = m.hidden, p.K = d.Hq;
       p.xplanes = c->at<__nv_bfloat16>(c->L.aplanes), p.x_ld = d.Hq;
-      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.sq_stride;
       p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(lp[3]);
       break;
     case G_GU:
       p.W = c->packed.empty() ? lp[4] : c->packed[4 * layer + 2], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
+      if (!c->packed.empty() && c->use_perm) p.perm = 1, p.perm_a = m.ffn;
       p.xplanes = xpl, p.x_ld = m.hidden;
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.n_sq;
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.sq_stride;
       p.out_planes = c->at<__nv_bfloat16>(c->L.splanes), p.planes_ld = m.ffn;
       break;
     case G_DOWN:
       p.W = c->packed.empty() ? lp[5] : c->packed[4 * layer + 3], p.N = m.hidden, p.K = m.ffn;
       p.xplanes = c->at<__nv_bfloat16>(c->L.splanes), p.x_ld = m.ffn;
-      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.n_sq;
+      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.sq_stride;
       if (layer + 1 < m.n_recurrent) {
         p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(c->layers[6 * (layer + 1)]);
       }
@@ -434,25 +438,32 @@ cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
   memset(&q, 0, sizeof q);
   q.tab = tab, q.hid = c->at<float>(c->L.hid), q.K = c->m.hidden, q.planes = c->at<__nv_bfloat16>(c->L.xplanes);
   if (readout) q.gain = c->final_norm, q.sumsq = c->at<float>(c->L.sumsq_ro), q.sq_stride = 1, q.readout_only = 1;
-  else q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.n_sq;
+  else q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.sq_stride;
   return launch_k(prep_planes_kernel, dim3(c->d.max_rows), dim3(256), 0, c->stream, q, c->use_pdl);
 }
 
 
 using PassFn = void (*)(const PassParams);
 PassFn pass_fn(int d, int G) {
-  if (d == 128) return G == 1 ? pass_kernel<1, 128, 1> : pass_kernel<1, 128, 4>;
-  return G == 1 ? pass_kernel<1, 64, 1> : pass_kernel<1, 64, 4>;
+  if (d == 128) return G == 1 ? pass_kernel<128, 1> : pass_kernel<128, 4>;
+  return G == 1 ? pass_kernel<64, 1> : pass_kernel<64, 4>;
+}
+
+void pass_launch_config(loopspec_ctx* c, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int n_clusters) {
+  memset(cfg, 0, sizeof *cfg);
+  cfg->gridDim = dim3(n_clusters * PASS_CS), cfg->blockDim = dim3(PASS_THREADS), cfg->dynamicSmemBytes = pass_smem_bytes();
+  cfg->stream = c->stream;
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = PASS_CS, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they meet at grid barriers
+  at[1].val.cooperative = 1;
+  cfg->attrs = at, cfg->numAttrs = c->pass_coop ? 2 : 1;
 }
 
 cudaError_t launch_pass(loopspec_ctx* c, const PassParams& pp) {
   cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3(c->pass_grid), cfg.blockDim = dim3(PASS_THREADS), cfg.dynamicSmemBytes = pass_smem_bytes(1), cfg.stream = c->stream;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they meet at grid barriers
-  at[0].val.cooperative = 1;
-  cfg.attrs = at, cfg.numAttrs = 1;
+  cudaLaunchAttribute at[2];
+  pass_launch_config(c, &cfg, at, pp.n_clusters);
   return cudaLaunchKernelEx(&cfg, pass_fn(c->m.head_dim, c->m.n_q_heads / c->m.n_kv_heads), pp);
 }
 
@@ -465,7 +476,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   if ((e = launch_prep(c, tab, false))) return e;
   if (n_launch) *n_launch += 1;
   if (c->use_mega && ng == 1) {
-    if ((e = cudaMemsetAsync(c->ws + c->L.bar, 0, 4, c->stream))) return e;
+    if ((e = cudaMemsetAsync(c->ws + c->L.bar, 0, 8, c->stream))) return e;
     PassParams pp = c->pass;
     pp.tab = tab;
     if ((e = launch_pass(c, pp))) return e;
@@ -764,10 +775,12 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // bf16 weights: repack every matrix once into the tile-major streaming layout held in the workspace
   if (m->weight_dtype == 1) {
     unsigned char* dst = c->ws + L.wpack;
-    auto pack = [&](const void* src, int N, int K) -> bool {
+    if (getenv("LOOPSPEC_NOPERM")) c->use_perm = false;  // tuning aid
+    auto pack = [&](const void* src, int N, int K, int perm = 0, int perm_a = 0) -> bool {
+      if (!c->use_perm) perm = 0;
       PackParams pp;
       pp.src = static_cast<const __nv_bfloat16*>(src), pp.dst = reinterpret_cast<__nv_bfloat16*>(dst), pp.N = N, pp.K = K;
-      pp.kpr = (K + 31) / 32;
+      pp.kpr = (K + 31) / 32, pp.perm = perm, pp.perm_a = perm_a, pp.perm_d = m->head_dim;
       pack_weights_kernel<<<n_sm * 8, 256, 0, c->stream>>>(pp);
       c->packed.push_back(dst);
       dst += packed_bytes(N, K);
@@ -776,19 +789,27 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     bool ok = true;
     for (int l = 0; l < m->n_recurrent && ok; ++l) {
       const void* const* lp = &c->layers[6 * l];
-      ok = pack(lp[1], d.Hq + 2 * d.Hkv, m->hidden) && pack(lp[2], m->hidden, d.Hq) && pack(lp[4], 2 * m->ffn, m->hidden) &&
-           pack(lp[5], m->hidden, m->ffn);
+      // rotary partners (QKV) and gate/up partners are stored as adjacent row tiles
+      ok = pack(lp[1], d.Hq + 2 * d.Hkv, m->hidden, 2, m->head_dim / 32) && pack(lp[2], m->hidden, d.Hq) &&
+           pack(lp[4], 2 * m->ffn, m->hidden, 1, m->ffn) && pack(lp[5], m->hidden, m->ffn);
     }
     ok = ok && pack(c->lm_head, m->vocab, m->hidden);
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
   }
   // persistent pass kernel: available for bf16 weights when a decode pass carries at most 8 rows
-  if (m->weight_dtype == 1 && c->ng_dec == 1) {
+  if (m->weight_dtype == 1 && c->use_perm && c->ng_dec == 1 && m->ffn % 16 == 0 && m->head_dim % 32 == 0 && m->hidden % 16 == 0) {
     PassFn fn = pass_fn(m->head_dim, m->n_q_heads / m->n_kv_heads);
-    int per_sm = 0;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pass_smem_bytes(1)) == cudaSuccess &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, PASS_THREADS, pass_smem_bytes(1)) == cudaSuccess && per_sm >= 1) {
-      c->pass_grid = n_sm * std::min(per_sm, 2);
+    int max_clusters = 0;
+    if (const char* env = getenv("LOOPSPEC_NOCOOP")) c->pass_coop = env[0] != '1';  // tuning aid
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute at[2];
+    pass_launch_config(c, &cfg, at, 1);
+    cfg.numAttrs = 1;  // the occupancy query takes the cluster shape only
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pass_smem_bytes()) == cudaSuccess &&
+        cudaOccupancyMaxActiveClusters(&max_clusters, fn, &cfg) == cudaSuccess && max_clusters >= 1) {
+      int nc = std::min(max_clusters, d.sq_stride);
+      if (const char* env = getenv("LOOPSPEC_NC")) nc = std::max(1, std::min(nc, atoi(env)));  // tuning aid
+      c->pass_grid = nc * PASS_CS;
       std::vector<const void*> tabs((size_t)m->n_recurrent * 10);
       for (int l = 0; l < m->n_recurrent; ++l) {
         for (int i = 0; i < 4; ++i) tabs[(size_t)l * 4 + i] = c->packed[(size_t)l * 4 + i];
@@ -799,36 +820,34 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         return bail(LOOPSPEC_ECUDA, "pointer table upload");
       PassParams& q = c->pass;
       memset(&q, 0, sizeof q);
-      q.L = m->n_recurrent;
+      q.L = m->n_recurrent, q.n_clusters = nc;
       q.wpacked = c->at<const void*>(L.ptrs), q.layer_w = c->at<const void*>(L.ptrs) + (size_t)m->n_recurrent * 4;
       q.H = m->hidden, q.Hq = d.Hq, q.Hkv = d.Hkv, q.F = m->ffn, q.n_q_heads = m->n_q_heads, q.n_kv_heads = m->n_kv_heads;
       q.head_dim = m->head_dim, q.slots = d.slots, q.eps = m->rms_eps, q.scale = 1.0f / sqrtf((float)m->head_dim);
       q.hid = c->at<float>(L.hid), q.xplanes = c->at<__nv_bfloat16>(L.xplanes), q.aplanes = c->at<__nv_bfloat16>(L.aplanes);
-      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq), q.n_sq = m->hidden / 128;
-      q.sq_stride = d.n_sq;
+      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq);
+      q.sq_stride = d.sq_stride;
       q.kv = c->at<__nv_bfloat16>(L.kv), q.kv_layer_stride = c->kv_layer_stride(), q.kv_plane_stride = c->kv_plane_stride();
       q.kv_sel_stride = c->kv_sel_stride(), q.rope = c->at<float2>(L.rope);
-      q.gpart = c->at<float>(L.gpart), q.gcnt = c->at<int>(L.gcnt), q.apart = c->at<float>(L.apart), q.acnt = c->at<int>(L.acnt);
+      q.apart = c->at<float>(L.apart), q.acnt = c->at<int>(L.acnt);
       q.max_chunks = d.max_chunks, q.bar = c->at<unsigned>(L.bar), q.err = c->host_flags_dev + HF_ERROR;
-      const int Ns[4] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden};
+      // stages: tile groups (rotary pairs, single tiles, gate/up pairs, single tiles)
+      const int groups[4] = {(m->n_q_heads + 2 * m->n_kv_heads) * (m->head_dim / 32), m->hidden / 16, m->ffn / 16, m->hidden / 16};
+      const int pairs[4] = {1, 0, 1, 0};
       bool fits = true;
       for (int i = 0; i < 4; ++i) {
-        q.n_rb[i] = (i == 1 || i == 3) ? m->hidden / 128 : n_rbs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.N[i] = Ns[i], q.K[i] = Ks[i];
-        int total = q.n_rb[i] * q.kpr[i];
-        q.upc[i] = (total + c->pass_grid - 1) / c->pass_grid;
-        int mc = 1;
-        for (int rb = 0; rb < q.n_rb[i]; ++rb)
-          mc = std::max(mc, ((rb + 1) * q.kpr[i] - 1) / q.upc[i] - (rb * q.kpr[i]) / q.upc[i] + 1);
-        q.max_contrib[i] = mc;
-        if ((size_t)q.n_rb[i] * mc > (size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4) fits = false;
+        q.n_groups[i] = groups[i], q.paired[i] = pairs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.K[i] = Ks[i];
+        const int nt_max = ((groups[i] + nc - 1) / nc) << pairs[i];  // row tiles of the busiest cluster
+        q.kh[i] = nt_max <= PASS_TPW * 4 ? 2 : 1;
+        if (nt_max > PASS_TPW * 8 || (!pairs[i] && nt_max * 16 > PASS_THREADS)) fits = false;
+        if ((q.kpr[i] + PASS_CS - 1) / PASS_CS > PASS_XCH) fits = false;
       }
-      // measured slower than the chain of cluster kernels (its stage hand-over through global partials and a
-      // grid barrier costs more than a kernel boundary), so it is opt-in: LOOPSPEC_MEGA=1
-      c->use_mega = false;
+      c->use_mega = false;  // opt-in: LOOPSPEC_MEGA=1
       if (const char* env = getenv("LOOPSPEC_MEGA")) c->use_mega = fits && env[0] == '1';
       if (getenv("LOOPSPEC_DBG")) {  // tuning aid: timestamps land in the unused tail of the partial buffer
         q.dbg = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + (1 << 20);
-        fprintf(stderr, "LOOPSPEC_DBG offset %zu\n", L.gpart + ((size_t)8 << 20));
+        fprintf(stderr, "LOOPSPEC_DBG offset %zu clusters %d (max %d) kh %d %d %d %d fits %d\n", L.gpart + ((size_t)8 << 20), nc, max_clusters,
+                q.kh[0], q.kh[1], q.kh[2], q.kh[3], (int)fits);
       }
     }
   }
@@ -1158,6 +1177,7 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
   if (launch_k(prep_planes_kernel, dim3(M), dim3(256), 0, st, q, false) != cudaSuccess) return LOOPSPEC_ECUDA;
   if (weight_dtype == 1) {  // stream from a tile-major copy, as the decode path does
     PackParams pp;
+    memset(&pp, 0, sizeof pp);
     pp.src = static_cast<const __nv_bfloat16*>(W), pp.N = N, pp.K = K, pp.kpr = (K + 31) / 32;
     pp.dst = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(scratch) + align_up((size_t)M * 3 * K * 2));
     pack_weights_kernel<<<296, 256, 0, st>>>(pp);

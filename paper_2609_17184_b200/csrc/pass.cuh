@@ -1,25 +1,34 @@
 // One persistent kernel for a whole batched pass through the shared block stack (Sec. 4.2 step 1): for every
 // layer QKV -> attention -> O -> gate/up -> down, separated by grid barriers instead of kernel boundaries.
 //
-// Why: each of the 5 x L stages streams only 1.3-7 us worth of weights, so hand-over latency between stages
-// decides the pass time.  Here every CTA walks a fixed, precomputed sequence of weight units (stream-K shares
-// of every stage of every layer) and keeps RING units of it in flight in a thread-private cp.async ring that
-// never drains at a stage boundary: while a CTA waits at a barrier or gathers activations, the weights of its
-// next stage are already arriving.
+// Why: each of the 5 x L stages streams only 1.3-7 us worth of weights, so the latency between stages decides
+// the pass time.  Here every warp walks a fixed sequence of weight units (all stages of all layers) and keeps
+// RING units of it in flight in a thread-private cp.async ring that never drains at a stage boundary: while a
+// CTA waits at a barrier, stages activations or reduces partial sums, the weights of its next stage arrive.
 //
-// Every stage is cut into equal contiguous shares of (row block x k-block) units, one per CTA.  A row block
-// shared by several CTAs is summed in fixed order by the CTA that finishes it last (a counter per row block),
-// which then runs the stage's epilogue.  Data written by other CTAs is read with L2 loads (ld.global.cg).
-// The barrier is a monotonic counter; a CTA that waits longer than a bound raises an error flag and leaves.
+// Decomposition.  The grid is n_clusters thread-block clusters of 8 CTAs.  In every stage a cluster owns a
+// contiguous set of output row tiles (16 rows each; rotary partners and gate/up partners are adjacent tiles of
+// the packed weights, so a cluster always holds both) and its 8 CTAs split K into equal contiguous ranges.  A
+// warp carries up to three row tiles through its k-blocks (activation fragments are loaded once per k-block
+// and reused for the tiles).  Partial sums are pushed into the shared memory of the CTA that finishes the
+// token column (rank c finishes column c; distributed shared memory stores + one cluster barrier), summed in
+// rank order, and the stage's epilogue runs there.  No atomics on data, no global partials: bit-reproducible.
+// The grid barrier is a monotonic counter touched by one thread per cluster; a wait that exceeds its bound
+// raises an error flag and every later barrier falls through (no CTA leaves early, nothing can hang).
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "gemm.cuh"
 
 namespace ls {
 
 constexpr int PASS_THREADS = 256;
-constexpr int PASS_XCH = 24;           // k-blocks of activations staged at a time (NG = 1)
-constexpr unsigned PASS_SPIN_LIMIT = 1u << 22;
+constexpr int PASS_CS = 8;             // CTAs per cluster = K ranges per stage = token columns of a pass
+constexpr int PASS_TPW = 3;            // row tiles a warp carries through a stage
+constexpr int PASS_XCH = 24;           // k-blocks of activations a CTA stages (its whole k-range)
+constexpr int PASS_RECV_FLOATS = 8 * PASS_TPW * 8 * 16;  // [contribution][tile][16 rows] of one token column
+constexpr unsigned PASS_SPIN_LIMIT = 1u << 20;
 enum { ST_QKV = 0, ST_O = 1, ST_GU = 2, ST_DOWN = 3, N_STAGES = 4 };
 
 struct PassParams {
@@ -32,159 +41,45 @@ struct PassParams {
   float* hid;
   __nv_bfloat16 *xplanes, *aplanes, *splanes;
   float* qbuf;
-  float* sumsq;                 // [row][n_sq]
-  int n_sq, sq_stride;
+  float* sumsq;                 // [row][sq_stride]: one partial per cluster
+  int sq_stride;
   __nv_bfloat16* kv;            // whole pool
   long long kv_layer_stride, kv_plane_stride, kv_sel_stride;
   const float2* rope;
-  float* gpart;                 // split-k partial tiles [rb][max_contrib][8*NG][128]
-  int* gcnt;                    // [max n_rb]
   float* apart;                 // attention partials
   int* acnt;
   int max_chunks;
-  unsigned* bar;                // grid barrier counter, zero at launch
+  unsigned* bar;                // [0] barrier counter, [1] set once a wait ran out; both zero at launch
   volatile int* err;            // host-visible flag
   unsigned long long* dbg;      // optional: per-stage timestamps of CTA 0 (null in production)
-  int n_rb[N_STAGES], kpr[N_STAGES], upc[N_STAGES], max_contrib[N_STAGES], N[N_STAGES], K[N_STAGES];
+  int n_clusters;
+  // per stage: tile groups (pairs of partner tiles or single tiles), k-halves per CTA, k-blocks per row, K
+  int n_groups[N_STAGES], paired[N_STAGES], kh[N_STAGES], kpr[N_STAGES], K[N_STAGES];
 };
 
-__device__ __forceinline__ int pass_row0(const PassParams& p, int st, int rb, int warp) {
-  if (st == ST_GU) {
-    int j = rb * 64 + (warp & 3) * 16;
-    if (j >= p.F) return -1;
-    return (warp < 4) ? j : p.F + j;
+// what one warp does in a stage
+struct StageGeo {
+  int KH, WG, wg, khalf;  // k-halves per CTA; warps per k-half; this warp's place
+  int g_lo, nt;           // first tile group and number of row tiles of this cluster
+  int kb_lo, upt;         // k-range of this CTA
+  int kb0, nkb;           // this warp's k-blocks: kb0, kb0 + KH, ... (nkb of them)
+  int my_nt;              // row tiles of this warp: local tiles wg, wg + WG, ...
+  __device__ __forceinline__ void set(const PassParams& p, int st, int cid, int rank, int warp) {
+    KH = p.kh[st], WG = 8 / KH, wg = warp % WG, khalf = warp / WG;
+    const int ng = p.n_groups[st];
+    g_lo = (int)((long long)cid * ng / p.n_clusters);
+    const int g_hi = (int)((long long)(cid + 1) * ng / p.n_clusters);
+    nt = (g_hi - g_lo) << p.paired[st];
+    int kb_hi;
+    gemm_krange(p.kpr[st], PASS_CS, rank, kb_lo, kb_hi);
+    upt = kb_hi - kb_lo;
+    kb0 = kb_lo + khalf;
+    nkb = upt > khalf ? (upt - khalf + KH - 1) / KH : 0;
+    my_nt = nt > wg ? (nt - wg + WG - 1) / WG : 0;
   }
-  int r = rb * RB_ROWS + warp * 16;
-  return r < p.N[st] ? r : -1;
-}
-
-// position of one CTA in its unit sequence: (layer, stage, unit) and the matching pointer into the packed weights
-struct UnitCursor {
-  int l, st, u, u_end, rb, kb;
-  const __nv_bfloat16* ptr;
-  bool ok, done;
-  __device__ __forceinline__ void set_block(const PassParams& p, int warp, int lane) {
-    rb = u / p.kpr[st];
-    kb = u - rb * p.kpr[st];
-    int r0 = pass_row0(p, st, rb, warp);
-    ok = r0 >= 0;
-    const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(p.wpacked[l * 4 + st]);
-    ptr = W + (ok ? ((size_t)(r0 >> 4) * p.kpr[st] + kb) * 512 : 0) + lane * 8;
-  }
-  __device__ __forceinline__ void enter(const PassParams& p, int warp, int lane) {  // first non-empty stage from (l, st)
-    for (;;) {
-      if (l >= p.L) { done = true; return; }
-      int total = p.n_rb[st] * p.kpr[st];
-      u = min((int)blockIdx.x * p.upc[st], total);
-      u_end = min(u + p.upc[st], total);
-      if (u < u_end) { set_block(p, warp, lane); return; }
-      if (++st == N_STAGES) st = 0, ++l;
-    }
-  }
-  __device__ __forceinline__ void init(const PassParams& p, int warp, int lane) {
-    l = 0, st = 0, done = false;
-    enter(p, warp, lane);
-  }
-  __device__ __forceinline__ void next(const PassParams& p, int warp, int lane) {
-    ++u, ptr += 512;
-    if (u == u_end) {
-      if (++st == N_STAGES) st = 0, ++l;
-      enter(p, warp, lane);
-    } else if (++kb == p.kpr[st]) {
-      set_block(p, warp, lane);
-    }
-  }
+  // index of this cluster's first tile in the packed weights (partner tiles are adjacent there)
+  __device__ __forceinline__ int tile0(const PassParams& p, int st) const { return g_lo << p.paired[st]; }
 };
-
-// all CTAs arrive; returns false if the bound ran out (the kernel then leaves)
-__device__ __forceinline__ bool grid_barrier(const PassParams& p, unsigned& generation, int* s_ok) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    ++generation;
-    const unsigned target = generation * gridDim.x;
-    __threadfence();
-    atomicAdd(p.bar, 1u);
-    unsigned spins = 0;
-    int ok = 1;
-    while (*reinterpret_cast<volatile unsigned*>(p.bar) < target) {
-      if (++spins > PASS_SPIN_LIMIT) { ok = 0; *p.err = 4; break; }
-      __nanosleep(20);
-    }
-    __threadfence();
-    *s_ok = ok;
-  }
-  __syncthreads();
-  return *s_ok != 0;
-}
-
-// ---- epilogue of a finished row block (tile [col][TILE_LD] in shared memory) ----------------------------------
-__device__ __forceinline__ void pass_epilogue(const PassParams& p, const RowTable* tab, int l, int st, int rb, int n_cols,
-                                              const float* tile, const float* s_rstd) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (st == ST_O || st == ST_DOWN) {
-    const float* gain_next = nullptr;
-    if (st == ST_O) gain_next = static_cast<const float*>(p.layer_w[l * 6 + 3]);
-    else if (l + 1 < p.L) gain_next = static_cast<const float*>(p.layer_w[(l + 1) * 6 + 0]);
-    const int n0 = rb * RB_ROWS;
-    for (int c = warp; c < n_cols; c += PASS_THREADS / 32) {
-      float4* h = reinterpret_cast<float4*>(p.hid + (size_t)tab->hid_idx[c] * p.H + n0) + lane;
-      float4 v = __ldcg(h);
-      const float* tr = tile + c * TILE_LD + lane * 4;
-      v.x += tr[0], v.y += tr[1], v.z += tr[2], v.w += tr[3];
-      *h = v;
-      float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
-      if (lane == 0) p.sumsq[c * p.sq_stride + rb] = ss;
-      if (gain_next) {
-        float4 gn = *reinterpret_cast<const float4*>(gain_next + n0 + lane * 4);
-        float xv[4] = {v.x * gn.x, v.y * gn.y, v.z * gn.z, v.w * gn.w};
-        unsigned short hh[4], mm[4], ll[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) split3(xv[i], hh[i], mm[i], ll[i]);
-        __nv_bfloat16* dst = p.xplanes + (size_t)c * 3 * p.H + n0 + lane * 4;
-        *reinterpret_cast<uint2*>(dst) = make_uint2(hh[0] | ((unsigned)hh[1] << 16), hh[2] | ((unsigned)hh[3] << 16));
-        *reinterpret_cast<uint2*>(dst + p.H) = make_uint2(mm[0] | ((unsigned)mm[1] << 16), mm[2] | ((unsigned)mm[3] << 16));
-        *reinterpret_cast<uint2*>(dst + 2 * p.H) = make_uint2(ll[0] | ((unsigned)ll[1] << 16), ll[2] | ((unsigned)ll[3] << 16));
-      }
-    }
-  } else if (st == ST_GU) {
-    const int j0 = rb * 64;
-    for (int idx = tid; idx < n_cols * 64; idx += PASS_THREADS) {
-      int c = idx >> 6, jj = idx & 63;
-      if (j0 + jj < p.F) {
-        float gt = tile[c * TILE_LD + jj] * s_rstd[c], up = tile[c * TILE_LD + 64 + jj] * s_rstd[c];
-        store_split(p.splanes + (size_t)c * 3 * p.F, p.F, j0 + jj, gt / (1.0f + expf(-gt)) * up);
-      }
-    }
-  } else {  // ST_QKV
-    const int d = p.head_dim, hd2 = d >> 1;
-    const int n0 = rb * RB_ROWS;
-    const int region = n0 < p.Hq ? 0 : (n0 < p.Hq + p.Hkv ? 1 : 2);
-    const int base = region == 0 ? 0 : (region == 1 ? p.Hq : p.Hq + p.Hkv);
-    __nv_bfloat16* kvl = p.kv + (size_t)l * p.kv_layer_stride;
-    for (int idx = tid; idx < n_cols * 64; idx += PASS_THREADS) {
-      int c = idx >> 6, pr = idx & 63;
-      int hh = pr / hd2, i = pr - hh * hd2;
-      float x1 = tile[c * TILE_LD + hh * d + i] * s_rstd[c], x2 = tile[c * TILE_LD + hh * d + i + hd2] * s_rstd[c];
-      float y1 = x1, y2 = x2;
-      if (region < 2) {
-        float2 cs = p.rope[(size_t)tab->pos[c] * hd2 + i];
-        y1 = x1 * cs.x - x2 * cs.y;
-        y2 = x2 * cs.x + x1 * cs.y;
-      }
-      int head = (n0 - base) / d + hh;
-      if (region == 0) {
-        float* q = p.qbuf + (size_t)c * p.Hq + head * d + i;
-        q[0] = y1;
-        q[hd2] = y2;
-      } else {
-        __nv_bfloat16* dst = kvl + (size_t)(tab->r[c] - 1) * p.kv_plane_stride + (size_t)(region - 1) * p.kv_sel_stride +
-                             ((size_t)(tab->seq[c] * p.n_kv_heads + head) * p.slots + tab->kv_slot[c]) * d + i;
-        dst[0] = __float2bfloat16_rn(y1);
-        dst[hd2] = __float2bfloat16_rn(y2);
-      }
-    }
-  }
-}
 
 // ---- attention work item on one half of the CTA (128 threads, own named barrier) ----------------------------------
 struct AttnSmem {
@@ -361,42 +256,103 @@ __device__ __forceinline__ void pass_attention_item(const PassParams& p, const R
   }
 }
 
-__host__ __device__ constexpr int pass_xbuf_uint4(int NG) { return 3 * (PASS_XCH / NG) * 8 * NG * 4; }
-__host__ __device__ constexpr int pass_smem_bytes(int NG) {
-  return RING * 2 * PASS_THREADS * 16 + pass_xbuf_uint4(NG) * 16 + 8 * NG * TILE_LD * 4 + 8 * NG * 4 + 64;
+__host__ __device__ constexpr int pass_xbuf_uint4() { return 3 * PASS_XCH * 8 * 4; }
+__host__ __device__ constexpr int pass_smem_bytes() {
+  return RING * 2 * PASS_THREADS * 16 + pass_xbuf_uint4() * 16 + PASS_RECV_FLOATS * 4 + 16 * 4 + 64;
 }
 
-template <int NG, int D, int G>
+// all clusters arrive: one thread per cluster touches the counter, the cluster barrier fans the release out
+template <typename Stamp>
+__device__ __forceinline__ void pass_grid_barrier(const PassParams& p, cg::cluster_group& cluster, unsigned& generation, Stamp stamp) {
+  __threadfence();  // this thread's global writes of the stage are ordered before the arrival
+  stamp();
+  cluster.sync();
+  stamp();
+  ++generation;
+  if (cluster.block_rank() == 0 && threadIdx.x == 0) {
+    volatile unsigned* bar = p.bar;
+    if (bar[1] == 0) {
+      const unsigned target = generation * (unsigned)p.n_clusters;
+      __threadfence();
+      atomicAdd(p.bar, 1u);
+      unsigned spins = 0;
+      while (bar[0] < target) {
+        if (++spins > PASS_SPIN_LIMIT) {  // give up: flag it; every later barrier falls through
+          bar[1] = 1;
+          *p.err = 4;
+          break;
+        }
+        __nanosleep(40);
+      }
+      __threadfence();
+    }
+  }
+  stamp();
+  cluster.sync();
+}
+
+template <int D, int G>
 __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_constant__ PassParams p) {
-  constexpr int NTOK = 8 * NG;
-  constexpr int XCH = PASS_XCH / NG;
-  constexpr int PIECES = 3 * XCH * NTOK * 4;
+  constexpr int XCH = PASS_XCH;
+  constexpr int PIECES = 3 * XCH * 8 * 4;
   constexpr int PPT = (PIECES + PASS_THREADS - 1) / PASS_THREADS;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint4* ring = reinterpret_cast<uint4*>(smem_raw);
-  uint4* xbuf = ring + RING * 2 * PASS_THREADS;
-  float* tile = reinterpret_cast<float*>(xbuf + pass_xbuf_uint4(NG));
-  float* s_rstd = tile + NTOK * TILE_LD;
-  AttnSmem* asm_ = reinterpret_cast<AttnSmem*>(xbuf);  // the activation buffer is idle during attention
-  static_assert(2 * sizeof(AttnSmem) <= (size_t)pass_xbuf_uint4(NG) * 16, "attention scratch must fit the activation buffer");
-  int* s_flag = reinterpret_cast<int*>(s_rstd + NTOK);
-  int* s_ok = s_flag + 1;
+  uint4* ring = reinterpret_cast<uint4*>(smem_raw);               // [RING][2][256], slot of thread tid only
+  uint4* xbuf = ring + RING * 2 * PASS_THREADS;                   // [3][XCH][8][4]
+  float* recv = reinterpret_cast<float*>(xbuf + pass_xbuf_uint4());  // [8 * KH][nt][16]
+  float* s_rstd = recv + PASS_RECV_FLOATS;                        // [8]
+  float* s_red = s_rstd + 8;                                      // [8]
+  AttnSmem* asm_ = reinterpret_cast<AttnSmem*>(xbuf);             // the activation buffer is idle during attention
+  static_assert(2 * sizeof(AttnSmem) <= (size_t)pass_xbuf_uint4() * 16, "attention scratch must fit the activation buffer");
 
+  cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int rank = (int)cluster.block_rank(), cid = blockIdx.x / PASS_CS;
 
-  // ---- weight ring, issue side: runs RING-1 units ahead of the consumer, across stages and layers ----------------
-  UnitCursor ic;
-  ic.init(p, warp, lane);
-  int i_cnt = 0;
+  // ---- weight ring, issue side: runs RING-1 units ahead of the consumer, across stages and layers.  Order of a
+  // warp's units in a stage: k-blocks outermost, its row tiles innermost (the consumer below walks the same way).
+  constexpr unsigned SLOT_BYTES = 2 * PASS_THREADS * 16, RING_MASK = RING * SLOT_BYTES - 1, HI_OFF = PASS_THREADS * 16;
+  const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring) + tid * 16;
+  unsigned i_slot = 0;
+  int i_l = 0, i_st = 0, i_s = 0, i_n = 0, i_kleft = 0;
+  bool i_done = false;
+  const char* i_ptr = nullptr;
+  long long i_tile_stride = 0, i_k_rewind = 0;
+  auto i_enter = [&]() {  // first stage from (i_l, i_st) in which this warp has units
+    for (;;) {
+      if (i_l >= p.L) {
+        i_done = true;
+        return;
+      }
+      StageGeo ge;
+      ge.set(p, i_st, cid, rank, warp);
+      if (ge.my_nt > 0 && ge.nkb > 0) {
+        const int kpr = p.kpr[i_st];
+        const char* W = static_cast<const char*>(p.wpacked[i_l * 4 + i_st]);
+        i_ptr = W + ((size_t)(ge.tile0(p, i_st) + ge.wg) * kpr + ge.kb0) * 1024 + lane * 16;
+        i_tile_stride = (long long)ge.WG * kpr * 1024;                       // next row tile of this warp
+        i_k_rewind = (long long)ge.KH * 1024 - (long long)ge.my_nt * i_tile_stride;  // back to the first tile, next k-block
+        i_n = ge.my_nt, i_s = 0, i_kleft = ge.nkb;
+        return;
+      }
+      if (++i_st == N_STAGES) i_st = 0, ++i_l;
+    }
+  };
+  i_enter();
   auto issue_unit = [&]() {
-    if (!ic.done) {
-      uint4* slot = ring + (i_cnt & (RING - 1)) * 2 * PASS_THREADS + tid;
-      const __nv_bfloat16* W0 = static_cast<const __nv_bfloat16*>(p.wpacked[0]);
-      cp_async16(slot, ic.ok ? ic.ptr : W0, ic.ok);
-      cp_async16(slot + PASS_THREADS, ic.ok ? ic.ptr + 256 : W0, ic.ok);
-      ++i_cnt;
-      ic.next(p, warp, lane);
+    if (!i_done) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + i_slot), "l"(i_ptr) : "memory");
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + i_slot + HI_OFF), "l"(i_ptr + 512) : "memory");
+      i_slot = (i_slot + SLOT_BYTES) & RING_MASK;
+      i_ptr += i_tile_stride;
+      if (++i_s == i_n) {
+        i_s = 0, i_ptr += i_k_rewind;
+        if (--i_kleft == 0) {
+          if (++i_st == N_STAGES) i_st = 0, ++i_l;
+          i_enter();
+        }
+      }
     }
     cp_async_commit();
   };
@@ -407,179 +363,207 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
   pdl_wait();
 
   const RowTable* tab = p.tab;
-  int n_cols = min(tab->n_rows, NTOK);
+  const int n_cols = min(tab->n_rows, 8);
   if (n_cols <= 0) {  // every CTA takes this exit together: no barrier is ever entered
     cp_async_wait<0>();
     return;
   }
   unsigned generation = 0;
-  int j = 0;  // units consumed by this CTA so far (ring position)
+  unsigned c_slot = 0;
   int dbg_n = 0;
   auto stamp = [&]() {
-    if (p.dbg && blockIdx.x == 0 && tid == 0) {
+    if (kTune && p.dbg && blockIdx.x == 0 && tid == 0) {
       unsigned long long tns;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tns));
       p.dbg[dbg_n++] = tns;
     }
   };
+  auto lds128 = [](unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+  };
+  const unsigned xs_s = (unsigned)__cvta_generic_to_shared(xbuf) + (g * 4 + t) * 16;
+  constexpr unsigned X_KB = 8 * 64, X_PLANE = XCH * 8 * 64;  // bytes per k-block / per plane in xbuf
+  const int c_own = rank;  // the token column this CTA finishes
+  const bool own = c_own < n_cols;
 
   for (int l = 0; l < p.L; ++l) {
     for (int st = 0; st < N_STAGES; ++st) {
-      // ================= weight-streaming stage =================
-      const int kpr = p.kpr[st], total = p.n_rb[st] * kpr, upc = p.upc[st];
-      int u = min((int)blockIdx.x * upc, total);
-      const int u_end = min(u + upc, total);
       stamp();
-      if (u < u_end) {
+      StageGeo ge;
+      ge.set(p, st, cid, rank, warp);
+      const int kpr = p.kpr[st], nt = ge.nt;
+      const bool paired = p.paired[st] != 0;
+      // ---- activations of this CTA's k-range -> MMA-fragment order (live columns only), 1/rms of the columns
+      {
         const __nv_bfloat16* xsrc = st == ST_O ? p.aplanes : (st == ST_DOWN ? p.splanes : p.xplanes);
         const int x_ld = p.K[st];
-        const bool normed = (st == ST_QKV || st == ST_GU);
-        if (tid < n_cols) {
-          float r = 1.0f;
-          if (normed) {
-            const int n_sq = (st == ST_QKV && l == 0) ? 1 : p.n_sq;
-            float ss = 0.f;
-            for (int q = 0; q < n_sq; ++q) ss += __ldcg(p.sumsq + tid * p.sq_stride + q);
-            r = 1.0f / sqrtf(ss / (float)p.H + p.eps);
+#pragma unroll
+        for (int i = 0; i < PPT; ++i) {
+          const int idx = tid + i * PASS_THREADS;
+          if (idx < PIECES) {
+            const int tt = idx & 3, c = (idx >> 2) & 7, r = idx >> 5, kbl = r % XCH, s = r / XCH;
+            const int k = (ge.kb_lo + kbl) * 32 + tt * 8;
+            const bool ok = kbl < ge.upt && k < x_ld && c < n_cols;
+            cp_async16(xbuf + idx, ok ? xsrc + ((size_t)c * 3 + s) * x_ld + k : xsrc, ok);
           }
-          s_rstd[tid] = r;
         }
-        while (u < u_end) {
-          const int rb = u / kpr, kb0 = u - rb * kpr;
-          const int seg_len = min(kpr - kb0, u_end - u);
-          const bool warp_valid = pass_row0(p, st, rb, warp) >= 0;
-          float acc[3][NG][4];
+        cp_async_commit();
+        stamp();
+        const bool normed = (st == ST_QKV || st == ST_GU);
+        {  // warp c sums the partial sums of squares of column c in a fixed order
+          const int c = warp;
+          float ss = 0.f;
+          if (normed && c < n_cols) {
+            const int n_sq = (st == ST_QKV && l == 0) ? 1 : p.n_clusters;
+            for (int j = lane; j < n_sq; j += 32) ss += __ldcg(p.sumsq + c * p.sq_stride + j);
+          }
+          ss = warp_sum(ss);
+          if (lane == 0) s_rstd[c] = normed ? 1.0f / sqrtf(ss / (float)p.H + p.eps) : 1.0f;
+        }
+        stamp();
+        cp_async_wait<0>();
+        stamp();
+        __syncthreads();
+        stamp();
+      }
+      // ---- main loop: this warp's row tiles over its k-blocks
+      float acc[3][PASS_TPW][4];
 #pragma unroll
-          for (int h = 0; h < 3; ++h)
+      for (int h = 0; h < 3; ++h)
 #pragma unroll
-            for (int n = 0; n < NG; ++n)
+        for (int s = 0; s < PASS_TPW; ++s)
 #pragma unroll
-              for (int i = 0; i < 4; ++i) acc[h][n][i] = 0.f;
-          for (int ck = 0; ck < seg_len; ck += XCH) {
-            const int nkb = min(XCH, seg_len - ck);
-            uint4 xr[PPT];
+          for (int i = 0; i < 4; ++i) acc[h][s][i] = 0.f;
+      {
+        unsigned xk = xs_s + ge.khalf * X_KB;
+        for (int kk = 0; kk < ge.nkb; ++kk) {
+          const uint4 b0 = lds128(xk), b1 = lds128(xk + X_PLANE), b2 = lds128(xk + 2 * X_PLANE);
 #pragma unroll
-            for (int i = 0; i < PPT; ++i) {
-              const int idx = tid + i * PASS_THREADS;
-              const int tt = idx & 3, c = (idx >> 2) % NTOK, r = idx / (4 * NTOK), kbl = r % XCH, s = r / XCH;
-              const int k = (kb0 + ck + kbl) * 32 + tt * 8;
-              xr[i] = make_uint4(0, 0, 0, 0);
-              if (idx < PIECES && kbl < nkb && c < n_cols && k < x_ld)
-                xr[i] = __ldcg(reinterpret_cast<const uint4*>(xsrc + ((size_t)c * 3 + s) * x_ld + k));
-            }
-            __syncthreads();  // everyone is done with the previous contents of xbuf
-#pragma unroll
-            for (int i = 0; i < PPT; ++i) {
-              const int idx = tid + i * PASS_THREADS;
-              if (idx < PIECES) xbuf[idx] = xr[i];
-            }
-            __syncthreads();
-            const uint4* xs = xbuf + g * 4 + t;
-            for (int kbl = 0; kbl < nkb; ++kbl, ++j) {
+          for (int s = 0; s < PASS_TPW; ++s) {
+            if (s < ge.my_nt) {
               issue_unit();
               cp_async_wait<RING - 1>();
-              if (warp_valid) {
-                const uint4* slot = ring + (j & (RING - 1)) * 2 * PASS_THREADS + tid;
-                const uint4 a_lo = slot[0], a_hi = slot[PASS_THREADS];
-#pragma unroll
-                for (int s = 0; s < 3; ++s) {
-#pragma unroll
-                  for (int n = 0; n < NG; ++n) {
-                    const uint4 b = xs[((s * XCH + kbl) * NTOK + n * 8) * 4];
-                    mma_bf16(acc[s][n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
-                    mma_bf16(acc[s][n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
-                  }
-                }
-              }
+              const uint4 a_lo = lds128(ring_s + c_slot), a_hi = lds128(ring_s + c_slot + HI_OFF);
+              c_slot = (c_slot + SLOT_BYTES) & RING_MASK;
+              mma_bf16(acc[0][s], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b0.x, b0.y);
+              mma_bf16(acc[0][s], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b0.z, b0.w);
+              mma_bf16(acc[1][s], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b1.x, b1.y);
+              mma_bf16(acc[1][s], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b1.z, b1.w);
+              mma_bf16(acc[2][s], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b2.x, b2.y);
+              mma_bf16(acc[2][s], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b2.z, b2.w);
             }
           }
-          // ---- publish this share of the row block; the last CTA to arrive sums all shares and finishes it --------
-          const int c_first = (rb * kpr) / upc, c_last = ((rb + 1) * kpr - 1) / upc;
-          const int n_contrib = c_last - c_first + 1;
-          const int rl = warp * 16 + g;
-          float tot[NG][4];
-#pragma unroll
-          for (int n = 0; n < NG; ++n)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) tot[n][i] = acc[0][n][i] + (acc[1][n][i] + acc[2][n][i]);
-          bool finish = true;
-          if (n_contrib == 1) {
-#pragma unroll
-            for (int n = 0; n < NG; ++n) {
-              const int c0 = n * 8 + 2 * t;
-              tile[c0 * TILE_LD + rl] = tot[n][0], tile[(c0 + 1) * TILE_LD + rl] = tot[n][1];
-              tile[c0 * TILE_LD + rl + 8] = tot[n][2], tile[(c0 + 1) * TILE_LD + rl + 8] = tot[n][3];
-            }
-            __syncthreads();
-          } else {
-            float* dst = p.gpart + ((size_t)rb * p.max_contrib[st] + ((int)blockIdx.x - c_first)) * (NTOK * RB_ROWS);
-#pragma unroll
-            for (int n = 0; n < NG; ++n) {
-              const int c0 = n * 8 + 2 * t;
-              if (c0 < n_cols) {
-                __stcg(dst + c0 * RB_ROWS + rl, tot[n][0]);
-                __stcg(dst + c0 * RB_ROWS + rl + 8, tot[n][2]);
-                if (c0 + 1 < n_cols) {
-                  __stcg(dst + (c0 + 1) * RB_ROWS + rl, tot[n][1]);
-                  __stcg(dst + (c0 + 1) * RB_ROWS + rl + 8, tot[n][3]);
-                }
-              }
-            }
-            __syncthreads();
-            if (tid == 0) {
-              __threadfence();
-              int old = atomicAdd(p.gcnt + rb, 1);
-              *s_flag = (old == n_contrib - 1);
-              __threadfence();
-            }
-            __syncthreads();
-            finish = *s_flag != 0;
-            if (finish) {
-              const float4* src = reinterpret_cast<const float4*>(p.gpart + (size_t)rb * p.max_contrib[st] * (NTOK * RB_ROWS));
-              for (int idx = tid; idx < n_cols * (RB_ROWS / 4); idx += PASS_THREADS) {
-                float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int o0 = 0; o0 < n_contrib; o0 += 4) {
-                  float4 v4[4];
-#pragma unroll
-                  for (int q = 0; q < 4; ++q)
-                    v4[q] = (o0 + q < n_contrib) ? __ldcg(src + (size_t)(o0 + q) * (NTOK * RB_ROWS / 4) + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) s4.x += v4[q].x, s4.y += v4[q].y, s4.z += v4[q].z, s4.w += v4[q].w;
-                }
-                const int c = idx / (RB_ROWS / 4), jj = (idx % (RB_ROWS / 4)) * 4;
-                float* tr = tile + c * TILE_LD + jj;
-                tr[0] = s4.x, tr[1] = s4.y, tr[2] = s4.z, tr[3] = s4.w;
-              }
-              if (tid == 0) p.gcnt[rb] = 0;
-              __syncthreads();
-            }
-          }
-          if (finish) pass_epilogue(p, tab, l, st, rb, n_cols, tile, s_rstd);
-          __syncthreads();
-          u += seg_len;
+          xk += X_KB * ge.KH;
         }
       }
       stamp();
-      if (!grid_barrier(p, generation, s_ok)) {
-        cp_async_wait<0>();
-        return;
+      // ---- the residual stream and next gain of this CTA's column are requested before the cluster barrier
+      const bool resid = (st == ST_O || st == ST_DOWN);
+      const float* gain_next = nullptr;
+      if (st == ST_O) gain_next = static_cast<const float*>(p.layer_w[l * 6 + 3]);
+      else if (st == ST_DOWN && l + 1 < p.L) gain_next = static_cast<const float*>(p.layer_w[(l + 1) * 6 + 0]);
+      float pre_h = 0.f, pre_g = 1.f;
+      float* h_ptr = nullptr;
+      const int n_glob = ge.g_lo * 16 + tid;  // single tiles: output row of thread tid
+      const bool live1 = resid && own && tid < nt * 16;
+      if (live1) {
+        h_ptr = p.hid + (size_t)tab->hid_idx[c_own] * p.H + n_glob;
+        pre_h = __ldcg(h_ptr);
+        if (gain_next) pre_g = gain_next[n_glob];
+      }
+      // ---- push the partial tiles to the ranks that finish the columns (hi + (mid + lo), fixed order)
+      {
+        const int v = rank * ge.KH + ge.khalf;  // contribution index: k-ranges in ascending order
+#pragma unroll
+        for (int s = 0; s < PASS_TPW; ++s) {
+          if (s < ge.my_nt) {
+            const int i = ge.wg + s * ge.WG;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int c = 2 * t + e;
+              if (c < n_cols) {
+                float* dst = cluster.map_shared_rank(recv, c) + ((size_t)v * nt + i) * 16 + g;
+                dst[0] = acc[0][s][e] + (acc[1][s][e] + acc[2][s][e]);
+                dst[8] = acc[0][s][2 + e] + (acc[1][s][2 + e] + acc[2][s][2 + e]);
+              }
+            }
+          }
+        }
       }
       stamp();
+      cluster.sync();
+      stamp();
+      // ---- finish column c_own: sum the contributions in order, epilogue
+      const int n_contrib = PASS_CS * ge.KH;
+      if (resid) {
+        float xn = 0.f;
+        if (live1) {
+          const float* src = recv + tid;
+          float v = src[0];
+          for (int q = 1; q < n_contrib; ++q) v += src[(size_t)q * nt * 16];
+          xn = pre_h + v;
+          *h_ptr = xn;
+          if (gain_next) store_split(p.xplanes + (size_t)c_own * 3 * p.H, p.H, n_glob, xn * pre_g);
+        }
+        const float ss = warp_sum(xn * xn);
+        if (lane == 0) s_red[warp] = ss;
+        __syncthreads();
+        if (own && tid == 0) {
+          float tsum = 0.f;
+          for (int w = 0; w < 8; ++w) tsum += s_red[w];
+          p.sumsq[c_own * p.sq_stride + cid] = tsum;
+        }
+      } else if (own && tid < nt * 8) {
+        const int gl = tid >> 4, r = tid & 15;
+        const float* sa = recv + (2 * gl) * 16 + r;
+        float a = sa[0], b = sa[16];
+        for (int q = 1; q < n_contrib; ++q) a += sa[(size_t)q * nt * 16], b += sa[(size_t)q * nt * 16 + 16];
+        a *= s_rstd[c_own], b *= s_rstd[c_own];
+        const int grp = ge.g_lo + gl;
+        if (st == ST_GU) {
+          store_split(p.splanes + (size_t)c_own * 3 * p.F, p.F, grp * 16 + r, a / (1.0f + expf(-a)) * b);
+        } else {  // QKV: group = (head, 16 rotary pairs); a, b are the two halves of the pairs
+          constexpr int TH = D / 32, HD2 = D / 2;
+          const int hh = grp / TH, i = (grp - hh * TH) * 16 + r;
+          const int region = hh < p.n_q_heads ? 0 : (hh < p.n_q_heads + p.n_kv_heads ? 1 : 2);
+          float y1 = a, y2 = b;
+          if (region < 2) {
+            const float2 csn = p.rope[(size_t)tab->pos[c_own] * HD2 + i];
+            y1 = a * csn.x - b * csn.y;
+            y2 = b * csn.x + a * csn.y;
+          }
+          if (region == 0) {
+            float* q = p.qbuf + (size_t)c_own * p.Hq + hh * D + i;
+            q[0] = y1;
+            q[HD2] = y2;
+          } else {
+            const int head = hh - p.n_q_heads - (region == 2 ? p.n_kv_heads : 0);
+            __nv_bfloat16* dst = p.kv + (size_t)l * p.kv_layer_stride + (size_t)(tab->r[c_own] - 1) * p.kv_plane_stride +
+                                 (size_t)(region - 1) * p.kv_sel_stride +
+                                 ((size_t)(tab->seq[c_own] * p.n_kv_heads + head) * p.slots + tab->kv_slot[c_own]) * D + i;
+            dst[0] = __float2bfloat16_rn(y1);
+            dst[HD2] = __float2bfloat16_rn(y2);
+          }
+        }
+      }
+      stamp();
+      pass_grid_barrier(p, cluster, generation, stamp);
       // ================= attention (after the QKV stage) =================
       if (st == ST_QKV) {
+        stamp();
         const int total_items = tab->attn_items * p.n_kv_heads;
         const int half = tid >> 7, htid = tid & 127;
         for (int item = (int)blockIdx.x * 2 + half; item < total_items; item += 2 * (int)gridDim.x)
           pass_attention_item<D, G>(p, tab, l, item, asm_[half], htid, 1 + half);
         stamp();
-        if (!grid_barrier(p, generation, s_ok)) {
-          cp_async_wait<0>();
-          return;
-        }
+        pass_grid_barrier(p, cluster, generation, stamp);
       }
     }
   }
   cp_async_wait<0>();
+  cluster.sync();  // nobody leaves while a sibling may still be addressed
 }
 
 }  // namespace ls
