@@ -141,6 +141,14 @@ __device__ __forceinline__ void timeline_mark(unsigned long long* tl, int id, bo
   }
 }
 
+// tuning aid for kernels without a timeline pointer of their own: a pointer set once by the host
+#ifdef LOOPSPEC_TUNE
+__device__ unsigned long long* g_tune_tl = nullptr;
+__device__ __forceinline__ void tune_mark(int id, bool end) { timeline_mark(g_tune_tl, id, end); }
+#else
+__device__ __forceinline__ void tune_mark(int, bool) {}
+#endif
+
 // programmatic dependent launch: wait for the kernels this launch depends on / let dependents start launching
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -60,16 +60,26 @@ __device__ __forceinline__ void nodes_store(const NodeSmem& s, const NodeTable& 
   }
 }
 
-// P of Eq. 1 for the Ouro layout: hidden state at depth 0 = embedding row of the prefix's last token
+// P of Eq. 1 for the Ouro layout: hidden state at depth 0 = embedding row of the prefix's last token.  All rows are
+// copied in one flat loop so that every load is in flight before the first store (H is a multiple of 128).  A node slot
+// freed and handed out again within one step appears twice in the list: the later entry is the live one.
 __device__ __forceinline__ void embed_rows(const int (*list)[2], int n, float* hid, int H, const void* embed, int wdt) {
-  for (int e = 0; e < n; ++e) {
-    float* dst = hid + (size_t)list[e][0] * H;
+  const int per_row = H / 8;  // 8 elements per thread and step
+  for (int idx = threadIdx.x; idx < n * per_row; idx += blockDim.x) {
+    const int e = idx / per_row, i = (idx - e * per_row) * 8;
+    bool superseded = false;
+    for (int e2 = e + 1; e2 < n; ++e2) superseded |= list[e2][0] == list[e][0];
+    if (superseded) continue;
+    float4* dst = reinterpret_cast<float4*>(hid + (size_t)list[e][0] * H + i);
     if (wdt == 1) {
-      const unsigned short* src = static_cast<const unsigned short*>(embed) + (size_t)list[e][1] * H;
-      for (int i = threadIdx.x; i < H; i += blockDim.x) dst[i] = bf16_bits_to_float(src[i]);
+      const uint4 w = *reinterpret_cast<const uint4*>(static_cast<const unsigned short*>(embed) + (size_t)list[e][1] * H + i);
+      dst[0] = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u), __uint_as_float(w.y << 16),
+                           __uint_as_float(w.y & 0xffff0000u));
+      dst[1] = make_float4(__uint_as_float(w.z << 16), __uint_as_float(w.z & 0xffff0000u), __uint_as_float(w.w << 16),
+                           __uint_as_float(w.w & 0xffff0000u));
     } else {
-      const float* src = static_cast<const float*>(embed) + (size_t)list[e][1] * H;
-      for (int i = threadIdx.x; i < H; i += blockDim.x) dst[i] = src[i];
+      const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(embed) + (size_t)list[e][1] * H + i);
+      dst[0] = src[0], dst[1] = src[1];
     }
   }
 }
@@ -129,16 +139,16 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
   __shared__ int s_sel_tok[MAX_ROWS], s_sel_aux[MAX_ROWS];
   __shared__ float s_sel_lse[MAX_ROWS], s_sel_z2[MAX_ROWS];
   __shared__ unsigned long long s_steps;
+  __shared__ int s_trace_n;
   const int tid = threadIdx.x;
   const int n_nodes = p.S * p.NB;
+  tune_mark(603, false);
   pdl_launch_dependents();
-  pdl_wait();
-  // everything the serial bookkeeping reads is pulled into shared memory with one round of parallel loads
-  if (tid < MAX_ROWS) {
-    s_sel_tok[tid] = p.sel_tok[tid], s_sel_aux[tid] = p.sel_aux[tid];
-    s_sel_lse[tid] = p.sel_lse[tid], s_sel_z2[tid] = p.sel_z2[tid];
-  }
+  // Everything the serial bookkeeping reads is pulled into shared memory with one round of parallel loads.  The branch
+  // table, the row table and the sequence state were last written by the previous step, so they are read while this
+  // step's readout kernels are still running; only the selection results have to wait for them.
   if (tid == MAX_ROWS) s_steps = p.ctr->steps;
+  if (tid == MAX_ROWS + 1) s_trace_n = *p.trace_n;
   nodes_load(nd, p.nodes, n_nodes);
   {
     const int* src = reinterpret_cast<const int*>(p.tab);
@@ -148,6 +158,11 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
   if (tid < p.S) {
     s_root[tid] = p.seqs.root[tid], s_nids[tid] = p.seqs.n_ids[tid], s_ndec[tid] = p.seqs.n_dec[tid];
     s_ntarget[tid] = p.seqs.n_target[tid], s_needv[tid] = p.seqs.need_verify[tid];
+  }
+  pdl_wait();
+  if (tid < MAX_ROWS) {
+    s_sel_tok[tid] = p.sel_tok[tid], s_sel_aux[tid] = p.sel_aux[tid];
+    s_sel_lse[tid] = p.sel_lse[tid], s_sel_z2[tid] = p.sel_z2[tid];
   }
   if (tid == 0) s_nemb = 0, s_err = 0;
   __syncthreads();
@@ -225,10 +240,11 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
   }
   __syncthreads();
   if (tid == 0) {
-    if (p.phases & PH_ADVANCE) {
-      p.ctr->steps += 1, p.ctr->rows_total += t.n_rows, p.ctr->readout_rows_total += t.n_readout;
-      if ((unsigned long long)t.n_rows > p.ctr->rows_max) p.ctr->rows_max = t.n_rows;
-      int k = *p.trace_n;
+    if (p.phases & PH_ADVANCE) {  // counters: no value is read back, so nothing here waits for memory
+      atomicAdd(&p.ctr->steps, 1ull), atomicAdd(&p.ctr->rows_total, (unsigned long long)t.n_rows);
+      atomicAdd(&p.ctr->readout_rows_total, (unsigned long long)t.n_readout);
+      atomicMax(&p.ctr->rows_max, (unsigned long long)t.n_rows);
+      const int k = s_trace_n;
       if (k < p.trace_cap) p.row_trace[k] = t.n_rows;
       *p.trace_n = k + 1;
     }
@@ -255,6 +271,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
     p.seqs.need_verify[tid] = s_needv[tid];
   }
   embed_rows(s_emb, s_nemb, p.hid, p.H, p.embed, p.weight_dtype);
+  tune_mark(603, true);
 }
 
 // ---- vanilla decoding (Fig. 1a): one row per sequence, R passes per token ---------------------------
@@ -407,8 +424,10 @@ struct KvCommitParams {
 
 __global__ void kv_commit_kernel(const __grid_constant__ KvCommitParams p) {
   // grid: (L, R, 2 * S); one CTA copies n_kv_heads rows of d bf16
+  tune_mark(604, false);
   pdl_launch_dependents();
   pdl_wait();
+  struct EndMark { __device__ ~EndMark() { tune_mark(604, true); } } end_mark;
   const int l = blockIdx.x, plane = blockIdx.y, sel = blockIdx.z & 1, s = blockIdx.z >> 1;
   const KvCopyCmd c = p.cmds[s];
   if (plane >= c.n_planes) return;

@@ -70,6 +70,7 @@ struct GemmParams {
   int slots, n_kv_heads, n_q_heads, head_dim;
   const float2* rope;     // [pos][d/2] (cos, sin)
   float* logits;          // LOGITS: [logit_idx][V]
+  float2* argpart;        // LOGITS: [column][row block] (largest logit of the block, its vocabulary index as int bits)
   int F;                  // SWIGLU: ffn width
   int perm, perm_a, perm_d;  // order of the row tiles in the packed weights (see packed_tile)
   const void* pf_ptr;     // region to prefetch into L2 for a later kernel of the chain (may be null)
@@ -177,6 +178,27 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
         if (EPI == EPI_PLAIN) p.out[(size_t)c * p.out_ld + n] = v;
         else p.logits[(size_t)ct[CT_LOGIT * ntok + c] * p.N + n] = v;
       }
+      if (EPI == EPI_LOGITS) {  // the block's largest logit (ties: lowest index), so that greedy selection reads
+                                // one partial per row block instead of the whole row
+        __shared__ float s_av[2][4];
+        __shared__ int s_ai[2][4];
+        float bv = (live && n < p.N) ? v : -INFINITY;
+        int bi = n;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (ov > bv || (ov == bv && oi < bi)) bv = ov, bi = oi;
+        }
+        if (lane == 0) s_av[half][hw] = bv, s_ai[half][hw] = bi;
+        __syncthreads();
+        if (c < n_cols && j == 0) {
+          for (int w = 1; w < 4; ++w)
+            if (s_av[half][w] > bv || (s_av[half][w] == bv && s_ai[half][w] < bi)) bv = s_av[half][w], bi = s_ai[half][w];
+          p.argpart[(size_t)c * p.n_rb + rb] = make_float2(bv, __int_as_float(bi));
+        }
+        __syncthreads();
+      }
     } else if (EPI == EPI_RESID) {
       const int n = rb * RBW + j;
       float xn = 0.f;
@@ -282,9 +304,11 @@ __device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float*
 
 // ======================================= bf16 weights: tensor cores ========================================
 template <int NG, int EPI>
-__global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
-  // the residual GEMMs have few output rows: 64-row blocks with two k-halves per CTA double the CTAs that stream
-  constexpr int KH = (EPI == EPI_RESID) ? 2 : 1;
+__global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? 96 : 255) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
+  // KH = 2 (64-row blocks, the warps of a CTA in two groups that alternate k-blocks) is supported by the helpers below
+  // and doubles the CTAs of a GEMM with few output rows; measured slower than 128-row blocks once the kernels of the
+  // chain overlap, so every epilogue runs with KH = 1
+  constexpr int KH = 1;
   constexpr int NTOK = 8 * NG;
   constexpr int XCH = xchunk_kblocks(NG);
 
@@ -306,6 +330,14 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   };
   stamp();
   timeline_mark(p.tl, p.tl_id, false);
+  if (kTune && p.tl && tid == 0 && (p.tl_id == 28 || p.tl_id == 29 || p.tl_id == 27)) {  // per-CTA start time and SM of one layer's kernels
+    unsigned long long tns;
+    unsigned smid;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tns));
+    asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+    p.tl[4096 + (p.tl_id - 27) * 1024 + blockIdx.x * 2] = tns;
+    p.tl[4096 + (p.tl_id - 27) * 1024 + blockIdx.x * 2 + 1] = smid;
+  }
   const int kpr = p.kb_per_rb;
   int kb_lo, kb_hi;
   gemm_krange(kpr, cs, rank, kb_lo, kb_hi);
@@ -346,7 +378,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
     }
     cp_async_commit();
   };
-#pragma unroll 1
+#pragma unroll
   for (int s = 0; s < RING - 1; ++s) issue_unit();
 
   // the row table was written before this pass started, so the live row count can be read ahead of the predecessor
@@ -472,6 +504,11 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_kernel(const __grid_co
   }
   cp_async_wait<0>();
   timeline_mark(p.tl, p.tl_id, true);
+  if (kTune && p.tl && tid == 0 && (p.tl_id == 28 || p.tl_id == 29 || p.tl_id == 27)) {
+    unsigned long long tns;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(tns));
+    p.tl[4096 + 3 * 1024 + (p.tl_id - 27) * 512 + blockIdx.x] = tns;
+  }
 }
 
 // ======================================= fp32 weights: CUDA cores ==========================================
@@ -619,6 +656,7 @@ struct PrepParams {
 
 __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant__ PrepParams p) {
   __shared__ float s_part[8];
+  tune_mark(600 + p.readout_only, false);
   pdl_launch_dependents();
   pdl_wait();
   const int c = blockIdx.x;
@@ -646,6 +684,7 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
     for (int w = 0; w < 8; ++w) tsum += s_part[w];
     p.sumsq[c * p.sq_stride] = tsum;
   }
+  tune_mark(600 + p.readout_only, true);
 }
 
 }  // namespace ls

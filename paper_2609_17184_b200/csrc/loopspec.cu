@@ -29,12 +29,16 @@ struct GemmPlan {
 // Cluster size = how many CTAs split K for one block of 128 output rows.  Enough CTAs to fill the resident
 // slots (two per SM), a k-range short enough that a decode pass keeps its activations staged once, and whole
 // rounds of row blocks per cluster so that every CTA streams the same number of bytes.
-GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only) {
+GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1) {
   GemmPlan g;
   g.n_rb = n_rb;
   g.kpr = (K + 31) / 32;
   int cs_min = (g.kpr + MAX_XCH_BLOCKS - 1) / MAX_XCH_BLOCKS;
   int cs = std::max(1, slots / std::max(n_rb, 1));
+  // a warp should keep at least 8 k-blocks: below that the fixed cost of a CTA (staging, reduction, epilogue)
+  // outweighs what more CTAs stream in parallel, and a smaller grid leaves room for the next kernel's CTAs to
+  // become resident (and prefetch) early  [measured: O projection, 8 -> 4 CTAs per cluster]
+  cs = std::min(cs, std::max(1, g.kpr / (8 * kh)));
   cs = std::max(cs, cs_min);
   cs = std::min(std::min(cs, 8), g.kpr);
   auto pow2_at_least = [&](int v) {
@@ -66,7 +70,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, argpart, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -155,7 +159,7 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->n_hid = d->S * d->NB + MAX_ROWS;
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
-  d->n_sq = m->hidden / (m->weight_dtype == 1 ? 64 : 128);  // residual row blocks: 64 rows (bf16 kernels), 128 (fp32)
+  d->n_sq = m->hidden / 128;  // row blocks of the residual GEMMs = partial sums of squares per row
   d->sq_stride = std::max(d->n_sq, 64);  // room for one partial per cluster of the persistent pass kernel
   d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
   d->trace_cap = 4 * s->max_ctx + 64;
@@ -193,6 +197,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sumsq = take(MR * d.sq_stride * 4);
   L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
+  L.argpart = take(MR * ((m->vocab + 127) / 128) * sizeof(float2));
   // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
   L.gpart = take((size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4 * MR * 128 * 4);
   L.ptrs = take((size_t)m->n_recurrent * 10 * sizeof(void*));
@@ -415,7 +420,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.W = c->packed.empty() ? c->lm_head : c->packed[4 * m.n_recurrent], p.N = m.vocab, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden, p.cols_from_readout = 1;
       p.sumsq = c->at<float>(c->L.sumsq_ro), p.n_sq = 1, p.sq_stride = 1;
-      p.logits = c->at<float>(c->L.logits);
+      p.logits = c->at<float>(c->L.logits), p.argpart = c->at<float2>(c->L.argpart);
       break;
   }
   return p;
@@ -520,7 +525,9 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
   cudaError_t e;
   if ((e = launch_prep(c, tab, true))) return e;
-  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gemm_params(c, G_LM, 0, tab), c->stream, c->use_pdl);
+  GemmParams gl = gemm_params(c, G_LM, 0, tab);
+  if (getenv("LOOPSPEC_DBG")) gl.tl = reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024, gl.tl_id = 120;  // tuning aid
+  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
 }
 
 cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) {
@@ -530,6 +537,7 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   sp.kinds_mask = kinds_mask;
   sp.sel_tok = c->at<int>(c->L.sel_tok), sp.sel_aux = c->at<int>(c->L.sel_aux);
   sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);
+  sp.argpart = c->at<float2>(c->L.argpart), sp.n_rb = c->plan[G_LM].n_rb;
   return launch_k(select_kernel, dim3(c->d.max_rows), dim3(SEL_THREADS), 0, c->stream, sp, c->use_pdl);
 }
 
@@ -676,6 +684,12 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   for (int i = 0; i < 6 * m->n_recurrent; ++i)
     if (!w->layer_ptrs[i]) return LOOPSPEC_EINVAL;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LOOPSPEC_EINVAL;
+  // every tensor is read with 16-byte loads
+  if ((reinterpret_cast<uintptr_t>(w->embed) & 15) || (w->lm_head && (reinterpret_cast<uintptr_t>(w->lm_head) & 15)) ||
+      (reinterpret_cast<uintptr_t>(w->final_norm) & 15))
+    return LOOPSPEC_EINVAL;
+  for (int i = 0; i < 6 * m->n_recurrent; ++i)
+    if (reinterpret_cast<uintptr_t>(w->layer_ptrs[i]) & 15) return LOOPSPEC_EINVAL;
   if (!cuda_stream) return LOOPSPEC_EINVAL;  // the legacy default stream cannot be captured into a graph
   int dev = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -693,12 +707,28 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * m->n_recurrent);
   c->ng_dec = ng_for_rows(d.max_rows_dec), c->ng_pf = ng_for_rows(d.max_rows_pf);
   c->prefilled.assign(d.S, 0);
-  const int resid_rows = m->weight_dtype == 1 ? 64 : 128;
+  const int resid_rows = 128;
   const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / resid_rows, (m->ffn + 63) / 64, m->hidden / resid_rows, (m->vocab + 127) / 128};
   const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
   int slots = n_sm * kCtasPerSm;
   if (const char* env = getenv("LOOPSPEC_SLOTS")) slots = std::max(1, atoi(env));  // tuning aid
   for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
+  if (const char* env = getenv("LOOPSPEC_NCL")) {  // tuning aid: clusters per GEMM "qkv,o,gateup,down,lmhead" (0 = keep)
+    int v[5];
+    if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
+      for (int i = 0; i < 5; ++i)
+        if (v[i] > 0 && v[i] <= c->plan[i].n_rb) c->plan[i].n_clusters = v[i], c->plan[i].grid = v[i] * c->plan[i].cs;
+  }
+  // Every kernel of the chain asks for the same (largest) shared-memory carve-out: the GEMM CTAs need it, and an SM
+  // whose partition was set by a small-shared-memory kernel would have to drain before it can host one.
+  if (!getenv("LOOPSPEC_NO_CARVEOUT")) {  // tuning aid
+    const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads), (const void*)prep_planes_kernel,
+                               (const void*)select_kernel, (const void*)control_kernel, (const void*)vanilla_control_kernel,
+                               (const void*)kv_commit_kernel};
+    for (const void* f : small_fns)
+      if (cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        (void)cudaGetLastError();
+  }
   for (int ng : {c->ng_dec, c->ng_pf})
     if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
@@ -709,7 +739,13 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
   if (const char* env = getenv("LOOPSPEC_L2PF")) c->use_l2pf = env[0] != '0', c->l2pf_only_o = env[0] == '2';  // tuning aid
-  if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
+  if (getenv("LOOPSPEC_DBG")) {
+    fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
+#ifdef LOOPSPEC_TUNE
+    unsigned long long* tl = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + 1024;
+    cudaMemcpyToSymbol(g_tune_tl, &tl, sizeof tl);
+#endif
+  }
   if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
     int v[5];
     if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
@@ -735,6 +771,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     cfg.attrs = at, cfg.numAttrs = 1;
     int n_active = 0;
     cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
+    if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gemm %d: cs %d clusters %d grid %d, max active clusters %d\n", i, g.cs, g.n_clusters, g.grid, n_active);
     if (e != cudaSuccess || n_active < 1) {
       (void)cudaGetLastError();
       g = plan_gemm(n_rbs[i], Ks[i], slots, true);

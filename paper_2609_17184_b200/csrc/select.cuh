@@ -27,6 +27,8 @@ struct SelectParams {
   int* sel_aux;         // RO_D2: gate open; RO_VERIFY: source 1/2/3
   float* sel_lse;       // RO_D1 / RO_D2: log-sum-exp of z/T
   float* sel_z2;        // RO_D2: normaliser of the residual proposal (0: the proposal is q2~ itself)
+  const float2* argpart;  // [readout column][row block]: per-block largest logit and its index, written by the lm_head
+  int n_rb;
 };
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
@@ -83,16 +85,35 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
   return r;
 }
 
+// argmax of the logits row of readout column `col` from the per-block maxima the lm_head epilogue left (ties to the
+// lowest index)
+__device__ __forceinline__ int greedy_argmax(const float2* argpart, int n_rb, int col, ArgMax* sh_am) {
+  ArgMax a = {-INFINITY, 0x7fffffff};
+  for (int b = threadIdx.x; b < n_rb; b += SEL_THREADS) {
+    const float2 v = __ldcg(argpart + (size_t)col * n_rb + b);
+    a = better(a, ArgMax{v.x, __float_as_int(v.y)});
+  }
+  return block_argmax(a, sh_am).i;
+}
+
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_constant__ SelectParams p) {
   __shared__ ArgMax sh_am[SEL_THREADS / 32];
   __shared__ float sh_f[SEL_THREADS / 32];
+  tune_mark(602, false);
   pdl_launch_dependents();
-  pdl_wait();
+  // the row table was written before this pass started: everything but the logits can be read ahead of the lm_head
   const RowTable* tab = p.tab;
-  if ((int)blockIdx.x >= tab->n_readout) return;
+  if ((int)blockIdx.x >= tab->n_readout) {  // every CTA waits: a kernel that ends early would release its dependents early
+    pdl_wait();
+    return;
+  }
+  struct EndMark { __device__ ~EndMark() { tune_mark(602, true); } } end_mark;
   const int row = tab->ro_rows[blockIdx.x];
   const int kind = tab->readout[row];
-  if (!((p.kinds_mask >> kind) & 1)) return;
+  if (!((p.kinds_mask >> kind) & 1)) {
+    pdl_wait();
+    return;
+  }
   const int V = p.V, tid = threadIdx.x;
   const float T = p.temperature;
   const float* z = p.logits + (size_t)tab->logit_idx[row] * V;
@@ -112,11 +133,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     s = block_sum(s, sh_f);
     return m + logf(s);
   };
-  auto greedy = [&](const float* zz) -> int {
-    ArgMax a = {-INFINITY, 0x7fffffff};
-    for (int v = tid; v < V; v += SEL_THREADS) a = better(a, ArgMax{zz[v], v});
-    return block_argmax(a, sh_am).i;
-  };
+  // greedy readouts are always taken from the row the lm_head just produced
+  auto greedy = [&](const float*) -> int { return greedy_argmax(p.argpart, p.n_rb, (int)blockIdx.x, sh_am); };
   // exponential race over weights given through logw(v) (-inf = zero weight)
   auto race = [&](auto logw, int purpose) -> int {
     ArgMax a = {-INFINITY, 0x7fffffff};
@@ -136,6 +154,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     return u01(philox4x32_10(make_uint4(0u, position, seq, (unsigned)purpose), key).x);
   };
 
+  pdl_wait();
   if (kind == RO_TARGET) {
     int tok = (T == 0.f) ? greedy(z) : race([&](int v) { return z[v] / T; }, PUR_VANILLA);
     if (tid == 0) p.sel_tok[row] = tok;
