@@ -29,7 +29,7 @@ import workloads as W  # noqa: E402
 
 # DRAM bytes (read + write) of ONE launch of the dominant kernel (gate/up GEMM, Ouro-1.4B shape, 4 rows),
 # taken from the ncu capture summarised in profiles/gemm_gateup_ouro1p4b.md.
-NCU_TRAFFIC_BYTES = {"ouro_1p4b": 46243072}  # profiles/gemm_gateup_ouro1p4b.md: 46.234 MB read + 0.009 MB written
+NCU_TRAFFIC_BYTES = {"ouro_1p4b": 46226944}  # profiles/gemm_gateup_ouro1p4b.md: dram bytes read + written per launch
 
 
 def measured_peaks():
