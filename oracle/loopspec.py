@@ -43,9 +43,10 @@ class Branch:                      # Algorithm 1: prefix X(b), hidden H_b, depth
 
 
 class Decoder:
-    def __init__(self, model, temperature=0.0, seed=0, seq=0, max_ctx=None):
+    def __init__(self, model, temperature=0.0, seed=0, seq=0, max_ctx=None, top_k=0, top_p=1.0):
         self.m = model
         self.T = float(temperature)
+        self.top_k, self.top_p = int(top_k), float(top_p)   # the optional filters of C (Sec. 3.1)
         self.seed, self.seq = seed, seq
         self.ids = []              # committed tokens (prompt + decoded)
         self.n_prompt = 0
@@ -68,7 +69,12 @@ class Decoder:
 
     # ---- readout C -----------------------------------------------------------------------------
     def probs(self, logits):
-        return nm.softmax(logits / self.T)
+        """C after the lm_head: temperature, optional top-k / top-p filtering, normalisation (Sec. 3.1)."""
+        p = nm.softmax(logits / self.T)
+        if self.top_k or self.top_p < 1.0:
+            p, margin = sp.top_k_top_p(p, self.top_k, self.top_p)
+            self.log.append(dict(kind="filter", margin=margin))
+        return p
 
     def _draw(self, weights, position, purpose):
         g = sp.gumbel(self.seed, self.seq, position, purpose, len(weights))
@@ -243,8 +249,9 @@ class Decoder:
                         q1 = b.records[0].q
                         q2t = self.probs(z2)
                         is_open = (q2t[x1] < q1[x1]) or not gate
-                        self.log.append(dict(kind="gate", pos=pos, open=is_open,
-                                             margin=abs(np.log(q2t[x1]) - np.log(q1[x1]))))
+                        with np.errstate(divide="ignore"):   # a filtered q2~ may give the candidate no mass
+                            gm = abs(np.log(q2t[x1]) - np.log(q1[x1]))
+                        self.log.append(dict(kind="gate", pos=pos, open=is_open, margin=gm))
                         if is_open:
                             q2 = sp.residual(q2t, q1) if residual_q2 else q2t
                             x2, margin = self._draw(q2, pos, sp.DRAFT2)

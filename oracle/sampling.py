@@ -9,7 +9,11 @@ sampler is lossless, Sec. 3.2):
   * uniform from a 32-bit word x: u = ((x >> 9) + 0.5) * 2^-23, in (0, 1);
   * categorical draw: exponential race / Gumbel-max, x = argmax_v log w_v + g_v,
     g_v = -log(-log u_v), u_v = word (v mod 4) of block v div 4; ties -> lowest v;
-  * acceptance uniforms: word 0 of block 0.
+  * acceptance uniforms: word 0 of block 0;
+  * the optional top-k / top-p filters of the post-layers C (Sec. 3.1): tokens are ranked by
+    decreasing probability (ties: lower index first); top-k keeps the first k and renormalises;
+    top-p then keeps the shortest prefix of that ranking whose mass reaches top_p and
+    renormalises.  The filtered distribution IS p_r, at every depth r.
 """
 import numpy as np
 
@@ -94,3 +98,36 @@ def residual(mu, nu):
 def accept_prob(rho, q, x):
     """min{1, rho(x)/q(x)} of Eq. 3 for a candidate x drawn from q (so q(x) > 0)."""
     return min(1.0, rho[x] / q[x])
+
+
+def top_k_top_p(p, top_k=0, top_p=1.0):
+    """The filters inside C (Sec. 3.1) applied to one probability vector.
+
+    Returns (filtered distribution, margin): margin is how far the decision "keep exactly this many
+    tokens" is from flipping - the smaller of the distance of the cumulative mass from top_p on
+    either side of the last kept token and, in probability units, the gap between the last kept
+    and the first dropped token (their order decides who is kept).
+    """
+    p = np.asarray(p, dtype=np.float64)
+    V = len(p)
+    order = np.lexsort((np.arange(V), -p))          # decreasing probability, then increasing index
+    margin = np.inf
+    m = V
+    if top_k and top_k < V:
+        m = int(top_k)
+        margin = min(margin, p[order[m - 1]] - p[order[m]])
+    kept = order[:m]
+    pk = p[kept] / p[kept].sum()
+    if top_p < 1.0:
+        cum = np.cumsum(pk)
+        j = int(np.searchsorted(cum, top_p, side="left")) + 1   # first prefix whose mass reaches top_p
+        j = min(j, m)
+        margin = min(margin, cum[j - 1] - top_p)
+        if j >= 2:
+            margin = min(margin, top_p - cum[j - 2])
+        if j < m:
+            margin = min(margin, pk[j - 1] - pk[j])
+        kept, pk = kept[:j], pk[:j] / pk[:j].sum()
+    out = np.zeros(V)
+    out[kept] = pk
+    return out, float(margin)

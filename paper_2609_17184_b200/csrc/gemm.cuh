@@ -27,8 +27,18 @@ enum { EPI_PLAIN = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_SWIGLU = 3, EPI_LOGITS = 4
 constexpr int GEMM_THREADS = 256;
 constexpr int RB_ROWS = 128;   // output rows per row block
 constexpr int TILE_LD = 132;   // padded leading dimension of the partial tile
-constexpr int RING = 8;        // weight stages in flight per thread (8 KB per stage per CTA)
-constexpr int MAX_XCH_BLOCKS = 24;  // k-blocks of activations one CTA keeps staged when NG = 1
+// shape of a GEMM CTA (overridable at build time for tuning): ring depth, staged k-blocks, register cap
+#ifndef LS_RING
+#define LS_RING 8
+#endif
+#ifndef LS_XCH
+#define LS_XCH 24
+#endif
+#ifndef LS_MAXREG
+#define LS_MAXREG 96
+#endif
+constexpr int RING = LS_RING;  // weight stages per thread (8 KB per stage per CTA), RING - 1 of them in flight
+constexpr int MAX_XCH_BLOCKS = LS_XCH;  // k-blocks of activations one CTA keeps staged when NG = 1
 // per-column copies of the row-table fields the epilogues need ([field][column] in shared memory)
 enum { CT_POS = 0, CT_R = 1, CT_SEQ = 2, CT_SLOT = 3, CT_HID = 4, CT_LOGIT = 5, CT_FIELDS = 6 };
 
@@ -304,7 +314,7 @@ __device__ __forceinline__ void gemm_push_tile(const float (&acc)[NG][4], float*
 
 // ======================================= bf16 weights: tensor cores ========================================
 template <int NG, int EPI>
-__global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? 96 : 255) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
+__global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG : 255) gemm_bf16_kernel(const __grid_constant__ GemmParams p) {
   // KH = 2 (64-row blocks, the warps of a CTA in two groups that alternate k-blocks) is supported by the helpers below
   // and doubles the CTAs of a GEMM with few output rows; measured slower than 128-row blocks once the kernels of the
   // chain overlap, so every epilogue runs with KH = 1
@@ -350,8 +360,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? 96 : 255) 
   // consumes per unit is contiguous and consecutive k-blocks of a 16-row tile follow each other, so every warp
   // streams one contiguous region and every request covers whole 128-byte lines.  The loop is kept to a few
   // instructions per unit: shared-memory addresses are 32-bit registers advanced by constants.
-  constexpr unsigned SLOT_BYTES = 2 * GEMM_THREADS * 16, RING_MASK = RING * SLOT_BYTES - 1, HI_OFF = GEMM_THREADS * 16;
-  static_assert((RING & (RING - 1)) == 0, "ring depth must be a power of two");
+  constexpr unsigned SLOT_BYTES = 2 * GEMM_THREADS * 16, RING_BYTES = RING * SLOT_BYTES, HI_OFF = GEMM_THREADS * 16;
   const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring) + tid * 16;
   const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
   const char* i_ptr = reinterpret_cast<const char*>(Wb);
@@ -370,7 +379,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? 96 : 255) 
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(ring_s + i_slot + HI_OFF), "l"(i_ptr + 512), "r"(i_size)
                    : "memory");
       i_ptr += 1024 * KH;
-      i_slot = (i_slot + SLOT_BYTES) & RING_MASK;
+      i_slot += SLOT_BYTES;
+      if (i_slot == RING_BYTES) i_slot = 0;
       if (--i_left == 0) {
         i_left = my_upt, i_rb += p.n_clusters;
         if (--i_tasks > 0) i_setup();
@@ -483,7 +493,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? 96 : 255) 
             }
           }
         }
-        c_slot = (c_slot + SLOT_BYTES) & RING_MASK;
+        c_slot += SLOT_BYTES;
+        if (c_slot == RING_BYTES) c_slot = 0;
         xk += X_KB * KH;
       }
     }

@@ -20,7 +20,10 @@ using namespace ls;
 
 namespace {
 
-constexpr int kCtasPerSm = 2;
+#ifndef LS_CTAS
+#define LS_CTAS 2
+#endif
+constexpr int kCtasPerSm = LS_CTAS;  // GEMM CTAs that fit one SM (shared memory and registers)
 
 struct GemmPlan {
   int n_rb, kpr, cs, n_clusters, grid;

@@ -26,6 +26,7 @@ namespace ls {
 constexpr int PASS_THREADS = 256;
 constexpr int PASS_CS = 8;             // CTAs per cluster = K ranges per stage = token columns of a pass
 constexpr int PASS_TPW = 3;            // row tiles a warp carries through a stage
+constexpr int PASS_RING = 8;            // weight stages per thread
 constexpr int PASS_XCH = 24;           // k-blocks of activations a CTA stages (its whole k-range)
 constexpr int PASS_RECV_FLOATS = 8 * PASS_TPW * 8 * 16;  // [contribution][tile][16 rows] of one token column
 constexpr unsigned PASS_SPIN_LIMIT = 1u << 20;
@@ -258,7 +259,7 @@ __device__ __forceinline__ void pass_attention_item(const PassParams& p, const R
 
 __host__ __device__ constexpr int pass_xbuf_uint4() { return 3 * PASS_XCH * 8 * 4; }
 __host__ __device__ constexpr int pass_smem_bytes() {
-  return RING * 2 * PASS_THREADS * 16 + pass_xbuf_uint4() * 16 + PASS_RECV_FLOATS * 4 + 16 * 4 + 64;
+  return PASS_RING * 2 * PASS_THREADS * 16 + pass_xbuf_uint4() * 16 + PASS_RECV_FLOATS * 4 + 16 * 4 + 64;
 }
 
 // all clusters arrive: one thread per cluster touches the counter, the cluster barrier fans the release out
@@ -299,7 +300,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint4* ring = reinterpret_cast<uint4*>(smem_raw);               // [RING][2][256], slot of thread tid only
-  uint4* xbuf = ring + RING * 2 * PASS_THREADS;                   // [3][XCH][8][4]
+  uint4* xbuf = ring + PASS_RING * 2 * PASS_THREADS;                   // [3][XCH][8][4]
   float* recv = reinterpret_cast<float*>(xbuf + pass_xbuf_uint4());  // [8 * KH][nt][16]
   float* s_rstd = recv + PASS_RECV_FLOATS;                        // [8]
   float* s_red = s_rstd + 8;                                      // [8]
@@ -312,7 +313,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
 
   // ---- weight ring, issue side: runs RING-1 units ahead of the consumer, across stages and layers.  Order of a
   // warp's units in a stage: k-blocks outermost, its row tiles innermost (the consumer below walks the same way).
-  constexpr unsigned SLOT_BYTES = 2 * PASS_THREADS * 16, RING_MASK = RING * SLOT_BYTES - 1, HI_OFF = PASS_THREADS * 16;
+  constexpr unsigned SLOT_BYTES = 2 * PASS_THREADS * 16, RING_MASK = PASS_RING * SLOT_BYTES - 1, HI_OFF = PASS_THREADS * 16;
   const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring) + tid * 16;
   unsigned i_slot = 0;
   int i_l = 0, i_st = 0, i_s = 0, i_n = 0, i_kleft = 0;
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
     cp_async_commit();
   };
 #pragma unroll
-  for (int s = 0; s < RING - 1; ++s) issue_unit();
+  for (int s = 0; s < PASS_RING - 1; ++s) issue_unit();
 
   pdl_launch_dependents();
   pdl_wait();
@@ -444,7 +445,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
           for (int s = 0; s < PASS_TPW; ++s) {
             if (s < ge.my_nt) {
               issue_unit();
-              cp_async_wait<RING - 1>();
+              cp_async_wait<PASS_RING - 1>();
               const uint4 a_lo = lds128(ring_s + c_slot), a_hi = lds128(ring_s + c_slot + HI_OFF);
               c_slot = (c_slot + SLOT_BYTES) & RING_MASK;
               mma_bf16(acc[0][s], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b0.x, b0.y);

@@ -111,6 +111,42 @@ def test_sampled_loopspec_matches_vanilla_in_distribution(models):
     assert stats.chisquare(obs, exp).pvalue > 1e-3
 
 
+def test_filtered_sampling_is_lossless_in_distribution_and_stays_in_the_nucleus(models):
+    """With top-k / top-p inside C (Sec. 3.1) the target is the filtered p_R: every committed token lies in its
+    support, and the first decoded token over many seeds follows it."""
+    shape = W.CONFIGS["tiny"].with_(vocab=16, hidden=32, n_q_heads=2, n_kv_heads=2, head_dim=16, ffn=48,
+                                    tied=False, std=0.35)
+    model = LoopedLM(shape, W.make_weights(shape, seed=9))
+    prompt = W.make_prompt(shape.vocab, 4, seed=3)
+    from scipy import stats
+    kw = dict(temperature=1.0, top_k=12, top_p=0.8)
+    base = Decoder(model, seed=0, **kw)
+    y0 = base.prefill(prompt, 2)
+    counts, target = np.zeros(shape.vocab), None
+    for seed in range(1200):
+        dec = Decoder(model, seed=seed, **kw)
+        dec.prefill(prompt, 2)
+        if dec.ids[-1] != y0:
+            continue
+        tok = dec.loopspec(1, 1, 2, keep_logits=True)[0]
+        counts[tok] += 1
+        target = dec.probs(dec.verify_logits[0])
+    assert counts.sum() > 100
+    assert 0 < np.count_nonzero(target) < shape.vocab          # the filter really cuts
+    assert counts[target == 0].sum() == 0                      # nothing outside the nucleus is ever committed
+    keep = target * counts.sum() > 5
+    obs = np.append(counts[keep], counts[~keep].sum())
+    exp = np.append(target[keep], target[~keep].sum()) * counts.sum()
+    if exp[-1] == 0:
+        obs, exp = obs[:-1], exp[:-1]
+    assert stats.chisquare(obs, exp).pvalue > 1e-3
+    # a longer run: reproducible, and equal to the unfiltered run only if the filters are off
+    a = Decoder(model, seed=5, **kw); a.prefill(prompt, 24)
+    b = Decoder(model, seed=5, **kw); b.prefill(prompt, 24)
+    assert a.loopspec(24, 1, 2) == b.loopspec(24, 1, 2)
+    assert any(e["kind"] == "filter" for e in a.log)
+
+
 class ScriptedModel:
     """A stub 'model' whose depth-R prediction for prefix ending in token t is t + 1 and whose early
     drafts are wrong exactly for the tokens listed in `bad_first` / `bad_second`."""

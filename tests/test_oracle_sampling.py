@@ -207,3 +207,70 @@ def test_greedy_verify_reduction():
         b = Branch(parent=None, token=0, pos=4, H=None)
         b.records = [Record(t, None, f"c{j + 1}") for j, t in enumerate(recs)]
         assert dec._verify(b, z) == want
+
+
+# ---- top-k / top-p filters of C (Sec. 3.1) -------------------------------------------------------
+def _filter_by_library_sort(p, top_k, top_p):
+    """The same filters written with torch's sort and cumsum (nucleus rule as it is usually stated:
+    drop a token when the mass ranked strictly before it already reaches top_p)."""
+    import torch
+    t = torch.tensor(p, dtype=torch.float64)
+    V = len(p)
+    idx = torch.arange(V)
+    # stable sort by decreasing probability keeps lower indices first among equals
+    order = torch.sort(-t, stable=True).indices
+    keep = torch.ones(V, dtype=torch.bool)
+    if top_k and top_k < V:
+        keep[order[top_k:]] = False
+    t = torch.where(keep, t, torch.zeros_like(t))
+    t = t / t.sum()
+    if top_p < 1.0:
+        ts = t[order]
+        before = torch.cumsum(ts, 0) - ts
+        drop = before >= top_p
+        t[order[drop]] = 0.0
+        t = t / t.sum()
+    return t.numpy()
+
+
+@pytest.mark.parametrize("top_k,top_p", [(0, 0.7), (5, 1.0), (6, 0.5), (0, 0.05), (1, 1.0), (3, 0.999)])
+def test_filters_match_the_library_sort_formulation_and_are_minimal(top_k, top_p):
+    rng = np.random.default_rng(3)
+    for V in (2, 7, 16, 300):
+        for _ in range(20):
+            p = random_dist(rng, V, conc=rng.choice([0.2, 1.0, 5.0]))
+            f, margin = sp.top_k_top_p(p, top_k, top_p)
+            np.testing.assert_allclose(f, _filter_by_library_sort(p, top_k, top_p), atol=1e-15)
+            assert abs(f.sum() - 1) < 1e-12 and margin >= 0
+            kept = np.flatnonzero(f)
+            # the kept tokens are the most probable ones and stay in proportion
+            assert p[kept].min() >= np.delete(p, kept).max(initial=0.0)
+            np.testing.assert_allclose(f[kept] / f[kept].sum(), p[kept] / p[kept].sum(), atol=1e-14)
+            if top_k:
+                assert len(kept) <= top_k
+            if top_p < 1.0:      # minimal: dropping the least probable kept token falls short of top_p
+                base = np.sort(p)[::-1][: (top_k or V)]
+                base = base / base.sum()
+                assert base[: len(kept)].sum() >= top_p - 1e-12
+                assert len(kept) == 1 or base[: len(kept) - 1].sum() < top_p
+
+
+def test_filter_special_cases():
+    p = np.array([0.1, 0.4, 0.4, 0.1])
+    np.testing.assert_allclose(sp.top_k_top_p(p, 0, 1.0)[0], p)                 # both off: C is the plain softmax
+    np.testing.assert_allclose(sp.top_k_top_p(p, 1, 1.0)[0], [0, 1, 0, 0])      # ties go to the lower index
+    np.testing.assert_allclose(sp.top_k_top_p(p, 0, 0.5)[0], [0, 0.5, 0.5, 0])  # 0.4 < 0.5 <= 0.8
+    np.testing.assert_allclose(sp.top_k_top_p(p, 0, 0.4)[0], [0, 1, 0, 0])      # mass 0.4 reaches 0.4
+    np.testing.assert_allclose(sp.top_k_top_p(p, 3, 0.9)[0], [1 / 9, 4 / 9, 4 / 9, 0])
+
+
+@pytest.mark.parametrize("V", [4, 6])
+def test_cascade_is_lossless_for_filtered_distributions(V):
+    """Losslessness holds for whatever C outputs (Sec. 3.2): with filtered p, q1, q2~ (supports differ, zeros
+    inside) the enumerated output law is still the filtered target."""
+    rng = np.random.default_rng(11)
+    for _ in range(60):
+        p, q1, q2t = (sp.top_k_top_p(random_dist(rng, V), int(rng.integers(0, V)), float(rng.uniform(0.3, 1.0)))[0]
+                      for _ in range(3))
+        law, _, _ = cascade_law(p, q1, q2t)
+        np.testing.assert_allclose(law, p, atol=1e-12)
