@@ -57,7 +57,12 @@ typedef struct {
  * d1 == d2 == 0 picks the pair from the closed form of Theorem 2 using (alpha, beta).
  * gate = 1 applies Eq. 6, gate = 0 always creates the second proposal; residual_q2 = 1 drafts it from
  * p_{d2} (-) p_{d1} (Eq. 5), 0 from p_{d2} itself.  temperature 0 = greedy.  max_prefill_rows (0 = default)
- * bounds how many prompt positions one prefill pass carries. */
+ * bounds how many prompt positions one prefill pass carries.
+ * top_k, top_p: the optional filters of the post-layers C (Sec. 3.1), applied at EVERY readout depth when
+ * temperature > 0: tokens are ranked by decreasing probability (ties: lower index first); top_k > 0 keeps the first
+ * top_k and renormalises; 0 < top_p < 1 then keeps the shortest prefix of the ranking whose mass reaches top_p and
+ * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off.  With filters on, the vocabulary must
+ * fit the selection kernel's shared memory (vocab <= 56320), else EUNSUPPORTED. */
 typedef struct {
   int32_t d1, d2;
   float alpha, beta;
@@ -66,6 +71,8 @@ typedef struct {
   uint64_t seed;
   int32_t max_seqs, max_ctx;
   int32_t max_prefill_rows;
+  int32_t top_k;
+  float top_p;
 } loopspec_sched;
 
 /* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:

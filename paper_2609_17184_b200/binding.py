@@ -35,7 +35,7 @@ class Model(C.Structure):
 class Sched(C.Structure):
     _fields_ = [("d1", C.c_int32), ("d2", C.c_int32), ("alpha", C.c_float), ("beta", C.c_float), ("gate", C.c_int32),
                 ("residual_q2", C.c_int32), ("temperature", C.c_float), ("seed", C.c_uint64), ("max_seqs", C.c_int32),
-                ("max_ctx", C.c_int32), ("max_prefill_rows", C.c_int32)]
+                ("max_ctx", C.c_int32), ("max_prefill_rows", C.c_int32), ("top_k", C.c_int32), ("top_p", C.c_float)]
 
 
 class Weights(C.Structure):
@@ -160,7 +160,7 @@ class LoopSpec:
     """One decoding context (see include/loopspec.h for the semantics of every call)."""
 
     def __init__(self, shape, weights, d1=1, d2=0, temperature=0.0, seed=0, gate=True, residual_q2=True, max_seqs=1,
-                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None):
+                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None, top_k=0, top_p=1.0):
         import torch
         self._torch = torch
         self.shape = shape
@@ -173,7 +173,7 @@ class LoopSpec:
                            shape.n_prelude, shape.n_recurrent, shape.n_coda, shape.R,
                            1 if shape.weight_dtype == "bf16" else 0, 1 if shape.tied else 0, shape.rms_eps, shape.rope_theta)
         self.sched = Sched(d1, d2, alpha, beta, int(gate), int(residual_q2), temperature, seed, max_seqs, max_ctx,
-                           max_prefill_rows)
+                           max_prefill_rows, int(top_k), float(top_p))
         nbytes = lib.loopspec_workspace_bytes(C.byref(self.model), C.byref(self.sched))
         if nbytes == 0:
             # let init report the precise status

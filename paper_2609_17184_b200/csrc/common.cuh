@@ -59,6 +59,8 @@ struct NodeTable {
   float* lse1;   // log-sum-exp of z/T of the first readout
   float* lse2;
   float* z2;     // sum of [q2~ - q1]_+ (normaliser of the residual proposal), 0 if it had no mass
+  float4* flt1;  // nucleus of the first readout when C filters (top-k / top-p): max z/T, kept mass, cut value, cut index
+  float4* flt2;
 };
 
 struct SeqState {

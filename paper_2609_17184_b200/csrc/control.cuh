@@ -23,6 +23,7 @@ struct ControlParams {
   const int* sel_aux;
   const float* sel_lse;
   const float* sel_z2;
+  const float4* sel_flt;  // nucleus of a drafted row's readout (null unless C filters)
   int phases;
   int* out_ids;      // [S][ids_cap] decoded tokens since prefill
   int ids_cap;
@@ -184,8 +185,10 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
           nd.parent[o + c] = gn - o, nd.child1[o + c] = nd.child2[o + c] = -1, nd.has2[o + c] = 0;
           if (ro == RO_D1) {
             nd.tok1[gn] = s_sel_tok[i], nd.child1[gn] = c, nd.lse1[gn] = s_sel_lse[i], nd.has2[gn] = 0, nd.child2[gn] = -1;
+            if (p.sel_flt) p.nodes.flt1[gn] = p.sel_flt[i];
           } else {
             nd.tok2[gn] = s_sel_tok[i], nd.child2[gn] = c, nd.lse2[gn] = s_sel_lse[i], nd.z2[gn] = s_sel_z2[i], nd.has2[gn] = 1;
+            if (p.sel_flt) p.nodes.flt2[gn] = p.sel_flt[i];
             atomicAdd(&p.ctr->gate_opens, 1ull);
           }
           int e = atomicAdd(&s_nemb, 1);

@@ -73,7 +73,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, argpart, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, argpart, flt, sel_flt, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -137,6 +137,7 @@ bool validate_model(const loopspec_model* m, int* why) {
 bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d, int* why) {
   *why = LOOPSPEC_EINVAL;
   if (!s || s->max_seqs <= 0 || s->max_ctx < 4 || s->temperature < 0 || s->max_prefill_rows < 0) return false;
+  if (s->top_k < 0 || s->top_p < 0.f || s->top_p != s->top_p) return false;
   int d1 = s->d1, d2 = s->d2;
   if (d1 == 0 && d2 == 0) {
     if (!(s->alpha > 0) || !(s->beta > 0)) return false;
@@ -210,6 +211,8 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.gcnt = take((size_t)((m->ffn + 63) / 64 + (d.Hq + 2 * d.Hkv) / 128 + 16) * 4);
   L.bar = take(256);
   L.nodes = take((size_t)13 * MAX_NODES * 4);
+  L.flt = take((size_t)2 * MAX_NODES * sizeof(float4));
+  L.sel_flt = take((size_t)MAX_ROWS * sizeof(float4));
   L.seqs = take((size_t)5 * MAX_ROWS * 4);
   L.ctr = take(sizeof(Counters));
   L.tab_dec = take(sizeof(RowTable));
@@ -257,6 +260,7 @@ struct loopspec_ctx {
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
   bool pass_coop = true, use_perm = true;
+  bool filters = false;  // C applies top-k / top-p (sampling only)
   int launches_per_step = 0;
   std::string err;
 
@@ -270,6 +274,7 @@ struct loopspec_ctx {
     n.tok2 = b + 8 * MAX_NODES, n.has2 = b + 9 * MAX_NODES;
     n.lse1 = reinterpret_cast<float*>(b + 10 * MAX_NODES), n.lse2 = reinterpret_cast<float*>(b + 11 * MAX_NODES);
     n.z2 = reinterpret_cast<float*>(b + 12 * MAX_NODES);
+    n.flt1 = at<float4>(L.flt), n.flt2 = n.flt1 + MAX_NODES;
     return n;
   }
   SeqState seqs() const {
@@ -541,7 +546,9 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   sp.sel_tok = c->at<int>(c->L.sel_tok), sp.sel_aux = c->at<int>(c->L.sel_aux);
   sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);
   sp.argpart = c->at<float2>(c->L.argpart), sp.n_rb = c->plan[G_LM].n_rb;
-  return launch_k(select_kernel, dim3(c->d.max_rows), dim3(SEL_THREADS), 0, c->stream, sp, c->use_pdl);
+  sp.top_k = c->filters ? c->s.top_k : 0, sp.top_p = c->filters ? c->s.top_p : 1.0f, sp.sel_flt = c->at<float4>(c->L.sel_flt);
+  const size_t smem = c->filters ? (size_t)c->m.vocab * sizeof(float) : 0;
+  return launch_k(select_kernel, dim3(c->d.max_rows), dim3(SEL_THREADS), smem, c->stream, sp, c->use_pdl);
 }
 
 ControlParams control_params(loopspec_ctx* c, int phases) {
@@ -551,6 +558,7 @@ ControlParams control_params(loopspec_ctx* c, int phases) {
   p.S = c->d.S, p.NB = c->d.NB, p.R = c->m.R, p.d1 = c->d.d1, p.d2 = c->d.d2, p.ctx_cap = c->s.max_ctx;
   p.sel_tok = c->at<int>(c->L.sel_tok), p.sel_aux = c->at<int>(c->L.sel_aux);
   p.sel_lse = c->at<float>(c->L.sel_lse), p.sel_z2 = c->at<float>(c->L.sel_z2);
+  p.sel_flt = c->filters ? c->at<float4>(c->L.sel_flt) : nullptr;
   p.phases = phases;
   p.out_ids = c->at<int>(c->L.out_ids), p.ids_cap = c->d.ids_cap, p.commits = c->at<int>(c->L.commits);
   p.row_trace = c->at<int>(c->L.trace), p.trace_n = c->at<int>(c->L.trace_n), p.trace_cap = c->d.trace_cap;
@@ -703,6 +711,17 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   loopspec_ctx* c = new loopspec_ctx();
   c->m = *m, c->s = *s, c->d = d, c->L = L, c->n_sm = n_sm;
   c->s.d1 = d.d1, c->s.d2 = d.d2;
+  if (c->s.top_p <= 0.f || c->s.top_p > 1.f) c->s.top_p = 1.f;  // 0 and anything above 1: no nucleus cut
+  c->filters = c->s.temperature > 0.f && ((c->s.top_k > 0 && c->s.top_k < m->vocab) || c->s.top_p < 1.f);
+  if (c->filters) {  // the selection kernel then keeps exp(z/T - max) of a whole row in shared memory
+    const size_t need = (size_t)m->vocab * sizeof(float);
+    if (need > 220 * 1024 ||
+        cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess) {
+      (void)cudaGetLastError();
+      delete c;
+      return LOOPSPEC_EUNSUPPORTED;
+    }
+  }
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   c->ws = static_cast<unsigned char*>(workspace);
   c->embed = w->embed, c->lm_head = m->tied_lm_head ? w->embed : w->lm_head;

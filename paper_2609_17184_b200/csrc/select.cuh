@@ -29,6 +29,36 @@ struct SelectParams {
   float* sel_z2;        // RO_D2: normaliser of the residual proposal (0: the proposal is q2~ itself)
   const float2* argpart;  // [readout column][row block]: per-block largest logit and its index, written by the lm_head
   int n_rb;
+  // optional filters of C (Sec. 3.1), used when temperature > 0: keep the top_k most probable tokens (0: all), then
+  // the shortest prefix of the ranking whose mass reaches top_p (>= 1: all).  The kernel then needs V floats of
+  // dynamic shared memory.
+  int top_k;
+  float top_p;
+  float4* sel_flt;      // per row: the nucleus of its readout (max of z/T, kept mass, cut value bits, cut index)
+};
+
+// A readout distribution C(H): softmax(z / T), optionally cut to a nucleus.  Ranking: decreasing e = exp(z/T - m)
+// (as fp32 bit patterns), ties to the lower index; the nucleus is everything ranked at or before (ecut, vcut).
+struct Dist {
+  const float* z;
+  float lse;      // unfiltered: log sum_v exp(z_v / T)
+  float m, s;     // filtered: max_v z_v / T and the mass of the kept exp(z_v / T - m)
+  unsigned ecut;
+  int vcut;
+  bool filt;
+  __device__ __forceinline__ bool kept(unsigned eb, int v) const { return eb > ecut || (eb == ecut && v <= vcut); }
+  __device__ __forceinline__ float prob(int v, float T) const {
+    if (!filt) return expf(z[v] / T - lse);
+    const float e = expf(z[v] / T - m);
+    return kept(__float_as_uint(e), v) ? e / s : 0.f;
+  }
+  // log of an unnormalised weight for the exponential race; -inf outside the support
+  __device__ __forceinline__ float logw(int v, float T) const {
+    if (!filt) return z[v] / T;
+    return kept(__float_as_uint(expf(z[v] / T - m)), v) ? z[v] / T : -INFINITY;
+  }
+  __device__ __forceinline__ float4 pack() const { return make_float4(m, s, __uint_as_float(ecut), __int_as_float(vcut)); }
+  __device__ __forceinline__ void unpack(float4 f) { m = f.x, s = f.y, ecut = __float_as_uint(f.z), vcut = __float_as_int(f.w), filt = true; }
 };
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
@@ -85,6 +115,77 @@ __device__ __forceinline__ float block_max(float v, float* sh) {
   return r;
 }
 
+__device__ __forceinline__ int block_sum_int(int v, int* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = 0;
+  for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh[w];
+  return r;
+}
+
+// Nucleus of softmax(z / T) under top-k and top-p.  e_v = exp(z_v/T - m) is kept in shared memory (a thread only ever
+// touches the elements it wrote); the cut is found by searching the bit pattern of e from the top bit down (e <= 1,
+// so 30 bits), then the index among equal values; every count / mass is a fixed-order block reduction, so the result
+// does not depend on timing.  top-k cuts first; top-p then applies to the renormalised top-k set.
+__device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, float top_p, float* e_sm, float* sh_f, int* sh_i) {
+  const int tid = threadIdx.x;
+  float m = -INFINITY;
+  for (int v = tid; v < V; v += SEL_THREADS) m = fmaxf(m, d.z[v] / T);
+  m = block_max(m, sh_f);
+  for (int v = tid; v < V; v += SEL_THREADS) e_sm[v] = expf(d.z[v] / T - m);
+  d.m = m, d.ecut = 0u, d.vcut = V - 1, d.filt = true;  // everything kept so far
+  auto count_if = [&](auto pred) {
+    int n = 0;
+    for (int v = tid; v < V; v += SEL_THREADS) n += pred(__float_as_uint(e_sm[v]), v) ? 1 : 0;
+    return block_sum_int(n, sh_i);
+  };
+  auto mass_if = [&](auto pred) {
+    float a = 0.f;
+    for (int v = tid; v < V; v += SEL_THREADS) a += pred(__float_as_uint(e_sm[v]), v) ? e_sm[v] : 0.f;
+    return block_sum(a, sh_f);
+  };
+  if (top_k > 0 && top_k < V) {
+    unsigned c = 0;  // largest c with at least top_k values >= c: the value of the top_k-th ranked token
+    for (int bit = 29; bit >= 0; --bit) {
+      const unsigned cand = c | (1u << bit);
+      if (count_if([&](unsigned eb, int) { return eb >= cand; }) >= top_k) c = cand;
+    }
+    const int need = top_k - count_if([&](unsigned eb, int) { return eb > c; });  // how many of the equal values stay
+    int lo = 0, hi = V - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (count_if([&](unsigned eb, int v) { return eb == c && v <= mid; }) >= need) hi = mid;
+      else lo = mid + 1;
+    }
+    d.ecut = c, d.vcut = lo;
+  }
+  if (top_p < 1.0f) {
+    const Dist dk = d;  // the top-k set
+    const float target = top_p * mass_if([&](unsigned eb, int v) { return dk.kept(eb, v); });
+    unsigned c = 0;     // largest c such that the kept values >= c carry at least the target mass
+    for (int bit = 29; bit >= 0; --bit) {
+      const unsigned cand = c | (1u << bit);
+      if (mass_if([&](unsigned eb, int v) { return dk.kept(eb, v) && eb >= cand; }) >= target) c = cand;
+    }
+    if (c < dk.ecut) c = dk.ecut;
+    const float m_gt = mass_if([&](unsigned eb, int v) { return dk.kept(eb, v) && eb > c; });
+    const float e_c = __uint_as_float(c);
+    int lo = 0, hi = (c == dk.ecut) ? dk.vcut : V - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      const int n = count_if([&](unsigned eb, int v) { return eb == c && v <= mid; });
+      if (m_gt + (float)n * e_c >= target) hi = mid;
+      else lo = mid + 1;
+    }
+    d.ecut = c, d.vcut = lo;
+  }
+  const Dist df = d;
+  d.s = mass_if([&](unsigned eb, int v) { return df.kept(eb, v); });
+}
+
 // argmax of the logits row of readout column `col` from the per-block maxima the lm_head epilogue left (ties to the
 // lowest index)
 __device__ __forceinline__ int greedy_argmax(const float2* argpart, int n_rb, int col, ArgMax* sh_am) {
@@ -124,14 +225,32 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   const unsigned seq = (unsigned)tab->seq[row];
   const uint2 key = make_uint2((unsigned)(p.seed & 0xffffffffull), (unsigned)(p.seed >> 32));
 
-  auto lse_of = [&](const float* zz) -> float {  // log sum_v exp(zz_v / T)
-    float m = -INFINITY;
-    for (int v = tid; v < V; v += SEL_THREADS) m = fmaxf(m, zz[v] / T);
-    m = block_max(m, sh_f);
-    float s = 0.f;
-    for (int v = tid; v < V; v += SEL_THREADS) s += expf(zz[v] / T - m);
-    s = block_sum(s, sh_f);
-    return m + logf(s);
+  const bool filt = T > 0.f && ((p.top_k > 0 && p.top_k < V) || p.top_p < 1.0f);
+  extern __shared__ float e_sm[];  // [V] when filters are on
+  __shared__ int sh_i[SEL_THREADS / 32];
+  // the distribution C(H) of a freshly computed logits row
+  auto fresh = [&](const float* zz) -> Dist {
+    Dist d;
+    d.z = zz, d.filt = false, d.lse = 0.f, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
+    if (filt) {
+      build_nucleus(d, V, T, p.top_k, p.top_p, e_sm, sh_f, sh_i);
+    } else {  // log sum_v exp(zz_v / T)
+      float m = -INFINITY;
+      for (int v = tid; v < V; v += SEL_THREADS) m = fmaxf(m, zz[v] / T);
+      m = block_max(m, sh_f);
+      float s = 0.f;
+      for (int v = tid; v < V; v += SEL_THREADS) s += expf(zz[v] / T - m);
+      s = block_sum(s, sh_f);
+      d.lse = m + logf(s);
+    }
+    return d;
+  };
+  // a distribution stored with a proposal record: its logits row, log-normaliser and (if filtered) nucleus
+  auto stored = [&](const float* zz, float lse, const float4* flt) -> Dist {
+    Dist d;
+    d.z = zz, d.filt = false, d.lse = lse, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
+    if (filt) d.unpack(*flt);
+    return d;
   };
   // greedy readouts are always taken from the row the lm_head just produced
   auto greedy = [&](const float*) -> int { return greedy_argmax(p.argpart, p.n_rb, (int)blockIdx.x, sh_am); };
@@ -156,7 +275,13 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
 
   pdl_wait();
   if (kind == RO_TARGET) {
-    int tok = (T == 0.f) ? greedy(z) : race([&](int v) { return z[v] / T; }, PUR_VANILLA);
+    int tok;
+    if (T == 0.f) {
+      tok = greedy(z);
+    } else {
+      const Dist dz = fresh(z);
+      tok = race([&](int v) { return dz.logw(v, T); }, PUR_VANILLA);
+    }
     if (tid == 0) p.sel_tok[row] = tok;
     return;
   }
@@ -165,9 +290,12 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       int tok = greedy(z);
       if (tid == 0) p.sel_tok[row] = tok, p.sel_lse[row] = 0.f;
     } else {
-      float lse = lse_of(z);
-      int tok = race([&](int v) { return z[v] / T; }, PUR_DRAFT1);
-      if (tid == 0) p.sel_tok[row] = tok, p.sel_lse[row] = lse;
+      const Dist dz = fresh(z);
+      int tok = race([&](int v) { return dz.logw(v, T); }, PUR_DRAFT1);
+      if (tid == 0) {
+        p.sel_tok[row] = tok, p.sel_lse[row] = dz.lse;
+        if (filt) p.sel_flt[row] = dz.pack();
+      }
     }
     return;
   }
@@ -178,25 +306,30 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       if (tid == 0) p.sel_tok[row] = top, p.sel_aux[row] = (top != x1) || !p.gate, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
       return;
     }
-    const float lse1 = p.nodes.lse1[gn];
-    const float lse2 = lse_of(z);
-    const bool open = (z[x1] / T - lse2 < z1[x1] / T - lse1) || !p.gate;
+    const Dist d1 = stored(z1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
+    const Dist d2 = fresh(z);
+    // Eq. 6; without filters the comparison is made on log-probabilities, as before
+    const bool lower = filt ? (d2.prob(x1, T) < d1.prob(x1, T)) : (z[x1] / T - d2.lse < z1[x1] / T - d1.lse);
+    const bool open = lower || !p.gate;
     int tok = 0;
     float Z2 = 0.f;
     if (open) {
       if (p.residual_q2) {
         float s = 0.f;
-        for (int v = tid; v < V; v += SEL_THREADS) s += fmaxf(expf(z[v] / T - lse2) - expf(z1[v] / T - lse1), 0.f);
+        for (int v = tid; v < V; v += SEL_THREADS) s += fmaxf(d2.prob(v, T) - d1.prob(v, T), 0.f);
         Z2 = block_sum(s, sh_f);
       }
       if (Z2 > 0.f)
         tok = race([&](int v) {
-          float w = expf(z[v] / T - lse2) - expf(z1[v] / T - lse1);
+          float w = d2.prob(v, T) - d1.prob(v, T);
           return w > 0.f ? logf(w) : -INFINITY; }, PUR_DRAFT2);
       else
-        tok = race([&](int v) { return z[v] / T; }, PUR_DRAFT2);
+        tok = race([&](int v) { return d2.logw(v, T); }, PUR_DRAFT2);
     }
-    if (tid == 0) p.sel_tok[row] = tok, p.sel_aux[row] = open, p.sel_lse[row] = lse2, p.sel_z2[row] = Z2;
+    if (tid == 0) {
+      p.sel_tok[row] = tok, p.sel_aux[row] = open, p.sel_lse[row] = d2.lse, p.sel_z2[row] = Z2;
+      if (filt) p.sel_flt[row] = d2.pack();
+    }
     return;
   }
   // ---- RO_VERIFY: z is the target readout p_R of the root branch ------------------------------------
@@ -207,11 +340,13 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     if (tid == 0) p.sel_tok[row] = top, p.sel_aux[row] = src;
     return;
   }
-  const float lse1 = p.nodes.lse1[gn], lse2 = p.nodes.lse2[gn], Z2 = p.nodes.z2[gn];
-  const float lsep = lse_of(z);
-  auto pp = [&](int v) { return expf(z[v] / T - lsep); };     // p_R
-  auto q1 = [&](int v) { return expf(z1[v] / T - lse1); };    // first proposal
-  auto q2t = [&](int v) { return expf(z2[v] / T - lse2); };   // deeper readout
+  const float Z2 = p.nodes.z2[gn];
+  const Dist d1 = stored(z1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
+  const Dist d2 = stored(z2, p.nodes.lse2[gn], p.nodes.flt2 + gn);
+  const Dist dp = fresh(z);
+  auto pp = [&](int v) { return dp.prob(v, T); };    // p_R
+  auto q1 = [&](int v) { return d1.prob(v, T); };    // first proposal
+  auto q2t = [&](int v) { return d2.prob(v, T); };   // deeper readout
   // first proposal: accept with probability min{1, p(x1)/q1(x1)} (Eq. 3)
   const float U1 = uniform(PUR_ACCEPT1);
   if (U1 < fminf(1.0f, pp(x1) / q1(x1))) {

@@ -20,9 +20,9 @@ def oracle_model(name, seed=0, gain_jitter=0.0):
 
 @functools.lru_cache(maxsize=None)
 def oracle_run(name, n_prompt, n_decode, d1, d2, T=0.0, seed=2, gate=True, residual_q2=True, prompt_seed=1, seq=0,
-               wseed=0, gain_jitter=0.0, vanilla=False):
+               wseed=0, gain_jitter=0.0, vanilla=False, top_k=0, top_p=1.0):
     shape = W.CONFIGS[name]
-    dec = Decoder(oracle_model(name, wseed, gain_jitter), temperature=T, seed=seed, seq=seq)
+    dec = Decoder(oracle_model(name, wseed, gain_jitter), temperature=T, seed=seed, seq=seq, top_k=top_k, top_p=top_p)
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=prompt_seed, seq=seq)
     first = dec.prefill(prompt, n_decode)
     if vanilla:

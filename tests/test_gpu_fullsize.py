@@ -1,7 +1,8 @@
 """Full-size parity on the Ouro-1.4B-shaped model (BASELINE config 1), in the launch configuration bench.py times.
 
 The oracle cannot decode 512 tokens of a 1.4B model in test time, so:
-  * the first tokens of the run (greedy and temperature 1) are compared with values the oracle computed once
+  * the first tokens of the run (greedy, temperature 1, temperature 1 with top-p 0.7) are compared with values the
+    oracle computed once
     (tests/golden/ouro_1p4b_oracle.json, written by tests/golden/make_ouro_golden.py, which calls only oracle/);
   * the whole 512-token run is checked through properties that hold at any size: greedy LoopSpec == greedy
     vanilla decoding on the device, the commit-gap schedule, and the counters' identities.
@@ -28,18 +29,18 @@ def setup():
     return ls, wl, shape, weights, prompt, json.load(open(GOLD))
 
 
-def make(setup, T):
+def make(setup, T, top_p=1.0):
     ls, wl, shape, weights, prompt, gold = setup
     return ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=T, seed=wl.sample_seed, gate=wl.gate, max_seqs=1,
-                       max_ctx=wl.prompt_len + wl.decode_len + 16, max_prefill_rows=64)
+                       max_ctx=wl.prompt_len + wl.decode_len + 16, max_prefill_rows=64, top_p=top_p)
 
 
-@pytest.mark.parametrize("run", ["greedy", "sampled_T1"])
+@pytest.mark.parametrize("run", ["greedy", "sampled_T1", "sampled_T1_top_p"])
 def test_first_tokens_match_the_oracle(setup, run):
     ls, wl, shape, weights, prompt, gold = setup
     g = gold["runs"][run]
     n = gold["n_tokens"]
-    ctx = make(setup, g["temperature"])
+    ctx = make(setup, g["temperature"], g.get("top_p", 1.0))
     assert ctx.prefill(prompt) == g["first_token"]
     z = ctx.debug_logits(0, 0)
     assert int(np.argmax(z)) == g["first_logits_argmax"]

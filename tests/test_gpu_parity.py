@@ -120,6 +120,52 @@ def test_sampled_decode_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate
     ctx.close()
 
 
+FILTERED_CASES = [
+    # name, n_prompt, n_decode, d1, d2, T, top_k, top_p
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, 0, 0.7),       # the paper's sampling setting: T = 1, top-p 0.7
+    ("tiny_bf16", 9, 40, 1, 3, 0.8, 20, 1.0),       # top-k alone
+    ("tiny", 16, 40, 2, 0, 1.2, 50, 0.9),           # both, fp32 weights, single proposal
+    ("small_bf16", 40, 32, 1, 2, 1.0, 0, 0.7),
+]
+
+
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,top_k,top_p", FILTERED_CASES)
+def test_filtered_sampling_matches_oracle(name, n_prompt, n_decode, d1, d2, T, top_k, top_p):
+    """top-k / top-p inside C (Sec. 3.1) at every readout depth: same nuclei, same draws, same decisions."""
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=2, top_k=top_k, top_p=top_p)
+    ctx = U.make_ctx(name, d1, d2, T=T, seed=2, max_ctx=n_prompt + n_decode + 8, top_k=top_k, top_p=top_p)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(n_decode)
+    got = [c["token"] for c in ctx.commits(0)]
+    assert got == ref["tokens"], (U.first_diff(got, ref["tokens"]), U.min_margin(ref["dec"]))
+    for g, o in zip(ctx.commits(0), ref["dec"].commits):
+        assert tuple(g[k] for k in U.COMMIT_KEYS) == tuple(o[k] for k in U.COMMIT_KEYS)
+    st, so = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
+        assert st[k] == so[k], (k, st[k], so[k])
+    # the filters change the stream (else the case tests nothing)
+    plain = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=2)
+    assert plain["tokens"] != ref["tokens"]
+    # vanilla decoding draws from the same filtered target
+    refv = U.oracle_run(name, n_prompt, 16, d1, d2, T=T, seed=2, top_k=top_k, top_p=top_p, vanilla=True)
+    assert ctx.prefill(refv["prompt"]) == refv["first"]
+    assert ctx.vanilla_decode(16)[0].tolist() == refv["tokens"]
+    ctx.close()
+
+
+def test_filters_off_values_and_unsupported_vocab():
+    """top_k = 0 with top_p = 0 or 1 is the plain softmax: bit-identical to a context built without the fields."""
+    ref = U.oracle_run("tiny_bf16", 16, 24, 1, 2, T=1.0, seed=2)
+    for top_p in (0.0, 1.0):
+        ctx = U.make_ctx("tiny_bf16", 1, 2, T=1.0, seed=2, max_ctx=64, top_k=0, top_p=top_p)
+        assert ctx.prefill(ref["prompt"]) == ref["first"]
+        assert ctx.decode(24)[0].tolist() == ref["tokens"]
+        ctx.close()
+    with pytest.raises(Exception) as e:
+        U.make_ctx("tiny_bf16", 1, 2, T=1.0, top_k=-1)
+    assert "EINVAL" in str(e.value)
+
+
 def test_sampled_vanilla_matches_oracle():
     ref = U.oracle_run("tiny_bf16", 16, 40, 1, 0, T=1.0, seed=5, vanilla=True)
     ctx = U.make_ctx("tiny_bf16", 1, 0, T=1.0, seed=5, max_ctx=80)
