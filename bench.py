@@ -171,7 +171,7 @@ def run_ours(args):
     t_setup = time.time() - t0
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed)
     ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
-                      max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64)
+                      max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64, top_k=wl.top_k, top_p=wl.top_p)
     stream = ctx.stream
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -238,7 +238,7 @@ def run_ours(args):
         "metric": "decode_tok_per_s", "value": round(value, 2), "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"{wl.name}: prompt {n_prompt}, decode {n_decode}, T={wl.temperature}, (d1,d2)=({wl.d1},{wl.d2}), "
+        "config": {"workload": f"{wl.name}: prompt {n_prompt}, decode {n_decode}, T={wl.temperature}{f', top-p {wl.top_p}' if wl.top_p < 1 else ''}{f', top-k {wl.top_k}' if wl.top_k else ''}, (d1,d2)=({wl.d1},{wl.d2}), "
                                f"gate={'on' if wl.gate else 'off'}, batch 1, R={shape.R}, L={shape.n_recurrent}",
                    "l2": "every pass streams the 2.5 GB shared stack, far larger than the 126 MB L2; no flush needed",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
@@ -323,7 +323,7 @@ def cpu_baseline(shape, wl, seconds_budget=25.0, n_prompt=32):
     cores = len(os.sched_getaffinity(0))
     model = LoopedLM(shape, W.make_weights(shape, seed=wl.weight_seed))
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed)
-    dec = Decoder(model, temperature=wl.temperature, seed=wl.sample_seed)
+    dec = Decoder(model, temperature=wl.temperature, seed=wl.sample_seed, top_k=wl.top_k, top_p=wl.top_p)
     dec.prefill(prompt, 64)
     t0 = time.perf_counter()
     n_v = 0
@@ -355,7 +355,7 @@ def run_reference(args):
     cores = len(os.sched_getaffinity(0))
     model = LoopedLM(shape, W.make_weights(shape, seed=wl.weight_seed))
     n_prompt, n_tok = 32, 2
-    dec = Decoder(model, temperature=wl.temperature, seed=wl.sample_seed)
+    dec = Decoder(model, temperature=wl.temperature, seed=wl.sample_seed, top_k=wl.top_k, top_p=wl.top_p)
     dec.prefill(W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed), n_tok * (args.steps + args.warmup) + 8)
     for _ in range(args.warmup):
         dec.loopspec(n_tok, wl.d1, wl.d2, gate=wl.gate)

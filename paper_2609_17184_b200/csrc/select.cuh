@@ -147,6 +147,13 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, f
     for (int v = tid; v < V; v += SEL_THREADS) a += pred(__float_as_uint(e_sm[v]), v) ? e_sm[v] : 0.f;
     return block_sum(a, sh_f);
   };
+  // lowest index of an element whose value is c (used when c occurs once: no search over the indices is needed)
+  auto first_index_of = [&](unsigned c) {
+    int best = V;
+    for (int v = tid; v < V; v += SEL_THREADS)
+      if (__float_as_uint(e_sm[v]) == c) best = min(best, v);
+    return -block_sum_int(best == V ? 0 : -best, sh_i);  // at most one thread holds it when the value is unique
+  };
   if (top_k > 0 && top_k < V) {
     unsigned c = 0;  // largest c with at least top_k values >= c: the value of the top_k-th ranked token
     for (int bit = 29; bit >= 0; --bit) {
@@ -155,6 +162,7 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, f
     }
     const int need = top_k - count_if([&](unsigned eb, int) { return eb > c; });  // how many of the equal values stay
     int lo = 0, hi = V - 1;
+    if (count_if([&](unsigned eb, int) { return eb == c; }) == 1) lo = hi = first_index_of(c);
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
       if (count_if([&](unsigned eb, int v) { return eb == c && v <= mid; }) >= need) hi = mid;
@@ -174,6 +182,7 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, f
     const float m_gt = mass_if([&](unsigned eb, int v) { return dk.kept(eb, v) && eb > c; });
     const float e_c = __uint_as_float(c);
     int lo = 0, hi = (c == dk.ecut) ? dk.vcut : V - 1;
+    if (count_if([&](unsigned eb, int) { return eb == c; }) == 1) lo = hi = first_index_of(c);
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
       const int n = count_if([&](unsigned eb, int v) { return eb == c && v <= mid; });

@@ -53,6 +53,8 @@ class Workload:
     prompt_seed: int = 1
     sample_seed: int = 2
     weight_seed: int = 0
+    top_k: int = 0            # filters of the readout (0 / 1.0 = off); only used when temperature > 0
+    top_p: float = 1.0
 
 
 CONFIGS = {
@@ -78,6 +80,9 @@ WORKLOADS = {
     "tiny": Workload("tiny", "tiny", prompt_len=16, decode_len=64, temperature=0.0, d1=1, d2=0),
     "ouro_1p4b": Workload("ouro_1p4b", "ouro_1p4b", prompt_len=512, decode_len=512, temperature=0.0, d1=1, d2=2),
     "ouro_2p6b": Workload("ouro_2p6b", "ouro_2p6b", prompt_len=1024, decode_len=1024, temperature=1.0, d1=1, d2=2),
+    # the paper's sampling setting for its reasoning models (Sec. 5.1: T = 1.0, top-p 0.7) on the headline shape
+    "ouro_1p4b_top_p": Workload("ouro_1p4b_top_p", "ouro_1p4b", prompt_len=512, decode_len=512, temperature=1.0, d1=1,
+                                d2=2, top_p=0.7),
     "kv_bound": Workload("kv_bound", "ouro_1p4b", prompt_len=8192, decode_len=256, temperature=0.7, d1=1, d2=2,
                          batch=8),
 }
