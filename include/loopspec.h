@@ -61,8 +61,7 @@ typedef struct {
  * top_k, top_p: the optional filters of the post-layers C (Sec. 3.1), applied at EVERY readout depth when
  * temperature > 0: tokens are ranked by decreasing probability (ties: lower index first); top_k > 0 keeps the first
  * top_k and renormalises; 0 < top_p < 1 then keeps the shortest prefix of the ranking whose mass reaches top_p and
- * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off.  With filters on, the vocabulary must
- * fit the selection kernel's shared memory (vocab <= 56320), else EUNSUPPORTED. */
+ * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off. */
 typedef struct {
   int32_t d1, d2;
   float alpha, beta;

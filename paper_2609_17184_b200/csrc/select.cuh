@@ -1,17 +1,24 @@
 // Readout decisions of one step: first-proposal draft at d1 (Sec. 4.2 step 2), gate and residual second
 // proposal at d2 (Eq. 5-6), cascade verification at R (Sec. 4.3; Algorithm 1 Verify), and the plain draw
-// x ~ C(H) used by prefill and vanilla decoding.  One CTA per reading-out row; every reduction over the
-// vocabulary is a fixed-order block reduction.
+// x ~ C(H) used by prefill and vanilla decoding.  One thread-block cluster per reading-out row: every CTA of
+// the cluster scans its slice of the vocabulary (a single SM ingests a 196 KB logits row in ~4 us, and the
+// sampled paths make several passes over up to three rows), and every reduction over the vocabulary is a
+// fixed-order block reduction followed by a fixed-order sum of the CTAs' partials exchanged through
+// distributed shared memory - so all CTAs of a cluster hold the same values and take the same branches.
 //
 // Random draws (the paper only says "x ~ q", "U ~ U(0,1)"): Philox4x32-10 keyed by the seed with counter
 // (block, position being decided, sequence, purpose); u = ((word >> 9) + 0.5) * 2^-23; categorical draws
 // by the exponential race argmax_v log w_v - log(-log u_v) with ties to the lowest index.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace ls {
+namespace cg = cooperative_groups;
 
-constexpr int SEL_THREADS = 1024;
+constexpr int SEL_THREADS = 512;
+constexpr int SEL_CS = 8;  // CTAs per reading-out row
 enum { PUR_DRAFT1 = 1, PUR_DRAFT2 = 2, PUR_ACCEPT1 = 3, PUR_ACCEPT2 = 4, PUR_RESAMPLE = 5, PUR_VANILLA = 6 };
 
 struct SelectParams {
@@ -81,78 +88,120 @@ struct ArgMax {
 };
 __device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b) { return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a; }
 
-__device__ __forceinline__ ArgMax block_argmax(ArgMax a, ArgMax* sh) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    ArgMax b;
-    b.v = __shfl_xor_sync(0xffffffffu, a.v, o);
-    b.i = __shfl_xor_sync(0xffffffffu, a.i, o);
-    a = better(a, b);
+// Reductions over the whole cluster.  Each CTA reduces its own threads (warp shuffles, then the warps' partials in
+// order), thread 0 writes the CTA's partial into slot [rank] of every CTA of the cluster, and after one cluster
+// barrier every thread combines the slots in rank order.  Two sets of slots alternate, so a CTA that is already in
+// the next reduction never overwrites what a slower sibling still reads.
+struct ClusterRed {
+  cg::cluster_group cluster;
+  int n_ranks, rank, phase;
+  float* sh_f;    // [SEL_THREADS / 32]
+  int* sh_i;      // [SEL_THREADS / 32]
+  ArgMax* sh_a;   // [SEL_THREADS / 32]
+  float* part_f;  // [2][SEL_CS]
+  int* part_i;    // [2][SEL_CS]
+  ArgMax* part_a; // [2][SEL_CS]
+
+  template <typename T>
+  __device__ __forceinline__ void publish(T* part, T v) {
+    if (threadIdx.x == 0)
+      for (int r = 0; r < n_ranks; ++r) *cluster.map_shared_rank(part + phase * SEL_CS + rank, r) = v;
+    cluster.sync();
   }
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = a;
-  __syncthreads();
-  ArgMax r = sh[0];
-  for (int w = 1; w < SEL_THREADS / 32; ++w) r = better(r, sh[w]);
-  return r;
-}
-__device__ __forceinline__ float block_sum(float v, float* sh) {
-  v = warp_sum(v);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-  __syncthreads();
-  float r = 0.f;
-  for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh[w];
-  return r;
-}
-__device__ __forceinline__ float block_max(float v, float* sh) {
-  v = warp_max(v);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-  __syncthreads();
-  float r = sh[0];
-  for (int w = 1; w < SEL_THREADS / 32; ++w) r = fmaxf(r, sh[w]);
-  return r;
-}
-
-__device__ __forceinline__ int block_sum_int(int v, int* sh) {
+  __device__ __forceinline__ float sum(float v) {
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh_f[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = 0.f;
+    for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh_f[w];
+    publish(part_f, r);
+    r = 0.f;
+    for (int q = 0; q < n_ranks; ++q) r += part_f[phase * SEL_CS + q];
+    phase ^= 1;
+    return r;
+  }
+  __device__ __forceinline__ float max(float v) {
+    v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh_f[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = sh_f[0];
+    for (int w = 1; w < SEL_THREADS / 32; ++w) r = fmaxf(r, sh_f[w]);
+    publish(part_f, r);
+    r = part_f[phase * SEL_CS];
+    for (int q = 1; q < n_ranks; ++q) r = fmaxf(r, part_f[phase * SEL_CS + q]);
+    phase ^= 1;
+    return r;
+  }
+  __device__ __forceinline__ int sum_int(int v) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-  __syncthreads();
-  int r = 0;
-  for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh[w];
-  return r;
-}
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh_i[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int r = 0;
+    for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh_i[w];
+    publish(part_i, r);
+    r = 0;
+    for (int q = 0; q < n_ranks; ++q) r += part_i[phase * SEL_CS + q];
+    phase ^= 1;
+    return r;
+  }
+  __device__ __forceinline__ ArgMax block_argmax(ArgMax a) {  // this CTA only
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ArgMax b;
+      b.v = __shfl_xor_sync(0xffffffffu, a.v, o);
+      b.i = __shfl_xor_sync(0xffffffffu, a.i, o);
+      a = better(a, b);
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh_a[threadIdx.x >> 5] = a;
+    __syncthreads();
+    ArgMax r = sh_a[0];
+    for (int w = 1; w < SEL_THREADS / 32; ++w) r = better(r, sh_a[w]);
+    return r;
+  }
+  __device__ __forceinline__ ArgMax argmax(ArgMax a) {
+    ArgMax r = block_argmax(a);
+    publish(part_a, r);
+    r = part_a[phase * SEL_CS];
+    for (int q = 1; q < n_ranks; ++q) r = better(r, part_a[phase * SEL_CS + q]);
+    phase ^= 1;
+    return r;
+  }
+};
 
-// Nucleus of softmax(z / T) under top-k and top-p.  e_v = exp(z_v/T - m) is kept in shared memory (a thread only ever
-// touches the elements it wrote); the cut is found by searching the bit pattern of e from the top bit down (e <= 1,
-// so 30 bits), then the index among equal values; every count / mass is a fixed-order block reduction, so the result
-// does not depend on timing.  top-k cuts first; top-p then applies to the renormalised top-k set.
-__device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, float top_p, float* e_sm, float* sh_f, int* sh_i) {
+// Nucleus of softmax(z / T) under top-k and top-p.  e_v = exp(z_v/T - m) of this CTA's slice [v_lo, v_hi) is kept in
+// shared memory (a thread only ever touches the elements it wrote); the cut is found by searching the bit pattern of
+// e from the top bit down (e <= 1, so 30 bits), then the index among equal values; every count / mass is a
+// fixed-order reduction, so the result does not depend on timing.  top-k cuts first; top-p then applies to the
+// renormalised top-k set.
+__device__ __noinline__ void build_nucleus(Dist& d, int V, int v_lo, int v_hi, float T, int top_k, float top_p, float* e_sm,
+                                           ClusterRed& R) {
   const int tid = threadIdx.x;
   float m = -INFINITY;
-  for (int v = tid; v < V; v += SEL_THREADS) m = fmaxf(m, d.z[v] / T);
-  m = block_max(m, sh_f);
-  for (int v = tid; v < V; v += SEL_THREADS) e_sm[v] = expf(d.z[v] / T - m);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, d.z[v] / T);
+  m = R.max(m);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) e_sm[v - v_lo] = expf(d.z[v] / T - m);
   d.m = m, d.ecut = 0u, d.vcut = V - 1, d.filt = true;  // everything kept so far
   auto count_if = [&](auto pred) {
     int n = 0;
-    for (int v = tid; v < V; v += SEL_THREADS) n += pred(__float_as_uint(e_sm[v]), v) ? 1 : 0;
-    return block_sum_int(n, sh_i);
+    for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) n += pred(__float_as_uint(e_sm[v - v_lo]), v) ? 1 : 0;
+    return R.sum_int(n);
   };
   auto mass_if = [&](auto pred) {
     float a = 0.f;
-    for (int v = tid; v < V; v += SEL_THREADS) a += pred(__float_as_uint(e_sm[v]), v) ? e_sm[v] : 0.f;
-    return block_sum(a, sh_f);
+    for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) a += pred(__float_as_uint(e_sm[v - v_lo]), v) ? e_sm[v - v_lo] : 0.f;
+    return R.sum(a);
   };
   // lowest index of an element whose value is c (used when c occurs once: no search over the indices is needed)
   auto first_index_of = [&](unsigned c) {
     int best = V;
-    for (int v = tid; v < V; v += SEL_THREADS)
-      if (__float_as_uint(e_sm[v]) == c) best = min(best, v);
-    return -block_sum_int(best == V ? 0 : -best, sh_i);  // at most one thread holds it when the value is unique
+    for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS)
+      if (__float_as_uint(e_sm[v - v_lo]) == c) best = min(best, v);
+    return -R.sum_int(best == V ? 0 : -best);  // exactly one thread of the cluster holds it when the value is unique
   };
   if (top_k > 0 && top_k < V) {
     unsigned c = 0;  // largest c with at least top_k values >= c: the value of the top_k-th ranked token
@@ -197,34 +246,45 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, float T, int top_k, f
 
 // argmax of the logits row of readout column `col` from the per-block maxima the lm_head epilogue left (ties to the
 // lowest index)
-__device__ __forceinline__ int greedy_argmax(const float2* argpart, int n_rb, int col, ArgMax* sh_am) {
+__device__ __forceinline__ int greedy_argmax(const float2* argpart, int n_rb, int col, ClusterRed& R) {
   ArgMax a = {-INFINITY, 0x7fffffff};
   for (int b = threadIdx.x; b < n_rb; b += SEL_THREADS) {
     const float2 v = __ldcg(argpart + (size_t)col * n_rb + b);
     a = better(a, ArgMax{v.x, __float_as_int(v.y)});
   }
-  return block_argmax(a, sh_am).i;
+  return R.block_argmax(a).i;  // every CTA of the cluster reads all partials: no exchange needed
 }
 
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_constant__ SelectParams p) {
   __shared__ ArgMax sh_am[SEL_THREADS / 32];
   __shared__ float sh_f[SEL_THREADS / 32];
+  __shared__ int sh_i[SEL_THREADS / 32];
+  __shared__ float part_f[2 * SEL_CS];
+  __shared__ int part_i[2 * SEL_CS];
+  __shared__ ArgMax part_a[2 * SEL_CS];
+  cg::cluster_group this_cl = cg::this_cluster();
+  ClusterRed R{this_cl, (int)this_cl.num_blocks(), (int)this_cl.block_rank(), 0, sh_f, sh_i, sh_am, part_f, part_i, part_a};
+  const int col = (int)blockIdx.x / R.n_ranks;  // readout column = this cluster
   tune_mark(602, false);
   pdl_launch_dependents();
   // the row table was written before this pass started: everything but the logits can be read ahead of the lm_head
   const RowTable* tab = p.tab;
-  if ((int)blockIdx.x >= tab->n_readout) {  // every CTA waits: a kernel that ends early would release its dependents early
+  if (col >= tab->n_readout) {  // every CTA waits: a kernel that ends early would release its dependents early
     pdl_wait();
     return;
   }
   struct EndMark { __device__ ~EndMark() { tune_mark(602, true); } } end_mark;
-  const int row = tab->ro_rows[blockIdx.x];
+  const int row = tab->ro_rows[col];
   const int kind = tab->readout[row];
   if (!((p.kinds_mask >> kind) & 1)) {
     pdl_wait();
     return;
   }
   const int V = p.V, tid = threadIdx.x;
+  const bool writer = R.rank == 0 && tid == 0;  // all CTAs of the cluster hold the same results; one thread stores them
+  // this CTA's slice of the vocabulary: whole Philox blocks of 4 indices
+  const int per = ((V / 4 + R.n_ranks - 1) / R.n_ranks) * 4;
+  const int v_lo = min(V, R.rank * per), v_hi = min(V, v_lo + per);
   const float T = p.temperature;
   const float* z = p.logits + (size_t)tab->logit_idx[row] * V;
   const int gn = tab->node[row];
@@ -235,21 +295,20 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   const uint2 key = make_uint2((unsigned)(p.seed & 0xffffffffull), (unsigned)(p.seed >> 32));
 
   const bool filt = T > 0.f && ((p.top_k > 0 && p.top_k < V) || p.top_p < 1.0f);
-  extern __shared__ float e_sm[];  // [V] when filters are on
-  __shared__ int sh_i[SEL_THREADS / 32];
+  extern __shared__ float e_sm[];  // this CTA's slice of exp(z/T - max) when filters are on
   // the distribution C(H) of a freshly computed logits row
   auto fresh = [&](const float* zz) -> Dist {
     Dist d;
     d.z = zz, d.filt = false, d.lse = 0.f, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
     if (filt) {
-      build_nucleus(d, V, T, p.top_k, p.top_p, e_sm, sh_f, sh_i);
+      build_nucleus(d, V, v_lo, v_hi, T, p.top_k, p.top_p, e_sm, R);
     } else {  // log sum_v exp(zz_v / T)
       float m = -INFINITY;
-      for (int v = tid; v < V; v += SEL_THREADS) m = fmaxf(m, zz[v] / T);
-      m = block_max(m, sh_f);
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, zz[v] / T);
+      m = R.max(m);
       float s = 0.f;
-      for (int v = tid; v < V; v += SEL_THREADS) s += expf(zz[v] / T - m);
-      s = block_sum(s, sh_f);
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += expf(zz[v] / T - m);
+      s = R.sum(s);
       d.lse = m + logf(s);
     }
     return d;
@@ -262,11 +321,11 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     return d;
   };
   // greedy readouts are always taken from the row the lm_head just produced
-  auto greedy = [&](const float*) -> int { return greedy_argmax(p.argpart, p.n_rb, (int)blockIdx.x, sh_am); };
+  auto greedy = [&](const float*) -> int { return greedy_argmax(p.argpart, p.n_rb, col, R); };
   // exponential race over weights given through logw(v) (-inf = zero weight)
   auto race = [&](auto logw, int purpose) -> int {
     ArgMax a = {-INFINITY, 0x7fffffff};
-    for (int b = tid; b < V / 4; b += SEL_THREADS) {
+    for (int b = v_lo / 4 + tid; b < v_hi / 4; b += SEL_THREADS) {
       uint4 w = philox4x32_10(make_uint4((unsigned)b, position, seq, (unsigned)purpose), key);
       const unsigned ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
@@ -276,7 +335,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
         if (lw > -INFINITY) a = better(a, ArgMax{lw + gumbel_of(ww[e]), v});
       }
     }
-    return block_argmax(a, sh_am).i;
+    return R.argmax(a).i;
   };
   auto uniform = [&](int purpose) -> float {
     return u01(philox4x32_10(make_uint4(0u, position, seq, (unsigned)purpose), key).x);
@@ -291,17 +350,17 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       const Dist dz = fresh(z);
       tok = race([&](int v) { return dz.logw(v, T); }, PUR_VANILLA);
     }
-    if (tid == 0) p.sel_tok[row] = tok;
+    if (writer) p.sel_tok[row] = tok;
     return;
   }
   if (kind == RO_D1) {
     if (T == 0.f) {
       int tok = greedy(z);
-      if (tid == 0) p.sel_tok[row] = tok, p.sel_lse[row] = 0.f;
+      if (writer) p.sel_tok[row] = tok, p.sel_lse[row] = 0.f;
     } else {
       const Dist dz = fresh(z);
       int tok = race([&](int v) { return dz.logw(v, T); }, PUR_DRAFT1);
-      if (tid == 0) {
+      if (writer) {
         p.sel_tok[row] = tok, p.sel_lse[row] = dz.lse;
         if (filt) p.sel_flt[row] = dz.pack();
       }
@@ -312,7 +371,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     const int x1 = p.nodes.tok1[gn];
     if (T == 0.f) {
       int top = greedy(z);
-      if (tid == 0) p.sel_tok[row] = top, p.sel_aux[row] = (top != x1) || !p.gate, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
+      if (writer) p.sel_tok[row] = top, p.sel_aux[row] = (top != x1) || !p.gate, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
       return;
     }
     const Dist d1 = stored(z1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
@@ -325,8 +384,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     if (open) {
       if (p.residual_q2) {
         float s = 0.f;
-        for (int v = tid; v < V; v += SEL_THREADS) s += fmaxf(d2.prob(v, T) - d1.prob(v, T), 0.f);
-        Z2 = block_sum(s, sh_f);
+        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(d2.prob(v, T) - d1.prob(v, T), 0.f);
+        Z2 = R.sum(s);
       }
       if (Z2 > 0.f)
         tok = race([&](int v) {
@@ -335,7 +394,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       else
         tok = race([&](int v) { return d2.logw(v, T); }, PUR_DRAFT2);
     }
-    if (tid == 0) {
+    if (writer) {
       p.sel_tok[row] = tok, p.sel_aux[row] = open, p.sel_lse[row] = d2.lse, p.sel_z2[row] = Z2;
       if (filt) p.sel_flt[row] = d2.pack();
     }
@@ -346,7 +405,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   if (T == 0.f) {
     int top = greedy(z);
     int src = (top == x1) ? 1 : ((has2 && top == x2) ? 2 : 3);
-    if (tid == 0) p.sel_tok[row] = top, p.sel_aux[row] = src;
+    if (writer) p.sel_tok[row] = top, p.sel_aux[row] = src;
     return;
   }
   const float Z2 = p.nodes.z2[gn];
@@ -359,32 +418,32 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   // first proposal: accept with probability min{1, p(x1)/q1(x1)} (Eq. 3)
   const float U1 = uniform(PUR_ACCEPT1);
   if (U1 < fminf(1.0f, pp(x1) / q1(x1))) {
-    if (tid == 0) p.sel_tok[row] = x1, p.sel_aux[row] = 1;
+    if (writer) p.sel_tok[row] = x1, p.sel_aux[row] = 1;
     return;
   }
   // rho1 = p (-) q1 (Eq. 2); if the positive part has no mass rho1 = p
   float s = 0.f;
-  for (int v = tid; v < V; v += SEL_THREADS) s += fmaxf(pp(v) - q1(v), 0.f);
-  const float Z1 = block_sum(s, sh_f);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(pp(v) - q1(v), 0.f);
+  const float Z1 = R.sum(s);
   auto rho1 = [&](int v) { return Z1 > 0.f ? fmaxf(pp(v) - q1(v), 0.f) / Z1 : pp(v); };
   if (!has2) {
     int tok = race([&](int v) { float w = rho1(v); return w > 0.f ? logf(w) : -INFINITY; }, PUR_RESAMPLE);
-    if (tid == 0) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
+    if (writer) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
     return;
   }
   auto q2 = [&](int v) { return Z2 > 0.f ? fmaxf(q2t(v) - q1(v), 0.f) / Z2 : q2t(v); };
   const float U2 = uniform(PUR_ACCEPT2);
   if (U2 < fminf(1.0f, rho1(x2) / q2(x2))) {
-    if (tid == 0) p.sel_tok[row] = x2, p.sel_aux[row] = 2;
+    if (writer) p.sel_tok[row] = x2, p.sel_aux[row] = 2;
     return;
   }
   s = 0.f;
-  for (int v = tid; v < V; v += SEL_THREADS) s += fmaxf(rho1(v) - q2(v), 0.f);
-  const float S2 = block_sum(s, sh_f);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(rho1(v) - q2(v), 0.f);
+  const float S2 = R.sum(s);
   int tok = race([&](int v) {
     float w = S2 > 0.f ? fmaxf(rho1(v) - q2(v), 0.f) : rho1(v);
     return w > 0.f ? logf(w) : -INFINITY; }, PUR_RESAMPLE);
-  if (tid == 0) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
+  if (writer) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
 }
 
 }  // namespace ls
