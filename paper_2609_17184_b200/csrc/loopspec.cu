@@ -261,6 +261,8 @@ struct loopspec_ctx {
   int pass_grid = 0;
   bool pass_coop = true, use_perm = true;
   bool filters = false;  // C applies top-k / top-p (sampling only)
+  int sel_staged = 0;    // the selection kernel keeps its row slices in shared memory
+  size_t sel_smem = 0;
   int launches_per_step = 0;
   std::string err;
 
@@ -547,9 +549,8 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);
   sp.argpart = c->at<float2>(c->L.argpart), sp.n_rb = c->plan[G_LM].n_rb;
   sp.top_k = c->filters ? c->s.top_k : 0, sp.top_p = c->filters ? c->s.top_p : 1.0f, sp.sel_flt = c->at<float4>(c->L.sel_flt);
-  // with filters on, every CTA keeps its slice of exp(z/T - max) in shared memory
-  const size_t smem = c->filters ? (size_t)((c->m.vocab / 4 + SEL_CS - 1) / SEL_CS) * 4 * sizeof(float) : 0;
-  return launch_k(select_kernel, dim3(c->d.max_rows * SEL_CS), dim3(SEL_THREADS), smem, c->stream, sp, c->use_pdl, SEL_CS);
+  sp.staged = c->sel_staged;
+  return launch_k(select_kernel, dim3(c->d.max_rows * SEL_CS), dim3(SEL_THREADS), c->sel_smem, c->stream, sp, c->use_pdl, SEL_CS);
 }
 
 ControlParams control_params(loopspec_ctx* c, int phases) {
@@ -714,11 +715,14 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->s.d1 = d.d1, c->s.d2 = d.d2;
   if (c->s.top_p <= 0.f || c->s.top_p > 1.f) c->s.top_p = 1.f;  // 0 and anything above 1: no nucleus cut
   c->filters = c->s.temperature > 0.f && ((c->s.top_k > 0 && c->s.top_k < m->vocab) || c->s.top_p < 1.f);
-  if (c->filters) {  // the selection kernel then keeps a slice of exp(z/T - max) of a row in shared memory
-    const size_t need = (size_t)((m->vocab / 4 + SEL_CS - 1) / SEL_CS) * 4 * sizeof(float);
-    if (need > 200 * 1024 ||
-        (need > 48 * 1024 &&
-         cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)) {
+  {  // selection kernel, sampling: every CTA stages its slice of up to three logits rows in shared memory, plus the
+     // slice of exp(z/T - max) when C filters; rows too long for that are read from global memory in every pass
+    const size_t slice = (size_t)((m->vocab / 4 + SEL_CS - 1) / SEL_CS) * 4 * sizeof(float);
+    c->sel_staged = c->s.temperature > 0.f && (3 + (c->filters ? 1 : 0)) * slice <= 200 * 1024;
+    c->sel_smem = (c->sel_staged ? 3 * slice : 0) + (c->filters ? slice : 0);
+    if (c->sel_smem > 200 * 1024 ||
+        (c->sel_smem > 48 * 1024 &&
+         cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->sel_smem) != cudaSuccess)) {
       (void)cudaGetLastError();
       delete c;
       return LOOPSPEC_EUNSUPPORTED;

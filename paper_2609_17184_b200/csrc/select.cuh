@@ -41,28 +41,33 @@ struct SelectParams {
   // dynamic shared memory.
   int top_k;
   float top_p;
+  int staged;           // 1: dynamic shared memory holds 3 row slices (+1 when filtering) of ceil(V/4/8)*4 floats each
   float4* sel_flt;      // per row: the nucleus of its readout (max of z/T, kept mass, cut value bits, cut index)
 };
 
 // A readout distribution C(H): softmax(z / T), optionally cut to a nucleus.  Ranking: decreasing e = exp(z/T - m)
 // (as fp32 bit patterns), ties to the lower index; the nucleus is everything ranked at or before (ecut, vcut).
 struct Dist {
-  const float* z;
+  const float* z;   // the logits row in global memory (any index)
+  const float* zs;  // the same row for indices of this CTA's vocabulary slice: a shared-memory copy when staged
   float lse;      // unfiltered: log sum_v exp(z_v / T)
   float m, s;     // filtered: max_v z_v / T and the mass of the kept exp(z_v / T - m)
   unsigned ecut;
   int vcut;
   bool filt;
   __device__ __forceinline__ bool kept(unsigned eb, int v) const { return eb > ecut || (eb == ecut && v <= vcut); }
-  __device__ __forceinline__ float prob(int v, float T) const {
-    if (!filt) return expf(z[v] / T - lse);
-    const float e = expf(z[v] / T - m);
+  __device__ __forceinline__ float prob_of(float zv, int v, float T) const {
+    if (!filt) return expf(zv / T - lse);
+    const float e = expf(zv / T - m);
     return kept(__float_as_uint(e), v) ? e / s : 0.f;
   }
-  // log of an unnormalised weight for the exponential race; -inf outside the support
+  __device__ __forceinline__ float prob(int v, float T) const { return prob_of(z[v], v, T); }    // any index
+  __device__ __forceinline__ float probs(int v, float T) const { return prob_of(zs[v], v, T); }  // index in the slice
+  // log of an unnormalised weight for the exponential race (slice indices); -inf outside the support
   __device__ __forceinline__ float logw(int v, float T) const {
-    if (!filt) return z[v] / T;
-    return kept(__float_as_uint(expf(z[v] / T - m)), v) ? z[v] / T : -INFINITY;
+    const float zv = zs[v];
+    if (!filt) return zv / T;
+    return kept(__float_as_uint(expf(zv / T - m)), v) ? zv / T : -INFINITY;
   }
   __device__ __forceinline__ float4 pack() const { return make_float4(m, s, __uint_as_float(ecut), __int_as_float(vcut)); }
   __device__ __forceinline__ void unpack(float4 f) { m = f.x, s = f.y, ecut = __float_as_uint(f.z), vcut = __float_as_int(f.w), filt = true; }
@@ -182,9 +187,9 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, int v_lo, int v_hi, f
                                            ClusterRed& R) {
   const int tid = threadIdx.x;
   float m = -INFINITY;
-  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, d.z[v] / T);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, d.zs[v] / T);
   m = R.max(m);
-  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) e_sm[v - v_lo] = expf(d.z[v] / T - m);
+  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) e_sm[v - v_lo] = expf(d.zs[v] / T - m);
   d.m = m, d.ecut = 0u, d.vcut = V - 1, d.filt = true;  // everything kept so far
   auto count_if = [&](auto pred) {
     int n = 0;
@@ -295,28 +300,41 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   const uint2 key = make_uint2((unsigned)(p.seed & 0xffffffffull), (unsigned)(p.seed >> 32));
 
   const bool filt = T > 0.f && ((p.top_k > 0 && p.top_k < V) || p.top_p < 1.0f);
-  extern __shared__ float e_sm[];  // this CTA's slice of exp(z/T - max) when filters are on
+  // dynamic shared memory: [staged ? 3 : 0] row slices, then the slice of exp(z/T - max) when filters are on
+  extern __shared__ __align__(16) float dyn_sm[];
+  float* e_sm = dyn_sm + (p.staged ? 3 * per : 0);
+  // Copy this CTA's slice of a logits row into shared memory with every load in flight at once (the sampled paths
+  // pass over up to three rows several times; from global memory each pass is a chain of L2 round trips).  Returns a
+  // pointer indexed by the vocabulary index.
+  auto stage = [&](const float* zz, int slot) -> const float* {
+    if (!p.staged) return zz;
+    float* dst = dyn_sm + slot * per;
+    const float4* src = reinterpret_cast<const float4*>(zz + v_lo);
+    for (int i = tid; i < (v_hi - v_lo) / 4; i += SEL_THREADS) reinterpret_cast<float4*>(dst)[i] = __ldcg(src + i);
+    __syncthreads();
+    return dst - v_lo;
+  };
   // the distribution C(H) of a freshly computed logits row
-  auto fresh = [&](const float* zz) -> Dist {
+  auto fresh = [&](const float* zz, int slot) -> Dist {
     Dist d;
-    d.z = zz, d.filt = false, d.lse = 0.f, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
+    d.z = zz, d.zs = stage(zz, slot), d.filt = false, d.lse = 0.f, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
     if (filt) {
       build_nucleus(d, V, v_lo, v_hi, T, p.top_k, p.top_p, e_sm, R);
     } else {  // log sum_v exp(zz_v / T)
       float m = -INFINITY;
-      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, zz[v] / T);
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) m = fmaxf(m, d.zs[v] / T);
       m = R.max(m);
       float s = 0.f;
-      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += expf(zz[v] / T - m);
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += expf(d.zs[v] / T - m);
       s = R.sum(s);
       d.lse = m + logf(s);
     }
     return d;
   };
   // a distribution stored with a proposal record: its logits row, log-normaliser and (if filtered) nucleus
-  auto stored = [&](const float* zz, float lse, const float4* flt) -> Dist {
+  auto stored = [&](const float* zz, int slot, float lse, const float4* flt) -> Dist {
     Dist d;
-    d.z = zz, d.filt = false, d.lse = lse, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
+    d.z = zz, d.zs = stage(zz, slot), d.filt = false, d.lse = lse, d.m = 0.f, d.s = 1.f, d.ecut = 0u, d.vcut = V - 1;
     if (filt) d.unpack(*flt);
     return d;
   };
@@ -347,7 +365,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     if (T == 0.f) {
       tok = greedy(z);
     } else {
-      const Dist dz = fresh(z);
+      const Dist dz = fresh(z, 0);
       tok = race([&](int v) { return dz.logw(v, T); }, PUR_VANILLA);
     }
     if (writer) p.sel_tok[row] = tok;
@@ -358,7 +376,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       int tok = greedy(z);
       if (writer) p.sel_tok[row] = tok, p.sel_lse[row] = 0.f;
     } else {
-      const Dist dz = fresh(z);
+      const Dist dz = fresh(z, 0);
       int tok = race([&](int v) { return dz.logw(v, T); }, PUR_DRAFT1);
       if (writer) {
         p.sel_tok[row] = tok, p.sel_lse[row] = dz.lse;
@@ -374,8 +392,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
       if (writer) p.sel_tok[row] = top, p.sel_aux[row] = (top != x1) || !p.gate, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
       return;
     }
-    const Dist d1 = stored(z1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
-    const Dist d2 = fresh(z);
+    const Dist d1 = stored(z1, 1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
+    const Dist d2 = fresh(z, 0);
     // Eq. 6; without filters the comparison is made on log-probabilities, as before
     const bool lower = filt ? (d2.prob(x1, T) < d1.prob(x1, T)) : (z[x1] / T - d2.lse < z1[x1] / T - d1.lse);
     const bool open = lower || !p.gate;
@@ -384,12 +402,12 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     if (open) {
       if (p.residual_q2) {
         float s = 0.f;
-        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(d2.prob(v, T) - d1.prob(v, T), 0.f);
+        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(d2.probs(v, T) - d1.probs(v, T), 0.f);
         Z2 = R.sum(s);
       }
       if (Z2 > 0.f)
         tok = race([&](int v) {
-          float w = d2.prob(v, T) - d1.prob(v, T);
+          float w = d2.probs(v, T) - d1.probs(v, T);
           return w > 0.f ? logf(w) : -INFINITY; }, PUR_DRAFT2);
       else
         tok = race([&](int v) { return d2.logw(v, T); }, PUR_DRAFT2);
@@ -409,15 +427,16 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     return;
   }
   const float Z2 = p.nodes.z2[gn];
-  const Dist d1 = stored(z1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
-  const Dist d2 = stored(z2, p.nodes.lse2[gn], p.nodes.flt2 + gn);
-  const Dist dp = fresh(z);
-  auto pp = [&](int v) { return dp.prob(v, T); };    // p_R
-  auto q1 = [&](int v) { return d1.prob(v, T); };    // first proposal
-  auto q2t = [&](int v) { return d2.prob(v, T); };   // deeper readout
+  const Dist d1 = stored(z1, 1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
+  const Dist d2 = has2 ? stored(z2, 2, p.nodes.lse2[gn], p.nodes.flt2 + gn) : d1;
+  const Dist dp = fresh(z, 0);
+  // p_R, the first proposal and the deeper readout: (v) for indices of this CTA's slice, (v, true) for any index
+  auto pp = [&](int v, bool any = false) { return any ? dp.prob(v, T) : dp.probs(v, T); };
+  auto q1 = [&](int v, bool any = false) { return any ? d1.prob(v, T) : d1.probs(v, T); };
+  auto q2t = [&](int v, bool any = false) { return any ? d2.prob(v, T) : d2.probs(v, T); };
   // first proposal: accept with probability min{1, p(x1)/q1(x1)} (Eq. 3)
   const float U1 = uniform(PUR_ACCEPT1);
-  if (U1 < fminf(1.0f, pp(x1) / q1(x1))) {
+  if (U1 < fminf(1.0f, pp(x1, true) / q1(x1, true))) {
     if (writer) p.sel_tok[row] = x1, p.sel_aux[row] = 1;
     return;
   }
@@ -425,15 +444,15 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   float s = 0.f;
   for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(pp(v) - q1(v), 0.f);
   const float Z1 = R.sum(s);
-  auto rho1 = [&](int v) { return Z1 > 0.f ? fmaxf(pp(v) - q1(v), 0.f) / Z1 : pp(v); };
+  auto rho1 = [&](int v, bool any = false) { return Z1 > 0.f ? fmaxf(pp(v, any) - q1(v, any), 0.f) / Z1 : pp(v, any); };
   if (!has2) {
     int tok = race([&](int v) { float w = rho1(v); return w > 0.f ? logf(w) : -INFINITY; }, PUR_RESAMPLE);
     if (writer) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
     return;
   }
-  auto q2 = [&](int v) { return Z2 > 0.f ? fmaxf(q2t(v) - q1(v), 0.f) / Z2 : q2t(v); };
+  auto q2 = [&](int v, bool any = false) { return Z2 > 0.f ? fmaxf(q2t(v, any) - q1(v, any), 0.f) / Z2 : q2t(v, any); };
   const float U2 = uniform(PUR_ACCEPT2);
-  if (U2 < fminf(1.0f, rho1(x2) / q2(x2))) {
+  if (U2 < fminf(1.0f, rho1(x2, true) / q2(x2, true))) {
     if (writer) p.sel_tok[row] = x2, p.sel_aux[row] = 2;
     return;
   }
