@@ -24,8 +24,6 @@ struct AttnParams {
   float* part;                // [row][n_kv][max_chunks][G][D + 2]
   int max_chunks;
   int* counters;              // [row][n_kv]
-  const void* pf_ptr;         // region to prefetch into L2 for a later kernel of the chain (may be null)
-  long long pf_bytes;
   long long* dbg;             // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
   unsigned long long* tl;     // tuning aid: kernel timeline (null in production)
   int tl_id;
@@ -51,7 +49,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_kernel(const __grid_const
   };
   stamp();
   timeline_mark(p.tl, p.tl_id, false);
-  if (threadIdx.x == 0) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
   const RowTable* tab = p.tab;   // written before this pass started: safe to read ahead of the predecessor
   const int n_rows = tab->n_rows;
   const int HQ = p.n_q_heads * D;

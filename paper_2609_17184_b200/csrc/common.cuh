@@ -7,7 +7,7 @@
 
 namespace ls {
 
-// tuning aids (cycle stamps, kernel timeline, L2 prefetch requests) are compiled in only with -DLOOPSPEC_TUNE:
+// tuning aids (cycle stamps, kernel timeline) are compiled in only with -DLOOPSPEC_TUNE:
 // the decode kernels run for a few microseconds each and every kilobyte of code they carry costs fetch time
 #ifdef LOOPSPEC_TUNE
 constexpr bool kTune = true;
@@ -111,24 +111,6 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* row_planes, int ld, i
   row_planes[k] = __ushort_as_bfloat16(h);
   row_planes[ld + k] = __ushort_as_bfloat16(m);
   row_planes[2 * ld + k] = __ushort_as_bfloat16(l);
-}
-
-// Ask L2 to fetch [ptr + slice * per, +per) of a region ahead of the kernel that will stream it (one request per
-// CTA; the region is cut into equal 16-byte-aligned slices).  Used to keep HBM busy with the NEXT kernel's
-// weights while the current kernel is in its latency-bound prologue / epilogue.
-__device__ __forceinline__ void l2_prefetch_slice(const void* ptr, long long bytes, int slice, int n_slices) {
-  if (!kTune || ptr == nullptr || bytes <= 0) return;
-  long long per = ((bytes + n_slices - 1) / n_slices + 15) & ~15ll;
-  long long off = (long long)slice * per;
-  if (off >= bytes) return;
-  long long n = bytes - off < per ? bytes - off : per;
-  n &= ~15ll;
-  const char* src = static_cast<const char*>(ptr) + off;
-  while (n > 0) {  // a single request carries a 32-bit size; keep each well below that
-    unsigned chunk = n > (1ll << 20) ? (1u << 20) : (unsigned)n;
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(chunk) : "memory");
-    src += chunk, n -= chunk;
-  }
 }
 
 // tuning aid: earliest CTA start / latest CTA end of kernel `id` on the global nanosecond timer

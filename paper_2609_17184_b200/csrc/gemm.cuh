@@ -83,8 +83,6 @@ struct GemmParams {
   float2* argpart;        // LOGITS: [column][row block] (largest logit of the block, its vocabulary index as int bits)
   int F;                  // SWIGLU: ffn width
   int perm, perm_a, perm_d;  // order of the row tiles in the packed weights (see packed_tile)
-  const void* pf_ptr;     // region to prefetch into L2 for a later kernel of the chain (may be null)
-  long long pf_bytes;
   long long* dbg;         // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
   unsigned long long* tl; // tuning aid: kernel timeline (null in production)
   int tl_id;
@@ -398,7 +396,6 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
   gemm_load_cols(p, n_cols, NTOK, s_ct);
   // the weights above are constants; everything below reads what earlier kernels of the pass produced
   stamp();
-  if (tid == GEMM_THREADS - 1) l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.x, gridDim.x);
   pdl_launch_dependents();
   pdl_wait();
   stamp();

@@ -256,10 +256,10 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false, use_l2pf = false, l2pf_only_o = false;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false;
   PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
   int pass_grid = 0;
-  bool pass_coop = true, use_perm = true;
+  bool pass_coop = true;
   bool filters = false;  // C applies top-k / top-p (sampling only)
   int sel_staged = 0;    // the selection kernel keeps its row slices in shared memory
   size_t sel_smem = 0;
@@ -398,7 +398,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.xplanes = xpl, p.x_ld = m.hidden;
       // layer 0 reads the full sums the preparation kernel wrote; later layers the down-projection's partials
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.sq_stride;
-      if (!c->packed.empty() && c->use_perm) p.perm = 2, p.perm_a = m.head_dim / 32, p.perm_d = m.head_dim;
+      if (!c->packed.empty() ) p.perm = 2, p.perm_a = m.head_dim / 32, p.perm_d = m.head_dim;
       p.qbuf = c->at<float>(c->L.qbuf);
       p.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)layer * c->kv_layer_stride();
       p.kv_plane_stride = c->kv_plane_stride(), p.kv_sel_stride = c->kv_sel_stride();
@@ -413,7 +413,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       break;
     case G_GU:
       p.W = c->packed.empty() ? lp[4] : c->packed[4 * layer + 2], p.N = 2 * m.ffn, p.K = m.hidden, p.F = m.ffn;
-      if (!c->packed.empty() && c->use_perm) p.perm = 1, p.perm_a = m.ffn;
+      if (!c->packed.empty() ) p.perm = 1, p.perm_a = m.ffn;
       p.xplanes = xpl, p.x_ld = m.hidden;
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.sq_stride;
       p.out_planes = c->at<__nv_bfloat16>(c->L.splanes), p.planes_ld = m.ffn;
@@ -434,18 +434,6 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       break;
   }
   return p;
-}
-
-// the region a kernel of the chain asks L2 to fetch for a later one: the packed weights of GEMM `which`, layer l
-void prefetch_target(loopspec_ctx* c, int which, int l, const void** ptr, long long* bytes) {
-  *ptr = nullptr, *bytes = 0;
-  if (c->packed.empty() || !c->use_l2pf || l >= c->m.n_recurrent) return;
-  if (c->l2pf_only_o && which != G_O) return;
-  const Derived& d = c->d;
-  const int Ns[4] = {d.Hq + 2 * d.Hkv, c->m.hidden, 2 * c->m.ffn, c->m.hidden};
-  const int Ks[4] = {c->m.hidden, d.Hq, c->m.hidden, c->m.ffn};
-  *ptr = c->packed[4 * l + which];
-  *bytes = (long long)packed_bytes(Ns[which], Ks[which]);
 }
 
 cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
@@ -502,7 +490,6 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     unsigned long long* tl = getenv("LOOPSPEC_DBG") ? reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024 : nullptr;  // tuning aid
     GemmParams gq = gemm_params(c, G_QKV, l, tab);
     gq.tl = tl, gq.tl_id = l * 5 + 0;
-    prefetch_target(c, G_O, l, &gq.pf_ptr, &gq.pf_bytes);          // QKV runs: fetch W_o
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
     AttnParams a;
     memset(&a, 0, sizeof a);
@@ -512,7 +499,6 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
-    prefetch_target(c, G_GU, l, &a.pf_ptr, &a.pf_bytes);           // attention runs: fetch W_gate/up
     if (l == 3 && getenv("LOOPSPEC_DBG")) a.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart) + 64;  // tuning aid
     a.tl = tl, a.tl_id = l * 5 + 1;
     if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
@@ -521,11 +507,9 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
     GemmParams gg = gemm_params(c, G_GU, l, tab);
     gg.tl = tl, gg.tl_id = l * 5 + 3;
-    prefetch_target(c, G_DOWN, l, &gg.pf_ptr, &gg.pf_bytes);       // gate/up runs: fetch W_down
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
     GemmParams gd = gemm_params(c, G_DOWN, l, tab);
     gd.tl = tl, gd.tl_id = l * 5 + 4;
-    prefetch_target(c, G_QKV, l + 1, &gd.pf_ptr, &gd.pf_bytes);    // down runs: fetch the next layer's W_qkv
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
   }
@@ -739,17 +723,10 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / resid_rows, (m->ffn + 63) / 64, m->hidden / resid_rows, (m->vocab + 127) / 128};
   const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
   int slots = n_sm * kCtasPerSm;
-  if (const char* env = getenv("LOOPSPEC_SLOTS")) slots = std::max(1, atoi(env));  // tuning aid
   for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
-  if (const char* env = getenv("LOOPSPEC_NCL")) {  // tuning aid: clusters per GEMM "qkv,o,gateup,down,lmhead" (0 = keep)
-    int v[5];
-    if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
-      for (int i = 0; i < 5; ++i)
-        if (v[i] > 0 && v[i] <= c->plan[i].n_rb) c->plan[i].n_clusters = v[i], c->plan[i].grid = v[i] * c->plan[i].cs;
-  }
   // Every kernel of the chain asks for the same (largest) shared-memory carve-out: the GEMM CTAs need it, and an SM
   // whose partition was set by a small-shared-memory kernel would have to drain before it can host one.
-  if (!getenv("LOOPSPEC_NO_CARVEOUT")) {  // tuning aid
+  {
     const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads), (const void*)prep_planes_kernel,
                                (const void*)select_kernel, (const void*)control_kernel, (const void*)vanilla_control_kernel,
                                (const void*)kv_commit_kernel};
@@ -766,7 +743,6 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           return LOOPSPEC_ECUDA;
         }
   if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
-  if (const char* env = getenv("LOOPSPEC_L2PF")) c->use_l2pf = env[0] != '0', c->l2pf_only_o = env[0] == '2';  // tuning aid
   if (getenv("LOOPSPEC_DBG")) {
     fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
 #ifdef LOOPSPEC_TUNE
@@ -840,9 +816,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // bf16 weights: repack every matrix once into the tile-major streaming layout held in the workspace
   if (m->weight_dtype == 1) {
     unsigned char* dst = c->ws + L.wpack;
-    if (getenv("LOOPSPEC_NOPERM")) c->use_perm = false;  // tuning aid
     auto pack = [&](const void* src, int N, int K, int perm = 0, int perm_a = 0) -> bool {
-      if (!c->use_perm) perm = 0;
       PackParams pp;
       pp.src = static_cast<const __nv_bfloat16*>(src), pp.dst = reinterpret_cast<__nv_bfloat16*>(dst), pp.N = N, pp.K = K;
       pp.kpr = (K + 31) / 32, pp.perm = perm, pp.perm_a = perm_a, pp.perm_d = m->head_dim;
@@ -862,10 +836,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
   }
   // persistent pass kernel: available for bf16 weights when a decode pass carries at most 8 rows
-  if (m->weight_dtype == 1 && c->use_perm && c->ng_dec == 1 && m->ffn % 16 == 0 && m->head_dim % 32 == 0 && m->hidden % 16 == 0) {
+  if (m->weight_dtype == 1 && c->ng_dec == 1 && m->ffn % 16 == 0 && m->head_dim % 32 == 0 && m->hidden % 16 == 0) {
     PassFn fn = pass_fn(m->head_dim, m->n_q_heads / m->n_kv_heads);
     int max_clusters = 0;
-    if (const char* env = getenv("LOOPSPEC_NOCOOP")) c->pass_coop = env[0] != '1';  // tuning aid
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute at[2];
     pass_launch_config(c, &cfg, at, 1);
@@ -873,7 +846,6 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pass_smem_bytes()) == cudaSuccess &&
         cudaOccupancyMaxActiveClusters(&max_clusters, fn, &cfg) == cudaSuccess && max_clusters >= 1) {
       int nc = std::min(max_clusters, d.sq_stride);
-      if (const char* env = getenv("LOOPSPEC_NC")) nc = std::max(1, std::min(nc, atoi(env)));  // tuning aid
       c->pass_grid = nc * PASS_CS;
       std::vector<const void*> tabs((size_t)m->n_recurrent * 10);
       for (int l = 0; l < m->n_recurrent; ++l) {
@@ -1198,7 +1170,6 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
       if (getenv("LOOPSPEC_DBG")) p.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart);  // tuning aid
-      if (getenv("LOOPSPEC_PFSELF") && which < 4) prefetch_target(c, which, (i + 1) % L, &p.pf_ptr, &p.pf_bytes);  // tuning aid
       cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }
