@@ -40,7 +40,7 @@ constexpr int TILE_LD = 132;   // padded leading dimension of the partial tile
 constexpr int RING = LS_RING;  // weight stages per thread (8 KB per stage per CTA), RING - 1 of them in flight
 constexpr int MAX_XCH_BLOCKS = LS_XCH;  // k-blocks of activations one CTA keeps staged when NG = 1
 // per-column copies of the row-table fields the epilogues need ([field][column] in shared memory)
-enum { CT_POS = 0, CT_R = 1, CT_SEQ = 2, CT_SLOT = 3, CT_HID = 4, CT_LOGIT = 5, CT_FIELDS = 6 };
+enum { CT_POS = 0, CT_R = 1, CT_SEQ = 2, CT_SLOT = 3, CT_HID = 4, CT_LOGIT = 5, CT_XROW = 6, CT_FIELDS = 7 };
 
 __host__ __device__ constexpr int xchunk_kblocks(int NG) { return MAX_XCH_BLOCKS / NG; }
 __host__ __device__ constexpr int xbuf_uint4(int NG) { return 3 * xchunk_kblocks(NG) * 8 * NG * 4; }
@@ -265,12 +265,13 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
 
 // 1/rms of every live column: warp w sums the partial sums of squares of columns w, w + 8, ... (one partial per lane,
 // butterfly sum: the same order in every launch)
-__device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float* s_rstd) {
+__device__ __forceinline__ void gemm_rstd(const GemmParams& p, int n_cols, float* s_rstd, const int* ct, int ntok) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int c = warp; c < n_cols; c += GEMM_THREADS / 32) {
+    const int xr = p.cols_from_readout ? ct[CT_XROW * ntok + c] : c;  // the lm_head's columns are the reading-out rows
     float ss = 0.f;
     if (p.sumsq)
-      for (int j = lane; j < p.n_sq; j += 32) ss += p.sumsq[c * p.sq_stride + j];
+      for (int j = lane; j < p.n_sq; j += 32) ss += p.sumsq[xr * p.sq_stride + j];
     ss = warp_sum(ss);
     if (lane == 0) s_rstd[c] = p.sumsq ? 1.0f / sqrtf(ss / (float)p.H + p.eps) : 1.0f;
   }
@@ -284,6 +285,7 @@ __device__ __forceinline__ void gemm_load_cols(const GemmParams& p, int n_cols, 
     const int row = p.cols_from_readout ? tab->ro_rows[c] : c;
     ct[CT_POS * ntok + c] = tab->pos[row], ct[CT_R * ntok + c] = tab->r[row], ct[CT_SEQ * ntok + c] = tab->seq[row];
     ct[CT_SLOT * ntok + c] = tab->kv_slot[row], ct[CT_HID * ntok + c] = tab->hid_idx[row], ct[CT_LOGIT * ntok + c] = tab->logit_idx[row];
+    ct[CT_XROW * ntok + c] = row;  // where the column's activation planes and sums of squares live
   }
 }
 
@@ -414,9 +416,10 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
     constexpr int KPR = GEMM_THREADS / (4 * NTOK);  // k-blocks per round
     const int tt = tid & 3, c = (tid >> 2) % NTOK, kq = tid / (4 * NTOK);
     if (c < n_cols) {
+      const int xr = p.cols_from_readout ? s_ct[CT_XROW * NTOK + c] : c;
 #pragma unroll
       for (int s = 0; s < 3; ++s) {
-        const __nv_bfloat16* src = p.xplanes + ((size_t)c * 3 + s) * p.x_ld + (kb0 + kq) * 32 + tt * 8;
+        const __nv_bfloat16* src = p.xplanes + ((size_t)xr * 3 + s) * p.x_ld + (kb0 + kq) * 32 + tt * 8;
         uint4* dst = xbuf + ((s * XCH + kq) * NTOK + c) * 4 + tt;
 #pragma unroll
         for (int j = 0; j < XCH; j += KPR) {
@@ -455,9 +458,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
       const int nkb = min(XCH, upt - ck);
       const bool first = task == 0 && ck == 0;
       if (first || !one_chunk) {  // wide passes (prefill) restage the activations chunk by chunk
-        if (!first) __syncthreads();
+        if (!first || p.cols_from_readout) __syncthreads();  // (the lm_head's staging reads the column table)
         x_stage(kb_lo + ck, nkb);
-        if (first) gemm_rstd(p, n_cols, s_rstd);
+        if (first) gemm_rstd(p, n_cols, s_rstd, s_ct, NTOK);
         cp_async_wait<0>();
         __syncthreads();
         if (first) stamp();
@@ -549,7 +552,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   if (n_cols > NTOK) n_cols = NTOK;
   if (n_cols <= 0) return;
   gemm_load_cols(p, n_cols, NTOK, s_ct);
-  gemm_rstd(p, n_cols, s_rstd);
+  __syncthreads();
+  gemm_rstd(p, n_cols, s_rstd, s_ct, NTOK);
 
   for (int task = 0; task < n_tasks; ++task) {
     const int rb = cid + task * p.n_clusters;
@@ -567,7 +571,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
         int k = (kb_lo + ck + kbl) * 32 + e;
         float v = 0.f;
         if (c < n_cols && k < p.K) {
-          const __nv_bfloat16* pl = p.xplanes + (size_t)c * 3 * p.x_ld + k;
+          const int xr = p.cols_from_readout ? s_ct[CT_XROW * NTOK + c] : c;
+          const __nv_bfloat16* pl = p.xplanes + (size_t)xr * 3 * p.x_ld + k;
           v = (__bfloat162float(pl[0]) + __bfloat162float(pl[p.x_ld])) + __bfloat162float(pl[2 * p.x_ld]);
         }
         xf[idx] = v;
@@ -659,21 +664,19 @@ struct PrepParams {
   __nv_bfloat16* planes;    // [col][3][K]
   float* sumsq;             // [col * sq_stride] full sum of squares (may be null)
   int sq_stride;
-  int readout_only;         // columns are the reading-out rows
 };
 
 __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant__ PrepParams p) {
   __shared__ float s_part[8];
-  tune_mark(600 + p.readout_only, false);
+  tune_mark(600, false);
   pdl_launch_dependents();
   pdl_wait();
   const int c = blockIdx.x;
-  int n = p.tab ? (p.readout_only ? p.tab->n_readout : p.tab->n_rows) : p.m_fixed;
+  int n = p.tab ? p.tab->n_rows : p.m_fixed;
   if (c >= n) return;
   const float* src;
   if (p.tab) {
-    int row = p.readout_only ? p.tab->ro_rows[c] : c;
-    src = p.hid + (size_t)p.tab->hid_idx[row] * p.K;
+    src = p.hid + (size_t)p.tab->hid_idx[c] * p.K;
   } else {
     src = p.x + (size_t)c * p.K;
   }
@@ -692,7 +695,7 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
     for (int w = 0; w < 8; ++w) tsum += s_part[w];
     p.sumsq[c * p.sq_stride] = tsum;
   }
-  tune_mark(600 + p.readout_only, true);
+  tune_mark(600, true);
 }
 
 }  // namespace ls

@@ -73,7 +73,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, sumsq_ro, logits, argpart, flt, sel_flt, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, flt, sel_flt, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -199,7 +199,6 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.aplanes = take(MR * 3 * d.Hq * 2);
   L.splanes = take(MR * 3 * m->ffn * 2);
   L.sumsq = take(MR * d.sq_stride * 4);
-  L.sumsq_ro = take(MR * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
   L.argpart = take(MR * ((m->vocab + 127) / 128) * sizeof(float2));
   // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
@@ -422,26 +421,27 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.W = c->packed.empty() ? lp[5] : c->packed[4 * layer + 3], p.N = m.hidden, p.K = m.ffn;
       p.xplanes = c->at<__nv_bfloat16>(c->L.splanes), p.x_ld = m.ffn;
       p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.sq_stride;
-      if (layer + 1 < m.n_recurrent) {
-        p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(c->layers[6 * (layer + 1)]);
-      }
+      // planes for the next consumer of the residual stream: the next layer's first norm, or - after the last
+      // layer - the final norm of the readout (the lm_head picks the reading-out rows out of them)
+      p.out_planes = xpl, p.planes_ld = m.hidden;
+      p.gain_next = layer + 1 < m.n_recurrent ? static_cast<const float*>(c->layers[6 * (layer + 1)]) : c->final_norm;
       break;
     default:
       p.W = c->packed.empty() ? c->lm_head : c->packed[4 * m.n_recurrent], p.N = m.vocab, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden, p.cols_from_readout = 1;
-      p.sumsq = c->at<float>(c->L.sumsq_ro), p.n_sq = 1, p.sq_stride = 1;
+      // 1/rms from the partial sums of squares the last down projection left for the row
+      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.sq_stride;
       p.logits = c->at<float>(c->L.logits), p.argpart = c->at<float2>(c->L.argpart);
       break;
   }
   return p;
 }
 
-cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, bool readout) {
+cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab) {
   PrepParams q;
   memset(&q, 0, sizeof q);
   q.tab = tab, q.hid = c->at<float>(c->L.hid), q.K = c->m.hidden, q.planes = c->at<__nv_bfloat16>(c->L.xplanes);
-  if (readout) q.gain = c->final_norm, q.sumsq = c->at<float>(c->L.sumsq_ro), q.sq_stride = 1, q.readout_only = 1;
-  else q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.sq_stride;
+  q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.sq_stride;
   return launch_k(prep_planes_kernel, dim3(c->d.max_rows), dim3(256), 0, c->stream, q, c->use_pdl);
 }
 
@@ -476,7 +476,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   const int G = m.n_q_heads / m.n_kv_heads;
   const bool pdl = c->use_pdl;
   cudaError_t e;
-  if ((e = launch_prep(c, tab, false))) return e;
+  if ((e = launch_prep(c, tab))) return e;
   if (n_launch) *n_launch += 1;
   if (c->use_mega && ng == 1) {
     if ((e = cudaMemsetAsync(c->ws + c->L.bar, 0, 8, c->stream))) return e;
@@ -517,9 +517,8 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
 }
 
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
-  cudaError_t e;
-  if ((e = launch_prep(c, tab, true))) return e;
   GemmParams gl = gemm_params(c, G_LM, 0, tab);
+  gl.n_sq = (c->use_mega && ng == 1) ? c->pass.n_clusters : c->d.n_sq;  // partials the layers of this pass left per row
   if (getenv("LOOPSPEC_DBG")) gl.tl = reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024, gl.tl_id = 120;  // tuning aid
   return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
 }
@@ -575,7 +574,7 @@ cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_com
   if ((e = launch_lm_head(c, tab, c->ng_dec))) return e;
   if ((e = launch_select(c, tab, kinds_mask))) return e;
   if ((e = launch_control(c, phases))) return e;
-  if (n_launch) *n_launch += 4;
+  if (n_launch) *n_launch += 3;
   if (kv_commit) {
     if ((e = launch_kv_commit(c))) return e;
     if (n_launch) *n_launch += 1;
@@ -857,7 +856,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         return bail(LOOPSPEC_ECUDA, "pointer table upload");
       PassParams& q = c->pass;
       memset(&q, 0, sizeof q);
-      q.L = m->n_recurrent, q.n_clusters = nc;
+      q.L = m->n_recurrent, q.n_clusters = nc, q.final_gain = c->final_norm;
       q.wpacked = c->at<const void*>(L.ptrs), q.layer_w = c->at<const void*>(L.ptrs) + (size_t)m->n_recurrent * 4;
       q.H = m->hidden, q.Hq = d.Hq, q.Hkv = d.Hkv, q.F = m->ffn, q.n_q_heads = m->n_q_heads, q.n_kv_heads = m->n_kv_heads;
       q.head_dim = m->head_dim, q.slots = d.slots, q.eps = m->rms_eps, q.scale = 1.0f / sqrtf((float)m->head_dim);
@@ -1144,7 +1143,7 @@ int loopspec_debug_logits(loopspec_ctx* c, int32_t seq, int32_t which, float* ou
 
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
-  *out = c->use_mega ? 8 : c->m.n_recurrent * 5 + 6;
+  *out = c->use_mega ? 6 : c->m.n_recurrent * 5 + 5;
   return LOOPSPEC_OK;
 }
 

@@ -37,6 +37,7 @@ struct PassParams {
   int L;
   const void* const* wpacked;   // device [L][4] tile-major weights: qkv, o, gate/up, down
   const void* const* layer_w;   // device [L][6] original pointers (norm gains: [0] norm1, [3] norm2)
+  const float* final_gain;      // gain of the readout's final norm (planes after the last layer)
   int H, Hq, Hkv, F, n_q_heads, n_kv_heads, head_dim, slots;
   float eps, scale;
   float* hid;
@@ -464,7 +465,7 @@ __global__ void __launch_bounds__(PASS_THREADS, 2) pass_kernel(const __grid_cons
       const bool resid = (st == ST_O || st == ST_DOWN);
       const float* gain_next = nullptr;
       if (st == ST_O) gain_next = static_cast<const float*>(p.layer_w[l * 6 + 3]);
-      else if (st == ST_DOWN && l + 1 < p.L) gain_next = static_cast<const float*>(p.layer_w[(l + 1) * 6 + 0]);
+      else if (st == ST_DOWN) gain_next = l + 1 < p.L ? static_cast<const float*>(p.layer_w[(l + 1) * 6 + 0]) : p.final_gain;
       float pre_h = 0.f, pre_g = 1.f;
       float* h_ptr = nullptr;
       const int n_glob = ge.g_lo * 16 + tid;  // single tiles: output row of thread tid
