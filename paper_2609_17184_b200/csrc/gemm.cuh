@@ -42,7 +42,9 @@ constexpr int MAX_XCH_BLOCKS = LS_XCH;  // k-blocks of activations one CTA keeps
 // per-column copies of the row-table fields the epilogues need ([field][column] in shared memory)
 enum { CT_POS = 0, CT_R = 1, CT_SEQ = 2, CT_SLOT = 3, CT_HID = 4, CT_LOGIT = 5, CT_XROW = 6, CT_FIELDS = 7 };
 
-__host__ __device__ constexpr int xchunk_kblocks(int NG) { return MAX_XCH_BLOCKS / NG; }
+// k-blocks of activations staged at a time.  The wide kernels (NG >= 4: prefill, batches) need too many registers for
+// two CTAs per SM anyway, so they take a larger staging buffer and restage less often.
+__host__ __device__ constexpr int xchunk_kblocks(int NG) { return NG >= 8 ? 8 : NG == 4 ? 12 : MAX_XCH_BLOCKS / NG; }
 __host__ __device__ constexpr int xbuf_uint4(int NG) { return 3 * xchunk_kblocks(NG) * 8 * NG * 4; }
 // partial columns received from the cluster's ranks: [rank][owned column][128 rows]
 __host__ __device__ constexpr int recv_floats(int NG) { return (8 * NG + 7) * RB_ROWS; }
