@@ -153,6 +153,24 @@ def test_filtered_sampling_matches_oracle(name, n_prompt, n_decode, d1, d2, T, t
     ctx.close()
 
 
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,top_k,top_p", [
+    ("tiny_bf16", 11, 40, 1, 2, 0.0, 0, 1.0), ("tiny_bf16", 16, 40, 1, 2, 1.0, 0, 1.0), ("tiny_bf16", 9, 40, 2, 0, 0.9, 0, 0.7),
+    ("tiny", 16, 40, 1, 3, 1.1, 30, 0.9), ("small_bf16", 33, 24, 1, 2, 1.0, 0, 1.0)])
+def test_parity_holds_across_seeds(name, n_prompt, n_decode, d1, d2, T, top_k, top_p):
+    """Not one lucky seed: eight prompt / sampling seeds per setting, tokens and counters equal to the oracle's."""
+    for seed in range(1, 9):
+        ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=seed, prompt_seed=seed + 10, top_k=top_k, top_p=top_p)
+        ctx = U.make_ctx(name, d1, d2, T=T, seed=seed, max_ctx=n_prompt + n_decode + 8, top_k=top_k, top_p=top_p)
+        assert ctx.prefill(ref["prompt"]) == ref["first"], seed
+        out = ctx.decode(n_decode)[0].tolist()
+        margins = sorted((e["margin"], e["kind"]) for e in ref["dec"].log if e["kind"] != "filter")[:3]
+        assert out == ref["tokens"], (seed, U.first_diff(out, ref["tokens"]), margins)
+        st, so = ctx.stats(), ref["dec"].stats
+        for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
+            assert st[k] == so[k], (seed, k, st[k], so[k])
+        ctx.close()
+
+
 def test_filters_off_values_and_unsupported_vocab():
     """top_k = 0 with top_p = 0 or 1 is the plain softmax: bit-identical to a context built without the fields."""
     ref = U.oracle_run("tiny_bf16", 16, 24, 1, 2, T=1.0, seed=2)
