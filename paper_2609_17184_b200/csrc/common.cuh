@@ -17,7 +17,20 @@ constexpr bool kTune = false;
 
 constexpr int MAX_ROWS = 64;  // rows (branches) one batched pass can carry: 8 token columns x up to 8 groups
 constexpr int MAX_SPEC = 8;   // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
-constexpr int ATT_CHUNK = 64; // key positions per attention work item (fixed by absolute position)
+constexpr int ATT_CHUNK = 64; // key positions per attention chunk (cut at fixed absolute positions)
+constexpr int ATT_MAX_RUNS = 32;  // attention work items per (row, kv head) at most
+constexpr int ATT_LONG_RUNS = 16; // ... and for contexts of more than ATT_MAX_RUNS chunks
+// A work item covers a run of consecutive chunks: one chunk for contexts up to ATT_MAX_RUNS chunks, beyond that as
+// many as leave ATT_LONG_RUNS items (a function of the row's own context only, so a row's arithmetic does not depend
+// on what shares the pass).
+__host__ __device__ inline int att_run_len(int n_canon) {
+  const int nc = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK;
+  return nc <= ATT_MAX_RUNS ? 1 : (nc + ATT_LONG_RUNS - 1) / ATT_LONG_RUNS;
+}
+__host__ __device__ inline int att_items(int n_canon) {
+  const int nc = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK, rl = att_run_len(n_canon);
+  return (nc + rl - 1) / rl;
+}
 
 // readout kinds of a row after its advance (Algorithm 1: r_b = d1, r_b = d2, r_b = R)
 enum { RO_NONE = 0, RO_D1 = 1, RO_D2 = 2, RO_VERIFY = 3, RO_TARGET = 4 /* x ~ C(H): prefill, vanilla */ };
@@ -26,7 +39,7 @@ enum { RO_NONE = 0, RO_D1 = 1, RO_D2 = 2, RO_VERIFY = 3, RO_TARGET = 4 /* x ~ C(
 struct RowTable {
   int n_rows;
   int n_readout;             // rows whose new depth is d1, d2 or R
-  int attn_items;            // sum over rows of attention chunks
+  int attn_items;            // sum over rows of attention work items (runs of chunks)
   int n_layers_done;         // unused, keeps the header 16 bytes
   int seq[MAX_ROWS];         // sequence of the row
   int r[MAX_ROWS];           // recurrence the row is advanced TO (1..R): KV plane it writes and reads
@@ -41,7 +54,7 @@ struct RowTable {
   int logit_idx[MAX_ROWS];   // which logits vector its readout fills
   int node[MAX_ROWS];        // global node index (seq * NB + node), -1 for prefill rows
   int ro_rows[MAX_ROWS];     // compact list of rows with readout != 0
-  int chunk_start[MAX_ROWS + 1];  // exclusive prefix sum of attention chunks per row
+  int chunk_start[MAX_ROWS + 1];  // exclusive prefix sum of attention work items per row
 };
 
 // Branch table of Algorithm 1 (a branch: prefix, hidden state, depth, proposal records), per sequence NB nodes.

@@ -124,7 +124,7 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       t.readout[i] = ro, t.logit_idx[i] = li;
       if (ro) t.ro_rows[n_ro++] = i;
       t.chunk_start[i] = items;
-      items += (t.n_canon[i] + ATT_CHUNK - 1) / ATT_CHUNK;
+      items += att_items(t.n_canon[i]);
     }
   }
   t.chunk_start[n_rows] = items;
@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
         t.n_safe[i] = pos;
         t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE;
         t.logit_idx[i] = p.p_logit_base + s, t.ro_rows[i] = i, t.chunk_start[i] = items;
-        items += (pos + 1 + ATT_CHUNK - 1) / ATT_CHUNK;
+        items += att_items(pos + 1);
       }
       t.chunk_start[n] = items;
       t.n_rows = n, t.n_readout = (r == p.R) ? n : 0, t.attn_items = items, t.n_layers_done = 0;
@@ -376,7 +376,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
       t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;
       if (last) t.ro_rows[n_ro++] = i;
       t.chunk_start[i] = items;
-      items += (pos + 1 + ATT_CHUNK - 1) / ATT_CHUNK;
+      items += att_items(pos + 1);
       s_emb[i][0] = p.hid_base + i, s_emb[i][1] = p.prompt[pos];
     }
     t.chunk_start[p.count] = items;

@@ -372,7 +372,11 @@ cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, cudaStrea
 }
 
 using AttnFn = void (*)(const AttnParams);
-AttnFn attn_fn(int d, int G) {
+AttnFn attn_fn(int d, int G, bool runs) {  // runs: contexts longer than ATT_MAX_RUNS chunks are possible
+  if (runs) {
+    if (d == 128) return G == 1 ? attn_runs_kernel<128, 1> : attn_runs_kernel<128, 4>;
+    return G == 1 ? attn_runs_kernel<64, 1> : attn_runs_kernel<64, 4>;
+  }
   if (d == 128) return G == 1 ? attn_kernel<128, 1> : attn_kernel<128, 4>;
   return G == 1 ? attn_kernel<64, 1> : attn_kernel<64, 4>;
 }
@@ -501,7 +505,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
     if (l == 3 && getenv("LOOPSPEC_DBG")) a.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart) + 64;  // tuning aid
     a.tl = tl, a.tl_id = l * 5 + 1;
-    if ((e = launch_k(attn_fn(m.head_dim, G), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
+    if ((e = launch_k(attn_fn(m.head_dim, G, d.max_chunks > ATT_MAX_RUNS), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
     GemmParams go = gemm_params(c, G_O, l, tab);
     go.tl = tl, go.tl_id = l * 5 + 2;
     if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
@@ -726,7 +730,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // Every kernel of the chain asks for the same (largest) shared-memory carve-out: the GEMM CTAs need it, and an SM
   // whose partition was set by a small-shared-memory kernel would have to drain before it can host one.
   {
-    const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads), (const void*)prep_planes_kernel,
+    const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads, d.max_chunks > ATT_MAX_RUNS), (const void*)prep_planes_kernel,
                                (const void*)select_kernel, (const void*)control_kernel, (const void*)vanilla_control_kernel,
                                (const void*)kv_commit_kernel};
     for (const void* f : small_fns)
@@ -879,6 +883,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         if ((q.kpr[i] + PASS_CS - 1) / PASS_CS > PASS_XCH) fits = false;
       }
       c->use_mega = false;  // opt-in: LOOPSPEC_MEGA=1
+      if (d.max_chunks > ATT_MAX_RUNS) fits = false;  // its attention stage works on single chunks
       if (const char* env = getenv("LOOPSPEC_MEGA")) c->use_mega = fits && env[0] == '1';
       if (getenv("LOOPSPEC_DBG")) {  // tuning aid: timestamps land in the unused tail of the partial buffer
         q.dbg = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + (1 << 20);
