@@ -18,7 +18,7 @@ constexpr bool kTune = false;
 constexpr int MAX_ROWS = 64;  // rows (branches) one batched pass can carry: 8 token columns x up to 8 groups
 constexpr int MAX_SPEC = 8;   // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
 constexpr int ATT_CHUNK = 64; // key positions per attention chunk (cut at fixed absolute positions)
-constexpr int ATT_MAX_RUNS = 32;  // attention work items per (row, kv head) at most
+constexpr int ATT_MAX_RUNS = 40;  // attention work items per (row, kv head) at most (contexts up to 2560: one chunk each)
 constexpr int ATT_LONG_RUNS = 8;  // ... and for contexts of more than ATT_MAX_RUNS chunks
 // A work item covers a run of consecutive chunks: one chunk for contexts up to ATT_MAX_RUNS chunks, beyond that as
 // many as leave ATT_LONG_RUNS items (a function of the row's own context only, so a row's arithmetic does not depend

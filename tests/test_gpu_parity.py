@@ -297,16 +297,14 @@ def test_depths_from_the_closed_form_are_used_when_none_are_given():
 
 
 @pytest.mark.parametrize("T", [0.0, 1.0])
-def test_context_beyond_2048_uses_runs_of_attention_chunks(T):
-    """A 2200-token prompt: more than 32 chunks per row, so attention work items are runs of several chunks folded with
-    the running-softmax rescaling (prefill positions beyond 2048 and every decode row)."""
-    ref = U.oracle_run("tiny_bf16", 2200, 16, 1, 2, T=T, seed=3)
-    ctx = U.make_ctx("tiny_bf16", 1, 2, T=T, seed=3, max_ctx=2240, max_prefill_rows=64)
+def test_context_beyond_2560_uses_runs_of_attention_chunks(T):
+    """A 2700-token prompt: more than 40 chunks per row, so attention work items are runs of several chunks folded with
+    the running-softmax rescaling (prefill positions beyond 2560 and every decode row)."""
+    ref = U.oracle_run("tiny_bf16", 2700, 16, 1, 2, T=T, seed=3)
+    ctx = U.make_ctx("tiny_bf16", 1, 2, T=T, seed=3, max_ctx=2740, max_prefill_rows=64)
     assert ctx.prefill(ref["prompt"]) == ref["first"]
     ctx.decode(16)
     U.assert_same_run(ctx, ref, 16)
-    # the same sequence in a context sized below the threshold for runs must not exist: sanity of the test itself
-    assert 2200 // 64 > 32
     ctx.close()
 
 
