@@ -393,6 +393,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   const GemmPlan& g = c->plan[which];
   p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.cluster_size = g.cs, p.n_clusters = g.n_clusters;
   p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
+  p.err = c->host_flags_dev + HF_ERROR;
   const void* const* lp = which == G_LM ? nullptr : &c->layers[6 * layer];
   __nv_bfloat16* xpl = c->at<__nv_bfloat16>(c->L.xplanes);
   switch (which) {
@@ -612,7 +613,7 @@ int check_device_error(loopspec_ctx* c) {
   if (!e) return LOOPSPEC_OK;
   c->host_flags[HF_ERROR] = 0;
   return fail(c, LOOPSPEC_ECAPACITY, "device scheduler reported %s",
-              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : e == 4 ? "a grid barrier timed out" : "speculative chain too deep");
+              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : e == 4 ? "a grid barrier timed out" : e == 5 ? "a bulk copy did not complete" : "speculative chain too deep");
 }
 
 int capture(loopspec_ctx* c, cudaGraphExec_t* out, bool vanilla) {
