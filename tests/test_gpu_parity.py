@@ -296,12 +296,25 @@ def test_depths_from_the_closed_form_are_used_when_none_are_given():
     ctx.close()
 
 
+@pytest.mark.parametrize("name", ["tiny_gqa", "tiny_gqa_f32"])
 @pytest.mark.parametrize("T", [0.0, 1.0])
-def test_context_beyond_2560_uses_runs_of_attention_chunks(T):
+def test_grouped_query_attention(name, T):
+    """Four query heads per KV head (the Raven-style head layout), head sizes 64 and 128, bf16 and fp32 weights; a
+    context of several attention chunks."""
+    ref = U.oracle_run(name, 150, 32, 1, 2, T=T, seed=6)
+    ctx = U.make_ctx(name, 1, 2, T=T, seed=6, max_ctx=200, max_prefill_rows=64)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(32)
+    U.assert_same_run(ctx, ref, 32)
+    ctx.close()
+
+
+@pytest.mark.parametrize("name,T", [("tiny_bf16", 0.0), ("tiny_bf16", 1.0), ("tiny_gqa", 1.0), ("tiny_gqa_f32", 0.0)])
+def test_context_beyond_2560_uses_runs_of_attention_chunks(name, T):
     """A 2700-token prompt: more than 40 chunks per row, so attention work items are runs of several chunks folded with
     the running-softmax rescaling (prefill positions beyond 2560 and every decode row)."""
-    ref = U.oracle_run("tiny_bf16", 2700, 16, 1, 2, T=T, seed=3)
-    ctx = U.make_ctx("tiny_bf16", 1, 2, T=T, seed=3, max_ctx=2740, max_prefill_rows=64)
+    ref = U.oracle_run(name, 2700, 16, 1, 2, T=T, seed=3)
+    ctx = U.make_ctx(name, 1, 2, T=T, seed=3, max_ctx=2740, max_prefill_rows=64)
     assert ctx.prefill(ref["prompt"]) == ref["first"]
     ctx.decode(16)
     U.assert_same_run(ctx, ref, 16)
