@@ -19,6 +19,7 @@ namespace cg = cooperative_groups;
 
 constexpr int SEL_THREADS = 512;
 constexpr int SEL_CS = 8;  // CTAs per reading-out row
+constexpr int SEL_NV = 7;  // values reduced together in the nucleus search (3 bits of the cut per pass)
 enum { PUR_DRAFT1 = 1, PUR_DRAFT2 = 2, PUR_ACCEPT1 = 3, PUR_ACCEPT2 = 4, PUR_RESAMPLE = 5, PUR_VANILLA = 6 };
 
 struct SelectParams {
@@ -106,6 +107,8 @@ struct ClusterRed {
   float* part_f;  // [2][SEL_CS]
   int* part_i;    // [2][SEL_CS]
   ArgMax* part_a; // [2][SEL_CS]
+  float* sh_n;    // [SEL_THREADS / 32][SEL_NV]: several values reduced at once (ints are passed as bit patterns)
+  float* part_n;  // [2][SEL_CS][SEL_NV]
 
   template <typename T>
   __device__ __forceinline__ void publish(T* part, T v) {
@@ -152,6 +155,54 @@ struct ClusterRed {
     for (int q = 0; q < n_ranks; ++q) r += part_i[phase * SEL_CS + q];
     phase ^= 1;
     return r;
+  }
+  // N <= SEL_NV sums at once, with one exchange: v[i] becomes the cluster-wide sum (floats or, with INT, integers)
+  template <int N, bool INT>
+  __device__ __forceinline__ void sum_n(float (&v)[N]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      if (INT) {
+        int x = __float_as_int(v[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        v[i] = __int_as_float(x);
+      } else {
+        v[i] = warp_sum(v[i]);
+      }
+    }
+    __syncthreads();
+    if (lane == 0)
+#pragma unroll
+      for (int i = 0; i < N; ++i) sh_n[warp * SEL_NV + i] = v[i];
+    __syncthreads();
+    if ((int)threadIdx.x < N) {  // thread i folds value i over the warps (in order) and hands it to every CTA
+      const int i = threadIdx.x;
+      float r;
+      if (INT) {
+        int x = 0;
+        for (int w = 0; w < SEL_THREADS / 32; ++w) x += __float_as_int(sh_n[w * SEL_NV + i]);
+        r = __int_as_float(x);
+      } else {
+        r = 0.f;
+        for (int w = 0; w < SEL_THREADS / 32; ++w) r += sh_n[w * SEL_NV + i];
+      }
+      for (int q = 0; q < n_ranks; ++q) *cluster.map_shared_rank(part_n + (phase * SEL_CS + rank) * SEL_NV + i, q) = r;
+    }
+    cluster.sync();
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      if (INT) {
+        int x = 0;
+        for (int q = 0; q < n_ranks; ++q) x += __float_as_int(part_n[(phase * SEL_CS + q) * SEL_NV + i]);
+        v[i] = __int_as_float(x);
+      } else {
+        float r = 0.f;
+        for (int q = 0; q < n_ranks; ++q) r += part_n[(phase * SEL_CS + q) * SEL_NV + i];
+        v[i] = r;
+      }
+    }
+    phase ^= 1;
   }
   __device__ __forceinline__ ArgMax block_argmax(ArgMax a) {  // this CTA only
 #pragma unroll
@@ -210,9 +261,21 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, int v_lo, int v_hi, f
   };
   if (top_k > 0 && top_k < V) {
     unsigned c = 0;  // largest c with at least top_k values >= c: the value of the top_k-th ranked token
-    for (int bit = 29; bit >= 0; --bit) {
-      const unsigned cand = c | (1u << bit);
-      if (count_if([&](unsigned eb, int) { return eb >= cand; }) >= top_k) c = cand;
+    for (int shift = 27; shift >= 0; shift -= 3) {  // three bits per pass: the seven candidates c | k << shift at once
+      float cnt[SEL_NV];
+#pragma unroll
+      for (int k = 0; k < SEL_NV; ++k) cnt[k] = __int_as_float(0);
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) {
+        const unsigned eb = __float_as_uint(e_sm[v - v_lo]);
+#pragma unroll
+        for (int k = 0; k < SEL_NV; ++k) cnt[k] = __int_as_float(__float_as_int(cnt[k]) + (eb >= (c | ((unsigned)(k + 1) << shift)) ? 1 : 0));
+      }
+      R.template sum_n<SEL_NV, true>(cnt);
+      unsigned best = 0;
+#pragma unroll
+      for (int k = 0; k < SEL_NV; ++k)
+        if (__float_as_int(cnt[k]) >= top_k) best = k + 1;  // the predicate is monotone in k
+      c |= best << shift;
     }
     const int need = top_k - count_if([&](unsigned eb, int) { return eb > c; });  // how many of the equal values stay
     int lo = 0, hi = V - 1;
@@ -228,9 +291,23 @@ __device__ __noinline__ void build_nucleus(Dist& d, int V, int v_lo, int v_hi, f
     const Dist dk = d;  // the top-k set
     const float target = top_p * mass_if([&](unsigned eb, int v) { return dk.kept(eb, v); });
     unsigned c = 0;     // largest c such that the kept values >= c carry at least the target mass
-    for (int bit = 29; bit >= 0; --bit) {
-      const unsigned cand = c | (1u << bit);
-      if (mass_if([&](unsigned eb, int v) { return dk.kept(eb, v) && eb >= cand; }) >= target) c = cand;
+    for (int shift = 27; shift >= 0; shift -= 3) {
+      float mass[SEL_NV];
+#pragma unroll
+      for (int k = 0; k < SEL_NV; ++k) mass[k] = 0.f;
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) {
+        const float e = e_sm[v - v_lo];
+        const unsigned eb = __float_as_uint(e);
+        const bool in_k = dk.kept(eb, v);
+#pragma unroll
+        for (int k = 0; k < SEL_NV; ++k) mass[k] += (in_k && eb >= (c | ((unsigned)(k + 1) << shift))) ? e : 0.f;
+      }
+      R.template sum_n<SEL_NV, false>(mass);
+      unsigned best = 0;
+#pragma unroll
+      for (int k = 0; k < SEL_NV; ++k)
+        if (mass[k] >= target) best = k + 1;
+      c |= best << shift;
     }
     if (c < dk.ecut) c = dk.ecut;
     const float m_gt = mass_if([&](unsigned eb, int v) { return dk.kept(eb, v) && eb > c; });
@@ -267,8 +344,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   __shared__ float part_f[2 * SEL_CS];
   __shared__ int part_i[2 * SEL_CS];
   __shared__ ArgMax part_a[2 * SEL_CS];
+  __shared__ float sh_n[(SEL_THREADS / 32) * SEL_NV];
+  __shared__ float part_n[2 * SEL_CS * SEL_NV];
   cg::cluster_group this_cl = cg::this_cluster();
-  ClusterRed R{this_cl, (int)this_cl.num_blocks(), (int)this_cl.block_rank(), 0, sh_f, sh_i, sh_am, part_f, part_i, part_a};
+  ClusterRed R{this_cl, (int)this_cl.num_blocks(), (int)this_cl.block_rank(), 0, sh_f, sh_i, sh_am, part_f, part_i, part_a, sh_n, part_n};
   const int col = (int)blockIdx.x / R.n_ranks;  // readout column = this cluster
   tune_mark(602, false);
   pdl_launch_dependents();
