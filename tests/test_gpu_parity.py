@@ -296,6 +296,21 @@ def test_depths_from_the_closed_form_are_used_when_none_are_given():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,T,d2", [("tiny_bf16", 0.0, 2), ("tiny_bf16", 1.0, 2), ("small_bf16", 1.0, 2), ("tiny_gqa", 0.0, 3)])
+def test_persistent_pass_kernel_matches_oracle(name, T, d2, monkeypatch):
+    """The opt-in persistent kernel (all layers of a pass in one launch, grid barriers between the stages) decodes the
+    same tokens as the oracle.  Its K split differs from the chain of kernels, so it is compared with the oracle, not
+    bit for bit with the default path."""
+    monkeypatch.setenv("LOOPSPEC_MEGA", "1")
+    ref = U.oracle_run(name, 40, 32, 1, d2, T=T, seed=7)
+    ctx = U.make_ctx(name, 1, d2, T=T, seed=7, max_ctx=100, max_prefill_rows=64)
+    assert ctx.launches_per_step() == 6          # preparation, pass, lm_head, selection, control, KV commit
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(32)
+    U.assert_same_run(ctx, ref, 32)
+    ctx.close()
+
+
 @pytest.mark.parametrize("name", ["tiny_gqa", "tiny_gqa_f32"])
 @pytest.mark.parametrize("T", [0.0, 1.0])
 def test_grouped_query_attention(name, T):
