@@ -137,6 +137,13 @@ int loopspec_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
 /* Baseline of Fig. 1(a): all R recurrences of a token before the next, from the same kernels. */
 int loopspec_vanilla_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
 
+/* Power-law envelope phi(r) = beta r^-alpha over a measured total-variation profile tv[r-1] = TV(p_r, p_R),
+ * r = 1..n (Sec. 4.1: "minimize the maximum ratio between phi(r) and the empirical TV over all depths"), read as:
+ * minimise max_r phi(r) / tv[r-1] subject to phi(r) >= tv[r-1] for every r, alpha > 0.  The pair feeds
+ * loopspec_pick_depths.  Host only.  tv: host array of n >= 2 positive values that decreases somewhere;
+ * EINVAL otherwise. */
+int loopspec_fit_envelope(const double* tv, int32_t n, double* alpha, double* beta);
+
 /* Theorem 2 / Eq. 8: real-valued optimum and the admissible integer pair (d1 | d2, d1 | R, d1 < d2 < R)
  * minimising the bound d1 + beta d1^-alpha d2 + 2 beta d2^-alpha R.  Host only; any output may be NULL. */
 int loopspec_pick_depths(float alpha, float beta, int32_t R, double* d1_star, double* d2_star, int32_t* d1,

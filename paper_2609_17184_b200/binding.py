@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libloopspec.so")
 
 EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loopspec_step", "loopspec_verify",
-           "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_max_branches",
+           "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_fit_envelope", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
            "loopspec_launches_per_step", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
            "loopspec_op_linear_static",
@@ -65,6 +65,7 @@ def _load():
     P, I, V = C.POINTER, C.c_int32, C.c_void_p
     lib.loopspec_workspace_bytes.restype = C.c_size_t
     lib.loopspec_workspace_bytes.argtypes = [P(Model), P(Sched)]
+    lib.loopspec_fit_envelope.argtypes = [P(C.c_double), I, P(C.c_double), P(C.c_double)]
     lib.loopspec_init.argtypes = [P(Model), P(Sched), P(Weights), V, C.c_size_t, V, P(V)]
     lib.loopspec_prefill.argtypes = [V, I, P(I), I, P(I)]
     lib.loopspec_step.argtypes = [V, P(I), P(I)]
@@ -103,6 +104,16 @@ def pick_depths(alpha, beta, R):
     if rc:
         raise LoopSpecError(rc)
     return a.value, b.value, x.value, y.value
+
+
+def fit_envelope(tv):
+    """(alpha, beta) of the power-law envelope over a measured TV profile tv[r-1] = TV(p_r, p_R)."""
+    arr = (C.c_double * len(tv))(*[float(x) for x in tv])
+    a, b = C.c_double(), C.c_double()
+    rc = lib.loopspec_fit_envelope(arr, len(tv), C.byref(a), C.byref(b))
+    if rc:
+        raise LoopSpecError(rc)
+    return a.value, b.value
 
 
 def max_branches(R, d1, d2):

@@ -668,6 +668,33 @@ int loopspec_pick_depths(float alpha, float beta, int32_t R, double* d1_star, do
   return LOOPSPEC_OK;
 }
 
+int loopspec_fit_envelope(const double* tv, int32_t n, double* alpha, double* beta) {
+  if (!tv || n < 2 || !alpha || !beta) return LOOPSPEC_EINVAL;
+  for (int i = 0; i < n; ++i)
+    if (!(tv[i] > 0)) return LOOPSPEC_EINVAL;
+  // With u_r(a) = log tv_r + a log r the constraint is log beta >= max_r u_r(a) and, at the tightest beta, the worst
+  // log-ratio is max_r u_r(a) - min_r u_r(a): convex and piecewise linear in a, so its minimum over a > 0 is at a slope
+  // where two of the lines u_i, u_j cross.  Every such slope is tried.
+  double best_gap = 0, best_a = 0, best_logb = 0;
+  bool have = false;
+  for (int i = 0; i < n; ++i)
+    for (int j = i + 1; j < n; ++j) {
+      const double a = -(std::log(tv[j]) - std::log(tv[i])) / (std::log((double)(j + 1)) - std::log((double)(i + 1)));
+      if (!(a > 0)) continue;
+      double hi = -1e300, lo = 1e300;
+      for (int r = 0; r < n; ++r) {
+        const double u = std::log(tv[r]) + a * std::log((double)(r + 1));
+        hi = std::max(hi, u), lo = std::min(lo, u);
+      }
+      if (!have || hi - lo < best_gap - 1e-15 || (std::fabs(hi - lo - best_gap) <= 1e-15 && a < best_a)) {
+        best_gap = hi - lo, best_a = a, best_logb = hi, have = true;
+      }
+    }
+  if (!have) return LOOPSPEC_EINVAL;  // the profile never decreases: no positive exponent fits
+  *alpha = best_a, *beta = std::exp(best_logb);
+  return LOOPSPEC_OK;
+}
+
 int32_t loopspec_max_branches(int32_t R, int32_t d1, int32_t d2) {
   if (d1 < 1 || R < 2 || d1 >= R || R % d1 || (d2 && (d2 <= d1 || d2 >= R || d2 % d1))) return 0;
   return max_branches(R, d1, d2);

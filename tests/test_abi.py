@@ -3,6 +3,7 @@ and its host-only entry points agree with the oracle."""
 import os
 import re
 
+import numpy as np
 import pytest
 
 import paper_2609_17184_b200 as ls
@@ -33,6 +34,28 @@ def test_pick_depths_matches_oracle():
         assert (d1, d2) == dp.snap_depths(float(__import__("numpy").float32(a)), float(__import__("numpy").float32(b)), R)
     with pytest.raises(ls.LoopSpecError):
         ls.pick_depths(-1.0, 0.2, 32)
+
+
+def test_fit_envelope_matches_oracle_and_recovers_exact_power_laws():
+    r = np.arange(1, 16, dtype=np.float64)
+    a, b = ls.fit_envelope(0.2 * r ** -1.1)          # an exact power law is its own envelope
+    assert abs(a - 1.1) < 1e-9 and abs(b - 0.2) < 1e-9
+    rng = np.random.default_rng(4)
+    for _ in range(40):
+        n = int(rng.integers(3, 33))
+        rr = np.arange(1, n + 1, dtype=np.float64)
+        tv = rng.uniform(0.05, 0.4) * rr ** -rng.uniform(0.3, 2.0) * np.exp(rng.normal(0, 0.15, n))
+        a, b = ls.fit_envelope(tv)
+        ao, bo = dp.fit_envelope(tv)
+        assert abs(a - ao) < 1e-9 * max(1, abs(ao)) and abs(b - bo) < 1e-9 * max(1, abs(bo))
+        phi = b * rr ** -a
+        assert (phi >= tv * (1 - 1e-12)).all() and a > 0       # an envelope: never below the measured profile
+    with pytest.raises(ls.LoopSpecError):
+        ls.fit_envelope([0.1, 0.2, 0.3])                       # never decreases: no positive exponent
+    with pytest.raises(ls.LoopSpecError):
+        ls.fit_envelope([0.1])
+    with pytest.raises(ls.LoopSpecError):
+        ls.fit_envelope([0.2, 0.0, 0.1])
 
 
 def test_max_branches_matches_oracle_and_paper():
