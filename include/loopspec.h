@@ -61,7 +61,10 @@ typedef struct {
  * top_k, top_p: the optional filters of the post-layers C (Sec. 3.1), applied at EVERY readout depth when
  * temperature > 0: tokens are ranked by decreasing probability (ties: lower index first); top_k > 0 keeps the first
  * top_k and renormalises; 0 < top_p < 1 then keeps the shortest prefix of the ranking whose mass reaches top_p and
- * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off. */
+ * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off.
+ * measure_tv = 1 (sampling only): every verification also records TV(p_d1, p_R) and, where a second-proposal record
+ * exists, TV(p_d2, p_R) of the readouts involved (Sec. 4.1's empirical profile; see loopspec_stats and
+ * loopspec_fit_envelope).  With the gate on, the depth-d2 readout exists only where the gate opened. */
 typedef struct {
   int32_t d1, d2;
   float alpha, beta;
@@ -72,6 +75,7 @@ typedef struct {
   int32_t max_prefill_rows;
   int32_t top_k;
   float top_p;
+  int32_t measure_tv;
 } loopspec_sched;
 
 /* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:
@@ -92,11 +96,15 @@ typedef struct {
   int32_t seq, n_committed, token, source, accepted1, accepted2, gate_open, step;
 } loopspec_commit;
 
-/* Counters of Sec. 5 (gamma), App. C (gate openings, effective batch size) and App. D (commit sources). */
+/* Counters of Sec. 5 (gamma), App. C (gate openings, effective batch size) and App. D (commit sources).
+ * tv_d1 / tv_d2: mean total-variation distance between the depth-d1 / depth-d2 readout and the target over the
+ * tv_n1 / tv_n2 verifications that had one (0 unless the scheduler was created with measure_tv). */
 typedef struct {
   int64_t steps, n_decode, n_accept1, n_accept2, n_restart, gate_evals, gate_opens, rows_total, rows_max,
       readout_rows_total;
   double gamma;
+  double tv_d1, tv_d2;
+  int64_t tv_n1, tv_n2;
 } loopspec_stats;
 
 /* Bytes of device workspace loopspec_init needs for this model and scheduler (0 on invalid input).  For bf16

@@ -54,6 +54,7 @@ class Decoder:
         self.K = self.V = None     # [R+1][layer] arrays [max_ctx, nkv, d]; index by recurrence 1..R
         self.log = []              # decision log
         self.rows_per_step = []
+        self.tv_log = []           # per verification (sampling): TV(p_d1, p_R) and TV(p_d2, p_R) or None (Sec. 4.1)
 
     # ---- committed, depth-indexed KV ---------------------------------------------------------
     def _alloc(self, n_total):
@@ -170,6 +171,10 @@ class Decoder:
             self.log.append(dict(kind="verify", pos=pos, source=3, token=top, margin=margin))
             return top, None, 3
         rho = self.probs(p_logits)
+        # the empirical profile of Sec. 4.1: total variation between the early readouts and the target
+        tv1 = 0.5 * float(np.abs(b.records[0].q - rho).sum())
+        tv2 = 0.5 * float(np.abs(self.probs(b.q2_logits) - rho).sum()) if len(b.records) > 1 else None
+        self.tv_log.append((tv1, tv2))
         for j, rec in enumerate(b.records):
             U = float(sp.uniform(self.seed, self.seq, pos, sp.ACCEPT1 + j))
             a = sp.accept_prob(rho, rec.q, rec.token)

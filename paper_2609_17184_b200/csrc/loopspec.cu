@@ -73,7 +73,7 @@ size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, flt, sel_flt, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, flt, sel_flt, tv, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -214,6 +214,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sel_flt = take((size_t)MAX_ROWS * sizeof(float4));
   L.seqs = take((size_t)5 * MAX_ROWS * 4);
   L.ctr = take(sizeof(Counters));
+  L.tv = take((size_t)MAX_ROWS * 4 * sizeof(double));
   L.tab_dec = take(sizeof(RowTable));
   L.tab_pf = take(sizeof(RowTable));
   L.tab_van = take(sizeof(RowTable) * m->R);
@@ -538,6 +539,7 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   sp.argpart = c->at<float2>(c->L.argpart), sp.n_rb = c->plan[G_LM].n_rb;
   sp.top_k = c->filters ? c->s.top_k : 0, sp.top_p = c->filters ? c->s.top_p : 1.0f, sp.sel_flt = c->at<float4>(c->L.sel_flt);
   sp.staged = c->sel_staged;
+  sp.tv_acc = (c->s.measure_tv && c->s.temperature > 0.f) ? c->at<double>(c->L.tv) : nullptr;
   return launch_k(select_kernel, dim3(c->d.max_rows * SEL_CS), dim3(SEL_THREADS), c->sel_smem, c->stream, sp, c->use_pdl, SEL_CS);
 }
 
@@ -977,6 +979,7 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
   CU(c, cudaGetLastError());
   // statistics and traces restart with the sequence set
   CU(c, cudaMemsetAsync(c->ws + c->L.ctr, 0, sizeof(Counters), c->stream));
+  CU(c, cudaMemsetAsync(c->ws + c->L.tv, 0, (size_t)MAX_ROWS * 4 * sizeof(double), c->stream));
   CU(c, cudaMemsetAsync(c->ws + c->L.trace_n, 0, 4, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   c->prefilled[seq] = 1;
@@ -1127,6 +1130,12 @@ int loopspec_get_stats(loopspec_ctx* c, loopspec_stats* out) {
   out->rows_total = k.rows_total, out->rows_max = k.rows_max, out->readout_rows_total = k.readout_rows_total;
   double den = (double)k.n_accept1 * c->d.d1 + (double)k.n_accept2 * c->d.d2 + (double)k.n_restart * c->m.R;
   out->gamma = den > 0 ? (double)k.n_decode * c->m.R / den : 0.0;  // Sec. 5, definition of gamma
+  double tv[MAX_ROWS * 4];
+  CU(c, cudaMemcpy(tv, c->ws + c->L.tv, sizeof tv, cudaMemcpyDeviceToHost));
+  double s1 = 0, n1 = 0, s2 = 0, n2 = 0;
+  for (int s = 0; s < c->d.S; ++s) s1 += tv[4 * s], n1 += tv[4 * s + 1], s2 += tv[4 * s + 2], n2 += tv[4 * s + 3];
+  out->tv_d1 = n1 > 0 ? s1 / n1 : 0.0, out->tv_d2 = n2 > 0 ? s2 / n2 : 0.0;
+  out->tv_n1 = (int64_t)n1, out->tv_n2 = (int64_t)n2;
   return LOOPSPEC_OK;
 }
 

@@ -43,6 +43,7 @@ struct SelectParams {
   int top_k;
   float top_p;
   int staged;           // 1: dynamic shared memory holds 3 row slices (+1 when filtering) of ceil(V/4/8)*4 floats each
+  double* tv_acc;       // [seq][4]: sum and count of TV(p_d1, p_R), sum and count of TV(p_d2, p_R); null: not measured
   float4* sel_flt;      // per row: the nucleus of its readout (max of z/T, kept mass, cut value bits, cut index)
 };
 
@@ -513,6 +514,27 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
   auto pp = [&](int v, bool any = false) { return any ? dp.prob(v, T) : dp.probs(v, T); };
   auto q1 = [&](int v, bool any = false) { return any ? d1.prob(v, T) : d1.probs(v, T); };
   auto q2t = [&](int v, bool any = false) { return any ? d2.prob(v, T) : d2.probs(v, T); };
+  // sum_v [p - q1]_+ : the normaliser of rho1 = p (-) q1 (Eq. 2) and, both being normalised, TV(q1, p)
+  auto mass_above_q1 = [&]() {
+    float a = 0.f;
+    for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) a += fmaxf(pp(v) - q1(v), 0.f);
+    return R.sum(a);
+  };
+  float Z1 = 0.f;
+  if (p.tv_acc) {  // the empirical TV profile of Sec. 4.1, recorded at every verification
+    Z1 = mass_above_q1();
+    float tv2 = 0.f;
+    if (has2) {
+      float a = 0.f;
+      for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) a += fmaxf(pp(v) - q2t(v), 0.f);
+      tv2 = R.sum(a);
+    }
+    if (writer) {  // one verification per sequence and pass: no other writer
+      double* acc = p.tv_acc + 4 * seq;
+      acc[0] += (double)Z1, acc[1] += 1.0;
+      if (has2) acc[2] += (double)tv2, acc[3] += 1.0;
+    }
+  }
   // first proposal: accept with probability min{1, p(x1)/q1(x1)} (Eq. 3)
   const float U1 = uniform(PUR_ACCEPT1);
   if (U1 < fminf(1.0f, pp(x1, true) / q1(x1, true))) {
@@ -520,9 +542,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     return;
   }
   // rho1 = p (-) q1 (Eq. 2); if the positive part has no mass rho1 = p
+  if (!p.tv_acc) Z1 = mass_above_q1();
   float s = 0.f;
-  for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(pp(v) - q1(v), 0.f);
-  const float Z1 = R.sum(s);
   auto rho1 = [&](int v, bool any = false) { return Z1 > 0.f ? fmaxf(pp(v, any) - q1(v, any), 0.f) / Z1 : pp(v, any); };
   if (!has2) {
     int tok = race([&](int v) { float w = rho1(v); return w > 0.f ? logf(w) : -INFINITY; }, PUR_RESAMPLE);

@@ -171,6 +171,42 @@ def test_parity_holds_across_seeds(name, n_prompt, n_decode, d1, d2, T, top_k, t
         ctx.close()
 
 
+@pytest.mark.parametrize("name,gate,top_p", [("tiny_bf16", True, 1.0), ("tiny_bf16", False, 1.0), ("small_bf16", False, 0.8)])
+def test_measured_tv_profile_matches_oracle_and_feeds_the_depth_picker(name, gate, top_p):
+    """measure_tv records TV(p_d1, p_R) and TV(p_d2, p_R) at every verification (Sec. 4.1); the means equal the
+    oracle's, and the fitted envelope gives an admissible depth pair."""
+    import paper_2609_17184_b200 as ls
+    R = W.CONFIGS[name].R
+    prof = {}
+    for d2 in (2, 3):
+        ref = U.oracle_run(name, 24, 40, 1, d2, T=1.0, seed=3, gate=gate, top_p=top_p)
+        ctx = U.make_ctx(name, 1, d2, T=1.0, seed=3, gate=gate, max_ctx=80, top_p=top_p, measure_tv=True)
+        assert ctx.prefill(ref["prompt"]) == ref["first"]
+        assert ctx.decode(40)[0].tolist() == ref["tokens"]      # measuring does not change the stream
+        st = ctx.stats()
+        tvs = ref["dec"].tv_log
+        t1 = [a for a, _ in tvs]
+        t2 = [b for _, b in tvs if b is not None]
+        assert st["tv_n1"] == len(t1) == 40 and st["tv_n2"] == len(t2)
+        # fp32 against fp64 probabilities; with a nucleus, which of the near-equal tokens sit at its edge may differ
+        tol = 2e-5 if top_p >= 1.0 else 2e-4
+        assert abs(st["tv_d1"] - np.mean(t1)) < tol
+        if t2:
+            assert abs(st["tv_d2"] - np.mean(t2)) < tol
+            prof[d2] = st["tv_d2"]
+        prof[1] = st["tv_d1"]
+        ctx.close()
+    assert sorted(prof) == [1, 2, 3]
+    alpha, beta = ls.fit_envelope([prof[r] for r in range(1, R)])
+    d1s, d2s, d1, d2 = ls.pick_depths(alpha, beta, R)
+    assert alpha > 0 and beta > 0 and 1 <= d1 < d2 < R and d2 % d1 == 0 and R % d1 == 0
+    # not measuring leaves the fields at zero
+    ctx = U.make_ctx(name, 1, 2, T=1.0, seed=3, max_ctx=80)
+    ctx.prefill(ref["prompt"]); ctx.decode(8)
+    assert ctx.stats()["tv_n1"] == 0 and ctx.stats()["tv_d1"] == 0.0
+    ctx.close()
+
+
 def test_filters_off_values_and_unsupported_vocab():
     """top_k = 0 with top_p = 0 or 1 is the plain softmax: bit-identical to a context built without the fields."""
     ref = U.oracle_run("tiny_bf16", 16, 24, 1, 2, T=1.0, seed=2)
