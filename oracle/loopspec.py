@@ -172,9 +172,12 @@ class Decoder:
             return top, None, 3
         rho = self.probs(p_logits)
         # the empirical profile of Sec. 4.1: total variation between the early readouts and the target
-        tv1 = 0.5 * float(np.abs(b.records[0].q - rho).sum())
-        tv2 = 0.5 * float(np.abs(self.probs(b.q2_logits) - rho).sum()) if len(b.records) > 1 else None
-        self.tv_log.append((tv1, tv2))
+        if b.records:
+            tv1 = 0.5 * float(np.abs(b.records[0].q - rho).sum())
+            tv2 = None
+            if len(b.records) > 1 and b.q2_logits is not None:
+                tv2 = 0.5 * float(np.abs(self.probs(b.q2_logits) - rho).sum())
+            self.tv_log.append((tv1, tv2))
         for j, rec in enumerate(b.records):
             U = float(sp.uniform(self.seed, self.seq, pos, sp.ACCEPT1 + j))
             a = sp.accept_prob(rho, rec.q, rec.token)
