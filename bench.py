@@ -148,6 +148,29 @@ def run_profile_pass(args):
     ctx.close()
 
 
+def select_depths(ls, shape, weights, prompt, wl, n_tokens=96):
+    """Depth pair from the closed form of Theorem 2 on a measured TV profile (Sec. 4.1, Sec. 5): short ungated runs at
+    (1, r), r = 2..R-1, record TV(p_1, p_R) and TV(p_r, p_R) on the device; the envelope fit and the snapping to an
+    admissible pair are the library's host functions."""
+    R = shape.R
+    tv = {}
+    for r in range(2, R):
+        ctx = ls.LoopSpec(shape, weights, d1=1, d2=r, temperature=wl.temperature, seed=wl.sample_seed, gate=False, max_seqs=1,
+                          max_ctx=len(prompt) + n_tokens + 16, max_prefill_rows=64, top_k=wl.top_k, top_p=wl.top_p,
+                          measure_tv=True)
+        ctx.prefill(prompt)
+        ctx.decode(n_tokens)
+        st = ctx.stats()
+        tv[1], tv[r] = st["tv_d1"], st["tv_d2"]
+        ctx.close()
+    profile = [tv[r] for r in range(1, R)]
+    alpha, beta = ls.fit_envelope(profile)
+    d1s, d2s, d1, d2 = ls.pick_depths(alpha, beta, R)
+    return d1, d2, {"tv_profile": [round(x, 5) for x in profile], "alpha": round(alpha, 4), "beta": round(beta, 4),
+                    "d1_star": round(d1s, 3), "d2_star": round(d2s, 3), "d1": d1, "d2": d2,
+                    "calibration_tokens_per_run": n_tokens}
+
+
 def run_ours(args):
     import torch
     import paper_2609_17184_b200 as ls
@@ -170,7 +193,10 @@ def run_ours(args):
     del wnp
     t_setup = time.time() - t0
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed)
-    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
+    d1, d2, depth_sel = wl.d1, wl.d2, None
+    if args.closed_form and wl.temperature > 0:
+        d1, d2, depth_sel = select_depths(ls, shape, weights, prompt, wl)
+    ctx = ls.LoopSpec(shape, weights, d1=d1, d2=d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
                       max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64, top_k=wl.top_k, top_p=wl.top_p)
     stream = ctx.stream
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -238,7 +264,7 @@ def run_ours(args):
         "metric": "decode_tok_per_s", "value": round(value, 2), "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"{wl.name}: prompt {n_prompt}, decode {n_decode}, T={wl.temperature}{f', top-p {wl.top_p}' if wl.top_p < 1 else ''}{f', top-k {wl.top_k}' if wl.top_k else ''}, (d1,d2)=({wl.d1},{wl.d2}), "
+        "config": {"workload": f"{wl.name}: prompt {n_prompt}, decode {n_decode}, T={wl.temperature}{f', top-p {wl.top_p}' if wl.top_p < 1 else ''}{f', top-k {wl.top_k}' if wl.top_k else ''}, (d1,d2)=({d1},{d2}), "
                                f"gate={'on' if wl.gate else 'off'}, batch 1, R={shape.R}, L={shape.n_recurrent}",
                    "l2": "every pass streams the 2.5 GB shared stack, far larger than the 126 MB L2; no flush needed",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
@@ -259,6 +285,7 @@ def run_ours(args):
                     "hbm_GBps": round(van_gbs, 1), "frac": round(van_gbs / peak, 4)},
         "speedup_vs_vanilla": round(statistics.mean(van_ms) / statistics.mean(dec_ms), 4),
         "greedy_equals_vanilla": lossless,
+        "depth_selection": depth_sel,
         "acceptance": {"gamma": round(stats["gamma"], 4), "first": round(stats["n_accept1"] / n, 4),
                        "second": round(stats["n_accept2"] / n, 4), "restart": round(stats["n_restart"] / n, 4),
                        "gate_open_rate": round(stats["gate_opens"] / max(stats["gate_evals"], 1), 4),
@@ -384,6 +411,8 @@ def main():
     ap.add_argument("--decode-len", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--calibrated", action="store_true", help="also run the acceptance-calibrated variant")
+    ap.add_argument("--closed-form", action="store_true",
+                    help="sampling workloads: pick (d1, d2) from Theorem 2 on a TV profile measured on the device first")
     ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")
     ap.add_argument("--profile-pass", type=int, default=0, help="prefill, decode this many tokens, exit (for profilers)")
     ap.add_argument("--rows", type=int, default=4)
