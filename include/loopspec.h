@@ -64,7 +64,11 @@ typedef struct {
  * renormalises.  top_k = 0 and top_p = 0 (or >= 1) switch the filters off.
  * measure_tv = 1 (sampling only): every verification also records TV(p_d1, p_R) and, where a second-proposal record
  * exists, TV(p_d2, p_R) of the readouts involved (Sec. 4.1's empirical profile; see loopspec_stats and
- * loopspec_fit_envelope).  With the gate on, the depth-d2 readout exists only where the gate opened. */
+ * loopspec_fit_envelope).  With the gate on, the depth-d2 readout exists only where the gate opened.
+ * mask_first = 1: the variant of the paper's second-proposal ablation (Sec. 5): the first candidate is removed from the
+ * second proposal's distribution (the residual one if it has mass elsewhere, else p_{d2}) and the rest renormalised, so
+ * the two candidates always differ; a branch whose p_{d2} has all its mass on the first candidate gets no second
+ * proposal.  Under greedy decoding the second candidate is then the best token other than the first. */
 typedef struct {
   int32_t d1, d2;
   float alpha, beta;
@@ -76,6 +80,7 @@ typedef struct {
   int32_t top_k;
   float top_p;
   int32_t measure_tv;
+  int32_t mask_first;
 } loopspec_sched;
 
 /* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:

@@ -190,7 +190,7 @@ class Decoder:
         self.log.append(dict(kind="resample", pos=pos, token=tok, margin=margin))
         return tok, None, 3
 
-    def loopspec(self, n_tokens, d1, d2=0, gate=True, residual_q2=True, keep_logits=False):
+    def loopspec(self, n_tokens, d1, d2=0, gate=True, residual_q2=True, keep_logits=False, mask_first=False):
         """Commit exactly n_tokens more tokens.  d2 = 0 disables the second proposal.
 
         Returns the committed tokens; `self.commits` lists, per token, its source and flags;
@@ -250,6 +250,9 @@ class Decoder:
                             # residual of two one-hot distributions: the deeper argmax; without the
                             # gate the two may coincide and the residual falls back to q2~ itself
                             x2 = top
+                            if mask_first and top == x1:   # second-proposal ablation (Sec. 5): the first candidate is masked out
+                                x2, margin = self._argmax(np.where(np.arange(len(z2)) == x1, -np.inf, z2))
+                                self.log.append(dict(kind="draft2", pos=pos, token=x2, margin=margin))
                             self.stats["gate_opens"] += 1
                             c2 = self._spawn(b, x2, pos)
                             b.records.append(Record(x2, None, c2))
@@ -260,8 +263,13 @@ class Decoder:
                         with np.errstate(divide="ignore"):   # a filtered q2~ may give the candidate no mass
                             gm = abs(np.log(q2t[x1]) - np.log(q1[x1]))
                         self.log.append(dict(kind="gate", pos=pos, open=is_open, margin=gm))
-                        if is_open:
+                        if is_open and mask_first:
+                            # second-proposal ablation (Sec. 5): the first candidate is masked out of the proposal
+                            q2 = sp.masked_second_proposal(q2t, q1, x1, residual_q2)
+                            is_open = q2 is not None      # q2~ puts all its mass on the first candidate: no proposal
+                        elif is_open:
                             q2 = sp.residual(q2t, q1) if residual_q2 else q2t
+                        if is_open:
                             x2, margin = self._draw(q2, pos, sp.DRAFT2)
                             self.log.append(dict(kind="draft2", pos=pos, token=x2, margin=margin))
                             self.stats["gate_opens"] += 1

@@ -95,6 +95,19 @@ def residual(mu, nu):
     return np.where(s > 0, d / np.where(s > 0, s, 1.0), mu)
 
 
+def masked_second_proposal(q2t, q1, x1, residual_q2=True):
+    """Second proposal with the first candidate x1 masked out (the variant of the second-proposal ablation, Sec. 5):
+    x1's mass is removed from the residual proposal norm([q2~ - q1]_+) if that leaves mass elsewhere (or if
+    residual_q2 is off, from q2~ directly), else from q2~, and the rest renormalised.  None when q2~ has all its mass
+    on x1: there is nothing else to propose."""
+    for base in ([positive_part_diff(q2t, q1)] if residual_q2 else []) + [np.asarray(q2t, dtype=np.float64)]:
+        base = base.copy()
+        base[x1] = 0.0
+        if base.sum() > 0:
+            return base / base.sum()
+    return None
+
+
 def accept_prob(rho, q, x):
     """min{1, rho(x)/q(x)} of Eq. 3 for a candidate x drawn from q (so q(x) > 0)."""
     return min(1.0, rho[x] / q[x])

@@ -36,7 +36,7 @@ class Sched(C.Structure):
     _fields_ = [("d1", C.c_int32), ("d2", C.c_int32), ("alpha", C.c_float), ("beta", C.c_float), ("gate", C.c_int32),
                 ("residual_q2", C.c_int32), ("temperature", C.c_float), ("seed", C.c_uint64), ("max_seqs", C.c_int32),
                 ("max_ctx", C.c_int32), ("max_prefill_rows", C.c_int32), ("top_k", C.c_int32), ("top_p", C.c_float),
-                ("measure_tv", C.c_int32)]
+                ("measure_tv", C.c_int32), ("mask_first", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -172,7 +172,7 @@ class LoopSpec:
     """One decoding context (see include/loopspec.h for the semantics of every call)."""
 
     def __init__(self, shape, weights, d1=1, d2=0, temperature=0.0, seed=0, gate=True, residual_q2=True, max_seqs=1,
-                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None, top_k=0, top_p=1.0, measure_tv=False):
+                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None, top_k=0, top_p=1.0, measure_tv=False, mask_first=False):
         import torch
         self._torch = torch
         self.shape = shape
@@ -185,7 +185,7 @@ class LoopSpec:
                            shape.n_prelude, shape.n_recurrent, shape.n_coda, shape.R,
                            1 if shape.weight_dtype == "bf16" else 0, 1 if shape.tied else 0, shape.rms_eps, shape.rope_theta)
         self.sched = Sched(d1, d2, alpha, beta, int(gate), int(residual_q2), temperature, seed, max_seqs, max_ctx,
-                           max_prefill_rows, int(top_k), float(top_p), int(measure_tv))
+                           max_prefill_rows, int(top_k), float(top_p), int(measure_tv), int(mask_first))
         nbytes = lib.loopspec_workspace_bytes(C.byref(self.model), C.byref(self.sched))
         if nbytes == 0:
             # let init report the precise status

@@ -72,6 +72,8 @@ GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1) {
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
+static_assert(SEL_ARG_BLOCK == RB_ROWS, "the selection reads one argmax partial per lm_head row block");
+
 struct Layout {  // byte offsets into the workspace
   size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, flt, sel_flt, tv, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
@@ -533,6 +535,7 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
   SelectParams sp;
   sp.tab = tab, sp.logits = c->at<float>(c->L.logits), sp.V = c->m.vocab, sp.NB = c->d.NB, sp.nodes = c->nodes();
   sp.temperature = c->s.temperature, sp.gate = c->s.gate, sp.residual_q2 = c->s.residual_q2, sp.seed = c->s.seed;
+  sp.mask_first = c->s.mask_first;
   sp.kinds_mask = kinds_mask;
   sp.sel_tok = c->at<int>(c->L.sel_tok), sp.sel_aux = c->at<int>(c->L.sel_aux);
   sp.sel_lse = c->at<float>(c->L.sel_lse), sp.sel_z2 = c->at<float>(c->L.sel_z2);

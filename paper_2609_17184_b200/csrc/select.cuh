@@ -20,6 +20,7 @@ namespace cg = cooperative_groups;
 constexpr int SEL_THREADS = 512;
 constexpr int SEL_CS = 8;  // CTAs per reading-out row
 constexpr int SEL_NV = 7;  // values reduced together in the nucleus search (3 bits of the cut per pass)
+constexpr int SEL_ARG_BLOCK = 128;  // vocabulary rows per argmax partial of the lm_head epilogue
 enum { PUR_DRAFT1 = 1, PUR_DRAFT2 = 2, PUR_ACCEPT1 = 3, PUR_ACCEPT2 = 4, PUR_RESAMPLE = 5, PUR_VANILLA = 6 };
 
 struct SelectParams {
@@ -29,6 +30,7 @@ struct SelectParams {
   NodeTable nodes;
   float temperature;
   int gate, residual_q2;
+  int mask_first;       // second-proposal ablation: the first candidate is removed from the second proposal
   unsigned long long seed;
   int kinds_mask;       // bit k set: handle readout kind k
   int* sel_tok;         // per row: drafted / committed token
@@ -469,28 +471,61 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     const int x1 = p.nodes.tok1[gn];
     if (T == 0.f) {
       int top = greedy(z);
-      if (writer) p.sel_tok[row] = top, p.sel_aux[row] = (top != x1) || !p.gate, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
+      const bool open = (top != x1) || !p.gate;
+      if (open && top == x1 && p.mask_first) {
+        // the best token other than the first candidate: the per-block maxima of the other blocks, and the logits of
+        // the candidate's own block one by one
+        ArgMax a = {-INFINITY, 0x7fffffff};
+        const int xb = x1 / SEL_ARG_BLOCK;
+        for (int b = tid; b < p.n_rb; b += SEL_THREADS)
+          if (b != xb) {
+            const float2 v = __ldcg(p.argpart + (size_t)col * p.n_rb + b);
+            a = better(a, ArgMax{v.x, __float_as_int(v.y)});
+          }
+        if (tid < SEL_ARG_BLOCK) {
+          const int v = xb * SEL_ARG_BLOCK + tid;
+          if (v < V && v != x1) a = better(a, ArgMax{__ldcg(z + v), v});
+        }
+        top = R.block_argmax(a).i;
+      }
+      if (writer) p.sel_tok[row] = top, p.sel_aux[row] = open, p.sel_lse[row] = 0.f, p.sel_z2[row] = 0.f;
       return;
     }
     const Dist d1 = stored(z1, 1, p.nodes.lse1[gn], p.nodes.flt1 + gn);
     const Dist d2 = fresh(z, 0);
     // Eq. 6; without filters the comparison is made on log-probabilities, as before
     const bool lower = filt ? (d2.prob(x1, T) < d1.prob(x1, T)) : (z[x1] / T - d2.lse < z1[x1] / T - d1.lse);
-    const bool open = lower || !p.gate;
+    bool open = lower || !p.gate;
+    const bool mask = p.mask_first != 0;
     int tok = 0;
+    // how the record's proposal is normalised: > 0: [q2~ - q1]_+ over this mass; < 0: q2~ over minus this mass
+    // (first candidate masked out); 0: q2~ as it is
     float Z2 = 0.f;
     if (open) {
       if (p.residual_q2) {
         float s = 0.f;
-        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS) s += fmaxf(d2.probs(v, T) - d1.probs(v, T), 0.f);
+        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS)
+          if (!(mask && v == x1)) s += fmaxf(d2.probs(v, T) - d1.probs(v, T), 0.f);
         Z2 = R.sum(s);
       }
-      if (Z2 > 0.f)
+      if (Z2 > 0.f) {
         tok = race([&](int v) {
-          float w = d2.probs(v, T) - d1.probs(v, T);
+          float w = (mask && v == x1) ? 0.f : d2.probs(v, T) - d1.probs(v, T);
           return w > 0.f ? logf(w) : -INFINITY; }, PUR_DRAFT2);
-      else
+      } else if (!mask) {
         tok = race([&](int v) { return d2.logw(v, T); }, PUR_DRAFT2);
+      } else {  // q2~ without the first candidate
+        float s = 0.f;
+        for (int v = v_lo + tid; v < v_hi; v += SEL_THREADS)
+          if (v != x1) s += d2.probs(v, T);
+        const float rest = R.sum(s);
+        if (rest > 0.f) {
+          Z2 = -rest;
+          tok = race([&](int v) { return v == x1 ? -INFINITY : d2.logw(v, T); }, PUR_DRAFT2);
+        } else {
+          open = false;  // all of q2~ sits on the first candidate: no second proposal
+        }
+      }
     }
     if (writer) {
       p.sel_tok[row] = tok, p.sel_aux[row] = open, p.sel_lse[row] = d2.lse, p.sel_z2[row] = Z2;
@@ -550,7 +585,12 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const __grid_consta
     if (writer) p.sel_tok[row] = tok, p.sel_aux[row] = 3;
     return;
   }
-  auto q2 = [&](int v, bool any = false) { return Z2 > 0.f ? fmaxf(q2t(v, any) - q1(v, any), 0.f) / Z2 : q2t(v, any); };
+  const bool mask = p.mask_first != 0;
+  auto q2 = [&](int v, bool any = false) {  // the second proposal as it was drafted (see the record's normaliser)
+    if (mask && v == x1) return 0.f;
+    if (Z2 > 0.f) return fmaxf(q2t(v, any) - q1(v, any), 0.f) / Z2;
+    return Z2 < 0.f ? q2t(v, any) / -Z2 : q2t(v, any);
+  };
   const float U2 = uniform(PUR_ACCEPT2);
   if (U2 < fminf(1.0f, rho1(x2, true) / q2(x2, true))) {
     if (writer) p.sel_tok[row] = x2, p.sel_aux[row] = 2;

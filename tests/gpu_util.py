@@ -20,7 +20,7 @@ def oracle_model(name, seed=0, gain_jitter=0.0):
 
 @functools.lru_cache(maxsize=None)
 def oracle_run(name, n_prompt, n_decode, d1, d2, T=0.0, seed=2, gate=True, residual_q2=True, prompt_seed=1, seq=0,
-               wseed=0, gain_jitter=0.0, vanilla=False, top_k=0, top_p=1.0):
+               wseed=0, gain_jitter=0.0, vanilla=False, top_k=0, top_p=1.0, mask_first=False):
     shape = W.CONFIGS[name]
     dec = Decoder(oracle_model(name, wseed, gain_jitter), temperature=T, seed=seed, seq=seq, top_k=top_k, top_p=top_p)
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=prompt_seed, seq=seq)
@@ -29,7 +29,8 @@ def oracle_run(name, n_prompt, n_decode, d1, d2, T=0.0, seed=2, gate=True, resid
         out, logits = dec.vanilla(n_decode, keep_logits=True)
         dec.verify_logits = logits
     else:
-        out = dec.loopspec(n_decode, d1, d2, gate=gate, residual_q2=residual_q2, keep_logits=True)
+        out = dec.loopspec(n_decode, d1, d2, gate=gate, residual_q2=residual_q2, keep_logits=True,
+                           mask_first=mask_first)
     return dict(prompt=prompt, first=first, tokens=out, dec=dec)
 
 

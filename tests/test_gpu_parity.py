@@ -120,6 +120,43 @@ def test_sampled_decode_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate
     ctx.close()
 
 
+MASKED_CASES = [
+    # name, n_prompt, n_decode, d1, d2, T, gate, residual, top_k, top_p
+    ("tiny", 16, 64, 1, 2, 0.0, False, True, 0, 1.0),         # greedy, ungated: the runner-up whenever the drafts agree
+    ("tiny_bf16", 16, 64, 1, 2, 0.0, False, True, 0, 1.0),
+    ("tiny_bf16", 16, 48, 1, 2, 0.0, True, True, 0, 1.0),     # greedy, gated: the mask never bites
+    ("tiny_bf16", 16, 64, 1, 2, 1.0, False, True, 0, 1.0),
+    ("tiny_bf16", 16, 64, 1, 2, 1.0, False, False, 0, 1.0),   # masked p_{d2} itself
+    ("tiny_bf16", 16, 48, 1, 3, 0.8, True, True, 0, 1.0),
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, False, True, 0, 0.7),    # with a nucleus
+    ("tiny", 16, 48, 1, 2, 1.0, False, False, 0, 0.6),
+    ("small_bf16", 40, 32, 1, 2, 1.0, False, True, 0, 1.0),
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, False, True, 2, 1.0),  # two-token nuclei: the residual can sit on the first candidate alone
+    ("tiny_bf16", 16, 48, 1, 2, 1.0, False, True, 1, 1.0),  # one-token nuclei: no second proposal where the drafts agree
+    ("tiny", 16, 48, 1, 2, 1.0, False, True, 2, 1.0),
+]
+
+
+@pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,gate,residual,top_k,top_p", MASKED_CASES)
+def test_masked_second_proposal_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate, residual, top_k, top_p):
+    """The variant of the second-proposal ablation (Sec. 5): the first candidate is masked out of the second
+    proposal; draws, decisions and tokens as the oracle's."""
+    kw = dict(T=T, seed=4, gate=gate, residual_q2=residual, top_k=top_k, top_p=top_p, mask_first=True)
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, **kw)
+    ctx = U.make_ctx(name, d1, d2, max_ctx=n_prompt + n_decode + 8, **kw)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(n_decode)
+    U.assert_same_run(ctx, ref, n_decode)
+    st, so = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
+        assert st[k] == so[k], (k, st[k], so[k])
+    if name == "tiny" and T == 0.0:   # the two drafts agree here, so the mask really picks runners-up
+        assert sum(e["kind"] == "draft2" for e in ref["dec"].log) > 10
+    if T == 0.0:
+        assert ref["tokens"] == U.oracle_run(name, n_prompt, n_decode, 0, 0, vanilla=True)["tokens"]
+    ctx.close()
+
+
 FILTERED_CASES = [
     # name, n_prompt, n_decode, d1, d2, T, top_k, top_p
     ("tiny_bf16", 16, 48, 1, 2, 1.0, 0, 0.7),       # the paper's sampling setting: T = 1, top-p 0.7

@@ -52,12 +52,12 @@ def random_dist(rng, V, conc=1.0):
     return rng.dirichlet(np.full(V, conc))
 
 
-def cascade_law(p, q1, q2t, gate=True, residual_q2=True):
+def cascade_law(p, q1, q2t, gate=True, residual_q2=True, mask_first=False):
     """Exact output law of drafting + cascade verification, by enumeration over (x1, x2)."""
     V = len(p)
     law = np.zeros(V)
     rho1 = sp.residual(p, q1)
-    q2 = sp.residual(q2t, q1) if residual_q2 else q2t
+    q2_plain = sp.residual(q2t, q1) if residual_q2 else q2t
     p_rej1 = p_rej_both = 0.0
     for x1 in range(V):
         if q1[x1] == 0:
@@ -67,6 +67,11 @@ def cascade_law(p, q1, q2t, gate=True, residual_q2=True):
         rej = q1[x1] * (1 - a1)
         p_rej1 += rej
         if gate and not (q2t[x1] < q1[x1]):
+            law += rej * rho1
+            p_rej_both += rej
+            continue
+        q2 = sp.masked_second_proposal(q2t, q1, x1, residual_q2) if mask_first else q2_plain
+        if q2 is None:                      # nothing left to propose: resample from the first residual
             law += rej * rho1
             p_rej_both += rej
             continue
@@ -89,6 +94,31 @@ def test_cascade_is_lossless_by_enumeration(V, gate, residual_q2):
         p, q1, q2t = (random_dist(rng, V, c) for c in (0.7, 1.0, 0.8))
         law, _, _ = cascade_law(p, q1, q2t, gate, residual_q2)
         np.testing.assert_allclose(law, p, atol=1e-12)
+
+
+def test_masked_second_proposal_definition_and_losslessness():
+    """Second-proposal ablation (Sec. 5): masking the first candidate gives a distribution with no mass on it, in
+    proportion to the unmasked proposal elsewhere; verification stays exact for it (any proposal is admissible)."""
+    rng = np.random.default_rng(21)
+    for V in (3, 6):
+        for _ in range(20):
+            p, q1, q2t = (random_dist(rng, V, c) for c in (0.7, 1.0, 0.8))
+            for residual_q2 in (True, False):
+                for gate in (True, False):
+                    law, _, _ = cascade_law(p, q1, q2t, gate, residual_q2, mask_first=True)
+                    np.testing.assert_allclose(law, p, atol=1e-12)
+                x1 = int(rng.integers(V))
+                q2 = sp.masked_second_proposal(q2t, q1, x1, residual_q2)
+                plain = sp.residual(q2t, q1) if residual_q2 else q2t
+                assert q2[x1] == 0 and abs(q2.sum() - 1) < 1e-12
+                others = np.arange(V) != x1
+                if plain[others].sum() > 0:
+                    np.testing.assert_allclose(q2[others], plain[others] / plain[others].sum(), atol=1e-12)
+    # degenerate cases: the residual sits on x1 alone -> q2~ without x1; q2~ sits on x1 alone -> no proposal
+    q1 = np.array([0.5, 0.5, 0.0]); q2t = np.array([0.7, 0.3, 0.0])
+    np.testing.assert_allclose(sp.masked_second_proposal(q2t, q1, 0), [0, 1, 0])
+    assert sp.masked_second_proposal(np.array([1.0, 0, 0]), q1, 0) is None
+    assert sp.masked_second_proposal(np.array([1.0, 0, 0]), q1, 0, residual_q2=False) is None
 
 
 def tv(a, b):
