@@ -8,6 +8,9 @@ it; it shares no code with the CUDA path.
 Parity status of what lives here:
   * model forward, depth-indexed KV  : pinned (cache-free library forward)
   * residual operator, cascade rule  : pinned (exact enumeration, chi-square, Thm 1)
+  * top-k / top-p filter, masked second proposal: pinned (definition on small
+    cases, exact enumeration of the output law)
+  * envelope fit (Sec. 4.1)           : pinned (closed form on power-law data)
   * Philox4x32-10                    : pinned (published known-answer vectors)
   * closed-form depths, branch bound : pinned (values printed in the paper)
   * scheduler (Algorithm 1)          : pinned (losslessness, commit-gap schedule)
