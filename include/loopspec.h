@@ -58,6 +58,9 @@ typedef struct {
  * gate = 1 applies Eq. 6, gate = 0 always creates the second proposal; residual_q2 = 1 drafts it from
  * p_{d2} (-) p_{d1} (Eq. 5), 0 from p_{d2} itself.  temperature 0 = greedy.  max_prefill_rows (0 = default)
  * bounds how many prompt positions one prefill pass carries.
+ * Capacity: max_ctx counts positions per sequence, the speculative ones included: a sequence needs
+ * max_ctx >= prompt + decoded tokens + R/d1 + 2 (the deepest chain of uncommitted positions); R/d1 may not exceed 8 and
+ * max_seqs times the branch bound of Sec. 4.3 may not exceed 64 rows (LOOPSPEC_ECAPACITY otherwise).
  * top_k, top_p: the optional filters of the post-layers C (Sec. 3.1), applied at EVERY readout depth when
  * temperature > 0: tokens are ranked by decreasing probability (ties: lower index first); top_k > 0 keeps the first
  * top_k and renormalises; 0 < top_p < 1 then keeps the shortest prefix of the ranking whose mass reaches top_p and

@@ -120,6 +120,30 @@ def test_sampled_decode_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate
     ctx.close()
 
 
+DEEP_LOOP_CASES = [
+    # name, d1, d2, T          (R = 8 / 16; up to ~50 rows in one pass, close to the branch bound of 54)
+    ("tiny_r8", 1, 2, 0.0), ("tiny_r8", 1, 2, 1.0), ("tiny_r8", 1, 4, 0.0), ("tiny_r8", 2, 6, 1.0), ("tiny_r8", 4, 0, 1.0),
+    ("tiny_r16", 2, 4, 0.0), ("tiny_r16", 2, 8, 1.0), ("tiny_r16", 4, 12, 1.0),
+]
+
+
+@pytest.mark.parametrize("name,d1,d2,T", DEEP_LOOP_CASES)
+def test_deeper_loops_match_oracle(name, d1, d2, T):
+    """More pipeline levels and wider passes than R = 4 gives (Sec. 4.3: the branch bound grows quickly with R / d1)."""
+    n_prompt, n_decode = 16, 40
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=2)
+    ctx = U.make_ctx(name, d1, d2, T=T, seed=2, max_ctx=n_prompt + n_decode + 24)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(n_decode)
+    U.assert_same_run(ctx, ref, n_decode)
+    st, so = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
+        assert st[k] == so[k], (k, st[k], so[k])
+    if (d1, d2) == (1, 2) or (name, d1, d2) == ("tiny_r16", 2, 4):
+        assert so["rows_max"] > 32           # the widest kernels (more than 32 rows) really run
+    ctx.close()
+
+
 MASKED_CASES = [
     # name, n_prompt, n_decode, d1, d2, T, gate, residual, top_k, top_p
     ("tiny", 16, 64, 1, 2, 0.0, False, True, 0, 1.0),         # greedy, ungated: the runner-up whenever the drafts agree

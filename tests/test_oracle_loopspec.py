@@ -56,6 +56,29 @@ def test_greedy_loopspec_equals_vanilla_for_every_admissible_depth_pair(models, 
         assert seen_sources == {1, 2, 3} or seen_sources == {2, 3}
 
 
+@pytest.mark.parametrize("name,pairs", [("tiny_r8", [(1, 2), (1, 4), (2, 4), (2, 6), (4, 0)]),
+                                        ("tiny_r16", [(2, 4), (2, 8), (4, 12), (8, 0)])])
+def test_deeper_loops_greedy_equals_vanilla_and_rows_stay_under_the_bound(name, pairs):
+    """Algorithm 1 for R = 8 and 16 (the Raven-style models loop 32 times): the greedy stream is the vanilla one, commit
+    gaps are d1 / d2 / R, and the rows in flight never exceed the branch bound of Sec. 4.3."""
+    shape, model = build(name)
+    Rn = shape.R
+    prompt = W.make_prompt(shape.vocab, 12)
+    n = 24
+    van = Decoder(model)
+    van.prefill(prompt, n)
+    ref = van.vanilla(n)
+    for d1, d2 in pairs:
+        dec = Decoder(model)
+        dec.prefill(prompt, n)
+        assert dec.loopspec(n, d1, d2) == ref, (name, d1, d2)
+        steps = [c["step"] for c in dec.commits]
+        cost = {1: d1, 2: d2, 3: Rn}
+        assert steps[0] == Rn
+        assert list(np.diff(steps)) == [cost[c["source"]] for c in dec.commits[:-1]]
+        assert dec.stats["rows_max"] <= dp.max_branches(Rn, d1, d2)
+
+
 def test_gamma_attains_R_over_d1_when_everything_is_accepted(models):
     shape, model = models["tiny"]
     dec = Decoder(model)

@@ -71,6 +71,11 @@ CONFIGS = {
     # and with head size 128, fp32 weights
     "tiny_gqa_f32": ModelShape("tiny_gqa_f32", vocab=512, hidden=512, n_q_heads=4, n_kv_heads=1, head_dim=128,
                                ffn=1024, n_recurrent=2, R=4, weight_dtype="fp32", tied=True),
+    # deeper loops (the Raven-style models run R = 32): more pipeline levels in flight, larger branch bounds
+    "tiny_r8": ModelShape("tiny_r8", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                          ffn=704, n_recurrent=2, R=8, weight_dtype="bf16", tied=False),
+    "tiny_r16": ModelShape("tiny_r16", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                           ffn=704, n_recurrent=1, R=16, weight_dtype="bf16", tied=False),
     # a mid-size bf16 model whose GEMMs span several tiles, K-slices and a ragged last tile
     "small_bf16": ModelShape("small_bf16", vocab=4000, hidden=768, n_q_heads=6, n_kv_heads=6, head_dim=128,
                              ffn=2000, n_recurrent=3, R=4, weight_dtype="bf16", tied=False),
