@@ -564,13 +564,31 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
 #else
           const uint4 a_lo = lds128(ring_s + c_slot), a_hi = lds128(ring_s + c_slot + HI_OFF);
 #endif
+          if (NG == 1) {
 #pragma unroll
-          for (int s = 0; s < 3; ++s) {
+            for (int s = 0; s < 3; ++s) {
+              const uint4 b = lds128(xk + s * X_PLANE);
+              mma_bf16(acc[s][0], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
+              mma_bf16(acc[s][0], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
+            }
+          } else {
+            // wide passes: a plane's B fragments are requested together, one plane ahead of the MMAs that use them
+            // (the asm statements keep their order, so a load placed next to its MMA would expose the shared-memory
+            // latency once per column group); the accumulation order of every chain is unchanged
+            uint4 b[2][NG];
 #pragma unroll
-            for (int n = 0; n < NG; ++n) {
-              const uint4 b = lds128(xk + s * X_PLANE + n * 512);
-              mma_bf16(acc[s][n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b.x, b.y);
-              mma_bf16(acc[s][n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b.z, b.w);
+            for (int n = 0; n < NG; ++n) b[0][n] = lds128(xk + n * 512);
+#pragma unroll
+            for (int s = 0; s < 3; ++s) {
+              if (s < 2) {
+#pragma unroll
+                for (int n = 0; n < NG; ++n) b[(s + 1) & 1][n] = lds128(xk + (s + 1) * X_PLANE + n * 512);
+              }
+              // the two k-halves of a chain depend on each other: all first halves, then all second halves
+#pragma unroll
+              for (int n = 0; n < NG; ++n) mma_bf16(acc[s][n], a_lo.x, a_hi.x, a_lo.y, a_hi.y, b[s & 1][n].x, b[s & 1][n].y);
+#pragma unroll
+              for (int n = 0; n < NG; ++n) mma_bf16(acc[s][n], a_lo.z, a_hi.z, a_lo.w, a_hi.w, b[s & 1][n].z, b[s & 1][n].w);
             }
           }
         }
