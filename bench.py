@@ -132,6 +132,53 @@ def run_kernel_only(args):
     ctx.close()
 
 
+def run_linear_tc(args):
+    """Time the stand-alone tcgen05 / TMA linear operator on one GEMM shape of the workload's model, next to the
+    mma.sync kernel of the decode pass on the same shape: prints its own JSON line.  Every launch reads another
+    layer's weights (the set is larger than L2); the operator's launches are replayed from a CUDA graph."""
+    import torch
+    import paper_2609_17184_b200 as ls
+    wl = W.WORKLOADS[args.workload]
+    sh = W.CONFIGS[wl.model]
+    hq, hkv = sh.n_q_heads * sh.head_dim, sh.n_kv_heads * sh.head_dim
+    N, K = {"qkv": (hq + 2 * hkv, sh.hidden), "o_proj": (sh.hidden, hq), "gate_up": (2 * sh.ffn, sh.hidden),
+            "down": (sh.hidden, sh.ffn), "lm_head": (sh.vocab, sh.hidden)}[args.linear_tc]
+    M = args.rows
+    n_w = max(4, min(24, int(400e6 // (N * K * 2)) + 1))
+    Ws = [torch.randn(N, K, device="cuda").mul_(0.02).to(torch.bfloat16) for _ in range(n_w)]
+    x = torch.randn(M, K, device="cuda")
+    sc = torch.empty(ls.lib.loopspec_linear_tc_scratch_bytes(M, N, K) + 256, dtype=torch.uint8, device="cuda")
+    sc2 = torch.zeros(ls.linear_scratch_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    st = torch.cuda.Stream()
+
+    def graph_us(fn):
+        with torch.cuda.stream(st):
+            for w in Ws[:2]:
+                fn(w)
+            st.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                for w in Ws:
+                    fn(w)
+            g.replay()
+            st.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for _ in range(args.iters):
+                g.replay()
+            e1.record(st)
+            e1.synchronize()
+        return e0.elapsed_time(e1) / (args.iters * len(Ws)) * 1e3
+
+    us_tc = graph_us(lambda w: ls.linear_tc(w, x, scratch=sc, check=False))
+    us_mma = graph_us(lambda w: ls.linear(w, x, scratch=sc2))
+    err = int(sc[(-sc.data_ptr()) % 256:][:4].view(torch.int32).item())
+    print(json.dumps({"linear_tc": args.linear_tc, "rows": M, "N": N, "K": K, "weight_sets": n_w, "bounded_wait_ran_out": err,
+                      "us_per_call_tcgen05_op": us_tc, "us_per_call_mma_sync_op": us_mma,
+                      "note": "whole operator per call inside a graph: tcgen05 = flag reset + split + GEMM + sum of k-splits "
+                              "(4 nodes); mma.sync = split + weight repack + GEMM (3 nodes; the repack reads W once more)"}))
+
+
 def run_profile_pass(args):
     """Prefill, then decode a few tokens and exit: the command profilers capture a steady-state pass from."""
     import paper_2609_17184_b200 as ls
@@ -414,12 +461,15 @@ def main():
     ap.add_argument("--closed-form", action="store_true",
                     help="sampling workloads: pick (d1, d2) from Theorem 2 on a TV profile measured on the device first")
     ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")
+    ap.add_argument("--linear-tc", choices=KERNELS, help="time the tcgen05 / TMA linear operator on this GEMM shape and exit")
     ap.add_argument("--profile-pass", type=int, default=0, help="prefill, decode this many tokens, exit (for profilers)")
     ap.add_argument("--rows", type=int, default=4)
     ap.add_argument("--iters", type=int, default=10)
     args = ap.parse_args()
     if args.kernel_only:
         return run_kernel_only(args)
+    if args.linear_tc:
+        return run_linear_tc(args)
     if args.profile_pass:
         return run_profile_pass(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

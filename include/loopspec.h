@@ -197,6 +197,18 @@ size_t loopspec_linear_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N,
                        int32_t K, void* scratch, size_t scratch_bytes, void* cuda_stream);
 
+/* The same linear map for bf16 weights on the tensor-memory path of sm_100a: weight tiles and activation planes arrive
+ * by TMA into a shared-memory ring, one thread issues tcgen05.mma (128 weight rows x up to 64 token columns per
+ * instruction, three exact bf16 planes of x per k-step, fp32 accumulator in tensor memory), K is split over CTAs and
+ * the partial sums are added in split order.  W is read in place (row-major, 16-byte aligned; no packed copy).
+ * All pointers device; x, y fp32; scratch: device, 256-byte aligned, loopspec_linear_tc_scratch_bytes(M, N, K) bytes
+ * (0 = unsupported shape).  1 <= M <= 64, N % 8 == 0, K % 64 == 0, else LOOPSPEC_EINVAL.  Stream-ordered; every wait
+ * inside the kernel is bounded: after the stream has been synchronised the first int32 of scratch is non-zero if one ran
+ * out (y is then undefined).  Stand-alone operator: the decode pass does not use it. */
+size_t loopspec_linear_tc_scratch_bytes(int32_t M, int32_t N, int32_t K);
+int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, int32_t N, int32_t K, void* scratch,
+                          size_t scratch_bytes, void* cuda_stream);
+
 /* The same linear map for callers that cannot allocate device memory at all.  (The paper has no counterpart;
  * this is a packaging convenience.)  Two kinds of caller are meant: a serving process whose allocator has reserved
  * the whole device up front, so that a later cudaMalloc -- theirs or ours -- fails or fragments the pool; and a

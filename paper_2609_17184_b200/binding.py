@@ -13,7 +13,7 @@ EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loo
            "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_fit_envelope", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
            "loopspec_launches_per_step", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
-           "loopspec_op_linear_static",
+           "loopspec_op_linear_static", "loopspec_linear_tc_scratch_bytes", "loopspec_op_linear_tc",
            "loopspec_last_error", "loopspec_destroy"]
 
 STATUS = {0: "OK", -1: "EINVAL", -2: "ESTATE", -3: "ECAPACITY", -4: "ECUDA", -5: "ETIMEOUT", -6: "EUNSUPPORTED"}
@@ -85,6 +85,9 @@ def _load():
     lib.loopspec_linear_scratch_bytes.restype = C.c_size_t
     lib.loopspec_linear_scratch_bytes.argtypes = [I, I, I]
     lib.loopspec_op_linear.argtypes = [V, I, V, V, I, I, I, V, C.c_size_t, V]
+    lib.loopspec_linear_tc_scratch_bytes.restype = C.c_size_t
+    lib.loopspec_linear_tc_scratch_bytes.argtypes = [I, I, I]
+    lib.loopspec_op_linear_tc.argtypes = [V, V, V, I, I, I, V, C.c_size_t, V]
     lib.loopspec_op_linear_static.argtypes = [V, I, V, V, I, I, I, V]
     lib.loopspec_last_error.restype = C.c_char_p
     lib.loopspec_last_error.argtypes = [V]
@@ -151,6 +154,30 @@ def linear(W, x, scratch=None):
                                 scratch.data_ptr(), scratch.numel(), torch.cuda.current_stream().cuda_stream)
     if rc:
         raise LoopSpecError(rc)
+    return y
+
+
+def linear_tc(W, x, scratch=None, check=True):
+    """y = x @ W.T through the tcgen05 / TMA operator.  W [N,K] bf16 (read in place), x [M,K] fp32 (cuda tensors).
+    check: synchronise and raise if a bounded wait inside the kernel ran out."""
+    import torch
+    M, K = x.shape
+    N = W.shape[0]
+    need = lib.loopspec_linear_tc_scratch_bytes(M, N, K)
+    if need == 0 or W.dtype != torch.bfloat16:
+        raise LoopSpecError(-1, "unsupported linear_tc shape or dtype")
+    if scratch is None:
+        scratch = torch.empty(need + 256, dtype=torch.uint8, device=x.device)
+    off = (-scratch.data_ptr()) % 256
+    y = torch.empty(M, N, dtype=torch.float32, device=x.device)
+    rc = lib.loopspec_op_linear_tc(W.data_ptr(), x.data_ptr(), y.data_ptr(), M, N, K, scratch.data_ptr() + off,
+                                   scratch.numel() - off, torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise LoopSpecError(rc, "op_linear_tc")
+    if check:
+        torch.cuda.current_stream().synchronize()
+        if int(scratch[off:off + 4].view(torch.int32).item()) != 0:
+            raise LoopSpecError(-5, "op_linear_tc: a bounded device-side wait ran out")
     return y
 
 

@@ -15,6 +15,7 @@
 #include "gemm.cuh"
 #include "pass.cuh"
 #include "select.cuh"
+#include "linear_tc.cuh"
 
 using namespace ls;
 
@@ -1300,6 +1301,94 @@ int loopspec_op_linear_static(const void* W, int32_t weight_dtype, const float* 
     scratch_of_device[dev] = ptr;
   }
   return loopspec_op_linear(W, weight_dtype, x, y, M, N, K, ptr, LOOPSPEC_STATIC_SCRATCH_BYTES, cuda_stream);
+}
+
+}  // extern "C"
+
+// ---- the same linear map on tcgen05 / TMA (stand-alone operator) ---------------------------------------------
+namespace {
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+// bf16 matrix [rows][K], K contiguous; box = 64 k x box_rows rows, 128-byte swizzle, zeros beyond the edges
+bool make_map_bf16(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+struct TcPlan {
+  int MP, stages, n_rb, n_split, kb_per_split;
+  size_t smem, planes_off, part_off, total;
+};
+bool plan_tc(int M, int N, int K, TcPlan* t) {
+  if (M < 1 || M > 64 || N < 8 || N % 8 || K < TC_BK || K % TC_BK) return false;
+  t->MP = (M + 15) / 16 * 16;
+  const int sb = tc_stage_bytes(t->MP);
+  // measured on the Ouro-1.4B shapes: up to 16 columns stream best from many small CTAs (two stages, four CTAs per
+  // SM); wider tiles from two CTAs per SM with deeper rings
+  const int kb_budget = t->MP <= 16 ? 56 : 100;
+  const int slots = t->MP <= 16 ? 592 : 296;
+  t->stages = std::max(2, std::min(TC_MAX_STAGES, (kb_budget * 1024) / sb));
+  t->smem = (size_t)t->stages * sb + 1024;
+  t->n_rb = (N + TC_BM - 1) / TC_BM;
+  const int total_kb = K / TC_BK;
+  int want = std::max(1, std::min(slots / t->n_rb, total_kb / 4));
+  t->kb_per_split = (total_kb + want - 1) / want;
+  t->n_split = (total_kb + t->kb_per_split - 1) / t->kb_per_split;
+  t->planes_off = 256;
+  t->part_off = t->planes_off + align_up((size_t)3 * t->MP * K * 2);
+  t->total = t->part_off + (t->n_split > 1 ? align_up((size_t)t->n_split * M * N * 4) : 0);
+  return true;
+}
+}  // namespace
+
+extern "C" {
+
+size_t loopspec_linear_tc_scratch_bytes(int32_t M, int32_t N, int32_t K) {
+  TcPlan t;
+  return plan_tc(M, N, K, &t) ? t.total : 0;
+}
+
+int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, int32_t N, int32_t K, void* scratch,
+                          size_t scratch_bytes, void* cuda_stream) {
+  TcPlan t;
+  if (!W || !x || !y || !plan_tc(M, N, K, &t) || (reinterpret_cast<uintptr_t>(W) & 15)) return LOOPSPEC_EINVAL;
+  if (!scratch || scratch_bytes < t.total || (reinterpret_cast<uintptr_t>(scratch) & 255)) return LOOPSPEC_ECAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* sc = static_cast<unsigned char*>(scratch);
+  __nv_bfloat16* planes = reinterpret_cast<__nv_bfloat16*>(sc + t.planes_off);
+  CUtensorMap map_w, map_x;
+  if (!make_map_bf16(&map_w, W, N, K, TC_BM) || !make_map_bf16(&map_x, planes, 3 * t.MP, K, 3 * t.MP)) return LOOPSPEC_ECUDA;
+  if (cudaMemsetAsync(sc, 0, 256, st) != cudaSuccess) return LOOPSPEC_ECUDA;
+  tc_split_kernel<<<t.MP, 256, 0, st>>>(x, planes, M, t.MP, K);
+  LinearTcParams p;
+  memset(&p, 0, sizeof p);
+  p.out = t.n_split > 1 ? reinterpret_cast<float*>(sc + t.part_off) : y;
+  p.M = M, p.MP = t.MP, p.N = N, p.K = K, p.kb_per_split = t.kb_per_split, p.stages = t.stages;
+  p.err = reinterpret_cast<int*>(sc);
+  if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t.smem) != cudaSuccess)
+    return LOOPSPEC_ECUDA;
+  linear_tc_kernel<<<dim3(t.n_rb, t.n_split), TC_THREADS, t.smem, st>>>(map_w, map_x, p);
+  if (t.n_split > 1) tc_sum_splits_kernel<<<296, 256, 0, st>>>(p.out, y, (size_t)M * N, t.n_split);
+  return cudaGetLastError() == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
 }
 
 }  // extern "C"

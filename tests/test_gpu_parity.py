@@ -39,6 +39,42 @@ def test_linear_matches_definition(dtype, M, N, K):
     assert np.array_equal(ls.linear(Wt, xt).cpu().numpy().view(np.uint32), y.view(np.uint32))
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 128, 64), (4, 768, 256), (7, 1408, 256), (8, 256, 704), (5, 2000, 768),
+                                   (3, 2048, 2048), (16, 768, 768), (29, 512, 1984), (64, 256, 256), (33, 2000, 768),
+                                   (2, 11264, 2048), (6, 2048, 5632), (64, 11264, 2048)])
+def test_linear_tc_matches_definition(M, N, K):
+    """The tcgen05 / TMA operator against the definition of the product (exact three-plane split of x, fp32
+    accumulation in tensor memory): ragged row blocks, several k-splits, every column-tile width."""
+    import paper_2609_17184_b200 as ls
+    rng = np.random.default_rng(N * 7 + K + M)
+    Wn = W.bf16_round((rng.standard_normal((N, K)) * 0.05).astype(np.float32))
+    x = rng.standard_normal((M, K)).astype(np.float32) * rng.uniform(0.1, 3.0, (M, 1)).astype(np.float32)
+    Wt = torch.from_numpy(Wn).cuda().to(torch.bfloat16)
+    xt = torch.from_numpy(x).cuda()
+    y = ls.linear_tc(Wt, xt).cpu().numpy()
+    ref = x.astype(np.float64) @ Wn.astype(np.float64).T
+    scale = np.abs(x).astype(np.float64) @ np.abs(Wn).astype(np.float64).T
+    assert (np.abs(y - ref) <= 2e-6 * scale + 1e-30).all(), np.abs(y - ref).max()
+    # reproducible bit for bit, and a row does not depend on the rows beside it in the same column tile
+    assert np.array_equal(ls.linear_tc(Wt, xt).cpu().numpy().view(np.uint32), y.view(np.uint32))
+    if M <= 16:
+        y1 = ls.linear_tc(Wt, xt[:1].contiguous()).cpu().numpy()
+        assert np.array_equal(y1[0].view(np.uint32), y[0].view(np.uint32))
+    # agrees with the mma.sync kernel of the decode pass to rounding
+    y2 = ls.linear(Wt, xt).cpu().numpy()
+    assert (np.abs(y - y2) <= 4e-6 * scale + 1e-30).all()
+
+
+def test_linear_tc_rejects_unsupported_shapes():
+    import paper_2609_17184_b200 as ls
+    assert ls.lib.loopspec_linear_tc_scratch_bytes(4, 256, 256) > 0
+    for M, N, K in [(0, 256, 256), (65, 256, 256), (4, 252, 256), (4, 256, 200), (4, 256, 32)]:
+        assert ls.lib.loopspec_linear_tc_scratch_bytes(M, N, K) == 0
+    Wt = torch.zeros(256, 200, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ls.LoopSpecError):
+        ls.linear_tc(Wt, torch.zeros(4, 200, device="cuda"))
+
+
 # ---- end-to-end parity -------------------------------------------------------------------------------
 GREEDY_CASES = [
     ("tiny", 16, 64, 1, 0, True),            # BASELINE config 0 as given
