@@ -170,10 +170,13 @@ def run_linear_tc(args):
             e1.synchronize()
         return e0.elapsed_time(e1) / (args.iters * len(Ws)) * 1e3
 
+    us_alone = ls.time_linear_tc(Ws, x, iters=args.iters)
     us_tc = graph_us(lambda w: ls.linear_tc(w, x, scratch=sc, check=False))
     us_mma = graph_us(lambda w: ls.linear(w, x, scratch=sc2))
     err = int(sc[(-sc.data_ptr()) % 256:][:4].view(torch.int32).item())
     print(json.dumps({"linear_tc": args.linear_tc, "rows": M, "N": N, "K": K, "weight_sets": n_w, "bounded_wait_ran_out": err,
+                      "us_per_launch_tcgen05_kernel_alone": us_alone, "GBps_kernel_alone": N * K * 2 / us_alone / 1e3,
+                      "frac_of_measured_hbm_peak": N * K * 2 / us_alone / 1e3 / measured_peaks()[0] if us_alone else None,
                       "us_per_call_tcgen05_op": us_tc, "us_per_call_mma_sync_op": us_mma,
                       "note": "whole operator per call inside a graph: tcgen05 = flag reset + split + GEMM + sum of k-splits "
                               "(4 nodes); mma.sync = split + weight repack + GEMM (3 nodes; the repack reads W once more)"}))

@@ -208,6 +208,14 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
 size_t loopspec_linear_tc_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, int32_t N, int32_t K, void* scratch,
                           size_t scratch_bytes, void* cuda_stream);
+/* Measurement aid for the operator above: the tcgen05 kernel alone, launched back to back with programmatic dependent
+ * launch (each launch requests its first weight tiles while the previous one still runs, as a kernel of the decode
+ * pass does), cycling over n_w (<= 64) weight matrices Ws[i] (HOST array of device pointers, each [N][K] bf16) so that
+ * consecutive launches stream different memory.  x is split once; the k-split partial sums stay in scratch (same size
+ * rule as above).  One untimed round over the matrices, then iters timed rounds; us_out (host) = mean microseconds per
+ * launch from CUDA events on cuda_stream.  Blocks until done. */
+int loopspec_time_linear_tc(const void* const* Ws, int32_t n_w, const float* x, int32_t M, int32_t N, int32_t K,
+                            void* scratch, size_t scratch_bytes, int32_t iters, float* us_out, void* cuda_stream);
 
 /* The same linear map for callers that cannot allocate device memory at all.  (The paper has no counterpart;
  * this is a packaging convenience.)  Two kinds of caller are meant: a serving process whose allocator has reserved

@@ -13,7 +13,7 @@ EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loo
            "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_fit_envelope", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
            "loopspec_launches_per_step", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
-           "loopspec_op_linear_static", "loopspec_linear_tc_scratch_bytes", "loopspec_op_linear_tc",
+           "loopspec_op_linear_static", "loopspec_linear_tc_scratch_bytes", "loopspec_op_linear_tc", "loopspec_time_linear_tc",
            "loopspec_last_error", "loopspec_destroy"]
 
 STATUS = {0: "OK", -1: "EINVAL", -2: "ESTATE", -3: "ECAPACITY", -4: "ECUDA", -5: "ETIMEOUT", -6: "EUNSUPPORTED"}
@@ -88,6 +88,7 @@ def _load():
     lib.loopspec_linear_tc_scratch_bytes.restype = C.c_size_t
     lib.loopspec_linear_tc_scratch_bytes.argtypes = [I, I, I]
     lib.loopspec_op_linear_tc.argtypes = [V, V, V, I, I, I, V, C.c_size_t, V]
+    lib.loopspec_time_linear_tc.argtypes = [C.POINTER(V), I, V, I, I, I, V, C.c_size_t, I, C.POINTER(C.c_float), V]
     lib.loopspec_op_linear_static.argtypes = [V, I, V, V, I, I, I, V]
     lib.loopspec_last_error.restype = C.c_char_p
     lib.loopspec_last_error.argtypes = [V]
@@ -179,6 +180,27 @@ def linear_tc(W, x, scratch=None, check=True):
         if int(scratch[off:off + 4].view(torch.int32).item()) != 0:
             raise LoopSpecError(-5, "op_linear_tc: a bounded device-side wait ran out")
     return y
+
+
+def time_linear_tc(Ws, x, iters=10):
+    """Mean microseconds per launch of the tcgen05 kernel alone, back to back over the weight matrices Ws."""
+    import torch
+    M, K = x.shape
+    N = Ws[0].shape[0]
+    need = lib.loopspec_linear_tc_scratch_bytes(M, N, K)
+    if need == 0:
+        raise LoopSpecError(-1, "unsupported linear_tc shape")
+    scratch = torch.empty(need + 256, dtype=torch.uint8, device=x.device)
+    off = (-scratch.data_ptr()) % 256
+    ptrs = (C.c_void_p * len(Ws))(*[w.data_ptr() for w in Ws])
+    us = C.c_float(0)
+    rc = lib.loopspec_time_linear_tc(ptrs, len(Ws), x.data_ptr(), M, N, K, scratch.data_ptr() + off, scratch.numel() - off,
+                                     iters, C.byref(us), torch.cuda.current_stream().cuda_stream)
+    if rc:
+        raise LoopSpecError(rc, "time_linear_tc")
+    if int(scratch[off:off + 4].view(torch.int32).item()) != 0:
+        raise LoopSpecError(-5, "time_linear_tc: a bounded device-side wait ran out")
+    return us.value
 
 
 def linear_static(W, x):

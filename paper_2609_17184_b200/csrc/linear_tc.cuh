@@ -100,7 +100,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   const int n_kb = min(p.kb_per_split, p.K / TC_BK - kb0);
   const unsigned tmem_cols = p.MP <= 32 ? 32u : 64u;
 
-  if (tid == 32) {  // the producer fetches the two tensor maps while the barriers and the tensor memory are set up
+  if (tid == 32) {  // the producer fetches the two tensor maps while the barriers are set up
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<unsigned long long>(&map_w)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<unsigned long long>(&map_x)) : "memory");
   }
@@ -110,6 +110,19 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  // The weights are constants, so the first ring-full of weight tiles is requested ahead of the predecessor's
+  // completion - and while warp 0 still allocates the tensor memory; the activation tiles (which the predecessor may
+  // still be writing) follow after the dependency wait, on the same barriers.
+  const int pre = min(p.stages, n_kb);
+  if (tid == 32) {
+    for (int kb = 0; kb < pre; ++kb) {
+      const unsigned bar = tc_smem_u32(&s_full[kb]);
+      tc_mbar_expect_tx(bar, (unsigned)stage_bytes);
+      tc_tma_load_2d(base + kb * stage_bytes, &map_w, bar, (kb0 + kb) * TC_BK, n0);
+    }
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&s_tmem)), "r"(tmem_cols)
@@ -121,12 +134,15 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem = s_tmem;
 
+  pdl_wait();
   if (tid == 32 && n_kb > 0) {
     // ---- producer: one thread keeps the ring of stages filled by TMA ----
+    for (int kb = 0; kb < pre; ++kb)
+      tc_tma_load_2d(base + kb * stage_bytes + TC_BM * TC_BK * 2, &map_x, tc_smem_u32(&s_full[kb]), (kb0 + kb) * TC_BK, 0);
     bool ok = true;
-    for (int kb = 0; kb < n_kb && ok; ++kb) {
+    for (int kb = pre; kb < n_kb && ok; ++kb) {
       const int s = kb % p.stages;
-      if (kb >= p.stages) ok = tc_mbar_wait(tc_smem_u32(&s_empty[s]), ((kb / p.stages) - 1) & 1);  // its MMAs are done
+      ok = tc_mbar_wait(tc_smem_u32(&s_empty[s]), ((kb / p.stages) - 1) & 1);  // the stage's MMAs are done
       if (!ok) break;
       const unsigned bar = tc_smem_u32(&s_full[s]);
       const unsigned a = base + s * stage_bytes, b = a + TC_BM * TC_BK * 2;
@@ -135,7 +151,8 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
       tc_tma_load_2d(b, &map_x, bar, (kb0 + kb) * TC_BK, 0);
     }
     if (!ok) s_fail = 1, *p.err = 1;
-  } else if (tid == 0 && n_kb > 0) {
+  }
+  if (tid == 0 && n_kb > 0) {
     // ---- MMA issuer: one thread, the accumulator lives in tensor memory ----
     const unsigned idesc = tc_idesc(TC_BM, p.MP);
     bool ok = true;

@@ -1355,7 +1355,7 @@ bool plan_tc(int M, int N, int K, TcPlan* t) {
   t->n_split = (total_kb + t->kb_per_split - 1) / t->kb_per_split;
   t->planes_off = 256;
   t->part_off = t->planes_off + align_up((size_t)3 * t->MP * K * 2);
-  t->total = t->part_off + (t->n_split > 1 ? align_up((size_t)t->n_split * M * N * 4) : 0);
+  t->total = t->part_off + align_up((size_t)t->n_split * M * N * 4);
   return true;
 }
 }  // namespace
@@ -1389,6 +1389,53 @@ int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, in
   linear_tc_kernel<<<dim3(t.n_rb, t.n_split), TC_THREADS, t.smem, st>>>(map_w, map_x, p);
   if (t.n_split > 1) tc_sum_splits_kernel<<<296, 256, 0, st>>>(p.out, y, (size_t)M * N, t.n_split);
   return cudaGetLastError() == cudaSuccess ? LOOPSPEC_OK : LOOPSPEC_ECUDA;
+}
+
+int loopspec_time_linear_tc(const void* const* Ws, int32_t n_w, const float* x, int32_t M, int32_t N, int32_t K,
+                            void* scratch, size_t scratch_bytes, int32_t iters, float* us_out, void* cuda_stream) {
+  TcPlan t;
+  if (!Ws || n_w < 1 || n_w > 64 || !x || !us_out || iters < 1 || !plan_tc(M, N, K, &t)) return LOOPSPEC_EINVAL;
+  const size_t part_bytes = align_up((size_t)t.n_split * M * N * 4);
+  if (!scratch || scratch_bytes < t.part_off + part_bytes || (reinterpret_cast<uintptr_t>(scratch) & 255)) return LOOPSPEC_ECAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* sc = static_cast<unsigned char*>(scratch);
+  __nv_bfloat16* planes = reinterpret_cast<__nv_bfloat16*>(sc + t.planes_off);
+  std::vector<CUtensorMap> maps(n_w);
+  CUtensorMap map_x;
+  for (int i = 0; i < n_w; ++i)
+    if (!Ws[i] || (reinterpret_cast<uintptr_t>(Ws[i]) & 15) || !make_map_bf16(&maps[i], Ws[i], N, K, TC_BM)) return LOOPSPEC_EINVAL;
+  if (!make_map_bf16(&map_x, planes, 3 * t.MP, K, 3 * t.MP)) return LOOPSPEC_ECUDA;
+  if (cudaMemsetAsync(sc, 0, 256, st) != cudaSuccess) return LOOPSPEC_ECUDA;
+  tc_split_kernel<<<t.MP, 256, 0, st>>>(x, planes, M, t.MP, K);
+  LinearTcParams p;
+  memset(&p, 0, sizeof p);
+  p.out = reinterpret_cast<float*>(sc + t.part_off);
+  p.M = M, p.MP = t.MP, p.N = N, p.K = K, p.kb_per_split = t.kb_per_split, p.stages = t.stages;
+  p.err = reinterpret_cast<int*>(sc);
+  if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t.smem) != cudaSuccess)
+    return LOOPSPEC_ECUDA;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(t.n_rb, t.n_split), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = t.smem, cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = 1;
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return LOOPSPEC_ECUDA;
+  cudaError_t e = cudaSuccess;
+  for (int rep = 0; rep < iters + 1 && e == cudaSuccess; ++rep) {  // the first round warms up
+    if (rep == 1) e = cudaEventRecord(e0, st);
+    for (int i = 0; i < n_w && e == cudaSuccess; ++i) e = cudaLaunchKernelEx(&cfg, linear_tc_kernel, maps[i], map_x, p);
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+  if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+  float ms = 0.f;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  cudaEventDestroy(e0), cudaEventDestroy(e1);
+  if (e != cudaSuccess) return LOOPSPEC_ECUDA;
+  *us_out = ms * 1e3f / ((float)iters * n_w);
+  return LOOPSPEC_OK;
 }
 
 }  // extern "C"
