@@ -801,4 +801,61 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
   tune_mark(600, true);
 }
 
+// ======================= fused epilogue for sums produced by the tcgen05 kernel (prefill passes) ==========================
+// linear_tc_kernel leaves raw k-split partial sums [split][column][N] in global memory; one CTA per row block adds the
+// splits in split order into the receive-buffer layout of a one-rank cluster and runs the same epilogue code as the
+// mma.sync kernels (1/rms, then RoPE + KV write / residual + sum of squares + planes / SwiGLU + planes).
+constexpr int TCE_MAX_COLS = 64;
+constexpr int TCE_GROUPS = 8;    // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
+struct TcEpiParams {
+  GemmParams g;        // cluster_size = TCE_GROUPS
+  const float* part;   // [n_split][cols_ld][N]
+  int n_split, cols_ld;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_constant__ TcEpiParams q) {
+  __shared__ float s_recv[TCE_MAX_COLS * RB_ROWS];
+  __shared__ float s_colbuf[2 * RB_ROWS];
+  __shared__ float s_rstd[TCE_MAX_COLS];
+  __shared__ int s_ct[CT_FIELDS * TCE_MAX_COLS];
+  const GemmParams& p = q.g;
+  const int tid = threadIdx.x, rb = blockIdx.x;
+  const RowTable* tab = p.tab;  // final before the pass starts
+  int n_cols = tab->n_rows;
+  if (n_cols > TCE_MAX_COLS) n_cols = TCE_MAX_COLS;
+  gemm_load_cols(p, n_cols, TCE_MAX_COLS, s_ct);
+  pdl_launch_dependents();
+  pdl_wait();
+  if ((int)blockIdx.y >= n_cols) return;  // no column for this group
+  gemm_rstd(p, n_cols, s_rstd, s_ct, TCE_MAX_COLS);
+  // row j of the block -> row of the weight matrix (gate/up: 64 gate rows, then the 64 matching up rows)
+  const int j = tid & (RB_ROWS - 1);
+  int n;
+  if (EPI == EPI_SWIGLU) {
+    const int f = rb * 64 + (j & 63);
+    n = f < p.F ? (j < 64 ? f : p.F + f) : -1;
+  } else {
+    n = rb * RB_ROWS + j;
+    if (n >= p.N) n = -1;
+  }
+  // blockIdx.y takes the columns c = y, y + TCE_GROUPS, ... exactly as rank y of a cluster of TCE_GROUPS CTAs would;
+  // the other ranks' contributions in the receive buffer are zeros (adding them changes nothing)
+  const int rank = blockIdx.y, own_max = TCE_MAX_COLS / TCE_GROUPS;
+  for (int i = tid; i < TCE_MAX_COLS * RB_ROWS; i += GEMM_THREADS) s_recv[i] = 0.f;
+  __syncthreads();
+  const size_t split_stride = (size_t)q.cols_ld * p.N;
+  for (int c = rank + TCE_GROUPS * (tid >> 7); c < n_cols; c += TCE_GROUPS * (GEMM_THREADS / RB_ROWS)) {
+    float v = 0.f;
+    if (n >= 0) {
+      const float* src = q.part + (size_t)c * p.N + n;
+      v = src[0];
+      for (int s = 1; s < q.n_split; ++s) v += src[(size_t)s * split_stride];
+    }
+    s_recv[(c / TCE_GROUPS) * RB_ROWS + j] = v;
+  }
+  __syncthreads();
+  gemm_reduce_epilogue<EPI>(p, s_ct, TCE_MAX_COLS, rb, n_cols, s_recv, own_max, s_colbuf, s_rstd, rank);
+}
+
 }  // namespace ls

@@ -8,7 +8,8 @@
 // Activations are fp32 split exactly into three bf16 planes, so each k-step issues three MMAs into one accumulator.
 // K may be split over blockIdx.y; the partial sums are added in split order by a second kernel (no atomics).
 //
-// Stand-alone operator (loopspec_op_linear_tc); the decode pass itself still runs gemm_bf16_kernel.
+// Used by the stand-alone operator loopspec_op_linear_tc and by the prefill passes (tc_epilogue_kernel then applies the
+// fused epilogue of the GEMM); the decode passes run gemm_bf16_kernel.
 #pragma once
 #include <cuda.h>
 
@@ -27,7 +28,10 @@ struct LinearTcParams {
   int M, MP, N, K;     // MP = M rounded up to 16: columns of the MMA
   int kb_per_split;    // 64-wide k-blocks per blockIdx.y
   int stages;
-  int* err;            // device flag: set to 1 when a bounded wait ran out
+  int* err;            // flag the host reads: set to err_code when a bounded wait ran out
+  int err_code;
+  int x3d;             // 0: x planes stacked [3][MP][K], one box; 1: the decode pass's layout [column][3][x_ld], a
+                       // three-dimensional map (k, plane, column) and one box per plane
 };
 
 __device__ __forceinline__ unsigned tc_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -56,6 +60,12 @@ __device__ __forceinline__ void tc_tma_load_2d(unsigned dst, const CUtensorMap* 
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
       "l"(reinterpret_cast<unsigned long long>(map)), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tc_tma_load_3d(unsigned dst, const CUtensorMap* map, unsigned bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+      "l"(reinterpret_cast<unsigned long long>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
 // shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart
@@ -135,10 +145,18 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   const unsigned tmem = s_tmem;
 
   pdl_wait();
+  auto load_x = [&](unsigned b, unsigned bar, int k) {  // the three planes of the activations, plane pl at b + pl * MP * 128
+    if (p.x3d) {
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl) tc_tma_load_3d(b + pl * p.MP * TC_BK * 2, &map_x, bar, k, pl, 0);
+    } else {
+      tc_tma_load_2d(b, &map_x, bar, k, 0);
+    }
+  };
   if (tid == 32 && n_kb > 0) {
     // ---- producer: one thread keeps the ring of stages filled by TMA ----
     for (int kb = 0; kb < pre; ++kb)
-      tc_tma_load_2d(base + kb * stage_bytes + TC_BM * TC_BK * 2, &map_x, tc_smem_u32(&s_full[kb]), (kb0 + kb) * TC_BK, 0);
+      load_x(base + kb * stage_bytes + TC_BM * TC_BK * 2, tc_smem_u32(&s_full[kb]), (kb0 + kb) * TC_BK);
     bool ok = true;
     for (int kb = pre; kb < n_kb && ok; ++kb) {
       const int s = kb % p.stages;
@@ -148,9 +166,9 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
       const unsigned a = base + s * stage_bytes, b = a + TC_BM * TC_BK * 2;
       tc_mbar_expect_tx(bar, (unsigned)stage_bytes);
       tc_tma_load_2d(a, &map_w, bar, (kb0 + kb) * TC_BK, n0);
-      tc_tma_load_2d(b, &map_x, bar, (kb0 + kb) * TC_BK, 0);
+      load_x(b, bar, (kb0 + kb) * TC_BK);
     }
-    if (!ok) s_fail = 1, *p.err = 1;
+    if (!ok) s_fail = 1, *p.err = p.err_code;
   }
   if (tid == 0 && n_kb > 0) {
     // ---- MMA issuer: one thread, the accumulator lives in tensor memory ----
@@ -173,7 +191,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
       tc_commit(tc_smem_u32(&s_empty[s]));  // arrives when the MMAs issued so far have read their operands
     }
     if (ok) tc_commit(tc_smem_u32(&s_done));
-    else s_fail = 1, *p.err = 1;
+    else s_fail = 1, *p.err = p.err_code;
   }
   // everyone: the accumulator is complete when the last commit arrives
   bool have = n_kb > 0;
@@ -200,7 +218,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
         if (c0 + j < p.M && n < p.N) out[(size_t)(c0 + j) * p.N + n] = __uint_as_float(v[j]);
     }
   } else if (tid == 0) {
-    *p.err = 1;
+    *p.err = p.err_code;
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -75,8 +75,67 @@ int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ?
 
 static_assert(SEL_ARG_BLOCK == RB_ROWS, "the selection reads one argmax partial per lm_head row block");
 
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+// bf16 matrix [rows][K], K contiguous; box = 64 k x box_rows rows, 128-byte swizzle, zeros beyond the edges
+bool make_map_bf16(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// the activation planes of a pass, [column][3][x_ld] bf16, as a (k, plane, column) tensor; box = 64 k x 1 plane x cols
+bool make_map_planes3d(CUtensorMap* map, const void* ptr, int K, int x_ld, int n_cols, int box_cols) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)K, 3, (cuuint64_t)n_cols};
+  cuuint64_t strides[2] = {(cuuint64_t)x_ld * 2, (cuuint64_t)x_ld * 6};
+  cuuint32_t box[3] = {(cuuint32_t)TC_BK, 1, (cuuint32_t)box_cols};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// k-split of a prefill GEMM on the tcgen05 kernel: a function of the matrix alone, so that a prompt position's sums
+// do not depend on how many positions share the pass
+struct TcPfPlan {
+  int n_tiles, n_split, kb_per_split;
+};
+TcPfPlan tc_pf_plan(int N, int K) {
+  TcPfPlan t;
+  t.n_tiles = (N + TC_BM - 1) / TC_BM;
+  const int total_kb = K / TC_BK;
+  const int want = std::max(1, std::min(296 / t.n_tiles, total_kb / 4));
+  t.kb_per_split = (total_kb + want - 1) / want;
+  t.n_split = (total_kb + t.kb_per_split - 1) / t.kb_per_split;
+  return t;
+}
+// the prefill passes can run their four layer GEMMs on the tcgen05 kernel: bf16 weights, every K a multiple of 64
+bool tc_prefill_shapes_ok(const loopspec_model* m) {
+  return m->weight_dtype == 1 && m->hidden % TC_BK == 0 && (m->n_q_heads * m->head_dim) % TC_BK == 0 && m->ffn % TC_BK == 0;
+}
+int tc_pf_cols(int max_rows_pf) { return (max_rows_pf + 15) / 16 * 16; }
+
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, flt, sel_flt, tv, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, tcpart, flt, sel_flt, tv, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
@@ -204,6 +263,15 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sumsq = take(MR * d.sq_stride * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
   L.argpart = take(MR * ((m->vocab + 127) / 128) * sizeof(float2));
+  {  // k-split partial sums of the prefill GEMMs on the tcgen05 kernel (the largest of the four)
+    size_t need = 0;
+    if (tc_prefill_shapes_ok(m)) {
+      const int Ns[4] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden}, Ks[4] = {m->hidden, d.Hq, m->hidden, m->ffn};
+      for (int i = 0; i < 4; ++i)
+        need = std::max(need, (size_t)tc_pf_plan(Ns[i], Ks[i]).n_split * tc_pf_cols(d.max_rows_pf) * Ns[i] * 4);
+    }
+    L.tcpart = take(need);
+  }
   // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
   L.gpart = take((size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4 * MR * 128 * 4);
   L.ptrs = take((size_t)m->n_recurrent * 10 * sizeof(void*));
@@ -252,6 +320,13 @@ struct loopspec_ctx {
   int n_sm = 148;
   int ng_dec = 1, ng_pf = 1;
   GemmPlan plan[5];
+  // prefill on the tcgen05 kernel: tensor maps of the row-major weights (4 per layer) and of the three plane buffers
+  bool tc_pf = false;
+  std::vector<CUtensorMap> tc_wmaps;
+  CUtensorMap tc_xmaps[3];
+  TcPfPlan tc_plan[4];
+  int tc_cols = 0, tc_stages = 0;
+  size_t tc_smem = 0;
   volatile int* host_flags = nullptr;  // pinned + mapped
   int* host_flags_dev = nullptr;
   int* pin_ids = nullptr;              // pinned staging for prompt / ids
@@ -479,7 +554,40 @@ cudaError_t launch_pass(loopspec_ctx* c, const PassParams& pp) {
   return cudaLaunchKernelEx(&cfg, pass_fn(c->m.head_dim, c->m.n_q_heads / c->m.n_kv_heads), pp);
 }
 
-cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch) {
+// one layer GEMM of a prefill pass on the tcgen05 kernel: raw k-split sums, then the fused epilogue
+template <int EPI>
+cudaError_t launch_tc_epi(const TcEpiParams& q, cudaStream_t st, bool pdl) {
+  return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
+}
+cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
+  const TcPfPlan& t = c->tc_plan[which];
+  TcEpiParams q;
+  q.g = gemm_params(c, which, layer, tab);
+  q.g.cluster_size = TCE_GROUPS;
+  q.part = c->at<float>(c->L.tcpart), q.n_split = t.n_split, q.cols_ld = c->tc_cols;
+  LinearTcParams p;
+  memset(&p, 0, sizeof p);
+  p.out = c->at<float>(c->L.tcpart);
+  p.M = c->tc_cols, p.MP = c->tc_cols, p.N = q.g.N, p.K = q.g.K, p.kb_per_split = t.kb_per_split, p.stages = c->tc_stages;
+  p.err = const_cast<int*>(c->host_flags_dev + HF_ERROR), p.err_code = 5, p.x3d = 1;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(t.n_tiles, t.n_split), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = c->tc_smem, cfg.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at, cfg.numAttrs = c->use_pdl ? 1 : 0;
+  const int xi = which == G_O ? 1 : which == G_DOWN ? 2 : 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel, c->tc_wmaps[4 * layer + which], c->tc_xmaps[xi], p);
+  if (e != cudaSuccess) return e;
+  switch (which) {
+    case G_QKV: return launch_tc_epi<EPI_QKV>(q, c->stream, c->use_pdl);
+    case G_GU: return launch_tc_epi<EPI_SWIGLU>(q, c->stream, c->use_pdl);
+    default: return launch_tc_epi<EPI_RESID>(q, c->stream, c->use_pdl);
+  }
+}
+
+cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
@@ -499,7 +607,7 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     unsigned long long* tl = getenv("LOOPSPEC_DBG") ? reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024 : nullptr;  // tuning aid
     GemmParams gq = gemm_params(c, G_QKV, l, tab);
     gq.tl = tl, gq.tl_id = l * 5 + 0;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
+    if ((e = tc ? launch_tc_gemm(c, G_QKV, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
     AttnParams a;
     memset(&a, 0, sizeof a);
     a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
@@ -513,13 +621,13 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     if ((e = launch_k(attn_fn(m.head_dim, G, d.max_chunks > ATT_MAX_RUNS), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
     GemmParams go = gemm_params(c, G_O, l, tab);
     go.tl = tl, go.tl_id = l * 5 + 2;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
+    if ((e = tc ? launch_tc_gemm(c, G_O, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
     GemmParams gg = gemm_params(c, G_GU, l, tab);
     gg.tl = tl, gg.tl_id = l * 5 + 3;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
+    if ((e = tc ? launch_tc_gemm(c, G_GU, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
     GemmParams gd = gemm_params(c, G_DOWN, l, tab);
     gd.tl = tl, gd.tl_id = l * 5 + 4;
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
+    if ((e = tc ? launch_tc_gemm(c, G_DOWN, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
     if (n_launch) *n_launch += 5;
   }
   return cudaSuccess;
@@ -818,6 +926,27 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       g = plan_gemm(n_rbs[i], Ks[i], slots, true);
     }
   }
+  // prefill passes on the tcgen05 kernel (LOOPSPEC_NO_TC_PREFILL=1: the mma.sync kernels, as the decode passes)
+  if (tc_prefill_shapes_ok(m) && !getenv("LOOPSPEC_NO_TC_PREFILL") && encode_tiled_fn()) {
+    const Derived& dd = c->d;
+    c->tc_cols = tc_pf_cols(dd.max_rows_pf);
+    const int sb = tc_stage_bytes(c->tc_cols);
+    c->tc_stages = std::max(2, std::min(TC_MAX_STAGES, (100 * 1024) / sb));
+    c->tc_smem = (size_t)c->tc_stages * sb + 1024;
+    const int Ns[4] = {dd.Hq + 2 * dd.Hkv, m->hidden, 2 * m->ffn, m->hidden}, Ks[4] = {m->hidden, dd.Hq, m->hidden, m->ffn};
+    const int w_idx[4] = {1, 2, 4, 5};  // qkv, o, gate/up, down among a layer's six pointers
+    bool ok = true;
+    c->tc_wmaps.resize((size_t)4 * m->n_recurrent);
+    for (int l = 0; l < m->n_recurrent && ok; ++l)
+      for (int i = 0; i < 4 && ok; ++i) ok = make_map_bf16(&c->tc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], TC_BM);
+    const size_t x_off[3] = {c->L.xplanes, c->L.aplanes, c->L.splanes};
+    const int x_k[3] = {m->hidden, dd.Hq, m->ffn};
+    for (int i = 0; i < 3 && ok; ++i) ok = make_map_planes3d(&c->tc_xmaps[i], c->ws + x_off[i], x_k[i], x_k[i], dd.max_rows, c->tc_cols);
+    for (int i = 0; i < 4; ++i) c->tc_plan[i] = tc_pf_plan(Ns[i], Ks[i]);
+    ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tc_smem) == cudaSuccess;
+    if (!ok) (void)cudaGetLastError();
+    c->tc_pf = ok;
+  }
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
     (void)what;
@@ -970,7 +1099,7 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
       pp.hid = c->at<float>(c->L.hid), pp.H = c->m.hidden, pp.embed = c->embed, pp.weight_dtype = c->m.weight_dtype;
       prefill_setup_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(pp);
       CU(c, cudaGetLastError());
-      CU(c, launch_layers(c, tab, c->ng_pf, nullptr));
+      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf && !(c->use_mega && c->ng_pf == 1)));
     }
   }
   CU(c, launch_lm_head(c, tab, c->ng_pf));
@@ -1307,33 +1436,6 @@ int loopspec_op_linear_static(const void* W, int32_t weight_dtype, const float* 
 
 // ---- the same linear map on tcgen05 / TMA (stand-alone operator) ---------------------------------------------
 namespace {
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-// bf16 matrix [rows][K], K contiguous; box = 64 k x box_rows rows, 128-byte swizzle, zeros beyond the edges
-bool make_map_bf16(CUtensorMap* map, const void* ptr, int rows, int K, int box_rows) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 struct TcPlan {
   int MP, stages, n_rb, n_split, kb_per_split;
   size_t smem, planes_off, part_off, total;
@@ -1383,7 +1485,7 @@ int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, in
   memset(&p, 0, sizeof p);
   p.out = t.n_split > 1 ? reinterpret_cast<float*>(sc + t.part_off) : y;
   p.M = M, p.MP = t.MP, p.N = N, p.K = K, p.kb_per_split = t.kb_per_split, p.stages = t.stages;
-  p.err = reinterpret_cast<int*>(sc);
+  p.err = reinterpret_cast<int*>(sc), p.err_code = 1;
   if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t.smem) != cudaSuccess)
     return LOOPSPEC_ECUDA;
   linear_tc_kernel<<<dim3(t.n_rb, t.n_split), TC_THREADS, t.smem, st>>>(map_w, map_x, p);
@@ -1411,7 +1513,7 @@ int loopspec_time_linear_tc(const void* const* Ws, int32_t n_w, const float* x, 
   memset(&p, 0, sizeof p);
   p.out = reinterpret_cast<float*>(sc + t.part_off);
   p.M = M, p.MP = t.MP, p.N = N, p.K = K, p.kb_per_split = t.kb_per_split, p.stages = t.stages;
-  p.err = reinterpret_cast<int*>(sc);
+  p.err = reinterpret_cast<int*>(sc), p.err_code = 1;
   if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t.smem) != cudaSuccess)
     return LOOPSPEC_ECUDA;
   cudaLaunchConfig_t cfg;
