@@ -204,7 +204,8 @@ int loopspec_op_linear(const void* W, int32_t weight_dtype, const float* x, floa
  * All pointers device; x, y fp32; scratch: device, 256-byte aligned, loopspec_linear_tc_scratch_bytes(M, N, K) bytes
  * (0 = unsupported shape).  1 <= M <= 64, N % 8 == 0, K % 64 == 0, else LOOPSPEC_EINVAL.  Stream-ordered; every wait
  * inside the kernel is bounded: after the stream has been synchronised the first int32 of scratch is non-zero if one ran
- * out (y is then undefined).  Stand-alone operator: the decode pass does not use it. */
+ * out (y is then undefined).  The prefill passes of a context run their layer GEMMs on the same kernel; the decode passes
+ * do not. */
 size_t loopspec_linear_tc_scratch_bytes(int32_t M, int32_t N, int32_t K);
 int loopspec_op_linear_tc(const void* W, const float* x, float* y, int32_t M, int32_t N, int32_t K, void* scratch,
                           size_t scratch_bytes, void* cuda_stream);

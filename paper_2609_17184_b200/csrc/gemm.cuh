@@ -806,7 +806,7 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
 // splits in split order into the receive-buffer layout of a one-rank cluster and runs the same epilogue code as the
 // mma.sync kernels (1/rms, then RoPE + KV write / residual + sum of squares + planes / SwiGLU + planes).
 constexpr int TCE_MAX_COLS = 64;
-constexpr int TCE_GROUPS = 8;    // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
+constexpr int TCE_GROUPS = 16;   // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
 struct TcEpiParams {
   GemmParams g;        // cluster_size = TCE_GROUPS
   const float* part;   // [n_split][cols_ld][N]
@@ -828,7 +828,16 @@ __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_
   pdl_launch_dependents();
   pdl_wait();
   if ((int)blockIdx.y >= n_cols) return;  // no column for this group
-  gemm_rstd(p, n_cols, s_rstd, s_ct, TCE_MAX_COLS);
+  {  // 1/rms of this group's columns only (gemm_rstd's arithmetic: one partial per lane, butterfly sum)
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int c = blockIdx.y + TCE_GROUPS * warp; c < n_cols; c += TCE_GROUPS * (GEMM_THREADS / 32)) {
+      float ss = 0.f;
+      if (p.sumsq)
+        for (int i = lane; i < p.n_sq; i += 32) ss += p.sumsq[c * p.sq_stride + i];
+      ss = warp_sum(ss);
+      if (lane == 0) s_rstd[c] = p.sumsq ? 1.0f / sqrtf(ss / (float)p.H + p.eps) : 1.0f;
+    }
+  }
   // row j of the block -> row of the weight matrix (gate/up: 64 gate rows, then the 64 matching up rows)
   const int j = tid & (RB_ROWS - 1);
   int n;
@@ -849,8 +858,15 @@ __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_
     float v = 0.f;
     if (n >= 0) {
       const float* src = q.part + (size_t)c * p.N + n;
-      v = src[0];
-      for (int s = 1; s < q.n_split; ++s) v += src[(size_t)s * split_stride];
+      v = __ldcg(src);
+      for (int s0 = 1; s0 < q.n_split; s0 += 8) {  // eight loads in flight, added in split order
+        float t[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) t[u] = s0 + u < q.n_split ? __ldcg(src + (size_t)(s0 + u) * split_stride) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (s0 + u < q.n_split) v += t[u];
+      }
     }
     s_recv[(c / TCE_GROUPS) * RB_ROWS + j] = v;
   }
