@@ -16,6 +16,7 @@
 #include "pass.cuh"
 #include "select.cuh"
 #include "linear_tc.cuh"
+#include "gemm_tc.cuh"
 
 using namespace ls;
 
@@ -327,6 +328,11 @@ struct loopspec_ctx {
   TcPfPlan tc_plan[4];
   int tc_cols = 0, tc_stages = 0;
   size_t tc_smem = 0;
+  // ... and in one kernel per GEMM (cluster reduction + epilogue inside): weight maps with 64-row boxes
+  bool tc_fused = false;
+  std::vector<CUtensorMap> gtc_wmaps;
+  int gtc_cs[4] = {1, 1, 1, 1}, gtc_stages = 0;
+  size_t gtc_smem = 0;
   volatile int* host_flags = nullptr;  // pinned + mapped
   int* host_flags_dev = nullptr;
   int* pin_ids = nullptr;              // pinned staging for prompt / ids
@@ -559,7 +565,43 @@ template <int EPI>
 cudaError_t launch_tc_epi(const TcEpiParams& q, cudaStream_t st, bool pdl) {
   return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
 }
+template <int EPI>
+cudaError_t launch_gtc_epi(loopspec_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, const GemmTcParams& q) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(q.g.n_rb * q.g.cluster_size), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = c->gtc_smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int n = 0;
+  if (c->use_pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (q.g.cluster_size > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = q.g.cluster_size, at[n].val.clusterDim.y = 1, at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = at, cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, mw, mx, q);
+}
+cudaError_t launch_gtc(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
+  GemmTcParams q;
+  q.g = gemm_params(c, which, layer, tab);
+  q.g.cluster_size = c->gtc_cs[which], q.g.n_clusters = q.g.n_rb;
+  q.g.err = c->host_flags_dev + HF_ERROR;
+  q.MP = c->tc_cols, q.stages = c->gtc_stages, q.err_code = 5;
+  const int xi = which == G_O ? 1 : which == G_DOWN ? 2 : 0;
+  const CUtensorMap& mw = c->gtc_wmaps[4 * layer + which];
+  switch (which) {
+    case G_QKV: return launch_gtc_epi<EPI_QKV>(c, mw, c->tc_xmaps[xi], q);
+    case G_GU: return launch_gtc_epi<EPI_SWIGLU>(c, mw, c->tc_xmaps[xi], q);
+    default: return launch_gtc_epi<EPI_RESID>(c, mw, c->tc_xmaps[xi], q);
+  }
+}
 cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
+  if (c->tc_fused) return launch_gtc(c, which, layer, tab);
   const TcPfPlan& t = c->tc_plan[which];
   TcEpiParams q;
   q.g = gemm_params(c, which, layer, tab);
@@ -946,6 +988,24 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tc_smem) == cudaSuccess;
     if (!ok) (void)cudaGetLastError();
     c->tc_pf = ok;
+    if (ok && getenv("LOOPSPEC_TC_FUSED")) {  // one kernel per GEMM: one CTA per SM, a cluster per row block
+      const int tail = gtc_tail_bytes(), gsb = gtc_stage_bytes(c->tc_cols);
+      c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (200 * 1024 - 1024 - tail) / gsb));
+      c->gtc_smem = (size_t)c->gtc_stages * gsb + 1024 + tail;
+      c->gtc_wmaps.resize((size_t)4 * m->n_recurrent);
+      bool ok2 = true;
+      for (int l = 0; l < m->n_recurrent && ok2; ++l)
+        for (int i = 0; i < 4 && ok2; ++i) ok2 = make_map_bf16(&c->gtc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], 64);
+      for (int i = 0; i < 4; ++i) {
+        const int n_rb = c->plan[i].n_rb, kb = Ks[i] / TC_BK;
+        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb), n_sm / std::max(1, n_rb)));
+      }
+      const void* fns[3] = {(const void*)gemm_tc_kernel<EPI_QKV>, (const void*)gemm_tc_kernel<EPI_RESID>, (const void*)gemm_tc_kernel<EPI_SWIGLU>};
+      for (int i = 0; i < 3 && ok2; ++i)
+        ok2 = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->gtc_smem) == cudaSuccess;
+      if (!ok2) (void)cudaGetLastError();
+      c->tc_fused = ok2;
+    }
   }
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
