@@ -24,9 +24,9 @@ struct GemmTcParams {
 };
 
 __host__ __device__ constexpr int gtc_stage_bytes(int MP) { return TC_BM * TC_BK * 2 + 3 * MP * TC_BK * 2; }
-__host__ __device__ constexpr int gtc_recv_floats() { return (GTC_COLS + 7) * RB_ROWS; }
-__host__ __device__ constexpr int gtc_tail_bytes() {
-  return gtc_recv_floats() * 4 + 2 * RB_ROWS * 4 + GTC_COLS * 4 + CT_FIELDS * GTC_COLS * 4;
+__host__ __device__ constexpr int gtc_recv_floats(int MP) { return (MP + 7) * RB_ROWS; }
+__host__ __device__ constexpr int gtc_tail_bytes(int MP) {
+  return gtc_recv_floats(MP) * 4 + 2 * RB_ROWS * 4 + GTC_COLS * 4 + CT_FIELDS * GTC_COLS * 4;
 }
 
 template <int EPI>
@@ -42,12 +42,12 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cs = p.cluster_size, rank = (int)cluster.block_rank(), rb = blockIdx.x / cs;
-  const int own_max = (GTC_COLS + cs - 1) / cs;
+  const int own_max = (q.MP + cs - 1) / cs;
   const unsigned base = (tc_smem_u32(gtc_smem_raw) + 1023u) & ~1023u;
   const int stage_bytes = gtc_stage_bytes(q.MP);
   unsigned char* tail = gtc_smem_raw + (base - tc_smem_u32(gtc_smem_raw)) + q.stages * stage_bytes;
   float* recv = reinterpret_cast<float*>(tail);                // [cs][own_max][128]
-  float* colbuf = recv + gtc_recv_floats();                    // [2][128]
+  float* colbuf = recv + gtc_recv_floats(q.MP);                    // [2][128]
   float* s_rstd = colbuf + 2 * RB_ROWS;
   int* s_ct = reinterpret_cast<int*>(s_rstd + GTC_COLS);       // [CT_FIELDS][GTC_COLS]
 

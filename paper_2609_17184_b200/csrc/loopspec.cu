@@ -329,7 +329,7 @@ struct loopspec_ctx {
   int tc_cols = 0, tc_stages = 0;
   size_t tc_smem = 0;
   // ... and in one kernel per GEMM (cluster reduction + epilogue inside): weight maps with 64-row boxes
-  bool tc_fused = false;
+  bool tc_fused = false, tc_all = false;
   std::vector<CUtensorMap> gtc_wmaps;
   int gtc_cs[4] = {1, 1, 1, 1}, gtc_stages = 0;
   size_t gtc_smem = 0;
@@ -630,6 +630,7 @@ cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable
 }
 
 cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false) {
+  tc = tc || c->tc_all;
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
@@ -988,9 +989,11 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tc_smem) == cudaSuccess;
     if (!ok) (void)cudaGetLastError();
     c->tc_pf = ok;
-    if (ok && getenv("LOOPSPEC_TC_FUSED")) {  // one kernel per GEMM: one CTA per SM, a cluster per row block
-      const int tail = gtc_tail_bytes(), gsb = gtc_stage_bytes(c->tc_cols);
-      c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (200 * 1024 - 1024 - tail) / gsb));
+    c->tc_all = ok && getenv("LOOPSPEC_TC_ALL") && tc_pf_cols(dd.max_rows) == c->tc_cols;  // experiment: decode passes too
+    if (ok && (getenv("LOOPSPEC_TC_FUSED") || c->tc_all)) {  // one kernel per GEMM, a cluster per row block
+      const int tail = gtc_tail_bytes(c->tc_cols), gsb = gtc_stage_bytes(c->tc_cols);
+      const int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
+      c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (budget * 1024 - 1024 - tail) / gsb));
       c->gtc_smem = (size_t)c->gtc_stages * gsb + 1024 + tail;
       c->gtc_wmaps.resize((size_t)4 * m->n_recurrent);
       bool ok2 = true;
@@ -998,7 +1001,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         for (int i = 0; i < 4 && ok2; ++i) ok2 = make_map_bf16(&c->gtc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], 64);
       for (int i = 0; i < 4; ++i) {
         const int n_rb = c->plan[i].n_rb, kb = Ks[i] / TC_BK;
-        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb), n_sm / std::max(1, n_rb)));
+        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb / 2), (c->tc_all ? 2 * n_sm : n_sm) / std::max(1, n_rb)));
       }
       const void* fns[3] = {(const void*)gemm_tc_kernel<EPI_QKV>, (const void*)gemm_tc_kernel<EPI_RESID>, (const void*)gemm_tc_kernel<EPI_SWIGLU>};
       for (int i = 0; i < 3 && ok2; ++i)

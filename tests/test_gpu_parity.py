@@ -452,15 +452,18 @@ def test_persistent_pass_kernel_matches_oracle(name, T, d2, monkeypatch):
 
 
 @pytest.mark.parametrize("name,T,rows", [("tiny_bf16", 0.0, 64), ("tiny_bf16", 1.0, 16), ("small_bf16", 1.0, 64), ("tiny_gqa", 0.0, 32)])
-@pytest.mark.parametrize("mode", ["two_kernels", "fused", "mma_sync"])
+@pytest.mark.parametrize("mode", ["two_kernels", "fused", "mma_sync", "all_passes_fused"])
 def test_prefill_paths_match_oracle(name, T, rows, mode, monkeypatch):
     """The three ways a prefill pass can run its layer GEMMs: tcgen05 kernel + fused-epilogue kernel (default), one
-    tcgen05 kernel with the cluster reduction and epilogue inside (opt-in), the mma.sync kernels of the decode pass.
+    tcgen05 kernel with the cluster reduction and epilogue inside (opt-in; also for the decode passes in the last mode),
+    the mma.sync kernels of the decode pass.
     Their K splits differ, so each is compared with the oracle, not bit for bit with the others."""
     if mode == "fused":
         monkeypatch.setenv("LOOPSPEC_TC_FUSED", "1")
     if mode == "mma_sync":
         monkeypatch.setenv("LOOPSPEC_NO_TC_PREFILL", "1")
+    if mode == "all_passes_fused":   # experiment: the decode passes on the one-kernel tcgen05 GEMM as well
+        monkeypatch.setenv("LOOPSPEC_TC_ALL", "1")
     ref = U.oracle_run(name, 150, 24, 1, 2, T=T, seed=9)
     ctx = U.make_ctx(name, 1, 2, T=T, seed=9, max_ctx=200, max_prefill_rows=rows)
     assert ctx.prefill(ref["prompt"]) == ref["first"]
