@@ -66,7 +66,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
   int row_a, row_b;
   if (EPI == EPI_SWIGLU) row_a = rb * 64, row_b = p.F + rb * 64;
   else row_a = rb * RB_ROWS, row_b = row_a + 64;
-  const unsigned tmem_cols = q.MP <= 32 ? 32u : 64u;
+  // the three planes of the activations are three groups of MP accumulator columns: one MMA of N = 3 MP per k-step,
+  // three separate chains as in the mma.sync kernels, folded hi + (mid + lo) when the accumulator is read
+  const unsigned tmem_cols = 3 * q.MP <= 64 ? 64u : (3 * q.MP <= 128 ? 128u : 256u);
 
   if (tid == 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<unsigned long long>(&map_w)) : "memory");
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
     if (!ok) *p.err = q.err_code;
   } else if (tid == 0) {
     // ---- MMA issuer ----
-    const unsigned idesc = tc_idesc(TC_BM, q.MP);
+    const unsigned idesc = tc_idesc(TC_BM, 3 * q.MP);
     bool ok = true;
     for (int kb = 0; kb < n_kb && ok; ++kb) {
       const int s = kb % q.stages;
@@ -135,13 +137,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const unsigned a = base + s * stage_bytes, b = a + TC_BM * TC_BK * 2;
       const unsigned long long adesc = tc_smem_desc(a);
+      const unsigned long long bdesc = tc_smem_desc(b);  // rows pl * MP + column: the planes stacked
 #pragma unroll
-      for (int ks = 0; ks < TC_BK / 16; ++ks)
-#pragma unroll
-        for (int pl = 0; pl < 3; ++pl) {
-          const unsigned long long bdesc = tc_smem_desc(b + pl * q.MP * TC_BK * 2);
-          tc_mma(tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, (kb | ks | pl) != 0);
-        }
+      for (int ks = 0; ks < TC_BK / 16; ++ks) tc_mma(tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, (kb | ks) != 0);
       tc_commit(tc_smem_u32(&s_empty[s]));
     }
     if (ok) tc_commit(tc_smem_u32(&s_done));
@@ -167,14 +165,22 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
     for (int c0 = 0; c0 < q.MP; c0 += 16) {
       unsigned v[16];
       if (have) {
-        const unsigned taddr = tmem + ((unsigned)(warp * 32) << 16) + (unsigned)c0;
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-              "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-            : "r"(taddr)
-            : "memory");
+        unsigned w[3][16];
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl) {
+          const unsigned taddr = tmem + ((unsigned)(warp * 32) << 16) + (unsigned)(pl * q.MP + c0);
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+              : "=r"(w[pl][0]), "=r"(w[pl][1]), "=r"(w[pl][2]), "=r"(w[pl][3]), "=r"(w[pl][4]), "=r"(w[pl][5]), "=r"(w[pl][6]),
+                "=r"(w[pl][7]), "=r"(w[pl][8]), "=r"(w[pl][9]), "=r"(w[pl][10]), "=r"(w[pl][11]), "=r"(w[pl][12]),
+                "=r"(w[pl][13]), "=r"(w[pl][14]), "=r"(w[pl][15])
+              : "r"(taddr)
+              : "memory");
+        }
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          v[j] = __float_as_uint(__uint_as_float(w[0][j]) + (__uint_as_float(w[1][j]) + __uint_as_float(w[2][j])));
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = 0u;  // a rank without k-blocks contributes zeros

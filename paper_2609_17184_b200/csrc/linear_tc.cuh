@@ -5,7 +5,8 @@
 // the row-major weights and of the activation planes arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle) in a
 // ring of shared-memory stages guarded by mbarriers; one thread issues tcgen05.mma (128 weight rows x up to 64 token
 // columns, K = 16 per instruction) with the accumulator in tensor memory; four warps read it back with tcgen05.ld.
-// Activations are fp32 split exactly into three bf16 planes, so each k-step issues three MMAs into one accumulator.
+// Activations are fp32 split exactly into three bf16 planes; the planes are stacked as 3 MP columns of one MMA per
+// k-step (three accumulator chains, as in the mma.sync kernels) and folded hi + (mid + lo) when the accumulator is read.
 // K may be split over blockIdx.y; the partial sums are added in split order by a second kernel (no atomics).
 //
 // Used by the stand-alone operator loopspec_op_linear_tc and by the prefill passes (tc_epilogue_kernel then applies the
@@ -108,7 +109,9 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   const int n0 = blockIdx.x * TC_BM;
   const int kb0 = blockIdx.y * p.kb_per_split;
   const int n_kb = min(p.kb_per_split, p.K / TC_BK - kb0);
-  const unsigned tmem_cols = p.MP <= 32 ? 32u : 64u;
+  // the three planes of the activations are three groups of MP accumulator columns: one MMA of N = 3 MP per k-step
+  // (three separate chains, as in the mma.sync kernels), folded hi + (mid + lo) when the accumulator is read
+  const unsigned tmem_cols = 3 * p.MP <= 64 ? 64u : (3 * p.MP <= 128 ? 128u : 256u);
 
   if (tid == 32) {  // the producer fetches the two tensor maps while the barriers are set up
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<unsigned long long>(&map_w)) : "memory");
@@ -172,7 +175,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   }
   if (tid == 0 && n_kb > 0) {
     // ---- MMA issuer: one thread, the accumulator lives in tensor memory ----
-    const unsigned idesc = tc_idesc(TC_BM, p.MP);
+    const unsigned idesc = tc_idesc(TC_BM, 3 * p.MP);
     bool ok = true;
     for (int kb = 0; kb < n_kb && ok; ++kb) {
       const int s = kb % p.stages;
@@ -181,13 +184,9 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const unsigned a = base + s * stage_bytes, b = a + TC_BM * TC_BK * 2;
       const unsigned long long adesc = tc_smem_desc(a);
+      const unsigned long long bdesc = tc_smem_desc(b);  // rows pl * MP + column: the hi, mid, lo planes stacked
 #pragma unroll
-      for (int ks = 0; ks < TC_BK / 16; ++ks)
-#pragma unroll
-        for (int pl = 0; pl < 3; ++pl) {  // hi, mid, lo plane of the activations: rows pl*MP .. of the x tile
-          const unsigned long long bdesc = tc_smem_desc(b + pl * p.MP * TC_BK * 2);
-          tc_mma(tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, (kb | ks | pl) != 0);
-        }
+      for (int ks = 0; ks < TC_BK / 16; ++ks) tc_mma(tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, (kb | ks) != 0);
       tc_commit(tc_smem_u32(&s_empty[s]));  // arrives when the MMAs issued so far have read their operands
     }
     if (ok) tc_commit(tc_smem_u32(&s_done));
@@ -204,15 +203,23 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
       if (n < p.N) out[(size_t)m * p.N + n] = 0.f;
   } else if (have) {
     for (int c0 = 0; c0 < p.MP; c0 += 16) {
-      unsigned v[16];
-      const unsigned taddr = tmem + ((unsigned)(warp * 32) << 16) + (unsigned)c0;
-      asm volatile(
-          "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-            "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-          : "r"(taddr)
-          : "memory");
+      unsigned w[3][16];
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl) {
+        const unsigned taddr = tmem + ((unsigned)(warp * 32) << 16) + (unsigned)(pl * p.MP + c0);
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(w[pl][0]), "=r"(w[pl][1]), "=r"(w[pl][2]), "=r"(w[pl][3]), "=r"(w[pl][4]), "=r"(w[pl][5]), "=r"(w[pl][6]),
+              "=r"(w[pl][7]), "=r"(w[pl][8]), "=r"(w[pl][9]), "=r"(w[pl][10]), "=r"(w[pl][11]), "=r"(w[pl][12]),
+              "=r"(w[pl][13]), "=r"(w[pl][14]), "=r"(w[pl][15])
+            : "r"(taddr)
+            : "memory");
+      }
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      unsigned v[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        v[j] = __float_as_uint(__uint_as_float(w[0][j]) + (__uint_as_float(w[1][j]) + __uint_as_float(w[2][j])));
 #pragma unroll
       for (int j = 0; j < 16; ++j)
         if (c0 + j < p.M && n < p.N) out[(size_t)(c0 + j) * p.N + n] = __uint_as_float(v[j]);

@@ -992,7 +992,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     c->tc_all = ok && getenv("LOOPSPEC_TC_ALL") && tc_pf_cols(dd.max_rows) == c->tc_cols;  // experiment: decode passes too
     if (ok && (getenv("LOOPSPEC_TC_FUSED") || c->tc_all)) {  // one kernel per GEMM, a cluster per row block
       const int tail = gtc_tail_bytes(c->tc_cols), gsb = gtc_stage_bytes(c->tc_cols);
-      const int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
+      int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
+      if (getenv("LOOPSPEC_GTC_KB")) budget = atoi(getenv("LOOPSPEC_GTC_KB"));
+      const int gslots = getenv("LOOPSPEC_GTC_SLOTS") ? atoi(getenv("LOOPSPEC_GTC_SLOTS")) : (c->tc_all ? 2 * n_sm : n_sm);
       c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (budget * 1024 - 1024 - tail) / gsb));
       c->gtc_smem = (size_t)c->gtc_stages * gsb + 1024 + tail;
       c->gtc_wmaps.resize((size_t)4 * m->n_recurrent);
@@ -1001,7 +1003,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
         for (int i = 0; i < 4 && ok2; ++i) ok2 = make_map_bf16(&c->gtc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], 64);
       for (int i = 0; i < 4; ++i) {
         const int n_rb = c->plan[i].n_rb, kb = Ks[i] / TC_BK;
-        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb / 2), (c->tc_all ? 2 * n_sm : n_sm) / std::max(1, n_rb)));
+        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb / 2), gslots / std::max(1, n_rb)));
       }
       const void* fns[3] = {(const void*)gemm_tc_kernel<EPI_QKV>, (const void*)gemm_tc_kernel<EPI_RESID>, (const void*)gemm_tc_kernel<EPI_SWIGLU>};
       for (int i = 0; i < 3 && ok2; ++i)
