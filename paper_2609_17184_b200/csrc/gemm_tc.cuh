@@ -145,6 +145,20 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
     if (ok) tc_commit(tc_smem_u32(&s_done));
     else *p.err = q.err_code;
   }
+  // operands of this CTA's first output column, requested ahead of the accumulator (as the mma.sync kernels do)
+  float pre_h = 0.f, pre_g = 1.f;
+  float2 pre_rope = make_float2(1.f, 0.f);
+  {
+    const int c = rank + cs * (tid >> 7), jr = tid & 127;
+    if (EPI == EPI_RESID && c < n_cols) {
+      pre_h = p.hid[(size_t)s_ct[CT_HID * GTC_COLS + c] * p.H + rb * RB_ROWS + jr];
+      if (p.out_planes) pre_g = p.gain_next[rb * RB_ROWS + jr];
+    }
+    if (EPI == EPI_QKV && c < n_cols && jr < 64) {
+      const int hd2 = p.head_dim >> 1;
+      pre_rope = p.rope[(size_t)s_ct[CT_POS * GTC_COLS + c] * hd2 + jr % hd2];
+    }
+  }
   // 1/rms of the columns this rank finishes (gemm_rstd's arithmetic), by the warps that do not read the accumulator
   if (warp >= 4) {
     for (int c = rank + cs * (warp - 4); c < n_cols; c += cs * 4) {
@@ -199,7 +213,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_tc_kernel(const __grid_cons
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   cluster.sync();
-  gemm_reduce_epilogue<EPI>(p, s_ct, GTC_COLS, rb, n_cols, recv, own_max, colbuf, s_rstd, rank);
+  gemm_reduce_epilogue<EPI>(p, s_ct, GTC_COLS, rb, n_cols, recv, own_max, colbuf, s_rstd, rank, pre_h, pre_g, pre_rope,
+                            EPI == EPI_RESID || EPI == EPI_QKV);
   __syncthreads();
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
 }

@@ -992,9 +992,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     c->tc_all = ok && getenv("LOOPSPEC_TC_ALL") && tc_pf_cols(dd.max_rows) == c->tc_cols;  // experiment: decode passes too
     if (ok && (getenv("LOOPSPEC_TC_FUSED") || c->tc_all)) {  // one kernel per GEMM, a cluster per row block
       const int tail = gtc_tail_bytes(c->tc_cols), gsb = gtc_stage_bytes(c->tc_cols);
-      int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
-      if (getenv("LOOPSPEC_GTC_KB")) budget = atoi(getenv("LOOPSPEC_GTC_KB"));
-      const int gslots = getenv("LOOPSPEC_GTC_SLOTS") ? atoi(getenv("LOOPSPEC_GTC_SLOTS")) : (c->tc_all ? 2 * n_sm : n_sm);
+      const int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
+      const int gslots = c->tc_all ? 2 * n_sm : n_sm;
       c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (budget * 1024 - 1024 - tail) / gsb));
       c->gtc_smem = (size_t)c->gtc_stages * gsb + 1024 + tail;
       c->gtc_wmaps.resize((size_t)4 * m->n_recurrent);
