@@ -306,6 +306,23 @@ def run_ours(args):
     for which, nm in enumerate(["qkv", "o_proj", "gate_up", "down", "lm_head"]):
         ms_k, b_k = ctx.time_kernel(which, min(rows_typ, 8), 240 if which < 4 else 40)
         per_kernel[nm] = {"us": round(ms_k * 1e3, 2), "GBps": round(b_k / (ms_k / 1e3) / 1e9, 1)}
+    # the same GEMM shapes on the tcgen05 / TMA kernel (used by the prefill passes; not by the decode passes that
+    # `value` times), alone and back to back over several weight matrices: reported beside, never instead of, the above
+    tc_alone = None
+    if shape.weight_dtype == "bf16" and rank == 0:
+        try:
+            tc_alone = {}
+            hq, hkv = shape.n_q_heads * shape.head_dim, shape.n_kv_heads * shape.head_dim
+            for nm, (N_, K_) in {"gate_up": (2 * shape.ffn, shape.hidden), "down": (shape.hidden, shape.ffn),
+                                 "qkv": (hq + 2 * hkv, shape.hidden), "lm_head": (shape.vocab, shape.hidden)}.items():
+                n_w = max(3, min(12, int(300e6 // (N_ * K_ * 2)) + 1))
+                Ws_ = [torch.randn(N_, K_, device="cuda").mul_(0.02).to(torch.bfloat16) for _ in range(n_w)]
+                us_ = ls.time_linear_tc(Ws_, torch.randn(min(rows_typ, 8), K_, device="cuda"), iters=10)
+                tc_alone[nm] = {"us": round(us_, 2), "GBps": round(N_ * K_ * 2 / us_ / 1e3, 1),
+                                "frac": round(N_ * K_ * 2 / us_ / 1e3 / peak, 4)}
+                del Ws_
+        except Exception as e:  # a reporting extra: never fails the bench
+            tc_alone = {"error": str(e)[:200]}
     total_b, w_b, w_c, kv_row = step_bytes(shape, n_prompt, n_decode, stats)
     step_gbs = total_b / (statistics.mean(dec_ms) / 1e3) / 1e9
     van_gbs = vanilla_bytes(shape, n_prompt, n_decode) / (statistics.mean(van_ms) / 1e3) / 1e9
@@ -328,6 +345,7 @@ def run_ours(args):
                      "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(wl.model),
                      "algorithmic_bytes_per_launch": k_bytes, "us_per_launch": round(k_ms * 1e3, 2), "rows": min(rows_typ, 8)},
         "kernels_alone": per_kernel,
+        "tcgen05_kernels_alone": tc_alone,
         "step_roofline": {"achieved": round(step_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(step_gbs / peak, 4),
                           "ms_per_pass": round(statistics.mean(dec_ms) / max(stats["steps"], 1), 4),
                           "bytes_per_pass": int(total_b / max(stats["steps"], 1))},
