@@ -3,7 +3,7 @@
 
 Metric: decode tokens/s at batch 1 on the Ouro-1.4B-shaped model (24 shared layers looped R=4, bf16),
 prompt 512, 512 greedy tokens, (d1, d2) = (1, 2) with the gate -- measured over the decode phase only,
-after prefill, as the paper does (Sec. 5 "Implementation and Metrics").  A bench "step" is one whole
+after prefill, as the paper does (Sec. 6 "Implementation and Metrics").  A bench "step" is one whole
 decode job (512 committed tokens) on a freshly prefilled sequence.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]

@@ -1,7 +1,7 @@
 /*
  * loopspec.h -- C ABI of the LoopSpec pipelined decode path for looped transformers on B200 (sm_100a).
  *
- * The library runs the decode loop of Algorithm 1 (App. G) of "LoopSpec: Pipelined Self-Speculative
+ * The library runs the decode loop of Algorithm 1 (App. H) of "LoopSpec: Pipelined Self-Speculative
  * Decoding for Looped Transformers": in every step all active branches -- the token being verified at
  * recurrent depth R, first-proposal drafts spawned at depth d1 and, when the gate of Eq. 6 opens,
  * residual second proposals spawned at depth d2 (Eq. 5) -- go through the shared block stack in ONE
@@ -37,7 +37,7 @@ typedef enum {
   LOOPSPEC_ESTATE = -2,       /* call out of order (step before prefill, verify with nothing at depth R, ...) */
   LOOPSPEC_ECAPACITY = -3,    /* max_ctx, max_seqs, node table or workspace too small */
   LOOPSPEC_ECUDA = -4,        /* a CUDA call failed; see loopspec_last_error */
-  LOOPSPEC_ETIMEOUT = -5,     /* reserved: a bounded device-side wait ran out */
+  LOOPSPEC_ETIMEOUT = -5,     /* a bounded device-side wait (mbarrier, grid barrier) ran out; the pass's results are void */
   LOOPSPEC_EUNSUPPORTED = -6  /* shape outside what the kernels support */
 } loopspec_status;
 
@@ -68,7 +68,7 @@ typedef struct {
  * measure_tv = 1 (sampling only): every verification also records TV(p_d1, p_R) and, where a second-proposal record
  * exists, TV(p_d2, p_R) of the readouts involved (Sec. 4.1's empirical profile; see loopspec_stats and
  * loopspec_fit_envelope).  With the gate on, the depth-d2 readout exists only where the gate opened.
- * mask_first = 1: the variant of the paper's second-proposal ablation (Sec. 5): the first candidate is removed from the
+ * mask_first = 1: the variant of the paper's second-proposal ablation (Sec. 6): the first candidate is removed from the
  * second proposal's distribution (the residual one if it has mass elsewhere, else p_{d2}) and the rest renormalised, so
  * the two candidates always differ; a branch whose p_{d2} has all its mass on the first candidate gets no second
  * proposal.  Under greedy decoding the second candidate is then the best token other than the first. */
@@ -97,14 +97,14 @@ typedef struct {
   const void* const* layer_ptrs;
 } loopspec_weights;
 
-/* One committed token (Algorithm 1, main loop: "commit a new decoded token"). source: 1 = accepted first
+/* One committed token (Algorithm 1, main loop, the commit after Verify). source: 1 = accepted first
  * proposal, 2 = accepted second proposal, 3 = resampled at depth R (restart). step = index (from 1) of the
  * batched pass after which it was committed. */
 typedef struct {
   int32_t seq, n_committed, token, source, accepted1, accepted2, gate_open, step;
 } loopspec_commit;
 
-/* Counters of Sec. 5 (gamma), App. C (gate openings, effective batch size) and App. D (commit sources).
+/* Counters of Sec. 6 (gamma), App. D (gate openings, effective batch size) and App. E (commit sources).
  * tv_d1 / tv_d2: mean total-variation distance between the depth-d1 / depth-d2 readout and the target over the
  * tv_n1 / tv_n2 verifications that had one (0 unless the scheduler was created with measure_tv). */
 typedef struct {
@@ -154,7 +154,7 @@ int loopspec_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
 int loopspec_vanilla_decode(loopspec_ctx*, int32_t n_tokens, int32_t* ids_out);
 
 /* Power-law envelope phi(r) = beta r^-alpha over a measured total-variation profile tv[r-1] = TV(p_r, p_R),
- * r = 1..n (Sec. 4.1: "minimize the maximum ratio between phi(r) and the empirical TV over all depths"), read as:
+ * r = 1..n (Sec. 4.1, the min-max-ratio fit of the envelope), read as:
  * minimise max_r phi(r) / tv[r-1] subject to phi(r) >= tv[r-1] for every r, alpha > 0.  The pair feeds
  * loopspec_pick_depths.  Host only.  tv: host array of n >= 2 positive values that decreases somewhere;
  * EINVAL otherwise. */

@@ -14,6 +14,7 @@ Parity status of what lives here:
   * Philox4x32-10                    : pinned (published known-answer vectors)
   * closed-form depths, branch bound : pinned (values printed in the paper)
   * scheduler (Algorithm 1)          : pinned (losslessness, commit-gap schedule)
+  * gamma, TV profile log            : pinned (hand values on scripted timelines / hand-made distributions)
   * sampled token streams / gamma on the large shapes: parity unpinned by the
     paper (it prints no token-level example); fixed only by the checks above.
 """

@@ -1,4 +1,4 @@
-"""Vanilla decoding and LoopSpec (Algorithm 1, App. G; Sec. 4.2-4.3), float64, one sequence.
+"""Vanilla decoding and LoopSpec (Algorithm 1, App. H; Sec. 4.2-4.3), float64, one sequence.
 
 `Decoder` holds the committed prefix and its depth-indexed KV.  `vanilla` finishes all R
 recurrences of a token before the next (Fig. 1a).  `loopspec` follows Algorithm 1 in its
@@ -250,7 +250,7 @@ class Decoder:
                             # residual of two one-hot distributions: the deeper argmax; without the
                             # gate the two may coincide and the residual falls back to q2~ itself
                             x2 = top
-                            if mask_first and top == x1:   # second-proposal ablation (Sec. 5): the first candidate is masked out
+                            if mask_first and top == x1:   # second-proposal ablation (Sec. 6): the first candidate is masked out
                                 x2, margin = self._argmax(np.where(np.arange(len(z2)) == x1, -np.inf, z2))
                                 self.log.append(dict(kind="draft2", pos=pos, token=x2, margin=margin))
                             self.stats["gate_opens"] += 1
@@ -264,7 +264,7 @@ class Decoder:
                             gm = abs(np.log(q2t[x1]) - np.log(q1[x1]))
                         self.log.append(dict(kind="gate", pos=pos, open=is_open, margin=gm))
                         if is_open and mask_first:
-                            # second-proposal ablation (Sec. 5): the first candidate is masked out of the proposal
+                            # second-proposal ablation (Sec. 6): the first candidate is masked out of the proposal
                             q2 = sp.masked_second_proposal(q2t, q1, x1, residual_q2)
                             is_open = q2 is not None      # q2~ puts all its mass on the first candidate: no proposal
                         elif is_open:

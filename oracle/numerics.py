@@ -54,12 +54,6 @@ def softmax(z, axis=-1):
     return e / np.sum(e, axis=axis, keepdims=True)
 
 
-def log_softmax(z, axis=-1):
-    m = np.max(z, axis=axis, keepdims=True)
-    s = z - m
-    return s - np.log(np.sum(np.exp(s), axis=axis, keepdims=True))
-
-
 def attend(q, K, V):
     """One query against its keys.  q [n_q_heads, d]; K, V [ctx, n_kv_heads, d].
 

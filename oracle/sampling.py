@@ -96,7 +96,7 @@ def residual(mu, nu):
 
 
 def masked_second_proposal(q2t, q1, x1, residual_q2=True):
-    """Second proposal with the first candidate x1 masked out (the variant of the second-proposal ablation, Sec. 5):
+    """Second proposal with the first candidate x1 masked out (the variant of the second-proposal ablation, Sec. 6):
     x1's mass is removed from the residual proposal norm([q2~ - q1]_+) if that leaves mass elsewhere (or if
     residual_q2 is off, from q2~ directly), else from q2~, and the rest renormalised.  None when q2~ has all its mass
     on x1: there is nothing else to propose."""

@@ -84,7 +84,7 @@ struct SeqState {
   int* need_verify;  // set by the step phase when the root reached R
 };
 
-struct Counters {  // App. C / App. D statistics
+struct Counters {  // App. D / App. E statistics
   unsigned long long steps, n_decode, n_accept1, n_accept2, n_restart, gate_evals, gate_opens, rows_total, rows_max,
       readout_rows_total;
 };

@@ -102,6 +102,9 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
     for (int n = 0; n < p.NB; ++n) {
       if (!nd.state[o + n]) continue;
       if (n_rows >= MAX_ROWS) { *err = ERR_NODES; break; }
+      // a position outside the KV pool is never scheduled (the host refuses such a decode before it starts; this is
+      // the second line of defence): the branch stays where it is and the flag tells the host
+      if (nd.pos[o + n] + 2 >= p.ctx_cap) { *err = ERR_CTX; continue; }
       const int i = n_rows++;
       const int r = nd.depth[o + n] + 1;
       const bool is_root = nd.parent[o + n] < 0;
@@ -109,7 +112,6 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       t.kv_slot[i] = is_root ? nd.pos[o + n] : p.ctx_cap + n;
       t.n_canon[i] = nd.pos[o + rt] + 1;
       t.n_safe[i] = is_root ? nd.pos[o + n] : t.n_canon[i];
-      if (nd.pos[o + n] + 2 >= p.ctx_cap) *err = ERR_CTX;
       int chain[MAX_SPEC], len = 0;
       for (int a = n; a >= 0 && nd.parent[o + a] >= 0; a = nd.parent[o + a]) {
         if (len >= MAX_SPEC) { *err = ERR_SPEC; break; }
@@ -312,6 +314,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
         int row = -1;
         for (int i = 0; i < cur.n_rows; ++i)
           if (cur.seq[i] == s) row = i;
+        if (row < 0) continue;  // the sequence had no row in the last pass (dropped at the capacity limit)
         int tok = p.sel_tok[row];
         int k = p.seqs.n_dec[s];
         if (k < p.ids_cap) p.out_ids[(size_t)s * p.ids_cap + k] = tok;
@@ -323,7 +326,10 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
       }
       p.nodes.depth[o + rt] = 0, p.nodes.child1[o + rt] = p.nodes.child2[o + rt] = -1, p.nodes.has2[o + rt] = 0;
       p.seqs.need_verify[s] = 0;
-      if (p.nodes.pos[o + rt] + 2 >= p.ctx_cap) p.host_flags[HF_ERROR] = ERR_CTX;
+      if (p.nodes.pos[o + rt] + 2 >= p.ctx_cap) {  // never schedule a position outside the KV pool
+        p.host_flags[HF_ERROR] = ERR_CTX;
+        continue;
+      }
       s_emb[n][0] = o + rt, s_emb[n][1] = p.nodes.token[o + rt];
       s_rowof[n] = s;
       ++n;

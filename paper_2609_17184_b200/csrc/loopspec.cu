@@ -1187,17 +1187,21 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
 
 // set every prefilled sequence's target to n more tokens and (re)build the decode rows
 static int arm_decode(loopspec_ctx* c, int n_tokens, bool unlimited = false) {
-  std::vector<int> ndec(MAX_ROWS), tgt(MAX_ROWS, 0);
+  std::vector<int> ndec(MAX_ROWS), nids(MAX_ROWS), tgt(MAX_ROWS, 0);
   CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
+  // Positions a sequence can reach: its committed ids, the tokens asked for (a manual step commits at most one) and
+  // the deepest chain of uncommitted drafts, R/d1; the scheduler wants two more below max_ctx.  Checked here, before
+  // anything is launched, so that no pass ever carries a row whose position lies outside the KV pool.
+  const int spec_depth = c->m.R / c->d.d1;
   for (int s = 0; s < c->d.S; ++s) {
     if (!c->prefilled[s]) continue;
-    if (unlimited) {
-      tgt[s] = c->d.ids_cap;
-      continue;
-    }
-    if ((long long)ndec[s] + n_tokens > c->d.ids_cap) return fail(c, LOOPSPEC_ECAPACITY, "decode would exceed max_ctx");
-    tgt[s] = ndec[s] + n_tokens;
+    const long long want = unlimited ? 1 : n_tokens;
+    if ((long long)nids[s] + want + spec_depth + 2 > c->s.max_ctx || (long long)ndec[s] + want > c->d.ids_cap)
+      return fail(c, LOOPSPEC_ECAPACITY, "sequence %d: %d committed ids + %lld more + %d speculative + 2 exceed max_ctx %d", s, nids[s],
+                  want, spec_depth, c->s.max_ctx);
+    tgt[s] = unlimited ? c->d.ids_cap : ndec[s] + n_tokens;
   }
   memcpy(c->pin_ids, tgt.data(), MAX_ROWS * 4);
   CU(c, cudaMemcpyAsync(c->seqs().n_target, c->pin_ids, MAX_ROWS * 4, cudaMemcpyHostToDevice, c->stream));
@@ -1301,11 +1305,13 @@ int loopspec_vanilla_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out)
   if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
   if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "decode before prefill");
   if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
-  std::vector<int> start(MAX_ROWS);
+  std::vector<int> start(MAX_ROWS), nids(MAX_ROWS);
   CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
-  for (int s = 0; s < c->d.S; ++s)
-    if (c->prefilled[s] && (long long)start[s] + n_tokens > c->d.ids_cap) return fail(c, LOOPSPEC_ECAPACITY, "decode would exceed max_ctx");
+  for (int s = 0; s < c->d.S; ++s)  // no drafts here: the last position is committed ids + n_tokens - 1, two more must fit
+    if (c->prefilled[s] && ((long long)nids[s] + n_tokens + 2 > c->s.max_ctx || (long long)start[s] + n_tokens > c->d.ids_cap))
+      return fail(c, LOOPSPEC_ECAPACITY, "sequence %d: %d committed ids + %d more + 2 exceed max_ctx %d", s, nids[s], n_tokens, c->s.max_ctx);
   vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 0));
   CU(c, cudaGetLastError());
   c->vanilla_mode = true;
@@ -1326,7 +1332,7 @@ int loopspec_get_stats(loopspec_ctx* c, loopspec_stats* out) {
   out->n_restart = k.n_restart, out->gate_evals = k.gate_evals, out->gate_opens = k.gate_opens;
   out->rows_total = k.rows_total, out->rows_max = k.rows_max, out->readout_rows_total = k.readout_rows_total;
   double den = (double)k.n_accept1 * c->d.d1 + (double)k.n_accept2 * c->d.d2 + (double)k.n_restart * c->m.R;
-  out->gamma = den > 0 ? (double)k.n_decode * c->m.R / den : 0.0;  // Sec. 5, definition of gamma
+  out->gamma = den > 0 ? (double)k.n_decode * c->m.R / den : 0.0;  // Sec. 6 "Implementation and Metrics", definition of gamma
   double tv[MAX_ROWS * 4];
   CU(c, cudaMemcpy(tv, c->ws + c->L.tv, sizeof tv, cudaMemcpyDeviceToHost));
   double s1 = 0, n1 = 0, s2 = 0, n2 = 0;

@@ -66,6 +66,16 @@ def assert_same_run(ctx, ref, n_decode, seq=0, logit_atol=3e-2, logit_rtol=2e-2)
     zo = dec.verify_logits[-1]
     err = np.abs(z - zo)
     assert (err <= logit_atol + logit_rtol * np.abs(zo)).all(), err.max()
+    # the proposal records Q_b of the surviving root branch: its depth-d1 and depth-d2 readouts, as stored for the
+    # cascade verification still to come (Algorithm 1, Spawn / Verify), against the oracle's at the same tolerance
+    root = next((b for b in getattr(dec, "active", []) if b.parent is None), None)
+    if root is not None:
+        for which, zq in ((1, root.q1_logits), (2, root.q2_logits)):
+            if zq is None:
+                continue
+            eq = np.abs(ctx.debug_logits(seq, which) - zq)
+            assert (eq <= logit_atol + logit_rtol * np.abs(zq)).all(), (which, eq.max())
+            err = np.maximum(err, eq)
     return err.max()
 
 

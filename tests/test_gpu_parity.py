@@ -1,7 +1,7 @@
 """GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same seeded inputs.
 
 Bar: token ids, accept/reject decisions, commit sources, gate bits, commit steps, per-step row counts and the
-App. C/D counters bit-exact; logits within max-abs 3e-2 + 2e-2 relative (the stated bf16 bound) -- and, because
+App. D/E counters bit-exact; logits within max-abs 3e-2 + 2e-2 relative (the stated bf16 bound) -- and, because
 the kernels keep activations fp32-faithful, within 2e-3 absolute in practice, which is also asserted.
 """
 import numpy as np
@@ -199,7 +199,7 @@ MASKED_CASES = [
 
 @pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,gate,residual,top_k,top_p", MASKED_CASES)
 def test_masked_second_proposal_matches_oracle(name, n_prompt, n_decode, d1, d2, T, gate, residual, top_k, top_p):
-    """The variant of the second-proposal ablation (Sec. 5): the first candidate is masked out of the second
+    """The variant of the second-proposal ablation (Sec. 6): the first candidate is masked out of the second
     proposal; draws, decisions and tokens as the oracle's."""
     kw = dict(T=T, seed=4, gate=gate, residual_q2=residual, top_k=top_k, top_p=top_p, mask_first=True)
     ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, **kw)
@@ -413,8 +413,19 @@ def test_error_paths_leave_the_context_usable():
     with pytest.raises(ls.LoopSpecError) as e:
         ctx.decode(1000)
     assert e.value.status == "ECAPACITY"
+    # fewer tokens than max_ctx, but prompt + tokens + the speculative chain would leave the KV pool: refused on the
+    # host, before any pass is launched (17 committed ids + 50 + R/d1 + 2 > 64), and nothing has been disturbed
+    for call in (lambda: ctx.decode(50), lambda: ctx.vanilla_decode(50)):
+        with pytest.raises(ls.LoopSpecError) as e:
+            call()
+        assert e.value.status == "ECAPACITY"
+    assert ctx.stats()["steps"] == 0
     ref = U.oracle_run("tiny_bf16", 16, 8, 1, 2)
     assert ctx.decode(8)[0].tolist() == ref["tokens"]
+    assert ctx.decode(64 - 17 - 8 - 4 - 2).shape[1] == 33       # exactly up to the limit is accepted
+    with pytest.raises(ls.LoopSpecError) as e:
+        ctx.decode(1)
+    assert e.value.status == "ECAPACITY"
     with pytest.raises(ls.LoopSpecError) as e:
         U.make_ctx("tiny_bf16", 3, 0)
     assert e.value.status == "EINVAL"

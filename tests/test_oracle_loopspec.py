@@ -135,7 +135,7 @@ def test_sampled_loopspec_matches_vanilla_in_distribution(models):
 
 
 def test_masked_second_proposal_keeps_greedy_lossless_and_candidates_distinct(models):
-    """Second-proposal ablation (Sec. 5): with the first candidate masked out and the gate off, every branch gets a
+    """Second-proposal ablation (Sec. 6): with the first candidate masked out and the gate off, every branch gets a
     second candidate different from the first; greedy output still equals vanilla, and more tokens are accepted
     from second proposals than without the mask."""
     shape, model = models["tiny_untied"]
@@ -252,6 +252,10 @@ def test_timeline_single_proposal_R4_d1_1():
     assert [c["step"] for c in dec.commits] == [4, 5, 6, 10]
     assert [c["source"] for c in dec.commits] == [1, 1, 3, 1]
     assert dec.rows_per_step == [1, 2, 3, 4, 4, 4, 1, 2, 3, 4]
+    # gamma by hand (Sec. 6 "Implementation and Metrics"): 4 tokens x R = 16 recurrences' worth of output over
+    # 3 first-proposal commits x d1 = 3 plus one restart x R = 4
+    assert dec.stats["gamma"] == pytest.approx(16 / 7, abs=1e-15)
+    assert (dec.stats["n_accept1"], dec.stats["n_accept2"], dec.stats["n_restart"]) == (3, 0, 1)
 
 
 def test_timeline_second_proposal_saves_d2_steps():
@@ -262,10 +266,53 @@ def test_timeline_second_proposal_saves_d2_steps():
     assert [c["source"] for c in dec.commits] == [1, 1, 2, 1, 1]
     assert [c["step"] for c in dec.commits] == [4, 5, 6, 8, 9]
     assert [c["gate_open"] for c in dec.commits] == [0, 0, 1, 0, 0]
+    # gamma by hand: 5 x 4 over 4 x d1 + 1 x d2 = 6; a second-proposal commit costs d2, not R (a formula with d2 and R
+    # exchanged would give 20 / 8 here)
+    assert dec.stats["gamma"] == pytest.approx(20 / 6, abs=1e-15)
     # both candidates wrong: restart, next commit R steps later
     dec = run_scripted(ScriptedModel(bad_first={2}), 4, 1, 2)
     assert [c["source"] for c in dec.commits] == [1, 1, 3, 1]
     assert [c["step"] for c in dec.commits] == [4, 5, 6, 10]
+    assert dec.stats["gamma"] == pytest.approx(16 / 7, abs=1e-15)
+    # R = 8 with (2, 4): every first draft right -> gamma = R / d1 = 4; the depth pair enters only through the costs
+    class Deep(ScriptedModel):
+        class s(ScriptedModel.s):
+            R = 8
+
+        def logits(self, x):
+            t, depth = int(x[0]), int(x[1])
+            z = np.zeros(self.V)
+            wrong = t in self.bad_first and (depth == 2 or (depth == 4 and t not in self.good_second))
+            z[(t + (30 if wrong else 1)) % self.V] = 1.0
+            return z
+    dec = run_scripted(Deep(bad_first={1, 3}, good_second={3}), 6, 2, 4)
+    assert [c["source"] for c in dec.commits] == [1, 3, 1, 2, 1, 1]
+    assert [c["step"] for c in dec.commits] == [8, 10, 18, 20, 24, 26]
+    assert dec.stats["gamma"] == pytest.approx(6 * 8 / (4 * 2 + 1 * 4 + 1 * 8), abs=1e-15)
+
+
+def test_tv_profile_of_a_verification_by_hand():
+    """Sec. 4.1's empirical profile as logged at a verification: TV(p_d1, p_R) and TV(p_d2, p_R) for hand-made
+    three-token distributions (0.5 x the L1 distance: 0.3 and 0.1)."""
+    from oracle.loopspec import Branch, Record
+    dec = Decoder(model=None, temperature=1.0, seed=4)
+    p = np.array([0.5, 0.3, 0.2])
+    q1 = np.array([0.2, 0.3, 0.5])
+    q2t = np.array([0.4, 0.4, 0.2])
+    b = Branch(parent=None, token=0, pos=5, H=None)
+    b.records = [Record(2, q1, None), Record(0, q2t, None)]
+    b.q2_logits = np.log(q2t) + 0.7          # any shift: C normalises
+    tok, child, source = dec._verify(b, np.log(p) - 1.3)
+    assert len(dec.tv_log) == 1
+    tv1, tv2 = dec.tv_log[0]
+    assert tv1 == pytest.approx(0.3, abs=1e-12) and tv2 == pytest.approx(0.1, abs=1e-12)
+    # without a second record only the first distance is logged; under greedy decoding nothing is
+    b.records = b.records[:1]
+    dec._verify(b, np.log(p))
+    assert dec.tv_log[1][0] == pytest.approx(0.3, abs=1e-12) and dec.tv_log[1][1] is None
+    g = Decoder(model=None, temperature=0.0)
+    g._verify(b, np.log(p))
+    assert g.tv_log == []
 
 
 def test_branch_census_reaches_the_bound_with_the_gate_forced_open():

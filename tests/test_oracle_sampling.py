@@ -1,4 +1,4 @@
-"""Pins for the random draws and the rejection rule (Sec. 3.2 Eq. 2-4; Sec. 4.3; Thm 1; App. F)."""
+"""Pins for the random draws and the rejection rule (Sec. 3.2 Eq. 2-4; Sec. 4.3; Thm 1; App. G)."""
 import itertools
 
 import numpy as np
@@ -97,7 +97,7 @@ def test_cascade_is_lossless_by_enumeration(V, gate, residual_q2):
 
 
 def test_masked_second_proposal_definition_and_losslessness():
-    """Second-proposal ablation (Sec. 5): masking the first candidate gives a distribution with no mass on it, in
+    """Second-proposal ablation (Sec. 6): masking the first candidate gives a distribution with no mass on it, in
     proportion to the unmasked proposal elsewhere; verification stays exact for it (any proposal is admissible)."""
     rng = np.random.default_rng(21)
     for V in (3, 6):
@@ -133,7 +133,7 @@ def test_acceptance_probability_is_one_minus_tv_and_theorem_1_bounds():
         _, rej1, rej_both_gated = cascade_law(p, q1, q2t, gate=True)
         _, _, rej_both_open = cascade_law(p, q1, q2t, gate=False)
         eps2 = tv(q2t, p)
-        assert abs((1 - rej1) - (1 - tv(q1, p))) < 1e-12           # Pr[accept] = 1 - TV (App. F)
+        assert abs((1 - rej1) - (1 - tv(q1, p))) < 1e-12           # Pr[accept] = 1 - TV (App. G)
         assert rej_both_open <= eps2 + 1e-12                        # Thm 1, no gate
         assert rej_both_gated <= 2 * eps2 + 1e-12                   # Thm 1, with gate
 

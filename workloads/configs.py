@@ -1,7 +1,7 @@
 """Model shapes and workloads of the synthetic stand-ins for the paper's models.
 
 The paper evaluates Ouro (R=4) and Raven (R=32) checkpoints on public
-benchmarks (Sec. 5, App. A); neither the checkpoints nor the datasets are
+benchmarks (Sec. 6, App. A); neither the checkpoints nor the datasets are
 available offline, so random weights of the same shapes and uniform-random
 prompts of the same lengths stand in for them.
 """
@@ -91,7 +91,7 @@ WORKLOADS = {
     "tiny": Workload("tiny", "tiny", prompt_len=16, decode_len=64, temperature=0.0, d1=1, d2=0),
     "ouro_1p4b": Workload("ouro_1p4b", "ouro_1p4b", prompt_len=512, decode_len=512, temperature=0.0, d1=1, d2=2),
     "ouro_2p6b": Workload("ouro_2p6b", "ouro_2p6b", prompt_len=1024, decode_len=1024, temperature=1.0, d1=1, d2=2),
-    # the paper's sampling setting for its reasoning models (Sec. 5.1: T = 1.0, top-p 0.7) on the headline shape
+    # the paper's sampling setting for its reasoning models (Sec. 6 "Models and Evaluations": T = 1.0, top-p 0.7) on the headline shape
     "ouro_1p4b_top_p": Workload("ouro_1p4b_top_p", "ouro_1p4b", prompt_len=512, decode_len=512, temperature=1.0, d1=1,
                                 d2=2, top_p=0.7),
     "kv_bound": Workload("kv_bound", "ouro_1p4b", prompt_len=8192, decode_len=256, temperature=0.7, d1=1, d2=2,
