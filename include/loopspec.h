@@ -84,6 +84,8 @@ typedef struct {
   float top_p;
   int32_t measure_tv;
   int32_t mask_first;
+  int32_t prefill_skinny; /* 1: the prefill passes run the layer GEMMs on the kernels of the decode passes instead of the
+                             wide tcgen05 kernels (slower; for comparing the two paths) */
 } loopspec_sched;
 
 /* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:
@@ -177,6 +179,16 @@ int loopspec_get_row_trace(loopspec_ctx*, int32_t* out, int32_t max_out, int32_t
 /* Copy fp32 logits (before temperature) to host out_V[vocab]: which = 0 the last verified target p_R
  * (or the prefill / vanilla readout), 1 / 2 the root branch's stored first / second proposal readout. */
 int loopspec_debug_logits(loopspec_ctx*, int32_t seq, int32_t which, float* out_V);
+
+/* Failure injection on the host side of the bounded device waits (App. B describes no failure handling; this serves the
+ * library's own tests).  Every wait inside the tcgen05 kernels (an mbarrier a TMA copy completes, a stage the tensor
+ * core releases, a cluster partner's partial sums) is bounded by the clock; when one runs out the kernel raises a flag,
+ * carries on with whatever data it has so that every barrier still receives its arrivals, and ends; the call that
+ * launched it returns LOOPSPEC_ETIMEOUT, the results of that pass are void, the context stays usable (prefill the
+ * sequence again).  This call makes such a wait run out: from now on CTA 0 of the readout GEMM never requests ring unit
+ * `unit` (unit >= 0), so the wait for it gives up after about wait_us microseconds.  unit = -1 restores normal operation
+ * (and the normal bound of ~0.2 s).  Nothing faults or hangs: the skipped copy is simply never issued. */
+int loopspec_debug_drop_tile(loopspec_ctx*, int32_t unit, int32_t wait_us);
 
 /* Number of kernels one decode step (one graph replay of loopspec_decode) launches. */
 int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);

@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libloopspec.so")
 EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loopspec_step", "loopspec_verify",
            "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_fit_envelope", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
-           "loopspec_launches_per_step", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
+           "loopspec_launches_per_step", "loopspec_debug_drop_tile", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
            "loopspec_op_linear_static", "loopspec_linear_tc_scratch_bytes", "loopspec_op_linear_tc", "loopspec_time_linear_tc",
            "loopspec_last_error", "loopspec_destroy"]
 
@@ -36,7 +36,7 @@ class Sched(C.Structure):
     _fields_ = [("d1", C.c_int32), ("d2", C.c_int32), ("alpha", C.c_float), ("beta", C.c_float), ("gate", C.c_int32),
                 ("residual_q2", C.c_int32), ("temperature", C.c_float), ("seed", C.c_uint64), ("max_seqs", C.c_int32),
                 ("max_ctx", C.c_int32), ("max_prefill_rows", C.c_int32), ("top_k", C.c_int32), ("top_p", C.c_float),
-                ("measure_tv", C.c_int32), ("mask_first", C.c_int32)]
+                ("measure_tv", C.c_int32), ("mask_first", C.c_int32), ("prefill_skinny", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -81,6 +81,7 @@ def _load():
     lib.loopspec_get_row_trace.argtypes = [V, P(I), I, P(I)]
     lib.loopspec_debug_logits.argtypes = [V, I, I, P(C.c_float)]
     lib.loopspec_launches_per_step.argtypes = [V, P(I)]
+    lib.loopspec_debug_drop_tile.argtypes = [V, I, I]
     lib.loopspec_time_kernel.argtypes = [V, I, I, I, P(C.c_float), P(C.c_double)]
     lib.loopspec_linear_scratch_bytes.restype = C.c_size_t
     lib.loopspec_linear_scratch_bytes.argtypes = [I, I, I]
@@ -221,7 +222,7 @@ class LoopSpec:
     """One decoding context (see include/loopspec.h for the semantics of every call)."""
 
     def __init__(self, shape, weights, d1=1, d2=0, temperature=0.0, seed=0, gate=True, residual_q2=True, max_seqs=1,
-                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None, top_k=0, top_p=1.0, measure_tv=False, mask_first=False):
+                 max_ctx=2048, alpha=0.0, beta=0.0, max_prefill_rows=0, stream=None, top_k=0, top_p=1.0, measure_tv=False, mask_first=False, prefill_skinny=False):
         import torch
         self._torch = torch
         self.shape = shape
@@ -234,7 +235,7 @@ class LoopSpec:
                            shape.n_prelude, shape.n_recurrent, shape.n_coda, shape.R,
                            1 if shape.weight_dtype == "bf16" else 0, 1 if shape.tied else 0, shape.rms_eps, shape.rope_theta)
         self.sched = Sched(d1, d2, alpha, beta, int(gate), int(residual_q2), temperature, seed, max_seqs, max_ctx,
-                           max_prefill_rows, int(top_k), float(top_p), int(measure_tv), int(mask_first))
+                           max_prefill_rows, int(top_k), float(top_p), int(measure_tv), int(mask_first), int(prefill_skinny))
         nbytes = lib.loopspec_workspace_bytes(C.byref(self.model), C.byref(self.sched))
         if nbytes == 0:
             # let init report the precise status
@@ -303,6 +304,9 @@ class LoopSpec:
 
     def vanilla_decode(self, n):
         return self._decode(lib.loopspec_vanilla_decode, n)
+
+    def debug_drop_tile(self, unit, wait_us=100):
+        self._check(lib.loopspec_debug_drop_tile(self.h, unit, wait_us))
 
     def stats(self):
         s = Stats()

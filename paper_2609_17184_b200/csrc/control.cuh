@@ -11,7 +11,7 @@ constexpr int CTRL_THREADS = 256;
 constexpr int MAX_NODES = 512;   // max_seqs * nodes-per-sequence
 enum { PH_ADVANCE = 1, PH_VERIFY = 2, PH_BUILD = 4 };
 enum { HF_ERROR = 0, HF_MIN_DEC = 1, HF_N_ROWS = 2, HF_NEED_VERIFY = 3, HF_FIRST_TOKEN = 4, HF_COUNT = 8 };
-enum { ERR_NODES = 1, ERR_CTX = 2, ERR_SPEC = 3 };
+enum { ERR_NODES = 1, ERR_CTX = 2, ERR_SPEC = 3, ERR_WAIT = 4 /* bounded wait, decode GEMM */, ERR_WAIT_PF = 5 /* prefill GEMM, grid barrier */ };
 
 struct ControlParams {
   RowTable* tab;

@@ -85,7 +85,7 @@ struct GemmParams {
   float2* argpart;        // LOGITS: [column][row block] (largest logit of the block, its vocabulary index as int bits)
   int F;                  // SWIGLU: ffn width
   int perm, perm_a, perm_d;  // order of the row tiles in the packed weights (see packed_tile)
-  volatile int* err;      // host-visible error flag (a bounded wait on a bulk copy ran out)
+  volatile int* err;      // host-visible error flag (a bounded wait in a tcgen05 kernel ran out)
   long long* dbg;         // tuning aid: cycle stamps of CTA 0 / thread 0 (null in production)
   unsigned long long* tl; // tuning aid: kernel timeline (null in production)
   int tl_id;
@@ -363,72 +363,6 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
   // consumes per unit is contiguous and consecutive k-blocks of a 16-row tile follow each other, so every warp
   // streams one contiguous region and every request covers whole 128-byte lines.  The loop is kept to a few
   // instructions per unit: shared-memory addresses are 32-bit registers advanced by constants.
-#ifdef LS_BULK
-  // Bulk variant: every warp owns RING slots of 1 KB, each filled by ONE bulk asynchronous copy (the unit is
-  // contiguous in the packed weights) that signals the slot's mbarrier; lane 0 issues, all lanes wait on the barrier.
-  __shared__ __align__(8) unsigned long long s_bar[GEMM_THREADS / 32][RING];
-  const unsigned ring_w = (unsigned)__cvta_generic_to_shared(ring) + warp * (RING * 1024);
-  const unsigned bar_w = (unsigned)__cvta_generic_to_shared(&s_bar[warp][0]);
-  if (lane == 0) {
-#pragma unroll
-    for (int sl = 0; sl < RING; ++sl) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_w + 8 * sl) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncwarp();
-  const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
-  const char* i_ptr = reinterpret_cast<const char*>(Wb);
-  unsigned i_slot = 0, c_slot = 0, c_phase = 0, pending = 0;  // slot indices; parity and in-flight bit per slot
-  bool i_valid = false, bulk_dead = false;
-  int i_rb = cid, i_left = my_upt, i_tasks = my_upt > 0 ? n_tasks : 0;
-  auto i_setup = [&]() {
-    int r0 = gemm_row0<EPI, KH>(p, i_rb, warp);
-    i_valid = r0 >= 0;  // rows beyond the matrix: nothing is copied and nothing is consumed
-    const int pt = r0 >= 0 ? packed_tile(p.perm, p.perm_a, p.perm_d, r0) : 0;
-    i_ptr = reinterpret_cast<const char*>(Wb + ((size_t)pt * kpr + kb_lo + khalf) * 512);
-  };
-  i_setup();
-  auto issue_unit = [&]() {
-    if (i_tasks > 0) {
-      __syncwarp();  // every lane has read what the slot held before
-      if (i_valid) {
-        if (lane == 0) {
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], 1024;" ::"r"(bar_w + 8 * i_slot) : "memory");
-          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 1024, [%2];" ::"r"(
-                           ring_w + 1024 * i_slot),
-                       "l"(i_ptr), "r"(bar_w + 8 * i_slot)
-                       : "memory");
-        }
-        pending |= 1u << i_slot;
-      }
-      i_ptr += 1024 * KH;
-      if (++i_slot == RING) i_slot = 0;
-      if (--i_left == 0) {
-        i_left = my_upt, i_rb += p.n_clusters;
-        if (--i_tasks > 0) i_setup();
-      }
-    }
-  };
-  // wait (bounded) until the copy into `slot` has landed
-  auto wait_slot = [&](unsigned slot) {
-    if (!(pending >> slot & 1u)) return;
-    const unsigned bar = bar_w + 8 * slot, par = (c_phase >> slot) & 1u;
-    unsigned done = bulk_dead ? 1u : 0u;
-    for (int spin = 0; !done && spin < (1 << 18); ++spin)
-      asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                   : "=r"(done)
-                   : "r"(bar), "r"(par)
-                   : "memory");
-    if (!done) {  // give up: flag it and stop waiting (the results of this pass are void)
-      bulk_dead = true;
-      if (p.err) *p.err = 5;
-    }
-    c_phase ^= 1u << slot, pending &= ~(1u << slot);
-  };
-  auto drain = [&]() {
-    for (unsigned sl = 0; sl < RING; ++sl) wait_slot(sl);
-  };
-#else
   constexpr unsigned SLOT_BYTES = 2 * GEMM_THREADS * 16, RING_BYTES = RING * SLOT_BYTES, HI_OFF = GEMM_THREADS * 16;
   const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ring) + tid * 16;
   const __nv_bfloat16* const Wb = static_cast<const __nv_bfloat16*>(p.W);
@@ -458,7 +392,6 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
     cp_async_commit();
   };
   auto drain = [&]() { cp_async_wait<0>(); };
-#endif
 #pragma unroll
   for (int s = 0; s < RING - 1; ++s) issue_unit();
 
@@ -508,9 +441,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
                         // how many rows share the pass
   const unsigned xs_s = (unsigned)__cvta_generic_to_shared(xbuf) + (g * 4 + t) * 16;
   constexpr unsigned X_KB = NTOK * 64, X_PLANE = XCH * NTOK * 64;  // bytes per k-block / per plane in xbuf
-#ifndef LS_BULK
   unsigned c_slot = 0;
-#endif
   auto lds128 = [](unsigned addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -553,17 +484,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
       unsigned xk = xs_s + kbl0 * X_KB;
       for (int kbl = kbl0; kbl < nkb; kbl += KH) {
         issue_unit();
-#ifdef LS_BULK
-        wait_slot(c_slot);
-#else
         cp_async_wait<RING - 1>();
-#endif
         if (warp_valid) {
-#ifdef LS_BULK
-          const uint4 a_lo = lds128(ring_w + 1024 * c_slot + lane * 16), a_hi = lds128(ring_w + 1024 * c_slot + 512 + lane * 16);
-#else
           const uint4 a_lo = lds128(ring_s + c_slot), a_hi = lds128(ring_s + c_slot + HI_OFF);
-#endif
           if (NG == 1) {
 #pragma unroll
             for (int s = 0; s < 3; ++s) {
@@ -592,12 +515,8 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
             }
           }
         }
-#ifdef LS_BULK
-        if (++c_slot == RING) c_slot = 0;
-#else
         c_slot += SLOT_BYTES;
         if (c_slot == RING_BYTES) c_slot = 0;
-#endif
         xk += X_KB * KH;
       }
     }

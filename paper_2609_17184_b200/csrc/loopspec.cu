@@ -13,10 +13,9 @@
 #include "common.cuh"
 #include "control.cuh"
 #include "gemm.cuh"
-#include "pass.cuh"
 #include "select.cuh"
 #include "linear_tc.cuh"
-#include "gemm_tc.cuh"
+#include "gemm_dec.cuh"
 
 using namespace ls;
 
@@ -72,6 +71,40 @@ GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1) {
 }
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+// ---- plan of a decode-pass GEMM on the tcgen05 kernel (dgemm_kernel) ----
+// One CTA per SM and kernel.  Among the cluster sizes the device can co-schedule, the one that gives the busiest CTA
+// the fewest (row block, k-block) units; ties go to the smaller cluster (fewer contributions to sum per column).
+struct DgPlan {
+  int n_rb, cs, n_clusters, stages, acc_bufs, recv_bufs;
+  size_t smem;
+};
+constexpr int kDgSmem = 200 * 1024;  // one CTA per SM: the ring takes (nearly) all of its shared memory
+int dg_mp_for_rows(int rows) { return rows <= 8 ? 8 : (rows + 15) / 16 * 16; }
+DgPlan plan_dg(int n_rb, int K, int MP, const int* max_clusters /* [9], by cluster size */) {
+  const int kb = (K + TC_BK - 1) / TC_BK;
+  DgPlan best{};
+  long long best_cost = -1;
+  for (int cs = 1; cs <= std::min(8, kb); ++cs) {
+    const int n_cl_max = max_clusters[cs];
+    if (n_cl_max < 1) continue;
+    const int n_cl = std::min(n_rb, n_cl_max);
+    const int tasks = (n_rb + n_cl - 1) / n_cl, kbm = (kb + cs - 1) / cs;
+    const long long cost = (long long)tasks * kbm;
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best.n_rb = n_rb, best.cs = cs, best.n_clusters = (n_rb + tasks - 1) / tasks;
+      best.recv_bufs = tasks > 1 ? 2 : 1;
+    }
+  }
+  if (best_cost < 0) return best;
+  best.acc_bufs = 2 * DG_CHAINS * dg_mma_n(MP) <= 512 ? 2 : 1;
+  const int budget = kDgSmem;
+  const int fixed = 1024 + best.recv_bufs * dg_recv_floats(MP, best.cs) * 4;
+  best.stages = std::max(2, std::min(DG_MAX_STAGES, (budget - fixed) / dg_stage_bytes(MP)));
+  best.smem = (size_t)dg_smem_bytes(MP, best.cs, best.stages, best.recv_bufs);
+  return best;
+}
 int ng_for_rows(int rows) { return rows <= 8 ? 1 : rows <= 16 ? 2 : rows <= 32 ? 4 : 8; }
 
 static_assert(SEL_ARG_BLOCK == RB_ROWS, "the selection reads one argmax partial per lm_head row block");
@@ -115,6 +148,18 @@ bool make_map_planes3d(CUtensorMap* map, const void* ptr, int K, int x_ld, int n
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// the same buffer with all three planes of `box_rows` rows in one box: the tile's 128-byte rows are (row, plane) pairs
+bool make_map_planes_all(CUtensorMap* map, const void* ptr, int K, int x_ld, int n_rows, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)K, 3, (cuuint64_t)n_rows};
+  cuuint64_t strides[2] = {(cuuint64_t)x_ld * 2, (cuuint64_t)x_ld * 6};
+  cuuint32_t box[3] = {(cuuint32_t)TC_BK, 3, (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 // k-split of a prefill GEMM on the tcgen05 kernel: a function of the matrix alone, so that a prompt position's sums
 // do not depend on how many positions share the pass
 struct TcPfPlan {
@@ -136,14 +181,13 @@ bool tc_prefill_shapes_ok(const loopspec_model* m) {
 int tc_pf_cols(int max_rows_pf) { return (max_rows_pf + 15) / 16 * 16; }
 
 struct Layout {  // byte offsets into the workspace
-  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, tcpart, flt, sel_flt, tv, gpart, ptrs, apart, acnt, gcnt, bar, nodes, seqs, ctr, tab_dec, tab_pf,
+  size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, tcpart, flt, sel_flt, tv, tune, tune_bytes, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
       tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
 struct Derived {
   int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, sq_stride, max_chunks,
       trace_cap, Hq, Hkv, d1, d2;
-  size_t gpart_floats, gcnt_ints;
 };
 
 int max_branches(int R, int d1, int d2) {
@@ -273,14 +317,11 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
     }
     L.tcpart = take(need);
   }
-  // persistent pass kernel: split-k partial tiles (<= 3 shares per row block), pointer tables
-  L.gpart = take((size_t)std::max((m->ffn + 63) / 64, (d.Hq + 2 * d.Hkv) / 128) * 4 * MR * 128 * 4);
-  L.ptrs = take((size_t)m->n_recurrent * 10 * sizeof(void*));
+  L.tune_bytes = kTune ? (size_t)1 << 20 : 0;  // kernel timeline of tuning builds
+  L.tune = take(L.tune_bytes);
   int G = m->n_q_heads / m->n_kv_heads;
   L.apart = take(MR * m->n_kv_heads * d.max_chunks * G * (m->head_dim + 2) * 4);
   L.acnt = take(MR * m->n_kv_heads * 4);
-  L.gcnt = take((size_t)((m->ffn + 63) / 64 + (d.Hq + 2 * d.Hkv) / 128 + 16) * 4);
-  L.bar = take(256);
   L.nodes = take((size_t)13 * MAX_NODES * 4);
   L.flt = take((size_t)2 * MAX_NODES * sizeof(float4));
   L.sel_flt = take((size_t)MAX_ROWS * sizeof(float4));
@@ -328,11 +369,14 @@ struct loopspec_ctx {
   TcPfPlan tc_plan[4];
   int tc_cols = 0, tc_stages = 0;
   size_t tc_smem = 0;
-  // ... and in one kernel per GEMM (cluster reduction + epilogue inside): weight maps with 64-row boxes
-  bool tc_fused = false, tc_all = false;
-  std::vector<CUtensorMap> gtc_wmaps;
-  int gtc_cs[4] = {1, 1, 1, 1}, gtc_stages = 0;
-  size_t gtc_smem = 0;
+  // readout GEMM of the decode passes on the tcgen05 kernel (bf16 weights): plan, tensor maps of the row-major lm_head
+  // (one box per 128-row tile) and of the hidden-state planes (all three planes of dg_mp rows in one box)
+  bool dg = false;
+  int dg_mp = 8;
+  DgPlan dgp;
+  CUtensorMap dg_wmap, dg_xmap;
+  long long dg_wait_cycles = TC_WAIT_CYCLES;
+  int dg_drop_unit = -1;  // test hook: see loopspec_debug_fail_next_step
   volatile int* host_flags = nullptr;  // pinned + mapped
   int* host_flags_dev = nullptr;
   int* pin_ids = nullptr;              // pinned staging for prompt / ids
@@ -340,10 +384,7 @@ struct loopspec_ctx {
   cudaGraphExec_t g_step = nullptr, g_vanilla = nullptr;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
-  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true, use_mega = false;
-  PassParams pass;  // persistent pass kernel (bf16 weights, at most 8 rows per decode pass)
-  int pass_grid = 0;
-  bool pass_coop = true;
+  bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true;
   bool filters = false;  // C applies top-k / top-p (sampling only)
   int sel_staged = 0;    // the selection kernel keeps its row slices in shared memory
   size_t sel_smem = 0;
@@ -466,6 +507,11 @@ AttnFn attn_fn(int d, int G, bool runs) {  // runs: contexts longer than ATT_MAX
   return G == 1 ? attn_kernel<64, 1> : attn_kernel<64, 4>;
 }
 
+// tuning builds (-DLOOPSPEC_TUNE) with LOOPSPEC_DBG set record a kernel timeline in a workspace region of their own
+unsigned long long* tune_timeline(loopspec_ctx* c) {
+  return (kTune && c->L.tune_bytes && getenv("LOOPSPEC_DBG")) ? reinterpret_cast<unsigned long long*>(c->ws + c->L.tune) : nullptr;
+}
+
 // ---- one batched pass through the shared block stack (all layers) on the rows of `tab` ------------------
 enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_LM = 4 };
 const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
@@ -536,72 +582,12 @@ cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab) {
 }
 
 
-using PassFn = void (*)(const PassParams);
-PassFn pass_fn(int d, int G) {
-  if (d == 128) return G == 1 ? pass_kernel<128, 1> : pass_kernel<128, 4>;
-  return G == 1 ? pass_kernel<64, 1> : pass_kernel<64, 4>;
-}
-
-void pass_launch_config(loopspec_ctx* c, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int n_clusters) {
-  memset(cfg, 0, sizeof *cfg);
-  cfg->gridDim = dim3(n_clusters * PASS_CS), cfg->blockDim = dim3(PASS_THREADS), cfg->dynamicSmemBytes = pass_smem_bytes();
-  cfg->stream = c->stream;
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = PASS_CS, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
-  at[1].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they meet at grid barriers
-  at[1].val.cooperative = 1;
-  cfg->attrs = at, cfg->numAttrs = c->pass_coop ? 2 : 1;
-}
-
-cudaError_t launch_pass(loopspec_ctx* c, const PassParams& pp) {
-  cudaLaunchConfig_t cfg;
-  cudaLaunchAttribute at[2];
-  pass_launch_config(c, &cfg, at, pp.n_clusters);
-  return cudaLaunchKernelEx(&cfg, pass_fn(c->m.head_dim, c->m.n_q_heads / c->m.n_kv_heads), pp);
-}
-
 // one layer GEMM of a prefill pass on the tcgen05 kernel: raw k-split sums, then the fused epilogue
 template <int EPI>
 cudaError_t launch_tc_epi(const TcEpiParams& q, cudaStream_t st, bool pdl) {
   return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
 }
-template <int EPI>
-cudaError_t launch_gtc_epi(loopspec_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, const GemmTcParams& q) {
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3(q.g.n_rb * q.g.cluster_size), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = c->gtc_smem;
-  cfg.stream = c->stream;
-  cudaLaunchAttribute at[2];
-  int n = 0;
-  if (c->use_pdl) {
-    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[n].val.programmaticStreamSerializationAllowed = 1;
-    ++n;
-  }
-  if (q.g.cluster_size > 1) {
-    at[n].id = cudaLaunchAttributeClusterDimension;
-    at[n].val.clusterDim.x = q.g.cluster_size, at[n].val.clusterDim.y = 1, at[n].val.clusterDim.z = 1;
-    ++n;
-  }
-  cfg.attrs = at, cfg.numAttrs = n;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI>, mw, mx, q);
-}
-cudaError_t launch_gtc(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
-  GemmTcParams q;
-  q.g = gemm_params(c, which, layer, tab);
-  q.g.cluster_size = c->gtc_cs[which], q.g.n_clusters = q.g.n_rb;
-  q.g.err = c->host_flags_dev + HF_ERROR;
-  q.MP = c->tc_cols, q.stages = c->gtc_stages, q.err_code = 5;
-  const int xi = which == G_O ? 1 : which == G_DOWN ? 2 : 0;
-  const CUtensorMap& mw = c->gtc_wmaps[4 * layer + which];
-  switch (which) {
-    case G_QKV: return launch_gtc_epi<EPI_QKV>(c, mw, c->tc_xmaps[xi], q);
-    case G_GU: return launch_gtc_epi<EPI_SWIGLU>(c, mw, c->tc_xmaps[xi], q);
-    default: return launch_gtc_epi<EPI_RESID>(c, mw, c->tc_xmaps[xi], q);
-  }
-}
 cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
-  if (c->tc_fused) return launch_gtc(c, which, layer, tab);
   const TcPfPlan& t = c->tc_plan[which];
   TcEpiParams q;
   q.g = gemm_params(c, which, layer, tab);
@@ -629,8 +615,43 @@ cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable
   }
 }
 
+using DgFn = void (*)(const CUtensorMap, const CUtensorMap, const DgParams);
+DgFn dg_fn(int epi) { return epi == EPI_LOGITS ? dgemm_kernel<EPI_LOGITS> : dgemm_kernel<EPI_PLAIN>; }
+cudaError_t launch_dg_raw(int epi, const DgPlan& g, const CUtensorMap& mw, const CUtensorMap& mx, const DgParams& q, cudaStream_t st,
+                          bool pdl) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(g.n_clusters * g.cs), cfg.blockDim = dim3(DG_THREADS), cfg.dynamicSmemBytes = g.smem, cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  int n = 0;
+  if (pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (g.cs > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = g.cs, at[n].val.clusterDim.y = 1, at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = at, cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, dg_fn(epi), mw, mx, q);
+}
+// the readout GEMM of a decode pass on the tcgen05 kernel
+cudaError_t launch_dg_lm(loopspec_ctx* c, const RowTable* tab) {
+  const DgPlan& g = c->dgp;
+  DgParams q;
+  memset(&q, 0, sizeof q);
+  q.g = gemm_params(c, G_LM, 0, tab);
+  q.g.cluster_size = g.cs, q.g.n_clusters = g.n_clusters, q.g.n_rb = g.n_rb;
+  q.g.err = c->host_flags_dev + HF_ERROR, q.g.tl_id = 120;
+  q.MP = c->dg_mp, q.stages = g.stages, q.acc_bufs = g.acc_bufs, q.recv_bufs = g.recv_bufs, q.err_code = ERR_WAIT;
+  q.wait_cycles = c->dg_wait_cycles;
+  q.drop_unit = c->dg_drop_unit;
+  return launch_dg_raw(EPI_LOGITS, g, c->dg_wmap, c->dg_xmap, q, c->stream, c->use_pdl);
+}
+
 cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false) {
-  tc = tc || c->tc_all;
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
@@ -638,16 +659,8 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   cudaError_t e;
   if ((e = launch_prep(c, tab))) return e;
   if (n_launch) *n_launch += 1;
-  if (c->use_mega && ng == 1) {
-    if ((e = cudaMemsetAsync(c->ws + c->L.bar, 0, 8, c->stream))) return e;
-    PassParams pp = c->pass;
-    pp.tab = tab;
-    if ((e = launch_pass(c, pp))) return e;
-    if (n_launch) *n_launch += 1;
-    return cudaSuccess;
-  }
   for (int l = 0; l < m.n_recurrent; ++l) {
-    unsigned long long* tl = getenv("LOOPSPEC_DBG") ? reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024 : nullptr;  // tuning aid
+    unsigned long long* tl = tune_timeline(c);
     GemmParams gq = gemm_params(c, G_QKV, l, tab);
     gq.tl = tl, gq.tl_id = l * 5 + 0;
     if ((e = tc ? launch_tc_gemm(c, G_QKV, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
@@ -659,7 +672,6 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
     a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
     a.scale = 1.0f / sqrtf((float)m.head_dim);
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
-    if (l == 3 && getenv("LOOPSPEC_DBG")) a.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart) + 64;  // tuning aid
     a.tl = tl, a.tl_id = l * 5 + 1;
     if ((e = launch_k(attn_fn(m.head_dim, G, d.max_chunks > ATT_MAX_RUNS), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
     GemmParams go = gemm_params(c, G_O, l, tab);
@@ -677,9 +689,9 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
 }
 
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
+  if (c->dg && tab != c->at<RowTable>(c->L.tab_pf)) return launch_dg_lm(c, tab);
   GemmParams gl = gemm_params(c, G_LM, 0, tab);
-  gl.n_sq = (c->use_mega && ng == 1) ? c->pass.n_clusters : c->d.n_sq;  // partials the layers of this pass left per row
-  if (getenv("LOOPSPEC_DBG")) gl.tl = reinterpret_cast<unsigned long long*>(c->ws + c->L.gpart) + 1024, gl.tl_id = 120;  // tuning aid
+  gl.tl = tune_timeline(c), gl.tl_id = 120;
   return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
 }
 
@@ -769,8 +781,10 @@ int check_device_error(loopspec_ctx* c) {
   int e = c->host_flags[HF_ERROR];
   if (!e) return LOOPSPEC_OK;
   c->host_flags[HF_ERROR] = 0;
+  if (e == ERR_WAIT || e == ERR_WAIT_PF)  // a bounded wait inside a kernel ran out: the pass's results are void, the context is not
+    return fail(c, LOOPSPEC_ETIMEOUT, "a bounded device-side wait ran out (%s)", e == ERR_WAIT ? "decode-pass GEMM" : "prefill GEMM or grid barrier");
   return fail(c, LOOPSPEC_ECAPACITY, "device scheduler reported %s",
-              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : e == 4 ? "a grid barrier timed out" : e == 5 ? "a bulk copy did not complete" : "speculative chain too deep");
+              e == ERR_NODES ? "node/row table overflow" : e == ERR_CTX ? "max_ctx exceeded" : "speculative chain too deep");
 }
 
 int capture(loopspec_ctx* c, cudaGraphExec_t* out, bool vanilla) {
@@ -930,26 +944,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
           delete c;
           return LOOPSPEC_ECUDA;
         }
-  if (const char* env = getenv("LOOPSPEC_NO_PDL")) c->use_pdl = !(env[0] == '1');
-  if (getenv("LOOPSPEC_DBG")) {
-    fprintf(stderr, "LOOPSPEC_DBG gpart %zu\n", L.gpart);
 #ifdef LOOPSPEC_TUNE
-    unsigned long long* tl = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + 1024;
-    cudaMemcpyToSymbol(g_tune_tl, &tl, sizeof tl);
+  if (unsigned long long* tl = tune_timeline(c)) cudaMemcpyToSymbol(g_tune_tl, &tl, sizeof tl);
 #endif
-  }
-  if (const char* env = getenv("LOOPSPEC_CS")) {  // tuning aid: explicit cluster sizes "qkv,o,gateup,down,lmhead"
-    int v[5];
-    if (sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5)
-      for (int i = 0; i < 5; ++i) {
-        GemmPlan& g = c->plan[i];
-        if (v[i] < 1 || v[i] > 8) continue;
-        g.cs = std::min(v[i], g.kpr);
-        int max_clusters = std::max(1, slots / g.cs);
-        int rounds = (g.n_rb + max_clusters - 1) / max_clusters;
-        g.n_clusters = (g.n_rb + rounds - 1) / rounds, g.grid = g.n_clusters * g.cs;
-      }
-  }
   // cluster sizes that are not powers of two are used only if the device can co-schedule them
   for (int i = 0; i < 5; ++i) {
     GemmPlan& g = c->plan[i];
@@ -963,14 +960,13 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     cfg.attrs = at, cfg.numAttrs = 1;
     int n_active = 0;
     cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
-    if (getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_DBG gemm %d: cs %d clusters %d grid %d, max active clusters %d\n", i, g.cs, g.n_clusters, g.grid, n_active);
     if (e != cudaSuccess || n_active < 1) {
       (void)cudaGetLastError();
       g = plan_gemm(n_rbs[i], Ks[i], slots, true);
     }
   }
-  // prefill passes on the tcgen05 kernel (LOOPSPEC_NO_TC_PREFILL=1: the mma.sync kernels, as the decode passes)
-  if (tc_prefill_shapes_ok(m) && !getenv("LOOPSPEC_NO_TC_PREFILL") && encode_tiled_fn()) {
+  // prefill passes on the tcgen05 kernel (shapes it does not take, and fp32 weights: the kernels of the decode passes)
+  if (tc_prefill_shapes_ok(m) && !s->prefill_skinny && encode_tiled_fn()) {
     const Derived& dd = c->d;
     c->tc_cols = tc_pf_cols(dd.max_rows_pf);
     const int sb = tc_stage_bytes(c->tc_cols);
@@ -989,27 +985,38 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tc_smem) == cudaSuccess;
     if (!ok) (void)cudaGetLastError();
     c->tc_pf = ok;
-    c->tc_all = ok && getenv("LOOPSPEC_TC_ALL") && tc_pf_cols(dd.max_rows) == c->tc_cols;  // experiment: decode passes too
-    if (ok && (getenv("LOOPSPEC_TC_FUSED") || c->tc_all)) {  // one kernel per GEMM, a cluster per row block
-      const int tail = gtc_tail_bytes(c->tc_cols), gsb = gtc_stage_bytes(c->tc_cols);
-      const int budget = c->tc_all ? 110 : 200;  // CTAs per SM: two (as the decode kernels) or one
-      const int gslots = c->tc_all ? 2 * n_sm : n_sm;
-      c->gtc_stages = std::max(2, std::min(TC_MAX_STAGES, (budget * 1024 - 1024 - tail) / gsb));
-      c->gtc_smem = (size_t)c->gtc_stages * gsb + 1024 + tail;
-      c->gtc_wmaps.resize((size_t)4 * m->n_recurrent);
-      bool ok2 = true;
-      for (int l = 0; l < m->n_recurrent && ok2; ++l)
-        for (int i = 0; i < 4 && ok2; ++i) ok2 = make_map_bf16(&c->gtc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], 64);
-      for (int i = 0; i < 4; ++i) {
-        const int n_rb = c->plan[i].n_rb, kb = Ks[i] / TC_BK;
-        c->gtc_cs[i] = std::max(1, std::min(std::min(8, kb / 2), gslots / std::max(1, n_rb)));
-      }
-      const void* fns[3] = {(const void*)gemm_tc_kernel<EPI_QKV>, (const void*)gemm_tc_kernel<EPI_RESID>, (const void*)gemm_tc_kernel<EPI_SWIGLU>};
-      for (int i = 0; i < 3 && ok2; ++i)
-        ok2 = cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->gtc_smem) == cudaSuccess;
-      if (!ok2) (void)cudaGetLastError();
-      c->tc_fused = ok2;
+  }
+  // readout GEMM of the decode passes on the tcgen05 kernel: bf16 weights whose rows are 16-byte multiples (TMA strides)
+  if (m->weight_dtype == 1 && encode_tiled_fn() && m->hidden % 8 == 0) {
+    const Derived& dd = c->d;
+    c->dg_mp = dg_mp_for_rows(dd.max_rows_dec);
+    bool ok = c->dg_mp <= DG_MAX_COLS;
+    const int budget = kDgSmem;
+    for (int epi : {EPI_LOGITS, EPI_PLAIN})
+      ok = ok && cudaFuncSetAttribute(dg_fn(epi), cudaFuncAttributeMaxDynamicSharedMemorySize, budget) == cudaSuccess;
+    int max_cl[9] = {0};
+    for (int cs = 1; cs <= 8 && ok; ++cs) {  // clusters of this size the device runs at once (one CTA per SM at most)
+      cudaLaunchConfig_t cfg;
+      memset(&cfg, 0, sizeof cfg);
+      cfg.gridDim = dim3(cs * n_sm), cfg.blockDim = dim3(DG_THREADS), cfg.dynamicSmemBytes = budget;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = cs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+      cfg.attrs = at, cfg.numAttrs = 1;
+      int n_active = 0;
+      if (cudaOccupancyMaxActiveClusters(&n_active, dg_fn(EPI_LOGITS), &cfg) != cudaSuccess) (void)cudaGetLastError(), n_active = 0;
+      // Inside the chain a kernel's clusters are placed while its predecessor's CTAs still leave: measured on the gate/up
+      // shape, three of the 45 clusters of three that the query (and a probe on the idle device) promised found no place
+      // and ran as a second wave, doubling the kernel's time; a tenth of the promise is left unused.
+      max_cl[cs] = std::min(n_active, n_sm / cs);
+      if (cs > 1) max_cl[cs] = max_cl[cs] * 9 / 10;
     }
+    if (ok) c->dgp = plan_dg((m->vocab + 127) / 128, m->hidden, c->dg_mp, max_cl);
+    ok = ok && c->dgp.cs >= 1;
+    ok = ok && make_map_bf16(&c->dg_wmap, c->lm_head, m->vocab, m->hidden, TC_BM);
+    ok = ok && make_map_planes_all(&c->dg_xmap, c->ws + c->L.xplanes, m->hidden, m->hidden, dd.max_rows, c->dg_mp);
+    if (!ok) (void)cudaGetLastError();
+    c->dg = ok;
   }
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
@@ -1065,60 +1072,6 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     ok = ok && pack(c->lm_head, m->vocab, m->hidden);
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
   }
-  // persistent pass kernel: available for bf16 weights when a decode pass carries at most 8 rows
-  if (m->weight_dtype == 1 && c->ng_dec == 1 && m->ffn % 16 == 0 && m->head_dim % 32 == 0 && m->hidden % 16 == 0) {
-    PassFn fn = pass_fn(m->head_dim, m->n_q_heads / m->n_kv_heads);
-    int max_clusters = 0;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute at[2];
-    pass_launch_config(c, &cfg, at, 1);
-    cfg.numAttrs = 1;  // the occupancy query takes the cluster shape only
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, pass_smem_bytes()) == cudaSuccess &&
-        cudaOccupancyMaxActiveClusters(&max_clusters, fn, &cfg) == cudaSuccess && max_clusters >= 1) {
-      int nc = std::min(max_clusters, d.sq_stride);
-      c->pass_grid = nc * PASS_CS;
-      std::vector<const void*> tabs((size_t)m->n_recurrent * 10);
-      for (int l = 0; l < m->n_recurrent; ++l) {
-        for (int i = 0; i < 4; ++i) tabs[(size_t)l * 4 + i] = c->packed[(size_t)l * 4 + i];
-        for (int i = 0; i < 6; ++i) tabs[(size_t)m->n_recurrent * 4 + (size_t)l * 6 + i] = c->layers[(size_t)l * 6 + i];
-      }
-      if (cudaMemcpyAsync(c->ws + L.ptrs, tabs.data(), tabs.size() * sizeof(void*), cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
-          cudaStreamSynchronize(c->stream) != cudaSuccess)
-        return bail(LOOPSPEC_ECUDA, "pointer table upload");
-      PassParams& q = c->pass;
-      memset(&q, 0, sizeof q);
-      q.L = m->n_recurrent, q.n_clusters = nc, q.final_gain = c->final_norm;
-      q.wpacked = c->at<const void*>(L.ptrs), q.layer_w = c->at<const void*>(L.ptrs) + (size_t)m->n_recurrent * 4;
-      q.H = m->hidden, q.Hq = d.Hq, q.Hkv = d.Hkv, q.F = m->ffn, q.n_q_heads = m->n_q_heads, q.n_kv_heads = m->n_kv_heads;
-      q.head_dim = m->head_dim, q.slots = d.slots, q.eps = m->rms_eps, q.scale = 1.0f / sqrtf((float)m->head_dim);
-      q.hid = c->at<float>(L.hid), q.xplanes = c->at<__nv_bfloat16>(L.xplanes), q.aplanes = c->at<__nv_bfloat16>(L.aplanes);
-      q.splanes = c->at<__nv_bfloat16>(L.splanes), q.qbuf = c->at<float>(L.qbuf), q.sumsq = c->at<float>(L.sumsq);
-      q.sq_stride = d.sq_stride;
-      q.kv = c->at<__nv_bfloat16>(L.kv), q.kv_layer_stride = c->kv_layer_stride(), q.kv_plane_stride = c->kv_plane_stride();
-      q.kv_sel_stride = c->kv_sel_stride(), q.rope = c->at<float2>(L.rope);
-      q.apart = c->at<float>(L.apart), q.acnt = c->at<int>(L.acnt);
-      q.max_chunks = d.max_chunks, q.bar = c->at<unsigned>(L.bar), q.err = c->host_flags_dev + HF_ERROR;
-      // stages: tile groups (rotary pairs, single tiles, gate/up pairs, single tiles)
-      const int groups[4] = {(m->n_q_heads + 2 * m->n_kv_heads) * (m->head_dim / 32), m->hidden / 16, m->ffn / 16, m->hidden / 16};
-      const int pairs[4] = {1, 0, 1, 0};
-      bool fits = true;
-      for (int i = 0; i < 4; ++i) {
-        q.n_groups[i] = groups[i], q.paired[i] = pairs[i], q.kpr[i] = (Ks[i] + 31) / 32, q.K[i] = Ks[i];
-        const int nt_max = ((groups[i] + nc - 1) / nc) << pairs[i];  // row tiles of the busiest cluster
-        q.kh[i] = nt_max <= PASS_TPW * 4 ? 2 : 1;
-        if (nt_max > PASS_TPW * 8 || (!pairs[i] && nt_max * 16 > PASS_THREADS)) fits = false;
-        if ((q.kpr[i] + PASS_CS - 1) / PASS_CS > PASS_XCH) fits = false;
-      }
-      c->use_mega = false;  // opt-in: LOOPSPEC_MEGA=1
-      if (d.max_chunks > ATT_MAX_RUNS) fits = false;  // its attention stage works on single chunks
-      if (const char* env = getenv("LOOPSPEC_MEGA")) c->use_mega = fits && env[0] == '1';
-      if (getenv("LOOPSPEC_DBG")) {  // tuning aid: timestamps land in the unused tail of the partial buffer
-        q.dbg = reinterpret_cast<unsigned long long*>(c->ws + L.gpart) + (1 << 20);
-        fprintf(stderr, "LOOPSPEC_DBG offset %zu clusters %d (max %d) kh %d %d %d %d fits %d\n", L.gpart + ((size_t)8 << 20), nc, max_clusters,
-                q.kh[0], q.kh[1], q.kh[2], q.kh[3], (int)fits);
-      }
-    }
-  }
   // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
   if (cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
       cudaMemsetAsync(c->ws + L.seqs, 0xff, (size_t)MAX_ROWS * 4, c->stream) != cudaSuccess ||  // root = -1
@@ -1163,7 +1116,7 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
       pp.hid = c->at<float>(c->L.hid), pp.H = c->m.hidden, pp.embed = c->embed, pp.weight_dtype = c->m.weight_dtype;
       prefill_setup_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(pp);
       CU(c, cudaGetLastError());
-      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf && !(c->use_mega && c->ng_pf == 1)));
+      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf));
     }
   }
   CU(c, launch_lm_head(c, tab, c->ng_pf));
@@ -1294,6 +1247,11 @@ int loopspec_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
     for (int s = 0; s < c->d.S; ++s)
       if (c->prefilled[s]) remaining = std::max(remaining, start[s] + n_tokens - ndec[s]);
     if (remaining <= 0) break;
+    if (kTune && getenv("LOOPSPEC_DBG_REPLAYS")) {  // tuning aid: a fixed number of replays, whatever they commit
+      for (int i = 0; i < atoi(getenv("LOOPSPEC_DBG_REPLAYS")); ++i) CU(c, cudaGraphLaunch(c->g_step, c->stream));
+      CU(c, cudaStreamSynchronize(c->stream));
+      return LOOPSPEC_OK;
+    }
     for (int i = 0; i < remaining * c->d.d1; ++i) CU(c, cudaGraphLaunch(c->g_step, c->stream));
   }
   return copy_ids_out(c, start, n_tokens, ids_out);
@@ -1386,9 +1344,19 @@ int loopspec_debug_logits(loopspec_ctx* c, int32_t seq, int32_t which, float* ou
   return LOOPSPEC_OK;
 }
 
+int loopspec_debug_drop_tile(loopspec_ctx* c, int32_t unit, int32_t wait_us) {
+  if (!c || unit < -1 || wait_us < 0) return LOOPSPEC_EINVAL;
+  if (!c->dg) return fail(c, LOOPSPEC_EUNSUPPORTED, "no tcgen05 readout kernel in this context (fp32 weights)");
+  c->dg_drop_unit = unit;
+  c->dg_wait_cycles = (unit >= 0 && wait_us > 0) ? (long long)wait_us * 2000 : TC_WAIT_CYCLES;
+  if (c->g_step) cudaGraphExecDestroy(c->g_step), c->g_step = nullptr;  // captured launches carry the old setting
+  if (c->g_vanilla) cudaGraphExecDestroy(c->g_vanilla), c->g_vanilla = nullptr;
+  return LOOPSPEC_OK;
+}
+
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
-  *out = c->use_mega ? 6 : c->m.n_recurrent * 5 + 5;
+  *out = c->m.n_recurrent * 5 + 5;
   return LOOPSPEC_OK;
 }
 
@@ -1413,8 +1381,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
       GemmParams p = gemm_params(c, which, i % L, tab);
-      if (getenv("LOOPSPEC_DBG")) p.dbg = reinterpret_cast<long long*>(c->ws + c->L.gpart);  // tuning aid
-      cudaError_t e = launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
+      cudaError_t e = (c->dg && which == G_LM) ? launch_dg_lm(c, tab) : launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }
     return cudaSuccess;
