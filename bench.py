@@ -27,9 +27,12 @@ sys.path.insert(0, ROOT)
 
 import workloads as W  # noqa: E402
 
-# DRAM bytes (read + write) of ONE launch of the dominant kernel (gate/up GEMM, Ouro-1.4B shape, 4 rows),
-# taken from the ncu capture summarised in profiles/gemm_gateup_ouro1p4b.md.
-NCU_TRAFFIC_BYTES = {"ouro_1p4b": 46226944}  # profiles/gemm_gateup_ouro1p4b.md: dram bytes read + written per launch
+# DRAM bytes (read + write) of ONE launch of the dominant kernel (gate/up GEMM, Ouro-1.4B shape, 4 rows): a profiler
+# counter, so it cannot be taken inside a timed run; this is the figure of the ncu capture of the same kernel in the same
+# launch configuration (`bench.py --kernel-only gate_up`), reported with its source and only for that model shape.
+NCU_TRAFFIC = {"ouro_1p4b": (46226944, "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch, captured on "
+                                       "`bench.py --kernel-only gate_up --rows 4` (not measured in this run)")}
+NOMINAL_HBM_GBS = 8000.0  # datasheet figure, for context beside the measured copy bandwidth
 
 
 def measured_peaks():
@@ -97,9 +100,9 @@ def step_bytes(shape, n_prompt, n_decode, stats):
     return steps * w_b + steps * w_c + stats["rows_total"] * kv_row, w_b, w_c, kv_row
 
 
-def vanilla_bytes(shape, n_prompt, n_decode):
+def vanilla_bytes(shape, n_prompt, n_decode, batch=1):
     _, w_b, w_c, kv_row = step_bytes(shape, n_prompt, n_decode, dict(steps=0, rows_total=0))
-    return n_decode * (shape.R * (w_b + kv_row) + w_c)
+    return n_decode * (shape.R * (w_b + batch * kv_row) + w_c)
 
 
 KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
@@ -242,12 +245,15 @@ def run_ours(args):
     weights = ls.upload_weights(shape, wnp)
     del wnp
     t_setup = time.time() - t0
-    prompt = W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed)
+    n_prompt = args.prompt_len or n_prompt
+    batch = wl.batch
+    prompts = [W.make_prompt(shape.vocab, n_prompt, seed=wl.prompt_seed, seq=s) for s in range(batch)]
+    prompt = prompts[0]
     d1, d2, depth_sel = wl.d1, wl.d2, None
     if args.closed_form and wl.temperature > 0:
         d1, d2, depth_sel = select_depths(ls, shape, weights, prompt, wl)
     ctx = ls.LoopSpec(shape, weights, d1=d1, d2=d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
-                      max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64, top_k=wl.top_k, top_p=wl.top_p)
+                      max_seqs=batch, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64, top_k=wl.top_k, top_p=wl.top_p)
     stream = ctx.stream
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -259,7 +265,8 @@ def run_ours(args):
     def one_job(decode_fn):
         """prefill (host ids -> device) then decode n_decode tokens; returns (decode ms on device, wall s of both)."""
         t_a = time.perf_counter()
-        ctx.prefill(prompt)
+        for s_, p_ in enumerate(prompts):      # every sequence of the batch is prefilled from its own host prompt
+            ctx.prefill(p_, seq=s_)
         with torch.cuda.stream(stream):
             ev0.record(stream)
             out = decode_fn(n_decode)
@@ -283,7 +290,6 @@ def run_ours(args):
     t_region = time.perf_counter() - t_region
     clocks = sampler.stop()
     stats = ctx.stats()
-    commits = ctx.commits(0)
     launches = ctx.launches_per_step() * stats["steps"] * args.steps
 
     # vanilla all-R decode from the same kernels (baseline of Fig. 1a)
@@ -292,9 +298,9 @@ def run_ours(args):
     for _ in range(max(2, min(args.steps, 3))):
         ms, _, vout = one_job(ctx.vanilla_decode)
         van_ms.append(ms)
-    lossless = bool((vout[0] == out[0]).all()) if wl.temperature == 0 else None
+    lossless = bool((vout == out).all()) if wl.temperature == 0 else None
 
-    value, e2e, tot_ms = replica_throughput(args.steps * n_decode, sum(dec_ms), sum(wall_s), dist, "cuda")
+    value, e2e, tot_ms = replica_throughput(args.steps * n_decode * batch, sum(dec_ms), sum(wall_s), dist, "cuda")
     ms_per_step = tot_ms / args.steps
 
     # roofline of the dominant kernel (gate/up GEMM), timed alone over the 24 layers' weights
@@ -325,31 +331,38 @@ def run_ours(args):
             tc_alone = {"error": str(e)[:200]}
     total_b, w_b, w_c, kv_row = step_bytes(shape, n_prompt, n_decode, stats)
     step_gbs = total_b / (statistics.mean(dec_ms) / 1e3) / 1e9
-    van_gbs = vanilla_bytes(shape, n_prompt, n_decode) / (statistics.mean(van_ms) / 1e3) / 1e9
+    van_gbs = vanilla_bytes(shape, n_prompt, n_decode, batch) / (statistics.mean(van_ms) / 1e3) / 1e9
     n = max(stats["n_decode"], 1)
     result = {
         "metric": "decode_tok_per_s", "value": round(value, 2), "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if shape.weight_dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": f"{wl.name}: prompt {n_prompt}, decode {n_decode}, T={wl.temperature}{f', top-p {wl.top_p}' if wl.top_p < 1 else ''}{f', top-k {wl.top_k}' if wl.top_k else ''}, (d1,d2)=({d1},{d2}), "
-                               f"gate={'on' if wl.gate else 'off'}, batch 1, R={shape.R}, L={shape.n_recurrent}",
+                               f"gate={'on' if wl.gate else 'off'}, batch {batch}, R={shape.R}, L={shape.n_recurrent}",
                    "l2": "every pass streams the 2.5 GB shared stack, far larger than the 126 MB L2; no flush needed",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks,
-        "e2e": {"value": round(e2e, 2), "unit": "tok/s", "h2d_bytes_per_step": int(n_prompt * 4),
-                "d2h_bytes_per_step": int(n_decode * 4 + 64),
-                "what": "wall clock of loopspec_prefill (host prompt ids) + loopspec_decode (host id buffer) per job"},
+        "e2e": {"value": round(e2e, 2), "unit": "tok/s", "h2d_bytes_per_step": int(batch * n_prompt * 4),
+                "d2h_bytes_per_step": int(batch * n_decode * 4 + 64),
+                "what": "wall clock of loopspec_prefill (host prompt ids, once per sequence) + loopspec_decode (host id buffer) per job"},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "gemm_kernel<bf16, NG=1, SwiGLU> (gate/up projection)",
+        "roofline": {"bound": "hbm", "kernel": "gemm_bf16_kernel<NG, SwiGLU> (gate/up projection of a decode pass; the kernel "
+                                               "with the largest share of a pass)",
                      "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                     "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(wl.model),
-                     "algorithmic_bytes_per_launch": k_bytes, "us_per_launch": round(k_ms * 1e3, 2), "rows": min(rows_typ, 8)},
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                     "traffic": NCU_TRAFFIC.get(wl.model, (None, None))[0], "traffic_source": NCU_TRAFFIC.get(wl.model, (None, None))[1],
+                     "algorithmic_bytes_per_launch": k_bytes, "us_per_launch": round(k_ms * 1e3, 2), "rows": min(rows_typ, 8),
+                     "how": "CUDA events around back-to-back launches in the decode launch configuration, cycling over the layers' weights"},
+        "readout_roofline": {"kernel": "dgemm_kernel<LOGITS> (lm_head of a decode pass: tcgen05.mma + TMA ring + cluster split-K)"
+                                       if shape.weight_dtype == "bf16" else "gemm_f32_kernel<LOGITS>",
+                             "achieved": per_kernel["lm_head"]["GBps"], "peak": peak, "unit": "GB/s",
+                             "frac": round(per_kernel["lm_head"]["GBps"] / peak, 4), "us_per_launch": per_kernel["lm_head"]["us"]},
         "kernels_alone": per_kernel,
-        "tcgen05_kernels_alone": tc_alone,
+        "prefill_tcgen05_kernels_alone": tc_alone,
         "step_roofline": {"achieved": round(step_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(step_gbs / peak, 4),
                           "ms_per_pass": round(statistics.mean(dec_ms) / max(stats["steps"], 1), 4),
                           "bytes_per_pass": int(total_b / max(stats["steps"], 1))},
-        "vanilla": {"tok_per_s": round(n_decode / (statistics.mean(van_ms) / 1e3), 2),
+        "vanilla": {"tok_per_s": round(batch * n_decode / (statistics.mean(van_ms) / 1e3), 2),
                     "hbm_GBps": round(van_gbs, 1), "frac": round(van_gbs / peak, 4)},
         "speedup_vs_vanilla": round(statistics.mean(van_ms) / statistics.mean(dec_ms), 4),
         "greedy_equals_vanilla": lossless,
@@ -361,11 +374,14 @@ def run_ours(args):
                        "passes": stats["steps"]},
         "setup_s": round(t_setup, 1), "timed_region_wall_s": round(t_region, 2),
     }
-    if args.calibrated and rank == 0:
+    if rank == 0 and world == 1 and batch == 1 and not args.no_calibrated and (args.calibrated or args.workload == "ouro_1p4b"):
+        ctx.close()
+        ctx = None
         result["calibrated_variant"] = run_calibrated(ls, shape, wl, prompt, n_prompt, n_decode, args)
     if rank == 0 and world == 1 and not args.no_cpu:
         result["cpu_baseline"] = cpu_baseline(shape, wl, seconds_budget=25.0)
-    ctx.close()
+    if ctx is not None:
+        ctx.close()
     if rank == 0:
         print(json.dumps(result))
     if dist is not None:
@@ -377,7 +393,7 @@ def run_calibrated(ls, shape, wl, prompt, n_prompt, n_decode, args):
     draft like trained checkpoints do (first-proposal share in the band the paper reports for Ouro-1.4B)."""
     import torch
     res = None
-    for scale in (0.0003, 0.0001, 0.001, 0.00003):
+    for scale in (0.0001, 0.0003, 0.001, 0.00003):
         w = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed, out_scale=scale))
         ctx = ls.LoopSpec(shape, w, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate,
                           max_seqs=1, max_ctx=n_prompt + n_decode + 16, max_prefill_rows=64)
@@ -385,23 +401,25 @@ def run_calibrated(ls, shape, wl, prompt, n_prompt, n_decode, args):
         times = {}
         for name, fn in (("loopspec", ctx.decode), ("vanilla", ctx.vanilla_decode)):
             ms = []
-            for i in range(3):
+            for i in range(2):
                 ctx.prefill(prompt)
                 ev0.record(ctx.stream)
                 fn(n_decode)
                 ev1.record(ctx.stream)
                 ev1.synchronize()
                 ms.append(ev0.elapsed_time(ev1))
-                if name == "loopspec" and i == 2:
+                if name == "loopspec" and i == 1:
                     st = ctx.stats()
-            times[name] = statistics.mean(ms[1:])
+            times[name] = ms[1]
         n = max(st["n_decode"], 1)
         res = {"out_scale": scale, "tok_per_s": round(n_decode / (times["loopspec"] / 1e3), 2),
                "vanilla_tok_per_s": round(n_decode / (times["vanilla"] / 1e3), 2),
                "speedup_vs_vanilla": round(times["vanilla"] / times["loopspec"], 4), "gamma": round(st["gamma"], 4),
                "first": round(st["n_accept1"] / n, 4), "second": round(st["n_accept2"] / n, 4),
                "restart": round(st["n_restart"] / n, 4),
-               "note": "NOT the config as given: out-projection scale tuned so acceptance resembles trained weights"}
+               "note": "NOT the config as given: the same shape and workload with the out-projection scale lowered until the "
+                       "first-proposal share lies in the band the paper reports for trained Ouro-1.4B weights (86.6-95.4 %); "
+                       "random weights at the given scale 0.3 draft far worse than trained ones"}
         ctx.close()
         del w
         torch.cuda.empty_cache()
@@ -478,7 +496,9 @@ def main():
     ap.add_argument("--workload", default="ouro_1p4b")
     ap.add_argument("--decode-len", type=int, default=0)
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
-    ap.add_argument("--calibrated", action="store_true", help="also run the acceptance-calibrated variant")
+    ap.add_argument("--calibrated", action="store_true", help="also run the acceptance-calibrated variant (default for ouro_1p4b)")
+    ap.add_argument("--no-calibrated", action="store_true", help="skip the acceptance-calibrated variant")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length")
     ap.add_argument("--closed-form", action="store_true",
                     help="sampling workloads: pick (d1, d2) from Theorem 2 on a TV profile measured on the device first")
     ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")

@@ -30,6 +30,9 @@ class Branch:                      # Algorithm 1: prefix X(b), hidden H_b, depth
     r: int = 0
     records: list = field(default_factory=list)
     kv: dict = field(default_factory=dict)      # recurrence -> [per layer (k, v)] while speculative
+    e: object = None               # Raven layout: prelude output of the last token (constant over the recurrences)
+    pre_kv: object = None          # ... its prelude keys/values [per layer (k, v)] while speculative
+    coda_kv: dict = field(default_factory=dict)  # ... readout depth -> [per coda layer (k, v)] while speculative
     q1_logits: object = None       # kept for inspection
     q2_logits: object = None
 
@@ -62,6 +65,23 @@ class Decoder:
         shp = (n_total, s.n_kv_heads, s.head_dim)
         self.K = [[np.zeros(shp) for _ in range(s.n_recurrent)] for _ in range(s.R + 1)]
         self.V = [[np.zeros(shp) for _ in range(s.n_recurrent)] for _ in range(s.R + 1)]
+        if getattr(self.m, "raven", False):   # prelude cache, and one coda cache per readout depth (App. B)
+            self.PK = [np.zeros(shp) for _ in range(s.n_prelude)]
+            self.PV = [np.zeros(shp) for _ in range(s.n_prelude)]
+            self.CK = {d: [np.zeros(shp) for _ in range(s.n_coda)] for d in self.readout_depths}
+            self.CV = {d: [np.zeros(shp) for _ in range(s.n_coda)] for d in self.readout_depths}
+
+    @property
+    def raven(self):
+        return getattr(self.m, "raven", False)
+
+    def _store_prelude(self, pos, per_layer_kv):
+        for l, (k, v) in enumerate(per_layer_kv):
+            self.PK[l][pos], self.PV[l][pos] = k, v
+
+    def _store_coda(self, d, pos, per_layer_kv):
+        for l, (k, v) in enumerate(per_layer_kv):
+            self.CK[d][l][pos], self.CV[d][l][pos] = k, v
 
     def _store_committed(self, r, pos, per_layer_kv):
         for l, (k, v) in enumerate(per_layer_kv):
@@ -94,18 +114,31 @@ class Decoder:
         return self._draw(self.probs(logits), position, purpose)
 
     # ---- prefill: all R recurrences over the prompt, first token from C(H^R) -------------------
-    def prefill(self, prompt, n_decode):
+    def prefill(self, prompt, n_decode, depths=None):
+        """depths = (d1, d2) of the LoopSpec run that follows (Raven layout only: the prompt must fill the coda cache of
+        every readout depth; None: only depth R, which is all vanilla decoding needs)."""
         s = self.m.s
         self.ids = [int(t) for t in prompt]
         self.n_prompt = n = len(self.ids)
+        self.readout_depths = sorted({s.R} | {d for d in (depths or ()) if d})
         self._alloc(self.max_ctx or (n + n_decode + 1))
         X = self.m.embed_tokens(self.ids)
+        E = None
+        if self.raven:
+            X, kv = self.m.prelude_prompt(X)
+            E = X
+            for l, (k, v) in enumerate(kv):
+                self.PK[l][:n], self.PV[l][:n] = k, v
         for r in range(1, s.R + 1):
-            X, kv = self.m.advance_prompt(X)
+            X, kv = self.m.advance_prompt(X, E)
             for l, (k, v) in enumerate(kv):
                 self.K[r][l][:n] = k
                 self.V[r][l][:n] = v
-        z = self.m.logits(X[-1])
+            if self.raven and r in self.readout_depths:
+                Xc, ckv = self.m.coda_prompt(X)
+                for l, (k, v) in enumerate(ckv):
+                    self.CK[r][l][:n], self.CV[r][l][:n] = k, v
+        z = self.m.logits(Xc[-1] if self.raven else X[-1])
         self.first_logits = z
         tok, margin = self._sample_target(z, n, sp.VANILLA)
         self.log.append(dict(kind="first", pos=n, token=tok, margin=margin))
@@ -119,10 +152,18 @@ class Decoder:
         for _ in range(n_tokens):
             pos = len(self.ids) - 1
             x = self.m.embed_tokens([self.ids[-1]])
+            e = None
+            if self.raven:
+                x, own = self.m.prelude_rows(x, [pos], lambda i, l: (self.PK[l][:pos], self.PV[l][:pos]))
+                self._store_prelude(pos, own[0])
+                e = x
             for r in range(1, s.R + 1):
                 x, own = self.m.advance_rows(
-                    x, [pos], lambda i, l, r=r: (self.K[r][l][:pos], self.V[r][l][:pos]))
+                    x, [pos], lambda i, l, r=r: (self.K[r][l][:pos], self.V[r][l][:pos]), e)
                 self._store_committed(r, pos, own[0])
+            if self.raven:
+                x, own = self.m.coda_rows(x, [pos], lambda i, l: (self.CK[s.R][l][:pos], self.CV[s.R][l][:pos]))
+                self._store_coda(s.R, pos, own[0])
             z = self.m.logits(x[0])
             tok, margin = self._sample_target(z, pos + 1, sp.VANILLA)
             self.log.append(dict(kind="vanilla", pos=pos + 1, token=tok, margin=margin))
@@ -134,9 +175,53 @@ class Decoder:
 
     # ---- LoopSpec ------------------------------------------------------------------------------
     def _spawn(self, parent, token, pos):
+        """Spawn(X || token): a branch at depth 0 with H0 = P(X || token) (Eq. 1; for the Raven layout the prelude blocks
+        run here, over the prelude keys/values of the branch's prefix)."""
         b = Branch(parent=parent, token=int(token), pos=pos, H=self.m.embed_tokens([token])[0])
+        if self.raven:
+            e, own = self.m.prelude_rows(b.H[None], [pos], lambda i, l: self._prefix_generic(
+                b, l, self.PK, self.PV, lambda a: a.pre_kv))
+            b.H = b.e = e[0]
+            if parent is None:
+                self._store_prelude(pos, own[0])
+            else:
+                b.pre_kv = own[0]
         self.active.append(b)
         return b
+
+    def _prefix_generic(self, b, layer, Kc, Vc, branch_kv):
+        """Keys/values of every position before b's own in b's prefix, for a cache with committed arrays Kc/Vc [layer] and
+        per-branch entries branch_kv(a) -> [per layer (k, v)] for the uncommitted ancestors."""
+        chain = []
+        a = b.parent
+        while a is not None:
+            chain.append(a)
+            a = a.parent
+        chain.reverse()
+        n_committed = b.pos if not chain else chain[0].pos
+        Ks, Vs = [Kc[layer][:n_committed]], [Vc[layer][:n_committed]]
+        for a in chain:
+            if a.parent is None:
+                Ks.append(Kc[layer][a.pos][None])
+                Vs.append(Vc[layer][a.pos][None])
+            else:
+                k, v = branch_kv(a)[layer]
+                Ks.append(k[None])
+                Vs.append(v[None])
+        return np.concatenate(Ks, axis=0), np.concatenate(Vs, axis=0)
+
+    def _readout_logits(self, b, depth):
+        """p_r = C(H^r) before temperature (Sec. 3.1): final norm + lm_head; for the Raven layout the coda blocks first, over
+        the coda cache of this readout depth (App. B), whose entry for b's own position is produced here."""
+        if not self.raven:
+            return self.m.logits(b.H)
+        x, own = self.m.coda_rows(b.H[None], [b.pos], lambda i, l: self._prefix_generic(
+            b, l, self.CK[depth], self.CV[depth], lambda a: a.coda_kv[depth]))
+        if b.parent is None:
+            self._store_coda(depth, b.pos, own[0])
+        else:
+            b.coda_kv[depth] = own[0]
+        return self.m.logits(x[0])
 
     def _prefix_kv(self, b, r, layer):
         """Keys/values, at recurrence r, of every position before b's own in b's prefix."""
@@ -199,6 +284,8 @@ class Decoder:
         s = self.m.s
         R = s.R
         assert 1 <= d1 < R and (d2 == 0 or d1 < d2 < R)
+        if self.raven:
+            assert {d for d in (d1, d2, R) if d} <= set(self.readout_depths), "prefill(..., depths=(d1, d2)) first"
         self.active = []
         self.commits, self.verify_logits = [], []
         self.stats = dict(steps=0, n_decode=0, n_accept1=0, n_accept2=0, n_restart=0,
@@ -209,7 +296,8 @@ class Decoder:
             cur = list(self.active)
             X = np.stack([b.H for b in cur])
             Xn, own = self.m.advance_rows(
-                X, [b.pos for b in cur], lambda i, l: self._prefix_kv(cur[i], cur[i].r + 1, l))
+                X, [b.pos for b in cur], lambda i, l: self._prefix_kv(cur[i], cur[i].r + 1, l),
+                np.stack([b.e for b in cur]) if self.raven else None)
             self.stats["steps"] += 1
             self.stats["rows_total"] += len(cur)
             self.stats["rows_max"] = max(self.stats["rows_max"], len(cur))
@@ -224,7 +312,7 @@ class Decoder:
             for b in cur:
                 pos = b.pos + 1                  # position this branch proposes for
                 if b.r == d1:                    # first proposal
-                    z1 = self.m.logits(b.H)
+                    z1 = self._readout_logits(b, d1)
                     self.stats["readout_rows_total"] += 1
                     b.q1_logits = z1
                     if self.T == 0.0:
@@ -237,7 +325,7 @@ class Decoder:
                     c1 = self._spawn(b, x1, pos)
                     b.records.append(Record(x1, q1, c1))
                 elif d2 and b.r == d2:           # gated residual second proposal
-                    z2 = self.m.logits(b.H)
+                    z2 = self._readout_logits(b, d2)
                     self.stats["readout_rows_total"] += 1
                     b.q2_logits = z2
                     x1 = b.records[0].token
@@ -278,7 +366,7 @@ class Decoder:
             bmax = max(self.active, key=lambda b: b.r)
             if bmax.r == R:
                 assert bmax.parent is None
-                p_logits = self.m.logits(bmax.H)
+                p_logits = self._readout_logits(bmax, R)
                 self.stats["readout_rows_total"] += 1
                 tok, child, source = self._verify(bmax, p_logits)
                 if keep_logits:
@@ -302,6 +390,11 @@ class Decoder:
                     for r, per_layer in child.kv.items():
                         self._store_committed(r, child.pos, per_layer)
                     child.kv = {}
+                    if self.raven:
+                        self._store_prelude(child.pos, child.pre_kv)
+                        for d, per_layer in child.coda_kv.items():
+                            self._store_coda(d, child.pos, per_layer)
+                        child.pre_kv, child.coda_kv = None, {}
         st = self.stats
         den = st["n_accept1"] * d1 + st["n_accept2"] * d2 + st["n_restart"] * R
         st["gamma"] = st["n_decode"] * R / den if den else float("nan")

@@ -79,12 +79,21 @@ CONFIGS = {
     # a mid-size bf16 model whose GEMMs span several tiles, K-slices and a ragged last tile
     "small_bf16": ModelShape("small_bf16", vocab=4000, hidden=768, n_q_heads=6, n_kv_heads=6, head_dim=128,
                              ffn=2000, n_recurrent=3, R=4, weight_dtype="bf16", tied=False),
+    # Raven layout at test size: prelude and coda blocks around the recurrent block, an adapter on [state; prelude output],
+    # grouped-query attention with head size 64 (the head layout of the Raven-style benchmark config), R = 16
+    "tiny_raven": ModelShape("tiny_raven", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=1, head_dim=64,
+                             ffn=704, n_recurrent=2, R=16, weight_dtype="bf16", tied=False, n_prelude=1, n_coda=1),
+    "tiny_raven_r4": ModelShape("tiny_raven_r4", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                                ffn=704, n_recurrent=2, R=4, weight_dtype="bf16", tied=False, n_prelude=2, n_coda=2),
     # config 1: Ouro-1.4B shape
     "ouro_1p4b": ModelShape("ouro_1p4b", vocab=49152, hidden=2048, n_q_heads=16, n_kv_heads=16, head_dim=128,
                             ffn=5632, n_recurrent=24, R=4, weight_dtype="bf16", tied=False),
     # config 2: Ouro-2.6B shape
     "ouro_2p6b": ModelShape("ouro_2p6b", vocab=49152, hidden=2048, n_q_heads=16, n_kv_heads=16, head_dim=128,
                             ffn=5632, n_recurrent=48, R=4, weight_dtype="bf16", tied=False),
+    # config 4: Raven-style prelude / recurrent / coda model
+    "raven": ModelShape("raven", vocab=128256, hidden=2048, n_q_heads=32, n_kv_heads=8, head_dim=64,
+                        ffn=8192, n_recurrent=4, R=16, weight_dtype="bf16", tied=False, n_prelude=2, n_coda=2),
 }
 
 WORKLOADS = {
@@ -94,6 +103,7 @@ WORKLOADS = {
     # the paper's sampling setting for its reasoning models (Sec. 6 "Models and Evaluations": T = 1.0, top-p 0.7) on the headline shape
     "ouro_1p4b_top_p": Workload("ouro_1p4b_top_p", "ouro_1p4b", prompt_len=512, decode_len=512, temperature=1.0, d1=1,
                                 d2=2, top_p=0.7),
+    "raven": Workload("raven", "raven", prompt_len=256, decode_len=512, temperature=0.0, d1=2, d2=8),
     "kv_bound": Workload("kv_bound", "ouro_1p4b", prompt_len=8192, decode_len=256, temperature=0.7, d1=1, d2=2,
                          batch=8),
 }

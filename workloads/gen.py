@@ -27,10 +27,15 @@ def weight_order(shape):
     if not shape.tied:
         out.append(("lm_head", (shape.vocab, h)))
     out.append(("final_norm", (h,)))
-    for l in range(shape.n_recurrent):
-        out += [(f"layers.{l}.norm1", (h,)), (f"layers.{l}.wqkv", (nq + 2 * nkv, h)),
-                (f"layers.{l}.wo", (h, nq)), (f"layers.{l}.norm2", (h,)),
-                (f"layers.{l}.wgateup", (2 * f, h)), (f"layers.{l}.wdown", (h, f))]
+    stacks = [("layers", shape.n_recurrent)]
+    if shape.n_prelude or shape.n_coda:   # Raven layout: adapter on [state; prelude output], then prelude, recurrent, coda blocks
+        out.append(("adapter", (h, 2 * h)))
+        stacks = [("prelude", shape.n_prelude), ("layers", shape.n_recurrent), ("coda", shape.n_coda)]
+    for prefix, n in stacks:
+        for l in range(n):
+            out += [(f"{prefix}.{l}.norm1", (h,)), (f"{prefix}.{l}.wqkv", (nq + 2 * nkv, h)),
+                    (f"{prefix}.{l}.wo", (h, nq)), (f"{prefix}.{l}.norm2", (h,)),
+                    (f"{prefix}.{l}.wgateup", (2 * f, h)), (f"{prefix}.{l}.wdown", (h, f))]
     return out
 
 
