@@ -42,10 +42,14 @@ typedef enum {
 } loopspec_status;
 
 /* Looped transformer of Sec. 3.1 (Eq. 1).  Ouro layout: n_prelude = n_coda = 0, P = embedding, C = final
- * RMSNorm + lm_head.  Blocks are pre-RMSNorm, rotary attention (rotate-half pairing), SwiGLU, no biases. */
+ * RMSNorm + lm_head.  Raven-style layout (n_prelude or n_coda > 0; Sec. 3.1: P and C hold transformer blocks too):
+ * P = embedding + n_prelude blocks giving e, H0 = e, one recurrence is H <- RecurrentBlocks(W_a [H; e]) with the adapter
+ * W_a [hidden][2 hidden], C = n_coda blocks + final RMSNorm + lm_head.  The prelude blocks have an ordinary KV cache, the
+ * coda blocks one cache per readout depth (d1, d2, R: App. B "KV Cache Management"); the prompt fills all of them.
+ * Blocks are pre-RMSNorm, rotary attention (rotate-half pairing), SwiGLU, no biases. */
 typedef struct {
   int32_t vocab, hidden, n_q_heads, n_kv_heads, head_dim, ffn;
-  int32_t n_prelude, n_recurrent, n_coda; /* layers in P, B, C; only n_prelude = n_coda = 0 is supported */
+  int32_t n_prelude, n_recurrent, n_coda; /* transformer blocks in P, B, C */
   int32_t R;                              /* recurrences of B */
   int32_t weight_dtype;                   /* 0 = fp32, 1 = bf16 (all matrices incl. embedding) */
   int32_t tied_lm_head;                   /* 1: lm_head pointer ignored, the embedding is used */
@@ -88,9 +92,11 @@ typedef struct {
                              wide tcgen05 kernels (slower; for comparing the two paths) */
 } loopspec_sched;
 
-/* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * n_recurrent device pointers, per layer:
+/* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * (n_prelude + n_recurrent + n_coda) device pointers -
+ * the prelude blocks, then the recurrent blocks, then the coda blocks - per block:
  * norm1 [H], wqkv [(nq + 2 nkv) * d][H] (q rows, then k rows, then v rows), wo [H][nq * d], norm2 [H],
- * wgateup [2F][H] (gate rows, then up rows), wdown [H][F].  adapter must be NULL. */
+ * wgateup [2F][H] (gate rows, then up rows), wdown [H][F].  adapter: [H][2H] (columns: state, then prelude output) for
+ * the Raven-style layout, NULL for the Ouro layout. */
 typedef struct {
   const void* embed;      /* [V][H] */
   const void* lm_head;    /* [V][H], ignored when tied */

@@ -242,13 +242,16 @@ class LoopSpec:
             nbytes = 256
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         names = ["norm1", "wqkv", "wo", "norm2", "wgateup", "wdown"]
-        ptrs = (C.c_void_p * (6 * shape.n_recurrent))()
-        for l in range(shape.n_recurrent):
+        blocks = [(f"prelude.{l}") for l in range(shape.n_prelude)] + [f"layers.{l}" for l in range(shape.n_recurrent)] + \
+                 [f"coda.{l}" for l in range(shape.n_coda)]
+        ptrs = (C.c_void_p * (6 * len(blocks)))()
+        for i, blk in enumerate(blocks):
             for j, n in enumerate(names):
-                ptrs[6 * l + j] = weights[f"layers.{l}.{n}"].data_ptr()
+                ptrs[6 * i + j] = weights[f"{blk}.{n}"].data_ptr()
         self._ptrs = ptrs
+        adapter = weights["adapter"].data_ptr() if (shape.n_prelude or shape.n_coda) else None
         wt = Weights(weights["embed"].data_ptr(), 0 if shape.tied else weights["lm_head"].data_ptr(),
-                     weights["final_norm"].data_ptr(), None, C.cast(ptrs, C.POINTER(C.c_void_p)))
+                     weights["final_norm"].data_ptr(), adapter, C.cast(ptrs, C.POINTER(C.c_void_p)))
         h = C.c_void_p()
         rc = lib.loopspec_init(C.byref(self.model), C.byref(self.sched), C.byref(wt), self.workspace.data_ptr(), nbytes,
                                self.stream.cuda_stream, C.byref(h))

@@ -54,6 +54,8 @@ struct RowTable {
   int logit_idx[MAX_ROWS];   // which logits vector its readout fills
   int node[MAX_ROWS];        // global node index (seq * NB + node), -1 for prefill rows
   int ro_rows[MAX_ROWS];     // compact list of rows with readout != 0
+  int src_hid[MAX_ROWS];     // >= 0: the pass works on a copy of this hidden state, made into hid_idx by its preparation
+                             // (the post-layers C of a Raven-style model must not disturb the branch's recurrent state)
   int chunk_start[MAX_ROWS + 1];  // exclusive prefix sum of attention work items per row
 };
 

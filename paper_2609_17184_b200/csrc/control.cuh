@@ -38,7 +38,51 @@ struct ControlParams {
   int weight_dtype;
   int p_logit_base;  // logits index of sequence 0's target readout
   volatile int* host_flags;  // pinned, host-mapped
+  // Raven-style layout (P and C hold transformer blocks, Sec. 3.1): the rows entering their first recurrence go through
+  // the prelude blocks first (tab_pre), the reading-out rows through the coda blocks on a copy of their state (tab_coda)
+  RowTable* tab_pre;   // null for the Ouro layout
+  RowTable* tab_coda;
+  int hid_coda_base;   // first hidden-state index of the coda pass's copies
 };
+
+// Sub-pass tables of the Raven-style layout, derived from the pass's rows (thread 0, straight to global memory).
+// class_of_readout: RO_D1 -> coda cache 1, RO_D2 -> 2, RO_VERIFY / RO_TARGET -> the last one (its plane index + 1 is `r`).
+__device__ void derive_raven_tables(const RowTable& t, RowTable* pre, RowTable* coda, int hid_coda_base, int n_classes) {
+  auto copy_row = [&](RowTable* dst, int j, int i) {
+    dst->seq[j] = t.seq[i], dst->pos[j] = t.pos[i], dst->kv_slot[j] = t.kv_slot[i], dst->n_canon[j] = t.n_canon[i];
+    dst->n_spec[j] = t.n_spec[i], dst->n_safe[j] = t.n_safe[i], dst->node[j] = t.node[i], dst->logit_idx[j] = t.logit_idx[i];
+    for (int k = 0; k < MAX_SPEC; ++k) dst->spec_slot[j][k] = t.spec_slot[i][k];
+  };
+  int items = 0;
+  if (pre) {
+    int np = 0;
+    for (int i = 0; i < t.n_rows; ++i) {
+      if (t.r[i] != 1) continue;  // P runs once per branch, before its first recurrence
+      copy_row(pre, np, i);
+      pre->r[np] = 1, pre->hid_idx[np] = t.hid_idx[i], pre->src_hid[np] = -1, pre->readout[np] = RO_NONE;
+      pre->chunk_start[np] = items;
+      items += att_items(t.n_canon[i]);
+      ++np;
+    }
+    pre->chunk_start[np] = items;
+    pre->n_rows = np, pre->n_readout = 0, pre->attn_items = items, pre->n_layers_done = 0;
+  }
+  int nc = 0;
+  items = 0;
+  for (int j = 0; j < t.n_readout; ++j) {
+    const int i = t.ro_rows[j];
+    copy_row(coda, nc, i);
+    const int ro = t.readout[i];
+    coda->r[nc] = ro == RO_D1 ? 1 : (ro == RO_D2 ? 2 : n_classes);
+    coda->hid_idx[nc] = hid_coda_base + nc, coda->src_hid[nc] = t.hid_idx[i];
+    coda->readout[nc] = ro, coda->ro_rows[nc] = nc;
+    coda->chunk_start[nc] = items;
+    items += att_items(t.n_canon[i]);
+    ++nc;
+  }
+  coda->chunk_start[nc] = items;
+  coda->n_rows = nc, coda->n_readout = nc, coda->attn_items = items, coda->n_layers_done = 0;
+}
 
 struct NodeSmem {
   int state[MAX_NODES], depth[MAX_NODES], pos[MAX_NODES], token[MAX_NODES], parent[MAX_NODES], child1[MAX_NODES],
@@ -110,6 +154,7 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       const bool is_root = nd.parent[o + n] < 0;
       t.seq[i] = s, t.r[i] = r, t.pos[i] = nd.pos[o + n], t.node[i] = o + n, t.hid_idx[i] = o + n;
       t.kv_slot[i] = is_root ? nd.pos[o + n] : p.ctx_cap + n;
+      t.src_hid[i] = -1;
       t.n_canon[i] = nd.pos[o + rt] + 1;
       t.n_safe[i] = is_root ? nd.pos[o + n] : t.n_canon[i];
       int chain[MAX_SPEC], len = 0;
@@ -260,7 +305,10 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
     }
     int err = s_err;
     // rows are rebuilt only when no verification is pending (the verify phase needs the current rows)
-    if ((p.phases & PH_BUILD) && need == 0) build_rows(t, nd, s_root, s_ndec, s_ntarget, p, &err);
+    if ((p.phases & PH_BUILD) && need == 0) {
+      build_rows(t, nd, s_root, s_ndec, s_ntarget, p, &err);
+      if (p.tab_pre) derive_raven_tables(t, p.tab_pre, p.tab_coda, p.hid_coda_base, p.d2 > 0 ? 3 : 2);
+    }
     p.host_flags[HF_MIN_DEC] = min_dec, p.host_flags[HF_N_ROWS] = t.n_rows, p.host_flags[HF_NEED_VERIFY] = need;
     if (err) p.host_flags[HF_ERROR] = err;
   }
@@ -294,6 +342,8 @@ struct VanillaParams {
   const void* embed;
   int weight_dtype, p_logit_base, ctx_cap;
   volatile int* host_flags;
+  RowTable* tab_coda;  // Raven-style layout: the readout rows of the last recurrence on copies of their states (else null)
+  int hid_coda_base, n_classes;
 };
 
 __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __grid_constant__ VanillaParams p) {
@@ -342,12 +392,15 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
         int s = s_rowof[i], gn = s_emb[i][0], pos = p.nodes.pos[gn];
         t.seq[i] = s, t.r[i] = r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
         t.n_safe[i] = pos;
-        t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE;
+        t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE, t.src_hid[i] = -1;
         t.logit_idx[i] = p.p_logit_base + s, t.ro_rows[i] = i, t.chunk_start[i] = items;
         items += att_items(pos + 1);
       }
       t.chunk_start[n] = items;
       t.n_rows = n, t.n_readout = (r == p.R) ? n : 0, t.attn_items = items, t.n_layers_done = 0;
+    }
+    if (p.tab_coda) {  // the prelude pass of a vanilla token is the first table itself (every row enters recurrence 1)
+      derive_raven_tables(p.tabs[p.R - 1], nullptr, p.tab_coda, p.hid_coda_base, p.n_classes);
     }
   }
   __syncthreads();
@@ -365,6 +418,9 @@ struct PrefillParams {
   int H;
   const void* embed;
   int weight_dtype;
+  RowTable* tab_coda;  // Raven-style layout: every prompt row goes through the coda blocks at the readout depths, on copies
+  int coda_class;      // cache of this recurrence's readout depth (1-based; 0: this recurrence is no readout depth)
+  int hid_coda_base;
 };
 
 __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const PrefillParams p) {
@@ -377,7 +433,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
       int pos = p.p0 + i;
       t.seq[i] = p.seq, t.r[i] = p.r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
       t.n_safe[i] = p.p0;
-      t.hid_idx[i] = p.hid_base + i, t.node[i] = -1;
+      t.hid_idx[i] = p.hid_base + i, t.node[i] = -1, t.src_hid[i] = -1;
       bool last = (p.r == p.R) && (pos == p.n_prompt - 1);
       t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;
       if (last) t.ro_rows[n_ro++] = i;
@@ -387,6 +443,18 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
     }
     t.chunk_start[p.count] = items;
     t.n_rows = p.count, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
+    if (p.tab_coda && p.coda_class > 0) {  // the same rows, on copies of their states, writing this depth's coda cache
+      RowTable& c = *p.tab_coda;
+      int nr = 0;
+      for (int i = 0; i < p.count; ++i) {
+        c.seq[i] = t.seq[i], c.r[i] = p.coda_class, c.pos[i] = t.pos[i], c.kv_slot[i] = t.kv_slot[i], c.n_canon[i] = t.n_canon[i];
+        c.n_spec[i] = 0, c.n_safe[i] = t.n_safe[i], c.hid_idx[i] = p.hid_coda_base + i, c.src_hid[i] = t.hid_idx[i], c.node[i] = -1;
+        c.readout[i] = t.readout[i], c.logit_idx[i] = t.logit_idx[i], c.chunk_start[i] = t.chunk_start[i];
+        if (t.readout[i]) c.ro_rows[nr++] = i;
+      }
+      c.chunk_start[p.count] = items;
+      c.n_rows = p.count, c.n_readout = nr, c.attn_items = items, c.n_layers_done = 0;
+    }
   }
   __syncthreads();
   if (p.r == 1) embed_rows(s_emb, p.count, p.hid, p.H, p.embed, p.weight_dtype);
@@ -429,6 +497,10 @@ struct KvCommitParams {
   __nv_bfloat16* kv;      // whole pool [L][R][2][S][n_kv][slots][d]
   long long layer_stride, plane_stride, sel_stride;
   int S, L, n_kv_heads, slots, d;
+  // Raven-style layout: the pool's layers are prelude blocks (one plane), recurrent blocks (a plane per recurrence) and coda
+  // blocks (a plane per readout depth); n_prelude = 0 and n_classes = 0 for the Ouro layout
+  int n_prelude, n_rec, n_classes;
+  int class_depth[3];
 };
 
 __global__ void kv_commit_kernel(const __grid_constant__ KvCommitParams p) {
@@ -439,7 +511,14 @@ __global__ void kv_commit_kernel(const __grid_constant__ KvCommitParams p) {
   struct EndMark { __device__ ~EndMark() { tune_mark(604, true); } } end_mark;
   const int l = blockIdx.x, plane = blockIdx.y, sel = blockIdx.z & 1, s = blockIdx.z >> 1;
   const KvCopyCmd c = p.cmds[s];
-  if (plane >= c.n_planes) return;
+  if (c.n_planes <= 0) return;                 // nothing kept for this sequence (n_planes = recurrent depth of the kept child)
+  if (l < p.n_prelude) {
+    if (plane != 0) return;                    // its prelude keys / values
+  } else if (l < p.n_prelude + p.n_rec) {
+    if (plane >= c.n_planes) return;           // the recurrences it has been through
+  } else {
+    if (plane >= p.n_classes || p.class_depth[plane] > c.n_planes) return;  // the readout depths it has reached
+  }
   __nv_bfloat16* base = p.kv + (size_t)l * p.layer_stride + (size_t)plane * p.plane_stride + (size_t)sel * p.sel_stride;
   const int per_head = p.d / 8;  // uint4 per head row
   for (int i = threadIdx.x; i < p.n_kv_heads * per_head; i += blockDim.x) {

@@ -74,6 +74,7 @@ struct GemmParams {
   int planes_ld;
   const float* gain_next;
   float* hid;             // RESID: residual stream [hid_idx][H]
+  int no_resid;           // RESID: the output REPLACES the stream (the adapter of a Raven-style model: H = W_a [H; e])
   float* sumsq_out;       // RESID: [row][n_sq_out]
   int n_sq_out;
   float* qbuf;            // QKV: [row][n_q_heads * d]
@@ -175,6 +176,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
         h_old = *h_ptr;
         if (p.out_planes) g_next = p.gain_next[rb * RBW + j];
       }
+      if (p.no_resid) h_old = 0.f;
     }
     float v = 0.f;
     if (live) {
@@ -680,13 +682,43 @@ struct PrepParams {
   const RowTable* tab;      // null: rows 0..m_fixed-1 of `x`
   int m_fixed;
   const float* x;           // stand-alone source [m][K]
-  const float* hid;         // row source [hid_idx][K]
+  float* hid;               // row source [hid_idx][K]
   int K;
   const float* gain;        // may be null
   __nv_bfloat16* planes;    // [col][3][K]
   float* sumsq;             // [col * sq_stride] full sum of squares (may be null)
   int sq_stride;
+  int use_src;              // rows with src_hid >= 0 are first copied from there (the copy is what the pass updates)
 };
+
+// ---- Raven-style recurrence input: the adapter reads [H; e] (Sec. 3.1 with P holding blocks: H0 = e = P(X), then
+// H <- B(W_a [H; e])).  Rows entering their first recurrence have H = e: their e is kept for the later recurrences. ----
+struct ConcatParams {
+  const RowTable* tab;
+  float* hid;               // [hid_idx][H] the rows' states
+  float* e_store;           // [hid_idx][H] the rows' prelude outputs
+  int H;
+  __nv_bfloat16* planes;    // [col][3][2 H]
+};
+__global__ void __launch_bounds__(256) raven_concat_kernel(const __grid_constant__ ConcatParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int c = blockIdx.x;
+  if (c >= p.tab->n_rows) return;
+  const int idx = p.tab->hid_idx[c];
+  const float* h = p.hid + (size_t)idx * p.H;
+  float* e = p.e_store + (size_t)idx * p.H;
+  const bool first = p.tab->r[c] == 1;
+  __nv_bfloat16* dst = p.planes + (size_t)c * 3 * 2 * p.H;
+  for (int k = threadIdx.x; k < p.H; k += blockDim.x) {
+    const float hv = h[k];
+    float ev = hv;
+    if (first) e[k] = hv;
+    else ev = e[k];
+    store_split(dst, 2 * p.H, k, hv);
+    store_split(dst, 2 * p.H, p.H + k, ev);
+  }
+}
 
 __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant__ PrepParams p) {
   __shared__ float s_part[8];
@@ -697,8 +729,10 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
   int n = p.tab ? p.tab->n_rows : p.m_fixed;
   if (c >= n) return;
   const float* src;
+  float* copy = nullptr;  // the pass works on a copy of another hidden state
   if (p.tab) {
     src = p.hid + (size_t)p.tab->hid_idx[c] * p.K;
+    if (p.use_src && p.tab->src_hid[c] >= 0) copy = p.hid + (size_t)p.tab->hid_idx[c] * p.K, src = p.hid + (size_t)p.tab->src_hid[c] * p.K;
   } else {
     src = p.x + (size_t)c * p.K;
   }
@@ -706,6 +740,7 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
   float ss = 0.f;
   for (int k = threadIdx.x; k < p.K; k += blockDim.x) {
     float v = src[k];
+    if (copy) copy[k] = v;
     ss += v * v;
     store_split(dst, p.K, k, p.gain ? v * p.gain[k] : v);
   }

@@ -182,12 +182,14 @@ int tc_pf_cols(int max_rows_pf) { return (max_rows_pf + 15) / 16 * 16; }
 
 struct Layout {  // byte offsets into the workspace
   size_t wpack, rope, kv, hid, qbuf, xplanes, aplanes, splanes, sumsq, logits, argpart, tcpart, flt, sel_flt, tv, tune, tune_bytes, apart, acnt, nodes, seqs, ctr, tab_dec, tab_pf,
-      tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
+      estore, cplanes, tab_pre, tab_coda, tab_pfc, tab_vanc, tab_van, sel_tok, sel_aux, sel_lse, sel_z2, kvcopy, out_ids, commits, trace, trace_n, prompt, total;
 };
 
 struct Derived {
   int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, sq_stride, max_chunks,
       trace_cap, Hq, Hkv, d1, d2;
+  // Raven-style layout (P and C hold transformer blocks): all layers in one list - prelude, recurrent, coda
+  int raven, n_pre, n_coda, NL, n_classes, class_depth[3], hid_coda_base;
 };
 
 int max_branches(int R, int d1, int d2) {
@@ -231,8 +233,8 @@ bool validate_model(const loopspec_model* m, int* why) {
       m->n_recurrent <= 0 || (m->weight_dtype != 0 && m->weight_dtype != 1) || !(m->rms_eps > 0) || !(m->rope_theta > 0))
     return false;
   if (m->n_q_heads % m->n_kv_heads) return false;
+  if (m->n_prelude < 0 || m->n_coda < 0) return false;
   *why = LOOPSPEC_EUNSUPPORTED;
-  if (m->n_prelude || m->n_coda) return false;
   if (m->head_dim != 64 && m->head_dim != 128) return false;
   int g = m->n_q_heads / m->n_kv_heads;
   if (g != 1 && g != 4) return false;
@@ -267,7 +269,13 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->max_rows = 8 * ng_for_rows(std::max(d->max_rows_dec, d->max_rows_pf));
   d->slots = s->max_ctx + d->NB;
   d->ids_cap = s->max_ctx;
-  d->n_hid = d->S * d->NB + MAX_ROWS;
+  d->n_pre = m->n_prelude, d->n_coda = m->n_coda, d->raven = (m->n_prelude || m->n_coda) ? 1 : 0;
+  d->NL = m->n_prelude + m->n_recurrent + m->n_coda;
+  d->n_classes = d->raven ? (d2 ? 3 : 2) : 0;  // coda caches: depth d1, depth d2 (if any), depth R
+  d->class_depth[0] = d1, d->class_depth[1] = d2 ? d2 : m->R, d->class_depth[2] = m->R;
+  if (d->raven && d->n_classes > m->R) return false;  // the pool gives every layer R planes
+  d->hid_coda_base = d->S * d->NB + MAX_ROWS;
+  d->n_hid = d->S * d->NB + MAX_ROWS + (d->raven ? MAX_ROWS : 0);  // branches, prefill rows, copies for the coda pass
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
   d->n_sq = m->hidden / 128;  // row blocks of the residual GEMMs = partial sums of squares per row
@@ -285,7 +293,7 @@ size_t packed_total_bytes(const loopspec_model* m, const Derived& d) {
   if (m->weight_dtype != 1) return 0;
   size_t per_layer = packed_bytes(d.Hq + 2 * d.Hkv, m->hidden) + packed_bytes(m->hidden, d.Hq) +
                      packed_bytes(2 * m->ffn, m->hidden) + packed_bytes(m->hidden, m->ffn);
-  return per_layer * m->n_recurrent + packed_bytes(m->vocab, m->hidden);
+  return per_layer * d.NL + packed_bytes(m->vocab, m->hidden) + (d.raven ? packed_bytes(m->hidden, 2 * m->hidden) : 0);
 }
 
 Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Derived& d) {
@@ -299,8 +307,10 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   const size_t MR = d.max_rows;
   L.wpack = take(packed_total_bytes(m, d));
   L.rope = take((size_t)s->max_ctx * (m->head_dim / 2) * sizeof(float2));
-  L.kv = take((size_t)m->n_recurrent * m->R * 2 * d.S * m->n_kv_heads * d.slots * m->head_dim * 2);
+  L.kv = take((size_t)d.NL * m->R * 2 * d.S * m->n_kv_heads * d.slots * m->head_dim * 2);
   L.hid = take((size_t)d.n_hid * m->hidden * 4);
+  L.estore = take(d.raven ? (size_t)d.n_hid * m->hidden * 4 : 0);
+  L.cplanes = take(d.raven ? MR * 3 * 2 * m->hidden * 2 : 0);
   L.qbuf = take(MR * d.Hq * 4);
   L.xplanes = take(MR * 3 * m->hidden * 2);
   L.aplanes = take(MR * 3 * d.Hq * 2);
@@ -330,6 +340,10 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.tv = take((size_t)MAX_ROWS * 4 * sizeof(double));
   L.tab_dec = take(sizeof(RowTable));
   L.tab_pf = take(sizeof(RowTable));
+  L.tab_pre = take(sizeof(RowTable));
+  L.tab_coda = take(sizeof(RowTable));
+  L.tab_pfc = take(sizeof(RowTable));
+  L.tab_vanc = take(sizeof(RowTable));
   L.tab_van = take(sizeof(RowTable) * m->R);
   L.sel_tok = take(MAX_ROWS * 4);
   L.sel_aux = take(MAX_ROWS * 4);
@@ -357,11 +371,12 @@ struct loopspec_ctx {
   const void* embed = nullptr;
   const void* lm_head = nullptr;
   const float* final_norm = nullptr;
-  std::vector<const void*> layers;  // 6 per layer
-  std::vector<const void*> packed;  // 4 per layer (qkv, o, gate/up, down) + lm_head; empty for fp32 weights
+  std::vector<const void*> layers;  // 6 per layer: prelude blocks, recurrent blocks, coda blocks
+  std::vector<const void*> packed;  // 4 per layer (qkv, o, gate/up, down), then lm_head, then the adapter; empty for fp32 weights
+  const void* adapter = nullptr;    // Raven-style layout: [H][2H]
   int n_sm = 148;
   int ng_dec = 1, ng_pf = 1;
-  GemmPlan plan[5];
+  GemmPlan plan[6];
   // prefill on the tcgen05 kernel: tensor maps of the row-major weights (4 per layer) and of the three plane buffers
   bool tc_pf = false;
   std::vector<CUtensorMap> tc_wmaps;
@@ -513,8 +528,13 @@ unsigned long long* tune_timeline(loopspec_ctx* c) {
 }
 
 // ---- one batched pass through the shared block stack (all layers) on the rows of `tab` ------------------
-enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_LM = 4 };
-const int kEpiOf[5] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS};
+enum { G_QKV = 0, G_O = 1, G_GU = 2, G_DOWN = 3, G_LM = 4, G_ADAPT = 5 };
+const int kEpiOf[6] = {EPI_QKV, EPI_RESID, EPI_SWIGLU, EPI_RESID, EPI_LOGITS, EPI_RESID};
+// `layer` is the index in the list prelude blocks | recurrent blocks | coda blocks
+bool first_of_stack(const Derived& d, int n_rec, int layer) { return layer == 0 || layer == d.n_pre || layer == d.n_pre + n_rec; }
+bool last_of_stack(const Derived& d, int n_rec, int layer) {
+  return layer == d.n_pre - 1 || layer == d.n_pre + n_rec - 1 || layer == d.NL - 1;
+}
 
 GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
   const loopspec_model& m = c->m;
@@ -525,14 +545,17 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.cluster_size = g.cs, p.n_clusters = g.n_clusters;
   p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
   p.err = c->host_flags_dev + HF_ERROR;
-  const void* const* lp = which == G_LM ? nullptr : &c->layers[6 * layer];
+  const void* const* lp = (which == G_LM || which == G_ADAPT) ? nullptr : &c->layers[6 * layer];
   __nv_bfloat16* xpl = c->at<__nv_bfloat16>(c->L.xplanes);
   switch (which) {
     case G_QKV:
       p.W = c->packed.empty() ? lp[1] : c->packed[4 * layer + 0], p.N = d.Hq + 2 * d.Hkv, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden;
-      // layer 0 reads the full sums the preparation kernel wrote; later layers the down-projection's partials
-      p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = layer == 0 ? 1 : d.n_sq, p.sq_stride = d.sq_stride;
+      // the first block of a stack reads the full sums its preparation kernel wrote (the recurrent blocks of a
+      // Raven-style model follow the adapter, which leaves partials like every other residual GEMM); later blocks
+      // read the down projection's partials
+      p.sumsq = c->at<float>(c->L.sumsq), p.sq_stride = d.sq_stride;
+      p.n_sq = (first_of_stack(d, m.n_recurrent, layer) && !(d.raven && layer == d.n_pre)) ? 1 : d.n_sq;
       if (!c->packed.empty() ) p.perm = 2, p.perm_a = m.head_dim / 32, p.perm_d = m.head_dim;
       p.qbuf = c->at<float>(c->L.qbuf);
       p.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)layer * c->kv_layer_stride();
@@ -560,10 +583,16 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       // planes for the next consumer of the residual stream: the next layer's first norm, or - after the last
       // layer - the final norm of the readout (the lm_head picks the reading-out rows out of them)
       p.out_planes = xpl, p.planes_ld = m.hidden;
-      p.gain_next = layer + 1 < m.n_recurrent ? static_cast<const float*>(c->layers[6 * (layer + 1)]) : c->final_norm;
+      p.gain_next = last_of_stack(d, m.n_recurrent, layer) ? c->final_norm : static_cast<const float*>(c->layers[6 * (layer + 1)]);
+      break;
+    case G_ADAPT:  // H <- W_a [H; e]: replaces the stream; leaves planes and sums of squares for the first recurrent block
+      p.W = c->packed.empty() ? c->adapter : c->packed[4 * d.NL + 1], p.N = m.hidden, p.K = 2 * m.hidden;
+      p.xplanes = c->at<__nv_bfloat16>(c->L.cplanes), p.x_ld = 2 * m.hidden, p.no_resid = 1;
+      p.sumsq_out = c->at<float>(c->L.sumsq), p.n_sq_out = d.sq_stride;
+      p.out_planes = xpl, p.planes_ld = m.hidden, p.gain_next = static_cast<const float*>(c->layers[6 * d.n_pre]);
       break;
     default:
-      p.W = c->packed.empty() ? c->lm_head : c->packed[4 * m.n_recurrent], p.N = m.vocab, p.K = m.hidden;
+      p.W = c->packed.empty() ? c->lm_head : c->packed[4 * d.NL], p.N = m.vocab, p.K = m.hidden;
       p.xplanes = xpl, p.x_ld = m.hidden, p.cols_from_readout = 1;
       // 1/rms from the partial sums of squares the last down projection left for the row
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.sq_stride;
@@ -573,11 +602,13 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   return p;
 }
 
-cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab) {
+// planes and sums of squares for the first block of a stack (`first_layer`); use_src: on copies of the rows' states
+cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, int first_layer = 0, bool use_src = false) {
   PrepParams q;
   memset(&q, 0, sizeof q);
   q.tab = tab, q.hid = c->at<float>(c->L.hid), q.K = c->m.hidden, q.planes = c->at<__nv_bfloat16>(c->L.xplanes);
-  q.gain = static_cast<const float*>(c->layers[0]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.sq_stride;
+  q.gain = static_cast<const float*>(c->layers[6 * first_layer]), q.sumsq = c->at<float>(c->L.sumsq), q.sq_stride = c->d.sq_stride;
+  q.use_src = use_src ? 1 : 0;
   return launch_k(prep_planes_kernel, dim3(c->d.max_rows), dim3(256), 0, c->stream, q, c->use_pdl);
 }
 
@@ -651,15 +682,14 @@ cudaError_t launch_dg_lm(loopspec_ctx* c, const RowTable* tab) {
   return launch_dg_raw(EPI_LOGITS, g, c->dg_wmap, c->dg_xmap, q, c->stream, c->use_pdl);
 }
 
-cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false) {
+// the blocks [l0, l0 + count) of the layer list on the rows of `tab`
+cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, int count, int* n_launch, bool tc) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
   const bool pdl = c->use_pdl;
   cudaError_t e;
-  if ((e = launch_prep(c, tab))) return e;
-  if (n_launch) *n_launch += 1;
-  for (int l = 0; l < m.n_recurrent; ++l) {
+  for (int l = l0; l < l0 + count; ++l) {
     unsigned long long* tl = tune_timeline(c);
     GemmParams gq = gemm_params(c, G_QKV, l, tab);
     gq.tl = tl, gq.tl_id = l * 5 + 0;
@@ -688,8 +718,44 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   return cudaSuccess;
 }
 
+// One batched pass of B over the rows of `tab` (Sec. 4.2 step 1).  Ouro layout: preparation + the shared blocks.
+// Raven-style layout: the rows entering their first recurrence (`tab_pre`, may be null) go through the prelude blocks,
+// then every row through the adapter on [H; e] and the recurrent blocks.
+cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false, const RowTable* tab_pre = nullptr) {
+  const loopspec_model& m = c->m;
+  const Derived& d = c->d;
+  cudaError_t e;
+  if (!d.raven) {
+    if ((e = launch_prep(c, tab))) return e;
+    if (n_launch) *n_launch += 1;
+    return launch_stack(c, tab, ng, 0, m.n_recurrent, n_launch, tc);
+  }
+  if (tab_pre && d.n_pre > 0) {
+    if ((e = launch_prep(c, tab_pre, 0))) return e;
+    if ((e = launch_stack(c, tab_pre, ng, 0, d.n_pre, n_launch, tc))) return e;
+    if (n_launch) *n_launch += 1;
+  }
+  ConcatParams cp;
+  cp.tab = tab, cp.hid = c->at<float>(c->L.hid), cp.e_store = c->at<float>(c->L.estore), cp.H = m.hidden;
+  cp.planes = c->at<__nv_bfloat16>(c->L.cplanes);
+  if ((e = launch_k(raven_concat_kernel, dim3(d.max_rows), dim3(256), 0, c->stream, cp, c->use_pdl))) return e;
+  if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_ADAPT, 0, tab), c->stream, c->use_pdl))) return e;
+  if (n_launch) *n_launch += 2;
+  return launch_stack(c, tab, ng, d.n_pre, m.n_recurrent, n_launch, tc);
+}
+
+// Raven-style layout: the post-layers' blocks on copies of the reading-out rows' states (`tab_coda`), writing the coda
+// cache of each row's readout depth; leaves the planes the lm_head reads
+cudaError_t launch_coda(loopspec_ctx* c, const RowTable* tab_coda, int ng, int* n_launch, bool tc = false) {
+  const Derived& d = c->d;
+  cudaError_t e;
+  if ((e = launch_prep(c, tab_coda, d.n_pre + c->m.n_recurrent, true))) return e;
+  if (n_launch) *n_launch += 1;
+  return launch_stack(c, tab_coda, ng, d.n_pre + c->m.n_recurrent, d.n_coda, n_launch, tc);
+}
+
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
-  if (c->dg && tab != c->at<RowTable>(c->L.tab_pf)) return launch_dg_lm(c, tab);
+  if (c->dg && tab != c->at<RowTable>(c->L.tab_pf) && tab != c->at<RowTable>(c->L.tab_pfc)) return launch_dg_lm(c, tab);
   GemmParams gl = gemm_params(c, G_LM, 0, tab);
   gl.tl = tune_timeline(c), gl.tl_id = 120;
   return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
@@ -724,6 +790,7 @@ ControlParams control_params(loopspec_ctx* c, int phases) {
   p.kvcopy = c->at<KvCopyCmd>(c->L.kvcopy);
   p.hid = c->at<float>(c->L.hid), p.H = c->m.hidden, p.embed = c->embed, p.weight_dtype = c->m.weight_dtype;
   p.p_logit_base = c->d.p_logit_base, p.host_flags = c->host_flags_dev;
+  if (c->d.raven) p.tab_pre = c->at<RowTable>(c->L.tab_pre), p.tab_coda = c->at<RowTable>(c->L.tab_coda), p.hid_coda_base = c->d.hid_coda_base;
   return p;
 }
 
@@ -735,8 +802,10 @@ cudaError_t launch_kv_commit(loopspec_ctx* c) {
   KvCommitParams k;
   k.cmds = c->at<KvCopyCmd>(c->L.kvcopy), k.kv = c->at<__nv_bfloat16>(c->L.kv);
   k.layer_stride = c->kv_layer_stride(), k.plane_stride = c->kv_plane_stride(), k.sel_stride = c->kv_sel_stride();
-  k.S = c->d.S, k.L = c->m.n_recurrent, k.n_kv_heads = c->m.n_kv_heads, k.slots = c->d.slots, k.d = c->m.head_dim;
-  dim3 grid(c->m.n_recurrent, c->m.R, 2 * c->d.S);
+  k.S = c->d.S, k.L = c->d.NL, k.n_kv_heads = c->m.n_kv_heads, k.slots = c->d.slots, k.d = c->m.head_dim;
+  k.n_prelude = c->d.n_pre, k.n_rec = c->m.n_recurrent, k.n_classes = c->d.n_classes;
+  for (int i = 0; i < 3; ++i) k.class_depth[i] = c->d.class_depth[i];
+  dim3 grid(c->d.NL, c->m.R, 2 * c->d.S);
   return launch_k(kv_commit_kernel, grid, dim3(128), 0, c->stream, k, c->use_pdl);
 }
 
@@ -744,8 +813,13 @@ cudaError_t launch_kv_commit(loopspec_ctx* c) {
 cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_commit, int* n_launch) {
   const RowTable* tab = c->at<RowTable>(c->L.tab_dec);
   cudaError_t e;
-  if ((e = launch_layers(c, tab, c->ng_dec, n_launch))) return e;
-  if ((e = launch_lm_head(c, tab, c->ng_dec))) return e;
+  if ((e = launch_layers(c, tab, c->ng_dec, n_launch, false, c->d.raven ? c->at<RowTable>(c->L.tab_pre) : nullptr))) return e;
+  const RowTable* tab_ro = tab;  // the rows the lm_head reads
+  if (c->d.raven && c->d.n_coda > 0) {
+    tab_ro = c->at<RowTable>(c->L.tab_coda);
+    if ((e = launch_coda(c, tab_ro, c->ng_dec, n_launch))) return e;
+  }
+  if ((e = launch_lm_head(c, tab_ro, c->ng_dec))) return e;
   if ((e = launch_select(c, tab, kinds_mask))) return e;
   if ((e = launch_control(c, phases))) return e;
   if (n_launch) *n_launch += 3;
@@ -764,15 +838,21 @@ VanillaParams vanilla_params(loopspec_ctx* c, int commit) {
   v.out_ids = c->at<int>(c->L.out_ids), v.ids_cap = c->d.ids_cap;
   v.hid = c->at<float>(c->L.hid), v.H = c->m.hidden, v.embed = c->embed, v.weight_dtype = c->m.weight_dtype;
   v.p_logit_base = c->d.p_logit_base, v.ctx_cap = c->s.max_ctx, v.host_flags = c->host_flags_dev;
+  if (c->d.raven && c->d.n_coda > 0) v.tab_coda = c->at<RowTable>(c->L.tab_vanc), v.hid_coda_base = c->d.hid_coda_base, v.n_classes = c->d.n_classes;
   return v;
 }
 
 cudaError_t launch_vanilla_token(loopspec_ctx* c) {
   cudaError_t e;
   RowTable* tabs = c->at<RowTable>(c->L.tab_van);
-  for (int r = 0; r < c->m.R; ++r)
-    if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr))) return e;
-  if ((e = launch_lm_head(c, tabs + c->m.R - 1, c->ng_dec))) return e;
+  for (int r = 0; r < c->m.R; ++r)  // every row enters recurrence 1 in the first pass: the prelude pass is that table itself
+    if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr, false, (c->d.raven && r == 0) ? tabs : nullptr))) return e;
+  const RowTable* tab_ro = tabs + c->m.R - 1;
+  if (c->d.raven && c->d.n_coda > 0) {
+    tab_ro = c->at<RowTable>(c->L.tab_vanc);
+    if ((e = launch_coda(c, tab_ro, c->ng_dec, nullptr))) return e;
+  }
+  if ((e = launch_lm_head(c, tab_ro, c->ng_dec))) return e;
   if ((e = launch_select(c, tabs + c->m.R - 1, 1 << RO_TARGET))) return e;
   return launch_k(vanilla_control_kernel, dim3(1), dim3(CTRL_THREADS), 0, c->stream, vanilla_params(c, 1), c->use_pdl);
 }
@@ -879,15 +959,17 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   Derived d;
   if (!validate_model(m, &why)) return why;
   if (!resolve_sched(m, s, &d, &why)) return why;
-  if (!w || !w->embed || !w->final_norm || !w->layer_ptrs || (!m->tied_lm_head && !w->lm_head) || w->adapter) return LOOPSPEC_EINVAL;
-  for (int i = 0; i < 6 * m->n_recurrent; ++i)
+  if (!w || !w->embed || !w->final_norm || !w->layer_ptrs || (!m->tied_lm_head && !w->lm_head)) return LOOPSPEC_EINVAL;
+  if ((d.raven != 0) != (w->adapter != nullptr)) return LOOPSPEC_EINVAL;  // the adapter belongs to the Raven-style layout
+  if (w->adapter && (reinterpret_cast<uintptr_t>(w->adapter) & 15)) return LOOPSPEC_EINVAL;
+  for (int i = 0; i < 6 * d.NL; ++i)
     if (!w->layer_ptrs[i]) return LOOPSPEC_EINVAL;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LOOPSPEC_EINVAL;
   // every tensor is read with 16-byte loads
   if ((reinterpret_cast<uintptr_t>(w->embed) & 15) || (w->lm_head && (reinterpret_cast<uintptr_t>(w->lm_head) & 15)) ||
       (reinterpret_cast<uintptr_t>(w->final_norm) & 15))
     return LOOPSPEC_EINVAL;
-  for (int i = 0; i < 6 * m->n_recurrent; ++i)
+  for (int i = 0; i < 6 * d.NL; ++i)
     if (reinterpret_cast<uintptr_t>(w->layer_ptrs[i]) & 15) return LOOPSPEC_EINVAL;
   if (!cuda_stream) return LOOPSPEC_EINVAL;  // the legacy default stream cannot be captured into a graph
   int dev = 0, n_sm = 0;
@@ -918,14 +1000,16 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   c->ws = static_cast<unsigned char*>(workspace);
   c->embed = w->embed, c->lm_head = m->tied_lm_head ? w->embed : w->lm_head;
   c->final_norm = static_cast<const float*>(w->final_norm);
-  c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * m->n_recurrent);
+  c->layers.assign(w->layer_ptrs, w->layer_ptrs + 6 * d.NL);
+  c->adapter = w->adapter;
   c->ng_dec = ng_for_rows(d.max_rows_dec), c->ng_pf = ng_for_rows(d.max_rows_pf);
   c->prefilled.assign(d.S, 0);
   const int resid_rows = 128;
-  const int n_rbs[5] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / resid_rows, (m->ffn + 63) / 64, m->hidden / resid_rows, (m->vocab + 127) / 128};
-  const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden};
+  const int n_rbs[6] = {(d.Hq + 2 * d.Hkv) / 128, m->hidden / resid_rows, (m->ffn + 63) / 64, m->hidden / resid_rows, (m->vocab + 127) / 128,
+                        m->hidden / resid_rows};
+  const int Ks[6] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden, 2 * m->hidden};
   int slots = n_sm * kCtasPerSm;
-  for (int i = 0; i < 5; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
+  for (int i = 0; i < 6; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
   // Every kernel of the chain asks for the same (largest) shared-memory carve-out: the GEMM CTAs need it, and an SM
   // whose partition was set by a small-shared-memory kernel would have to drain before it can host one.
   {
@@ -948,7 +1032,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   if (unsigned long long* tl = tune_timeline(c)) cudaMemcpyToSymbol(g_tune_tl, &tl, sizeof tl);
 #endif
   // cluster sizes that are not powers of two are used only if the device can co-schedule them
-  for (int i = 0; i < 5; ++i) {
+  for (int i = 0; i < 6; ++i) {
     GemmPlan& g = c->plan[i];
     if ((g.cs & (g.cs - 1)) == 0) continue;
     cudaLaunchConfig_t cfg;
@@ -975,8 +1059,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     const int Ns[4] = {dd.Hq + 2 * dd.Hkv, m->hidden, 2 * m->ffn, m->hidden}, Ks[4] = {m->hidden, dd.Hq, m->hidden, m->ffn};
     const int w_idx[4] = {1, 2, 4, 5};  // qkv, o, gate/up, down among a layer's six pointers
     bool ok = true;
-    c->tc_wmaps.resize((size_t)4 * m->n_recurrent);
-    for (int l = 0; l < m->n_recurrent && ok; ++l)
+    c->tc_wmaps.resize((size_t)4 * dd.NL);
+    for (int l = 0; l < dd.NL && ok; ++l)
       for (int i = 0; i < 4 && ok; ++i) ok = make_map_bf16(&c->tc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], TC_BM);
     const size_t x_off[3] = {c->L.xplanes, c->L.aplanes, c->L.splanes};
     const int x_k[3] = {m->hidden, dd.Hq, m->ffn};
@@ -1063,13 +1147,14 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       return cudaGetLastError() == cudaSuccess;
     };
     bool ok = true;
-    for (int l = 0; l < m->n_recurrent && ok; ++l) {
+    for (int l = 0; l < d.NL && ok; ++l) {
       const void* const* lp = &c->layers[6 * l];
       // rotary partners (QKV) and gate/up partners are stored as adjacent row tiles
       ok = pack(lp[1], d.Hq + 2 * d.Hkv, m->hidden, 2, m->head_dim / 32) && pack(lp[2], m->hidden, d.Hq) &&
            pack(lp[4], 2 * m->ffn, m->hidden, 1, m->ffn) && pack(lp[5], m->hidden, m->ffn);
     }
     ok = ok && pack(c->lm_head, m->vocab, m->hidden);
+    if (d.raven) ok = ok && pack(c->adapter, m->hidden, 2 * m->hidden);
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) return bail(LOOPSPEC_ECUDA, "weight repack");
   }
   // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
@@ -1114,15 +1199,24 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
       pp.tab = tab, pp.prompt = c->at<int>(c->L.prompt), pp.seq = seq, pp.p0 = p0, pp.count = cnt, pp.r = r, pp.R = c->m.R;
       pp.n_prompt = n, pp.hid_base = c->d.S * c->d.NB, pp.p_logit_base = c->d.p_logit_base;
       pp.hid = c->at<float>(c->L.hid), pp.H = c->m.hidden, pp.embed = c->embed, pp.weight_dtype = c->m.weight_dtype;
+      pp.tab_coda = nullptr, pp.coda_class = 0, pp.hid_coda_base = c->d.hid_coda_base;
+      if (c->d.raven && c->d.n_coda > 0) {  // the prompt fills the coda cache of every readout depth (App. B)
+        pp.tab_coda = c->at<RowTable>(c->L.tab_pfc);
+        for (int k = 0; k < c->d.n_classes; ++k)
+          if (c->d.class_depth[k] == r && pp.coda_class == 0) pp.coda_class = k + 1;
+        if (r == c->m.R) pp.coda_class = c->d.n_classes;
+      }
       prefill_setup_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(pp);
       CU(c, cudaGetLastError());
-      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf));
+      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf, (c->d.raven && r == 1) ? tab : nullptr));
+      if (pp.coda_class > 0) CU(c, launch_coda(c, pp.tab_coda, c->ng_pf, nullptr, c->tc_pf));
     }
   }
+  if (c->d.raven && c->d.n_coda > 0) tab = c->at<RowTable>(c->L.tab_pfc);  // its last state: last chunk, depth R
   CU(c, launch_lm_head(c, tab, c->ng_pf));
   CU(c, launch_select(c, tab, 1 << RO_TARGET));
   PrefillFinishParams fp;
-  fp.tab = tab, fp.nodes = c->nodes(), fp.seqs = c->seqs(), fp.seq = seq, fp.NB = c->d.NB, fp.n_prompt = n, fp.n_target = 0;
+  fp.tab = c->at<RowTable>(c->L.tab_pf), fp.nodes = c->nodes(), fp.seqs = c->seqs(), fp.seq = seq, fp.NB = c->d.NB, fp.n_prompt = n, fp.n_target = 0;
   fp.sel_tok = c->at<int>(c->L.sel_tok), fp.hid = c->at<float>(c->L.hid), fp.H = c->m.hidden, fp.embed = c->embed;
   fp.weight_dtype = c->m.weight_dtype, fp.host_flags = c->host_flags_dev;
   prefill_finish_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(fp);
@@ -1356,7 +1450,11 @@ int loopspec_debug_drop_tile(loopspec_ctx* c, int32_t unit, int32_t wait_us) {
 
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
-  *out = c->m.n_recurrent * 5 + 5;
+  const Derived& d = c->d;
+  int n = c->m.n_recurrent * 5 + 5;  // preparation, five kernels per block, lm_head, selection, control, KV commit
+  if (d.raven)  // prelude pass (preparation + blocks), concatenation + adapter instead of the preparation, coda pass
+    n = (d.n_pre ? 1 + 5 * d.n_pre : 0) + 2 + 5 * c->m.n_recurrent + (d.n_coda ? 1 + 5 * d.n_coda : 0) + 4;
+  *out = n;
   return LOOPSPEC_OK;
 }
 

@@ -24,7 +24,7 @@ def oracle_run(name, n_prompt, n_decode, d1, d2, T=0.0, seed=2, gate=True, resid
     shape = W.CONFIGS[name]
     dec = Decoder(oracle_model(name, wseed, gain_jitter), temperature=T, seed=seed, seq=seq, top_k=top_k, top_p=top_p)
     prompt = W.make_prompt(shape.vocab, n_prompt, seed=prompt_seed, seq=seq)
-    first = dec.prefill(prompt, n_decode)
+    first = dec.prefill(prompt, n_decode, depths=None if vanilla else (d1, d2))
     if vanilla:
         out, logits = dec.vanilla(n_decode, keep_logits=True)
         dec.verify_logits = logits

@@ -432,6 +432,35 @@ def test_error_paths_leave_the_context_usable():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,d1,d2,T,gate", [
+    ("tiny_raven_r4", 1, 2, 0.0, True), ("tiny_raven_r4", 1, 2, 1.0, True), ("tiny_raven_r4", 1, 3, 0.8, False),
+    ("tiny_raven_r4", 2, 0, 1.0, True), ("tiny_raven", 2, 8, 0.0, True), ("tiny_raven", 2, 8, 1.0, True),
+    ("tiny_raven", 4, 8, 1.0, False), ("tiny_raven", 2, 4, 0.7, True)])
+def test_raven_layout_matches_oracle(name, d1, d2, T, gate):
+    """Raven-style layout (Sec. 3.1: P and C hold transformer blocks; App. B: prelude cache, one coda cache per readout
+    depth): prelude pass for the rows entering their first recurrence, adapter on [state; prelude output], recurrent
+    blocks, coda pass on copies of the reading-out rows' states - tokens, decisions, counters and the stored proposal
+    logits as the oracle's; greedy LoopSpec equals vanilla decoding on the device."""
+    n_prompt, n_decode = 40, 24
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=5, gate=gate)
+    ctx = U.make_ctx(name, d1, d2, T=T, seed=5, gate=gate, max_ctx=n_prompt + n_decode + 24, max_prefill_rows=16)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    z0 = ref["dec"].first_logits      # 16 recurrences deep: the stated bf16 tolerance, not the tighter bound of the shallow models
+    assert (np.abs(ctx.debug_logits(0, 0) - z0) <= 3e-2 + 2e-2 * np.abs(z0)).all()
+    ctx.decode(n_decode)
+    U.assert_same_run(ctx, ref, n_decode)
+    st, ost = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total", "rows_max", "readout_rows_total"):
+        assert st[k] == ost[k], k
+    assert ctx.row_trace().tolist() == ref["dec"].rows_per_step
+    van = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=5, vanilla=True)
+    ctx.prefill(van["prompt"])
+    assert ctx.vanilla_decode(n_decode)[0].tolist() == van["tokens"]
+    if T == 0.0:
+        assert van["tokens"] == ref["tokens"]
+    ctx.close()
+
+
 def test_a_bounded_device_wait_that_runs_out_is_reported_and_survived():
     """Failure detection without a fault: a ring tile of the readout GEMM is never requested, so the MMA issuer's wait
     for it runs out after ~0.1 ms; the kernel raises its flag, carries on and ends; the call returns ETIMEOUT; after the

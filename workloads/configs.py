@@ -81,7 +81,7 @@ CONFIGS = {
                              ffn=2000, n_recurrent=3, R=4, weight_dtype="bf16", tied=False),
     # Raven layout at test size: prelude and coda blocks around the recurrent block, an adapter on [state; prelude output],
     # grouped-query attention with head size 64 (the head layout of the Raven-style benchmark config), R = 16
-    "tiny_raven": ModelShape("tiny_raven", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=1, head_dim=64,
+    "tiny_raven": ModelShape("tiny_raven", vocab=512, hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=64,
                              ffn=704, n_recurrent=2, R=16, weight_dtype="bf16", tied=False, n_prelude=1, n_coda=1),
     "tiny_raven_r4": ModelShape("tiny_raven_r4", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
                                 ffn=704, n_recurrent=2, R=4, weight_dtype="bf16", tied=False, n_prelude=2, n_coda=2),
