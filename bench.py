@@ -92,11 +92,22 @@ def step_bytes(shape, n_prompt, n_decode, stats):
     wb = 2 if shape.weight_dtype == "bf16" else 4
     h, f, d = shape.hidden, shape.ffn, shape.head_dim
     hq, hkv = shape.n_q_heads * d, shape.n_kv_heads * d
-    w_b = shape.n_recurrent * ((hq + 2 * hkv) * h + h * hq + 3 * f * h) * wb
+    block = ((hq + 2 * hkv) * h + h * hq + 3 * f * h) * wb
+    w_b = shape.n_recurrent * block
     w_c = shape.vocab * h * wb
     ctx = n_prompt + n_decode / 2.0
     kv_row = ctx * 2 * hkv * 2 * shape.n_recurrent
     steps = stats["steps"]
+    if shape.n_prelude or shape.n_coda:
+        # Raven-style layout: the adapter with every pass; the prelude blocks and the coda blocks + lm_head only in the
+        # passes that spawn / read out - every d1-th pass, because all branch depths are congruent modulo d1 (App. B
+        # "Depth Configuration"); their K/V reads are counted per reading-out row
+        w_b += 2 * h * h * wb
+        ro_passes = steps / max(stats.get("d1", 1), 1)
+        kv_ro = ctx * 2 * hkv * 2 * (shape.n_prelude + shape.n_coda)
+        total = steps * w_b + ro_passes * ((shape.n_prelude + shape.n_coda) * block + w_c) + stats["rows_total"] * kv_row + \
+            stats.get("readout_rows_total", 0) * kv_ro
+        return total, w_b, w_c + (shape.n_prelude + shape.n_coda) * block, kv_row
     return steps * w_b + steps * w_c + stats["rows_total"] * kv_row, w_b, w_c, kv_row
 
 
@@ -290,6 +301,7 @@ def run_ours(args):
     t_region = time.perf_counter() - t_region
     clocks = sampler.stop()
     stats = ctx.stats()
+    stats["d1"] = d1
     launches = ctx.launches_per_step() * stats["steps"] * args.steps
 
     # vanilla all-R decode from the same kernels (baseline of Fig. 1a)

@@ -63,8 +63,10 @@ typedef struct {
  * p_{d2} (-) p_{d1} (Eq. 5), 0 from p_{d2} itself.  temperature 0 = greedy.  max_prefill_rows (0 = default)
  * bounds how many prompt positions one prefill pass carries.
  * Capacity: max_ctx counts positions per sequence, the speculative ones included: a sequence needs
- * max_ctx >= prompt + decoded tokens + R/d1 + 2 (the deepest chain of uncommitted positions); R/d1 may not exceed 8 and
- * max_seqs times the branch bound of Sec. 4.3 may not exceed 64 rows (LOOPSPEC_ECAPACITY otherwise).
+ * max_ctx >= prompt + decoded tokens + R/d1 + 2 (the deepest chain of uncommitted positions); R/d1 may not exceed 16,
+ * max_seqs 64, and max_seqs times the branch bound of Sec. 4.3 256 rows per pass (LOOPSPEC_ECAPACITY otherwise; the bound
+ * for R = 32 with (d1, d2) = (2, 8) is 249).  Passes that can carry more than 64 rows run every GEMM once per group of 64
+ * rows, i.e. stream the weights once per group.
  * top_k, top_p: the optional filters of the post-layers C (Sec. 3.1), applied at EVERY readout depth when
  * temperature > 0: tokens are ranked by decreasing probability (ties: lower index first); top_k > 0 keeps the first
  * top_k and renormalises; 0 < top_p < 1 then keeps the shortest prefix of the ranking whose mass reaches top_p and

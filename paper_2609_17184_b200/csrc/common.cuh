@@ -15,8 +15,11 @@ constexpr bool kTune = true;
 constexpr bool kTune = false;
 #endif
 
-constexpr int MAX_ROWS = 64;  // rows (branches) one batched pass can carry: 8 token columns x up to 8 groups
-constexpr int MAX_SPEC = 8;   // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
+constexpr int MAX_ROWS = 256; // rows (branches) one batched pass can carry (Sec. 4.3: the branch bound for R = 32 with
+                              // (d1, d2) = (2, 8) is 249); the GEMMs take them in groups of up to 64 token columns
+constexpr int GROUP_ROWS = 64;  // token columns one GEMM launch carries
+constexpr int MAX_SEQS = 64;  // sequences a context can hold
+constexpr int MAX_SPEC = 16;  // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
 constexpr int ATT_CHUNK = 64; // key positions per attention chunk (cut at fixed absolute positions)
 constexpr int ATT_MAX_RUNS = 40;  // attention work items per (row, kv head) at most (contexts up to 2560: one chunk each)
 constexpr int ATT_LONG_RUNS = 8;  // ... and for contexts of more than ATT_MAX_RUNS chunks

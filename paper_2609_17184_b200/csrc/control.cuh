@@ -178,14 +178,25 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
   t.n_rows = n_rows, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
 }
 
+// dynamic shared memory of control_kernel: the branch table, the row table and the per-row selection results
+struct ControlSmem {
+  NodeSmem nd;
+  RowTable t;
+  int emb[2 * MAX_ROWS][2];
+  int sel_tok[MAX_ROWS], sel_aux[MAX_ROWS];
+  float sel_lse[MAX_ROWS], sel_z2[MAX_ROWS];
+};
+
 __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_constant__ ControlParams p) {
-  __shared__ NodeSmem nd;
-  __shared__ RowTable t;
-  __shared__ int s_root[MAX_ROWS], s_nids[MAX_ROWS], s_ndec[MAX_ROWS], s_ntarget[MAX_ROWS], s_needv[MAX_ROWS];
-  __shared__ int s_emb[2 * MAX_ROWS][2];
+  extern __shared__ __align__(16) unsigned char ctrl_smem_raw[];
+  ControlSmem& sm = *reinterpret_cast<ControlSmem*>(ctrl_smem_raw);
+  NodeSmem& nd = sm.nd;
+  RowTable& t = sm.t;
+  int (*s_emb)[2] = sm.emb;
+  int *s_sel_tok = sm.sel_tok, *s_sel_aux = sm.sel_aux;
+  float *s_sel_lse = sm.sel_lse, *s_sel_z2 = sm.sel_z2;
+  __shared__ int s_root[MAX_SEQS], s_nids[MAX_SEQS], s_ndec[MAX_SEQS], s_ntarget[MAX_SEQS], s_needv[MAX_SEQS];
   __shared__ int s_nemb, s_err;
-  __shared__ int s_sel_tok[MAX_ROWS], s_sel_aux[MAX_ROWS];
-  __shared__ float s_sel_lse[MAX_ROWS], s_sel_z2[MAX_ROWS];
   __shared__ unsigned long long s_steps;
   __shared__ int s_trace_n;
   const int tid = threadIdx.x;
@@ -195,8 +206,8 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
   // Everything the serial bookkeeping reads is pulled into shared memory with one round of parallel loads.  The branch
   // table, the row table and the sequence state were last written by the previous step, so they are read while this
   // step's readout kernels are still running; only the selection results have to wait for them.
-  if (tid == MAX_ROWS) s_steps = p.ctr->steps;
-  if (tid == MAX_ROWS + 1) s_trace_n = *p.trace_n;
+  if (tid == CTRL_THREADS - 1) s_steps = p.ctr->steps;
+  if (tid == CTRL_THREADS - 2) s_trace_n = *p.trace_n;
   nodes_load(nd, p.nodes, n_nodes);
   {
     const int* src = reinterpret_cast<const int*>(p.tab);
@@ -208,9 +219,9 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
     s_ntarget[tid] = p.seqs.n_target[tid], s_needv[tid] = p.seqs.need_verify[tid];
   }
   pdl_wait();
-  if (tid < MAX_ROWS) {
-    s_sel_tok[tid] = p.sel_tok[tid], s_sel_aux[tid] = p.sel_aux[tid];
-    s_sel_lse[tid] = p.sel_lse[tid], s_sel_z2[tid] = p.sel_z2[tid];
+  for (int i = tid; i < MAX_ROWS; i += CTRL_THREADS) {
+    s_sel_tok[i] = p.sel_tok[i], s_sel_aux[i] = p.sel_aux[i];
+    s_sel_lse[i] = p.sel_lse[i], s_sel_z2[i] = p.sel_z2[i];
   }
   if (tid == 0) s_nemb = 0, s_err = 0;
   __syncthreads();
@@ -347,8 +358,8 @@ struct VanillaParams {
 };
 
 __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __grid_constant__ VanillaParams p) {
-  __shared__ int s_emb[MAX_ROWS][2];
-  __shared__ int s_rowof[MAX_ROWS];
+  __shared__ int s_emb[MAX_SEQS][2];
+  __shared__ int s_rowof[MAX_SEQS];
   __shared__ int s_n;
   const int tid = threadIdx.x;
   pdl_launch_dependents();

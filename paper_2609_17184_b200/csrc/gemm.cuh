@@ -62,6 +62,8 @@ struct GemmParams {
   int x_ld;
   const RowTable* tab;
   int m_fixed;            // tab == nullptr: number of rows of a stand-alone call
+  int col0;               // first column (row of the pass, or reading-out row) this launch carries: passes wider than one
+                          // launch's columns run as several launches; the per-column buffers below are offset by the host
   int cols_from_readout;  // columns are the reading-out rows (lm_head)
   // fused RMSNorm: scale column c by 1/sqrt(sum_j sumsq[c*sq_stride + j] / H + eps); sumsq == nullptr: none
   const float* sumsq;
@@ -287,10 +289,10 @@ __device__ __forceinline__ void gemm_load_cols(const GemmParams& p, int n_cols, 
   const int c = threadIdx.x;
   const RowTable* tab = p.tab;
   if (tab && c < n_cols) {
-    const int row = p.cols_from_readout ? tab->ro_rows[c] : c;
+    const int row = p.cols_from_readout ? tab->ro_rows[p.col0 + c] : p.col0 + c;
     ct[CT_POS * ntok + c] = tab->pos[row], ct[CT_R * ntok + c] = tab->r[row], ct[CT_SEQ * ntok + c] = tab->seq[row];
     ct[CT_SLOT * ntok + c] = tab->kv_slot[row], ct[CT_HID * ntok + c] = tab->hid_idx[row], ct[CT_LOGIT * ntok + c] = tab->logit_idx[row];
-    ct[CT_XROW * ntok + c] = row;  // where the column's activation planes and sums of squares live
+    ct[CT_XROW * ntok + c] = row;  // where a reading-out column's activation planes and sums of squares live
   }
 }
 
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) __maxnreg__(NG == 1 ? LS_MAXREG 
 
   // the row table was written before this pass started, so the live row count can be read ahead of the predecessor
   const RowTable* tab = p.tab;
-  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
+  int n_cols = (tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed) - p.col0;
   if (n_cols > NTOK) n_cols = NTOK;
   gemm_load_cols(p, n_cols, NTOK, s_ct);
   // the weights above are constants; everything below reads what earlier kernels of the pass produced
@@ -572,7 +574,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_f32_kernel(const __grid_con
   pdl_launch_dependents();
   pdl_wait();
   const RowTable* tab = p.tab;
-  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed;
+  int n_cols = (tab ? (p.cols_from_readout ? tab->n_readout : tab->n_rows) : p.m_fixed) - p.col0;
   if (n_cols > NTOK) n_cols = NTOK;
   if (n_cols <= 0) return;
   gemm_load_cols(p, n_cols, NTOK, s_ct);

@@ -179,6 +179,16 @@ __global__ void __launch_bounds__(DG_THREADS) dgemm_kernel(const __grid_constant
 
   pdl_launch_dependents();
   tune_mark(p.tl_id, false);
+  // the row table of a pass is final before the pass starts: read ahead of the predecessor
+  const RowTable* tab = p.tab;
+  int n_rows = tab ? tab->n_rows : p.m_fixed;          // rows of the pass = live MMA columns
+  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : n_rows) : p.m_fixed;  // columns this GEMM finishes
+  if (n_rows > MP) n_rows = MP;
+  if (n_cols > MP) n_cols = MP;
+  if (n_cols <= 0) {  // uniform over the grid: nothing reads out in this pass - nothing is requested, nothing allocated
+    pdl_wait();     // (a kernel that ended before its predecessor would release its own dependents too early)
+    return;
+  }
 
   int kb_lo, kb_hi;
   gemm_krange((p.K + TC_BK - 1) / TC_BK, cs, rank, kb_lo, kb_hi);
@@ -229,12 +239,6 @@ __global__ void __launch_bounds__(DG_THREADS) dgemm_kernel(const __grid_constant
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // the row table of a pass is final before the pass starts: read ahead of the predecessor
-  const RowTable* tab = p.tab;
-  int n_rows = tab ? tab->n_rows : p.m_fixed;          // rows of the pass = live MMA columns
-  int n_cols = tab ? (p.cols_from_readout ? tab->n_readout : n_rows) : p.m_fixed;  // columns this GEMM finishes
-  if (n_rows > MP) n_rows = MP;
-  if (n_cols > MP) n_cols = MP;
   if (warp < 4) {
     if (tid < DG_MAX_COLS) s_colof[tid] = (!p.cols_from_readout && tid < n_cols) ? tid : -1;
     gemm_load_cols(p, n_cols, DG_MAX_COLS, s_ct);
@@ -246,16 +250,6 @@ __global__ void __launch_bounds__(DG_THREADS) dgemm_kernel(const __grid_constant
   const unsigned tmem = s_tmem;
   if (cs > 1) cluster.sync();  // every rank's barriers exist before anybody arrives on them remotely
   else __syncthreads();
-
-  if (n_cols <= 0) {  // uniform over the grid: nothing to compute; the copies already requested must land first
-    if (tid == 128)
-      for (int u = 0; u < pre; ++u)
-        if (!(dropper && u == q.drop_unit)) dg_wait(tc_smem_u32(&s_full[u]), 0, limit);
-    pdl_wait();
-    __syncthreads();
-    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
-    return;
-  }
 
   if (warp == 4) {
     if (lane < S) {

@@ -262,11 +262,14 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->B = max_branches(m->R, d1, d2);
   d->NB = 2 * d->B + 1;
   if (m->R / d1 > MAX_SPEC) return false;
-  if (d->S > MAX_ROWS || d->S * d->NB > MAX_NODES || d->S * d->B > MAX_ROWS) return false;
+  if (d->S > MAX_SEQS || d->S * d->NB > MAX_NODES || d->S * d->B > MAX_ROWS) return false;
   d->max_rows_dec = d->S * d->B;
   d->max_rows_pf = s->max_prefill_rows ? s->max_prefill_rows : 32;
-  if (d->max_rows_pf > MAX_ROWS) return false;
-  d->max_rows = 8 * ng_for_rows(std::max(d->max_rows_dec, d->max_rows_pf));
+  if (d->max_rows_pf > GROUP_ROWS) return false;
+  {  // rows of the pass buffers: one group of 8 / 16 / 32 / 64 token columns, or whole groups of 64
+    const int need = std::max(d->max_rows_dec, d->max_rows_pf);
+    d->max_rows = need <= GROUP_ROWS ? 8 * ng_for_rows(need) : (need + GROUP_ROWS - 1) / GROUP_ROWS * GROUP_ROWS;
+  }
   d->slots = s->max_ctx + d->NB;
   d->ids_cap = s->max_ctx;
   d->n_pre = m->n_prelude, d->n_coda = m->n_coda, d->raven = (m->n_prelude || m->n_coda) ? 1 : 0;
@@ -274,14 +277,14 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->n_classes = d->raven ? (d2 ? 3 : 2) : 0;  // coda caches: depth d1, depth d2 (if any), depth R
   d->class_depth[0] = d1, d->class_depth[1] = d2 ? d2 : m->R, d->class_depth[2] = m->R;
   if (d->raven && d->n_classes > m->R) return false;  // the pool gives every layer R planes
-  d->hid_coda_base = d->S * d->NB + MAX_ROWS;
-  d->n_hid = d->S * d->NB + MAX_ROWS + (d->raven ? MAX_ROWS : 0);  // branches, prefill rows, copies for the coda pass
+  d->hid_coda_base = d->S * d->NB + GROUP_ROWS;
+  d->n_hid = d->S * d->NB + GROUP_ROWS + (d->raven ? MAX_ROWS : 0);  // branches, prefill rows, copies for the coda pass
   d->p_logit_base = d->S * d->NB * 2;
   d->n_logit_vecs = d->p_logit_base + d->S;
   d->n_sq = m->hidden / 128;  // row blocks of the residual GEMMs = partial sums of squares per row
   d->sq_stride = std::max(d->n_sq, 64);  // room for one partial per cluster of the persistent pass kernel
   d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
-  d->trace_cap = 4 * s->max_ctx + 64;
+  d->trace_cap = m->R * s->max_ctx + 64;  // a token can take R passes (restart)
   d->Hq = m->n_q_heads * m->head_dim;
   d->Hkv = m->n_kv_heads * m->head_dim;
   return true;
@@ -335,9 +338,9 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.nodes = take((size_t)13 * MAX_NODES * 4);
   L.flt = take((size_t)2 * MAX_NODES * sizeof(float4));
   L.sel_flt = take((size_t)MAX_ROWS * sizeof(float4));
-  L.seqs = take((size_t)5 * MAX_ROWS * 4);
+  L.seqs = take((size_t)5 * MAX_SEQS * 4);
   L.ctr = take(sizeof(Counters));
-  L.tv = take((size_t)MAX_ROWS * 4 * sizeof(double));
+  L.tv = take((size_t)MAX_SEQS * 4 * sizeof(double));
   L.tab_dec = take(sizeof(RowTable));
   L.tab_pf = take(sizeof(RowTable));
   L.tab_pre = take(sizeof(RowTable));
@@ -349,7 +352,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sel_aux = take(MAX_ROWS * 4);
   L.sel_lse = take(MAX_ROWS * 4);
   L.sel_z2 = take(MAX_ROWS * 4);
-  L.kvcopy = take(MAX_ROWS * sizeof(KvCopyCmd));
+  L.kvcopy = take(MAX_SEQS * sizeof(KvCopyCmd));
   L.out_ids = take((size_t)d.S * d.ids_cap * 4);
   L.commits = take((size_t)d.S * d.ids_cap * 8 * 4);
   L.trace = take((size_t)d.trace_cap * 4);
@@ -422,7 +425,7 @@ struct loopspec_ctx {
   SeqState seqs() const {
     int* b = at<int>(L.seqs);
     SeqState q;
-    q.root = b, q.n_ids = b + MAX_ROWS, q.n_dec = b + 2 * MAX_ROWS, q.n_target = b + 3 * MAX_ROWS, q.need_verify = b + 4 * MAX_ROWS;
+    q.root = b, q.n_ids = b + MAX_SEQS, q.n_dec = b + 2 * MAX_SEQS, q.n_target = b + 3 * MAX_SEQS, q.need_verify = b + 4 * MAX_SEQS;
     return q;
   }
   long long kv_sel_stride() const { return (long long)d.S * m.n_kv_heads * d.slots * m.head_dim; }
@@ -536,7 +539,7 @@ bool last_of_stack(const Derived& d, int n_rec, int layer) {
   return layer == d.n_pre - 1 || layer == d.n_pre + n_rec - 1 || layer == d.NL - 1;
 }
 
-GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
+GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* tab, int col0 = 0) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   GemmParams p;
@@ -598,6 +601,18 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
       p.sumsq = c->at<float>(c->L.sumsq), p.n_sq = d.n_sq, p.sq_stride = d.sq_stride;
       p.logits = c->at<float>(c->L.logits), p.argpart = c->at<float2>(c->L.argpart);
       break;
+  }
+  if (col0 > 0) {  // a later group of token columns: its slices of the per-column buffers
+    p.col0 = col0;
+    if (which == G_LM) {
+      p.argpart += (size_t)col0 * p.n_rb;  // the planes and sums of squares are addressed by pass row, not by column
+    } else {
+      p.xplanes += (size_t)col0 * 3 * p.x_ld;
+      if (p.out_planes) p.out_planes += (size_t)col0 * 3 * p.planes_ld;
+      if (p.sumsq) p.sumsq += (size_t)col0 * p.sq_stride;
+      if (p.sumsq_out) p.sumsq_out += (size_t)col0 * p.n_sq_out;
+      if (p.qbuf) p.qbuf += (size_t)col0 * d.Hq;
+    }
   }
   return p;
 }
@@ -682,6 +697,13 @@ cudaError_t launch_dg_lm(loopspec_ctx* c, const RowTable* tab) {
   return launch_dg_raw(EPI_LOGITS, g, c->dg_wmap, c->dg_xmap, q, c->stream, c->use_pdl);
 }
 
+// launches a GEMM of a pass over `tab` takes: decode passes that can carry more than 64 rows run every GEMM once per group of
+// 64 token columns (a launch whose group holds no row returns at once); prefill passes carry at most 64 rows
+int col_groups(loopspec_ctx* c, const RowTable* tab) {
+  if (tab == c->at<RowTable>(c->L.tab_pf) || tab == c->at<RowTable>(c->L.tab_pfc)) return 1;
+  return (c->d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;
+}
+
 // the blocks [l0, l0 + count) of the layer list on the rows of `tab`
 cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, int count, int* n_launch, bool tc) {
   const loopspec_model& m = c->m;
@@ -689,11 +711,21 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
   const int G = m.n_q_heads / m.n_kv_heads;
   const bool pdl = c->use_pdl;
   cudaError_t e;
+  const int groups = col_groups(c, tab);
+  // a GEMM of the pass: one launch per group of token columns (one group unless a decode pass can carry more than 64 rows)
+  auto gemm = [&](int which, int l, int tl_id) -> cudaError_t {
+    if (tc) return launch_tc_gemm(c, which, l, tab);
+    for (int g = 0; g < groups; ++g) {
+      GemmParams gp = gemm_params(c, which, l, tab, g * GROUP_ROWS);
+      gp.tl = tune_timeline(c), gp.tl_id = tl_id;
+      cudaError_t e2 = launch_gemm(m.weight_dtype, ng, kEpiOf[which], gp, c->stream, pdl);
+      if (e2) return e2;
+    }
+    return cudaSuccess;
+  };
   for (int l = l0; l < l0 + count; ++l) {
     unsigned long long* tl = tune_timeline(c);
-    GemmParams gq = gemm_params(c, G_QKV, l, tab);
-    gq.tl = tl, gq.tl_id = l * 5 + 0;
-    if ((e = tc ? launch_tc_gemm(c, G_QKV, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_QKV, gq, c->stream, pdl))) return e;
+    if ((e = gemm(G_QKV, l, l * 5 + 0))) return e;
     AttnParams a;
     memset(&a, 0, sizeof a);
     a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
@@ -704,16 +736,10 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
     a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
     a.tl = tl, a.tl_id = l * 5 + 1;
     if ((e = launch_k(attn_fn(m.head_dim, G, d.max_chunks > ATT_MAX_RUNS), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
-    GemmParams go = gemm_params(c, G_O, l, tab);
-    go.tl = tl, go.tl_id = l * 5 + 2;
-    if ((e = tc ? launch_tc_gemm(c, G_O, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_RESID, go, c->stream, pdl))) return e;
-    GemmParams gg = gemm_params(c, G_GU, l, tab);
-    gg.tl = tl, gg.tl_id = l * 5 + 3;
-    if ((e = tc ? launch_tc_gemm(c, G_GU, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_SWIGLU, gg, c->stream, pdl))) return e;
-    GemmParams gd = gemm_params(c, G_DOWN, l, tab);
-    gd.tl = tl, gd.tl_id = l * 5 + 4;
-    if ((e = tc ? launch_tc_gemm(c, G_DOWN, l, tab) : launch_gemm(m.weight_dtype, ng, EPI_RESID, gd, c->stream, pdl))) return e;
-    if (n_launch) *n_launch += 5;
+    if ((e = gemm(G_O, l, l * 5 + 2))) return e;
+    if ((e = gemm(G_GU, l, l * 5 + 3))) return e;
+    if ((e = gemm(G_DOWN, l, l * 5 + 4))) return e;
+    if (n_launch) *n_launch += 1 + 4 * (tc ? 2 : groups);
   }
   return cudaSuccess;
 }
@@ -739,8 +765,10 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   cp.tab = tab, cp.hid = c->at<float>(c->L.hid), cp.e_store = c->at<float>(c->L.estore), cp.H = m.hidden;
   cp.planes = c->at<__nv_bfloat16>(c->L.cplanes);
   if ((e = launch_k(raven_concat_kernel, dim3(d.max_rows), dim3(256), 0, c->stream, cp, c->use_pdl))) return e;
-  if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_ADAPT, 0, tab), c->stream, c->use_pdl))) return e;
-  if (n_launch) *n_launch += 2;
+  const int groups = col_groups(c, tab);
+  for (int g = 0; g < groups; ++g)
+    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_ADAPT, 0, tab, g * GROUP_ROWS), c->stream, c->use_pdl))) return e;
+  if (n_launch) *n_launch += 1 + groups;
   return launch_stack(c, tab, ng, d.n_pre, m.n_recurrent, n_launch, tc);
 }
 
@@ -756,9 +784,14 @@ cudaError_t launch_coda(loopspec_ctx* c, const RowTable* tab_coda, int ng, int* 
 
 cudaError_t launch_lm_head(loopspec_ctx* c, const RowTable* tab, int ng) {
   if (c->dg && tab != c->at<RowTable>(c->L.tab_pf) && tab != c->at<RowTable>(c->L.tab_pfc)) return launch_dg_lm(c, tab);
-  GemmParams gl = gemm_params(c, G_LM, 0, tab);
-  gl.tl = tune_timeline(c), gl.tl_id = 120;
-  return launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
+  const int groups = col_groups(c, tab);
+  for (int g = 0; g < groups; ++g) {
+    GemmParams gl = gemm_params(c, G_LM, 0, tab, g * GROUP_ROWS);
+    gl.tl = tune_timeline(c), gl.tl_id = 120;
+    cudaError_t e = launch_gemm(c->m.weight_dtype, ng, EPI_LOGITS, gl, c->stream, c->use_pdl);
+    if (e) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) {
@@ -795,7 +828,7 @@ ControlParams control_params(loopspec_ctx* c, int phases) {
 }
 
 cudaError_t launch_control(loopspec_ctx* c, int phases) {
-  return launch_k(control_kernel, dim3(1), dim3(CTRL_THREADS), 0, c->stream, control_params(c, phases), c->use_pdl);
+  return launch_k(control_kernel, dim3(1), dim3(CTRL_THREADS), sizeof(ControlSmem), c->stream, control_params(c, phases), c->use_pdl);
 }
 
 cudaError_t launch_kv_commit(loopspec_ctx* c) {
@@ -1020,6 +1053,10 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       if (cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
         (void)cudaGetLastError();
   }
+  if (cudaFuncSetAttribute(control_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ControlSmem)) != cudaSuccess) {
+    delete c;
+    return LOOPSPEC_ECUDA;
+  }
   for (int ng : {c->ng_dec, c->ng_pf})
     if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
@@ -1159,7 +1196,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   }
   // clear everything after the KV pool's predecessor tables: scratch counters must start at zero, tables idle
   if (cudaMemsetAsync(c->ws + L.acnt, 0, L.total - L.acnt, c->stream) != cudaSuccess ||
-      cudaMemsetAsync(c->ws + L.seqs, 0xff, (size_t)MAX_ROWS * 4, c->stream) != cudaSuccess ||  // root = -1
+      cudaMemsetAsync(c->ws + L.seqs, 0xff, (size_t)MAX_SEQS * 4, c->stream) != cudaSuccess ||  // root = -1
       cudaStreamSynchronize(c->stream) != cudaSuccess)
     return bail(LOOPSPEC_ECUDA, "workspace clear");
   *out = c;
@@ -1223,7 +1260,7 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
   CU(c, cudaGetLastError());
   // statistics and traces restart with the sequence set
   CU(c, cudaMemsetAsync(c->ws + c->L.ctr, 0, sizeof(Counters), c->stream));
-  CU(c, cudaMemsetAsync(c->ws + c->L.tv, 0, (size_t)MAX_ROWS * 4 * sizeof(double), c->stream));
+  CU(c, cudaMemsetAsync(c->ws + c->L.tv, 0, (size_t)MAX_SEQS * 4 * sizeof(double), c->stream));
   CU(c, cudaMemsetAsync(c->ws + c->L.trace_n, 0, 4, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   c->prefilled[seq] = 1;
@@ -1234,9 +1271,9 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
 
 // set every prefilled sequence's target to n more tokens and (re)build the decode rows
 static int arm_decode(loopspec_ctx* c, int n_tokens, bool unlimited = false) {
-  std::vector<int> ndec(MAX_ROWS), nids(MAX_ROWS), tgt(MAX_ROWS, 0);
-  CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
-  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  std::vector<int> ndec(MAX_SEQS), nids(MAX_SEQS), tgt(MAX_SEQS, 0);
+  CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   // Positions a sequence can reach: its committed ids, the tokens asked for (a manual step commits at most one) and
   // the deepest chain of uncommitted drafts, R/d1; the scheduler wants two more below max_ctx.  Checked here, before
@@ -1250,8 +1287,8 @@ static int arm_decode(loopspec_ctx* c, int n_tokens, bool unlimited = false) {
                   want, spec_depth, c->s.max_ctx);
     tgt[s] = unlimited ? c->d.ids_cap : ndec[s] + n_tokens;
   }
-  memcpy(c->pin_ids, tgt.data(), MAX_ROWS * 4);
-  CU(c, cudaMemcpyAsync(c->seqs().n_target, c->pin_ids, MAX_ROWS * 4, cudaMemcpyHostToDevice, c->stream));
+  memcpy(c->pin_ids, tgt.data(), MAX_SEQS * 4);
+  CU(c, cudaMemcpyAsync(c->seqs().n_target, c->pin_ids, MAX_SEQS * 4, cudaMemcpyHostToDevice, c->stream));
   if (c->vanilla_mode) {  // drop back from vanilla decoding: the root restarts at depth 0
     vanilla_control_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(vanilla_params(c, 0));
     CU(c, cudaGetLastError());
@@ -1285,12 +1322,12 @@ int loopspec_verify(loopspec_ctx* c, loopspec_commit* out, int32_t max_out, int3
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (!c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "no branch is at depth R");
   if (max_out < 0 || (max_out > 0 && !out)) return fail(c, LOOPSPEC_EINVAL, "bad output array");
-  std::vector<int> before(MAX_ROWS), after(MAX_ROWS);
-  CU(c, cudaMemcpyAsync(before.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  std::vector<int> before(MAX_SEQS), after(MAX_SEQS);
+  CU(c, cudaMemcpyAsync(before.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, launch_select(c, c->at<RowTable>(c->L.tab_dec), 1 << RO_VERIFY));
   CU(c, launch_control(c, PH_VERIFY | PH_BUILD));
   CU(c, launch_kv_commit(c));
-  CU(c, cudaMemcpyAsync(after.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(after.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   c->pending_verify = false;
   int n = 0;
@@ -1326,15 +1363,15 @@ int loopspec_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
   if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
   if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "decode before prefill");
   if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
-  std::vector<int> start(MAX_ROWS);
-  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  std::vector<int> start(MAX_SEQS);
+  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
   int rc = arm_decode(c, n_tokens);
   if (rc) return rc;
   if (!c->g_step && (rc = capture(c, &c->g_step, false))) return rc;
   // every commit needs at least d1 more passes, so `remaining * d1` replays can never overshoot
-  std::vector<int> ndec(MAX_ROWS);
+  std::vector<int> ndec(MAX_SEQS);
   for (;;) {
-    CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(c, cudaMemcpyAsync(ndec.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
     if ((rc = check_device_error(c))) return rc;
     int remaining = 0;
@@ -1357,9 +1394,9 @@ int loopspec_vanilla_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out)
   if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
   if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "decode before prefill");
   if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
-  std::vector<int> start(MAX_ROWS), nids(MAX_ROWS);
-  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
-  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_ROWS * 4, cudaMemcpyDeviceToHost, c->stream));
+  std::vector<int> start(MAX_SEQS), nids(MAX_SEQS);
+  CU(c, cudaMemcpyAsync(start.data(), c->seqs().n_dec, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(nids.data(), c->seqs().n_ids, MAX_SEQS * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   for (int s = 0; s < c->d.S; ++s)  // no drafts here: the last position is committed ids + n_tokens - 1, two more must fit
     if (c->prefilled[s] && ((long long)nids[s] + n_tokens + 2 > c->s.max_ctx || (long long)start[s] + n_tokens > c->d.ids_cap))
@@ -1385,7 +1422,7 @@ int loopspec_get_stats(loopspec_ctx* c, loopspec_stats* out) {
   out->rows_total = k.rows_total, out->rows_max = k.rows_max, out->readout_rows_total = k.readout_rows_total;
   double den = (double)k.n_accept1 * c->d.d1 + (double)k.n_accept2 * c->d.d2 + (double)k.n_restart * c->m.R;
   out->gamma = den > 0 ? (double)k.n_decode * c->m.R / den : 0.0;  // Sec. 6 "Implementation and Metrics", definition of gamma
-  double tv[MAX_ROWS * 4];
+  double tv[MAX_SEQS * 4];
   CU(c, cudaMemcpy(tv, c->ws + c->L.tv, sizeof tv, cudaMemcpyDeviceToHost));
   double s1 = 0, n1 = 0, s2 = 0, n2 = 0;
   for (int s = 0; s < c->d.S; ++s) s1 += tv[4 * s], n1 += tv[4 * s + 1], s2 += tv[4 * s + 2], n2 += tv[4 * s + 3];
@@ -1451,9 +1488,11 @@ int loopspec_debug_drop_tile(loopspec_ctx* c, int32_t unit, int32_t wait_us) {
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
   const Derived& d = c->d;
-  int n = c->m.n_recurrent * 5 + 5;  // preparation, five kernels per block, lm_head, selection, control, KV commit
+  const int g = (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;  // launches per GEMM (groups of 64 token columns)
+  const int per_block = 1 + 4 * g, lm = c->dg ? 1 : g;            // attention + four GEMMs
+  int n = 1 + c->m.n_recurrent * per_block + lm + 3;               // preparation, blocks, lm_head, selection, control, KV commit
   if (d.raven)  // prelude pass (preparation + blocks), concatenation + adapter instead of the preparation, coda pass
-    n = (d.n_pre ? 1 + 5 * d.n_pre : 0) + 2 + 5 * c->m.n_recurrent + (d.n_coda ? 1 + 5 * d.n_coda : 0) + 4;
+    n = (d.n_pre ? 1 + per_block * d.n_pre : 0) + 1 + g + per_block * c->m.n_recurrent + (d.n_coda ? 1 + per_block * d.n_coda : 0) + lm + 3;
   *out = n;
   return LOOPSPEC_OK;
 }

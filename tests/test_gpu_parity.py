@@ -461,6 +461,30 @@ def test_raven_layout_matches_oracle(name, d1, d2, T, gate):
     ctx.close()
 
 
+@pytest.mark.parametrize("name,d1,d2,T,gate", [("tiny_r32", 2, 8, 1.0, False), ("tiny_raven_r32", 2, 8, 1.0, True),
+                                                ("tiny_r32", 2, 10, 1.0, True), ("tiny_r32", 4, 8, 0.0, True)])
+def test_thirty_two_recurrences_with_hundreds_of_rows_per_pass(name, d1, d2, T, gate):
+    """The Raven family's loop count, R = 32, with the paper's depth pairs (2, 8) and (2, 10) (Sec. 4.3 "Gating Mechanism":
+    up to B = 249 branches; appendix on the effective batch size: observed peaks of 176-239 rows): passes of up to 249 rows
+    (GEMMs in groups of 64 token columns), chains of up to 16 uncommitted positions - tokens, decisions, row counts per
+    pass and counters as the oracle's."""
+    import paper_2609_17184_b200 as ls
+    n_prompt, n_decode = 24, 16
+    ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=5, gate=gate)
+    ctx = U.make_ctx(name, d1, d2, T=T, seed=5, gate=gate, max_ctx=n_prompt + n_decode + 40, max_prefill_rows=16)
+    assert ctx.prefill(ref["prompt"]) == ref["first"]
+    ctx.decode(n_decode)
+    U.assert_same_run(ctx, ref, n_decode)
+    st, ost = ctx.stats(), ref["dec"].stats
+    for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total", "rows_max", "readout_rows_total"):
+        assert st[k] == ost[k], k
+    assert ctx.row_trace().tolist() == ref["dec"].rows_per_step
+    assert st["rows_max"] <= ls.max_branches(32, d1, d2)
+    if (d1, d2, gate) == (2, 8, False):
+        assert st["rows_max"] == 249 == ls.max_branches(32, 2, 8)     # the bound of Sec. 4.3 is reached
+    ctx.close()
+
+
 def test_a_bounded_device_wait_that_runs_out_is_reported_and_survived():
     """Failure detection without a fault: a ring tile of the readout GEMM is never requested, so the MMA issuer's wait
     for it runs out after ~0.1 ms; the kernel raises its flag, carries on and ends; the call returns ETIMEOUT; after the

@@ -76,6 +76,11 @@ CONFIGS = {
                           ffn=704, n_recurrent=2, R=8, weight_dtype="bf16", tied=False),
     "tiny_r16": ModelShape("tiny_r16", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
                            ffn=704, n_recurrent=1, R=16, weight_dtype="bf16", tied=False),
+    # the Raven family's loop count: R = 32, where (d1, d2) = (2, 8) allows up to 249 branches in a pass (Sec. 4.3)
+    "tiny_r32": ModelShape("tiny_r32", vocab=512, hidden=256, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                           ffn=704, n_recurrent=1, R=32, weight_dtype="bf16", tied=False),
+    "tiny_raven_r32": ModelShape("tiny_raven_r32", vocab=512, hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=64,
+                                 ffn=704, n_recurrent=1, R=32, weight_dtype="bf16", tied=False, n_prelude=1, n_coda=1),
     # a mid-size bf16 model whose GEMMs span several tiles, K-slices and a ragged last tile
     "small_bf16": ModelShape("small_bf16", vocab=4000, hidden=768, n_q_heads=6, n_kv_heads=6, head_dim=128,
                              ffn=2000, n_recurrent=3, R=4, weight_dtype="bf16", tied=False),
