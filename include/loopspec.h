@@ -248,7 +248,13 @@ int loopspec_time_linear_tc(const void* const* Ws, int32_t n_w, const float* x, 
  *   - Sizes: loopspec_linear_scratch_bytes(M, N, K) must not exceed 16 MiB (roughly N*K <= 8M bf16 weights);
  *     larger requests return LOOPSPEC_ECAPACITY and do nothing.  Bad shapes return LOOPSPEC_EINVAL.
  *   - The first call on each device looks up the array's device address (with that device current); make that
- *     first call outside any stream capture.  Later calls only launch kernels on cuda_stream.
+ *     first call outside any stream capture.  Later calls only launch kernels on cuda_stream.  With lazy module
+ *     loading that first call is also when the library's device image -- the 16 MiB array with it -- becomes
+ *     resident on the device: make it BEFORE the process's pool reserves the device's memory (a warm-up call on a
+ *     small shape is enough); made afterwards it can return LOOPSPEC_ECUDA for lack of memory.
+ *   - The array is the CURRENT device's (cudaGetDevice at the time of the call): cuda_stream, W, x and y must
+ *     belong to that device.  Nothing checks this; a stream or pointer of another device gives a CUDA error or
+ *     wrong results.  The first-call look-up is safe to race from several host threads.
  *   - All calls on a device share the one array, which keeps whatever the previous call left there.  Nothing in
  *     it has to start at zero: every call overwrites the part it reads.  Two calls that overlap on the GPU (different
  *     streams, or threads racing on one stream's ordering) overwrite each other's scratch and give wrong results:

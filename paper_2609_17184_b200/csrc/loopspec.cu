@@ -2,6 +2,7 @@
 // sequence of one batched pass, CUDA-graph capture of the decode step and the host side of the scheduler.
 #include "../../include/loopspec.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -1589,19 +1590,22 @@ static __device__ __align__(256) unsigned char g_static_scratch[LOOPSPEC_STATIC_
 
 int loopspec_op_linear_static(const void* W, int32_t weight_dtype, const float* x, float* y, int32_t M, int32_t N, int32_t K,
                               void* cuda_stream) {
-  static void* scratch_of_device[64] = {nullptr};
+  // one slot per device; the address of a device symbol never changes, so two threads racing on a first call store
+  // the same value and the atomic only makes the publication well defined
+  static std::atomic<void*> scratch_of_device[64];
   size_t need = loopspec_linear_scratch_bytes(M, N, K);
   if (!need) return LOOPSPEC_EINVAL;
   if (need > LOOPSPEC_STATIC_SCRATCH_BYTES) return LOOPSPEC_ECAPACITY;  // beyond the built-in scratch: use loopspec_op_linear
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOOPSPEC_ECUDA;
-  void* ptr = scratch_of_device[dev];
-  if (!ptr) {  // first call on this device (it is the current one): resolve the array's device address
+  void* ptr = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!ptr) {  // first call on this device (it is the current one): resolve the array's device address; this is
+               // also the moment the library's device image, the 16 MiB array included, becomes resident there
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
       (void)cudaGetLastError();
       return LOOPSPEC_ECUDA;
     }
-    scratch_of_device[dev] = ptr;
+    scratch_of_device[dev].store(ptr, std::memory_order_release);
   }
   return loopspec_op_linear(W, weight_dtype, x, y, M, N, K, ptr, LOOPSPEC_STATIC_SCRATCH_BYTES, cuda_stream);
 }

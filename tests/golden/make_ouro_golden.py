@@ -1,5 +1,5 @@
 """Writes tests/golden/ouro_1p4b_oracle.json: what the float64 oracle decodes on the Ouro-1.4B-shaped model
-(BASELINE config 1: prompt 512, greedy, (d1, d2) = (1, 2), gate on) for the first tokens of the run, the same
+(the headline workload: prompt 512, greedy, (d1, d2) = (1, 2), gate on) for the first tokens of the run, the same
 with temperature-1 sampling, and the same with the paper's sampling setting (temperature 1, top-p 0.7).  Calls only
 `oracle/` and the seeded input generators.  Takes ~15 minutes and ~20 GB.  Runs already in the file are kept
 (they are deterministic); pass --force to recompute them.

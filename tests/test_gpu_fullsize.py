@@ -1,4 +1,4 @@
-"""Full-size parity on the Ouro-1.4B-shaped model (BASELINE config 1), in the launch configuration bench.py times.
+"""Full-size parity on the Ouro-1.4B-shaped model (the headline workload: prompt 512, 512 greedy tokens), in the launch configuration bench.py times.
 
 The oracle cannot decode 512 tokens of a 1.4B model in test time, so:
   * the first tokens of the run (greedy, temperature 1, temperature 1 with top-p 0.7) are compared with values the

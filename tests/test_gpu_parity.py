@@ -77,7 +77,7 @@ def test_linear_tc_rejects_unsupported_shapes():
 
 # ---- end-to-end parity -------------------------------------------------------------------------------
 GREEDY_CASES = [
-    ("tiny", 16, 64, 1, 0, True),            # BASELINE config 0 as given
+    ("tiny", 16, 64, 1, 0, True),            # the small greedy workload (16-token prompt, 64 tokens, d1 = 1, no second proposal)
     ("tiny", 16, 40, 1, 2, True),
     ("tiny", 9, 30, 2, 0, True),
     ("tiny_bf16", 16, 64, 1, 2, True),
@@ -250,29 +250,42 @@ def test_filtered_sampling_matches_oracle(name, n_prompt, n_decode, d1, d2, T, t
     ctx.close()
 
 
+# runs of the seed sweep whose closest decision in the oracle is below the 1e-5 threshold (found by running the oracle
+# alone): greedy tiny_bf16 with (d1, d2) = (1, 2), seed 4, a gate score 1.9e-6 from its threshold at position 37
+NEAR_TIES = {("tiny_bf16", 1, 2, 0.0, 0, 1.0): {4}}
+
+
 @pytest.mark.parametrize("name,n_prompt,n_decode,d1,d2,T,top_k,top_p", [
     ("tiny_bf16", 11, 40, 1, 2, 0.0, 0, 1.0), ("tiny_bf16", 16, 40, 1, 2, 1.0, 0, 1.0), ("tiny_bf16", 9, 40, 2, 0, 0.9, 0, 0.7),
     ("tiny", 16, 40, 1, 3, 1.1, 30, 0.9), ("small_bf16", 33, 24, 1, 2, 1.0, 0, 1.0)])
 def test_parity_holds_across_seeds(name, n_prompt, n_decode, d1, d2, T, top_k, top_p):
-    """Not one lucky seed: eight prompt / sampling seeds per setting, tokens and counters equal to the oracle's."""
-    undecidable = 0
+    """Not one lucky seed: eight prompt / sampling seeds per setting, tokens and counters equal to the oracle's.
+
+    A run whose closest decision in the oracle has a margin below 1e-5 cannot be compared decision by decision: fp32
+    logits (error ~3e-5 here) do not resolve it, and either outcome is a correct execution of the step.  Such runs
+    are listed by name in NEAR_TIES (the list is checked, so none is passed over silently) and still run on the
+    device: the tokens before the tied position must agree, and under greedy decoding the whole stream must, because
+    the output of a lossless scheme does not depend on what a gate or a proposal decided."""
+    seen = set()
     for seed in range(1, 9):
         ref = U.oracle_run(name, n_prompt, n_decode, d1, d2, T=T, seed=seed, prompt_seed=seed + 10, top_k=top_k, top_p=top_p)
-        if min(e["margin"] for e in ref["dec"].log if e["kind"] != "filter") < 1e-5:
-            # a decision closer than fp32 logits resolve (their error is ~3e-5 here): either outcome is a correct
-            # fp32 execution of the same step, so the run cannot be compared decision by decision
-            undecidable += 1
-            continue
+        decisions = sorted((e["margin"], e["kind"], e.get("pos", -1)) for e in ref["dec"].log if e["kind"] != "filter")
         ctx = U.make_ctx(name, d1, d2, T=T, seed=seed, max_ctx=n_prompt + n_decode + 8, top_k=top_k, top_p=top_p)
         assert ctx.prefill(ref["prompt"]) == ref["first"], seed
         out = ctx.decode(n_decode)[0].tolist()
-        margins = sorted((e["margin"], e["kind"]) for e in ref["dec"].log if e["kind"] != "filter")[:3]
-        assert out == ref["tokens"], (seed, U.first_diff(out, ref["tokens"]), margins)
+        if decisions[0][0] < 1e-5:
+            seen.add(seed)
+            tie_pos = min(pos for m, _, pos in decisions if m < 1e-5)
+            keep = n_decode if T == 0.0 else max(0, tie_pos - n_prompt - 2)
+            assert out[:keep] == ref["tokens"][:keep], (seed, U.first_diff(out, ref["tokens"]), decisions[:3])
+            ctx.close()
+            continue
+        assert out == ref["tokens"], (seed, U.first_diff(out, ref["tokens"]), decisions[:3])
         st, so = ctx.stats(), ref["dec"].stats
         for k in ("steps", "n_accept1", "n_accept2", "n_restart", "gate_evals", "gate_opens", "rows_total"):
             assert st[k] == so[k], (seed, k, st[k], so[k])
         ctx.close()
-    assert undecidable <= 1
+    assert seen == NEAR_TIES.get((name, d1, d2, T, top_k, top_p), set()), seen
 
 
 @pytest.mark.parametrize("name,gate,top_p", [("tiny_bf16", True, 1.0), ("tiny_bf16", False, 1.0), ("small_bf16", False, 0.8)])

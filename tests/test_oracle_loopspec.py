@@ -219,7 +219,7 @@ class ScriptedModel:
     def embed_tokens(self, ids):
         return np.array([[float(t), 0.0] for t in ids])
 
-    def advance_rows(self, X, pos, prefix_kv):
+    def advance_rows(self, X, pos, prefix_kv, E=None):
         X = np.array(X, dtype=np.float64)
         X[:, 1] += 1
         return X, [[] for _ in pos]
