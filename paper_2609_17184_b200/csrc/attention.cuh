@@ -10,6 +10,13 @@
 
 namespace ls {
 
+// 16-byte asynchronous copy into shared memory; !valid: the 16 bytes are zero-filled and nothing is read
+__device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, bool valid) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+  const int n = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(n) : "memory");
+}
+
 constexpr int ATT_THREADS = 256;  // 8 warps per work item; at most 64 registers per thread so that the
                                    // neighbouring GEMM kernels' CTAs can be resident (and prefetching) alongside
 
@@ -267,38 +274,56 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_kernel(const __grid_const
 }
 
 // The same attention for contexts of more than ATT_MAX_RUNS chunks: a work item is a run of consecutive chunks (a
-// function of the row's own context only), folded one after the other with the usual softmax rescaling, so that the
-// per-item costs (row lookup, partial write, counter) are paid once per run and a (row, kv head) never has more than
-// ATT_MAX_RUNS partials.  Kept apart from attn_kernel, whose single-chunk items are the ones the batch-1 decode uses.
+// function of the row's own context only), so that the per-item costs (row lookup, partial write, counter) are paid
+// once per run and a (row, kv head) never has more than ATT_MAX_RUNS partials.  This is the kernel of the KV-bound
+// regime, built to stream: every thread owns a ring of (key piece, value piece) slots in shared memory that it fills
+// with cp.async and reads back itself, so the K/V of the next rounds are in flight while the current one is used and
+// the main loop has no block-wide barrier.  A key position is shared by the D/8 lanes of a group, 8 dims each (groups
+// of 4 lanes with D/4 dims each need fewer shuffles and softmax updates per byte but leave too few warps to hide
+// their longer dependent chains: 3.6 TB/s against 5.6 TB/s measured on 34 rows x 8192 positions).  Each lane group keeps
+// a running softmax (max, mass, weighted values) over the positions it is dealt - position j of a chunk always goes
+// to group j mod PPR - the groups of a warp are folded by a fixed butterfly, the warps in ascending order, once per
+// run.  Kept apart from attn_kernel, whose single-chunk items are the ones the batch-1 decode uses.
 template <int D, int G>
-__global__ void __launch_bounds__(ATT_THREADS, 4) attn_runs_kernel(const __grid_constant__ AttnParams p) {
-  constexpr int LPP = D / 8;            // lanes per key position (8 bf16 = 16 bytes per lane)
-  constexpr int PPW = 32 / LPP;         // positions per warp per load
-  constexpr int PPR = PPW * (ATT_THREADS / 32);  // positions per round of the whole CTA
-  constexpr int NPOS = ATT_CHUNK + MAX_SPEC;     // the last chunk of a row also carries its speculative slots
-  constexpr int ROUNDS = (NPOS + PPR - 1) / PPR;
-  constexpr int PSTRIDE = D + 2;
+struct AtsCfg {
+  static constexpr int NP = 1;                     // 16-byte pieces of a key (and of a value) per lane
+  static constexpr int DPL = 8 * NP;               // dims per lane
+  static constexpr int LPP = D / DPL;              // lanes per key position
+  static constexpr int PPW = 32 / LPP;             // positions per warp per round
+  static constexpr int PPR = PPW * (ATT_THREADS / 32);  // positions per round of the whole CTA
+  static constexpr int UNIT_BYTES = 2 * NP * ATT_THREADS * 16;  // one round of the CTA: K and V pieces of every thread
+  static constexpr int MIN_CTAS = G == 1 ? 4 : 2;  // per SM (grouped-query attention keeps G accumulators per lane)
+  static constexpr int UNITS = (G == 1 ? 48 : 96) * 1024 / UNIT_BYTES;  // ring depth: 48 KB in flight per CTA
+  static constexpr int COMB_BYTES = (ATT_THREADS / 32) * G * (D + 2) * 4;
+  static constexpr int SMEM_BYTES = UNITS * UNIT_BYTES + COMB_BYTES;
+};
 
-  __shared__ float s_score[G][ROUNDS * PPR];
-  __shared__ float s_red[ATT_THREADS / 32][G][D];
-  __shared__ float s_stat[G][2];
+template <int D, int G>
+__global__ void __launch_bounds__(ATT_THREADS, (AtsCfg<D, G>::MIN_CTAS)) attn_runs_kernel(const __grid_constant__ AttnParams p) {
+  using C = AtsCfg<D, G>;
+  constexpr int NP = C::NP, DPL = C::DPL, LPP = C::LPP, PPW = C::PPW, PPR = C::PPR, UNITS = C::UNITS;
+  constexpr int PSTRIDE = D + 2;
+  constexpr int EPT = (G * D + ATT_THREADS - 1) / ATT_THREADS;  // output elements (head, dim) a thread folds
+  constexpr unsigned PIECE = ATT_THREADS * 16, V_OFF = NP * PIECE, UNIT_BYTES = C::UNIT_BYTES, RING_BYTES = UNITS * UNIT_BYTES;
+
+  extern __shared__ __align__(16) unsigned char ats_smem[];
+  float* s_comb = reinterpret_cast<float*>(ats_smem + RING_BYTES);  // [warp][G][PSTRIDE]
   __shared__ int s_last;
 
-  int dbg_n = 0;
-  auto stamp = [&]() {
-    if (kTune && p.dbg && blockIdx.x == 0 && threadIdx.x == 0) p.dbg[dbg_n++] = clock64();
-  };
-  stamp();
   timeline_mark(p.tl, p.tl_id, false);
   const RowTable* tab = p.tab;   // written before this pass started: safe to read ahead of the predecessor
   const int n_rows = tab->n_rows;
   const int HQ = p.n_q_heads * D;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int sub = lane / LPP, dl = lane % LPP;  // which position of the warp's group, which 8-dim slice
+  const int sub = lane / LPP, dl = lane % LPP;  // which position of the warp's group, which DPL-dim slice
+  const int jl = warp * PPW + sub;              // this lane group's position within a round
   const int total = tab->attn_items * p.n_kv_heads;
+  const unsigned ring_s = (unsigned)__cvta_generic_to_shared(ats_smem) + tid * 16;
   bool waited = false;
 
-  constexpr int EPT = (G * D + ATT_THREADS - 1) / ATT_THREADS;  // output elements (head, dim) a thread folds
+  struct Cursor {  // a round of a chunk of the run, with the chunk's geometry
+    int chunk, rd, n_can, n_here, n_safe, rounds;
+  };
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     const int kvh = item % p.n_kv_heads;
     const int rr = item / p.n_kv_heads;
@@ -321,153 +346,202 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_runs_kernel(const __grid_
 
     const size_t plane = (size_t)(tab->r[row] - 1) * p.kv_plane_stride;
     const size_t headbase = (size_t)(tab->seq[row] * p.n_kv_heads + kvh) * p.slots * D;
-    const __nv_bfloat16* Kb = p.kv + plane + headbase;
-    const __nv_bfloat16* Vb = p.kv + plane + p.kv_sel_stride + headbase;
+    const __nv_bfloat16* Kb = p.kv + plane + headbase + dl * DPL;
+    const __nv_bfloat16* Vb = Kb + p.kv_sel_stride;
 
-    // running softmax state of the run, per output element of this thread: max, mass, weighted values
-    float run_m[EPT], run_l[EPT], run_a[EPT];
-    for (int chunk = chunk_lo; chunk < chunk_hi; ++chunk) {
+    auto setup = [&](Cursor& c, int chunk) {
       const int p0 = chunk * ATT_CHUNK;
-      const int n_can_here = min(ATT_CHUNK, n_canon - p0);
-      const int n_spec = (chunk == n_chunks - 1) ? row_spec : 0;
-      const int n_here = n_can_here + n_spec;
+      const int n_spec = (chunk == n_chunks - 1) ? row_spec : 0;  // the last chunk of a row also carries its speculative slots
+      c.chunk = chunk, c.rd = 0;
+      c.n_can = min(ATT_CHUNK, n_canon - p0);
+      c.n_here = c.n_can + n_spec;
       // positions below n_safe were cached by earlier passes; the others are written by this pass's QKV kernel
-      const int n_safe_can = min(n_can_here, max(0, row_safe - p0));
-      const int n_safe = (n_spec > 0) ? n_can_here + n_spec - 1 : n_safe_can;
-
-      auto slot_of = [&](int jpos) -> int { return jpos < n_can_here ? p0 + jpos : tab->spec_slot[row][jpos - n_can_here]; };
-      uint4 kreg[ROUNDS], vreg[ROUNDS];
-      auto load_kv = [&](int lo, int hi) {
+      c.n_safe = (n_spec > 0) ? c.n_can + n_spec - 1 : min(c.n_can, max(0, row_safe - p0));
+      c.rounds = (c.n_here + PPR - 1) / PPR;
+    };
+    auto advance = [&](Cursor& c) {
+      if (++c.rd == c.rounds) {
+        if (c.chunk + 1 < chunk_hi) setup(c, c.chunk + 1);
+        else c.chunk = chunk_hi;
+      }
+    };
+    // ---- ring, issue side: one unit = this thread's pieces of a key and of a value of one round ------------------
+    Cursor ic;
+    setup(ic, chunk_lo);
+    unsigned i_slot = 0, c_slot = 0;
+    auto issue = [&]() {
+      if (ic.chunk < chunk_hi) {
+        const int jpos = ic.rd * PPR + jl;
+        if (jpos < ic.n_here) {
+          const int slot = jpos < ic.n_can ? ic.chunk * ATT_CHUNK + jpos : tab->spec_slot[row][jpos - ic.n_can];
+          const size_t off = (size_t)slot * D;
 #pragma unroll
-        for (int rd = 0; rd < ROUNDS; ++rd) {
-          const int jpos = rd * PPR + warp * PPW + sub;
-          if (jpos >= lo && jpos < hi) {
-            const size_t off = (size_t)slot_of(jpos) * D + dl * 8;
-            kreg[rd] = *reinterpret_cast<const uint4*>(Kb + off);
-            vreg[rd] = *reinterpret_cast<const uint4*>(Vb + off);
+          for (int pc = 0; pc < NP; ++pc) {
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + i_slot + pc * PIECE), "l"(Kb + off + pc * 8) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_s + i_slot + V_OFF + pc * PIECE), "l"(Vb + off + pc * 8)
+                         : "memory");
           }
         }
-      };
-#pragma unroll
-      for (int rd = 0; rd < ROUNDS; ++rd) kreg[rd] = vreg[rd] = make_uint4(0, 0, 0, 0);
-      stamp();
-      load_kv(0, n_safe);
-      stamp();
-      if (!waited) {
-        pdl_launch_dependents();
-        pdl_wait();
-        waited = true;
-        timeline_mark(p.tl, p.tl_id + 256, false);
+        advance(ic);
       }
-      stamp();
-      load_kv(n_safe, n_here);
+      i_slot += UNIT_BYTES;
+      if (i_slot == RING_BYTES) i_slot = 0;
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int issued = 0;
+    if (!waited) {
+      // rounds whose positions were all cached by earlier passes are requested ahead of the predecessor's completion
+      while (issued < UNITS - 1 && ic.chunk < chunk_hi && min((ic.rd + 1) * PPR, ic.n_here) <= ic.n_safe) issue(), ++issued;
+      pdl_launch_dependents();
+      pdl_wait();
+      waited = true;
+      timeline_mark(p.tl, p.tl_id + 256, false);
+    }
+    for (; issued < UNITS - 1; ++issued) issue();
 
-      float q[G][8];  // (re-read for every chunk of a run: a cache hit, and it keeps the registers free in between)
+    float q[G][DPL];
+#pragma unroll
+    for (int gq = 0; gq < G; ++gq) {
+      const float4* qp =
+          reinterpret_cast<const float4*>(p.qbuf + (size_t)row * p.n_q_heads * D + (size_t)(kvh * G + gq) * D + dl * DPL);
+#pragma unroll
+      for (int i = 0; i < DPL / 4; ++i) {
+        const float4 a = qp[i];
+        q[gq][4 * i] = a.x, q[gq][4 * i + 1] = a.y, q[gq][4 * i + 2] = a.z, q[gq][4 * i + 3] = a.w;
+      }
+    }
+
+    // ---- main loop: running softmax of this lane group over its positions of the run ----------------------------
+    float gm[G], gl[G], o[G][DPL];
+#pragma unroll
+    for (int gq = 0; gq < G; ++gq) {
+      gm[gq] = -INFINITY, gl[gq] = 0.f;
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) o[gq][i] = 0.f;
+    }
+    auto lds128 = [](unsigned addr) {
+      uint4 v;
+      asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+      return v;
+    };
+    Cursor cc;
+    setup(cc, chunk_lo);
+    while (cc.chunk < chunk_hi) {
+      issue();
+      asm volatile("cp.async.wait_group %0;" ::"n"(UNITS - 1) : "memory");
+      const bool valid = cc.rd * PPR + jl < cc.n_here;
+      float sc[G];
+#pragma unroll
+      for (int gq = 0; gq < G; ++gq) sc[gq] = 0.f;
+#pragma unroll
+      for (int pc = 0; pc < NP; ++pc) {  // one chain per piece, folded in piece order
+        const uint4 kk = valid ? lds128(ring_s + c_slot + pc * PIECE) : make_uint4(0, 0, 0, 0);
+        const unsigned kw[4] = {kk.x, kk.y, kk.z, kk.w};
+        float sp[G];
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq) sp[gq] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float k0 = __uint_as_float(kw[i] << 16), k1 = __uint_as_float(kw[i] & 0xffff0000u);
+#pragma unroll
+          for (int gq = 0; gq < G; ++gq) sp[gq] = fmaf(q[gq][pc * 8 + 2 * i + 1], k1, fmaf(q[gq][pc * 8 + 2 * i], k0, sp[gq]));
+        }
+#pragma unroll
+        for (int gq = 0; gq < G; ++gq) sc[gq] += sp[gq];
+      }
+      float wb[G];
 #pragma unroll
       for (int gq = 0; gq < G; ++gq) {
-        const float4* qp =
-            reinterpret_cast<const float4*>(p.qbuf + (size_t)row * p.n_q_heads * D + (size_t)(kvh * G + gq) * D + dl * 8);
-        float4 a = qp[0], b = qp[1];
-        q[gq][0] = a.x, q[gq][1] = a.y, q[gq][2] = a.z, q[gq][3] = a.w;
-        q[gq][4] = b.x, q[gq][5] = b.y, q[gq][6] = b.z, q[gq][7] = b.w;
-      }
-      __syncthreads();  // shared buffers of the previous chunk are free
-      stamp();
-
-      // ---- scores ------------------------------------------------------------------------------------
 #pragma unroll
-      for (int rd = 0; rd < ROUNDS; ++rd) {
-        const int jpos = rd * PPR + warp * PPW + sub;
-        const unsigned w[4] = {kreg[rd].x, kreg[rd].y, kreg[rd].z, kreg[rd].w};
-        float kf[8];
+        for (int off = LPP / 2; off > 0; off >>= 1) sc[gq] += __shfl_xor_sync(0xffffffffu, sc[gq], off);  // (every lane takes part)
+        wb[gq] = 0.f;
+        if (valid) {
+          const float sv = sc[gq] * p.scale;
+          if (sv > gm[gq]) {  // a new maximum: rescale what has been gathered (the first position finds -inf: weight 0)
+            const float wa = expf(gm[gq] - sv);
+            gl[gq] *= wa;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          kf[2 * i] = __uint_as_float(w[i] << 16);
-          kf[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-#pragma unroll
-        for (int gq = 0; gq < G; ++gq) {
-          float s = 0.f;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) s = fmaf(q[gq][i], kf[i], s);
-#pragma unroll
-          for (int o = LPP / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-          if (dl == 0) s_score[gq][jpos] = (jpos < n_here) ? s * p.scale : -INFINITY;
+            for (int i = 0; i < DPL; ++i) o[gq][i] *= wa;
+            gm[gq] = sv;
+          }
+          wb[gq] = expf(sv - gm[gq]);
+          gl[gq] += wb[gq];
         }
       }
-      __syncthreads();
-      stamp();
-
-      // ---- chunk softmax statistics (one warp per query head, round robin) ----------------------------
-      for (int gq = warp; gq < G; gq += ATT_THREADS / 32) {
-        float m = -INFINITY;
-        for (int jj = lane; jj < ROUNDS * PPR; jj += 32) m = fmaxf(m, s_score[gq][jj]);
-        m = warp_max(m);
-        float l = 0.f;
-        for (int jj = lane; jj < ROUNDS * PPR; jj += 32) {
-          float e = (jj < n_here) ? expf(s_score[gq][jj] - m) : 0.f;
-          s_score[gq][jj] = e;
-          l += e;
-        }
-        l = warp_sum(l);
-        if (lane == 0) s_stat[gq][0] = m, s_stat[gq][1] = l;
-      }
-      __syncthreads();
-      stamp();
-
-      // ---- weighted values ----------------------------------------------------------------------------
-      float o[G][8];
+      if (valid) {
 #pragma unroll
-      for (int gq = 0; gq < G; ++gq)
+        for (int pc = 0; pc < NP; ++pc) {
+          const uint4 vv = lds128(ring_s + c_slot + V_OFF + pc * PIECE);
+          const unsigned vw[4] = {vv.x, vv.y, vv.z, vv.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) o[gq][i] = 0.f;
+          for (int i = 0; i < 4; ++i) {
+            const float v0 = __uint_as_float(vw[i] << 16), v1 = __uint_as_float(vw[i] & 0xffff0000u);
 #pragma unroll
-      for (int rd = 0; rd < ROUNDS; ++rd) {
-        const int jpos = rd * PPR + warp * PPW + sub;
-        const unsigned w[4] = {vreg[rd].x, vreg[rd].y, vreg[rd].z, vreg[rd].w};
-        float vf[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          vf[2 * i] = __uint_as_float(w[i] << 16);
-          vf[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-#pragma unroll
-        for (int gq = 0; gq < G; ++gq) {
-          float pw = s_score[gq][jpos];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) o[gq][i] = fmaf(pw, vf[i], o[gq][i]);
-        }
-      }
-      // fold the PPW position groups of the warp, then the warps, in fixed order
-#pragma unroll
-      for (int gq = 0; gq < G; ++gq)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float v = o[gq][i];
-#pragma unroll
-          for (int off = LPP; off < 32; off <<= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-          if (sub == 0) s_red[warp][gq][dl * 8 + i] = v;
-        }
-      __syncthreads();
-      stamp();
-
-      // ---- fold the chunk into the run: the first chunk is taken as it is, later ones by the usual rescaling ------
-#pragma unroll
-      for (int e = 0; e < EPT; ++e) {
-        const int idx = tid + e * ATT_THREADS;
-        if (idx < G * D) {
-          const int gq = idx / D, dd = idx % D;
-          float v = 0.f;
-#pragma unroll
-          for (int w2 = 0; w2 < ATT_THREADS / 32; ++w2) v += s_red[w2][gq][dd];
-          const float m_c = s_stat[gq][0], l_c = s_stat[gq][1];
-          if (chunk == chunk_lo) {
-            run_m[e] = m_c, run_l[e] = l_c, run_a[e] = v;
-          } else {
-            const float mn = fmaxf(run_m[e], m_c), wa = expf(run_m[e] - mn), wb = expf(m_c - mn);
-            run_a[e] = fmaf(run_a[e], wa, v * wb), run_l[e] = fmaf(run_l[e], wa, l_c * wb), run_m[e] = mn;
+            for (int gq = 0; gq < G; ++gq) {
+              o[gq][pc * 8 + 2 * i] = fmaf(wb[gq], v0, o[gq][pc * 8 + 2 * i]);
+              o[gq][pc * 8 + 2 * i + 1] = fmaf(wb[gq], v1, o[gq][pc * 8 + 2 * i + 1]);
+            }
           }
         }
+      }
+      c_slot += UNIT_BYTES;
+      if (c_slot == RING_BYTES) c_slot = 0;
+      advance(cc);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");  // (only empty groups are left)
+
+    // ---- fold the lane groups of a warp: a butterfly in which the lower lane's state always comes first ---------
+#pragma unroll
+    for (int off = LPP; off < 32; off <<= 1) {
+      const bool upper = (lane & off) != 0;
+#pragma unroll
+      for (int gq = 0; gq < G; ++gq) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, gm[gq], off), l2 = __shfl_xor_sync(0xffffffffu, gl[gq], off);
+        const float ma = upper ? m2 : gm[gq], mb = upper ? gm[gq] : m2;  // a: the lower lane's state
+        const float la = upper ? l2 : gl[gq], lb = upper ? gl[gq] : l2;
+        const float mn = fmaxf(ma, mb);
+        const float wa = ma == -INFINITY ? 0.f : expf(ma - mn), wb2 = mb == -INFINITY ? 0.f : expf(mb - mn);
+        gl[gq] = fmaf(la, wa, lb * wb2), gm[gq] = mn;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) {
+          const float o2 = __shfl_xor_sync(0xffffffffu, o[gq][i], off);
+          const float oa = upper ? o2 : o[gq][i], ob = upper ? o[gq][i] : o2;
+          o[gq][i] = fmaf(oa, wa, ob * wb2);
+        }
+      }
+    }
+    // ---- ... and the warps in ascending order -----------------------------------------------------------------
+    __syncthreads();  // the previous item's readers are done with s_comb
+    if (sub == 0) {
+#pragma unroll
+      for (int gq = 0; gq < G; ++gq) {
+        float* dst = s_comb + ((size_t)warp * G + gq) * PSTRIDE;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) dst[dl * DPL + i] = o[gq][i];
+        if (dl == 0) dst[D] = gm[gq], dst[D + 1] = gl[gq];
+      }
+    }
+    __syncthreads();
+    float run_m[EPT], run_l[EPT], run_a[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+      const int idx = tid + e * ATT_THREADS;
+      run_m[e] = -INFINITY, run_l[e] = 0.f, run_a[e] = 0.f;
+      if (idx < G * D) {
+        const int gq = idx / D, dd = idx % D;
+        const float* src = s_comb + (size_t)gq * PSTRIDE;
+        float m = -INFINITY;
+#pragma unroll
+        for (int w2 = 0; w2 < ATT_THREADS / 32; ++w2) m = fmaxf(m, src[(size_t)w2 * G * PSTRIDE + D]);
+        float l = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w2 = 0; w2 < ATT_THREADS / 32; ++w2) {
+          const float* pc = src + (size_t)w2 * G * PSTRIDE;
+          const float wgt = pc[D] == -INFINITY ? 0.f : expf(pc[D] - m);  // a warp that was dealt no position
+          l = fmaf(pc[D + 1], wgt, l);
+          acc = fmaf(pc[dd], wgt, acc);
+        }
+        run_m[e] = m, run_l[e] = l, run_a[e] = acc;
       }
     }
 
@@ -501,26 +575,24 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_runs_kernel(const __grid_
       __threadfence();
     }
     __syncthreads();
-    stamp();
     if (s_last) {  // combine the runs in ascending order
-      const int n_chunks = n_runs;  // (partials per pair)
       const float* base = p.part + (size_t)pair * p.max_chunks * G * PSTRIDE;
       for (int idx = tid; idx < G * D; idx += ATT_THREADS) {
         int gq = idx / D, dd = idx % D;
         float m = -INFINITY;
-        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+        for (int c0 = 0; c0 < n_runs; c0 += 8) {
           float mm[8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) mm[u] = (c0 + u < n_chunks) ? __ldcg(base + ((size_t)(c0 + u) * G + gq) * PSTRIDE + D) : -INFINITY;
+          for (int u = 0; u < 8; ++u) mm[u] = (c0 + u < n_runs) ? __ldcg(base + ((size_t)(c0 + u) * G + gq) * PSTRIDE + D) : -INFINITY;
 #pragma unroll
           for (int u = 0; u < 8; ++u) m = fmaxf(m, mm[u]);
         }
         float l = 0.f, acc = 0.f;
-        for (int c0 = 0; c0 < n_chunks; c0 += 8) {
+        for (int c0 = 0; c0 < n_runs; c0 += 8) {
           float mc[8], lc[8], oc[8];
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
-            const bool ok = c0 + u < n_chunks;
+            const bool ok = c0 + u < n_runs;
             const float* pc = base + ((size_t)(ok ? c0 + u : 0) * G + gq) * PSTRIDE;
             mc[u] = ok ? __ldcg(pc + D) : -INFINITY;
             lc[u] = ok ? __ldcg(pc + D + 1) : 0.f;
@@ -537,13 +609,274 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_runs_kernel(const __grid_
       }
       if (tid == 0) p.counters[pair] = 0;
     }
-    stamp();
   }
   if (!waited) {
     pdl_launch_dependents();
     pdl_wait();
   }
   timeline_mark(p.tl, p.tl_id, true);
+}
+
+// ======================= prefill attention: the rows of a pass share every key / value chunk ========================
+// A prefill pass carries consecutive prompt positions p0 .. p0 + n - 1 of one sequence at one recurrence, so all its rows
+// read the same cached keys and values (row i up to its own position).  A work item is (query head, run of chunks) for
+// ALL rows of the pass: a chunk's keys and values are brought into shared memory once, the scores of the 64 x 64 (row,
+// key) tile and the weighted values are register-tiled fp32 FMAs (the query is fp32, keys and values are bf16 values held
+// exactly in fp32: the same products as the decode kernels form), and every row keeps a running softmax over the
+// chunks of the run.  Runs are cut at fixed absolute positions - every chunk below position ATT_PF_SINGLE * 64 is a run
+// of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending order by the CTA that
+// finishes the row's last one, so a row's result depends on its own prefix only, not on how the prompt was cut into
+// passes.
+constexpr int ATT_PF_SINGLE = 40;
+constexpr int ATT_PF_RUN = 16;
+__host__ __device__ inline int att_pf_run_of_chunk(int c) { return c < ATT_PF_SINGLE ? c : ATT_PF_SINGLE + (c - ATT_PF_SINGLE) / ATT_PF_RUN; }
+__host__ __device__ inline int att_pf_run_first_chunk(int run) {
+  return run < ATT_PF_SINGLE ? run : ATT_PF_SINGLE + (run - ATT_PF_SINGLE) * ATT_PF_RUN;
+}
+constexpr int ATT_PF_ROWS = 64;  // rows of a pass at most (one group of token columns)
+template <int D>
+struct AtpCfg {
+  static constexpr int QS = D + 4;           // floats per query row in shared memory
+  static constexpr int KS = D * 2 + 16;      // bytes per key row (the pad spreads the keys a quarter warp reads over the banks)
+  static constexpr int VS = D * 2;           // bytes per value row
+  static constexpr int SS = ATT_CHUNK + 1;   // floats per score row
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = Q_OFF + ATT_PF_ROWS * QS * 4;
+  static constexpr int V_OFF = K_OFF + ATT_CHUNK * KS;
+  static constexpr int S_OFF = V_OFF + ATT_CHUNK * VS;
+  static constexpr int ST_OFF = S_OFF + ATT_PF_ROWS * SS * 4;   // per row: running max, running mass, rescale of this chunk
+  static constexpr int SMEM_BYTES = ST_OFF + ATT_PF_ROWS * 4 * 4;
+};
+
+template <int D>
+__global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
+  using C = AtpCfg<D>;
+  constexpr int PSTRIDE = D + 2;
+  constexpr int DPT = D / 16;  // dims of the output a thread accumulates (for each of its 4 rows)
+  extern __shared__ __align__(16) unsigned char atp_smem[];
+  float* s_q = reinterpret_cast<float*>(atp_smem + C::Q_OFF);
+  unsigned char* s_k = atp_smem + C::K_OFF;
+  unsigned char* s_v = atp_smem + C::V_OFF;
+  float* s_s = reinterpret_cast<float*>(atp_smem + C::S_OFF);
+  float* s_st = reinterpret_cast<float*>(atp_smem + C::ST_OFF);  // [row][4]
+  __shared__ int s_lastrow[ATT_PF_ROWS];
+
+  const RowTable* tab = p.tab;  // written before this pass started
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int n_rows = min(tab->n_rows, ATT_PF_ROWS);
+  pdl_launch_dependents();
+  pdl_wait();  // the queries, and the keys / values of the pass's own positions, come from this pass's QKV kernel
+  if (n_rows <= 0) return;
+  const int p0 = tab->pos[0], seq = tab->seq[0];
+  const int n_ctx = p0 + n_rows;                                   // keys 0 .. n_ctx - 1
+  const int n_runs_all = att_pf_run_of_chunk((n_ctx - 1) / ATT_CHUNK) + 1;
+  const int G = p.n_q_heads / p.n_kv_heads, HQ = p.n_q_heads * D;
+  const size_t plane = (size_t)(tab->r[0] - 1) * p.kv_plane_stride;
+  const int total = p.n_q_heads * n_runs_all;
+
+  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+    const int h = item % p.n_q_heads, run = item / p.n_q_heads;
+    const int kvh = h / G, gq = h - kvh * G;
+    const int c_lo = att_pf_run_first_chunk(run), c_hi = min(att_pf_run_first_chunk(run + 1), (n_ctx + ATT_CHUNK - 1) / ATT_CHUNK);
+    const __nv_bfloat16* Kb = p.kv + plane + (size_t)(seq * p.n_kv_heads + kvh) * p.slots * D;
+    const __nv_bfloat16* Vb = Kb + p.kv_sel_stride;
+    __syncthreads();  // the previous item is done with the shared buffers
+    // queries of every row for this head (fp32), and the rows' softmax state
+    for (int idx = tid; idx < n_rows * (D / 4); idx += ATT_THREADS) {
+      const int row = idx / (D / 4), d4 = idx - row * (D / 4);
+      *reinterpret_cast<float4*>(s_q + row * C::QS + d4 * 4) =
+          *reinterpret_cast<const float4*>(p.qbuf + (size_t)row * HQ + (size_t)h * D + d4 * 4);
+    }
+    for (int idx = tid; idx < (ATT_PF_ROWS - n_rows) * (D / 4); idx += ATT_THREADS) {  // rows the pass does not have: zeros
+      const int row = n_rows + idx / (D / 4), d4 = idx % (D / 4);
+      *reinterpret_cast<float4*>(s_q + row * C::QS + d4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (tid < ATT_PF_ROWS) s_st[tid * 4] = -INFINITY, s_st[tid * 4 + 1] = 0.f, s_st[tid * 4 + 2] = 1.f;
+    float o[4][DPT];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int i = 0; i < DPT; ++i) o[a][i] = 0.f;
+
+    for (int chunk = c_lo; chunk < c_hi; ++chunk) {
+      const int k0 = chunk * ATT_CHUNK;
+      const int n_keys = min(ATT_CHUNK, n_ctx - k0);  // keys of this chunk that exist (all of them written)
+      if (chunk > c_lo) __syncthreads();               // the previous chunk's readers are done
+      // ---- the chunk's keys and values, once for all rows -------------------------------------------------------
+      for (int idx = tid; idx < ATT_CHUNK * (D / 8); idx += ATT_THREADS) {
+        const int key = idx / (D / 8), pc = idx - key * (D / 8);
+        const bool ok = key < n_keys;
+        const size_t off = (size_t)(k0 + (ok ? key : 0)) * D + pc * 8;
+        cp_async16_zfill(s_k + key * C::KS + pc * 16, Kb + off, ok);
+        cp_async16_zfill(s_v + key * C::VS + pc * 16, Vb + off, ok);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+      // ---- scores: thread (ty, tx) takes rows 4 ty .. 4 ty + 3 and keys tx, tx + 16, tx + 32, tx + 48 ---------------
+      float sc[4][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) sc[a][b] = 0.f;
+#pragma unroll 2
+      for (int d = 0; d < D; d += 8) {
+        float4 qa[4], qb[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          qa[a] = *reinterpret_cast<const float4*>(s_q + (4 * ty + a) * C::QS + d);
+          qb[a] = *reinterpret_cast<const float4*>(s_q + (4 * ty + a) * C::QS + d + 4);
+        }
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const uint4 kw = *reinterpret_cast<const uint4*>(s_k + (tx + 16 * b) * C::KS + d * 2);
+          const float k0f = __uint_as_float(kw.x << 16), k1f = __uint_as_float(kw.x & 0xffff0000u);
+          const float k2f = __uint_as_float(kw.y << 16), k3f = __uint_as_float(kw.y & 0xffff0000u);
+          const float k4f = __uint_as_float(kw.z << 16), k5f = __uint_as_float(kw.z & 0xffff0000u);
+          const float k6f = __uint_as_float(kw.w << 16), k7f = __uint_as_float(kw.w & 0xffff0000u);
+#pragma unroll
+          for (int a = 0; a < 4; ++a) {  // dims in ascending order, one chain per (row, key)
+            float v = sc[a][b];
+            v = fmaf(qa[a].x, k0f, v), v = fmaf(qa[a].y, k1f, v), v = fmaf(qa[a].z, k2f, v), v = fmaf(qa[a].w, k3f, v);
+            v = fmaf(qb[a].x, k4f, v), v = fmaf(qb[a].y, k5f, v), v = fmaf(qb[a].z, k6f, v), v = fmaf(qb[a].w, k7f, v);
+            sc[a][b] = v;
+          }
+        }
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int row = 4 * ty + a, pos = p0 + row;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int key = tx + 16 * b;
+          const bool ok = row < n_rows && key < n_keys && k0 + key <= pos;  // causal
+          s_s[row * C::SS + key] = ok ? sc[a][b] * p.scale : -INFINITY;
+        }
+      }
+      __syncthreads();
+      // ---- running softmax of every row: four threads per row, 16 keys each, folded in a fixed order ----------------
+      {
+        const int row = tid >> 2, part = tid & 3;
+        float* sr = s_s + row * C::SS + part * 16;
+        float m = -INFINITY;
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) m = fmaxf(m, sr[jj]);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        const float m_old = s_st[row * 4], l_old = s_st[row * 4 + 1];
+        const float m_new = fmaxf(m_old, m);
+        float l = 0.f;
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+          const float e = (sr[jj] == -INFINITY) ? 0.f : expf(sr[jj] - m_new);
+          sr[jj] = e;
+          l += e;
+        }
+        const float l1 = __shfl_xor_sync(0xffffffffu, l, 1);
+        const float lp = (part & 1) ? l1 + l : l + l1;         // (part 0 + part 1), (part 2 + part 3)
+        const float l2 = __shfl_xor_sync(0xffffffffu, lp, 2);
+        const float lc = (part & 2) ? l2 + lp : lp + l2;       // lower pair first
+        __syncwarp();
+        if (part == 0) {
+          const float wa = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);  // (a row that has seen no key yet: nothing to rescale)
+          s_st[row * 4] = m_new, s_st[row * 4 + 1] = fmaf(l_old, wa, lc), s_st[row * 4 + 2] = (m_new == -INFINITY) ? 1.f : wa;
+        }
+      }
+      __syncthreads();
+      // ---- weighted values: thread (ty, tx) takes rows 4 ty .. + 3 and dims tx * DPT .. + DPT - 1, keys in ascending order --
+      {
+        float wa[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) wa[a] = s_st[(4 * ty + a) * 4 + 2];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int i = 0; i < DPT; ++i) o[a][i] *= wa[a];
+        for (int key = 0; key < n_keys; ++key) {
+          float vf[DPT];
+          if (DPT == 8) {
+            const uint4 vw = *reinterpret_cast<const uint4*>(s_v + key * C::VS + tx * 16);
+            const unsigned w[4] = {vw.x, vw.y, vw.z, vw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) vf[2 * i] = __uint_as_float(w[i] << 16), vf[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+          } else {
+            const uint2 vw = *reinterpret_cast<const uint2*>(s_v + key * C::VS + tx * 8);
+            vf[0] = __uint_as_float(vw.x << 16), vf[1] = __uint_as_float(vw.x & 0xffff0000u);
+            vf[2] = __uint_as_float(vw.y << 16), vf[3] = __uint_as_float(vw.y & 0xffff0000u);
+          }
+#pragma unroll
+          for (int a = 0; a < 4; ++a) {
+            const float pw = s_s[(4 * ty + a) * C::SS + key];
+#pragma unroll
+            for (int i = 0; i < DPT; ++i) o[a][i] = fmaf(pw, vf[i], o[a][i]);
+          }
+        }
+      }
+    }
+    __syncthreads();  // every thread has read the final state
+    // ---- the run is done: rows with one run only are finished here, the others leave a partial -----------------------
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int row = 4 * ty + a, pos = p0 + row;
+      if (row >= n_rows || c_lo * ATT_CHUNK > pos) continue;   // the row does not reach this run
+      const int n_runs_row = att_pf_run_of_chunk(pos / ATT_CHUNK) + 1;
+      const float m = s_st[row * 4], l = s_st[row * 4 + 1];
+      if (n_runs_row == 1) {
+#pragma unroll
+        for (int i = 0; i < DPT; ++i) store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + tx * DPT + i, o[a][i] / l);
+      } else {
+        float* mypart = p.part + (((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks + run) * G + gq) * PSTRIDE;
+#pragma unroll
+        for (int i = 0; i < DPT; ++i) __stcg(mypart + tx * DPT + i, o[a][i]);
+        if (tx == 0) __stcg(mypart + D, m), __stcg(mypart + D + 1, l);
+      }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid < ATT_PF_ROWS) {
+      const int row = tid, pos = p0 + row;
+      int last = 0;
+      if (row < n_rows && c_lo * ATT_CHUNK <= pos) {
+        const int n_runs_row = att_pf_run_of_chunk(pos / ATT_CHUNK) + 1;
+        if (n_runs_row > 1) {
+          const int old = atomicAdd(p.counters + row * p.n_q_heads + h, 1);
+          last = (old == n_runs_row - 1) ? n_runs_row : 0;
+        }
+      }
+      s_lastrow[row] = last;
+      __threadfence();
+    }
+    __syncthreads();
+    // ---- rows whose last run this was: fold their runs in ascending order (two rows at a time, one thread per dim) ----
+    for (int r0 = 0; r0 < n_rows; r0 += 2) {
+      const int row = r0 + (tid >> 7), dd = tid & 127;
+      if (row >= n_rows || dd >= D) continue;
+      const int n_runs_row = s_lastrow[row];
+      if (n_runs_row == 0) continue;
+      const float* base = p.part + ((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks * G + gq) * PSTRIDE;
+      const size_t rstride = (size_t)G * PSTRIDE;
+      float m = -INFINITY;
+      for (int c0 = 0; c0 < n_runs_row; ++c0) m = fmaxf(m, __ldcg(base + c0 * rstride + D));
+      float l = 0.f, acc = 0.f;
+      for (int c0 = 0; c0 < n_runs_row; c0 += 4) {
+        float mc[4], lc[4], oc[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool ok = c0 + u < n_runs_row;
+          const float* pc = base + (size_t)(ok ? c0 + u : 0) * rstride;
+          mc[u] = ok ? __ldcg(pc + D) : -INFINITY, lc[u] = ok ? __ldcg(pc + D + 1) : 0.f, oc[u] = ok ? __ldcg(pc + dd) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float wgt = (mc[u] == -INFINITY) ? 0.f : expf(mc[u] - m);
+          l = fmaf(lc[u], wgt, l);
+          acc = fmaf(oc[u], wgt, acc);
+        }
+      }
+      store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + dd, acc / l);
+      if (dd == 0) p.counters[row * p.n_q_heads + h] = 0;
+    }
+  }
 }
 
 }  // namespace ls

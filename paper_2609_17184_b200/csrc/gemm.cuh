@@ -77,6 +77,7 @@ struct GemmParams {
   const float* gain_next;
   float* hid;             // RESID: residual stream [hid_idx][H]
   int no_resid;           // RESID: the output REPLACES the stream (the adapter of a Raven-style model: H = W_a [H; e])
+  int recv_ranks;         // contributions per column in the receive buffer (0: one per rank of the cluster)
   float* sumsq_out;       // RESID: [row][n_sq_out]
   int n_sq_out;
   float* qbuf;            // QKV: [row][n_q_heads * d]
@@ -162,7 +163,7 @@ __device__ __forceinline__ void gemm_reduce_epilogue(const GemmParams& p, const 
                                                      float pre_g = 1.f, float2 pre_rope = make_float2(1.f, 0.f), bool pre_valid = false) {
   constexpr int RBW = RB_ROWS / KH;  // rows of this row block
   const int tid = threadIdx.x, half = tid >> 7, j = tid & 127, lane = tid & 31, hw = (tid >> 5) & 3;
-  const int cs = p.cluster_size, vcs = cs * KH;
+  const int cs = p.cluster_size, vcs = p.recv_ranks ? p.recv_ranks : cs * KH;
   __shared__ float s_ss[2][4];
   for (int base = rank; base < n_cols; base += 2 * cs) {
     const int c = base + cs * half;
@@ -771,7 +772,7 @@ struct TcEpiParams {
 
 template <int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_constant__ TcEpiParams q) {
-  __shared__ float s_recv[TCE_MAX_COLS * RB_ROWS];
+  __shared__ float s_recv[(TCE_MAX_COLS / TCE_GROUPS) * RB_ROWS];
   __shared__ float s_colbuf[2 * RB_ROWS];
   __shared__ float s_rstd[TCE_MAX_COLS];
   __shared__ int s_ct[CT_FIELDS * TCE_MAX_COLS];
@@ -804,11 +805,9 @@ __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_
     n = rb * RB_ROWS + j;
     if (n >= p.N) n = -1;
   }
-  // blockIdx.y takes the columns c = y, y + TCE_GROUPS, ... exactly as rank y of a cluster of TCE_GROUPS CTAs would;
-  // the other ranks' contributions in the receive buffer are zeros (adding them changes nothing)
+  // blockIdx.y takes the columns c = y, y + TCE_GROUPS, ... exactly as rank y of a cluster of TCE_GROUPS CTAs would, with
+  // one contribution per column in the receive buffer (recv_ranks = 1): the k-split sums added below
   const int rank = blockIdx.y, own_max = TCE_MAX_COLS / TCE_GROUPS;
-  for (int i = tid; i < TCE_MAX_COLS * RB_ROWS; i += GEMM_THREADS) s_recv[i] = 0.f;
-  __syncthreads();
   const size_t split_stride = (size_t)q.cols_ld * p.N;
   for (int c = rank + TCE_GROUPS * (tid >> 7); c < n_cols; c += TCE_GROUPS * (GEMM_THREADS / RB_ROWS)) {
     float v = 0.f;

@@ -322,12 +322,13 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.sumsq = take(MR * d.sq_stride * 4);
   L.logits = take((size_t)d.n_logit_vecs * m->vocab * 4);
   L.argpart = take(MR * ((m->vocab + 127) / 128) * sizeof(float2));
-  {  // k-split partial sums of the prefill GEMMs on the tcgen05 kernel (the largest of the four)
+  {  // k-split partial sums of the GEMMs that run on the tcgen05 kernel (the largest of them, prefill or decode columns)
     size_t need = 0;
     if (tc_prefill_shapes_ok(m)) {
-      const int Ns[4] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden}, Ks[4] = {m->hidden, d.Hq, m->hidden, m->ffn};
-      for (int i = 0; i < 4; ++i)
-        need = std::max(need, (size_t)tc_pf_plan(Ns[i], Ks[i]).n_split * tc_pf_cols(d.max_rows_pf) * Ns[i] * 4);
+      const int Ns[5] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden, m->hidden};
+      const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, 2 * m->hidden};
+      const int cols = std::max(tc_pf_cols(d.max_rows_pf), tc_pf_cols(std::min(d.max_rows_dec, (int)GROUP_ROWS)));
+      for (int i = 0; i < (d.raven ? 5 : 4); ++i) need = std::max(need, (size_t)tc_pf_plan(Ns[i], Ks[i]).n_split * cols * Ns[i] * 4);
     }
     L.tcpart = take(need);
   }
@@ -335,7 +336,7 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
   L.tune = take(L.tune_bytes);
   int G = m->n_q_heads / m->n_kv_heads;
   L.apart = take(MR * m->n_kv_heads * d.max_chunks * G * (m->head_dim + 2) * 4);
-  L.acnt = take(MR * m->n_kv_heads * 4);
+  L.acnt = take(MR * m->n_q_heads * 4);  // arrival counters per (row, kv head) of the decode kernels, (row, query head) of the prefill kernel
   L.nodes = take((size_t)13 * MAX_NODES * 4);
   L.flt = take((size_t)2 * MAX_NODES * sizeof(float4));
   L.sel_flt = take((size_t)MAX_ROWS * sizeof(float4));
@@ -382,12 +383,17 @@ struct loopspec_ctx {
   int ng_dec = 1, ng_pf = 1;
   GemmPlan plan[6];
   // prefill on the tcgen05 kernel: tensor maps of the row-major weights (4 per layer) and of the three plane buffers
-  bool tc_pf = false;
-  std::vector<CUtensorMap> tc_wmaps;
-  CUtensorMap tc_xmaps[3];
-  TcPfPlan tc_plan[4];
-  int tc_cols = 0, tc_stages = 0;
-  size_t tc_smem = 0;
+  // ... and the decode passes of contexts whose passes carry 9 to 64 rows (batches, deep recurrences), where the
+  // mma.sync kernels are bound by their three-plane arithmetic rather than by the weight stream
+  struct TcCfg {
+    bool on = false;
+    int cols = 0, stages = 0;   // token columns of a launch (multiple of 16), ring stages
+    size_t smem = 0;
+    CUtensorMap xmaps[4];       // planes read by QKV and gate/up, by O, by down, by the adapter
+  };
+  TcCfg tc[2];                  // 0: prefill passes, 1: decode passes
+  std::vector<CUtensorMap> tc_wmaps;  // 4 per block, then the adapter
+  TcPfPlan tc_plan[5];          // qkv, o, gate/up, down, adapter
   // readout GEMM of the decode passes on the tcgen05 kernel (bf16 weights): plan, tensor maps of the row-major lm_head
   // (one box per 128-row tile) and of the hidden-state planes (all three planes of dg_mp rows in one box)
   bool dg = false;
@@ -404,6 +410,7 @@ struct loopspec_ctx {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   std::vector<char> prefilled;
   bool pending_verify = false, sticky = false, vanilla_mode = false, use_pdl = true;
+  bool pf_attn = false;  // prefill passes run the attention kernel that shares K/V chunks among the rows
   bool filters = false;  // C applies top-k / top-p (sampling only)
   int sel_staged = 0;    // the selection kernel keeps its row slices in shared memory
   size_t sel_smem = 0;
@@ -526,6 +533,15 @@ AttnFn attn_fn(int d, int G, bool runs) {  // runs: contexts longer than ATT_MAX
   return G == 1 ? attn_kernel<64, 1> : attn_kernel<64, 4>;
 }
 
+// dynamic shared memory and grid of the attention launch (the streaming kernel of long contexts: its rings, and one
+// CTA per slot the SMs offer)
+size_t attn_smem(int d, int G, bool runs) {
+  if (!runs) return 0;
+  if (d == 128) return G == 1 ? AtsCfg<128, 1>::SMEM_BYTES : AtsCfg<128, 4>::SMEM_BYTES;
+  return G == 1 ? AtsCfg<64, 1>::SMEM_BYTES : AtsCfg<64, 4>::SMEM_BYTES;
+}
+int attn_grid(int n_sm, int G, bool runs) { return runs ? n_sm * (G == 1 ? AtsCfg<128, 1>::MIN_CTAS : AtsCfg<128, 4>::MIN_CTAS) : n_sm * 8; }
+
 // tuning builds (-DLOOPSPEC_TUNE) with LOOPSPEC_DBG set record a kernel timeline in a workspace region of their own
 unsigned long long* tune_timeline(loopspec_ctx* c) {
   return (kTune && c->L.tune_bytes && getenv("LOOPSPEC_DBG")) ? reinterpret_cast<unsigned long long*>(c->ws + c->L.tune) : nullptr;
@@ -634,26 +650,29 @@ template <int EPI>
 cudaError_t launch_tc_epi(const TcEpiParams& q, cudaStream_t st, bool pdl) {
   return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
 }
-cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab) {
-  const TcPfPlan& t = c->tc_plan[which];
+cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab, int cfg_i) {
+  const loopspec_ctx::TcCfg& tc = c->tc[cfg_i];
+  const int pi = which == G_ADAPT ? 4 : which;
+  const TcPfPlan& t = c->tc_plan[pi];
   TcEpiParams q;
   q.g = gemm_params(c, which, layer, tab);
-  q.g.cluster_size = TCE_GROUPS;
-  q.part = c->at<float>(c->L.tcpart), q.n_split = t.n_split, q.cols_ld = c->tc_cols;
+  q.g.cluster_size = TCE_GROUPS, q.g.recv_ranks = 1;
+  q.part = c->at<float>(c->L.tcpart), q.n_split = t.n_split, q.cols_ld = tc.cols;
   LinearTcParams p;
   memset(&p, 0, sizeof p);
   p.out = c->at<float>(c->L.tcpart);
-  p.M = c->tc_cols, p.MP = c->tc_cols, p.N = q.g.N, p.K = q.g.K, p.kb_per_split = t.kb_per_split, p.stages = c->tc_stages;
+  p.M = tc.cols, p.MP = tc.cols, p.N = q.g.N, p.K = q.g.K, p.kb_per_split = t.kb_per_split, p.stages = tc.stages;
   p.err = const_cast<int*>(c->host_flags_dev + HF_ERROR), p.err_code = 5, p.x3d = 1;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3(t.n_tiles, t.n_split), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = c->tc_smem, cfg.stream = c->stream;
+  cfg.gridDim = dim3(t.n_tiles, t.n_split), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = tc.smem, cfg.stream = c->stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at, cfg.numAttrs = c->use_pdl ? 1 : 0;
-  const int xi = which == G_O ? 1 : which == G_DOWN ? 2 : 0;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel, c->tc_wmaps[4 * layer + which], c->tc_xmaps[xi], p);
+  const int xi = which == G_O ? 1 : which == G_DOWN ? 2 : which == G_ADAPT ? 3 : 0;
+  const CUtensorMap& wm = which == G_ADAPT ? c->tc_wmaps[4 * c->d.NL] : c->tc_wmaps[4 * layer + which];
+  cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel, wm, tc.xmaps[xi], p);
   if (e != cudaSuccess) return e;
   switch (which) {
     case G_QKV: return launch_tc_epi<EPI_QKV>(q, c->stream, c->use_pdl);
@@ -705,8 +724,32 @@ int col_groups(loopspec_ctx* c, const RowTable* tab) {
   return (c->d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;
 }
 
+// decode attention of block `l` on the rows of `tab`
+cudaError_t launch_attention(loopspec_ctx* c, const RowTable* tab, int l, unsigned long long* tl, int tl_id, bool prefill_rows = false) {
+  const loopspec_model& m = c->m;
+  const Derived& d = c->d;
+  const int G = m.n_q_heads / m.n_kv_heads;
+  AttnParams a;
+  memset(&a, 0, sizeof a);
+  a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
+  a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
+  a.kv_plane_stride = c->kv_plane_stride(), a.kv_sel_stride = c->kv_sel_stride();
+  a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
+  a.scale = 1.0f / sqrtf((float)m.head_dim);
+  a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
+  a.tl = tl, a.tl_id = tl_id;
+  if (prefill_rows && c->pf_attn) {  // consecutive prompt positions of one sequence: the rows share every K/V chunk
+    if (m.head_dim == 128)
+      return launch_k(attn_prefill_kernel<128>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<128>::SMEM_BYTES, c->stream, a, c->use_pdl);
+    return launch_k(attn_prefill_kernel<64>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<64>::SMEM_BYTES, c->stream, a, c->use_pdl);
+  }
+  const bool runs = d.max_chunks > ATT_MAX_RUNS;
+  return launch_k(attn_fn(m.head_dim, G, runs), dim3(attn_grid(c->n_sm, G, runs)), dim3(ATT_THREADS), attn_smem(m.head_dim, G, runs), c->stream, a,
+                  c->use_pdl);
+}
+
 // the blocks [l0, l0 + count) of the layer list on the rows of `tab`
-cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, int count, int* n_launch, bool tc) {
+cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, int count, int* n_launch, int tc) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   const int G = m.n_q_heads / m.n_kv_heads;
@@ -715,7 +758,7 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
   const int groups = col_groups(c, tab);
   // a GEMM of the pass: one launch per group of token columns (one group unless a decode pass can carry more than 64 rows)
   auto gemm = [&](int which, int l, int tl_id) -> cudaError_t {
-    if (tc) return launch_tc_gemm(c, which, l, tab);
+    if (tc >= 0) return launch_tc_gemm(c, which, l, tab, tc);
     for (int g = 0; g < groups; ++g) {
       GemmParams gp = gemm_params(c, which, l, tab, g * GROUP_ROWS);
       gp.tl = tune_timeline(c), gp.tl_id = tl_id;
@@ -727,20 +770,11 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
   for (int l = l0; l < l0 + count; ++l) {
     unsigned long long* tl = tune_timeline(c);
     if ((e = gemm(G_QKV, l, l * 5 + 0))) return e;
-    AttnParams a;
-    memset(&a, 0, sizeof a);
-    a.tab = tab, a.qbuf = c->at<float>(c->L.qbuf), a.aplanes = c->at<__nv_bfloat16>(c->L.aplanes);
-    a.kv = c->at<__nv_bfloat16>(c->L.kv) + (size_t)l * c->kv_layer_stride();
-    a.kv_plane_stride = c->kv_plane_stride(), a.kv_sel_stride = c->kv_sel_stride();
-    a.slots = d.slots, a.n_kv_heads = m.n_kv_heads, a.n_q_heads = m.n_q_heads;
-    a.scale = 1.0f / sqrtf((float)m.head_dim);
-    a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
-    a.tl = tl, a.tl_id = l * 5 + 1;
-    if ((e = launch_k(attn_fn(m.head_dim, G, d.max_chunks > ATT_MAX_RUNS), dim3(c->n_sm * 8), dim3(ATT_THREADS), 0, c->stream, a, pdl))) return e;
+    if ((e = launch_attention(c, tab, l, tl, l * 5 + 1, tab == c->at<RowTable>(c->L.tab_pf) || tab == c->at<RowTable>(c->L.tab_pfc)))) return e;
     if ((e = gemm(G_O, l, l * 5 + 2))) return e;
     if ((e = gemm(G_GU, l, l * 5 + 3))) return e;
     if ((e = gemm(G_DOWN, l, l * 5 + 4))) return e;
-    if (n_launch) *n_launch += 1 + 4 * (tc ? 2 : groups);
+    if (n_launch) *n_launch += 1 + 4 * (tc >= 0 ? 2 : groups);
   }
   return cudaSuccess;
 }
@@ -748,7 +782,7 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
 // One batched pass of B over the rows of `tab` (Sec. 4.2 step 1).  Ouro layout: preparation + the shared blocks.
 // Raven-style layout: the rows entering their first recurrence (`tab_pre`, may be null) go through the prelude blocks,
 // then every row through the adapter on [H; e] and the recurrent blocks.
-cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, bool tc = false, const RowTable* tab_pre = nullptr) {
+cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_launch, int tc = -1, const RowTable* tab_pre = nullptr) {
   const loopspec_model& m = c->m;
   const Derived& d = c->d;
   cudaError_t e;
@@ -767,15 +801,19 @@ cudaError_t launch_layers(loopspec_ctx* c, const RowTable* tab, int ng, int* n_l
   cp.planes = c->at<__nv_bfloat16>(c->L.cplanes);
   if ((e = launch_k(raven_concat_kernel, dim3(d.max_rows), dim3(256), 0, c->stream, cp, c->use_pdl))) return e;
   const int groups = col_groups(c, tab);
-  for (int g = 0; g < groups; ++g)
-    if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_ADAPT, 0, tab, g * GROUP_ROWS), c->stream, c->use_pdl))) return e;
-  if (n_launch) *n_launch += 1 + groups;
+  if (tc >= 0) {
+    if ((e = launch_tc_gemm(c, G_ADAPT, 0, tab, tc))) return e;
+  } else {
+    for (int g = 0; g < groups; ++g)
+      if ((e = launch_gemm(m.weight_dtype, ng, EPI_RESID, gemm_params(c, G_ADAPT, 0, tab, g * GROUP_ROWS), c->stream, c->use_pdl))) return e;
+  }
+  if (n_launch) *n_launch += 1 + (tc >= 0 ? 2 : groups);
   return launch_stack(c, tab, ng, d.n_pre, m.n_recurrent, n_launch, tc);
 }
 
 // Raven-style layout: the post-layers' blocks on copies of the reading-out rows' states (`tab_coda`), writing the coda
 // cache of each row's readout depth; leaves the planes the lm_head reads
-cudaError_t launch_coda(loopspec_ctx* c, const RowTable* tab_coda, int ng, int* n_launch, bool tc = false) {
+cudaError_t launch_coda(loopspec_ctx* c, const RowTable* tab_coda, int ng, int* n_launch, int tc = -1) {
   const Derived& d = c->d;
   cudaError_t e;
   if ((e = launch_prep(c, tab_coda, d.n_pre + c->m.n_recurrent, true))) return e;
@@ -847,11 +885,12 @@ cudaError_t launch_kv_commit(loopspec_ctx* c) {
 cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_commit, int* n_launch) {
   const RowTable* tab = c->at<RowTable>(c->L.tab_dec);
   cudaError_t e;
-  if ((e = launch_layers(c, tab, c->ng_dec, n_launch, false, c->d.raven ? c->at<RowTable>(c->L.tab_pre) : nullptr))) return e;
+  const int tc = c->tc[1].on ? 1 : -1;  // decode passes of 9 to 64 rows: the layers' GEMMs on the tcgen05 kernel
+  if ((e = launch_layers(c, tab, c->ng_dec, n_launch, tc, c->d.raven ? c->at<RowTable>(c->L.tab_pre) : nullptr))) return e;
   const RowTable* tab_ro = tab;  // the rows the lm_head reads
   if (c->d.raven && c->d.n_coda > 0) {
     tab_ro = c->at<RowTable>(c->L.tab_coda);
-    if ((e = launch_coda(c, tab_ro, c->ng_dec, n_launch))) return e;
+    if ((e = launch_coda(c, tab_ro, c->ng_dec, n_launch, tc))) return e;
   }
   if ((e = launch_lm_head(c, tab_ro, c->ng_dec))) return e;
   if ((e = launch_select(c, tab, kinds_mask))) return e;
@@ -880,11 +919,11 @@ cudaError_t launch_vanilla_token(loopspec_ctx* c) {
   cudaError_t e;
   RowTable* tabs = c->at<RowTable>(c->L.tab_van);
   for (int r = 0; r < c->m.R; ++r)  // every row enters recurrence 1 in the first pass: the prelude pass is that table itself
-    if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr, false, (c->d.raven && r == 0) ? tabs : nullptr))) return e;
+    if ((e = launch_layers(c, tabs + r, c->ng_dec, nullptr, c->tc[1].on ? 1 : -1, (c->d.raven && r == 0) ? tabs : nullptr))) return e;
   const RowTable* tab_ro = tabs + c->m.R - 1;
   if (c->d.raven && c->d.n_coda > 0) {
     tab_ro = c->at<RowTable>(c->L.tab_vanc);
-    if ((e = launch_coda(c, tab_ro, c->ng_dec, nullptr))) return e;
+    if ((e = launch_coda(c, tab_ro, c->ng_dec, nullptr, c->tc[1].on ? 1 : -1))) return e;
   }
   if ((e = launch_lm_head(c, tab_ro, c->ng_dec))) return e;
   if ((e = launch_select(c, tabs + c->m.R - 1, 1 << RO_TARGET))) return e;
@@ -1054,6 +1093,22 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       if (cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
         (void)cudaGetLastError();
   }
+  {
+    const int G = m->n_q_heads / m->n_kv_heads;
+    const bool runs = d.max_chunks > ATT_MAX_RUNS;
+    if (runs && cudaFuncSetAttribute((const void*)attn_fn(m->head_dim, G, runs), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)attn_smem(m->head_dim, G, runs)) != cudaSuccess) {
+      delete c;
+      return LOOPSPEC_ECUDA;
+    }
+  }
+  if (!s->prefill_skinny) {  // (prefill_skinny keeps the decode kernels for the prefill passes, attention included)
+    const bool ok = m->head_dim == 128
+                        ? cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<128>::SMEM_BYTES) == cudaSuccess
+                        : cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<64>::SMEM_BYTES) == cudaSuccess;
+    if (!ok) (void)cudaGetLastError();
+    c->pf_attn = ok;
+  }
   if (cudaFuncSetAttribute(control_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ControlSmem)) != cudaSuccess) {
     delete c;
     return LOOPSPEC_ECUDA;
@@ -1087,26 +1142,38 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
       g = plan_gemm(n_rbs[i], Ks[i], slots, true);
     }
   }
-  // prefill passes on the tcgen05 kernel (shapes it does not take, and fp32 weights: the kernels of the decode passes)
-  if (tc_prefill_shapes_ok(m) && !s->prefill_skinny && encode_tiled_fn()) {
+  // prefill passes on the tcgen05 kernel (shapes it does not take, and fp32 weights: the kernels of the decode passes);
+  // decode passes too when they carry 9 to 64 rows
+  if (tc_prefill_shapes_ok(m) && encode_tiled_fn()) {
     const Derived& dd = c->d;
-    c->tc_cols = tc_pf_cols(dd.max_rows_pf);
-    const int sb = tc_stage_bytes(c->tc_cols);
-    c->tc_stages = std::max(2, std::min(TC_MAX_STAGES, (100 * 1024) / sb));
-    c->tc_smem = (size_t)c->tc_stages * sb + 1024;
-    const int Ns[4] = {dd.Hq + 2 * dd.Hkv, m->hidden, 2 * m->ffn, m->hidden}, Ks[4] = {m->hidden, dd.Hq, m->hidden, m->ffn};
+    const int Ns[5] = {dd.Hq + 2 * dd.Hkv, m->hidden, 2 * m->ffn, m->hidden, m->hidden};
+    const int Ks[5] = {m->hidden, dd.Hq, m->hidden, m->ffn, 2 * m->hidden};
     const int w_idx[4] = {1, 2, 4, 5};  // qkv, o, gate/up, down among a layer's six pointers
     bool ok = true;
-    c->tc_wmaps.resize((size_t)4 * dd.NL);
+    c->tc_wmaps.resize((size_t)4 * dd.NL + 1);
     for (int l = 0; l < dd.NL && ok; ++l)
       for (int i = 0; i < 4 && ok; ++i) ok = make_map_bf16(&c->tc_wmaps[4 * l + i], c->layers[6 * l + w_idx[i]], Ns[i], Ks[i], TC_BM);
-    const size_t x_off[3] = {c->L.xplanes, c->L.aplanes, c->L.splanes};
-    const int x_k[3] = {m->hidden, dd.Hq, m->ffn};
-    for (int i = 0; i < 3 && ok; ++i) ok = make_map_planes3d(&c->tc_xmaps[i], c->ws + x_off[i], x_k[i], x_k[i], dd.max_rows, c->tc_cols);
-    for (int i = 0; i < 4; ++i) c->tc_plan[i] = tc_pf_plan(Ns[i], Ks[i]);
-    ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->tc_smem) == cudaSuccess;
+    if (dd.raven) ok = ok && make_map_bf16(&c->tc_wmaps[4 * dd.NL], c->adapter, Ns[4], Ks[4], TC_BM);
+    for (int i = 0; i < 5; ++i) c->tc_plan[i] = tc_pf_plan(Ns[i], Ks[i]);
+    const size_t x_off[4] = {c->L.xplanes, c->L.aplanes, c->L.splanes, c->L.cplanes};
+    const int x_k[4] = {m->hidden, dd.Hq, m->ffn, 2 * m->hidden};
+    const bool want[2] = {!s->prefill_skinny, c->ng_dec > 1 && dd.max_rows_dec <= GROUP_ROWS};
+    const int rows[2] = {dd.max_rows_pf, dd.max_rows_dec};
+    size_t smem_max = 0;
+    for (int k = 0; k < 2 && ok; ++k) {
+      if (!want[k]) continue;
+      loopspec_ctx::TcCfg& tc = c->tc[k];
+      tc.cols = tc_pf_cols(rows[k]);
+      const int sb = tc_stage_bytes(tc.cols);
+      tc.stages = std::max(2, std::min(TC_MAX_STAGES, (100 * 1024) / sb));
+      tc.smem = (size_t)tc.stages * sb + 1024;
+      smem_max = std::max(smem_max, tc.smem);
+      for (int i = 0; i < (dd.raven ? 4 : 3) && ok; ++i)
+        ok = make_map_planes3d(&tc.xmaps[i], c->ws + x_off[i], x_k[i], x_k[i], dd.max_rows, tc.cols);
+    }
+    if (smem_max) ok = ok && cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) == cudaSuccess;
     if (!ok) (void)cudaGetLastError();
-    c->tc_pf = ok;
+    for (int k = 0; k < 2; ++k) c->tc[k].on = ok && want[k];
   }
   // readout GEMM of the decode passes on the tcgen05 kernel: bf16 weights whose rows are 16-byte multiples (TMA strides)
   if (m->weight_dtype == 1 && encode_tiled_fn() && m->hidden % 8 == 0) {
@@ -1246,8 +1313,8 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
       }
       prefill_setup_kernel<<<1, CTRL_THREADS, 0, c->stream>>>(pp);
       CU(c, cudaGetLastError());
-      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc_pf, (c->d.raven && r == 1) ? tab : nullptr));
-      if (pp.coda_class > 0) CU(c, launch_coda(c, pp.tab_coda, c->ng_pf, nullptr, c->tc_pf));
+      CU(c, launch_layers(c, tab, c->ng_pf, nullptr, c->tc[0].on ? 0 : -1, (c->d.raven && r == 1) ? tab : nullptr));
+      if (pp.coda_class > 0) CU(c, launch_coda(c, pp.tab_coda, c->ng_pf, nullptr, c->tc[0].on ? 0 : -1));
     }
   }
   if (c->d.raven && c->d.n_coda > 0) tab = c->at<RowTable>(c->L.tab_pfc);  // its last state: last chunk, depth R
@@ -1489,8 +1556,9 @@ int loopspec_debug_drop_tile(loopspec_ctx* c, int32_t unit, int32_t wait_us) {
 int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
   const Derived& d = c->d;
-  const int g = (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;  // launches per GEMM (groups of 64 token columns)
-  const int per_block = 1 + 4 * g, lm = c->dg ? 1 : g;            // attention + four GEMMs
+  // launches per GEMM: one per group of 64 token columns, or the tcgen05 kernel and its epilogue
+  const int g = c->tc[1].on ? 2 : (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;
+  const int per_block = 1 + 4 * g, lm = c->dg ? 1 : (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;  // attention + four GEMMs
   int n = 1 + c->m.n_recurrent * per_block + lm + 3;               // preparation, blocks, lm_head, selection, control, KV commit
   if (d.raven)  // prelude pass (preparation + blocks), concatenation + adapter instead of the preparation, coda pass
     n = (d.n_pre ? 1 + per_block * d.n_pre : 0) + 1 + g + per_block * c->m.n_recurrent + (d.n_coda ? 1 + per_block * d.n_coda : 0) + lm + 3;
@@ -1499,7 +1567,7 @@ int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
 }
 
 int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_out, double* bytes_out) {
-  if (!c || which < 0 || which > 4 || rows < 1 || rows > 8 * c->ng_dec || iters < 1 || !ms_out) return LOOPSPEC_EINVAL;
+  if (!c || which < 0 || which > 5 || rows < 1 || rows > 8 * c->ng_dec || iters < 1 || !ms_out) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
   // a scratch row table with `rows` plain rows on sequence 0 (hidden states of the prefill area; outputs go to
@@ -1512,14 +1580,34 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
     t.logit_idx[i] = c->d.p_logit_base, t.node[i] = -1, t.chunk_start[i] = i;
   }
   t.chunk_start[rows] = rows, t.attn_items = rows;
+  if (which == 5) {
+    // attention: row i reads the whole cached context (the capacity minus one chunk) of sequence i mod S at recurrence
+    // 1 + (i / S) mod R, so that no two rows share keys or values (as rows at different depths do not)
+    const int ctx = std::max(1, c->d.ids_cap - ATT_CHUNK);
+    int items = 0;
+    for (int i = 0; i < rows; ++i) {
+      t.seq[i] = i % c->d.S, t.r[i] = 1 + (i / c->d.S) % c->m.R;
+      t.n_canon[i] = ctx, t.n_safe[i] = ctx, t.n_spec[i] = 0, t.chunk_start[i] = items;
+      items += att_items(ctx);
+    }
+    t.chunk_start[rows] = items, t.attn_items = items;
+  }
   CU(c, cudaMemcpyAsync(c->ws + c->L.tab_pf, &t, sizeof t, cudaMemcpyHostToDevice, c->stream));
   CU(c, cudaMemsetAsync(c->ws + c->L.hid + (size_t)c->d.S * c->d.NB * c->m.hidden * 4, 0, (size_t)rows * c->m.hidden * 4, c->stream));
   const RowTable* tab = c->at<RowTable>(c->L.tab_pf);
-  const int L = c->m.n_recurrent;
+  int L = c->m.n_recurrent;
+  if (kTune && getenv("LOOPSPEC_TK_LAYERS")) L = std::max(1, std::min(L, atoi(getenv("LOOPSPEC_TK_LAYERS"))));  // L2-resident weights
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
+      if (which == 5) {
+        cudaError_t e = launch_attention(c, tab, i % L, nullptr, 0);
+        if (e) return e;
+        continue;
+      }
       GemmParams p = gemm_params(c, which, i % L, tab);
-      cudaError_t e = (c->dg && which == G_LM) ? launch_dg_lm(c, tab) : launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
+      cudaError_t e = (c->dg && which == G_LM)         ? launch_dg_lm(c, tab)
+                      : (c->tc[1].on && which != G_LM) ? launch_tc_gemm(c, which, i % L, tab, 1)
+                                                       : launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
       if (e) return e;
     }
     return cudaSuccess;
@@ -1536,7 +1624,10 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   const Derived& d = c->d;
   double nk[5] = {(double)(d.Hq + 2 * d.Hkv) * c->m.hidden, (double)c->m.hidden * d.Hq, 2.0 * c->m.ffn * c->m.hidden,
                   (double)c->m.hidden * c->m.ffn, (double)c->m.vocab * c->m.hidden};
-  if (bytes_out) *bytes_out = nk[which] * wb;
+  if (bytes_out) {
+    *bytes_out = which < 5 ? nk[which] * wb
+                           : 2.0 * rows * c->m.n_kv_heads * (double)std::max(1, d.ids_cap - ATT_CHUNK) * c->m.head_dim * 2;  // K and V, bf16
+  }
   // the timed launches touched sequence state only through scratch; mark sequences as needing a new prefill
   std::fill(c->prefilled.begin(), c->prefilled.end(), 0);
   return LOOPSPEC_OK;
