@@ -116,7 +116,7 @@ def vanilla_bytes(shape, n_prompt, n_decode, batch=1):
     return n_decode * (shape.R * (w_b + batch * kv_row) + w_c)
 
 
-KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
+KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head", "attention"]
 
 
 def replica_throughput(tokens_per_rank, device_ms, wall_s, dist=None, device=None):
@@ -139,7 +139,10 @@ def run_kernel_only(args):
     wl = W.WORKLOADS[args.workload]
     shape = W.CONFIGS[wl.model]
     weights = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed))
-    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, max_seqs=1, max_ctx=wl.prompt_len + wl.decode_len + 16)
+    # (attention: every row reads a cached context of max_ctx - 64 positions at a recurrence of its own; --prompt-len
+    # sets the context, e.g. 4096 for the streaming kernel of long contexts on a few GB of KV pool)
+    n_ctx = (args.prompt_len or wl.prompt_len) + (0 if args.kernel_only == "attention" else wl.decode_len) + 64
+    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, max_seqs=1, max_ctx=n_ctx)
     ms, nbytes = ctx.time_kernel(KERNELS.index(args.kernel_only), args.rows, args.iters)
     print(json.dumps({"kernel": args.kernel_only, "rows": args.rows, "iters": args.iters, "us_per_launch": ms * 1e3,
                       "GBps": nbytes / (ms / 1e3) / 1e9}))
@@ -273,11 +276,14 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    prefill_s = []
+
     def one_job(decode_fn):
         """prefill (host ids -> device) then decode n_decode tokens; returns (decode ms on device, wall s of both)."""
         t_a = time.perf_counter()
         for s_, p_ in enumerate(prompts):      # every sequence of the batch is prefilled from its own host prompt
-            ctx.prefill(p_, seq=s_)
+            ctx.prefill(p_, seq=s_)          # (returns the first token: the call ends when the prefill has)
+        prefill_s.append(time.perf_counter() - t_a)
         with torch.cuda.stream(stream):
             ev0.record(stream)
             out = decode_fn(n_decode)
@@ -291,6 +297,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
+    prefill_s.clear()
     dec_ms, wall_s = [], []
     t_region = time.perf_counter()
     for _ in range(args.steps):
@@ -300,6 +307,7 @@ def run_ours(args):
     barrier()
     t_region = time.perf_counter() - t_region
     clocks = sampler.stop()
+    prefill_ms_seq = 1e3 * statistics.mean(prefill_s) / batch
     stats = ctx.stats()
     stats["d1"] = d1
     launches = ctx.launches_per_step() * stats["steps"] * args.steps
@@ -324,6 +332,14 @@ def run_ours(args):
     for which, nm in enumerate(["qkv", "o_proj", "gate_up", "down", "lm_head"]):
         ms_k, b_k = ctx.time_kernel(which, min(rows_typ, 8), 240 if which < 4 else 40)
         per_kernel[nm] = {"us": round(ms_k * 1e3, 2), "GBps": round(b_k / (ms_k / 1e3) / 1e9, 1)}
+    # the attention kernel alone, every row on a cached context of its own at this context's capacity
+    att_rows = max(1, min(rows_typ, 8 * (1 if batch == 1 else 8)))
+    try:
+        ms_k, b_k = ctx.time_kernel(5, att_rows, 20)
+        per_kernel["attention"] = {"us": round(ms_k * 1e3, 2), "GBps": round(b_k / (ms_k / 1e3) / 1e9, 1), "rows": att_rows,
+                                   "context": int(b_k / (att_rows * shape.n_kv_heads * shape.head_dim * 4))}
+    except Exception as e:  # (a row count the context cannot carry)
+        per_kernel["attention"] = {"error": str(e)[:120]}
     # the same GEMM shapes on the tcgen05 / TMA kernel (used by the prefill passes; not by the decode passes that
     # `value` times), alone and back to back over several weight matrices: reported beside, never instead of, the above
     tc_alone = None
@@ -370,6 +386,8 @@ def run_ours(args):
                              "achieved": per_kernel["lm_head"]["GBps"], "peak": peak, "unit": "GB/s",
                              "frac": round(per_kernel["lm_head"]["GBps"] / peak, 4), "us_per_launch": per_kernel["lm_head"]["us"]},
         "kernels_alone": per_kernel,
+        "prefill": {"ms_per_sequence": round(prefill_ms_seq, 2), "prompt_len": n_prompt,
+                    "tok_per_s": round(n_prompt / (prefill_ms_seq / 1e3), 1), "what": "wall clock of loopspec_prefill (host ids in, first token out)"},
         "prefill_tcgen05_kernels_alone": tc_alone,
         "step_roofline": {"achieved": round(step_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(step_gbs / peak, 4),
                           "ms_per_pass": round(statistics.mean(dec_ms) / max(stats["steps"], 1), 4),
@@ -386,6 +404,18 @@ def run_ours(args):
                        "passes": stats["steps"]},
         "setup_s": round(t_setup, 1), "timed_region_wall_s": round(t_region, 2),
     }
+    att = per_kernel.get("attention", {})
+    if "GBps" in att and stats["rows_total"] * kv_row > stats["steps"] * (w_b + w_c):
+        # K/V bytes exceed weight bytes in a pass: the attention kernel is the dominant one
+        result["gemm_roofline"] = result["roofline"]
+        result["roofline"] = {"bound": "hbm", "kernel": "attn_runs_kernel (decode attention over the cached context: per-thread cp.async ring, "
+                              "running softmax per lane group)", "achieved": att["GBps"], "peak": peak, "unit": "GB/s",
+                              "frac": round(att["GBps"] / peak, 4), "peak_kind": f"of {peak_kind}",
+                              "frac_of_nominal_8TBs": round(att["GBps"] / NOMINAL_HBM_GBS, 4), "traffic": None, "traffic_source": None,
+                              "algorithmic_bytes_per_launch": att["rows"] * shape.n_kv_heads * att["context"] * shape.head_dim * 4,
+                              "us_per_launch": att["us"], "rows": att["rows"],
+                              "how": "CUDA events around back-to-back launches, cycling over the layers' KV pools; every row reads K and V "
+                                     "of its own (sequence, recurrence) at the context's capacity"}
     if rank == 0 and world == 1 and batch == 1 and not args.no_calibrated and (args.calibrated or args.workload == "ouro_1p4b"):
         ctx.close()
         ctx = None
@@ -514,7 +544,7 @@ def main():
     ap.add_argument("--closed-form", action="store_true",
                     help="sampling workloads: pick (d1, d2) from Theorem 2 on a TV profile measured on the device first")
     ap.add_argument("--kernel-only", choices=KERNELS, help="time one kernel of the pass alone and exit")
-    ap.add_argument("--linear-tc", choices=KERNELS, help="time the tcgen05 / TMA linear operator on this GEMM shape and exit")
+    ap.add_argument("--linear-tc", choices=KERNELS[:5], help="time the tcgen05 / TMA linear operator on this GEMM shape and exit")
     ap.add_argument("--profile-pass", type=int, default=0, help="prefill, decode this many tokens, exit (for profilers)")
     ap.add_argument("--rows", type=int, default=4)
     ap.add_argument("--iters", type=int, default=10)

@@ -204,7 +204,9 @@ int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);
 /* Time `iters` back-to-back launches of one kernel of the pass in the decode launch configuration, cycling
  * over the layers' weights (so successive launches read different memory): which = 0 qkv, 1 o-proj,
  * 2 gate/up, 3 down, 4 lm_head, 5 the attention kernel with every row reading a cached context of (max_ctx - 64)
- * positions of its own (row i: sequence i mod max_seqs, recurrence 1 + (i / max_seqs) mod R).  rows = token rows
+ * positions of its own (row i: sequence i mod max_seqs, recurrence 1 + (i / max_seqs) mod R), 6 the attention of a
+ * prefill pass: `rows` (<= max_prefill_rows) consecutive positions of sequence 0 ending at position max_ctx - 65, which
+ * share the cached keys and values (bytes_out: those of one context).  rows = token rows
  * carried.  ms_out: mean milliseconds per launch measured with CUDA events on the context's stream; bytes_out: weight
  * (which = 5: key and value) bytes one launch streams.  Sequences need a new prefill afterwards. */
 int loopspec_time_kernel(loopspec_ctx*, int32_t which, int32_t rows, int32_t iters, float* ms_out,

@@ -624,11 +624,11 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtsCfg<D, G>::MIN_CTAS)) attn_ru
 // key) tile and the weighted values are register-tiled fp32 FMAs (the query is fp32, keys and values are bf16 values held
 // exactly in fp32: the same products as the decode kernels form), and every row keeps a running softmax over the
 // chunks of the run.  Runs are cut at fixed absolute positions - every chunk below position ATT_PF_SINGLE * 64 is a run
-// of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending order by the CTA that
-// finishes the row's last one, so a row's result depends on its own prefix only, not on how the prompt was cut into
+// of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending order by a second kernel
+// (attn_prefill_fold_kernel), so a row's result depends on its own prefix only, not on how the prompt was cut into
 // passes.
 constexpr int ATT_PF_SINGLE = 40;
-constexpr int ATT_PF_RUN = 16;
+constexpr int ATT_PF_RUN = 4;
 __host__ __device__ inline int att_pf_run_of_chunk(int c) { return c < ATT_PF_SINGLE ? c : ATT_PF_SINGLE + (c - ATT_PF_SINGLE) / ATT_PF_RUN; }
 __host__ __device__ inline int att_pf_run_first_chunk(int run) {
   return run < ATT_PF_SINGLE ? run : ATT_PF_SINGLE + (run - ATT_PF_SINGLE) * ATT_PF_RUN;
@@ -659,7 +659,6 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
   unsigned char* s_v = atp_smem + C::V_OFF;
   float* s_s = reinterpret_cast<float*>(atp_smem + C::S_OFF);
   float* s_st = reinterpret_cast<float*>(atp_smem + C::ST_OFF);  // [row][4]
-  __shared__ int s_lastrow[ATT_PF_ROWS];
 
   const RowTable* tab = p.tab;  // written before this pass started
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
@@ -831,52 +830,55 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
         if (tx == 0) __stcg(mypart + D, m), __stcg(mypart + D + 1, l);
       }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid < ATT_PF_ROWS) {
-      const int row = tid, pos = p0 + row;
-      int last = 0;
-      if (row < n_rows && c_lo * ATT_CHUNK <= pos) {
-        const int n_runs_row = att_pf_run_of_chunk(pos / ATT_CHUNK) + 1;
-        if (n_runs_row > 1) {
-          const int old = atomicAdd(p.counters + row * p.n_q_heads + h, 1);
-          last = (old == n_runs_row - 1) ? n_runs_row : 0;
-        }
-      }
-      s_lastrow[row] = last;
-      __threadfence();
+  }
+}
+
+// ... and the fold of a row's runs, in ascending order: one CTA per (row, query head), one lane per four dims.  A
+// kernel of its own so that the folds of a pass (up to 64 rows x all heads x up to ATT_PF_SINGLE + max_ctx / 1024 runs)
+// spread over the whole device instead of queuing in whichever CTA finished a head last.
+template <int D>
+__global__ void __launch_bounds__(D / 4) attn_prefill_fold_kernel(const __grid_constant__ AttnParams p) {
+  constexpr int PSTRIDE = D + 2;
+  const RowTable* tab = p.tab;
+  const int row = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (row >= min(tab->n_rows, ATT_PF_ROWS)) return;
+  const int n_runs = att_pf_run_of_chunk(tab->pos[row] / ATT_CHUNK) + 1;
+  if (n_runs == 1) return;  // finished by the attention kernel itself
+  const int G = p.n_q_heads / p.n_kv_heads, HQ = p.n_q_heads * D, kvh = h / G, gq = h - kvh * G;
+  const float* base = p.part + ((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks * G + gq) * PSTRIDE;
+  const size_t rstride = (size_t)G * PSTRIDE;
+  float m = -INFINITY;
+  for (int c0 = 0; c0 < n_runs; c0 += 8) {
+    float mm[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) mm[u] = (c0 + u < n_runs) ? __ldcg(base + (size_t)(c0 + u) * rstride + D) : -INFINITY;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) m = fmaxf(m, mm[u]);
+  }
+  float l = 0.f, acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int c0 = 0; c0 < n_runs; c0 += 8) {
+    float mc[8], lc[8];
+    float2 oa[8], ob[8];  // (a partial's D + 2 floats keep 8-byte alignment only)
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const bool ok = c0 + u < n_runs;
+      const float* pc = base + (size_t)(ok ? c0 + u : 0) * rstride;
+      mc[u] = ok ? __ldcg(pc + D) : -INFINITY, lc[u] = ok ? __ldcg(pc + D + 1) : 0.f;
+      oa[u] = ok ? __ldcg(reinterpret_cast<const float2*>(pc + tid * 4)) : make_float2(0.f, 0.f);
+      ob[u] = ok ? __ldcg(reinterpret_cast<const float2*>(pc + tid * 4 + 2)) : make_float2(0.f, 0.f);
     }
-    __syncthreads();
-    // ---- rows whose last run this was: fold their runs in ascending order (two rows at a time, one thread per dim) ----
-    for (int r0 = 0; r0 < n_rows; r0 += 2) {
-      const int row = r0 + (tid >> 7), dd = tid & 127;
-      if (row >= n_rows || dd >= D) continue;
-      const int n_runs_row = s_lastrow[row];
-      if (n_runs_row == 0) continue;
-      const float* base = p.part + ((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks * G + gq) * PSTRIDE;
-      const size_t rstride = (size_t)G * PSTRIDE;
-      float m = -INFINITY;
-      for (int c0 = 0; c0 < n_runs_row; ++c0) m = fmaxf(m, __ldcg(base + c0 * rstride + D));
-      float l = 0.f, acc = 0.f;
-      for (int c0 = 0; c0 < n_runs_row; c0 += 4) {
-        float mc[4], lc[4], oc[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const bool ok = c0 + u < n_runs_row;
-          const float* pc = base + (size_t)(ok ? c0 + u : 0) * rstride;
-          mc[u] = ok ? __ldcg(pc + D) : -INFINITY, lc[u] = ok ? __ldcg(pc + D + 1) : 0.f, oc[u] = ok ? __ldcg(pc + dd) : 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const float wgt = (mc[u] == -INFINITY) ? 0.f : expf(mc[u] - m);
-          l = fmaf(lc[u], wgt, l);
-          acc = fmaf(oc[u], wgt, acc);
-        }
-      }
-      store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + dd, acc / l);
-      if (dd == 0) p.counters[row * p.n_q_heads + h] = 0;
+    for (int u = 0; u < 8; ++u) {
+      const float wgt = (mc[u] == -INFINITY) ? 0.f : expf(mc[u] - m);
+      l = fmaf(lc[u], wgt, l);
+      acc[0] = fmaf(oa[u].x, wgt, acc[0]), acc[1] = fmaf(oa[u].y, wgt, acc[1]);
+      acc[2] = fmaf(ob[u].x, wgt, acc[2]), acc[3] = fmaf(ob[u].y, wgt, acc[3]);
     }
   }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + tid * 4 + i, acc[i] / l);
 }
 
 }  // namespace ls

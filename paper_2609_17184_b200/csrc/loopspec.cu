@@ -739,9 +739,16 @@ cudaError_t launch_attention(loopspec_ctx* c, const RowTable* tab, int l, unsign
   a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
   a.tl = tl, a.tl_id = tl_id;
   if (prefill_rows && c->pf_attn) {  // consecutive prompt positions of one sequence: the rows share every K/V chunk
-    if (m.head_dim == 128)
-      return launch_k(attn_prefill_kernel<128>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<128>::SMEM_BYTES, c->stream, a, c->use_pdl);
-    return launch_k(attn_prefill_kernel<64>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<64>::SMEM_BYTES, c->stream, a, c->use_pdl);
+    const dim3 fold_grid(d.max_rows_pf, m.n_q_heads);
+    cudaError_t e;
+    if (m.head_dim == 128) {
+      if ((e = launch_k(attn_prefill_kernel<128>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<128>::SMEM_BYTES, c->stream, a, c->use_pdl)))
+        return e;
+      return launch_k(attn_prefill_fold_kernel<128>, fold_grid, dim3(32), 0, c->stream, a, c->use_pdl);
+    }
+    if ((e = launch_k(attn_prefill_kernel<64>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtpCfg<64>::SMEM_BYTES, c->stream, a, c->use_pdl)))
+      return e;
+    return launch_k(attn_prefill_fold_kernel<64>, fold_grid, dim3(16), 0, c->stream, a, c->use_pdl);
   }
   const bool runs = d.max_chunks > ATT_MAX_RUNS;
   return launch_k(attn_fn(m.head_dim, G, runs), dim3(attn_grid(c->n_sm, G, runs)), dim3(ATT_THREADS), attn_smem(m.head_dim, G, runs), c->stream, a,
@@ -1567,7 +1574,8 @@ int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
 }
 
 int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_out, double* bytes_out) {
-  if (!c || which < 0 || which > 5 || rows < 1 || rows > 8 * c->ng_dec || iters < 1 || !ms_out) return LOOPSPEC_EINVAL;
+  if (!c || which < 0 || which > 6 || rows < 1 || rows > (which == 6 ? c->d.max_rows_pf : 8 * c->ng_dec) || iters < 1 || !ms_out)
+    return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "verification pending");
   // a scratch row table with `rows` plain rows on sequence 0 (hidden states of the prefill area; outputs go to
@@ -1592,6 +1600,19 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
     }
     t.chunk_start[rows] = items, t.attn_items = items;
   }
+  if (which == 6) {
+    // prefill attention: `rows` consecutive prompt positions of sequence 0 at recurrence 1, the last one at the end of
+    // the cached context (the capacity minus one chunk)
+    const int ctx = std::max(rows, c->d.ids_cap - ATT_CHUNK);
+    int items = 0;
+    for (int i = 0; i < rows; ++i) {
+      const int pos = ctx - rows + i;
+      t.seq[i] = 0, t.r[i] = 1, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_safe[i] = ctx - rows, t.n_spec[i] = 0;
+      t.chunk_start[i] = items;
+      items += att_items(pos + 1);
+    }
+    t.chunk_start[rows] = items, t.attn_items = items;
+  }
   CU(c, cudaMemcpyAsync(c->ws + c->L.tab_pf, &t, sizeof t, cudaMemcpyHostToDevice, c->stream));
   CU(c, cudaMemsetAsync(c->ws + c->L.hid + (size_t)c->d.S * c->d.NB * c->m.hidden * 4, 0, (size_t)rows * c->m.hidden * 4, c->stream));
   const RowTable* tab = c->at<RowTable>(c->L.tab_pf);
@@ -1599,8 +1620,8 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   if (kTune && getenv("LOOPSPEC_TK_LAYERS")) L = std::max(1, std::min(L, atoi(getenv("LOOPSPEC_TK_LAYERS"))));  // L2-resident weights
   auto run = [&](int n) -> cudaError_t {
     for (int i = 0; i < n; ++i) {
-      if (which == 5) {
-        cudaError_t e = launch_attention(c, tab, i % L, nullptr, 0);
+      if (which >= 5) {
+        cudaError_t e = launch_attention(c, tab, i % L, nullptr, 0, which == 6);
         if (e) return e;
         continue;
       }
@@ -1625,8 +1646,8 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   double nk[5] = {(double)(d.Hq + 2 * d.Hkv) * c->m.hidden, (double)c->m.hidden * d.Hq, 2.0 * c->m.ffn * c->m.hidden,
                   (double)c->m.hidden * c->m.ffn, (double)c->m.vocab * c->m.hidden};
   if (bytes_out) {
-    *bytes_out = which < 5 ? nk[which] * wb
-                           : 2.0 * rows * c->m.n_kv_heads * (double)std::max(1, d.ids_cap - ATT_CHUNK) * c->m.head_dim * 2;  // K and V, bf16
+    const double kv_ctx = 2.0 * c->m.n_kv_heads * (double)std::max(1, d.ids_cap - ATT_CHUNK) * c->m.head_dim * 2;  // K and V of a context, bf16
+    *bytes_out = which < 5 ? nk[which] * wb : which == 5 ? rows * kv_ctx : kv_ctx;  // (the rows of a prefill pass share one context)
   }
   // the timed launches touched sequence state only through scratch; mark sequences as needing a new prefill
   std::fill(c->prefilled.begin(), c->prefilled.end(), 0);
