@@ -634,25 +634,30 @@ __host__ __device__ inline int att_pf_run_first_chunk(int run) {
   return run < ATT_PF_SINGLE ? run : ATT_PF_SINGLE + (run - ATT_PF_SINGLE) * ATT_PF_RUN;
 }
 constexpr int ATT_PF_ROWS = 64;  // rows of a pass at most (one group of token columns)
-template <int D>
+// RT = rows per thread: a work item carries 16 RT rows of the pass.  Smaller items finish sooner (short prompts, where a
+// pass offers only heads x chunks items), larger ones reuse a staged chunk for more rows; a row's arithmetic is the same.
+template <int D, int RT>
 struct AtpCfg {
+  static constexpr int IR = 16 * RT;         // rows per item
   static constexpr int QS = D + 4;           // floats per query row in shared memory
   static constexpr int KS = D * 2 + 16;      // bytes per key row (the pad spreads the keys a quarter warp reads over the banks)
   static constexpr int VS = D * 2;           // bytes per value row
   static constexpr int SS = ATT_CHUNK + 1;   // floats per score row
   static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = Q_OFF + ATT_PF_ROWS * QS * 4;
+  static constexpr int K_OFF = Q_OFF + IR * QS * 4;
   static constexpr int V_OFF = K_OFF + ATT_CHUNK * KS;
   static constexpr int S_OFF = V_OFF + ATT_CHUNK * VS;
-  static constexpr int ST_OFF = S_OFF + ATT_PF_ROWS * SS * 4;   // per row: running max, running mass, rescale of this chunk
-  static constexpr int SMEM_BYTES = ST_OFF + ATT_PF_ROWS * 4 * 4;
+  static constexpr int ST_OFF = S_OFF + IR * SS * 4;   // per row: running max, running mass, rescale of this chunk
+  static constexpr int SMEM_BYTES = ST_OFF + IR * 4 * 4;
+  static constexpr int MIN_CTAS = RT >= 4 ? 2 : 3;
 };
 
-template <int D>
-__global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
-  using C = AtpCfg<D>;
+template <int D, int RT>
+__global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
+  using C = AtpCfg<D, RT>;
+  constexpr int IR = C::IR;
   constexpr int PSTRIDE = D + 2;
-  constexpr int DPT = D / 16;  // dims of the output a thread accumulates (for each of its 4 rows)
+  constexpr int DPT = D / 16;  // dims of the output a thread accumulates (for each of its RT rows)
   extern __shared__ __align__(16) unsigned char atp_smem[];
   float* s_q = reinterpret_cast<float*>(atp_smem + C::Q_OFF);
   unsigned char* s_k = atp_smem + C::K_OFF;
@@ -669,31 +674,34 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
   const int p0 = tab->pos[0], seq = tab->seq[0];
   const int n_ctx = p0 + n_rows;                                   // keys 0 .. n_ctx - 1
   const int n_runs_all = att_pf_run_of_chunk((n_ctx - 1) / ATT_CHUNK) + 1;
+  const int n_blocks = (n_rows + IR - 1) / IR;
   const int G = p.n_q_heads / p.n_kv_heads, HQ = p.n_q_heads * D;
   const size_t plane = (size_t)(tab->r[0] - 1) * p.kv_plane_stride;
-  const int total = p.n_q_heads * n_runs_all;
+  const int total = p.n_q_heads * n_blocks * n_runs_all;
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
-    const int h = item % p.n_q_heads, run = item / p.n_q_heads;
+    const int h = item % p.n_q_heads, rest = item / p.n_q_heads;
+    const int blk = rest % n_blocks, run = rest / n_blocks;
+    const int row0 = blk * IR, rows_here = min(IR, n_rows - row0);  // this item's rows of the pass
     const int kvh = h / G, gq = h - kvh * G;
-    const int c_lo = att_pf_run_first_chunk(run), c_hi = min(att_pf_run_first_chunk(run + 1), (n_ctx + ATT_CHUNK - 1) / ATT_CHUNK);
+    const int c_lo = att_pf_run_first_chunk(run);
+    // keys beyond the block's last position are never visible to it: the run ends there
+    const int c_hi = min(att_pf_run_first_chunk(run + 1), (p0 + row0 + rows_here - 1) / ATT_CHUNK + 1);
+    if (c_lo >= c_hi) continue;  // (uniform over the CTA) none of the block's rows reaches this run
     const __nv_bfloat16* Kb = p.kv + plane + (size_t)(seq * p.n_kv_heads + kvh) * p.slots * D;
     const __nv_bfloat16* Vb = Kb + p.kv_sel_stride;
     __syncthreads();  // the previous item is done with the shared buffers
-    // queries of every row for this head (fp32), and the rows' softmax state
-    for (int idx = tid; idx < n_rows * (D / 4); idx += ATT_THREADS) {
-      const int row = idx / (D / 4), d4 = idx - row * (D / 4);
-      *reinterpret_cast<float4*>(s_q + row * C::QS + d4 * 4) =
-          *reinterpret_cast<const float4*>(p.qbuf + (size_t)row * HQ + (size_t)h * D + d4 * 4);
+    // queries of the block's rows for this head (fp32), and the rows' softmax state
+    for (int idx = tid; idx < IR * (D / 4); idx += ATT_THREADS) {
+      const int lr = idx / (D / 4), d4 = idx - lr * (D / 4);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);  // rows the pass does not have: zeros
+      if (lr < rows_here) v = *reinterpret_cast<const float4*>(p.qbuf + (size_t)(row0 + lr) * HQ + (size_t)h * D + d4 * 4);
+      *reinterpret_cast<float4*>(s_q + lr * C::QS + d4 * 4) = v;
     }
-    for (int idx = tid; idx < (ATT_PF_ROWS - n_rows) * (D / 4); idx += ATT_THREADS) {  // rows the pass does not have: zeros
-      const int row = n_rows + idx / (D / 4), d4 = idx % (D / 4);
-      *reinterpret_cast<float4*>(s_q + row * C::QS + d4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    if (tid < ATT_PF_ROWS) s_st[tid * 4] = -INFINITY, s_st[tid * 4 + 1] = 0.f, s_st[tid * 4 + 2] = 1.f;
-    float o[4][DPT];
+    if (tid < IR) s_st[tid * 4] = -INFINITY, s_st[tid * 4 + 1] = 0.f, s_st[tid * 4 + 2] = 1.f;
+    float o[RT][DPT];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < RT; ++a)
 #pragma unroll
       for (int i = 0; i < DPT; ++i) o[a][i] = 0.f;
 
@@ -701,7 +709,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
       const int k0 = chunk * ATT_CHUNK;
       const int n_keys = min(ATT_CHUNK, n_ctx - k0);  // keys of this chunk that exist (all of them written)
       if (chunk > c_lo) __syncthreads();               // the previous chunk's readers are done
-      // ---- the chunk's keys and values, once for all rows -------------------------------------------------------
+      // ---- the chunk's keys and values, once for all rows of the block ------------------------------------------
       for (int idx = tid; idx < ATT_CHUNK * (D / 8); idx += ATT_THREADS) {
         const int key = idx / (D / 8), pc = idx - key * (D / 8);
         const bool ok = key < n_keys;
@@ -712,19 +720,19 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       __syncthreads();
-      // ---- scores: thread (ty, tx) takes rows 4 ty .. 4 ty + 3 and keys tx, tx + 16, tx + 32, tx + 48 ---------------
-      float sc[4][4];
+      // ---- scores: thread (ty, tx) takes rows RT ty .. RT ty + RT - 1 and keys tx, tx + 16, tx + 32, tx + 48 ---------
+      float sc[RT][4];
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+      for (int a = 0; a < RT; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) sc[a][b] = 0.f;
 #pragma unroll 2
       for (int d = 0; d < D; d += 8) {
-        float4 qa[4], qb[4];
+        float4 qa[RT], qb[RT];
 #pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          qa[a] = *reinterpret_cast<const float4*>(s_q + (4 * ty + a) * C::QS + d);
-          qb[a] = *reinterpret_cast<const float4*>(s_q + (4 * ty + a) * C::QS + d + 4);
+        for (int a = 0; a < RT; ++a) {
+          qa[a] = *reinterpret_cast<const float4*>(s_q + (RT * ty + a) * C::QS + d);
+          qb[a] = *reinterpret_cast<const float4*>(s_q + (RT * ty + a) * C::QS + d + 4);
         }
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
@@ -734,7 +742,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
           const float k4f = __uint_as_float(kw.z << 16), k5f = __uint_as_float(kw.z & 0xffff0000u);
           const float k6f = __uint_as_float(kw.w << 16), k7f = __uint_as_float(kw.w & 0xffff0000u);
 #pragma unroll
-          for (int a = 0; a < 4; ++a) {  // dims in ascending order, one chain per (row, key)
+          for (int a = 0; a < RT; ++a) {  // dims in ascending order, one chain per (row, key)
             float v = sc[a][b];
             v = fmaf(qa[a].x, k0f, v), v = fmaf(qa[a].y, k1f, v), v = fmaf(qa[a].z, k2f, v), v = fmaf(qa[a].w, k3f, v);
             v = fmaf(qb[a].x, k4f, v), v = fmaf(qb[a].y, k5f, v), v = fmaf(qb[a].z, k6f, v), v = fmaf(qb[a].w, k7f, v);
@@ -743,26 +751,26 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
         }
       }
 #pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        const int row = 4 * ty + a, pos = p0 + row;
+      for (int a = 0; a < RT; ++a) {
+        const int lr = RT * ty + a, pos = p0 + row0 + lr;
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           const int key = tx + 16 * b;
-          const bool ok = row < n_rows && key < n_keys && k0 + key <= pos;  // causal
-          s_s[row * C::SS + key] = ok ? sc[a][b] * p.scale : -INFINITY;
+          const bool ok = lr < rows_here && key < n_keys && k0 + key <= pos;  // causal
+          s_s[lr * C::SS + key] = ok ? sc[a][b] * p.scale : -INFINITY;
         }
       }
       __syncthreads();
       // ---- running softmax of every row: four threads per row, 16 keys each, folded in a fixed order ----------------
-      {
-        const int row = tid >> 2, part = tid & 3;
-        float* sr = s_s + row * C::SS + part * 16;
+      if (tid < 4 * IR) {
+        const int lr = tid >> 2, part = tid & 3;
+        float* sr = s_s + lr * C::SS + part * 16;
         float m = -INFINITY;
 #pragma unroll
         for (int jj = 0; jj < 16; ++jj) m = fmaxf(m, sr[jj]);
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-        const float m_old = s_st[row * 4], l_old = s_st[row * 4 + 1];
+        const float m_old = s_st[lr * 4], l_old = s_st[lr * 4 + 1];
         const float m_new = fmaxf(m_old, m);
         float l = 0.f;
 #pragma unroll
@@ -778,17 +786,17 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
         __syncwarp();
         if (part == 0) {
           const float wa = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);  // (a row that has seen no key yet: nothing to rescale)
-          s_st[row * 4] = m_new, s_st[row * 4 + 1] = fmaf(l_old, wa, lc), s_st[row * 4 + 2] = (m_new == -INFINITY) ? 1.f : wa;
+          s_st[lr * 4] = m_new, s_st[lr * 4 + 1] = fmaf(l_old, wa, lc), s_st[lr * 4 + 2] = (m_new == -INFINITY) ? 1.f : wa;
         }
       }
       __syncthreads();
-      // ---- weighted values: thread (ty, tx) takes rows 4 ty .. + 3 and dims tx * DPT .. + DPT - 1, keys in ascending order --
+      // ---- weighted values: thread (ty, tx) takes its RT rows and dims tx * DPT .. + DPT - 1, keys in ascending order --
       {
-        float wa[4];
+        float wa[RT];
 #pragma unroll
-        for (int a = 0; a < 4; ++a) wa[a] = s_st[(4 * ty + a) * 4 + 2];
+        for (int a = 0; a < RT; ++a) wa[a] = s_st[(RT * ty + a) * 4 + 2];
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+        for (int a = 0; a < RT; ++a)
 #pragma unroll
           for (int i = 0; i < DPT; ++i) o[a][i] *= wa[a];
         for (int key = 0; key < n_keys; ++key) {
@@ -804,8 +812,8 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
             vf[2] = __uint_as_float(vw.y << 16), vf[3] = __uint_as_float(vw.y & 0xffff0000u);
           }
 #pragma unroll
-          for (int a = 0; a < 4; ++a) {
-            const float pw = s_s[(4 * ty + a) * C::SS + key];
+          for (int a = 0; a < RT; ++a) {
+            const float pw = s_s[(RT * ty + a) * C::SS + key];
 #pragma unroll
             for (int i = 0; i < DPT; ++i) o[a][i] = fmaf(pw, vf[i], o[a][i]);
           }
@@ -813,13 +821,13 @@ __global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_kernel(const __gr
       }
     }
     __syncthreads();  // every thread has read the final state
-    // ---- the run is done: rows with one run only are finished here, the others leave a partial -----------------------
+    // ---- the run is done: rows with one run only are finished here, the others leave a partial for the fold -----------
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const int row = 4 * ty + a, pos = p0 + row;
-      if (row >= n_rows || c_lo * ATT_CHUNK > pos) continue;   // the row does not reach this run
+    for (int a = 0; a < RT; ++a) {
+      const int lr = RT * ty + a, row = row0 + lr, pos = p0 + row;
+      if (lr >= rows_here || c_lo * ATT_CHUNK > pos) continue;   // the row does not reach this run
       const int n_runs_row = att_pf_run_of_chunk(pos / ATT_CHUNK) + 1;
-      const float m = s_st[row * 4], l = s_st[row * 4 + 1];
+      const float m = s_st[lr * 4], l = s_st[lr * 4 + 1];
       if (n_runs_row == 1) {
 #pragma unroll
         for (int i = 0; i < DPT; ++i) store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + tx * DPT + i, o[a][i] / l);
