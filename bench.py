@@ -32,6 +32,11 @@ import workloads as W  # noqa: E402
 # launch configuration (`bench.py --kernel-only gate_up`), reported with its source and only for that model shape.
 NCU_TRAFFIC = {"ouro_1p4b": (46226944, "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch, captured on "
                                        "`bench.py --kernel-only gate_up --rows 4` (not measured in this run)")}
+# the streaming attention kernel: ncu DRAM bytes of one launch on a small case (4 rows x 4096 cached positions: 137.7 MB
+# against 134.2 MB algorithmic); its traffic grows in proportion to rows x context, so a full-size launch is scaled by
+# the units it processes
+ATTN_TRAFFIC = (137.7e6 / 134.2e6, "ncu dram__bytes.sum of one launch of `bench.py --kernel-only attention --rows 4 --prompt-len 4096` "
+                                   "(137.7 MB for 134.2 MB algorithmic), scaled to this launch's rows x context (not measured in this run)")
 NOMINAL_HBM_GBS = 8000.0  # datasheet figure, for context beside the measured copy bandwidth
 
 
@@ -117,6 +122,11 @@ def vanilla_bytes(shape, n_prompt, n_decode, batch=1):
 
 
 KERNELS = ["qkv", "o_proj", "gate_up", "down", "lm_head", "attention"]
+GATE_UP_KERNEL = ["gemm_bf16_kernel<1, SwiGLU> (gate/up projection of a decode pass on mma.sync cluster kernels; the kernel with the "
+                  "largest share of a pass)",
+                  "linear_tc_kernel + tc_epilogue_kernel<SwiGLU> (gate/up projection of a decode pass of 9 to 64 rows: TMA + tcgen05.mma, "
+                  "k-split sums folded by the epilogue kernel; both launches are timed)",
+                  "gemm_f32_kernel<NG, SwiGLU> (gate/up projection of a decode pass, fp32 weights on CUDA cores)"]
 
 
 def replica_throughput(tokens_per_rank, device_ms, wall_s, dist=None, device=None):
@@ -336,7 +346,7 @@ def run_ours(args):
     att_rows = max(1, min(rows_typ, 8 * (1 if batch == 1 else 8)))
     try:
         ms_k, b_k = ctx.time_kernel(5, att_rows, 20)
-        per_kernel["attention"] = {"us": round(ms_k * 1e3, 2), "GBps": round(b_k / (ms_k / 1e3) / 1e9, 1), "rows": att_rows,
+        per_kernel["attention"] = {"us": round(ms_k * 1e3, 2), "GBps": round(b_k / (ms_k / 1e3) / 1e9, 1), "rows": att_rows, "path": ctx.decode_paths()[1],
                                    "context": int(b_k / (att_rows * shape.n_kv_heads * shape.head_dim * 4))}
     except Exception as e:  # (a row count the context cannot carry)
         per_kernel["attention"] = {"error": str(e)[:120]}
@@ -361,6 +371,8 @@ def run_ours(args):
     step_gbs = total_b / (statistics.mean(dec_ms) / 1e3) / 1e9
     van_gbs = vanilla_bytes(shape, n_prompt, n_decode, batch) / (statistics.mean(van_ms) / 1e3) / 1e9
     n = max(stats["n_decode"], 1)
+    # (the captured traffic figure is the mma.sync gate/up kernel's: it does not describe the tcgen05 path of wide passes)
+    gu_traffic = NCU_TRAFFIC.get(wl.model, (None, None)) if ctx.decode_paths()[0] == 0 else (None, None)
     result = {
         "metric": "decode_tok_per_s", "value": round(value, 2), "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 3), "higher_is_better": True, "scaling": "weak",
@@ -374,11 +386,10 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(batch * n_decode * 4 + 64),
                 "what": "wall clock of loopspec_prefill (host prompt ids, once per sequence) + loopspec_decode (host id buffer) per job"},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "gemm_bf16_kernel<NG, SwiGLU> (gate/up projection of a decode pass; the kernel "
-                                               "with the largest share of a pass)",
+        "roofline": {"bound": "hbm", "kernel": GATE_UP_KERNEL[ctx.decode_paths()[0] if shape.weight_dtype == "bf16" else 2],
                      "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
-                     "traffic": NCU_TRAFFIC.get(wl.model, (None, None))[0], "traffic_source": NCU_TRAFFIC.get(wl.model, (None, None))[1],
+                     "traffic": gu_traffic[0], "traffic_source": gu_traffic[1],
                      "algorithmic_bytes_per_launch": k_bytes, "us_per_launch": round(k_ms * 1e3, 2), "rows": min(rows_typ, 8),
                      "how": "CUDA events around back-to-back launches in the decode launch configuration, cycling over the layers' weights"},
         "readout_roofline": {"kernel": "dgemm_kernel<LOGITS> (lm_head of a decode pass: tcgen05.mma + TMA ring + cluster split-K)"
@@ -408,11 +419,14 @@ def run_ours(args):
     if "GBps" in att and stats["rows_total"] * kv_row > stats["steps"] * (w_b + w_c):
         # K/V bytes exceed weight bytes in a pass: the attention kernel is the dominant one
         result["gemm_roofline"] = result["roofline"]
-        result["roofline"] = {"bound": "hbm", "kernel": "attn_runs_kernel (decode attention over the cached context: per-thread cp.async ring, "
-                              "running softmax per lane group)", "achieved": att["GBps"], "peak": peak, "unit": "GB/s",
+        att_bytes = att["rows"] * shape.n_kv_heads * att["context"] * shape.head_dim * 4
+        result["roofline"] = {"bound": "hbm", "kernel": ("attn_runs_kernel (decode attention over the cached context: per-thread cp.async ring, "
+                              "running softmax per lane group)") if att.get("path") else "attn_kernel (decode attention, one work item per 64-position chunk)", "achieved": att["GBps"], "peak": peak, "unit": "GB/s",
                               "frac": round(att["GBps"] / peak, 4), "peak_kind": f"of {peak_kind}",
-                              "frac_of_nominal_8TBs": round(att["GBps"] / NOMINAL_HBM_GBS, 4), "traffic": None, "traffic_source": None,
-                              "algorithmic_bytes_per_launch": att["rows"] * shape.n_kv_heads * att["context"] * shape.head_dim * 4,
+                              "frac_of_nominal_8TBs": round(att["GBps"] / NOMINAL_HBM_GBS, 4),
+                              "traffic": int(att_bytes * ATTN_TRAFFIC[0]) if att.get("path") else None,
+                              "traffic_source": ATTN_TRAFFIC[1] if att.get("path") else None,
+                              "algorithmic_bytes_per_launch": att_bytes,
                               "us_per_launch": att["us"], "rows": att["rows"],
                               "how": "CUDA events around back-to-back launches, cycling over the layers' KV pools; every row reads K and V "
                                      "of its own (sequence, recurrence) at the context's capacity"}

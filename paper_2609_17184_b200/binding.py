@@ -12,7 +12,7 @@ _LIB_PATH = os.path.join(_HERE, "libloopspec.so")
 EXPORTS = ["loopspec_workspace_bytes", "loopspec_init", "loopspec_prefill", "loopspec_step", "loopspec_verify",
            "loopspec_decode", "loopspec_vanilla_decode", "loopspec_pick_depths", "loopspec_fit_envelope", "loopspec_max_branches",
            "loopspec_get_stats", "loopspec_get_commits", "loopspec_get_row_trace", "loopspec_debug_logits",
-           "loopspec_launches_per_step", "loopspec_debug_drop_tile", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
+           "loopspec_launches_per_step", "loopspec_decode_paths", "loopspec_debug_drop_tile", "loopspec_time_kernel", "loopspec_linear_scratch_bytes", "loopspec_op_linear",
            "loopspec_op_linear_static", "loopspec_linear_tc_scratch_bytes", "loopspec_op_linear_tc", "loopspec_time_linear_tc",
            "loopspec_last_error", "loopspec_destroy"]
 
@@ -81,6 +81,7 @@ def _load():
     lib.loopspec_get_row_trace.argtypes = [V, P(I), I, P(I)]
     lib.loopspec_debug_logits.argtypes = [V, I, I, P(C.c_float)]
     lib.loopspec_launches_per_step.argtypes = [V, P(I)]
+    lib.loopspec_decode_paths.argtypes = [V, P(I), P(I)]
     lib.loopspec_debug_drop_tile.argtypes = [V, I, I]
     lib.loopspec_time_kernel.argtypes = [V, I, I, I, P(C.c_float), P(C.c_double)]
     lib.loopspec_linear_scratch_bytes.restype = C.c_size_t
@@ -339,6 +340,12 @@ class LoopSpec:
         n = C.c_int32()
         self._check(lib.loopspec_launches_per_step(self.h, C.byref(n)))
         return n.value
+
+    def decode_paths(self):
+        """(gemm_path, attention_path) of this context's decode passes: see loopspec_decode_paths."""
+        g, a = C.c_int32(), C.c_int32()
+        self._check(lib.loopspec_decode_paths(self.h, C.byref(g), C.byref(a)))
+        return g.value, a.value
 
     def time_kernel(self, which, rows, iters):
         ms, nbytes = C.c_float(), C.c_double()

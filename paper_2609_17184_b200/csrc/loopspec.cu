@@ -1588,6 +1588,13 @@ int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   return LOOPSPEC_OK;
 }
 
+int loopspec_decode_paths(loopspec_ctx* c, int32_t* gemm_path, int32_t* attention_path) {
+  if (!c) return LOOPSPEC_EINVAL;
+  if (gemm_path) *gemm_path = c->tc[1].on ? 1 : 0;
+  if (attention_path) *attention_path = c->d.max_chunks > ATT_MAX_RUNS ? 1 : 0;
+  return LOOPSPEC_OK;
+}
+
 int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_out, double* bytes_out) {
   if (!c || which < 0 || which > 6 || rows < 1 || rows > (which == 6 ? c->d.max_rows_pf : 8 * c->ng_dec) || iters < 1 || !ms_out)
     return LOOPSPEC_EINVAL;
