@@ -6,7 +6,8 @@ Only tests, the smoke check and the benchmark's CPU-baseline leg may import
 it; it shares no code with the CUDA path.
 
 Parity status of what lives here:
-  * model forward, depth-indexed KV  : pinned (cache-free library forward)
+  * model forward, depth-indexed KV  : pinned (cache-free library forward; for the prelude / recurrent / coda layout
+    also the adapter on [state; prelude output], the prelude cache and every readout depth's coda cache)
   * residual operator, cascade rule  : pinned (exact enumeration, chi-square, Thm 1)
   * top-k / top-p filter, masked second proposal: pinned (definition on small
     cases, exact enumeration of the output law)
