@@ -1229,6 +1229,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     if (!ok) (void)cudaGetLastError();
     c->dg = ok;
   }
+  if (kTune && getenv("LOOPSPEC_DBG")) fprintf(stderr, "LOOPSPEC_TUNE region at workspace offset %zu\n", c->L.tune);
   auto bail = [&](int code, const char* what) {
     loopspec_destroy(c);
     (void)what;
@@ -1648,6 +1649,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
         continue;
       }
       GemmParams p = gemm_params(c, which, i % L, tab);
+      if (kTune && tune_timeline(c)) p.dbg = reinterpret_cast<long long*>(tune_timeline(c));  // phase stamps of CTA 0 (tuning builds)
       cudaError_t e = (c->dg && which == G_LM)         ? launch_dg_lm(c, tab)
                       : (c->tc[1].on && which != G_LM) ? launch_tc_gemm(c, which, i % L, tab, 1)
                                                        : launch_gemm(c->m.weight_dtype, c->ng_dec, kEpiOf[which], p, c->stream, c->use_pdl);
