@@ -8,7 +8,10 @@
                           shape with 2600-token prompts (contexts beyond 40 attention chunks), temperature 0.7,
                           (d1, d2) = (1, 2): tokens, commit records and row counts per sequence.
 
-    python tests/golden/make_config_goldens.py 2p6b|kv [--force]
+  raven_oracle.json       the Raven-style workload at full size (2 prelude + 4 recurrent + 2 coda blocks, R = 16, prompt
+                          256, greedy, (d1, d2) = (2, 8)): the first tokens with commit records, row counts and logit probes.
+
+    python tests/golden/make_config_goldens.py 2p6b|kv|raven [--force]
 
 Each takes tens of minutes and 12-25 GB of memory.
 """
@@ -120,9 +123,33 @@ def golden_kv(path):
     print("written in", round(time.time() - t0), "s", flush=True)
 
 
+def golden_raven(path):
+    wl = W.WORKLOADS["raven"]
+    shape = W.CONFIGS[wl.model]
+    n_tokens = 12
+    t0 = time.time()
+    model = LoopedLM(shape, W.make_weights(shape, seed=wl.weight_seed))
+    prompt = W.make_prompt(shape.vocab, wl.prompt_len, seed=wl.prompt_seed)
+    dec = Decoder(model, temperature=wl.temperature, seed=wl.sample_seed)
+    first = dec.prefill(prompt, n_tokens + 4, depths=(wl.d1, wl.d2))
+    print("prefill done", round(time.time() - t0), "s", flush=True)
+    toks = dec.loopspec(n_tokens, wl.d1, wl.d2, gate=wl.gate, keep_logits=True)
+    probe = [i for i in PROBE if i < shape.vocab] + [shape.vocab - 1]
+    rec = run_record(dec, toks)
+    rec["last_verify_logits_probe"] = {str(i): float(dec.verify_logits[-1][i]) for i in probe}
+    out = {"workload": "raven", "prompt_len": wl.prompt_len, "temperature": wl.temperature, "seed": wl.sample_seed,
+           "d1": wl.d1, "d2": wl.d2, "written_by": "tests/golden/make_config_goldens.py (oracle only)",
+           "first_token": first, "first_logits_probe": {str(i): float(dec.first_logits[i]) for i in probe},
+           "first_logits_argmax": int(np.argmax(dec.first_logits)), "n_tokens": n_tokens, "run": rec}
+    with open(path, "w") as f:
+        json.dump(out, f)
+    print("written in", round(time.time() - t0), "s", "min margin", rec["min_margin"], flush=True)
+
+
 if __name__ == "__main__":
     which = [a for a in sys.argv[1:] if not a.startswith("--")]
-    jobs = {"2p6b": ("ouro_2p6b_oracle.json", golden_2p6b), "kv": ("kv_bound_small_oracle.json", golden_kv)}
+    jobs = {"2p6b": ("ouro_2p6b_oracle.json", golden_2p6b), "kv": ("kv_bound_small_oracle.json", golden_kv),
+            "raven": ("raven_oracle.json", golden_raven)}
     for w in which or list(jobs):
         name, fn = jobs[w]
         path = os.path.join(HERE, name)
