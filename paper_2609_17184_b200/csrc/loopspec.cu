@@ -10,6 +10,11 @@
 #include <string>
 #include <vector>
 
+#if __has_include(<nvtx3/nvToolsExt.h>)
+#include <nvtx3/nvToolsExt.h>  // header-only: ranges show up when a profiler injects the NVTX library, cost nothing otherwise
+#define LOOPSPEC_NVTX 1
+#endif
+
 #include "attention.cuh"
 #include "common.cuh"
 #include "control.cuh"
@@ -442,6 +447,16 @@ struct loopspec_ctx {
 };
 
 namespace {
+
+// a named range around a C-ABI call (prefill, step, verify, decode), visible on a profiler's timeline
+struct Range {
+#ifdef LOOPSPEC_NVTX
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+#else
+  explicit Range(const char*) {}
+#endif
+};
 
 int fail(loopspec_ctx* c, int code, const char* fmt, ...) {
   if (c) {
@@ -1309,6 +1324,7 @@ int loopspec_destroy(loopspec_ctx* c) {
 const char* loopspec_last_error(loopspec_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
 int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* first_token) {
+  Range nvtx_range("loopspec_prefill");
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (seq < 0 || seq >= c->d.S || !prompt_ids || n < 1) return fail(c, LOOPSPEC_EINVAL, "bad prefill arguments");
@@ -1391,6 +1407,7 @@ static int arm_decode(loopspec_ctx* c, int n_tokens, bool unlimited = false) {
 }
 
 int loopspec_step(loopspec_ctx* c, int32_t* n_rows_out, int32_t* n_need_verify_out) {
+  Range nvtx_range("loopspec_step");
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (!any_prefilled(c)) return fail(c, LOOPSPEC_ESTATE, "step before prefill");
@@ -1409,6 +1426,7 @@ int loopspec_step(loopspec_ctx* c, int32_t* n_rows_out, int32_t* n_need_verify_o
 }
 
 int loopspec_verify(loopspec_ctx* c, loopspec_commit* out, int32_t max_out, int32_t* n_out) {
+  Range nvtx_range("loopspec_verify");
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (!c->pending_verify) return fail(c, LOOPSPEC_ESTATE, "no branch is at depth R");
@@ -1449,6 +1467,7 @@ static int copy_ids_out(loopspec_ctx* c, const std::vector<int>& start, int n_to
 }
 
 int loopspec_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
+  Range nvtx_range("loopspec_decode");
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");
@@ -1480,6 +1499,7 @@ int loopspec_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
 }
 
 int loopspec_vanilla_decode(loopspec_ctx* c, int32_t n_tokens, int32_t* ids_out) {
+  Range nvtx_range("loopspec_vanilla_decode");
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (n_tokens < 1) return fail(c, LOOPSPEC_EINVAL, "n_tokens must be positive");

@@ -178,3 +178,45 @@ def test_kv_bound_regime_at_reduced_size_matches_the_oracle():
         assert [c["step"] for c in alone.commits(s)] == [c[2] for c in g["seqs"][s]["commits"]]
         assert np.array_equal(alone.debug_logits(s, 0).view(np.uint32), logits[s].view(np.uint32))
         alone.close()
+
+
+# ---- Raven-style workload at full size (prelude / adapter / recurrent / coda blocks, R = 16, GQA 32:8 x 64, V = 128256) --------
+GOLD_RAVEN = os.path.join(os.path.dirname(__file__), "golden", "raven_oracle.json")
+
+
+def test_raven_style_workload_at_full_size_matches_the_oracle():
+    """Prompt 256, greedy, (d1, d2) = (2, 8), in the launch configuration bench.py times (passes of up to 18 rows: the
+    layers' GEMMs on the tcgen05 kernel, readout on the cluster kernel): first token, its logits, the first tokens of
+    the run with their commit records and row counts, the last verified logits; and greedy LoopSpec == vanilla."""
+    import paper_2609_17184_b200 as ls
+    g = json.load(open(GOLD_RAVEN))
+    wl = W.WORKLOADS["raven"]
+    shape = W.CONFIGS[wl.model]
+    assert (g["d1"], g["d2"], g["prompt_len"]) == (wl.d1, wl.d2, wl.prompt_len)
+    weights = ls.upload_weights(shape, W.make_weights(shape, seed=wl.weight_seed))
+    prompt = W.make_prompt(shape.vocab, wl.prompt_len, seed=wl.prompt_seed)
+    ctx = ls.LoopSpec(shape, weights, d1=wl.d1, d2=wl.d2, temperature=wl.temperature, seed=wl.sample_seed, gate=wl.gate, max_seqs=1,
+                      max_ctx=wl.prompt_len + wl.decode_len + 16, max_prefill_rows=64)
+    assert ctx.decode_paths()[0] == 1
+    assert ctx.prefill(prompt) == g["first_token"]
+    z = ctx.debug_logits(0, 0)
+    assert int(np.argmax(z)) == g["first_logits_argmax"]
+    for i, v in g["first_logits_probe"].items():
+        assert abs(z[int(i)] - v) <= 3e-2 + 2e-2 * abs(v)
+    run, n = g["run"], g["n_tokens"]
+    out = ctx.decode(n)[0].tolist()
+    decisions = sorted(m[2] for m in run["margins"] if m[0] != "filter")
+    assert out == run["tokens"], ("oracle's closest decisions", decisions[:3])
+    commits = ctx.commits(0)
+    assert [[c["source"], c["gate_open"], c["step"]] for c in commits] == run["commits"]
+    assert ctx.row_trace().tolist() == run["rows_per_step"]
+    st = ctx.stats()
+    for k, v in run["stats"].items():
+        if k != "gamma":
+            assert st[k] == v, k
+    z = ctx.debug_logits(0, 0)
+    for i, v in run["last_verify_logits_probe"].items():
+        assert abs(z[int(i)] - v) <= 3e-2 + 2e-2 * abs(v)
+    ctx.prefill(prompt)
+    assert ctx.vanilla_decode(n)[0].tolist() == run["tokens"]
+    ctx.close()
