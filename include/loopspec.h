@@ -202,8 +202,9 @@ int loopspec_debug_drop_tile(loopspec_ctx*, int32_t unit, int32_t wait_us);
 int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);
 
 /* Which kernels a decode pass of this context runs (fixed at loopspec_init by the row capacity of a pass and the
- * context capacity): *gemm_path = 0 the mma.sync cluster kernels (passes of up to 8 rows, fp32 weights, passes of
- * more than 64 rows), 1 the tcgen05 / TMA kernel + epilogue kernel (bf16 weights, passes of 9 to 64 rows);
+ * context capacity): *gemm_path = 0 the mma.sync cluster kernels (passes of up to 8 rows, fp32 weights), 1 the
+ * tcgen05 / TMA kernel + epilogue kernel (bf16 weights, passes of 9 or more rows, one pair of launches per group of 64
+ * token columns);
  * *attention_path = 0 one work item per 64-position chunk (context capacity up to 2560), 1 the streaming kernel over
  * runs of chunks.  Either pointer may be null. */
 int loopspec_decode_paths(loopspec_ctx*, int32_t* gemm_path, int32_t* attention_path);

@@ -765,9 +765,10 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
 constexpr int TCE_MAX_COLS = 64;
 constexpr int TCE_GROUPS = 16;   // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
 struct TcEpiParams {
-  GemmParams g;        // cluster_size = TCE_GROUPS
-  const float* part;   // [n_split][cols_ld][N]
+  GemmParams g;        // cluster_size = TCE_GROUPS; the per-column buffers start at the pass's first column
+  const float* part;   // [group][n_split][cols_ld][N]
   int n_split, cols_ld;
+  int Hq;              // query width (rows of the query buffer)
 };
 
 template <int EPI>
@@ -776,10 +777,20 @@ __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_
   __shared__ float s_colbuf[2 * RB_ROWS];
   __shared__ float s_rstd[TCE_MAX_COLS];
   __shared__ int s_ct[CT_FIELDS * TCE_MAX_COLS];
-  const GemmParams& p = q.g;
+  // blockIdx.z = group of TCE_MAX_COLS token columns: its slices of the per-column buffers
+  GemmParams p = q.g;
+  {
+    const int col0 = (int)blockIdx.z * TCE_MAX_COLS;
+    p.col0 = col0;
+    if (p.out_planes) p.out_planes += (size_t)col0 * 3 * p.planes_ld;
+    if (p.sumsq) p.sumsq += (size_t)col0 * p.sq_stride;
+    if (p.sumsq_out) p.sumsq_out += (size_t)col0 * p.n_sq_out;
+    if (p.qbuf) p.qbuf += (size_t)col0 * q.Hq;
+  }
+  const float* part = q.part + (size_t)blockIdx.z * q.n_split * q.cols_ld * p.N;
   const int tid = threadIdx.x, rb = blockIdx.x;
   const RowTable* tab = p.tab;  // final before the pass starts
-  int n_cols = tab->n_rows;
+  int n_cols = tab->n_rows - p.col0;  // this group's live columns
   if (n_cols > TCE_MAX_COLS) n_cols = TCE_MAX_COLS;
   gemm_load_cols(p, n_cols, TCE_MAX_COLS, s_ct);
   pdl_launch_dependents();
@@ -812,7 +823,7 @@ __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_
   for (int c = rank + TCE_GROUPS * (tid >> 7); c < n_cols; c += TCE_GROUPS * (GEMM_THREADS / RB_ROWS)) {
     float v = 0.f;
     if (n >= 0) {
-      const float* src = q.part + (size_t)c * p.N + n;
+      const float* src = part + (size_t)c * p.N + n;
       v = __ldcg(src);
       for (int s0 = 1; s0 < q.n_split; s0 += 8) {  // eight loads in flight, added in split order
         float t[8];

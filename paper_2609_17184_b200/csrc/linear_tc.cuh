@@ -33,6 +33,10 @@ struct LinearTcParams {
   int err_code;
   int x3d;             // 0: x planes stacked [3][MP][K], one box; 1: the decode pass's layout [column][3][x_ld], a
                        // three-dimensional map (k, plane, column) and one box per plane
+  int row0;            // x3d: first column of the map this launch carries; blockIdx.z adds group_cols to it and
+  int group_cols;      //      group_stride floats to `out` (passes wider than one MMA's columns: one grid plane per
+  long long group_stride;  //  group of columns)
+  const int* n_live;   // x3d: number of live columns of the pass (may be null); a group beyond it has nothing to do
 };
 
 __device__ __forceinline__ unsigned tc_smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -126,6 +130,11 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   }
   __syncthreads();
   pdl_launch_dependents();
+  const int row0 = p.row0 + (int)blockIdx.z * p.group_cols;
+  if (p.n_live && *p.n_live <= row0) {  // (final before the pass starts; uniform over the CTA) this group of columns is empty
+    pdl_wait();  // a kernel that ended before its predecessor would release its own dependents too early
+    return;
+  }
   // The weights are constants, so the first ring-full of weight tiles is requested ahead of the predecessor's
   // completion - and while warp 0 still allocates the tensor memory; the activation tiles (which the predecessor may
   // still be writing) follow after the dependency wait, on the same barriers.
@@ -151,7 +160,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   auto load_x = [&](unsigned b, unsigned bar, int k) {  // the three planes of the activations, plane pl at b + pl * MP * 128
     if (p.x3d) {
 #pragma unroll
-      for (int pl = 0; pl < 3; ++pl) tc_tma_load_3d(b + pl * p.MP * TC_BK * 2, &map_x, bar, k, pl, 0);
+      for (int pl = 0; pl < 3; ++pl) tc_tma_load_3d(b + pl * p.MP * TC_BK * 2, &map_x, bar, k, pl, row0);
     } else {
       tc_tma_load_2d(b, &map_x, bar, k, 0);
     }
@@ -197,7 +206,7 @@ __global__ void __launch_bounds__(TC_THREADS) linear_tc_kernel(const __grid_cons
   if (have) have = tc_mbar_wait(tc_smem_u32(&s_done), 0);
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const int n = n0 + warp * 32 + lane;  // this thread's weight row = its TMEM lane
-  float* out = p.out + (size_t)blockIdx.y * p.M * p.N;
+  float* out = p.out + (size_t)blockIdx.z * p.group_stride + (size_t)blockIdx.y * p.M * p.N;
   if (n_kb <= 0) {
     for (int m = 0; m < p.M; ++m)
       if (n < p.N) out[(size_t)m * p.N + n] = 0.f;

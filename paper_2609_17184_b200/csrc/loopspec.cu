@@ -5,6 +5,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstdarg>
+#include <cstddef>
 #include <cstdio>
 #include <cstring>
 #include <string>
@@ -332,7 +333,8 @@ Layout make_layout(const loopspec_model* m, const loopspec_sched* s, const Deriv
     if (tc_prefill_shapes_ok(m)) {
       const int Ns[5] = {d.Hq + 2 * d.Hkv, m->hidden, 2 * m->ffn, m->hidden, m->hidden};
       const int Ks[5] = {m->hidden, d.Hq, m->hidden, m->ffn, 2 * m->hidden};
-      const int cols = std::max(tc_pf_cols(d.max_rows_pf), tc_pf_cols(std::min(d.max_rows_dec, (int)GROUP_ROWS)));
+      const int groups = (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;  // decode passes: one slice per group of 64 columns
+      const size_t cols = std::max((size_t)tc_pf_cols(d.max_rows_pf), (size_t)groups * tc_pf_cols(std::min(d.max_rows_dec, (int)GROUP_ROWS)));
       for (int i = 0; i < (d.raven ? 5 : 4); ++i) need = std::max(need, (size_t)tc_pf_plan(Ns[i], Ks[i]).n_split * cols * Ns[i] * 4);
     }
     L.tcpart = take(need);
@@ -660,27 +662,32 @@ cudaError_t launch_prep(loopspec_ctx* c, const RowTable* tab, int first_layer = 
 }
 
 
+int col_groups(loopspec_ctx* c, const RowTable* tab);
 // one layer GEMM of a prefill pass on the tcgen05 kernel: raw k-split sums, then the fused epilogue
 template <int EPI>
-cudaError_t launch_tc_epi(const TcEpiParams& q, cudaStream_t st, bool pdl) {
-  return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
+cudaError_t launch_tc_epi(const TcEpiParams& q, int groups, cudaStream_t st, bool pdl) {
+  return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS, groups), dim3(GEMM_THREADS), 0, st, q, pdl);
 }
 cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab, int cfg_i) {
   const loopspec_ctx::TcCfg& tc = c->tc[cfg_i];
   const int pi = which == G_ADAPT ? 4 : which;
   const TcPfPlan& t = c->tc_plan[pi];
   TcEpiParams q;
+  // one grid plane per group of 64 token columns (a plane whose group holds no row returns at once)
+  const int groups = cfg_i == 1 ? col_groups(c, tab) : 1;
   q.g = gemm_params(c, which, layer, tab);
-  q.g.cluster_size = TCE_GROUPS, q.g.recv_ranks = 1;
+  q.g.cluster_size = TCE_GROUPS, q.g.recv_ranks = 1, q.Hq = c->d.Hq;
   q.part = c->at<float>(c->L.tcpart), q.n_split = t.n_split, q.cols_ld = tc.cols;
   LinearTcParams p;
   memset(&p, 0, sizeof p);
   p.out = c->at<float>(c->L.tcpart);
   p.M = tc.cols, p.MP = tc.cols, p.N = q.g.N, p.K = q.g.K, p.kb_per_split = t.kb_per_split, p.stages = tc.stages;
   p.err = const_cast<int*>(c->host_flags_dev + HF_ERROR), p.err_code = 5, p.x3d = 1;
+  p.row0 = 0, p.group_cols = GROUP_ROWS, p.group_stride = (long long)t.n_split * tc.cols * q.g.N;
+  p.n_live = reinterpret_cast<const int*>(reinterpret_cast<const char*>(tab) + offsetof(RowTable, n_rows));
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3(t.n_tiles, t.n_split), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = tc.smem, cfg.stream = c->stream;
+  cfg.gridDim = dim3(t.n_tiles, t.n_split, groups), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = tc.smem, cfg.stream = c->stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -690,9 +697,9 @@ cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable
   cudaError_t e = cudaLaunchKernelEx(&cfg, linear_tc_kernel, wm, tc.xmaps[xi], p);
   if (e != cudaSuccess) return e;
   switch (which) {
-    case G_QKV: return launch_tc_epi<EPI_QKV>(q, c->stream, c->use_pdl);
-    case G_GU: return launch_tc_epi<EPI_SWIGLU>(q, c->stream, c->use_pdl);
-    default: return launch_tc_epi<EPI_RESID>(q, c->stream, c->use_pdl);
+    case G_QKV: return launch_tc_epi<EPI_QKV>(q, groups, c->stream, c->use_pdl);
+    case G_GU: return launch_tc_epi<EPI_SWIGLU>(q, groups, c->stream, c->use_pdl);
+    default: return launch_tc_epi<EPI_RESID>(q, groups, c->stream, c->use_pdl);
   }
 }
 
@@ -790,7 +797,7 @@ cudaError_t launch_stack(loopspec_ctx* c, const RowTable* tab, int ng, int l0, i
   const int groups = col_groups(c, tab);
   // a GEMM of the pass: one launch per group of token columns (one group unless a decode pass can carry more than 64 rows)
   auto gemm = [&](int which, int l, int tl_id) -> cudaError_t {
-    if (tc >= 0) return launch_tc_gemm(c, which, l, tab, tc);
+    if (tc >= 0) return launch_tc_gemm(c, which, l, tab, tc);  // (all groups of token columns in one pair of launches)
     for (int g = 0; g < groups; ++g) {
       GemmParams gp = gemm_params(c, which, l, tab, g * GROUP_ROWS);
       gp.tl = tune_timeline(c), gp.tl_id = tl_id;
@@ -1194,8 +1201,8 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     for (int i = 0; i < 5; ++i) c->tc_plan[i] = tc_pf_plan(Ns[i], Ks[i]);
     const size_t x_off[4] = {c->L.xplanes, c->L.aplanes, c->L.splanes, c->L.cplanes};
     const int x_k[4] = {m->hidden, dd.Hq, m->ffn, 2 * m->hidden};
-    const bool want[2] = {!s->prefill_skinny, c->ng_dec > 1 && dd.max_rows_dec <= GROUP_ROWS};
-    const int rows[2] = {dd.max_rows_pf, dd.max_rows_dec};
+    const bool want[2] = {!s->prefill_skinny, c->ng_dec > 1};
+    const int rows[2] = {dd.max_rows_pf, std::min(dd.max_rows_dec, (int)GROUP_ROWS)};  // (wider decode passes: groups of 64 columns)
     size_t smem_max = 0;
     for (int k = 0; k < 2 && ok; ++k) {
       if (!want[k]) continue;
@@ -1600,8 +1607,9 @@ int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
   if (!c || !out) return LOOPSPEC_EINVAL;
   const Derived& d = c->d;
   // launches per GEMM: one per group of 64 token columns, or the tcgen05 kernel and its epilogue
-  const int g = c->tc[1].on ? 2 : (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;
-  const int per_block = 1 + 4 * g, lm = c->dg ? 1 : (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;  // attention + four GEMMs
+  const int groups = (d.max_rows_dec + GROUP_ROWS - 1) / GROUP_ROWS;
+  const int g = c->tc[1].on ? 2 : groups;
+  const int per_block = 1 + 4 * g, lm = c->dg ? 1 : groups;  // attention + four GEMMs
   int n = 1 + c->m.n_recurrent * per_block + lm + 3;               // preparation, blocks, lm_head, selection, control, KV commit
   if (d.raven)  // prelude pass (preparation + blocks), concatenation + adapter instead of the preparation, coda pass
     n = (d.n_pre ? 1 + per_block * d.n_pre : 0) + 1 + g + per_block * c->m.n_recurrent + (d.n_coda ? 1 + per_block * d.n_coda : 0) + lm + 3;
