@@ -40,7 +40,7 @@ struct GemmPlan {
 // Cluster size = how many CTAs split K for one block of 128 output rows.  Enough CTAs to fill the resident
 // slots (two per SM), a k-range short enough that a decode pass keeps its activations staged once, and whole
 // rounds of row blocks per cluster so that every CTA streams the same number of bytes.
-GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1) {
+GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1, int cs_cap = 8) {
   GemmPlan g;
   g.n_rb = n_rb;
   g.kpr = (K + 31) / 32;
@@ -51,7 +51,7 @@ GemmPlan plan_gemm(int n_rb, int K, int slots, bool pow2_only, int kh = 1) {
   // become resident (and prefetch) early  [measured: O projection, 8 -> 4 CTAs per cluster]
   cs = std::min(cs, std::max(1, g.kpr / (8 * kh)));
   cs = std::max(cs, cs_min);
-  cs = std::min(std::min(cs, 8), g.kpr);
+  cs = std::min(std::min(cs, cs_cap), g.kpr);
   auto pow2_at_least = [&](int v) {
     int q = 1;
     while (q < v) q <<= 1;
@@ -1124,14 +1124,18 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
                         m->hidden / resid_rows};
   const int Ks[6] = {m->hidden, d.Hq, m->hidden, m->ffn, m->hidden, 2 * m->hidden};
   int slots = n_sm * kCtasPerSm;
-  for (int i = 0; i < 6; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
+  // Passes of up to 8 rows may split K over up to 11 CTAs (clusters beyond 8 are opt-in; a rank's slot of the receive
+  // buffer holds one column then): the down projection's 176 k-blocks over 11 ranks instead of 8 [measured: pass 1.122 ->
+  // 1.099 ms; 12 ranks 1.110 ms, 16 ranks 1.21 ms - they no longer fit at once]
+  const int cs_cap = c->ng_dec == 1 ? 11 : 8;
+  for (int i = 0; i < 6; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false, 1, cs_cap);
   if (kTune) {  // tuning aid: cluster size of GEMM i from LOOPSPEC_CS_i
     for (int i = 0; i < 6; ++i) {
       char name[32];
       snprintf(name, sizeof name, "LOOPSPEC_CS_%d", i);
       if (const char* v = getenv(name)) {
         GemmPlan& g = c->plan[i];
-        g.cs = std::max(1, std::min(8, atoi(v)));
+        g.cs = std::max(1, std::min(16, atoi(v)));
         const int max_clusters = std::max(1, slots / g.cs), rounds = (g.n_rb + max_clusters - 1) / max_clusters;
         g.n_clusters = (g.n_rb + rounds - 1) / rounds, g.grid = g.n_clusters * g.cs;
       }
@@ -1172,6 +1176,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     delete c;
     return LOOPSPEC_ECUDA;
   }
+  for (int epi = 0; epi < 5; ++epi)  // clusters of more than 8 CTAs (the O and down projections' k-split) are opt-in
+    if (cudaFuncSetAttribute(gemm_fn(m->weight_dtype, c->ng_dec, epi), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+      (void)cudaGetLastError();
   for (int ng : {c->ng_dec, c->ng_pf})
     if (gemm_smem(m->weight_dtype, ng) > 48 * 1024)
       for (int epi = 0; epi < 5; ++epi)
@@ -1186,7 +1193,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // cluster sizes that are not powers of two are used only if the device can co-schedule them
   for (int i = 0; i < 6; ++i) {
     GemmPlan& g = c->plan[i];
-    if ((g.cs & (g.cs - 1)) == 0) continue;
+    if ((g.cs & (g.cs - 1)) == 0 && g.cs <= 8) continue;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(g.grid), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = gemm_smem(m->weight_dtype, c->ng_dec);
@@ -1196,9 +1203,9 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
     cfg.attrs = at, cfg.numAttrs = 1;
     int n_active = 0;
     cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
-    if (e != cudaSuccess || n_active < 1) {
+    if (e != cudaSuccess || n_active < 1 || (g.cs > 8 && n_active < g.n_clusters)) {
       (void)cudaGetLastError();
-      g = plan_gemm(n_rbs[i], Ks[i], slots, true);
+      g = g.cs > 8 ? plan_gemm(n_rbs[i], Ks[i], slots, false) : plan_gemm(n_rbs[i], Ks[i], slots, true);
     }
   }
   // prefill passes on the tcgen05 kernel (shapes it does not take, and fp32 weights: the kernels of the decode passes);
