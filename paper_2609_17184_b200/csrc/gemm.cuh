@@ -771,15 +771,19 @@ struct TcEpiParams {
   int Hq;              // query width (rows of the query buffer)
 };
 
-template <int EPI>
+template <int EPI, bool GROUPED>
 __global__ void __launch_bounds__(GEMM_THREADS) tc_epilogue_kernel(const __grid_constant__ TcEpiParams q) {
   __shared__ float s_recv[(TCE_MAX_COLS / TCE_GROUPS) * RB_ROWS];
   __shared__ float s_colbuf[2 * RB_ROWS];
   __shared__ float s_rstd[TCE_MAX_COLS];
   __shared__ int s_ct[CT_FIELDS * TCE_MAX_COLS];
-  // blockIdx.z = group of TCE_MAX_COLS token columns: its slices of the per-column buffers
-  GemmParams p = q.g;
-  {
+  // GROUPED: blockIdx.z = group of TCE_MAX_COLS token columns, with its slices of the per-column buffers (a private copy
+  // of the parameters; passes of up to TCE_MAX_COLS rows read them where they are)
+  GemmParams p_grp;
+  if (GROUPED) p_grp = q.g;
+  const GemmParams& p = GROUPED ? p_grp : q.g;
+  if (GROUPED) {
+    GemmParams& p = p_grp;
     const int col0 = (int)blockIdx.z * TCE_MAX_COLS;
     p.col0 = col0;
     if (p.out_planes) p.out_planes += (size_t)col0 * 3 * p.planes_ld;

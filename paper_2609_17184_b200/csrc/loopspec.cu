@@ -391,7 +391,10 @@ struct loopspec_ctx {
   const void* adapter = nullptr;    // Raven-style layout: [H][2H]
   int n_sm = 148;
   int ng_dec = 1, ng_pf = 1;
-  GemmPlan plan[6];
+  GemmPlan plan[6];      // mma.sync kernels of the decode passes
+  GemmPlan plan_pf[6];   // ... of prefill passes that run on them (clusters of up to 8: the receive buffer of a wide pass
+                         // holds several columns per rank)
+  const GemmPlan* cur_plan = plan;  // the set the launch helpers read (loopspec_prefill switches it for its duration)
   // prefill on the tcgen05 kernel: tensor maps of the row-major weights (4 per layer) and of the three plane buffers
   // ... and the decode passes of contexts whose passes carry 9 to 64 rows (batches, deep recurrences), where the
   // mma.sync kernels are bound by their three-plane arithmetic rather than by the weight stream
@@ -581,7 +584,7 @@ GemmParams gemm_params(loopspec_ctx* c, int which, int layer, const RowTable* ta
   const Derived& d = c->d;
   GemmParams p;
   memset(&p, 0, sizeof p);
-  const GemmPlan& g = c->plan[which];
+  const GemmPlan& g = c->cur_plan[which];
   p.n_rb = g.n_rb, p.kb_per_rb = g.kpr, p.cluster_size = g.cs, p.n_clusters = g.n_clusters;
   p.hid = c->at<float>(c->L.hid), p.H = m.hidden, p.eps = m.rms_eps, p.tab = tab;
   p.err = c->host_flags_dev + HF_ERROR;
@@ -669,7 +672,8 @@ int col_groups(loopspec_ctx* c, const RowTable* tab);
 // one layer GEMM of a prefill pass on the tcgen05 kernel: raw k-split sums, then the fused epilogue
 template <int EPI>
 cudaError_t launch_tc_epi(const TcEpiParams& q, int groups, cudaStream_t st, bool pdl) {
-  return launch_k(tc_epilogue_kernel<EPI>, dim3(q.g.n_rb, TCE_GROUPS, groups), dim3(GEMM_THREADS), 0, st, q, pdl);
+  if (groups > 1) return launch_k(tc_epilogue_kernel<EPI, true>, dim3(q.g.n_rb, TCE_GROUPS, groups), dim3(GEMM_THREADS), 0, st, q, pdl);
+  return launch_k(tc_epilogue_kernel<EPI, false>, dim3(q.g.n_rb, TCE_GROUPS), dim3(GEMM_THREADS), 0, st, q, pdl);
 }
 cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable* tab, int cfg_i) {
   const loopspec_ctx::TcCfg& tc = c->tc[cfg_i];
@@ -687,7 +691,8 @@ cudaError_t launch_tc_gemm(loopspec_ctx* c, int which, int layer, const RowTable
   p.M = tc.cols, p.MP = tc.cols, p.N = q.g.N, p.K = q.g.K, p.kb_per_split = t.kb_per_split, p.stages = tc.stages;
   p.err = const_cast<int*>(c->host_flags_dev + HF_ERROR), p.err_code = 5, p.x3d = 1;
   p.row0 = 0, p.group_cols = GROUP_ROWS, p.group_stride = (long long)t.n_split * tc.cols * q.g.N;
-  p.n_live = reinterpret_cast<const int*>(reinterpret_cast<const char*>(tab) + offsetof(RowTable, n_rows));
+  // (only a pass of several groups can have an empty one worth skipping)
+  p.n_live = groups > 1 ? reinterpret_cast<const int*>(reinterpret_cast<const char*>(tab) + offsetof(RowTable, n_rows)) : nullptr;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3(t.n_tiles, t.n_split, groups), cfg.blockDim = dim3(TC_THREADS), cfg.dynamicSmemBytes = tc.smem, cfg.stream = c->stream;
@@ -1129,6 +1134,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // 1.099 ms; 12 ranks 1.110 ms, 16 ranks 1.21 ms - they no longer fit at once]
   const int cs_cap = c->ng_dec == 1 ? 11 : 8;
   for (int i = 0; i < 6; ++i) c->plan[i] = plan_gemm(n_rbs[i], Ks[i], slots, false, 1, cs_cap);
+  for (int i = 0; i < 6; ++i) c->plan_pf[i] = plan_gemm(n_rbs[i], Ks[i], slots, false);
   if (kTune) {  // tuning aid: cluster size of GEMM i from LOOPSPEC_CS_i
     for (int i = 0; i < 6; ++i) {
       char name[32];
@@ -1191,21 +1197,23 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   if (unsigned long long* tl = tune_timeline(c)) cudaMemcpyToSymbol(g_tune_tl, &tl, sizeof tl);
 #endif
   // cluster sizes that are not powers of two are used only if the device can co-schedule them
-  for (int i = 0; i < 6; ++i) {
-    GemmPlan& g = c->plan[i];
+  for (int i = 0; i < 12; ++i) {
+    const bool pf = i >= 6;
+    GemmPlan& g = pf ? c->plan_pf[i - 6] : c->plan[i];
     if ((g.cs & (g.cs - 1)) == 0 && g.cs <= 8) continue;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(g.grid), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = gemm_smem(m->weight_dtype, c->ng_dec);
+    const int ng = pf ? c->ng_pf : c->ng_dec;
+    cfg.gridDim = dim3(g.grid), cfg.blockDim = dim3(GEMM_THREADS), cfg.dynamicSmemBytes = gemm_smem(m->weight_dtype, ng);
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = g.cs, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
     cfg.attrs = at, cfg.numAttrs = 1;
     int n_active = 0;
-    cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, c->ng_dec, kEpiOf[i]), &cfg);
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n_active, gemm_fn(m->weight_dtype, ng, kEpiOf[i % 6]), &cfg);
     if (e != cudaSuccess || n_active < 1 || (g.cs > 8 && n_active < g.n_clusters)) {
       (void)cudaGetLastError();
-      g = g.cs > 8 ? plan_gemm(n_rbs[i], Ks[i], slots, false) : plan_gemm(n_rbs[i], Ks[i], slots, true);
+      g = g.cs > 8 ? plan_gemm(n_rbs[i % 6], Ks[i % 6], slots, false) : plan_gemm(n_rbs[i % 6], Ks[i % 6], slots, true);
     }
   }
   // prefill passes on the tcgen05 kernel (shapes it does not take, and fp32 weights: the kernels of the decode passes);
@@ -1354,6 +1362,15 @@ const char* loopspec_last_error(loopspec_ctx* c) { return c ? c->err.c_str() : "
 
 int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, int32_t n, int32_t* first_token) {
   Range nvtx_range("loopspec_prefill");
+  struct PlanGuard {  // prefill passes on the mma.sync kernels use their own cluster plans
+    loopspec_ctx* c;
+    explicit PlanGuard(loopspec_ctx* c_) : c(c_) {
+      if (c) c->cur_plan = c->plan_pf;
+    }
+    ~PlanGuard() {
+      if (c) c->cur_plan = c->plan;
+    }
+  } plan_guard(c);
   if (!c) return LOOPSPEC_EINVAL;
   if (c->sticky) return LOOPSPEC_ECUDA;
   if (seq < 0 || seq >= c->d.S || !prompt_ids || n < 1) return fail(c, LOOPSPEC_EINVAL, "bad prefill arguments");
