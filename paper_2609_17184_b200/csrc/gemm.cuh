@@ -763,7 +763,10 @@ __global__ void __launch_bounds__(256) prep_planes_kernel(const __grid_constant_
 // splits in split order into the receive-buffer layout of a one-rank cluster and runs the same epilogue code as the
 // mma.sync kernels (1/rms, then RoPE + KV write / residual + sum of squares + planes / SwiGLU + planes).
 constexpr int TCE_MAX_COLS = 64;
-constexpr int TCE_GROUPS = 16;   // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
+#ifndef LS_TCE_GROUPS
+#define LS_TCE_GROUPS 32  // measured on the 512-token prefill of the 1.4B shape: 8 / 16 / 32 / 64 groups -> 80.3 / 70.9 / 67.9 / 71.7 ms
+#endif
+constexpr int TCE_GROUPS = LS_TCE_GROUPS;   // column groups = CTAs per row block (the epilogue code sees a cluster of this size)
 struct TcEpiParams {
   GemmParams g;        // cluster_size = TCE_GROUPS; the per-column buffers start at the pass's first column
   const float* part;   // [group][n_split][cols_ld][N]

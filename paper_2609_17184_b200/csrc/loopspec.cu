@@ -179,7 +179,10 @@ TcPfPlan tc_pf_plan(int N, int K) {
   TcPfPlan t;
   t.n_tiles = (N + TC_BM - 1) / TC_BM;
   const int total_kb = K / TC_BK;
-  const int want = std::max(1, std::min(296 / t.n_tiles, total_kb / 4));
+#ifndef LS_TC_SLOTS
+#define LS_TC_SLOTS 296
+#endif
+  const int want = std::max(1, std::min(LS_TC_SLOTS / t.n_tiles, total_kb / 4));
   t.kb_per_split = (total_kb + want - 1) / want;
   t.n_split = (total_kb + t.kb_per_split - 1) / t.kb_per_split;
   return t;
