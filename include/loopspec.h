@@ -205,8 +205,8 @@ int loopspec_launches_per_step(loopspec_ctx*, int32_t* out);
  * context capacity): *gemm_path = 0 the mma.sync cluster kernels (passes of up to 8 rows, fp32 weights), 1 the
  * tcgen05 / TMA kernel + epilogue kernel (bf16 weights, passes of 9 or more rows, one pair of launches per group of 64
  * token columns);
- * *attention_path = 0 one work item per 64-position chunk (context capacity up to 2560), 1 the streaming kernel over
- * runs of chunks.  Either pointer may be null. */
+ * *attention_path = 0 one work item per 64-position chunk (context capacity up to 2560 positions; up to 512 when the
+ * context holds several sequences), 1 the streaming kernel over runs of chunks.  Either pointer may be null. */
 int loopspec_decode_paths(loopspec_ctx*, int32_t* gemm_path, int32_t* attention_path);
 
 /* Time `iters` back-to-back launches of one kernel of the pass in the decode launch configuration, cycling

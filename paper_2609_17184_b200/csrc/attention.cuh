@@ -273,8 +273,9 @@ __global__ void __launch_bounds__(ATT_THREADS, 4) attn_kernel(const __grid_const
   timeline_mark(p.tl, p.tl_id, true);
 }
 
-// The same attention for contexts of more than ATT_MAX_RUNS chunks: a work item is a run of consecutive chunks (a
-// function of the row's own context only), so that the per-item costs (row lookup, partial write, counter) are paid
+// The same attention for contexts whose rows can have more chunks than single-chunk items are cut for (more than
+// ATT_MAX_RUNS chunks; more than ATT_BATCH_SINGLE in contexts of several sequences): a work item is a run of consecutive
+// chunks (a function of the row's own context only), so that the per-item costs (row lookup, partial write, counter) are paid
 // once per run and a (row, kv head) never has more than ATT_MAX_RUNS partials.  This is the kernel of the KV-bound
 // regime, built to stream: every thread owns a ring of (key piece, value piece) slots in shared memory that it fills
 // with cp.async and reads back itself, so the K/V of the next rounds are in flight while the current one is used and
@@ -340,7 +341,7 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtsCfg<D, G>::MIN_CTAS)) attn_ru
     const int n_runs = tab->chunk_start[row + 1] - tab->chunk_start[row];
     const int n_canon = tab->n_canon[row];
     const int n_chunks = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK;
-    const int run_len = att_run_len(n_canon);
+    const int run_len = att_run_len(n_canon, tab->att_mode);
     const int chunk_lo = run * run_len, chunk_hi = min(n_chunks, chunk_lo + run_len);
     const int row_spec = tab->n_spec[row], row_safe = tab->n_safe[row];
 

@@ -22,16 +22,19 @@ constexpr int MAX_SEQS = 64;  // sequences a context can hold
 constexpr int MAX_SPEC = 16;  // speculative ancestors (incl. the row itself) a row can attend to: R/d1 levels
 constexpr int ATT_CHUNK = 64; // key positions per attention chunk (cut at fixed absolute positions)
 constexpr int ATT_MAX_RUNS = 40;  // attention work items per (row, kv head) at most (contexts up to 2560: one chunk each)
-constexpr int ATT_LONG_RUNS = 8;  // ... and for contexts of more than ATT_MAX_RUNS chunks
-// A work item covers a run of consecutive chunks: one chunk for contexts up to ATT_MAX_RUNS chunks, beyond that as
-// many as leave ATT_LONG_RUNS items (a function of the row's own context only, so a row's arithmetic does not depend
-// on what shares the pass).
-__host__ __device__ inline int att_run_len(int n_canon) {
+constexpr int ATT_LONG_RUNS = 8;  // ... and for longer contexts
+constexpr int ATT_BATCH_SINGLE = 8;  // contexts that hold several sequences: single-chunk items only up to 8 chunks
+// A work item covers a run of consecutive chunks.  mode 0 (a context of one sequence: few rows per pass, every chunk in
+// parallel matters): one chunk for contexts up to ATT_MAX_RUNS chunks, beyond that as many as leave ATT_LONG_RUNS items.
+// mode 1 (contexts of several sequences: many rows per pass, the stream matters): one chunk up to ATT_BATCH_SINGLE
+// chunks, beyond that as many as leave ATT_LONG_RUNS items.  Either way a function of the row's own context only, so a
+// row's arithmetic does not depend on what shares the pass.
+__host__ __device__ inline int att_run_len(int n_canon, int mode) {
   const int nc = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK;
-  return nc <= ATT_MAX_RUNS ? 1 : (nc + ATT_LONG_RUNS - 1) / ATT_LONG_RUNS;
+  return nc <= (mode ? ATT_BATCH_SINGLE : ATT_MAX_RUNS) ? 1 : (nc + ATT_LONG_RUNS - 1) / ATT_LONG_RUNS;
 }
-__host__ __device__ inline int att_items(int n_canon) {
-  const int nc = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK, rl = att_run_len(n_canon);
+__host__ __device__ inline int att_items(int n_canon, int mode) {
+  const int nc = (n_canon + ATT_CHUNK - 1) / ATT_CHUNK, rl = att_run_len(n_canon, mode);
   return (nc + rl - 1) / rl;
 }
 
@@ -43,7 +46,7 @@ struct RowTable {
   int n_rows;
   int n_readout;             // rows whose new depth is d1, d2 or R
   int attn_items;            // sum over rows of attention work items (runs of chunks)
-  int n_layers_done;         // unused, keeps the header 16 bytes
+  int att_mode;              // how attention work items are cut (see att_run_len)
   int seq[MAX_ROWS];         // sequence of the row
   int r[MAX_ROWS];           // recurrence the row is advanced TO (1..R): KV plane it writes and reads
   int pos[MAX_ROWS];         // position of the row's token (rotary index)

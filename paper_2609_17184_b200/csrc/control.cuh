@@ -14,6 +14,7 @@ enum { HF_ERROR = 0, HF_MIN_DEC = 1, HF_N_ROWS = 2, HF_NEED_VERIFY = 3, HF_FIRST
 enum { ERR_NODES = 1, ERR_CTX = 2, ERR_SPEC = 3, ERR_WAIT = 4 /* bounded wait, decode GEMM */, ERR_WAIT_PF = 5 /* prefill GEMM, grid barrier */ };
 
 struct ControlParams {
+  int att_mode;     // how attention work items are cut (att_run_len)
   RowTable* tab;
   NodeTable nodes;
   SeqState seqs;
@@ -61,11 +62,11 @@ __device__ void derive_raven_tables(const RowTable& t, RowTable* pre, RowTable* 
       copy_row(pre, np, i);
       pre->r[np] = 1, pre->hid_idx[np] = t.hid_idx[i], pre->src_hid[np] = -1, pre->readout[np] = RO_NONE;
       pre->chunk_start[np] = items;
-      items += att_items(t.n_canon[i]);
+      items += att_items(t.n_canon[i], t.att_mode);
       ++np;
     }
     pre->chunk_start[np] = items;
-    pre->n_rows = np, pre->n_readout = 0, pre->attn_items = items, pre->n_layers_done = 0;
+    pre->n_rows = np, pre->n_readout = 0, pre->attn_items = items, pre->att_mode = t.att_mode;
   }
   int nc = 0;
   items = 0;
@@ -77,11 +78,11 @@ __device__ void derive_raven_tables(const RowTable& t, RowTable* pre, RowTable* 
     coda->hid_idx[nc] = hid_coda_base + nc, coda->src_hid[nc] = t.hid_idx[i];
     coda->readout[nc] = ro, coda->ro_rows[nc] = nc;
     coda->chunk_start[nc] = items;
-    items += att_items(t.n_canon[i]);
+    items += att_items(t.n_canon[i], t.att_mode);
     ++nc;
   }
   coda->chunk_start[nc] = items;
-  coda->n_rows = nc, coda->n_readout = nc, coda->attn_items = items, coda->n_layers_done = 0;
+  coda->n_rows = nc, coda->n_readout = nc, coda->attn_items = items, coda->att_mode = t.att_mode;
 }
 
 struct NodeSmem {
@@ -171,11 +172,11 @@ __device__ void build_rows(RowTable& t, const NodeSmem& nd, const int* root, con
       t.readout[i] = ro, t.logit_idx[i] = li;
       if (ro) t.ro_rows[n_ro++] = i;
       t.chunk_start[i] = items;
-      items += att_items(t.n_canon[i]);
+      items += att_items(t.n_canon[i], p.att_mode);
     }
   }
   t.chunk_start[n_rows] = items;
-  t.n_rows = n_rows, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
+  t.n_rows = n_rows, t.n_readout = n_ro, t.attn_items = items, t.att_mode = p.att_mode;
 }
 
 // dynamic shared memory of control_kernel: the branch table, the row table and the per-row selection results
@@ -340,6 +341,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) control_kernel(const __grid_cons
 
 // ---- vanilla decoding (Fig. 1a): one row per sequence, R passes per token ---------------------------
 struct VanillaParams {
+  int att_mode;     // how attention work items are cut (att_run_len)
   RowTable* tabs;   // [R] one table per recurrence
   NodeTable nodes;
   SeqState seqs;
@@ -405,10 +407,10 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
         t.n_safe[i] = pos;
         t.hid_idx[i] = gn, t.node[i] = gn, t.readout[i] = (r == p.R) ? RO_TARGET : RO_NONE, t.src_hid[i] = -1;
         t.logit_idx[i] = p.p_logit_base + s, t.ro_rows[i] = i, t.chunk_start[i] = items;
-        items += att_items(pos + 1);
+        items += att_items(pos + 1, p.att_mode);
       }
       t.chunk_start[n] = items;
-      t.n_rows = n, t.n_readout = (r == p.R) ? n : 0, t.attn_items = items, t.n_layers_done = 0;
+      t.n_rows = n, t.n_readout = (r == p.R) ? n : 0, t.attn_items = items, t.att_mode = p.att_mode;
     }
     if (p.tab_coda) {  // the prelude pass of a vanilla token is the first table itself (every row enters recurrence 1)
       derive_raven_tables(p.tabs[p.R - 1], nullptr, p.tab_coda, p.hid_coda_base, p.n_classes);
@@ -420,6 +422,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) vanilla_control_kernel(const __g
 
 // ---- prefill (Algorithm 1, lines before the main loop): rows = consecutive prompt positions ---------
 struct PrefillParams {
+  int att_mode;       // how attention work items are cut (att_run_len)
   RowTable* tab;
   const int* prompt;  // device ids of the sequence
   int seq, p0, count, r, R, n_prompt;
@@ -449,11 +452,11 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
       t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;
       if (last) t.ro_rows[n_ro++] = i;
       t.chunk_start[i] = items;
-      items += att_items(pos + 1);
+      items += att_items(pos + 1, p.att_mode);
       s_emb[i][0] = p.hid_base + i, s_emb[i][1] = p.prompt[pos];
     }
     t.chunk_start[p.count] = items;
-    t.n_rows = p.count, t.n_readout = n_ro, t.attn_items = items, t.n_layers_done = 0;
+    t.n_rows = p.count, t.n_readout = n_ro, t.attn_items = items, t.att_mode = p.att_mode;
     if (p.tab_coda && p.coda_class > 0) {  // the same rows, on copies of their states, writing this depth's coda cache
       RowTable& c = *p.tab_coda;
       int nr = 0;
@@ -464,7 +467,7 @@ __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const Prefi
         if (t.readout[i]) c.ro_rows[nr++] = i;
       }
       c.chunk_start[p.count] = items;
-      c.n_rows = p.count, c.n_readout = nr, c.attn_items = items, c.n_layers_done = 0;
+      c.n_rows = p.count, c.n_readout = nr, c.attn_items = items, c.att_mode = p.att_mode;
     }
   }
   __syncthreads();

@@ -199,6 +199,8 @@ struct Layout {  // byte offsets into the workspace
 };
 
 struct Derived {
+  int att_mode;   // attention work items: 0 one sequence per context, 1 several (see att_run_len)
+  int att_runs;   // the context's rows can have items of several chunks: the streaming attention kernel runs
   int S, NB, B, max_rows_dec, max_rows_pf, max_rows, slots, ids_cap, n_hid, n_logit_vecs, p_logit_base, n_sq, sq_stride, max_chunks,
       trace_cap, Hq, Hkv, d1, d2;
   // Raven-style layout (P and C hold transformer blocks): all layers in one list - prelude, recurrent, coda
@@ -297,6 +299,8 @@ bool resolve_sched(const loopspec_model* m, const loopspec_sched* s, Derived* d,
   d->n_sq = m->hidden / 128;  // row blocks of the residual GEMMs = partial sums of squares per row
   d->sq_stride = std::max(d->n_sq, 64);  // room for one partial per cluster of the persistent pass kernel
   d->max_chunks = (s->max_ctx + ATT_CHUNK - 1) / ATT_CHUNK;
+  d->att_mode = d->S >= 2 ? 1 : 0;
+  d->att_runs = d->max_chunks > (d->att_mode ? ATT_BATCH_SINGLE : ATT_MAX_RUNS) ? 1 : 0;
   d->trace_cap = m->R * s->max_ctx + 64;  // a token can take R passes (restart)
   d->Hq = m->n_q_heads * m->head_dim;
   d->Hkv = m->n_kv_heads * m->head_dim;
@@ -550,7 +554,7 @@ cudaError_t launch_gemm(int wdt, int ng, int epi, const GemmParams& p, cudaStrea
 }
 
 using AttnFn = void (*)(const AttnParams);
-AttnFn attn_fn(int d, int G, bool runs) {  // runs: contexts longer than ATT_MAX_RUNS chunks are possible
+AttnFn attn_fn(int d, int G, bool runs) {  // runs: rows of this context can have work items of several chunks
   if (runs) {
     if (d == 128) return G == 1 ? attn_runs_kernel<128, 1> : attn_runs_kernel<128, 4>;
     return G == 1 ? attn_runs_kernel<64, 1> : attn_runs_kernel<64, 4>;
@@ -793,7 +797,7 @@ cudaError_t launch_attention(loopspec_ctx* c, const RowTable* tab, int l, unsign
     if (e) return e;
     return launch_k(attn_prefill_fold_kernel<64>, fold_grid, dim3(16), 0, c->stream, a, c->use_pdl);
   }
-  const bool runs = d.max_chunks > ATT_MAX_RUNS;
+  const bool runs = d.att_runs != 0;
   return launch_k(attn_fn(m.head_dim, G, runs), dim3(attn_grid(c->n_sm, G, runs)), dim3(ATT_THREADS), attn_smem(m.head_dim, G, runs), c->stream, a,
                   c->use_pdl);
 }
@@ -901,6 +905,7 @@ cudaError_t launch_select(loopspec_ctx* c, const RowTable* tab, int kinds_mask) 
 ControlParams control_params(loopspec_ctx* c, int phases) {
   ControlParams p;
   memset(&p, 0, sizeof p);
+  p.att_mode = c->d.att_mode;
   p.tab = c->at<RowTable>(c->L.tab_dec), p.nodes = c->nodes(), p.seqs = c->seqs(), p.ctr = c->at<Counters>(c->L.ctr);
   p.S = c->d.S, p.NB = c->d.NB, p.R = c->m.R, p.d1 = c->d.d1, p.d2 = c->d.d2, p.ctx_cap = c->s.max_ctx;
   p.sel_tok = c->at<int>(c->L.sel_tok), p.sel_aux = c->at<int>(c->L.sel_aux);
@@ -956,6 +961,7 @@ cudaError_t launch_step(loopspec_ctx* c, int kinds_mask, int phases, bool kv_com
 VanillaParams vanilla_params(loopspec_ctx* c, int commit) {
   VanillaParams v;
   memset(&v, 0, sizeof v);
+  v.att_mode = c->d.att_mode;
   v.tabs = c->at<RowTable>(c->L.tab_van), v.nodes = c->nodes(), v.seqs = c->seqs();
   v.S = c->d.S, v.NB = c->d.NB, v.R = c->m.R, v.sel_tok = c->at<int>(c->L.sel_tok), v.commit = commit;
   v.out_ids = c->at<int>(c->L.out_ids), v.ids_cap = c->d.ids_cap;
@@ -1153,7 +1159,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   // Every kernel of the chain asks for the same (largest) shared-memory carve-out: the GEMM CTAs need it, and an SM
   // whose partition was set by a small-shared-memory kernel would have to drain before it can host one.
   {
-    const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads, d.max_chunks > ATT_MAX_RUNS), (const void*)prep_planes_kernel,
+    const void* small_fns[] = {(const void*)attn_fn(m->head_dim, m->n_q_heads / m->n_kv_heads, d.att_runs != 0), (const void*)prep_planes_kernel,
                                (const void*)select_kernel, (const void*)control_kernel, (const void*)vanilla_control_kernel,
                                (const void*)kv_commit_kernel};
     for (const void* f : small_fns)
@@ -1162,7 +1168,7 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   }
   {
     const int G = m->n_q_heads / m->n_kv_heads;
-    const bool runs = d.max_chunks > ATT_MAX_RUNS;
+    const bool runs = d.att_runs != 0;
     if (runs && cudaFuncSetAttribute((const void*)attn_fn(m->head_dim, G, runs), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)attn_smem(m->head_dim, G, runs)) != cudaSuccess) {
       delete c;
@@ -1389,6 +1395,7 @@ int loopspec_prefill(loopspec_ctx* c, int32_t seq, const int32_t* prompt_ids, in
     int cnt = std::min(chunk, n - p0);
     for (int r = 1; r <= c->m.R; ++r) {
       PrefillParams pp;
+      pp.att_mode = c->d.att_mode;
       pp.tab = tab, pp.prompt = c->at<int>(c->L.prompt), pp.seq = seq, pp.p0 = p0, pp.count = cnt, pp.r = r, pp.R = c->m.R;
       pp.n_prompt = n, pp.hid_base = c->d.S * c->d.NB, pp.p_logit_base = c->d.p_logit_base;
       pp.hid = c->at<float>(c->L.hid), pp.H = c->m.hidden, pp.embed = c->embed, pp.weight_dtype = c->m.weight_dtype;
@@ -1662,7 +1669,7 @@ int loopspec_launches_per_step(loopspec_ctx* c, int32_t* out) {
 int loopspec_decode_paths(loopspec_ctx* c, int32_t* gemm_path, int32_t* attention_path) {
   if (!c) return LOOPSPEC_EINVAL;
   if (gemm_path) *gemm_path = c->tc[1].on ? 1 : 0;
-  if (attention_path) *attention_path = c->d.max_chunks > ATT_MAX_RUNS ? 1 : 0;
+  if (attention_path) *attention_path = c->d.att_runs != 0 ? 1 : 0;
   return LOOPSPEC_OK;
 }
 
@@ -1675,7 +1682,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
   // the pass buffers and to KV slot 0 of plane 1, which the next prefill overwrites)
   RowTable t;
   memset(&t, 0, sizeof t);
-  t.n_rows = rows, t.n_readout = rows;
+  t.n_rows = rows, t.n_readout = rows, t.att_mode = c->d.att_mode;
   for (int i = 0; i < rows; ++i) {
     t.r[i] = 1, t.hid_idx[i] = c->d.S * c->d.NB + i, t.ro_rows[i] = i, t.readout[i] = RO_TARGET, t.n_canon[i] = 1, t.n_safe[i] = 0;
     t.logit_idx[i] = c->d.p_logit_base, t.node[i] = -1, t.chunk_start[i] = i;
@@ -1689,7 +1696,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
     for (int i = 0; i < rows; ++i) {
       t.seq[i] = i % c->d.S, t.r[i] = 1 + (i / c->d.S) % c->m.R;
       t.n_canon[i] = ctx, t.n_safe[i] = ctx, t.n_spec[i] = 0, t.chunk_start[i] = items;
-      items += att_items(ctx);
+      items += att_items(ctx, c->d.att_mode);
     }
     t.chunk_start[rows] = items, t.attn_items = items;
   }
@@ -1702,7 +1709,7 @@ int loopspec_time_kernel(loopspec_ctx* c, int32_t which, int32_t rows, int32_t i
       const int pos = ctx - rows + i;
       t.seq[i] = 0, t.r[i] = 1, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_safe[i] = ctx - rows, t.n_spec[i] = 0;
       t.chunk_start[i] = items;
-      items += att_items(pos + 1);
+      items += att_items(pos + 1, c->d.att_mode);
     }
     t.chunk_start[rows] = items, t.attn_items = items;
   }

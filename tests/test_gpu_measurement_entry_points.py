@@ -11,10 +11,13 @@ pytestmark = pytest.mark.gpu
 
 def test_decode_paths_follow_the_row_and_context_capacity():
     """Passes of up to 8 rows: mma.sync cluster kernels; 9 to 64 rows of a bf16 model: the tcgen05 kernel + epilogue;
-    a context capacity beyond 2560 positions: the streaming attention kernel; fp32 weights never leave the CUDA cores."""
+    a context capacity beyond 2560 positions (512 when the context holds several sequences): the streaming attention kernel;
+    fp32 weights never leave the CUDA cores."""
     cases = [(dict(name="tiny_bf16", max_seqs=1, max_ctx=256), (0, 0)),
              (dict(name="tiny_bf16", max_seqs=4, max_ctx=256), (1, 0)),
              (dict(name="tiny_bf16", max_seqs=1, max_ctx=3000), (0, 1)),
+             (dict(name="tiny_bf16", max_seqs=4, max_ctx=1024), (1, 1)),
+             (dict(name="tiny_bf16", max_seqs=4, max_ctx=512), (1, 0)),
              (dict(name="tiny_raven", max_seqs=1, max_ctx=256), (1, 0)),
              (dict(name="tiny", max_seqs=4, max_ctx=256), (0, 0))]
     for kw, want in cases:

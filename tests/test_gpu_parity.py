@@ -385,6 +385,26 @@ def test_batch_of_sequences_equals_each_alone():
     ctx.close()
 
 
+@pytest.mark.parametrize("name,T", [("tiny_bf16", 0.9), ("tiny_gqa", 0.0)])
+def test_batch_of_mid_length_contexts_streams_runs_of_chunks(name, T):
+    """Several sequences with contexts of 9 to 17 attention chunks: in a context that holds more than one sequence the
+    attention work items are runs of chunks from 8 chunks on (the streaming kernel); each sequence must still decode exactly
+    as the oracle decodes it alone, whatever the other rows of the pass are."""
+    S, n = 3, 20
+    lens = [600, 830, 1050]
+    refs = [U.oracle_run(name, lens[s], n, 1, 2, T=T, seed=9, seq=s) for s in range(S)]
+    ctx = U.make_ctx(name, 1, 2, T=T, seed=9, max_seqs=S, max_ctx=1100, max_prefill_rows=64)
+    assert ctx.decode_paths()[1] == 1
+    for s in range(S):
+        assert ctx.prefill(refs[s]["prompt"], seq=s) == refs[s]["first"]
+    out = ctx.decode(n)
+    for s in range(S):
+        assert out[s].tolist() == refs[s]["tokens"], (s, U.min_margin(refs[s]["dec"]))
+        got = ctx.commits(s)
+        assert [(c["source"], c["gate_open"]) for c in got] == [(c["source"], c["gate_open"]) for c in refs[s]["dec"].commits]
+    ctx.close()
+
+
 def test_prefill_chunking_does_not_change_results():
     name = "tiny_bf16"
     ref = U.oracle_run(name, 37, 16, 1, 2)
