@@ -587,12 +587,14 @@ def test_grouped_query_attention(name, T):
     ctx.close()
 
 
-@pytest.mark.parametrize("name,T", [("tiny_bf16", 0.0), ("tiny_bf16", 1.0), ("tiny_gqa", 1.0), ("tiny_gqa_f32", 0.0)])
-def test_context_beyond_2560_uses_runs_of_attention_chunks(name, T):
+@pytest.mark.parametrize("name,T,skinny", [("tiny_bf16", 0.0, False), ("tiny_bf16", 1.0, False), ("tiny_gqa", 1.0, False),
+                                           ("tiny_gqa_f32", 0.0, False), ("tiny_bf16", 1.0, True), ("tiny_gqa", 0.0, True)])
+def test_context_beyond_2560_uses_runs_of_attention_chunks(name, T, skinny):
     """A 2700-token prompt: more than 40 chunks per row, so attention work items are runs of several chunks folded with
-    the running-softmax rescaling (prefill positions beyond 2560 and every decode row)."""
+    the running-softmax rescaling (every decode row; with `prefill_skinny` also the prompt's rows, whose passes write
+    the last positions they attend to - otherwise the prompt runs the prefill attention kernel)."""
     ref = U.oracle_run(name, 2700, 16, 1, 2, T=T, seed=3)
-    ctx = U.make_ctx(name, 1, 2, T=T, seed=3, max_ctx=2740, max_prefill_rows=64)
+    ctx = U.make_ctx(name, 1, 2, T=T, seed=3, max_ctx=2740, max_prefill_rows=64, prefill_skinny=skinny)
     assert ctx.prefill(ref["prompt"]) == ref["first"]
     ctx.decode(16)
     U.assert_same_run(ctx, ref, 16)
