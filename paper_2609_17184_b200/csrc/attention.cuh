@@ -2,9 +2,15 @@
 // recurrence r attends to the keys/values that its prefix produced at the SAME recurrence r -- the
 // committed slots [0, n_canon) of plane r plus the speculative slots of its uncommitted ancestors and itself.
 //
-// Work item = (row, kv head, chunk of ATT_CHUNK key positions).  Chunks are cut at fixed absolute positions
-// and combined in ascending order by the CTA that finishes a (row, kv head) last, so a row's result does
-// not depend on what else is in the pass.  Softmax statistics are reduced with warp shuffles.
+// Three kernels, by regime:
+//   attn_kernel          work item = (row, kv head, chunk of ATT_CHUNK key positions): every chunk in parallel, for the few
+//                        rows and short contexts of a single sequence's decode pass (latency matters);
+//   attn_runs_kernel     work item = (row, kv head, run of chunks) streamed through a per-thread cp.async ring: long
+//                        contexts and contexts of several sequences (bandwidth matters);
+//   attn_prefill_kernel  work item = (query head, block of rows, run of chunks) for the consecutive positions of a prefill
+//                        pass, which share their keys and values.
+// Chunks and runs are cut at fixed absolute positions (or as a function of the row's own context) and folded in
+// ascending order, so a row's result does not depend on what else is in the pass.
 #pragma once
 #include "common.cuh"
 

@@ -7,10 +7,12 @@
 // columns, K = 16 per instruction) with the accumulator in tensor memory; four warps read it back with tcgen05.ld.
 // Activations are fp32 split exactly into three bf16 planes; the planes are stacked as 3 MP columns of one MMA per
 // k-step (three accumulator chains, as in the mma.sync kernels) and folded hi + (mid + lo) when the accumulator is read.
-// K may be split over blockIdx.y; the partial sums are added in split order by a second kernel (no atomics).
+// K may be split over blockIdx.y; the partial sums are added in split order by a second kernel (no atomics).  Passes of
+// more than 64 token columns put one group of 64 columns in each blockIdx.z plane.
 //
-// Used by the stand-alone operator loopspec_op_linear_tc and by the prefill passes (tc_epilogue_kernel then applies the
-// fused epilogue of the GEMM); the decode passes run gemm_bf16_kernel.
+// Used by the stand-alone operator loopspec_op_linear_tc, by the prefill passes and by the decode passes that carry 9 or
+// more rows (tc_epilogue_kernel then applies the fused epilogue of the GEMM); decode passes of up to 8 rows run
+// gemm_bf16_kernel, whose launch is cheaper than this pair's.
 #pragma once
 #include <cuda.h>
 
