@@ -7,7 +7,7 @@
 //                        rows and short contexts of a single sequence's decode pass (latency matters);
 //   attn_runs_kernel     work item = (row, kv head, run of chunks) streamed through a per-thread cp.async ring: long
 //                        contexts and contexts of several sequences (bandwidth matters);
-//   attn_prefill_kernel  work item = (query head, block of rows, run of chunks) for the consecutive positions of a prefill
+//   attn_prefill_mma_kernel  work item = (query head, block of rows, run of chunks) for the consecutive positions of a prefill
 //                        pass, which share their keys and values.
 // Chunks and runs are cut at fixed absolute positions (or as a function of the row's own context) and folded in
 // ascending order, so a row's result does not depend on what else is in the pass.
@@ -626,14 +626,12 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtsCfg<D, G>::MIN_CTAS)) attn_ru
 
 // ======================= prefill attention: the rows of a pass share every key / value chunk ========================
 // A prefill pass carries consecutive prompt positions p0 .. p0 + n - 1 of one sequence at one recurrence, so all its rows
-// read the same cached keys and values (row i up to its own position).  A work item is (query head, run of chunks) for
-// ALL rows of the pass: a chunk's keys and values are brought into shared memory once, the scores of the 64 x 64 (row,
-// key) tile and the weighted values are register-tiled fp32 FMAs (the query is fp32, keys and values are bf16 values held
-// exactly in fp32: the same products as the decode kernels form), and every row keeps a running softmax over the
-// chunks of the run.  Runs are cut at fixed absolute positions - every chunk below position ATT_PF_SINGLE * 64 is a run
-// of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending order by a second kernel
-// (attn_prefill_fold_kernel), so a row's result depends on its own prefix only, not on how the prompt was cut into
-// passes.
+// read the same cached keys and values (row i up to its own position).  A work item is (query head, block of 32 rows, run
+// of chunks): a chunk's keys and values are brought into shared memory once for the block, and every row keeps a running
+// softmax over the chunks of the run.  Runs are cut at fixed absolute positions - every chunk below position
+// ATT_PF_SINGLE * 64 is a run of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending
+// order by a second kernel (attn_prefill_fold_kernel), so a row's result depends on its own prefix only, not on how the
+// prompt was cut into passes.
 constexpr int ATT_PF_SINGLE = 40;
 constexpr int ATT_PF_RUN = 4;
 __host__ __device__ inline int att_pf_run_of_chunk(int c) { return c < ATT_PF_SINGLE ? c : ATT_PF_SINGLE + (c - ATT_PF_SINGLE) / ATT_PF_RUN; }
@@ -641,39 +639,50 @@ __host__ __device__ inline int att_pf_run_first_chunk(int run) {
   return run < ATT_PF_SINGLE ? run : ATT_PF_SINGLE + (run - ATT_PF_SINGLE) * ATT_PF_RUN;
 }
 constexpr int ATT_PF_ROWS = 64;  // rows of a pass at most (one group of token columns)
-// RT = rows per thread: a work item carries 16 RT rows of the pass.  Smaller items finish sooner (short prompts, where a
-// pass offers only heads x chunks items), larger ones reuse a staged chunk for more rows; a row's arithmetic is the same.
-template <int D, int RT>
-struct AtpCfg {
-  static constexpr int IR = 16 * RT;         // rows per item
-  static constexpr int QS = D + 4;           // floats per query row in shared memory
-  static constexpr int KS = D * 2 + 16;      // bytes per key row (the pad spreads the keys a quarter warp reads over the banks)
-  static constexpr int VS = D * 2;           // bytes per value row
-  static constexpr int SS = ATT_CHUNK + 1;   // floats per score row
-  static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = Q_OFF + IR * QS * 4;
-  static constexpr int V_OFF = K_OFF + ATT_CHUNK * KS;
-  static constexpr int S_OFF = V_OFF + ATT_CHUNK * VS;
-  static constexpr int ST_OFF = S_OFF + IR * SS * 4;   // per row: running max, running mass, rescale of this chunk
+
+// Scores and weighted values of a (32 rows x 64 keys) tile are mma.sync.m16n8k16 contractions (bf16 x bf16 -> fp32).  Keys
+// and values are bf16 already; the fp32 queries and the fp32 softmax weights are split exactly into three bf16 planes
+// (hi + mid + lo), one accumulator chain per plane, folded hi + (mid + lo) - the arithmetic of the GEMM kernels, so every
+// product is exact and a row's result depends on its own operands only (not on its place in the tile, nor on the other
+// rows).  (The same tiles as fp32 FMAs in registers took 29 us per layer at 512 positions and 211 us at 8192 against 18 us
+// and 134 us here.)
+template <int D>
+struct AtmCfg {
+  static constexpr int IR = 32;                 // rows per item: two 16-row MMA tiles
+  static constexpr int QS = D + 8;              // bf16 per row of a query plane (the pad keeps fragment loads off each other's banks)
+  static constexpr int KS = D + 8;              // bf16 per key / value row
+  static constexpr int PS = ATT_CHUNK + 8;      // bf16 per row of a softmax-weight plane
+  static constexpr int SS = ATT_CHUNK + 1;      // floats per score row
+  static constexpr int Q_OFF = 0;                                   // [3][IR][QS] bf16
+  static constexpr int K_OFF = Q_OFF + 3 * IR * QS * 2;             // [64][KS] bf16
+  static constexpr int V_OFF = K_OFF + ATT_CHUNK * KS * 2;          // [64][KS] bf16
+  static constexpr int P_OFF = V_OFF + ATT_CHUNK * KS * 2;          // [3][IR][PS] bf16
+  static constexpr int S_OFF = P_OFF + 3 * IR * PS * 2;             // [IR][SS] fp32
+  static constexpr int ST_OFF = S_OFF + IR * SS * 4;                // [IR][4] fp32
   static constexpr int SMEM_BYTES = ST_OFF + IR * 4 * 4;
-  static constexpr int MIN_CTAS = RT >= 4 ? 2 : 3;
 };
 
-template <int D, int RT>
-__global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
-  using C = AtpCfg<D, RT>;
-  constexpr int IR = C::IR;
-  constexpr int PSTRIDE = D + 2;
-  constexpr int DPT = D / 16;  // dims of the output a thread accumulates (for each of its RT rows)
-  extern __shared__ __align__(16) unsigned char atp_smem[];
-  float* s_q = reinterpret_cast<float*>(atp_smem + C::Q_OFF);
-  unsigned char* s_k = atp_smem + C::K_OFF;
-  unsigned char* s_v = atp_smem + C::V_OFF;
-  float* s_s = reinterpret_cast<float*>(atp_smem + C::S_OFF);
-  float* s_st = reinterpret_cast<float*>(atp_smem + C::ST_OFF);  // [row][4]
+__device__ __forceinline__ void att_mma(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int D>
+__global__ void __launch_bounds__(ATT_THREADS, 2) attn_prefill_mma_kernel(const __grid_constant__ AttnParams p) {
+  using C = AtmCfg<D>;
+  constexpr int IR = C::IR, PSTRIDE = D + 2;
+  constexpr int NTO = D / 32;  // 8-dim output tiles per warp (each warp: one 16-row tile x NTO column tiles)
+  extern __shared__ __align__(16) unsigned char atm_smem[];
+  __nv_bfloat16* s_q = reinterpret_cast<__nv_bfloat16*>(atm_smem + C::Q_OFF);
+  __nv_bfloat16* s_k = reinterpret_cast<__nv_bfloat16*>(atm_smem + C::K_OFF);
+  __nv_bfloat16* s_v = reinterpret_cast<__nv_bfloat16*>(atm_smem + C::V_OFF);
+  __nv_bfloat16* s_p = reinterpret_cast<__nv_bfloat16*>(atm_smem + C::P_OFF);
+  float* s_s = reinterpret_cast<float*>(atm_smem + C::S_OFF);
+  float* s_st = reinterpret_cast<float*>(atm_smem + C::ST_OFF);  // [row][4]: running max, running mass, rescale of this chunk
 
   const RowTable* tab = p.tab;  // written before this pass started
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int n_rows = min(tab->n_rows, ATT_PF_ROWS);
   pdl_launch_dependents();
   pdl_wait();  // the queries, and the keys / values of the pass's own positions, come from this pass's QKV kernel
@@ -685,6 +694,8 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_p
   const int G = p.n_q_heads / p.n_kv_heads, HQ = p.n_q_heads * D;
   const size_t plane = (size_t)(tab->r[0] - 1) * p.kv_plane_stride;
   const int total = p.n_q_heads * n_blocks * n_runs_all;
+  const int mt = warp & 1;   // this warp's 16-row tile
+  const int wq = warp >> 1;  // ... and its quarter of the columns (keys of the score tile, dims of the output tile)
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     const int h = item % p.n_q_heads, rest = item / p.n_q_heads;
@@ -698,80 +709,84 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_p
     const __nv_bfloat16* Kb = p.kv + plane + (size_t)(seq * p.n_kv_heads + kvh) * p.slots * D;
     const __nv_bfloat16* Vb = Kb + p.kv_sel_stride;
     __syncthreads();  // the previous item is done with the shared buffers
-    // queries of the block's rows for this head (fp32), and the rows' softmax state
+    // the block's queries for this head, split into three bf16 planes; rows the pass does not have are zeros
     for (int idx = tid; idx < IR * (D / 4); idx += ATT_THREADS) {
       const int lr = idx / (D / 4), d4 = idx - lr * (D / 4);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);  // rows the pass does not have: zeros
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (lr < rows_here) v = *reinterpret_cast<const float4*>(p.qbuf + (size_t)(row0 + lr) * HQ + (size_t)h * D + d4 * 4);
-      *reinterpret_cast<float4*>(s_q + lr * C::QS + d4 * 4) = v;
+      const float x[4] = {v.x, v.y, v.z, v.w};
+      unsigned short hh[4], mm[4], ll[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) split3(x[i], hh[i], mm[i], ll[i]);
+      __nv_bfloat16* q0 = s_q + lr * C::QS + d4 * 4;
+      *reinterpret_cast<uint2*>(q0) = make_uint2(hh[0] | ((unsigned)hh[1] << 16), hh[2] | ((unsigned)hh[3] << 16));
+      *reinterpret_cast<uint2*>(q0 + IR * C::QS) = make_uint2(mm[0] | ((unsigned)mm[1] << 16), mm[2] | ((unsigned)mm[3] << 16));
+      *reinterpret_cast<uint2*>(q0 + 2 * IR * C::QS) = make_uint2(ll[0] | ((unsigned)ll[1] << 16), ll[2] | ((unsigned)ll[3] << 16));
     }
     if (tid < IR) s_st[tid * 4] = -INFINITY, s_st[tid * 4 + 1] = 0.f, s_st[tid * 4 + 2] = 1.f;
-    float o[RT][DPT];
+    float o[NTO][4];  // running weighted values: rows 16 mt + g (elements 0, 1) and + 8 (2, 3), dims 8 (wq NTO + j) + 2 t, + 1
 #pragma unroll
-    for (int a = 0; a < RT; ++a)
+    for (int j = 0; j < NTO; ++j)
 #pragma unroll
-      for (int i = 0; i < DPT; ++i) o[a][i] = 0.f;
+      for (int i = 0; i < 4; ++i) o[j][i] = 0.f;
 
     for (int chunk = c_lo; chunk < c_hi; ++chunk) {
       const int k0 = chunk * ATT_CHUNK;
       const int n_keys = min(ATT_CHUNK, n_ctx - k0);  // keys of this chunk that exist (all of them written)
       if (chunk > c_lo) __syncthreads();               // the previous chunk's readers are done
-      // ---- the chunk's keys and values, once for all rows of the block ------------------------------------------
+      // ---- the chunk's keys and values, once for all rows of the block (missing keys: zeros) ----------------------
       for (int idx = tid; idx < ATT_CHUNK * (D / 8); idx += ATT_THREADS) {
         const int key = idx / (D / 8), pc = idx - key * (D / 8);
         const bool ok = key < n_keys;
         const size_t off = (size_t)(k0 + (ok ? key : 0)) * D + pc * 8;
-        cp_async16_zfill(s_k + key * C::KS + pc * 16, Kb + off, ok);
-        cp_async16_zfill(s_v + key * C::VS + pc * 16, Vb + off, ok);
+        cp_async16_zfill(s_k + key * C::KS + pc * 8, Kb + off, ok);
+        cp_async16_zfill(s_v + key * C::KS + pc * 8, Vb + off, ok);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       __syncthreads();
-      // ---- scores: thread (ty, tx) takes rows RT ty .. RT ty + RT - 1 and keys tx, tx + 16, tx + 32, tx + 48 ---------
-      float sc[RT][4];
+      // ---- scores: this warp's 16 rows x 16 keys (two 8-key tiles), three plane chains each --------------------------
+      {
+        float acc[3][2][4];
 #pragma unroll
-      for (int a = 0; a < RT; ++a)
+        for (int pl = 0; pl < 3; ++pl)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) sc[a][b] = 0.f;
+          for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[pl][j][i] = 0.f;
 #pragma unroll 2
-      for (int d = 0; d < D; d += 8) {
-        float4 qa[RT], qb[RT];
+        for (int ks = 0; ks < D / 16; ++ks) {
+          unsigned a[3][4];
 #pragma unroll
-        for (int a = 0; a < RT; ++a) {
-          qa[a] = *reinterpret_cast<const float4*>(s_q + (RT * ty + a) * C::QS + d);
-          qb[a] = *reinterpret_cast<const float4*>(s_q + (RT * ty + a) * C::QS + d + 4);
-        }
+          for (int pl = 0; pl < 3; ++pl) {
+            const __nv_bfloat16* qa = s_q + (pl * IR + 16 * mt + g) * C::QS + 16 * ks + 2 * t;
+            a[pl][0] = *reinterpret_cast<const unsigned*>(qa), a[pl][1] = *reinterpret_cast<const unsigned*>(qa + 8 * C::QS);
+            a[pl][2] = *reinterpret_cast<const unsigned*>(qa + 8), a[pl][3] = *reinterpret_cast<const unsigned*>(qa + 8 * C::QS + 8);
+          }
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const uint4 kw = *reinterpret_cast<const uint4*>(s_k + (tx + 16 * b) * C::KS + d * 2);
-          const float k0f = __uint_as_float(kw.x << 16), k1f = __uint_as_float(kw.x & 0xffff0000u);
-          const float k2f = __uint_as_float(kw.y << 16), k3f = __uint_as_float(kw.y & 0xffff0000u);
-          const float k4f = __uint_as_float(kw.z << 16), k5f = __uint_as_float(kw.z & 0xffff0000u);
-          const float k6f = __uint_as_float(kw.w << 16), k7f = __uint_as_float(kw.w & 0xffff0000u);
+          for (int j = 0; j < 2; ++j) {
+            const __nv_bfloat16* kb = s_k + (8 * (2 * wq + j) + g) * C::KS + 16 * ks + 2 * t;
+            const unsigned b0 = *reinterpret_cast<const unsigned*>(kb), b1 = *reinterpret_cast<const unsigned*>(kb + 8);
 #pragma unroll
-          for (int a = 0; a < RT; ++a) {  // dims in ascending order, one chain per (row, key)
-            float v = sc[a][b];
-            v = fmaf(qa[a].x, k0f, v), v = fmaf(qa[a].y, k1f, v), v = fmaf(qa[a].z, k2f, v), v = fmaf(qa[a].w, k3f, v);
-            v = fmaf(qb[a].x, k4f, v), v = fmaf(qb[a].y, k5f, v), v = fmaf(qb[a].z, k6f, v), v = fmaf(qb[a].w, k7f, v);
-            sc[a][b] = v;
+            for (int pl = 0; pl < 3; ++pl) att_mma(acc[pl][j], a[pl], b0, b1);
           }
         }
-      }
 #pragma unroll
-      for (int a = 0; a < RT; ++a) {
-        const int lr = RT * ty + a, pos = p0 + row0 + lr;
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int key = tx + 16 * b;
-          const bool ok = lr < rows_here && key < n_keys && k0 + key <= pos;  // causal
-          s_s[lr * C::SS + key] = ok ? sc[a][b] * p.scale : -INFINITY;
-        }
+          for (int i = 0; i < 4; ++i) {
+            const int lr = 16 * mt + g + (i >> 1) * 8, key = 8 * (2 * wq + j) + 2 * t + (i & 1);
+            const float sv = acc[0][j][i] + (acc[1][j][i] + acc[2][j][i]);
+            const bool ok = lr < rows_here && key < n_keys && k0 + key <= p0 + row0 + lr;  // causal
+            s_s[lr * C::SS + key] = ok ? sv * p.scale : -INFINITY;
+          }
       }
       __syncthreads();
-      // ---- running softmax of every row: four threads per row, 16 keys each, folded in a fixed order ----------------
+      // ---- running softmax of every row: four threads per row, 16 keys each, folded in a fixed order; the weights go
+      // to three bf16 planes for the second contraction -------------------------------------------------------------
       if (tid < 4 * IR) {
         const int lr = tid >> 2, part = tid & 3;
-        float* sr = s_s + lr * C::SS + part * 16;
+        const float* sr = s_s + lr * C::SS + part * 16;
         float m = -INFINITY;
 #pragma unroll
         for (int jj = 0; jj < 16; ++jj) m = fmaxf(m, sr[jj]);
@@ -781,15 +796,23 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_p
         const float m_new = fmaxf(m_old, m);
         float l = 0.f;
 #pragma unroll
-        for (int jj = 0; jj < 16; ++jj) {
-          const float e = (sr[jj] == -INFINITY) ? 0.f : expf(sr[jj] - m_new);
-          sr[jj] = e;
-          l += e;
+        for (int jj = 0; jj < 16; jj += 2) {
+          const float e0 = (sr[jj] == -INFINITY) ? 0.f : expf(sr[jj] - m_new);
+          const float e1 = (sr[jj + 1] == -INFINITY) ? 0.f : expf(sr[jj + 1] - m_new);
+          l += e0;
+          l += e1;
+          unsigned short h0, m0, l0, h1, m1, l1;
+          split3(e0, h0, m0, l0);
+          split3(e1, h1, m1, l1);
+          __nv_bfloat16* pp = s_p + lr * C::PS + part * 16 + jj;
+          *reinterpret_cast<unsigned*>(pp) = h0 | ((unsigned)h1 << 16);
+          *reinterpret_cast<unsigned*>(pp + IR * C::PS) = m0 | ((unsigned)m1 << 16);
+          *reinterpret_cast<unsigned*>(pp + 2 * IR * C::PS) = l0 | ((unsigned)l1 << 16);
         }
-        const float l1 = __shfl_xor_sync(0xffffffffu, l, 1);
-        const float lp = (part & 1) ? l1 + l : l + l1;         // (part 0 + part 1), (part 2 + part 3)
-        const float l2 = __shfl_xor_sync(0xffffffffu, lp, 2);
-        const float lc = (part & 2) ? l2 + lp : lp + l2;       // lower pair first
+        const float l1s = __shfl_xor_sync(0xffffffffu, l, 1);
+        const float lp = (part & 1) ? l1s + l : l + l1s;       // (part 0 + part 1), (part 2 + part 3)
+        const float l2s = __shfl_xor_sync(0xffffffffu, lp, 2);
+        const float lc = (part & 2) ? l2s + lp : lp + l2s;     // lower pair first
         __syncwarp();
         if (part == 0) {
           const float wa = (m_old == -INFINITY) ? 0.f : expf(m_old - m_new);  // (a row that has seen no key yet: nothing to rescale)
@@ -797,53 +820,61 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtpCfg<D, RT>::MIN_CTAS)) attn_p
         }
       }
       __syncthreads();
-      // ---- weighted values: thread (ty, tx) takes its RT rows and dims tx * DPT .. + DPT - 1, keys in ascending order --
+      // ---- weighted values: this warp's 16 rows x NTO tiles of 8 dims, keys in four steps of 16 ---------------------------
       {
-        float wa[RT];
+        float acc[3][NTO][4];
 #pragma unroll
-        for (int a = 0; a < RT; ++a) wa[a] = s_st[(RT * ty + a) * 4 + 2];
+        for (int pl = 0; pl < 3; ++pl)
 #pragma unroll
-        for (int a = 0; a < RT; ++a)
+          for (int j = 0; j < NTO; ++j)
 #pragma unroll
-          for (int i = 0; i < DPT; ++i) o[a][i] *= wa[a];
-        for (int key = 0; key < n_keys; ++key) {
-          float vf[DPT];
-          if (DPT == 8) {
-            const uint4 vw = *reinterpret_cast<const uint4*>(s_v + key * C::VS + tx * 16);
-            const unsigned w[4] = {vw.x, vw.y, vw.z, vw.w};
+            for (int i = 0; i < 4; ++i) acc[pl][j][i] = 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) vf[2 * i] = __uint_as_float(w[i] << 16), vf[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-          } else {
-            const uint2 vw = *reinterpret_cast<const uint2*>(s_v + key * C::VS + tx * 8);
-            vf[0] = __uint_as_float(vw.x << 16), vf[1] = __uint_as_float(vw.x & 0xffff0000u);
-            vf[2] = __uint_as_float(vw.y << 16), vf[3] = __uint_as_float(vw.y & 0xffff0000u);
+        for (int ks = 0; ks < ATT_CHUNK / 16; ++ks) {
+          unsigned a[3][4];
+#pragma unroll
+          for (int pl = 0; pl < 3; ++pl) {
+            const __nv_bfloat16* pa = s_p + (pl * IR + 16 * mt + g) * C::PS + 16 * ks + 2 * t;
+            a[pl][0] = *reinterpret_cast<const unsigned*>(pa), a[pl][1] = *reinterpret_cast<const unsigned*>(pa + 8 * C::PS);
+            a[pl][2] = *reinterpret_cast<const unsigned*>(pa + 8), a[pl][3] = *reinterpret_cast<const unsigned*>(pa + 8 * C::PS + 8);
           }
 #pragma unroll
-          for (int a = 0; a < RT; ++a) {
-            const float pw = s_s[(RT * ty + a) * C::SS + key];
+          for (int j = 0; j < NTO; ++j) {
+            // B fragment of V[key][dim] (keys = the contraction index): transposing matrix load, lanes 0-15 name the key rows
+            const unsigned addr = (unsigned)__cvta_generic_to_shared(s_v + (16 * ks + (lane & 15)) * C::KS + 8 * (wq * NTO + j));
+            unsigned b0, b1;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
 #pragma unroll
-            for (int i = 0; i < DPT; ++i) o[a][i] = fmaf(pw, vf[i], o[a][i]);
+            for (int pl = 0; pl < 3; ++pl) att_mma(acc[pl][j], a[pl], b0, b1);
           }
         }
+        const float wa0 = s_st[(16 * mt + g) * 4 + 2], wa1 = s_st[(16 * mt + g + 8) * 4 + 2];
+#pragma unroll
+        for (int j = 0; j < NTO; ++j)
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            o[j][i] = fmaf(o[j][i], (i >> 1) ? wa1 : wa0, acc[0][j][i] + (acc[1][j][i] + acc[2][j][i]));
       }
     }
     __syncthreads();  // every thread has read the final state
     // ---- the run is done: rows with one run only are finished here, the others leave a partial for the fold -----------
 #pragma unroll
-    for (int a = 0; a < RT; ++a) {
-      const int lr = RT * ty + a, row = row0 + lr, pos = p0 + row;
+    for (int hf = 0; hf < 2; ++hf) {
+      const int lr = 16 * mt + g + 8 * hf, row = row0 + lr, pos = p0 + row;
       if (lr >= rows_here || c_lo * ATT_CHUNK > pos) continue;   // the row does not reach this run
       const int n_runs_row = att_pf_run_of_chunk(pos / ATT_CHUNK) + 1;
       const float m = s_st[lr * 4], l = s_st[lr * 4 + 1];
-      if (n_runs_row == 1) {
+      float* mypart = p.part + (((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks + run) * G + gq) * PSTRIDE;
 #pragma unroll
-        for (int i = 0; i < DPT; ++i) store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + tx * DPT + i, o[a][i] / l);
-      } else {
-        float* mypart = p.part + (((size_t)(row * p.n_kv_heads + kvh) * p.max_chunks + run) * G + gq) * PSTRIDE;
+      for (int j = 0; j < NTO; ++j)
 #pragma unroll
-        for (int i = 0; i < DPT; ++i) __stcg(mypart + tx * DPT + i, o[a][i]);
-        if (tx == 0) __stcg(mypart + D, m), __stcg(mypart + D + 1, l);
-      }
+        for (int e = 0; e < 2; ++e) {
+          const int dd = 8 * (wq * NTO + j) + 2 * t + e;
+          const float v = o[j][2 * hf + e];
+          if (n_runs_row == 1) store_split(p.aplanes + (size_t)row * 3 * HQ, HQ, h * D + dd, v / l);
+          else __stcg(mypart + dd, v);
+        }
+      if (n_runs_row > 1 && wq == 0 && t == 0) __stcg(mypart + D, m), __stcg(mypart + D + 1, l);
     }
   }
 }

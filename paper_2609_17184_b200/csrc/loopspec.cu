@@ -776,25 +776,15 @@ cudaError_t launch_attention(loopspec_ctx* c, const RowTable* tab, int l, unsign
   a.part = c->at<float>(c->L.apart), a.max_chunks = d.max_chunks, a.counters = c->at<int>(c->L.acnt);
   a.tl = tl, a.tl_id = tl_id;
   if (prefill_rows && c->pf_attn) {  // consecutive prompt positions of one sequence: the rows share every K/V chunk
-    // contexts of up to 1280 positions offer few items per pass (heads x chunks): items of 32 rows finish sooner (29 us
-    // against 33 us per layer at 512 positions); longer contexts have items to spare and reuse a staged chunk for all 64
-    // rows (62 us against 74 us at 2048 positions, 211 us against 256 us at 8192)
     const dim3 fold_grid(d.max_rows_pf, m.n_q_heads);
-    const bool small_items = d.max_chunks <= 20;
     cudaError_t e;
     if (m.head_dim == 128) {
-      e = small_items ? launch_k(attn_prefill_kernel<128, 2>, dim3(c->n_sm * AtpCfg<128, 2>::MIN_CTAS), dim3(ATT_THREADS),
-                                 (size_t)AtpCfg<128, 2>::SMEM_BYTES, c->stream, a, c->use_pdl)
-                      : launch_k(attn_prefill_kernel<128, 4>, dim3(c->n_sm * AtpCfg<128, 4>::MIN_CTAS), dim3(ATT_THREADS),
-                                 (size_t)AtpCfg<128, 4>::SMEM_BYTES, c->stream, a, c->use_pdl);
-      if (e) return e;
+      if ((e = launch_k(attn_prefill_mma_kernel<128>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtmCfg<128>::SMEM_BYTES, c->stream, a, c->use_pdl)))
+        return e;
       return launch_k(attn_prefill_fold_kernel<128>, fold_grid, dim3(32), 0, c->stream, a, c->use_pdl);
     }
-    e = small_items ? launch_k(attn_prefill_kernel<64, 2>, dim3(c->n_sm * AtpCfg<64, 2>::MIN_CTAS), dim3(ATT_THREADS),
-                               (size_t)AtpCfg<64, 2>::SMEM_BYTES, c->stream, a, c->use_pdl)
-                    : launch_k(attn_prefill_kernel<64, 4>, dim3(c->n_sm * AtpCfg<64, 4>::MIN_CTAS), dim3(ATT_THREADS),
-                               (size_t)AtpCfg<64, 4>::SMEM_BYTES, c->stream, a, c->use_pdl);
-    if (e) return e;
+    if ((e = launch_k(attn_prefill_mma_kernel<64>, dim3(c->n_sm * 2), dim3(ATT_THREADS), (size_t)AtmCfg<64>::SMEM_BYTES, c->stream, a, c->use_pdl)))
+      return e;
     return launch_k(attn_prefill_fold_kernel<64>, fold_grid, dim3(16), 0, c->stream, a, c->use_pdl);
   }
   const bool runs = d.att_runs != 0;
@@ -1177,13 +1167,10 @@ int loopspec_init(const loopspec_model* m, const loopspec_sched* s, const loopsp
   }
   if (!s->prefill_skinny) {  // (prefill_skinny keeps the decode kernels for the prefill passes, attention included)
     bool ok = true;
-    if (m->head_dim == 128) {
-      ok = ok && cudaFuncSetAttribute(attn_prefill_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<128, 2>::SMEM_BYTES) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(attn_prefill_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<128, 4>::SMEM_BYTES) == cudaSuccess;
-    } else {
-      ok = ok && cudaFuncSetAttribute(attn_prefill_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<64, 2>::SMEM_BYTES) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(attn_prefill_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtpCfg<64, 4>::SMEM_BYTES) == cudaSuccess;
-    }
+    if (m->head_dim == 128)
+      ok = cudaFuncSetAttribute(attn_prefill_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtmCfg<128>::SMEM_BYTES) == cudaSuccess;
+    else
+      ok = cudaFuncSetAttribute(attn_prefill_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AtmCfg<64>::SMEM_BYTES) == cudaSuccess;
     if (!ok) (void)cudaGetLastError();
     c->pf_attn = ok;
   }
