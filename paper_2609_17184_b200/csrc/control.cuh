@@ -440,34 +440,36 @@ struct PrefillParams {
 __global__ void __launch_bounds__(CTRL_THREADS) prefill_setup_kernel(const PrefillParams p) {
   __shared__ int s_emb[MAX_ROWS][2];
   const int tid = threadIdx.x;
-  if (tid == 0) {
-    RowTable& t = *p.tab;
-    int items = 0, n_ro = 0;
-    for (int i = 0; i < p.count; ++i) {
-      int pos = p.p0 + i;
-      t.seq[i] = p.seq, t.r[i] = p.r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
-      t.n_safe[i] = p.p0;
-      t.hid_idx[i] = p.hid_base + i, t.node[i] = -1, t.src_hid[i] = -1;
-      bool last = (p.r == p.R) && (pos == p.n_prompt - 1);
-      t.readout[i] = last ? RO_TARGET : RO_NONE, t.logit_idx[i] = p.p_logit_base + p.seq;
-      if (last) t.ro_rows[n_ro++] = i;
-      t.chunk_start[i] = items;
-      items += att_items(pos + 1, p.att_mode);
-      s_emb[i][0] = p.hid_base + i, s_emb[i][1] = p.prompt[pos];
-    }
-    t.chunk_start[p.count] = items;
-    t.n_rows = p.count, t.n_readout = n_ro, t.attn_items = items, t.att_mode = p.att_mode;
-    if (p.tab_coda && p.coda_class > 0) {  // the same rows, on copies of their states, writing this depth's coda cache
-      RowTable& c = *p.tab_coda;
-      int nr = 0;
-      for (int i = 0; i < p.count; ++i) {
-        c.seq[i] = t.seq[i], c.r[i] = p.coda_class, c.pos[i] = t.pos[i], c.kv_slot[i] = t.kv_slot[i], c.n_canon[i] = t.n_canon[i];
-        c.n_spec[i] = 0, c.n_safe[i] = t.n_safe[i], c.hid_idx[i] = p.hid_coda_base + i, c.src_hid[i] = t.hid_idx[i], c.node[i] = -1;
-        c.readout[i] = t.readout[i], c.logit_idx[i] = t.logit_idx[i], c.chunk_start[i] = t.chunk_start[i];
-        if (t.readout[i]) c.ro_rows[nr++] = i;
+  // one thread per row (rows are independent: consecutive positions of one sequence); the reading-out row, if the
+  // pass has one, is the prompt's last position at the last recurrence
+  RowTable& t = *p.tab;
+  RowTable* c = (p.tab_coda && p.coda_class > 0) ? p.tab_coda : nullptr;  // the same rows, on copies of their states,
+                                                                          // writing this depth's coda cache
+  const int ro_row = (p.r == p.R && p.n_prompt - 1 >= p.p0 && p.n_prompt - 1 < p.p0 + p.count) ? p.n_prompt - 1 - p.p0 : -1;
+  for (int i = tid; i <= p.count; i += CTRL_THREADS) {
+    int items = 0;  // work items of the rows before this one
+    for (int k = 0; k < i; ++k) items += att_items(p.p0 + k + 1, p.att_mode);
+    t.chunk_start[i] = items;
+    if (c) c->chunk_start[i] = items;
+    if (i == p.count) {
+      t.n_rows = p.count, t.n_readout = ro_row >= 0 ? 1 : 0, t.attn_items = items, t.att_mode = p.att_mode;
+      if (ro_row >= 0) t.ro_rows[0] = ro_row;
+      if (c) {
+        c->n_rows = p.count, c->n_readout = ro_row >= 0 ? 1 : 0, c->attn_items = items, c->att_mode = p.att_mode;
+        if (ro_row >= 0) c->ro_rows[0] = ro_row;
       }
-      c.chunk_start[p.count] = items;
-      c.n_rows = p.count, c.n_readout = nr, c.attn_items = items, c.att_mode = p.att_mode;
+      break;
+    }
+    const int pos = p.p0 + i, ro = i == ro_row ? RO_TARGET : RO_NONE;
+    t.seq[i] = p.seq, t.r[i] = p.r, t.pos[i] = pos, t.kv_slot[i] = pos, t.n_canon[i] = pos + 1, t.n_spec[i] = 0;
+    t.n_safe[i] = p.p0;
+    t.hid_idx[i] = p.hid_base + i, t.node[i] = -1, t.src_hid[i] = -1;
+    t.readout[i] = ro, t.logit_idx[i] = p.p_logit_base + p.seq;
+    s_emb[i][0] = p.hid_base + i, s_emb[i][1] = p.prompt[pos];
+    if (c) {
+      c->seq[i] = p.seq, c->r[i] = p.coda_class, c->pos[i] = pos, c->kv_slot[i] = pos, c->n_canon[i] = pos + 1;
+      c->n_spec[i] = 0, c->n_safe[i] = p.p0, c->hid_idx[i] = p.hid_coda_base + i, c->src_hid[i] = p.hid_base + i, c->node[i] = -1;
+      c->readout[i] = ro, c->logit_idx[i] = p.p_logit_base + p.seq;
     }
   }
   __syncthreads();
