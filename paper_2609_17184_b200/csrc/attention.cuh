@@ -632,8 +632,8 @@ __global__ void __launch_bounds__(ATT_THREADS, (AtsCfg<D, G>::MIN_CTAS)) attn_ru
 // ATT_PF_SINGLE * 64 is a run of its own, beyond that runs of ATT_PF_RUN chunks - and a row's runs are folded in ascending
 // order by a second kernel (attn_prefill_fold_kernel), so a row's result depends on its own prefix only, not on how the
 // prompt was cut into passes.
-constexpr int ATT_PF_SINGLE = 40;
-constexpr int ATT_PF_RUN = 4;
+constexpr int ATT_PF_SINGLE = 8;  // [measured per layer at 2048 / 4096 / 8192 positions, 64 rows: single chunks up to 8 and runs of 4
+constexpr int ATT_PF_RUN = 4;     //  beyond: 43 / 68 / 106 us; up to 16: 47 / 66 / 120 us; up to 40: 51 / 78 / 133 us; runs of 8: slower]
 __host__ __device__ inline int att_pf_run_of_chunk(int c) { return c < ATT_PF_SINGLE ? c : ATT_PF_SINGLE + (c - ATT_PF_SINGLE) / ATT_PF_RUN; }
 __host__ __device__ inline int att_pf_run_first_chunk(int run) {
   return run < ATT_PF_SINGLE ? run : ATT_PF_SINGLE + (run - ATT_PF_SINGLE) * ATT_PF_RUN;
