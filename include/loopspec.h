@@ -90,8 +90,9 @@ typedef struct {
   float top_p;
   int32_t measure_tv;
   int32_t mask_first;
-  int32_t prefill_skinny; /* 1: the prefill passes run the layer GEMMs on the kernels of the decode passes instead of the
-                             wide tcgen05 kernels (slower; for comparing the two paths) */
+  int32_t prefill_skinny; /* 1: the prefill passes run the kernels of the decode passes - layer GEMMs on mma.sync instead of
+                             the wide tcgen05 kernel, attention row by row instead of the kernel that shares K/V among the
+                             rows of a pass (slower; for comparing the two paths) */
 } loopspec_sched;
 
 /* Device pointers to the weights.  layer_ptrs is a HOST array of 6 * (n_prelude + n_recurrent + n_coda) device pointers -
